@@ -1,0 +1,205 @@
+/*
+ * huffllm — Huffman-compressed 16-bit LLM weights that stay compressed in GPU memory and are
+ * decoded on the fly inside the matrix-vector / small-batch matrix products that consume them.
+ *
+ * The method is Huff-LLM's: each weight is split into bit fields, the sign (and, for BF16, the
+ * seven mantissa bits) stay raw, the exponent fields are Huffman coded (BF16 {1,4,4,7}:
+ * Section 5.1; FP16 {1,5,5,5}: Section 3.1), compression happens once, offline, on the CPU
+ * (Section 3.1), weights stay compressed everywhere and are decompressed only to be multiplied
+ * with activations (Section 1, contributions), and the decoder knows a fixed bound L_max on the
+ * codeword length (Section 3.2).
+ *
+ * Conventions for every call
+ *   - C ABI, plain pointers and sizes.  "host" / "device" on a pointer says where it must live.
+ *   - The caller owns every buffer.  The only object the library allocates is the codebook
+ *     (create with huffllm_build_codebook, release with huffllm_codebook_free).
+ *   - Weights are row-major [rows = out_features][cols = in_features], as 16-bit patterns.
+ *   - Device calls are asynchronous on `stream`, never synchronise, never allocate.
+ *   - Every call returns a huffllm_status; huffllm_last_error() gives a thread-local message.
+ *     Nothing aborts, throws, or traps on the device.
+ */
+#ifndef HUFFLLM_H
+#define HUFFLLM_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    HUFFLLM_OK = 0,
+    HUFFLLM_ERR_INVALID_ARG = 1,      /* null pointer, zero size, misaligned device pointer, bad enum        */
+    HUFFLLM_ERR_UNSUPPORTED = 2,      /* valid request this build does not implement (nothing was launched)  */
+    HUFFLLM_ERR_BUFFER_TOO_SMALL = 3, /* blob / workspace capacity below what the call needs                 */
+    HUFFLLM_ERR_CORRUPT = 4,          /* blob fails validation                                               */
+    HUFFLLM_ERR_CUDA = 5,             /* a CUDA runtime call failed; message holds cudaGetErrorString        */
+    HUFFLLM_ERR_NOMEM = 6             /* host allocation failed                                              */
+} huffllm_status;
+
+typedef enum { HUFFLLM_BF16 = 0, HUFFLLM_FP16 = 1 } huffllm_dtype;
+
+/* A CUDA stream handle (cudaStream_t), spelled without the CUDA headers. */
+typedef struct CUstream_st *huffllm_stream;
+
+/* Opaque host object: per-field symbol counts, code lengths, canonical codewords, decode table. */
+typedef struct huffllm_codebook huffllm_codebook;
+
+/*
+ * Descriptor of an encoded tensor.  It is also, byte for byte, the first 256 bytes of the blob,
+ * so a blob saved to disk describes itself (huffllm_validate_blob re-reads it).  Little endian.
+ *
+ * Blob layout (every section starts on a 256-byte boundary):
+ *   header    this struct
+ *   codebook  uint8 lengths[3][32]; 0 = symbol unused; codewords are canonical: symbols ordered by
+ *             (length, symbol), first codeword 0, next = (previous + 1) << (length growth); a
+ *             codeword's most significant bit comes first in the stream
+ *   LUT       uint32[1 << lut_bits], indexed by the next lut_bits stream bits (first bit = bit 0);
+ *             BF16 entry = exponent << 23 | (length of hi-nibble code + length of lo-nibble code)
+ *   index     uint32[n_chunks + 1]: record offsets from off_payload, in units of 128 bytes
+ *   payload   one record per chunk, chunk id = row_group * col_chunks + col_chunk
+ *
+ * A chunk is a tile of 16 rows x chunk_cols (= chunk_elems / 16) columns, cut into blocks of 32
+ * columns (the last column chunk may hold fewer blocks).  It is decoded by 32 lanes; lane
+ * l = 4 g + t (g < 8, t < 4) owns rows g and g + 8 of the tile and columns 8t .. 8t+7 of every
+ * block.  Its sequence is, block after block, row g's eight weights then row g+8's eight weights.
+ * Positions outside the tensor hold `pad_word`.  Record = raw bytes [block][lane][16]
+ * (BF16 raw byte = sign << 7 | mantissa), then W rows of 32 little-endian uint32 (row j, lane l):
+ * lane l's bit sequence, bit i in word i / 32 at bit i % 32.  The sequence starts with `lag_bits`
+ * zero bits, then for every weight code(exponent >> 4) code(exponent & 15); bits after the last
+ * codeword are zero.  W is the largest lane length of the chunk in words (lanes are padded to it).
+ */
+typedef struct huffllm_desc {
+    char     magic[4];        /* "HFLM"                                                    */
+    uint32_t version;         /* 1                                                         */
+    uint32_t dtype;           /* huffllm_dtype                                             */
+    uint32_t chunk_elems;     /* weights per chunk: a multiple of 512 in [512, 16384]      */
+    uint64_t rows, cols;
+    uint32_t tile_rows;       /* 16                                                        */
+    uint32_t chunk_cols;      /* chunk_elems / 16                                          */
+    uint32_t row_groups;      /* ceil(rows / 16)                                           */
+    uint32_t col_chunks;      /* ceil(cols / chunk_cols)                                   */
+    uint64_t n_chunks;        /* row_groups * col_chunks                                   */
+    uint32_t lut_bits;        /* L_max of one weight's coded fields together (8 .. 12)     */
+    uint32_t lag_bits;        /* 7                                                         */
+    uint32_t n_fields;        /* coded fields per weight: 2 (BF16)                         */
+    uint8_t  caps[4];         /* per-field maximum code length chosen under lut_bits       */
+    uint16_t pad_word;        /* weight stored at positions outside the tensor            */
+    uint16_t reserved0;
+    uint32_t max_words;       /* largest W over all chunks                                 */
+    uint64_t off_codebook, off_lut, off_index, off_payload;   /* byte offsets in the blob */
+    uint64_t payload_bytes;   /* 128 * index[n_chunks]                                     */
+    uint64_t blob_bytes;      /* total size: what the device kernels stream from HBM       */
+    uint64_t coded_bits;      /* sum of codeword lengths over all stored weights           */
+    uint64_t raw_bits;        /* raw bits of the rows*cols real weights                    */
+    uint64_t payload_checksum;/* sum over chunks of (2 id + 1) * FNV-1a-64(record bytes)   */
+    uint8_t  reserved[104];
+} huffllm_desc;
+
+/* ------------------------------------------------------------------ host: compress once, offline */
+
+/*
+ * Count the coded fields of `w` (host, rows*cols 16-bit words) and build one Huffman code per
+ * field for this tensor (Sections 3.1 and 5.1).  `max_code_len` is L_max (Section 3.2) for the
+ * coded fields of one weight taken together: for BF16 the hi- and lo-nibble code lengths are
+ * capped at (c0, c1) with c0 + c1 <= max_code_len, chosen to minimise the coded size, each code
+ * being the optimal length-limited prefix code for its cap; where plain Huffman already fits,
+ * the result is plain Huffman.  0 selects the default (8); supported range 8..12.
+ * A field with a single used symbol gets a 1-bit code.  An empty tensor is INVALID_ARG.
+ * On success *out owns a new codebook.  HUFFLLM_FP16 returns UNSUPPORTED in this build.
+ */
+huffllm_status huffllm_build_codebook(const uint16_t *w_host, uint64_t rows, uint64_t cols, huffllm_dtype dtype,
+                                      uint32_t max_code_len, huffllm_codebook **out);
+
+/* Read one field of a codebook: number of symbols of the field's alphabet, and per symbol its
+ * count, code length (0 = unused) and canonical codeword.  Arrays hold 32 entries.            */
+huffllm_status huffllm_codebook_get(const huffllm_codebook *cb, uint32_t field, uint32_t *n_symbols,
+                                    uint64_t counts[32], uint8_t lengths[32], uint32_t codes[32]);
+
+void huffllm_codebook_free(huffllm_codebook *cb);
+
+/* Upper bound, in bytes, of the blob huffllm_encode can produce for this shape (any codebook).  */
+huffllm_status huffllm_encode_bound(uint64_t rows, uint64_t cols, huffllm_dtype dtype, uint32_t chunk_elems,
+                                    size_t *max_bytes);
+
+/*
+ * Encode `w` (host) with `cb` into `blob` (host, capacity blob_cap, 256-byte aligned recommended):
+ * chunked bitstreams with a per-chunk offset index so that chunks decode in parallel.  Every
+ * weight must use only symbols the codebook has codewords for (always true for the tensor the
+ * codebook was built from), else INVALID_ARG.  *desc receives the descriptor (= blob header).
+ */
+huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w_host, uint64_t rows, uint64_t cols,
+                              uint32_t chunk_elems, void *blob_host, size_t blob_cap, huffllm_desc *desc);
+
+/*
+ * Check a blob held in host memory before it is uploaded: header fields and geometry, section
+ * bounds, Kraft sums of the stored code lengths, the LUT against the codebook, a monotone record
+ * index, record sizes, and a walk over every lane's bits (each lane must hold exactly its number
+ * of codewords inside its W words, with zero lag and tail bits) and the payload checksum.  Returns CORRUPT on any
+ * failure.  On success *desc_out (optional) receives the descriptor.
+ */
+huffllm_status huffllm_validate_blob(const void *blob_host, size_t bytes, huffllm_desc *desc_out);
+
+/* --------------------------------------------------------- device: decode, and decode fused with products */
+
+/*
+ * Scratch bytes the fused products need for `batch` activation vectors.  The workspace must be
+ * zero-filled once after allocation; every call leaves it zero-filled again.  Calls that share a
+ * workspace must not overlap on the GPU.
+ */
+huffllm_status huffllm_workspace_bytes(const huffllm_desc *desc, uint32_t batch, size_t *bytes);
+
+/*
+ * Decompress a blob (device, 256-byte aligned) to its original 16-bit weights, bit for bit
+ * (Section 3.2: sign, exponent and mantissa are concatenated back into the 16-bit weight).
+ * `out` (device) receives rows*cols words, row-major.  `err_flag` (device int32, may be null) is
+ * set non-zero if the kernel met an out-of-range record offset or a copy that never arrived.
+ */
+huffllm_status huffllm_decode(const huffllm_desc *desc, const void *blob_dev, uint16_t *out_dev,
+                              int32_t *err_flag_dev, huffllm_stream stream);
+
+/*
+ * y = W x with W taken straight from the compressed blob: weights are decoded in registers and
+ * multiplied at once, so only compressed bytes cross the memory bus (Section 1: weights are
+ * decompressed only when needed, to multiply with activations).  x: device, cols words of the
+ * blob's dtype.  y: device, rows floats.  Products are exact, sums are accumulated in fp32.
+ * Results are bitwise reproducible from run to run.
+ */
+huffllm_status huffllm_decode_gemv(const huffllm_desc *desc, const void *blob_dev, const uint16_t *x_dev, float *y_dev,
+                                   void *workspace_dev, size_t workspace_bytes, int32_t *err_flag_dev,
+                                   huffllm_stream stream);
+
+/*
+ * Small-batch version: x is [batch][cols] row-major (device), y is [batch][rows] floats (device).
+ * batch 1..64.
+ */
+huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob_dev, const uint16_t *x_dev, uint32_t batch,
+                                   float *y_dev, void *workspace_dev, size_t workspace_bytes, int32_t *err_flag_dev,
+                                   huffllm_stream stream);
+
+/*
+ * The same product called with HOST activations and a HOST result: copies x to `x_stage_dev`
+ * (device, batch*cols words), runs huffllm_decode_gemm, copies y from `y_stage_dev` (device,
+ * batch*rows floats) to y_host and waits for the stream.  x_host / y_host should be pinned.
+ */
+huffllm_status huffllm_decode_gemm_host(const huffllm_desc *desc, const void *blob_dev, const uint16_t *x_host,
+                                        uint32_t batch, float *y_host, uint16_t *x_stage_dev, float *y_stage_dev,
+                                        void *workspace_dev, size_t workspace_bytes, int32_t *err_flag_dev,
+                                        huffllm_stream stream);
+
+/*
+ * Reference point for the compressed path: y = W x for an UNCOMPRESSED bf16 matrix (device,
+ * row-major, 16-byte aligned rows, cols a multiple of 8), same fp32 accumulation.  This is the
+ * dense product whose memory traffic the compression removes (Section 6).
+ */
+huffllm_status huffllm_plain_gemv(const uint16_t *w_dev, uint64_t rows, uint64_t cols, const uint16_t *x_dev,
+                                  float *y_dev, huffllm_stream stream);
+
+/* Message of the last failing call on this thread ("" if none). */
+const char *huffllm_last_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HUFFLLM_H */

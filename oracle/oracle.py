@@ -277,7 +277,7 @@ def decode_tensor(enc) -> np.ndarray:
 #   32 u32 tile_rows | 36 u32 chunk_cols | 40 u32 row_groups | 44 u32 col_chunks | 48 u64 n_chunks
 #   56 u32 lut_bits | 60 u32 lag_bits | 64 u32 n_fields | 68 u8 caps[4] | 72 u16 pad_word | 74 u16 0
 #   76 u32 max_words | 80 u64 off_codebook | 88 u64 off_lut | 96 u64 off_index | 104 u64 off_payload
-#   112 u64 payload_bytes | 120 u64 blob_bytes | 128 u64 coded_bits | 136 u64 raw_bits
+#   112 u64 payload_bytes | 120 u64 blob_bytes | 128 u64 coded_bits | 136 u64 raw_bits | 144 u64 checksum
 # codebook: u8 lengths[3][32].  LUT: u32[1 << lut_bits], entry = E << 23 | (len0 + len1), indexed by the
 # next lut_bits stream bits (first bit = bit 0).  index: u32[n_chunks + 1], record offsets in 128-byte
 # units from off_payload.  Record of a chunk with nkb blocks: raw bytes [nkb][32 lanes][16], then W rows

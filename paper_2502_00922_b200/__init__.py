@@ -1,0 +1,10 @@
+"""huffllm: Huffman-compressed bf16 weights decoded on the fly inside GPU matrix products.
+
+The Python layer only marshals arguments into the C-ABI library (``libhuffllm.so``); every
+step of the method runs in that library.  Importing this package fails loudly when the
+library has not been built — there is no fallback path.
+"""
+from .binding import (  # noqa: F401
+    BF16, FP16, HuffllmError, Codebook, Desc, lib, build_codebook, encode_bound, encode, validate_blob,
+    workspace_bytes, decode, decode_gemv, decode_gemm, decode_gemm_host, plain_gemv, last_error, exported_symbols,
+)

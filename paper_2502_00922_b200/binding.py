@@ -1,0 +1,192 @@
+"""ctypes binding of include/huffllm.h: same names, argument marshalling only."""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import numpy as np
+
+BF16, FP16 = 0, 1
+_SO = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libhuffllm.so")
+_lib = None
+
+STATUS = {0: "OK", 1: "INVALID_ARG", 2: "UNSUPPORTED", 3: "BUFFER_TOO_SMALL", 4: "CORRUPT", 5: "CUDA", 6: "NOMEM"}
+
+
+class HuffllmError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__(f"huffllm: {STATUS.get(status, status)}: {message}")
+        self.status = status
+        self.status_name = STATUS.get(status, str(status))
+
+
+class Desc(C.Structure):
+    """huffllm_desc: descriptor of an encoded tensor = first 256 bytes of the blob."""
+    _fields_ = [("magic", C.c_char * 4), ("version", C.c_uint32), ("dtype", C.c_uint32), ("chunk_elems", C.c_uint32),
+                ("rows", C.c_uint64), ("cols", C.c_uint64), ("tile_rows", C.c_uint32), ("chunk_cols", C.c_uint32),
+                ("row_groups", C.c_uint32), ("col_chunks", C.c_uint32), ("n_chunks", C.c_uint64),
+                ("lut_bits", C.c_uint32), ("lag_bits", C.c_uint32), ("n_fields", C.c_uint32), ("caps", C.c_uint8 * 4),
+                ("pad_word", C.c_uint16), ("reserved0", C.c_uint16), ("max_words", C.c_uint32),
+                ("off_codebook", C.c_uint64), ("off_lut", C.c_uint64), ("off_index", C.c_uint64),
+                ("off_payload", C.c_uint64), ("payload_bytes", C.c_uint64), ("blob_bytes", C.c_uint64),
+                ("coded_bits", C.c_uint64), ("raw_bits", C.c_uint64), ("payload_checksum", C.c_uint64),
+                ("reserved", C.c_uint8 * 104)]
+
+
+assert C.sizeof(Desc) == 256
+
+_SIGNATURES = {
+    "huffllm_build_codebook": [C.c_void_p, C.c_uint64, C.c_uint64, C.c_int, C.c_uint32, C.POINTER(C.c_void_p)],
+    "huffllm_codebook_get": [C.c_void_p, C.c_uint32, C.POINTER(C.c_uint32), C.c_void_p, C.c_void_p, C.c_void_p],
+    "huffllm_codebook_free": [C.c_void_p],
+    "huffllm_encode_bound": [C.c_uint64, C.c_uint64, C.c_int, C.c_uint32, C.POINTER(C.c_size_t)],
+    "huffllm_encode": [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint32, C.c_void_p, C.c_size_t, C.POINTER(Desc)],
+    "huffllm_validate_blob": [C.c_void_p, C.c_size_t, C.POINTER(Desc)],
+    "huffllm_workspace_bytes": [C.POINTER(Desc), C.c_uint32, C.POINTER(C.c_size_t)],
+    "huffllm_decode": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
+    "huffllm_decode_gemv": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
+    "huffllm_decode_gemm": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
+    "huffllm_decode_gemm_host": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                 C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
+    "huffllm_plain_gemv": [C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p],
+    "huffllm_last_error": [],
+}
+
+
+def exported_symbols():
+    """Names include/huffllm.h declares; the library must export every one of them."""
+    return sorted(_SIGNATURES)
+
+
+def lib():
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_SO):
+            raise ImportError(f"{_SO} is missing: build it with `python -m paper_2502_00922_b200.build` "
+                              "(there is no fallback implementation)")
+        L = C.CDLL(_SO)
+        for name, args in _SIGNATURES.items():
+            fn = getattr(L, name)
+            fn.argtypes = args
+            fn.restype = C.c_int
+        L.huffllm_codebook_free.restype = None
+        L.huffllm_last_error.restype = C.c_char_p
+        _lib = L
+    return _lib
+
+
+def last_error() -> str:
+    return lib().huffllm_last_error().decode()
+
+
+def _check(status: int):
+    if status != 0:
+        raise HuffllmError(status, last_error())
+
+
+def _ptr(t):
+    """Address of a torch tensor, a numpy array, an int, or None."""
+    if t is None:
+        return None
+    if isinstance(t, int):
+        return t
+    if isinstance(t, np.ndarray):
+        return t.ctypes.data
+    return t.data_ptr()
+
+
+def _stream(stream):
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    return stream if isinstance(stream, int) else stream.cuda_stream
+
+
+class Codebook:
+    """Owner of a huffllm_codebook*."""
+
+    def __init__(self, handle):
+        self._h = handle
+
+    def get(self, field: int):
+        n = C.c_uint32()
+        counts = np.zeros(32, np.uint64)
+        lengths = np.zeros(32, np.uint8)
+        codes = np.zeros(32, np.uint32)
+        _check(lib().huffllm_codebook_get(self._h, field, C.byref(n), counts.ctypes.data, lengths.ctypes.data, codes.ctypes.data))
+        return n.value, counts, lengths, codes
+
+    def free(self):
+        if self._h:
+            lib().huffllm_codebook_free(self._h)
+            self._h = None
+
+    def __del__(self):
+        try:
+            self.free()
+        except Exception:
+            pass
+
+
+def build_codebook(w: np.ndarray, dtype: int = BF16, max_code_len: int = 0) -> Codebook:
+    w = np.ascontiguousarray(w, dtype=np.uint16)
+    rows, cols = w.shape if w.ndim == 2 else (1, w.size)
+    h = C.c_void_p()
+    _check(lib().huffllm_build_codebook(w.ctypes.data, rows, cols, dtype, max_code_len, C.byref(h)))
+    return Codebook(h)
+
+
+def encode_bound(rows: int, cols: int, dtype: int = BF16, chunk_elems: int = 4096) -> int:
+    n = C.c_size_t()
+    _check(lib().huffllm_encode_bound(rows, cols, dtype, chunk_elems, C.byref(n)))
+    return n.value
+
+
+def encode(cb: Codebook, w: np.ndarray, chunk_elems: int = 4096):
+    """Returns (blob as a numpy uint8 array trimmed to its size, Desc)."""
+    w = np.ascontiguousarray(w, dtype=np.uint16)
+    rows, cols = w.shape
+    cap = encode_bound(rows, cols, BF16, chunk_elems)
+    buf = np.empty(cap, dtype=np.uint8)
+    d = Desc()
+    _check(lib().huffllm_encode(cb._h, w.ctypes.data, rows, cols, chunk_elems, buf.ctypes.data, cap, C.byref(d)))
+    return buf[:d.blob_bytes].copy(), d
+
+
+def validate_blob(blob: np.ndarray) -> Desc:
+    blob = np.ascontiguousarray(blob, dtype=np.uint8)
+    d = Desc()
+    _check(lib().huffllm_validate_blob(blob.ctypes.data, blob.size, C.byref(d)))
+    return d
+
+
+def workspace_bytes(desc: Desc, batch: int = 1) -> int:
+    n = C.c_size_t()
+    _check(lib().huffllm_workspace_bytes(C.byref(desc), batch, C.byref(n)))
+    return n.value
+
+
+def decode(desc: Desc, blob_dev, out_dev, err_flag_dev=None, stream=None):
+    _check(lib().huffllm_decode(C.byref(desc), _ptr(blob_dev), _ptr(out_dev), _ptr(err_flag_dev), _stream(stream)))
+
+
+def decode_gemv(desc: Desc, blob_dev, x_dev, y_dev, workspace_dev, workspace_bytes_: int, err_flag_dev=None, stream=None):
+    _check(lib().huffllm_decode_gemv(C.byref(desc), _ptr(blob_dev), _ptr(x_dev), _ptr(y_dev), _ptr(workspace_dev),
+                                     workspace_bytes_, _ptr(err_flag_dev), _stream(stream)))
+
+
+def decode_gemm(desc: Desc, blob_dev, x_dev, batch: int, y_dev, workspace_dev, workspace_bytes_: int, err_flag_dev=None,
+                stream=None):
+    _check(lib().huffllm_decode_gemm(C.byref(desc), _ptr(blob_dev), _ptr(x_dev), batch, _ptr(y_dev), _ptr(workspace_dev),
+                                     workspace_bytes_, _ptr(err_flag_dev), _stream(stream)))
+
+
+def decode_gemm_host(desc: Desc, blob_dev, x_host, batch: int, y_host, x_stage_dev, y_stage_dev, workspace_dev,
+                     workspace_bytes_: int, err_flag_dev=None, stream=None):
+    _check(lib().huffllm_decode_gemm_host(C.byref(desc), _ptr(blob_dev), _ptr(x_host), batch, _ptr(y_host),
+                                          _ptr(x_stage_dev), _ptr(y_stage_dev), _ptr(workspace_dev), workspace_bytes_,
+                                          _ptr(err_flag_dev), _stream(stream)))
+
+
+def plain_gemv(w_dev, rows: int, cols: int, x_dev, y_dev, stream=None):
+    _check(lib().huffllm_plain_gemv(_ptr(w_dev), rows, cols, _ptr(x_dev), _ptr(y_dev), _stream(stream)))

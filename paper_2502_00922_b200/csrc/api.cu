@@ -1,0 +1,177 @@
+// C-ABI entry points that run on the device: argument checks, launch geometry, launches.
+// No allocation and no synchronisation here (huffllm_decode_gemm_host, which exists to be timed
+// end to end with host buffers, is the one call that waits for its stream).
+#include <cuda_runtime.h>
+#include <cstring>
+
+#include "internal.h"
+#include "kernels.h"
+
+using namespace huffllm;
+
+namespace {
+
+constexpr uint32_t kMaxGrid = 512;        // CTAs the scratch layout provides for
+constexpr uint32_t kKernelBatch = 8;      // activation vectors one launch multiplies
+constexpr uint32_t kStaticSmem = 1024;    // barriers and tags the kernel declares statically (rounded up)
+
+struct DeviceInfo {
+    bool known = false;
+    int sms = 0, smem_optin = 0;
+};
+DeviceInfo g_dev[64];
+
+huffllm_status device_info(DeviceInfo **out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+    if (dev < 0 || dev >= 64) return fail(HUFFLLM_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
+    DeviceInfo &d = g_dev[dev];
+    if (!d.known) {
+        if ((e = cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess ||
+            (e = cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess)
+            return fail(HUFFLLM_ERR_CUDA, "cudaDeviceGetAttribute: %s", cudaGetErrorString(e));
+        d.known = true;
+    }
+    *out = &d;
+    return HUFFLLM_OK;
+}
+
+// Scratch layout: [0,256) ticket | [256, 256 + 8*kMaxGrid) row-group tags | partial sums
+size_t ws_partial_offset() { return 256 + (size_t)kMaxGrid * 2 * sizeof(int); }
+size_t ws_bytes_for(uint32_t batch) {
+    uint32_t b = batch < kKernelBatch ? batch : kKernelBatch;
+    return ws_partial_offset() + (size_t)kMaxGrid * 2 * 16 * b * sizeof(float);
+}
+
+huffllm_status fill_args(const huffllm_desc *desc, const void *blob, uint32_t batch, bool product, const DeviceInfo &dev,
+                         KernelArgs *k, uint32_t *grid) {
+    huffllm_status st = check_desc(desc);
+    if (st != HUFFLLM_OK) return st;
+    if (!blob || ((uintptr_t)blob & 255)) return fail(HUFFLLM_ERR_INVALID_ARG, "blob must be a 256-byte aligned device pointer");
+    if (desc->lut_bits > 9)
+        return fail(HUFFLLM_ERR_UNSUPPORTED, "device kernels take max_code_len 8 or 9 (this blob: %u)", desc->lut_bits);
+    memset(k, 0, sizeof(*k));
+    k->blob = (const uint8_t *)blob;
+    k->off_lut = desc->off_lut;
+    k->off_index = desc->off_index;
+    k->off_payload = desc->off_payload;
+    k->payload_units = (uint32_t)(desc->payload_bytes / kRecordUnit);
+    k->rows = desc->rows;
+    k->cols = desc->cols;
+    k->n_chunks = desc->n_chunks;
+    k->chunk_cols = desc->chunk_cols;
+    k->col_chunks = desc->col_chunks;
+    k->lut_bits = desc->lut_bits;
+    k->slot_bytes = (desc->max_words + 1) * 128;
+    const uint32_t checks_per_block = desc->lut_bits == 8 ? 6 : 8;
+    k->guard_bytes = 128 * (3 + checks_per_block * (desc->chunk_cols / kBlockCols));
+    k->part_bytes = product ? 2 * 32 * 16 * batch * (uint32_t)sizeof(float) : 0;
+    k->dyn_smem_bytes = (uint32_t)dev.smem_optin - kStaticSmem;
+    k->batch = batch;
+    // worst case for the table's alignment gap is covered by assuming the window starts within 4 KB of zero
+    uint64_t fixed = (128ull << desc->lut_bits) + k->guard_bytes + k->part_bytes + 4096;
+    if (fixed + 2ull * k->slot_bytes > k->dyn_smem_bytes)
+        return fail(HUFFLLM_ERR_UNSUPPORTED, "chunk records too large for shared memory (max_words %u)", desc->max_words);
+    uint64_t g = desc->n_chunks < (uint64_t)dev.sms ? desc->n_chunks : (uint64_t)dev.sms;
+    *grid = (uint32_t)(g < kMaxGrid ? g : kMaxGrid);
+    return HUFFLLM_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+huffllm_status huffllm_workspace_bytes(const huffllm_desc *desc, uint32_t batch, size_t *bytes) {
+    clear_error();
+    if (!bytes) return fail(HUFFLLM_ERR_INVALID_ARG, "bytes is null");
+    huffllm_status st = check_desc(desc);
+    if (st != HUFFLLM_OK) return st;
+    if (batch == 0 || batch > 64) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be in [1, 64]");
+    *bytes = ws_bytes_for(batch);
+    return HUFFLLM_OK;
+}
+
+huffllm_status huffllm_decode(const huffllm_desc *desc, const void *blob, uint16_t *out, int32_t *err_flag, huffllm_stream stream) {
+    clear_error();
+    DeviceInfo *dev;
+    huffllm_status st = device_info(&dev);
+    if (st != HUFFLLM_OK) return st;
+    if (!out || ((uintptr_t)out & 15)) return fail(HUFFLLM_ERR_INVALID_ARG, "out must be a 16-byte aligned device pointer");
+    KernelArgs k;
+    uint32_t grid;
+    if ((st = fill_args(desc, blob, 1, false, *dev, &k, &grid)) != HUFFLLM_OK) return st;
+    k.out = out;
+    k.err = err_flag;
+    cudaError_t e = launch_decode(k, grid, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "decode launch: %s", cudaGetErrorString(e));
+    return HUFFLLM_OK;
+}
+
+huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, const uint16_t *x, uint32_t batch, float *y,
+                                   void *workspace, size_t workspace_bytes, int32_t *err_flag, huffllm_stream stream) {
+    clear_error();
+    DeviceInfo *dev;
+    huffllm_status st = device_info(&dev);
+    if (st != HUFFLLM_OK) return st;
+    if (!x || !y || !workspace) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
+    if (batch == 0 || batch > 64) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be in [1, 64]");
+    if (((uintptr_t)x & 15) || ((uintptr_t)y & 3) || ((uintptr_t)workspace & 255))
+        return fail(HUFFLLM_ERR_INVALID_ARG, "x must be 16-byte, y 4-byte, workspace 256-byte aligned");
+    if (workspace_bytes < ws_bytes_for(batch)) return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "workspace too small");
+    st = check_desc(desc);
+    if (st != HUFFLLM_OK) return st;
+    if (desc->cols % 8) return fail(HUFFLLM_ERR_UNSUPPORTED, "fused products need cols to be a multiple of 8");
+    if (desc->cols % kBlockCols && ((desc->pad_word >> 7) & 0xFF) == 0xFF)
+        return fail(HUFFLLM_ERR_UNSUPPORTED, "pad weights are not finite for this tensor");
+    for (uint32_t b0 = 0; b0 < batch; b0 += kKernelBatch) {
+        uint32_t nb = batch - b0 < kKernelBatch ? batch - b0 : kKernelBatch;
+        KernelArgs k;
+        uint32_t grid;
+        if ((st = fill_args(desc, blob, nb, true, *dev, &k, &grid)) != HUFFLLM_OK) return st;
+        k.x = x + (uint64_t)b0 * desc->cols;
+        k.y = y + (uint64_t)b0 * desc->rows;
+        k.ws_ticket = (unsigned int *)workspace;
+        k.ws_rg = (int *)((uint8_t *)workspace + 256);
+        k.ws_partial = (float *)((uint8_t *)workspace + ws_partial_offset());
+        k.err = err_flag;
+        cudaError_t e = launch_gemm(k, grid, (cudaStream_t)stream);
+        if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "product launch: %s", cudaGetErrorString(e));
+    }
+    return HUFFLLM_OK;
+}
+
+huffllm_status huffllm_decode_gemv(const huffllm_desc *desc, const void *blob, const uint16_t *x, float *y, void *workspace,
+                                   size_t workspace_bytes, int32_t *err_flag, huffllm_stream stream) {
+    return huffllm_decode_gemm(desc, blob, x, 1, y, workspace, workspace_bytes, err_flag, stream);
+}
+
+huffllm_status huffllm_decode_gemm_host(const huffllm_desc *desc, const void *blob, const uint16_t *x_host, uint32_t batch,
+                                        float *y_host, uint16_t *x_stage, float *y_stage, void *workspace,
+                                        size_t workspace_bytes, int32_t *err_flag, huffllm_stream stream) {
+    clear_error();
+    if (!desc || !x_host || !y_host || !x_stage || !y_stage) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
+    cudaStream_t s = (cudaStream_t)stream;
+    cudaError_t e = cudaMemcpyAsync(x_stage, x_host, (size_t)batch * desc->cols * 2, cudaMemcpyHostToDevice, s);
+    if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "copy of x: %s", cudaGetErrorString(e));
+    huffllm_status st = huffllm_decode_gemm(desc, blob, x_stage, batch, y_stage, workspace, workspace_bytes, err_flag, stream);
+    if (st != HUFFLLM_OK) return st;
+    e = cudaMemcpyAsync(y_host, y_stage, (size_t)batch * desc->rows * 4, cudaMemcpyDeviceToHost, s);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "copy of y: %s", cudaGetErrorString(e));
+    return HUFFLLM_OK;
+}
+
+huffllm_status huffllm_plain_gemv(const uint16_t *w, uint64_t rows, uint64_t cols, const uint16_t *x, float *y, huffllm_stream stream) {
+    clear_error();
+    DeviceInfo *dev;
+    huffllm_status st = device_info(&dev);
+    if (st != HUFFLLM_OK) return st;
+    if (!w || !x || !y || rows == 0 || cols == 0) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer or empty matrix");
+    if (cols % 8 || ((uintptr_t)w & 15) || ((uintptr_t)x & 15)) return fail(HUFFLLM_ERR_UNSUPPORTED, "cols must be a multiple of 8 and pointers 16-byte aligned");
+    cudaError_t e = launch_plain_gemv(w, rows, cols, x, y, (uint32_t)dev->sms, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "plain gemv launch: %s", cudaGetErrorString(e));
+    return HUFFLLM_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,554 @@
+// Host side of the library: codebook construction, encoder, blob validator.
+//
+// Compression runs once, offline, on the CPU (Section 3.1).  The field split is the paper's
+// BF16 {1,4,4,7} scheme (Section 5.1): sign and mantissa stay raw, the exponent is coded as two
+// 4-bit groups, each with its own Huffman code.  Code lengths are bounded by a fixed L_max
+// (Section 3.2) — here a joint bound on the two nibble codes of one weight, so that the device
+// can resolve both with a single table lookup.
+#include <algorithm>
+#include <atomic>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+#include <thread>
+#include <vector>
+
+#include "internal.h"
+
+namespace huffllm {
+
+static thread_local char g_err[512] = "";
+
+huffllm_status fail(huffllm_status st, const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return st;
+}
+void clear_error() { g_err[0] = 0; }
+
+static inline uint64_t align_up(uint64_t v, uint64_t a) { return (v + a - 1) / a * a; }
+
+// Order-independent checksum term of one chunk record.
+static inline uint64_t record_checksum(const uint8_t *p, uint64_t n, uint64_t chunk_id) {
+    uint64_t h = 1469598103934665603ull;
+    for (uint64_t i = 0; i < n; ++i) h = (h ^ p[i]) * 1099511628211ull;
+    return h * (2 * chunk_id + 1);
+}
+
+huffllm_status check_desc(const huffllm_desc *d) {
+    if (!d) return fail(HUFFLLM_ERR_INVALID_ARG, "descriptor is null");
+    if (memcmp(d->magic, "HFLM", 4) != 0 || d->version != 1) return fail(HUFFLLM_ERR_CORRUPT, "bad magic or version");
+    if (d->dtype != HUFFLLM_BF16) return fail(HUFFLLM_ERR_UNSUPPORTED, "only bf16 blobs are supported");
+    if (d->rows == 0 || d->cols == 0 || d->rows > (1ull << 31) || d->cols > (1ull << 31))
+        return fail(HUFFLLM_ERR_CORRUPT, "bad shape");
+    if (d->chunk_elems % (kTileRows * kBlockCols) || d->chunk_elems < 512 || d->chunk_elems > 16384)
+        return fail(HUFFLLM_ERR_CORRUPT, "bad chunk_elems");
+    if (d->tile_rows != kTileRows || d->chunk_cols != d->chunk_elems / kTileRows || d->lag_bits != kLagBits ||
+        d->n_fields != 2)
+        return fail(HUFFLLM_ERR_CORRUPT, "bad tile geometry");
+    if (d->row_groups != (d->rows + kTileRows - 1) / kTileRows ||
+        d->col_chunks != (d->cols + d->chunk_cols - 1) / d->chunk_cols ||
+        d->n_chunks != (uint64_t)d->row_groups * d->col_chunks)
+        return fail(HUFFLLM_ERR_CORRUPT, "chunk counts do not match the shape");
+    if (d->lut_bits < kMinBudget || d->lut_bits > kMaxBudget) return fail(HUFFLLM_ERR_CORRUPT, "bad lut_bits");
+    uint32_t max_steps = d->chunk_cols / kBlockCols * 16;
+    uint32_t w_bound = (kLagBits + max_steps * d->lut_bits + 31) / 32;
+    if (d->max_words == 0 || d->max_words > w_bound) return fail(HUFFLLM_ERR_CORRUPT, "bad max_words");
+    if (d->off_codebook % 256 || d->off_lut % 256 || d->off_index % 256 || d->off_payload % 256 ||
+        d->off_codebook < 256 || d->off_lut < d->off_codebook + 96 ||
+        d->off_index < d->off_lut + (4ull << d->lut_bits) || d->off_payload < d->off_index + 4 * (d->n_chunks + 1) ||
+        d->payload_bytes % kRecordUnit || d->blob_bytes < d->off_payload + d->payload_bytes ||
+        d->payload_bytes / kRecordUnit > 0xFFFFFFFFull)
+        return fail(HUFFLLM_ERR_CORRUPT, "bad section offsets");
+    return HUFFLLM_OK;
+}
+
+// ------------------------------------------------------------------ code construction
+
+// Optimal prefix-code lengths with every length <= cap, by exhaustive dynamic programming over
+// the Kraft budget: state = (symbols placed, budget spent in units of 2^-cap).
+static bool limited_lengths(const uint64_t *counts, int nsym, int cap, uint8_t *len) {
+    std::vector<int> used;
+    for (int s = 0; s < nsym; ++s) {
+        len[s] = 0;
+        if (counts[s]) used.push_back(s);
+    }
+    int n = (int)used.size();
+    if (n == 0) return false;
+    if (n == 1) { len[used[0]] = 1; return true; }
+    if (cap < 1 || cap > 15 || (1 << cap) < n) return false;
+    std::stable_sort(used.begin(), used.end(), [&](int a, int b) { return counts[a] > counts[b]; });
+    const int U = 1 << cap;
+    const uint64_t INF = ~0ull;
+    std::vector<uint64_t> cost((size_t)(n + 1) * (U + 1), INF);
+    std::vector<uint8_t> choice((size_t)(n + 1) * (U + 1), 0);
+    cost[0] = 0;
+    for (int i = 0; i < n; ++i)
+        for (int b = 0; b <= U; ++b) {
+            uint64_t c = cost[(size_t)i * (U + 1) + b];
+            if (c == INF) continue;
+            for (int l = 1; l <= cap; ++l) {
+                int nb = b + (U >> l);
+                if (nb > U) continue;
+                uint64_t v = c + counts[used[i]] * (uint64_t)l;
+                size_t k = (size_t)(i + 1) * (U + 1) + nb;
+                if (v < cost[k]) { cost[k] = v; choice[k] = (uint8_t)l; }
+            }
+        }
+    int best_b = -1;
+    for (int b = 0; b <= U; ++b)
+        if (cost[(size_t)n * (U + 1) + b] != INF &&
+            (best_b < 0 || cost[(size_t)n * (U + 1) + b] < cost[(size_t)n * (U + 1) + best_b]))
+            best_b = b;
+    if (best_b < 0) return false;
+    for (int i = n, b = best_b; i > 0; --i) {
+        int l = choice[(size_t)i * (U + 1) + b];
+        len[used[i - 1]] = (uint8_t)l;
+        b -= U >> l;
+    }
+    return true;
+}
+
+static uint64_t code_cost(const uint64_t *counts, const uint8_t *len, int nsym) {
+    uint64_t c = 0;
+    for (int s = 0; s < nsym; ++s) c += counts[s] * len[s];
+    return c;
+}
+
+static void canonical_codes(const uint8_t *len, int nsym, uint32_t *code) {
+    std::vector<int> order;
+    for (int s = 0; s < nsym; ++s) {
+        code[s] = 0;
+        if (len[s]) order.push_back(s);
+    }
+    std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return len[a] < len[b]; });
+    uint32_t next = 0;
+    for (size_t i = 0; i < order.size(); ++i) {
+        if (i) next = (next + 1) << (len[order[i]] - len[order[i - 1]]);
+        code[order[i]] = next;
+    }
+}
+
+static uint32_t reverse_bits(uint32_t v, int n) {
+    uint32_t r = 0;
+    for (int i = 0; i < n; ++i) r |= ((v >> i) & 1u) << (n - 1 - i);
+    return r;
+}
+
+}  // namespace huffllm
+
+using namespace huffllm;
+
+struct huffllm_codebook {
+    uint32_t dtype, budget;
+    uint64_t counts[3][32];
+    uint8_t len[3][32];
+    uint32_t code[3][32];
+    uint8_t caps[4];
+    uint16_t pad_word;
+    uint8_t len8[256];    // code length of a whole exponent byte (hi + lo), 0 = no codeword
+    uint32_t bits8[256];  // its stream bits, first bit in bit 0
+    std::vector<uint32_t> lut;
+};
+
+// Fill len8 / bits8 / lut / pad_word from len[] and code[].
+static void finish_codebook(huffllm_codebook *cb) {
+    memset(cb->len8, 0, sizeof(cb->len8));
+    memset(cb->bits8, 0, sizeof(cb->bits8));
+    cb->lut.assign((size_t)1 << cb->budget, 0u);
+    for (int e = 0; e < 256; ++e) {
+        int h = e >> 4, l = e & 15;
+        int lh = cb->len[0][h], ll = cb->len[1][l];
+        if (!lh || !ll) continue;
+        uint32_t seq = reverse_bits(cb->code[0][h], lh) | (reverse_bits(cb->code[1][l], ll) << lh);
+        int L = lh + ll;
+        cb->len8[e] = (uint8_t)L;
+        cb->bits8[e] = seq;
+        for (uint32_t hi = 0; hi < (1u << (cb->budget - L)); ++hi)
+            cb->lut[seq | (hi << L)] = ((uint32_t)e << 23) | (uint32_t)L;
+    }
+    int f[2];
+    for (int k = 0; k < 2; ++k) {
+        int best = -1;
+        for (int s = 0; s < 16; ++s)
+            if (cb->len[k][s] && (best < 0 || cb->len[k][s] < cb->len[k][best])) best = s;
+        f[k] = best;
+    }
+    cb->pad_word = (uint16_t)(((f[0] << 4) | f[1]) << 7);
+}
+
+extern "C" {
+
+const char *huffllm_last_error(void) { return g_err; }
+
+huffllm_status huffllm_build_codebook(const uint16_t *w, uint64_t rows, uint64_t cols, huffllm_dtype dtype,
+                                      uint32_t max_code_len, huffllm_codebook **out) {
+    clear_error();
+    if (!w || !out || rows == 0 || cols == 0) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer or empty tensor");
+    if (dtype == HUFFLLM_FP16) return fail(HUFFLLM_ERR_UNSUPPORTED, "fp16 {1,5,5,5} is not built yet");
+    if (dtype != HUFFLLM_BF16) return fail(HUFFLLM_ERR_INVALID_ARG, "bad dtype");
+    uint32_t budget = max_code_len ? max_code_len : kDefaultBudget;
+    if (budget < kMinBudget || budget > kMaxBudget)
+        return fail(HUFFLLM_ERR_UNSUPPORTED, "max_code_len must be 0 or in [%u, %u]", kMinBudget, kMaxBudget);
+    huffllm_codebook *cb = new (std::nothrow) huffllm_codebook();
+    if (!cb) return fail(HUFFLLM_ERR_NOMEM, "out of host memory");
+    cb->dtype = dtype;
+    cb->budget = budget;
+    memset(cb->counts, 0, sizeof(cb->counts));
+    memset(cb->len, 0, sizeof(cb->len));
+    memset(cb->code, 0, sizeof(cb->code));
+    memset(cb->caps, 0, sizeof(cb->caps));
+
+    // histogram of the exponent byte, threaded over slices, then folded into the two nibble fields
+    const uint64_t n = rows * cols;
+    unsigned nt = std::max(1u, std::min(16u, std::thread::hardware_concurrency()));
+    if (n < (1u << 20)) nt = 1;
+    std::vector<std::vector<uint64_t>> part(nt, std::vector<uint64_t>(256, 0));
+    std::vector<std::thread> th;
+    for (unsigned t = 0; t < nt; ++t)
+        th.emplace_back([&, t] {
+            uint64_t a = n * t / nt, b = n * (t + 1) / nt;
+            uint64_t *h = part[t].data();
+            for (uint64_t i = a; i < b; ++i) h[(w[i] >> 7) & 0xFF]++;
+        });
+    for (auto &x : th) x.join();
+    for (unsigned t = 0; t < nt; ++t)
+        for (int e = 0; e < 256; ++e) {
+            cb->counts[0][e >> 4] += part[t][e];
+            cb->counts[1][e & 15] += part[t][e];
+        }
+
+    bool have = false;
+    uint64_t best = 0;
+    uint8_t l0[32], l1[32];
+    for (uint32_t c0 = 1; c0 < budget; ++c0) {
+        uint32_t c1 = budget - c0;
+        if (!limited_lengths(cb->counts[0], 16, (int)c0, l0) || !limited_lengths(cb->counts[1], 16, (int)c1, l1)) continue;
+        uint64_t cost = code_cost(cb->counts[0], l0, 16) + code_cost(cb->counts[1], l1, 16);
+        if (!have || cost < best) {
+            have = true;
+            best = cost;
+            cb->caps[0] = (uint8_t)c0;
+            cb->caps[1] = (uint8_t)c1;
+            memcpy(cb->len[0], l0, 16);
+            memcpy(cb->len[1], l1, 16);
+        }
+    }
+    if (!have) {
+        delete cb;
+        return fail(HUFFLLM_ERR_INVALID_ARG, "no code fits max_code_len");
+    }
+    canonical_codes(cb->len[0], 16, cb->code[0]);
+    canonical_codes(cb->len[1], 16, cb->code[1]);
+    finish_codebook(cb);
+    *out = cb;
+    return HUFFLLM_OK;
+}
+
+huffllm_status huffllm_codebook_get(const huffllm_codebook *cb, uint32_t field, uint32_t *n_symbols, uint64_t counts[32],
+                                    uint8_t lengths[32], uint32_t codes[32]) {
+    clear_error();
+    if (!cb || field >= 2) return fail(HUFFLLM_ERR_INVALID_ARG, "bad codebook or field");
+    if (n_symbols) *n_symbols = 16;
+    for (int s = 0; s < 32; ++s) {
+        if (counts) counts[s] = cb->counts[field][s];
+        if (lengths) lengths[s] = cb->len[field][s];
+        if (codes) codes[s] = cb->code[field][s];
+    }
+    return HUFFLLM_OK;
+}
+
+void huffllm_codebook_free(huffllm_codebook *cb) { delete cb; }
+
+}  // extern "C"
+
+// ------------------------------------------------------------------------------ encoder
+
+namespace {
+
+struct Geometry {
+    uint64_t rows, cols;
+    uint32_t Kc, RG, KC;
+};
+
+bool make_geometry(uint64_t rows, uint64_t cols, uint32_t chunk_elems, Geometry *g) {
+    if (chunk_elems % (kTileRows * kBlockCols) || chunk_elems < 512 || chunk_elems > 16384) return false;
+    if (rows == 0 || cols == 0 || rows > (1ull << 31) || cols > (1ull << 31)) return false;
+    g->rows = rows;
+    g->cols = cols;
+    g->Kc = chunk_elems / kTileRows;
+    g->RG = (uint32_t)((rows + kTileRows - 1) / kTileRows);
+    g->KC = (uint32_t)((cols + g->Kc - 1) / g->Kc);
+    return true;
+}
+
+inline uint32_t blocks_of(const Geometry &g, uint32_t kc) {
+    uint64_t left = g.cols - (uint64_t)kc * g.Kc;
+    return (uint32_t)((std::min<uint64_t>(left, g.Kc) + kBlockCols - 1) / kBlockCols);
+}
+
+// The weight at (chunk, lane, step) of the element map, or the pad word outside the tensor.
+inline uint16_t weight_at(const uint16_t *w, const Geometry &g, uint32_t rg, uint32_t kc, uint32_t lane, uint32_t step,
+                          uint16_t pad) {
+    uint32_t gg = lane >> 2, t = lane & 3, kb = step >> 4, half = (step >> 3) & 1, i = step & 7;
+    uint64_t r = (uint64_t)rg * 16 + gg + 8 * half;
+    uint64_t c = (uint64_t)kc * g.Kc + (uint64_t)kb * 32 + t * 8 + i;
+    return (r < g.rows && c < g.cols) ? w[r * g.cols + c] : pad;
+}
+
+template <class F>
+void parallel_chunks(uint64_t n, F f) {
+    unsigned nt = std::max(1u, std::min(16u, std::thread::hardware_concurrency()));
+    if (n < 64) nt = 1;
+    std::atomic<uint64_t> next{0};
+    std::vector<std::thread> th;
+    for (unsigned t = 0; t < nt; ++t)
+        th.emplace_back([&] {
+            for (;;) {
+                uint64_t a = next.fetch_add(16);
+                if (a >= n) break;
+                for (uint64_t c = a; c < std::min(n, a + 16); ++c) f(c);
+            }
+        });
+    for (auto &x : th) x.join();
+}
+
+}  // namespace
+
+extern "C" {
+
+huffllm_status huffllm_encode_bound(uint64_t rows, uint64_t cols, huffllm_dtype dtype, uint32_t chunk_elems,
+                                    size_t *max_bytes) {
+    clear_error();
+    Geometry g;
+    if (!max_bytes) return fail(HUFFLLM_ERR_INVALID_ARG, "max_bytes is null");
+    if (dtype != HUFFLLM_BF16) return fail(HUFFLLM_ERR_UNSUPPORTED, "only bf16 is supported");
+    if (!make_geometry(rows, cols, chunk_elems, &g)) return fail(HUFFLLM_ERR_INVALID_ARG, "bad shape or chunk_elems");
+    uint64_t payload = 0;
+    for (uint32_t kc = 0; kc < g.KC; ++kc) {
+        uint32_t nkb = blocks_of(g, kc);
+        uint64_t w = (kLagBits + (uint64_t)nkb * 16 * kMaxBudget + 31) / 32;
+        payload += (uint64_t)g.RG * (nkb * 512ull + w * 128ull);
+    }
+    uint64_t n_chunks = (uint64_t)g.RG * g.KC;
+    *max_bytes = (size_t)(256 + 256 + align_up(4ull << kMaxBudget, 256) + align_up(4 * (n_chunks + 1), 256) + payload + 256);
+    return HUFFLLM_OK;
+}
+
+huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uint64_t rows, uint64_t cols,
+                              uint32_t chunk_elems, void *blob, size_t blob_cap, huffllm_desc *desc) {
+    clear_error();
+    if (!cb || !w || !blob || !desc) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
+    Geometry g;
+    if (!make_geometry(rows, cols, chunk_elems, &g)) return fail(HUFFLLM_ERR_INVALID_ARG, "bad shape or chunk_elems");
+    const uint64_t n_chunks = (uint64_t)g.RG * g.KC;
+
+    huffllm_desc d;
+    memset(&d, 0, sizeof(d));
+    memcpy(d.magic, "HFLM", 4);
+    d.version = 1;
+    d.dtype = cb->dtype;
+    d.chunk_elems = chunk_elems;
+    d.rows = rows;
+    d.cols = cols;
+    d.tile_rows = kTileRows;
+    d.chunk_cols = g.Kc;
+    d.row_groups = g.RG;
+    d.col_chunks = g.KC;
+    d.n_chunks = n_chunks;
+    d.lut_bits = cb->budget;
+    d.lag_bits = kLagBits;
+    d.n_fields = 2;
+    memcpy(d.caps, cb->caps, 4);
+    d.pad_word = cb->pad_word;
+    d.off_codebook = 256;
+    d.off_lut = 512;
+    d.off_index = d.off_lut + align_up(4ull << cb->budget, 256);
+    d.off_payload = d.off_index + align_up(4 * (n_chunks + 1), 256);
+    if (blob_cap < d.off_payload) return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "blob capacity below the fixed sections");
+
+    // pass 1: words per lane row (W) of every chunk, from the code lengths alone
+    std::vector<uint32_t> words(n_chunks);
+    std::vector<uint64_t> chunk_bits(n_chunks);
+    std::atomic<int> bad{0};
+    const uint8_t *len8 = cb->len8;
+    const uint16_t pad = cb->pad_word;
+    parallel_chunks(n_chunks, [&](uint64_t c) {
+        uint32_t rg = (uint32_t)(c / g.KC), kc = (uint32_t)(c % g.KC), steps = blocks_of(g, kc) * 16;
+        uint32_t max_bits = 0;
+        uint64_t sum = 0;
+        for (uint32_t lane = 0; lane < 32; ++lane) {
+            uint32_t bits = 0;
+            for (uint32_t s = 0; s < steps; ++s) {
+                uint32_t l = len8[(weight_at(w, g, rg, kc, lane, s, pad) >> 7) & 0xFF];
+                if (!l) bad.store(1);
+                bits += l;
+            }
+            sum += bits;
+            max_bits = std::max(max_bits, bits + kLagBits);
+        }
+        words[c] = std::max(1u, (max_bits + 31) / 32);
+        chunk_bits[c] = sum;
+    });
+    if (bad.load()) return fail(HUFFLLM_ERR_INVALID_ARG, "a weight uses a symbol the codebook has no codeword for");
+
+    uint8_t *base = (uint8_t *)blob;
+    std::vector<uint64_t> rec(n_chunks + 1, 0);
+    uint32_t max_words = 0;
+    uint64_t coded_bits = 0;
+    for (uint64_t c = 0; c < n_chunks; ++c) {
+        uint32_t nkb = blocks_of(g, (uint32_t)(c % g.KC));
+        rec[c + 1] = rec[c] + (nkb * 512ull + words[c] * 128ull) / kRecordUnit;
+        max_words = std::max(max_words, words[c]);
+        coded_bits += chunk_bits[c];
+    }
+    d.max_words = max_words;
+    d.payload_bytes = rec[n_chunks] * kRecordUnit;
+    d.blob_bytes = d.off_payload + d.payload_bytes;
+    d.coded_bits = coded_bits;
+    d.raw_bits = 8 * rows * cols;
+    if (rec[n_chunks] > 0xFFFFFFFFull) return fail(HUFFLLM_ERR_UNSUPPORTED, "payload exceeds the 32-bit record index");
+    if (blob_cap < d.blob_bytes)
+        return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "blob needs %llu bytes, capacity is %llu", (unsigned long long)d.blob_bytes,
+                    (unsigned long long)blob_cap);
+
+    memset(base, 0, d.off_payload);
+    memcpy(base, &d, sizeof(d));
+    for (int k = 0; k < 3; ++k) memcpy(base + d.off_codebook + 32 * k, cb->len[k], 32);
+    memcpy(base + d.off_lut, cb->lut.data(), 4ull << cb->budget);
+    uint32_t *index = (uint32_t *)(base + d.off_index);
+    for (uint64_t c = 0; c <= n_chunks; ++c) index[c] = (uint32_t)rec[c];
+
+    // pass 2: write the records
+    const uint32_t *bits8 = cb->bits8;
+    std::atomic<uint64_t> checksum{0};
+    parallel_chunks(n_chunks, [&](uint64_t c) {
+        uint32_t rg = (uint32_t)(c / g.KC), kc = (uint32_t)(c % g.KC), nkb = blocks_of(g, kc), steps = nkb * 16;
+        uint32_t W = words[c];
+        uint8_t *raw = base + d.off_payload + rec[c] * kRecordUnit;
+        uint32_t *coded = (uint32_t *)(raw + nkb * 512ull);
+        memset(coded, 0, (size_t)W * 128);
+        for (uint32_t lane = 0; lane < 32; ++lane) {
+            uint64_t acc = 0;
+            uint32_t nacc = kLagBits, j = 0;
+            for (uint32_t s = 0; s < steps; ++s) {
+                uint16_t v = weight_at(w, g, rg, kc, lane, s, pad);
+                raw[(s >> 4) * 512 + lane * 16 + (s & 15)] = (uint8_t)(((v >> 8) & 0x80) | (v & 0x7F));
+                uint32_t e = (v >> 7) & 0xFF;
+                acc |= (uint64_t)bits8[e] << nacc;
+                nacc += len8[e];
+                if (nacc >= 32) {
+                    coded[(size_t)j++ * 32 + lane] = (uint32_t)acc;
+                    acc >>= 32;
+                    nacc -= 32;
+                }
+            }
+            if (nacc) coded[(size_t)j * 32 + lane] = (uint32_t)acc;
+        }
+        checksum.fetch_add(record_checksum(raw, nkb * 512ull + (uint64_t)W * 128, c));
+    });
+    d.payload_checksum = checksum.load();
+    memcpy(base, &d, sizeof(d));
+    *desc = d;
+    return HUFFLLM_OK;
+}
+
+huffllm_status huffllm_validate_blob(const void *blob, size_t bytes, huffllm_desc *desc_out) {
+    clear_error();
+    if (!blob || bytes < 256) return fail(HUFFLLM_ERR_CORRUPT, "blob shorter than its header");
+    huffllm_desc d;
+    memcpy(&d, blob, sizeof(d));
+    huffllm_status st = check_desc(&d);
+    if (st != HUFFLLM_OK) return st == HUFFLLM_ERR_UNSUPPORTED ? st : HUFFLLM_ERR_CORRUPT;
+    if (d.blob_bytes != bytes) return fail(HUFFLLM_ERR_CORRUPT, "blob_bytes does not match the buffer size");
+    const uint8_t *base = (const uint8_t *)blob;
+
+    // codebook: used symbols must form a complete prefix code (a single 1-bit code is the one exception)
+    huffllm_codebook cb;
+    memset(cb.counts, 0, sizeof(cb.counts));
+    memset(cb.code, 0, sizeof(cb.code));
+    cb.dtype = d.dtype;
+    cb.budget = d.lut_bits;
+    for (int k = 0; k < 3; ++k) memcpy(cb.len[k], base + d.off_codebook + 32 * k, 32);
+    for (int k = 0; k < 2; ++k) {
+        uint64_t kraft = 0;
+        int used = 0, mx = 0;
+        for (int s = 0; s < 32; ++s) {
+            int l = cb.len[k][s];
+            if (!l) continue;
+            if (s >= 16 || l > 15) return fail(HUFFLLM_ERR_CORRUPT, "code length out of range");
+            kraft += 1ull << (16 - l);
+            ++used;
+            mx = std::max(mx, l);
+        }
+        if (used == 0) return fail(HUFFLLM_ERR_CORRUPT, "field %d has no codewords", k);
+        if (!(kraft == (1ull << 16) || (used == 1 && mx == 1))) return fail(HUFFLLM_ERR_CORRUPT, "field %d is not a complete prefix code", k);
+        if (mx > d.caps[k]) return fail(HUFFLLM_ERR_CORRUPT, "field %d exceeds its cap", k);
+    }
+    for (int s = 0; s < 32; ++s)
+        if (cb.len[2][s]) return fail(HUFFLLM_ERR_CORRUPT, "unexpected third field");
+    if (d.caps[0] + d.caps[1] > (int)d.lut_bits) return fail(HUFFLLM_ERR_CORRUPT, "caps exceed lut_bits");
+    canonical_codes(cb.len[0], 16, cb.code[0]);
+    canonical_codes(cb.len[1], 16, cb.code[1]);
+    finish_codebook(&cb);
+    if (memcmp(cb.lut.data(), base + d.off_lut, 4ull << d.lut_bits) != 0) return fail(HUFFLLM_ERR_CORRUPT, "LUT does not match the codebook");
+    if (cb.pad_word != d.pad_word) return fail(HUFFLLM_ERR_CORRUPT, "pad_word does not match the codebook");
+
+    Geometry g;
+    make_geometry(d.rows, d.cols, d.chunk_elems, &g);
+    const uint32_t *index = (const uint32_t *)(base + d.off_index);
+    if (index[0] != 0 || (uint64_t)index[d.n_chunks] * kRecordUnit != d.payload_bytes)
+        return fail(HUFFLLM_ERR_CORRUPT, "record index does not span the payload");
+    std::atomic<int> bad{0};
+    std::atomic<uint64_t> total_bits{0}, checksum{0};
+    std::atomic<uint32_t> max_words{0};
+    const uint32_t mask = (1u << d.lut_bits) - 1;
+    parallel_chunks(d.n_chunks, [&](uint64_t c) {
+        uint32_t kc = (uint32_t)(c % g.KC), rg = (uint32_t)(c / g.KC), nkb = blocks_of(g, kc), steps = nkb * 16;
+        if (index[c + 1] <= index[c]) { bad.store(1); return; }
+        uint64_t size = (uint64_t)(index[c + 1] - index[c]) * kRecordUnit;
+        if (size <= nkb * 512ull) { bad.store(2); return; }
+        uint32_t W = (uint32_t)((size - nkb * 512ull) / 128);
+        if (W > d.max_words) { bad.store(3); return; }
+        uint32_t seen = max_words.load();
+        while (W > seen && !max_words.compare_exchange_weak(seen, W)) {}
+        const uint8_t *raw = base + d.off_payload + (uint64_t)index[c] * kRecordUnit;
+        const uint32_t *coded = (const uint32_t *)(raw + nkb * 512ull);
+        uint64_t sum = 0;
+        for (uint32_t lane = 0; lane < 32; ++lane) {
+            auto word = [&](uint32_t j) -> uint64_t { return j < W ? coded[(size_t)j * 32 + lane] : 0; };
+            if (word(0) & ((1u << kLagBits) - 1)) { bad.store(4); return; }
+            uint32_t pos = kLagBits;
+            for (uint32_t s = 0; s < steps; ++s) {
+                uint64_t win = (word(pos >> 5) | (word((pos >> 5) + 1) << 32)) >> (pos & 31);
+                uint32_t e = cb.lut[(uint32_t)win & mask];
+                uint32_t l = e & 0x7FFFFF;
+                if (!l) { bad.store(5); return; }
+                uint32_t gg = lane >> 2, t = lane & 3, kb = s >> 4, half = (s >> 3) & 1, i = s & 7;
+                uint64_t r = (uint64_t)rg * 16 + gg + 8 * half, col = (uint64_t)kc * g.Kc + kb * 32ull + t * 8 + i;
+                if (r >= g.rows || col >= g.cols) {
+                    uint8_t rb = raw[(s >> 4) * 512 + lane * 16 + (s & 15)];
+                    if (rb != 0 || (e >> 23) != ((d.pad_word >> 7) & 0xFFu)) { bad.store(6); return; }
+                }
+                pos += l;
+                sum += l;
+            }
+            if (pos > W * 32) { bad.store(7); return; }
+            for (uint32_t p = pos; p < W * 32; ++p)
+                if ((word(p >> 5) >> (p & 31)) & 1) { bad.store(8); return; }
+        }
+        total_bits.fetch_add(sum);
+        checksum.fetch_add(record_checksum(raw, size, c));
+    });
+    if (bad.load()) return fail(HUFFLLM_ERR_CORRUPT, "payload check %d failed", bad.load());
+    if (total_bits.load() != d.coded_bits) return fail(HUFFLLM_ERR_CORRUPT, "coded_bits does not match the payload");
+    if (max_words.load() != d.max_words) return fail(HUFFLLM_ERR_CORRUPT, "max_words does not match the payload");
+    if (checksum.load() != d.payload_checksum) return fail(HUFFLLM_ERR_CORRUPT, "payload checksum mismatch");
+    if (d.raw_bits != 8 * d.rows * d.cols) return fail(HUFFLLM_ERR_CORRUPT, "raw_bits does not match the shape");
+    if (desc_out) *desc_out = d;
+    return HUFFLLM_OK;
+}
+
+}  // extern "C"

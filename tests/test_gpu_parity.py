@@ -1,0 +1,236 @@
+"""Parity of the CUDA path against the CPU oracle, through the C-ABI.  Needs a GPU."""
+import numpy as np
+import pytest
+
+import workloads as wl
+from oracle import oracle as orc
+
+pytestmark = pytest.mark.gpu
+
+TOL = 2e-3   # |y_gpu - y_oracle| <= TOL * sum_k |w x|, per output
+
+
+@pytest.fixture(scope="module")
+def hl():
+    import paper_2502_00922_b200 as m
+    m.lib()
+    return m
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch as t
+    assert t.cuda.is_available()
+    return t
+
+
+class Uploaded:
+    """A tensor encoded on the host and resident on the device, with its scratch buffers."""
+
+    def __init__(self, hl, torch, w, chunk_elems=4096, budget=0, batch=1):
+        self.w = w
+        cb = hl.build_codebook(w, hl.BF16, budget)
+        self.blob, self.desc = hl.encode(cb, w, chunk_elems)
+        cb.free()
+        hl.validate_blob(self.blob)
+        self.blob_dev = torch.from_numpy(self.blob).cuda()
+        assert self.blob_dev.data_ptr() % 256 == 0
+        self.ws_bytes = hl.workspace_bytes(self.desc, batch)
+        self.ws = torch.zeros(self.ws_bytes, dtype=torch.uint8, device="cuda")
+        self.err = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+
+def gpu_decode(hl, torch, up):
+    rows, cols = up.w.shape
+    out = torch.full((rows * cols + 64,), 0x5A5A, dtype=torch.int16, device="cuda")   # canary behind the output
+    hl.decode(up.desc, up.blob_dev, out, up.err)
+    torch.cuda.synchronize()
+    assert int(up.err.item()) == 0
+    res = out.cpu().numpy().view(np.uint16)
+    assert np.all(res[rows * cols:] == 0x5A5A)
+    return res[:rows * cols].reshape(rows, cols)
+
+
+def gpu_gemm(hl, torch, up, x):
+    rows, cols = up.w.shape
+    batch = x.shape[0]
+    x_dev = torch.from_numpy(x.view(np.int16)).cuda()
+    y = torch.full((batch * rows + 16,), float("nan"), dtype=torch.float32, device="cuda")
+    if batch == 1:
+        hl.decode_gemv(up.desc, up.blob_dev, x_dev, y, up.ws, up.ws_bytes, up.err)
+    else:
+        hl.decode_gemm(up.desc, up.blob_dev, x_dev, batch, y, up.ws, up.ws_bytes, up.err)
+    torch.cuda.synchronize()
+    assert int(up.err.item()) == 0
+    assert int(up.ws.count_nonzero().item()) == 0, "scratch must be left zero-filled"
+    res = y.cpu().numpy()
+    assert np.all(np.isnan(res[batch * rows:]))
+    return res[:batch * rows].reshape(batch, rows)
+
+
+def check_product(y_gpu, w, x):
+    y, d = orc.matmul(w, x)
+    err = np.abs(y_gpu.astype(np.float64) - y)
+    assert np.all(err <= TOL * d + 1e-30), f"max err/bound = {np.max(err / (TOL * d + 1e-30))}"
+    assert np.all(y_gpu[d == 0] == 0)
+    return float(np.max(err / np.maximum(d, 1e-300)))
+
+
+DECODE_CASES = [
+    # rows, cols, chunk_elems, budget, generator
+    (1024, 1024, 4096, 0, "gauss"),        # the small benchmark configuration
+    (16, 256, 4096, 0, "gauss"),           # exactly one chunk
+    (37, 300, 1024, 0, "student"),         # ragged rows and columns, scalar stores
+    (48, 1056, 4096, 0, "gauss"),          # ragged last column chunk
+    (5, 31, 512, 0, "patterns"),           # smaller than one tile
+    (272, 2080, 16384, 0, "gauss"),        # largest chunk size
+    (64, 8192, 1024, 0, "uniform"),        # worst-case exponents, smallest benchmark chunk size
+    (256, 2048, 4096, 0, "patterns"),      # every bit pattern incl. NaN / Inf / denormals
+    (96, 4096, 4096, 9, "student"),        # the other table size
+    (2368, 512, 512, 0, "gauss"),          # more chunks than warps, many per warp
+    (16, 512, 512, 0, "constant"),         # single-symbol codes
+]
+
+
+def make(gen, rows, cols, seed):
+    return {"gauss": lambda: wl.gaussian_weights(rows, cols, 0.02, seed),
+            "student": lambda: wl.student_t_weights(rows, cols, seed),
+            "uniform": lambda: wl.uniform_exponent_weights(rows, cols, seed),
+            "patterns": lambda: wl.all_patterns_weights(rows, cols, seed),
+            "constant": lambda: np.full((rows, cols), 0xBD33, dtype=np.uint16)}[gen]()
+
+
+@pytest.mark.parametrize("rows,cols,ce,budget,gen", DECODE_CASES)
+def test_decode_is_bit_exact(hl, torch, rows, cols, ce, budget, gen):
+    w = make(gen, rows, cols, 100 + rows)
+    up = Uploaded(hl, torch, w, ce, budget)
+    got = gpu_decode(hl, torch, up)
+    if rows * cols <= 300_000:
+        ref, _ = orc.decode_blob(up.blob)          # the oracle's bit-serial decode of the same blob
+        assert np.array_equal(ref, w)
+    assert np.array_equal(got, w)                  # lossless: the oracle's result is the original tensor
+
+
+GEMM_CASES = [
+    (1024, 1024, 4096, 0, "gauss", 1),
+    (16, 256, 4096, 0, "gauss", 1),
+    (48, 1056, 4096, 0, "gauss", 1),
+    (40, 2056, 1024, 0, "student", 3),            # ragged rows, cols a multiple of 8 only
+    (16, 65536, 4096, 0, "gauss", 1),             # one row group split over every CTA
+    (32, 32768, 4096, 0, "gauss", 8),
+    (2368, 512, 512, 0, "gauss", 2),
+    (272, 2080, 16384, 0, "gauss", 4),
+    (512, 4096, 4096, 9, "student", 5),
+    (256, 2048, 4096, 0, "uniform", 8),
+    (128, 1024, 1024, 0, "gauss", 16),            # two passes of 8
+    (64, 1024, 4096, 0, "gauss", 23),
+]
+
+
+@pytest.mark.parametrize("rows,cols,ce,budget,gen,batch", GEMM_CASES)
+def test_fused_product_matches_oracle(hl, torch, rows, cols, ce, budget, gen, batch):
+    w = make(gen, rows, cols, 200 + rows)
+    x = wl.activations(batch, cols, 300 + cols)
+    up = Uploaded(hl, torch, w, ce, budget, batch)
+    y1 = gpu_gemm(hl, torch, up, x)
+    check_product(y1, w, x)
+    y2 = gpu_gemm(hl, torch, up, x)
+    assert np.array_equal(y1, y2), "results must be bitwise reproducible"
+
+
+def test_product_closed_forms(hl, torch):
+    rows, cols = 64, 1024
+    ones = np.full((rows, cols), 0x3F80, dtype=np.uint16)
+    up = Uploaded(hl, torch, ones)
+    y = gpu_gemm(hl, torch, up, np.full((1, cols), 0x3F80, dtype=np.uint16))
+    assert np.all(y == cols)
+    w = wl.gaussian_weights(rows, cols, 0.02, 7)
+    up = Uploaded(hl, torch, w)
+    for k in (0, 519, cols - 1):                   # one-hot x returns column k exactly
+        x = np.zeros((1, cols), dtype=np.uint16)
+        x[0, k] = 0x3F80
+        assert np.array_equal(gpu_gemm(hl, torch, up, x)[0], wl.bf16_bits_to_f32(w[:, k]))
+
+
+def test_plain_gemv_matches_oracle(hl, torch):
+    rows, cols = 520, 4096
+    w = wl.gaussian_weights(rows, cols, 0.02, 9)
+    x = wl.activations(1, cols, 10)
+    y = torch.zeros(rows, dtype=torch.float32, device="cuda")
+    hl.plain_gemv(torch.from_numpy(w.view(np.int16)).cuda(), rows, cols, torch.from_numpy(x.view(np.int16)).cuda(), y)
+    torch.cuda.synchronize()
+    check_product(y.cpu().numpy()[None, :], w, x)
+
+
+def test_host_buffer_call(hl, torch):
+    rows, cols, batch = 256, 2048, 4
+    w = wl.gaussian_weights(rows, cols, 0.02, 11)
+    x = wl.activations(batch, cols, 12)
+    up = Uploaded(hl, torch, w, batch=batch)
+    x_host = torch.from_numpy(x.view(np.int16)).pin_memory()
+    y_host = torch.zeros(batch * rows, dtype=torch.float32).pin_memory()
+    x_stage = torch.zeros(batch * cols, dtype=torch.int16, device="cuda")
+    y_stage = torch.zeros(batch * rows, dtype=torch.float32, device="cuda")
+    hl.decode_gemm_host(up.desc, up.blob_dev, x_host, batch, y_host, x_stage, y_stage, up.ws, up.ws_bytes, up.err)
+    check_product(y_host.numpy().reshape(batch, rows), w, x)
+
+
+def test_bad_record_offsets_are_reported_not_followed(hl, torch):
+    """A record index pointing outside the payload (made on the host) sets the error flag; the kernel
+    skips that chunk, touches nothing out of range, and every other chunk still decodes."""
+    rows, cols = 64, 1024
+    w = wl.gaussian_weights(rows, cols, 0.02, 13)
+    up = Uploaded(hl, torch, w)
+    blob = up.blob.copy()
+    idx = blob[up.desc.off_index:up.desc.off_index + 4 * (up.desc.n_chunks + 1)].view(np.uint32)
+    idx[5] = 0x7FFFFFF0                            # chunk 4 ends / chunk 5 starts far outside
+    with pytest.raises(hl.HuffllmError):
+        hl.validate_blob(blob)                     # the host check refuses it
+    dev = torch.from_numpy(blob).cuda()
+    out = torch.zeros(rows * cols, dtype=torch.int16, device="cuda")
+    hl.decode(up.desc, dev, out, up.err)
+    torch.cuda.synchronize()
+    assert int(up.err.item()) != 0
+    got = out.cpu().numpy().view(np.uint16).reshape(rows, cols)
+    good = np.ones((rows, cols), dtype=bool)
+    kc_cols = up.desc.chunk_cols
+    for c in (4, 5):
+        rg, kc = divmod(c, up.desc.col_chunks)
+        good[rg * 16:(rg + 1) * 16, kc * kc_cols:(kc + 1) * kc_cols] = False
+    assert np.array_equal(got[good], w[good])
+
+
+def test_unsupported_requests_fail_before_launch(hl, torch):
+    w = wl.gaussian_weights(16, 516, 0.02, 14)     # cols not a multiple of 8
+    up = Uploaded(hl, torch, w, 512)
+    x = torch.zeros(516, dtype=torch.int16, device="cuda")
+    y = torch.zeros(16, dtype=torch.float32, device="cuda")
+    with pytest.raises(hl.HuffllmError) as e:
+        hl.decode_gemv(up.desc, up.blob_dev, x, y, up.ws, up.ws_bytes, up.err)
+    assert e.value.status_name == "UNSUPPORTED"
+    w = wl.gaussian_weights(16, 512, 0.02, 15)
+    up = Uploaded(hl, torch, w, 512, budget=12)    # larger codes than the device table handles
+    with pytest.raises(hl.HuffllmError) as e:
+        hl.decode(up.desc, up.blob_dev, torch.zeros(16 * 512, dtype=torch.int16, device="cuda"), up.err)
+    assert e.value.status_name == "UNSUPPORTED"
+    with pytest.raises(hl.HuffllmError) as e:      # misaligned blob pointer
+        hl.decode(up.desc, up.blob_dev.data_ptr() + 8, torch.zeros(16 * 512, dtype=torch.int16, device="cuda"), up.err)
+    assert e.value.status_name == "INVALID_ARG"
+
+
+def test_full_size_layer_matrix_sampled(hl, torch):
+    """gate/up projection of the Llama-7B-shaped layer at full size, in the launch configuration the
+    benchmark times: decode compared everywhere with the original tensor, the product on sampled rows."""
+    rows, cols = 11008, 4096
+    w = wl.gaussian_weights(rows, cols, 0.02, 2004)
+    x = wl.activations(1, cols, 2504)
+    up = Uploaded(hl, torch, w)
+    got = gpu_decode(hl, torch, up)
+    assert np.array_equal(got, w)
+    y = gpu_gemm(hl, torch, up, x)
+    rs = np.random.default_rng(0).choice(rows, 64, replace=False)
+    yo, d = orc.matmul(w[rs], x)
+    assert np.all(np.abs(y[0, rs] - yo[0]) <= TOL * d[0])
+    # a property that holds at any size: y(-x) = -y exactly (sign flips commute with every rounding)
+    yn = gpu_gemm(hl, torch, up, x ^ np.uint16(0x8000))
+    assert np.array_equal(yn, -y)

@@ -1,0 +1,152 @@
+"""Host side of the library (codebook, encoder, validator) against the CPU oracle.  No GPU needed."""
+import ctypes
+import os
+
+import numpy as np
+import pytest
+
+import paper_2502_00922_b200 as hl
+import workloads as wl
+from oracle import oracle as orc
+
+
+def kraft_ok(lens):
+    used = [int(l) for l in lens if l]
+    return sum(1 << (16 - l) for l in used) == 1 << 16 or used == [1]
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(os.path.dirname(hl.__file__), "..", "include", "huffllm.h")).read()
+    import re
+    declared = set(re.findall(r"\b(huffllm_[a-z_]+)\s*\(", header))
+    assert declared == set(hl.exported_symbols())
+    so = ctypes.CDLL(os.path.join(os.path.dirname(hl.__file__), "libhuffllm.so"))
+    for name in declared:
+        assert getattr(so, name) is not None
+
+
+DATASETS = {
+    "gauss": lambda: wl.gaussian_weights(64, 2048, 0.02, 21),
+    "gauss015": lambda: wl.gaussian_weights(64, 2048, 0.015, 22),
+    "student": lambda: wl.student_t_weights(128, 1024, 23),
+    "uniform": lambda: wl.uniform_exponent_weights(64, 1024, 24),
+    "patterns": lambda: wl.all_patterns_weights(64, 2048, 25),
+    "constant": lambda: np.full((16, 512), 0x3C12, dtype=np.uint16),
+}
+
+
+@pytest.mark.parametrize("name", sorted(DATASETS))
+@pytest.mark.parametrize("budget", [0, 8, 9, 10, 12])
+def test_codebook_cost_matches_oracle(name, budget):
+    w = DATASETS[name]()
+    cb = hl.build_codebook(w, hl.BF16, budget)
+    counts = orc.histogram(w)
+    olens, ocaps = orc.build_lengths(counts, orc.BF16, budget or 8)
+    total = 0
+    for f in range(2):
+        n, c, lens, codes = cb.get(f)
+        assert n == 16 and np.array_equal(c[:16], counts[f][:16])
+        assert kraft_ok(lens) and max(lens) <= (budget or 8)
+        assert np.array_equal(codes, orc.canonical_codes(lens))           # same canonical rule on both sides
+        total += orc.code_cost(c, lens)
+    assert total == orc.code_cost(counts[0], olens[0]) + orc.code_cost(counts[1], olens[1])
+    cb.free()
+
+
+@pytest.mark.parametrize("rows,cols,ce,budget,gen", [
+    (48, 1056, 4096, 8, "gauss"), (37, 300, 1024, 8, "student"), (16, 256, 4096, 9, "gauss"),
+    (5, 31, 512, 8, "patterns"), (33, 2080, 16384, 8, "gauss"), (64, 1024, 4096, 12, "uniform"),
+    (20, 520, 1024, 10, "patterns"), (1, 8, 512, 8, "gauss")])
+def test_blob_decodes_with_oracle_and_bits_match(rows, cols, ce, budget, gen):
+    w = {"gauss": lambda: wl.gaussian_weights(rows, cols, 0.02, 31),
+         "student": lambda: wl.student_t_weights(rows, cols, 32),
+         "uniform": lambda: wl.uniform_exponent_weights(rows, cols, 33),
+         "patterns": lambda: wl.all_patterns_weights(rows, cols, 34)}[gen]()
+    cb = hl.build_codebook(w, hl.BF16, budget)
+    blob, d = hl.encode(cb, w, ce)
+    assert d.blob_bytes == blob.size <= hl.encode_bound(rows, cols, hl.BF16, ce)
+    hl.validate_blob(blob)
+    back, used = orc.decode_blob(blob)                  # slow reader + bit-serial decoder; checks lag/tail/pad bits
+    assert np.array_equal(back, w)
+    # the oracle's own encoding with the blob's code lengths gives the same bits, lane by lane
+    parsed = orc.parse_blob(blob)
+    lens, codes = parsed["lens"], parsed["codes"]
+    flat = np.append(w.ravel(), np.uint16(d.pad_word))
+    assert d.pad_word == orc.pad_word(lens)
+    for chunk_ids, idx in orc.element_map(rows, cols, ce):
+        n, _, steps = idx.shape
+        bits, off, raw = orc.encode_sequences(flat[idx.reshape(n * 32, steps)], lens, codes)
+        for a, cid in enumerate(chunk_ids):
+            pbits, poff, praw = parsed["chunks"][int(cid)]
+            per = pbits.reshape(32, -1)
+            for l in range(32):
+                lo, hi = int(off[a * 32 + l]), int(off[a * 32 + l + 1])
+                assert int(used[int(cid)][l]) == hi - lo
+                assert np.array_equal(per[l, :hi - lo], bits[lo:hi])
+            assert np.array_equal(praw, raw[a * 32:a * 32 + 32])
+    # the LUT is what a bit-serial decode of every index gives
+    assert np.array_equal(parsed["lut"], orc.lut_from_code(lens, codes, d.lut_bits))
+    # accounting
+    assert d.coded_bits == sum(int(u.sum()) for u in used.values()) and d.raw_bits == 8 * rows * cols
+    cb.free()
+
+
+def test_validator_rejects_damaged_blobs():
+    w = wl.gaussian_weights(48, 1056, 0.02, 41)
+    cb = hl.build_codebook(w)
+    blob, d = hl.encode(cb, w, 4096)
+    hl.validate_blob(blob)
+
+    def damaged(offset, xor=0xFF):
+        b = blob.copy()
+        b[offset] ^= xor
+        with pytest.raises(hl.HuffllmError) as e:
+            hl.validate_blob(b)
+        assert e.value.status_name in ("CORRUPT", "UNSUPPORTED")
+
+    damaged(0)                                   # magic
+    damaged(16, 1)                               # rows
+    damaged(56, 1)                               # lut_bits
+    damaged(76, 1)                               # max_words
+    damaged(d.off_codebook + 6, 1)               # a code length
+    damaged(d.off_lut + 40, 1)                   # a LUT entry
+    damaged(d.off_index + 4, 1)                  # record index
+    damaged(d.off_payload + 8 * 512 + 0, 1)      # lag bit of chunk 0 lane 0
+    damaged(d.off_payload + 8 * 512 + 200)       # coded bits
+    damaged(d.off_payload + d.payload_bytes - 1, 0x80)  # tail padding of the last record
+    with pytest.raises(hl.HuffllmError):
+        hl.validate_blob(blob[:-128])            # truncated
+
+
+def test_argument_errors():
+    w = wl.gaussian_weights(16, 64, 0.02, 51)
+    with pytest.raises(hl.HuffllmError) as e:
+        hl.build_codebook(w, hl.FP16)
+    assert e.value.status_name == "UNSUPPORTED"
+    with pytest.raises(hl.HuffllmError) as e:
+        hl.build_codebook(w, hl.BF16, 5)
+    assert e.value.status_name == "UNSUPPORTED"
+    cb = hl.build_codebook(w)
+    with pytest.raises(hl.HuffllmError) as e:
+        hl.encode(cb, w, 1000)
+    assert e.value.status_name == "INVALID_ARG"
+    other = wl.uniform_exponent_weights(16, 64, 52, 1, 250)     # uses exponents the codebook never saw
+    with pytest.raises(hl.HuffllmError) as e:
+        hl.encode(cb, other, 512)
+    assert e.value.status_name == "INVALID_ARG" and "codeword" in str(e.value)
+    blob, d = hl.encode(cb, w, 512)
+    assert hl.workspace_bytes(d, 1) > 0
+    with pytest.raises(hl.HuffllmError):
+        hl.workspace_bytes(d, 65)
+
+
+def test_compression_accounting_on_paper_shaped_weights():
+    # Section 5.1: BF16 lands at 11.59-11.68 bits/param on real checkpoints; the synthetic stand-in gives ~11.7-11.8
+    w = wl.gaussian_weights(256, 4096, 0.02, 61)
+    cb = hl.build_codebook(w)
+    blob, d = hl.encode(cb, w, 4096)
+    n = w.size
+    payload_bits = (d.coded_bits + d.raw_bits) / n
+    assert 11.6 <= payload_bits <= 11.9
+    total_ratio = 2.0 * n / d.blob_bytes
+    assert 1.25 <= total_ratio <= 1.37          # lane padding and side tables cost a few percent
