@@ -145,8 +145,9 @@ huffllm_status huffllm_validate_blob(const void *blob_host, size_t bytes, huffll
 
 /*
  * Scratch bytes the fused products need for `batch` activation vectors.  The workspace must be
- * zero-filled once after allocation; every call leaves it zero-filled again.  Calls that share a
- * workspace must not overlap on the GPU.
+ * zero-filled once after allocation; its first 256 bytes are control words that every call
+ * leaves zero again, the rest is overwritten freely.  Calls that share a workspace must not
+ * overlap on the GPU.
  */
 huffllm_status huffllm_workspace_bytes(const huffllm_desc *desc, uint32_t batch, size_t *bytes);
 
