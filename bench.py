@@ -1,0 +1,353 @@
+#!/usr/bin/env python
+"""Benchmark of the decode-fused GEMV path.
+
+One "step" is one pass of the whole hot path over one batch of synthetic input: every matrix of the
+workload's decoder layer, held Huffman-compressed in HBM, is multiplied with one bf16 activation
+vector by the fused kernel (stream the compressed bytes, decode in registers, multiply, reduce).
+
+    python bench.py --gpus 1 --steps 20 --warmup 5            # this library
+    python bench.py --impl reference --steps 3 --warmup 1     # the CPU oracle on a bounded sample
+    python -m torch.distributed.run --nproc-per-node N ... bench.py --gpus N   # N independent replicas
+
+Prints ONE JSON line (rank 0).  metric = uncompressed-equivalent weight GB/s (2 bytes per weight over
+the step time); roofline = compressed bytes the kernels must read over their measured duration, against
+the measured HBM copy bandwidth of this GPU pool.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+import workloads as wl  # noqa: E402
+
+METRIC = "decode-fused GEMV uncompressed-equiv weight GB/s; % HBM roofline on comp. bytes"
+UNIT = "GB/s"
+WORKLOADS = {
+    # name: (layer table, std, seed, description)
+    "small_1024": ([("w", 1024, 1024)], 0.02, 1000, "single 1024x1024 bf16 matrix (oracle-sized case)"),
+    "llama7b_layer": (wl.LAYER_LLAMA7B, 0.02, 2000, "Llama-7B-shaped decoder layer, 7 matrices, batch 1"),
+    "8b_layer": (wl.LAYER_8B, 0.02, 3000, "8B-shaped decoder layer (GQA k/v 1024x4096, FFN 14336), batch 1"),
+    "ffn70b": (wl.FFN_70B, 0.015, 4000, "70B-FFN-shaped pair 28672x8192 / 8192x28672"),
+}
+FALLBACK_HBM_GBS = 6650.0
+# dram__bytes_read.sum + dram__bytes_write.sum of one fused-product launch over its algorithmic bytes, from the
+# ncu capture summarised in profiles/ (None until a capture exists); traffic = ratio * algorithmic bytes.
+NCU_TRAFFIC_RATIO = None
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback (earlier measurement on this pool)"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+         "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.uuid, self.proc, self.lines = uuid, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.uuid, "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def prepare(workload: str, chunk_elems: int, hl, torch, dev):
+    """Generate, encode (host) and upload every matrix of the workload."""
+    table, std, seed, _ = WORKLOADS[workload]
+    mats = []
+    for i, (name, rows, cols) in enumerate(table):
+        w = wl.gaussian_weights(rows, cols, std, seed + i)
+        cb = hl.build_codebook(w)
+        blob, desc = hl.encode(cb, w, chunk_elems)
+        cb.free()
+        x = wl.activations(1, cols, seed + 500 + i)
+        ws_bytes = hl.workspace_bytes(desc, 1)
+        alg_bytes = (desc.payload_bytes + 4 * (desc.n_chunks + 1) + (4 << desc.lut_bits) + 2 * cols + 4 * rows)
+        mats.append(dict(name=name, rows=rows, cols=cols, desc=desc, blob_dev=torch.from_numpy(blob).to(dev),
+                         x_host=torch.from_numpy(x.view(np.int16).reshape(-1)).pin_memory(),
+                         y_host=torch.zeros(rows, dtype=torch.float32).pin_memory(),
+                         x_dev=torch.from_numpy(x.view(np.int16).reshape(-1)).to(dev),
+                         y_dev=torch.zeros(rows, dtype=torch.float32, device=dev),
+                         ws=torch.zeros(ws_bytes, dtype=torch.uint8, device=dev), ws_bytes=ws_bytes,
+                         alg_bytes=int(alg_bytes), coded_bits=int(desc.coded_bits), raw_bits=int(desc.raw_bits),
+                         blob_bytes=int(desc.blob_bytes), w_sample=w[:512].copy() if i == 0 else None,
+                         x_np=x if i == 0 else None))
+        del w
+    return mats
+
+
+def oracle_sample_time(hl, w_sample, x_np, chunk_elems: int, repeats: int = 1):
+    """Time the CPU oracle (bit-serial decode of the library's blob + fp64 product) on a sample tensor."""
+    from oracle import oracle as orc
+    cb = hl.build_codebook(w_sample)
+    blob, _ = hl.encode(cb, w_sample, chunk_elems)
+    cb.free()
+    orc.lib()
+    best = None
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        back, _ = orc.decode_blob(blob)
+        y, _ = orc.matmul(back, x_np)
+        dt = time.perf_counter() - t0
+        best = dt if best is None else min(best, dt)
+    assert np.array_equal(back, w_sample)
+    return best
+
+
+def run_reference(args):
+    """The oracle arm: the CPU oracle, as it stands, on a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import paper_2502_00922_b200 as hl   # host encoder only: it produces the blob the oracle decodes
+    table, std, seed, desc_text = WORKLOADS[args.workload]
+    name, rows, cols = table[0]
+    sample_rows = min(rows, 128)
+    w = wl.gaussian_weights(rows, cols, std, seed)[:sample_rows].copy()
+    x = wl.activations(1, cols, seed + 500)
+    times = []
+    for i in range(args.warmup + args.steps):
+        dt = oracle_sample_time(hl, w, x, args.chunk_elems)
+        if i >= args.warmup:
+            times.append(dt)
+    t = sum(times) / len(times)
+    value = 2.0 * w.size / t / 1e9
+    sample = f"rows 0..{sample_rows - 1} of matrix '{name}' ({w.size} weights) per step; decode of the blob + fp64 product"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": t * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16", "data": "synthetic", "config": {"workload": args.workload, "what": desc_text, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=20)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama7b_layer", choices=sorted(WORKLOADS))
+    ap.add_argument("--chunk-elems", type=int, default=4096)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+
+    import torch
+    import paper_2502_00922_b200 as hl
+    hl.lib()   # fails loudly when the CUDA library has not been built
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device; there is no CPU path")
+    rank, world = int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    args.warmup = max(args.warmup, 3)
+
+    mats = prepare(args.workload, args.chunk_elems, hl, torch, dev)
+    err = torch.zeros(1, dtype=torch.int32, device=dev)
+    n_weights = sum(m["rows"] * m["cols"] for m in mats)
+    unc_bytes = 2 * n_weights
+    alg_bytes = sum(m["alg_bytes"] for m in mats)
+    stream = torch.cuda.current_stream()
+
+    def step_device():
+        for m in mats:
+            hl.decode_gemv(m["desc"], m["blob_dev"], m["x_dev"], m["y_dev"], m["ws"], m["ws_bytes"], err, stream)
+
+    def step_host():
+        for m in mats:
+            hl.decode_gemm_host(m["desc"], m["blob_dev"], m["x_host"], 1, m["y_host"], m["x_dev"], m["y_dev"], m["ws"],
+                                m["ws_bytes"], err, stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(v: float) -> float:
+        if dist is None:
+            return v
+        t = torch.tensor([v], dtype=torch.float64, device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- device-resident timing: K steps between one pair of events on the launching stream
+    for _ in range(args.warmup):
+        step_device()
+    uuid = str(getattr(torch.cuda.get_device_properties(dev), "uuid", local))
+    sampler = ClockSampler(uuid if uuid.startswith("GPU-") or uuid.isdigit() else "GPU-" + uuid)
+    barrier()
+    sampler.start()
+    time.sleep(0.3)                       # let the sampler come up before the timed region starts
+    t_beg, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_beg.record(stream)
+    for s in range(args.steps):
+        step_device()
+    t_end.record(stream)
+    barrier()
+    clocks = sampler.stop()
+    ms_step = max_over_ranks(t_beg.elapsed_time(t_end) / args.steps)
+    assert int(err.item()) == 0, "device error flag set"
+
+    # ---- per-matrix durations (a second, shorter pass with an event after every launch)
+    n_b = min(args.steps, 50)
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(mats) + 1)] for _ in range(n_b)]
+    for s in range(n_b):
+        ev[s][0].record(stream)
+        for i, m in enumerate(mats):
+            hl.decode_gemv(m["desc"], m["blob_dev"], m["x_dev"], m["y_dev"], m["ws"], m["ws_bytes"], err, stream)
+            ev[s][i + 1].record(stream)
+    barrier()
+    per_mat_ms = [statistics.median(ev[s][i].elapsed_time(ev[s][i + 1]) for s in range(n_b)) for i in range(len(mats))]
+    kernel_ms_step = ms_step              # launches run back to back: average launch duration = step time / launches
+
+    # ---- end to end through the host-buffer call: x from pinned host memory, y back to the host, every launch
+    for _ in range(args.warmup):
+        step_host()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step_host()
+    barrier()
+    e2e_ms = max_over_ranks((time.perf_counter() - t0) * 1e3 / args.steps)
+
+    # ---- the dense product the compression competes with: same layer, uncompressed bf16, own kernel and cuBLAS
+    plain_ms = cublas_ms = None
+    if rank == 0:
+        try:
+            dense = [(torch.randint(-2**15, 2**15, (m["rows"], m["cols"]), dtype=torch.int16, device=dev), m) for m in mats]
+            for w_dev, m in dense:
+                w_dev.view(torch.bfloat16).normal_(0, 0.02)
+            def plain():
+                for w_dev, m in dense:
+                    hl.plain_gemv(w_dev, m["rows"], m["cols"], m["x_dev"], m["y_dev"], stream)
+            def cublas():
+                for w_dev, m in dense:
+                    torch.mv(w_dev.view(torch.bfloat16), m["x_dev"].view(torch.bfloat16))
+            for fn, key in ((plain, "plain"), (cublas, "cublas")):
+                for _ in range(args.warmup):
+                    fn()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                torch.cuda.synchronize()
+                a.record(stream)
+                for _ in range(args.steps):
+                    fn()
+                b.record(stream)
+                torch.cuda.synchronize()
+                if key == "plain":
+                    plain_ms = a.elapsed_time(b) / args.steps
+                else:
+                    cublas_ms = a.elapsed_time(b) / args.steps
+            del dense
+        except Exception as ex:   # the comparison point must never take the benchmark down
+            print(f"[bench] dense comparison skipped: {ex}", file=sys.stderr)
+
+    # ---- the CPU oracle on a bounded sample of the same workload (rank 0, single GPU run only)
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        m0 = mats[0]
+        dt = oracle_sample_time(hl, m0["w_sample"], m0["x_np"], args.chunk_elems, repeats=1)
+        cpu = {"value": 2.0 * m0["w_sample"].size / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"rows 0..{m0['w_sample'].shape[0] - 1} of matrix '{m0['name']}' ({m0['w_sample'].size} weights, "
+                         f"{dt:.1f} s): bit-serial decode of the blob + fp64 product, one thread"}
+
+    if rank != 0:
+        return
+    peak, peak_src = measured_peak()
+    value = world * unc_bytes / (ms_step * 1e-3) / 1e9
+    achieved = alg_bytes / (kernel_ms_step * 1e-3) / 1e9
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "data": "synthetic",
+        "config": {"workload": args.workload, "what": WORKLOADS[args.workload][3], "chunk_elems": args.chunk_elems,
+                   "max_code_len": int(mats[0]["desc"].lut_bits), "weights_per_step": n_weights,
+                   "uncompressed_bytes": unc_bytes, "compressed_bytes": sum(m["blob_bytes"] for m in mats),
+                   "compression_ratio_total": unc_bytes / sum(m["blob_bytes"] for m in mats),
+                   "compression_ratio_payload": 16.0 * n_weights / sum(m["coded_bits"] + m["raw_bits"] for m in mats),
+                   "bits_per_param_payload": sum(m["coded_bits"] + m["raw_bits"] for m in mats) / n_weights,
+                   "l2": "inputs larger than L2: the step streams %.0f MB of compressed weights, L2 is 126 MB" % (alg_bytes / 1e6),
+                   "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "tokens_per_s_equiv_one_layer": 1e3 / ms_step},
+        "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
+                     "traffic": None if NCU_TRAFFIC_RATIO is None else NCU_TRAFFIC_RATIO * alg_bytes / len(mats),
+                     "peak_source": peak_src, "kernel": "huff_kernel<product>", "launches_per_step": len(mats),
+                     "algorithmic_bytes_per_step": alg_bytes, "kernel_ms_per_step": kernel_ms_step,
+                     "frac_of_nominal_8TBs": achieved / 8000.0,
+                     "per_matrix": [{"name": m["name"], "rows": m["rows"], "cols": m["cols"], "ms": t,
+                                     "comp_GBs": m["alg_bytes"] / (t * 1e-3) / 1e9} for m, t in zip(mats, per_mat_ms)]},
+        "cpu_baseline": cpu,
+        "e2e": {"value": world * unc_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
+                "h2d_bytes_per_step": sum(2 * m["cols"] for m in mats), "d2h_bytes_per_step": sum(4 * m["rows"] for m in mats)},
+        "gpu_launches": len(mats) * args.steps,
+        "clocks": clocks,
+        "dense_bf16_gemv": {"own_kernel_ms_per_step": plain_ms, "cublas_mv_ms_per_step": cublas_ms,
+                            "own_kernel_GBs": None if not plain_ms else unc_bytes / (plain_ms * 1e-3) / 1e9,
+                            "speedup_vs_own_dense": None if not plain_ms else plain_ms / ms_step},
+    }
+    print(json.dumps(out))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

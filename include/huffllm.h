@@ -56,19 +56,22 @@ typedef struct huffllm_codebook huffllm_codebook;
  *             (length, symbol), first codeword 0, next = (previous + 1) << (length growth); a
  *             codeword's most significant bit comes first in the stream
  *   LUT       uint32[1 << lut_bits], indexed by the next lut_bits stream bits (first bit = bit 0);
- *             BF16 entry = exponent << 23 | (length of hi-nibble code + length of lo-nibble code)
+ *             BF16 entry = (length of hi-nibble code + length of lo-nibble code) << 16 | exponent << 7,
+ *             i.e. the exponent already sits where a bf16 word has it
  *   index     uint32[n_chunks + 1]: record offsets from off_payload, in units of 128 bytes
  *   payload   one record per chunk, chunk id = row_group * col_chunks + col_chunk
  *
  * A chunk is a tile of 16 rows x chunk_cols (= chunk_elems / 16) columns, cut into blocks of 32
  * columns (the last column chunk may hold fewer blocks).  It is decoded by 32 lanes; lane
  * l = 4 g + t (g < 8, t < 4) owns rows g and g + 8 of the tile and columns 8t .. 8t+7 of every
- * block.  Its sequence is, block after block, row g's eight weights then row g+8's eight weights.
- * Positions outside the tensor hold `pad_word`.  Record = raw bytes [block][lane][16]
- * (BF16 raw byte = sign << 7 | mantissa), then W rows of 32 little-endian uint32 (row j, lane l):
- * lane l's bit sequence, bit i in word i / 32 at bit i % 32.  The sequence starts with `lag_bits`
- * zero bits, then for every weight code(exponent >> 4) code(exponent & 15); bits after the last
- * codeword are zero.  W is the largest lane length of the chunk in words (lanes are padded to it).
+ * block, as two independent bit sequences: sequence l holds row g's weights, sequence 32 + l
+ * holds row g + 8's, block after block (eight weights per block each).  Positions outside the
+ * tensor hold `pad_word`.  Record = raw bytes [block][lane][16] (BF16 raw byte = sign << 7 |
+ * mantissa; a lane's 16 bytes are row g's eight weights, then row g + 8's), then W rows of 64
+ * little-endian uint32 (row j, sequence s): the sequence's bits, bit i in word i / 32 at bit
+ * i % 32.  A sequence starts with `lag_bits` zero bits, then for every weight
+ * code(exponent >> 4) code(exponent & 15); bits after the last codeword are zero.  W is the
+ * longest sequence of the chunk in words (all 64 are padded to it).
  */
 typedef struct huffllm_desc {
     char     magic[4];        /* "HFLM"                                                    */
@@ -145,7 +148,7 @@ huffllm_status huffllm_validate_blob(const void *blob_host, size_t bytes, huffll
 
 /*
  * Scratch bytes the fused products need for `batch` activation vectors.  The workspace must be
- * zero-filled once after allocation; its first 256 bytes are control words that every call
+ * zero-filled once after allocation; its first 4096 bytes are control words that every call
  * leaves zero again, the rest is overwritten freely.  Calls that share a workspace must not
  * overlap on the GPU.
  */

@@ -183,12 +183,13 @@ def matmul(w: np.ndarray, x: np.ndarray, dtype=BF16):
 # ------------------------------------------------------- blob element map
 # A chunk is a tile of 16 rows by Kc = chunk_elems/16 columns, cut into blocks of 32 columns.
 # Lane l = 4*g + t (g = 0..7, t = 0..3) owns rows g and g+8 of the tile and, in every 32-column
-# block, the 8 columns 8t..8t+7.  Its sequence is, block after block: row g's 8 weights, then
-# row g+8's 8 weights (16 steps per block).
+# block, the 8 columns 8t..8t+7.  Each lane carries TWO independent bit sequences: sequence l holds
+# row g's weights, sequence 32 + l holds row g+8's, block after block (8 steps per block each).
 
 TILE_ROWS = 16
 BLOCK_COLS = 32
 LAG_BITS = 7
+SEQS = 64          # bit sequences per chunk
 
 
 def geometry(rows: int, cols: int, chunk_elems: int):
@@ -203,27 +204,28 @@ def blocks_in_chunk(cols: int, Kc: int, kc: int) -> int:
 
 
 def element_map(rows: int, cols: int, chunk_elems: int):
-    """Yield groups (chunk_ids[n], idx[n][32][steps]): flat tensor index of every (chunk, lane, step),
+    """Yield groups (chunk_ids[n], idx[n][64][steps]): flat tensor index of every (chunk, sequence, step),
     -1 where the position lies outside the tensor (a pad weight).  Chunks are numbered rg*KC + kc; the
     chunks of the last column-chunk form their own group when they hold fewer blocks."""
     geo = geometry(rows, cols, chunk_elems)
     Kc, RG, KC = geo["Kc"], geo["RG"], geo["KC"]
-    lane = np.arange(32)
+    seq = np.arange(SEQS)
+    half, lane = seq // 32, seq % 32
     g, t = lane // 4, lane % 4
     groups = {}
     for kc in range(KC):
         groups.setdefault(blocks_in_chunk(cols, Kc, kc), []).append(kc)
     for nkb, kcs in groups.items():
-        steps = np.arange(nkb * 16)
-        kb, half, i = steps // 16, (steps % 16) // 8, steps % 8
+        steps = np.arange(nkb * 8)
+        kb, i = steps // 8, steps % 8
         rg = np.arange(RG)
         kcs = np.asarray(kcs)
-        row = rg[:, None, None, None] * 16 + g[None, None, :, None] + 8 * half[None, None, None, :]
+        row = rg[:, None, None, None] * 16 + (g + 8 * half)[None, None, :, None] + 0 * steps[None, None, None, :]
         col = kcs[None, :, None, None] * Kc + kb[None, None, None, :] * 32 + t[None, None, :, None] * 8 + i[None, None, None, :]
         row, col = np.broadcast_arrays(row, col)
         idx = np.where((row < rows) & (col < cols), row.astype(np.int64) * cols + col, -1)
         chunk_ids = (rg[:, None] * KC + kcs[None, :]).ravel()
-        yield chunk_ids, idx.reshape(len(chunk_ids), 32, nkb * 16)
+        yield chunk_ids, idx.reshape(len(chunk_ids), SEQS, nkb * 8)
 
 
 def pad_word(lens: np.ndarray, dtype=BF16) -> int:
@@ -238,8 +240,8 @@ def pad_word(lens: np.ndarray, dtype=BF16) -> int:
 
 
 def encode_tensor(w: np.ndarray, chunk_elems: int = 4096, budget: int = 8, dtype=BF16):
-    """Oracle-side encoding of a whole tensor in the blob's lane order.  Returns a dict with the code
-    (lens, codes, caps), and per chunk id: (bits, bit_off, raw) of its 32 lane sequences."""
+    """Oracle-side encoding of a whole tensor in the blob's sequence order.  Returns a dict with the code
+    (lens, codes, caps), and per chunk id: (bits, bit_off, raw) of its 64 sequences."""
     w = np.ascontiguousarray(w, dtype=np.uint16)
     rows, cols = w.shape
     counts = histogram(w, dtype)
@@ -250,11 +252,11 @@ def encode_tensor(w: np.ndarray, chunk_elems: int = 4096, budget: int = 8, dtype
     chunks = {}
     for chunk_ids, idx in element_map(rows, cols, chunk_elems):
         n, _, steps = idx.shape
-        seq = flat[idx.reshape(n * 32, steps)]
+        seq = flat[idx.reshape(n * SEQS, steps)]
         bits, off, raw = encode_sequences(seq, lens, codes, dtype)
         for a, cid in enumerate(chunk_ids):
-            lo, hi = off[a * 32], off[a * 32 + 32]
-            chunks[int(cid)] = (bits[lo:hi], (off[a * 32:a * 32 + 33] - lo).copy(), raw[a * 32:a * 32 + 32])
+            lo, hi = off[a * SEQS], off[a * SEQS + SEQS]
+            chunks[int(cid)] = (bits[lo:hi], (off[a * SEQS:a * SEQS + SEQS + 1] - lo).copy(), raw[a * SEQS:a * SEQS + SEQS])
     return dict(rows=rows, cols=cols, chunk_elems=chunk_elems, dtype=dtype, counts=counts, lens=lens,
                 codes=codes, caps=caps, pad=pad, chunks=chunks)
 
@@ -278,11 +280,12 @@ def decode_tensor(enc) -> np.ndarray:
 #   56 u32 lut_bits | 60 u32 lag_bits | 64 u32 n_fields | 68 u8 caps[4] | 72 u16 pad_word | 74 u16 0
 #   76 u32 max_words | 80 u64 off_codebook | 88 u64 off_lut | 96 u64 off_index | 104 u64 off_payload
 #   112 u64 payload_bytes | 120 u64 blob_bytes | 128 u64 coded_bits | 136 u64 raw_bits | 144 u64 checksum
-# codebook: u8 lengths[3][32].  LUT: u32[1 << lut_bits], entry = E << 23 | (len0 + len1), indexed by the
+# codebook: u8 lengths[3][32].  LUT: u32[1 << lut_bits], entry = (len0 + len1) << 16 | E << 7, indexed by the
 # next lut_bits stream bits (first bit = bit 0).  index: u32[n_chunks + 1], record offsets in 128-byte
-# units from off_payload.  Record of a chunk with nkb blocks: raw bytes [nkb][32 lanes][16], then W rows
-# of 32 little-endian u32 (row j, lane l): the lane's bit sequence, bit i in word i // 32 at bit i % 32,
-# starting with LAG_BITS zero bits; unused bits after the last codeword are zero.
+# units from off_payload.  Record of a chunk with nkb blocks: raw bytes [nkb][32 lanes][16] (a lane's 16
+# bytes: row g's eight weights, then row g+8's), then W rows of 64 little-endian u32 (row j, sequence s):
+# the sequence's bits, bit i in word i // 32 at bit i % 32, starting with LAG_BITS zero bits; unused bits
+# after the last codeword are zero.
 
 HEADER = struct.Struct("<4sIIIQQIIIIQIII4sHHIQQQQQQQQ")
 
@@ -317,23 +320,23 @@ def parse_blob(blob) -> dict:
     index = np.frombuffer(blob, dtype=np.uint32, count=h["n_chunks"] + 1, offset=h["off_index"]).astype(np.int64)
     assert index[0] == 0 and np.all(np.diff(index) > 0) and index[-1] * 128 == h["payload_bytes"]
     assert h["off_payload"] + h["payload_bytes"] <= len(blob)
-    chunks, max_words, coded_bits = {}, 0, 0
+    chunks, max_words = {}, 0
     for chunk_ids, idx in element_map(rows, cols, ce):
         steps = idx.shape[2]
-        nkb = steps // 16
+        nkb = steps // 8
         for a, cid in enumerate(chunk_ids):
             beg = h["off_payload"] + int(index[cid]) * 128
             size = int(index[cid + 1] - index[cid]) * 128
-            W = (size - nkb * 512) // 128
-            assert W >= 1 and nkb * 512 + W * 128 == size
+            W = (size - nkb * 512) // 256
+            assert W >= 1 and nkb * 512 + W * 256 == size
             max_words = max(max_words, W)
-            raw = np.frombuffer(blob, dtype=np.uint8, count=nkb * 512, offset=beg).reshape(nkb, 32, 16)
-            raw = raw.transpose(1, 0, 2).reshape(32, steps).copy()
-            words = np.frombuffer(blob, dtype="<u4", count=W * 32, offset=beg + nkb * 512).reshape(W, 32)
-            lane_bits = ((words.T[:, :, None] >> np.arange(32, dtype=np.uint32)) & 1).astype(np.uint8).reshape(32, W * 32)
-            assert not lane_bits[:, :LAG_BITS].any(), "lag bits must be zero"
-            body = np.ascontiguousarray(lane_bits[:, LAG_BITS:])
-            off = (np.arange(33, dtype=np.uint64) * np.uint64(body.shape[1]))
+            raw = np.frombuffer(blob, dtype=np.uint8, count=nkb * 512, offset=beg).reshape(nkb, 32, 2, 8)
+            raw = raw.transpose(2, 1, 0, 3).reshape(SEQS, steps).copy()        # [half][lane] -> sequence
+            words = np.frombuffer(blob, dtype="<u4", count=W * SEQS, offset=beg + nkb * 512).reshape(W, SEQS)
+            seq_bits = ((words.T[:, :, None] >> np.arange(32, dtype=np.uint32)) & 1).astype(np.uint8).reshape(SEQS, W * 32)
+            assert not seq_bits[:, :LAG_BITS].any(), "lag bits must be zero"
+            body = np.ascontiguousarray(seq_bits[:, LAG_BITS:])
+            off = (np.arange(SEQS + 1, dtype=np.uint64) * np.uint64(body.shape[1]))
             chunks[int(cid)] = (body.ravel(), off, raw)
     enc = dict(rows=rows, cols=cols, chunk_elems=ce, dtype=dtype, lens=lens, codes=codes, caps=list(h["caps"][:3]),
                pad=h["pad_word"], chunks=chunks, header=h, lut=lut)
@@ -342,8 +345,8 @@ def parse_blob(blob) -> dict:
 
 
 def decode_blob(blob):
-    """Full slow decode of a library blob: (tensor, per-chunk per-lane bits used).  Also checks that every
-    bit after a lane's last codeword is zero and that pad positions hold the pad word."""
+    """Full slow decode of a library blob: (tensor, per-chunk per-sequence bits used).  Also checks that
+    every bit after a sequence's last codeword is zero and that pad positions hold the pad word."""
     enc = parse_blob(blob)
     rows, cols, dtype = enc["rows"], enc["cols"], enc["dtype"]
     out = np.zeros(rows * cols + 1, dtype=np.uint16)
@@ -353,8 +356,8 @@ def decode_blob(blob):
         for a, cid in enumerate(chunk_ids):
             bits, off, raw = enc["chunks"][int(cid)]
             seq, used = decode_sequences(bits, off, raw, enc["lens"], enc["codes"], dtype)
-            per = bits.reshape(32, -1)
-            for l in range(32):
+            per = bits.reshape(SEQS, -1)
+            for l in range(SEQS):
                 assert not per[l, int(used[l]):].any(), "non-zero bits after the last codeword"
             assert np.all(seq[idx[a] < 0] == enc["pad"]), "pad positions must hold the pad word"
             out[idx[a]] = seq
@@ -377,5 +380,5 @@ def lut_from_code(lens, codes, lut_bits: int) -> np.ndarray:
             seq, used = decode_sequences(idx_bits[i], off, raw, lens, codes, BF16)
         except ValueError:
             continue                                   # no codeword pair is a prefix of this index
-        out[i] = (((int(seq[0, 0]) >> 7) & 0xFF) << 23) | int(used[0])
+        out[i] = (int(used[0]) << 16) | (((int(seq[0, 0]) >> 7) & 0xFF) << 7)
     return out

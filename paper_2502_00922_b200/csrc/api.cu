@@ -13,7 +13,7 @@ namespace {
 
 constexpr uint32_t kMaxGrid = 512;        // CTAs the scratch layout provides for
 constexpr uint32_t kKernelBatch = 8;      // activation vectors one launch multiplies
-constexpr uint32_t kStaticSmem = 1024;    // barriers and tags the kernel declares statically (rounded up)
+constexpr uint32_t kStaticSmem = 2048;    // barriers and tables the kernel declares statically (rounded up)
 
 struct DeviceInfo {
     bool known = false;
@@ -37,8 +37,8 @@ huffllm_status device_info(DeviceInfo **out) {
     return HUFFLLM_OK;
 }
 
-// Scratch layout: [0,256) ticket | [256, 256 + 8*kMaxGrid) row-group tags | partial sums
-size_t ws_partial_offset() { return 256 + (size_t)kMaxGrid * 2 * sizeof(int); }
+// Scratch layout: [0, 4096) arrival counters (one per CTA, zero between calls) | partial sums
+size_t ws_partial_offset() { return 4096; }
 size_t ws_bytes_for(uint32_t batch) {
     uint32_t b = batch < kKernelBatch ? batch : kKernelBatch;
     return ws_partial_offset() + (size_t)kMaxGrid * 2 * 16 * b * sizeof(float);
@@ -51,6 +51,7 @@ huffllm_status fill_args(const huffllm_desc *desc, const void *blob, uint32_t ba
     if (!blob || ((uintptr_t)blob & 255)) return fail(HUFFLLM_ERR_INVALID_ARG, "blob must be a 256-byte aligned device pointer");
     if (desc->lut_bits > 9)
         return fail(HUFFLLM_ERR_UNSUPPORTED, "device kernels take max_code_len 8 or 9 (this blob: %u)", desc->lut_bits);
+    if (desc->n_chunks >= (1ull << 31)) return fail(HUFFLLM_ERR_UNSUPPORTED, "too many chunks for one launch");
     memset(k, 0, sizeof(*k));
     k->blob = (const uint8_t *)blob;
     k->off_lut = desc->off_lut;
@@ -63,9 +64,10 @@ huffllm_status fill_args(const huffllm_desc *desc, const void *blob, uint32_t ba
     k->chunk_cols = desc->chunk_cols;
     k->col_chunks = desc->col_chunks;
     k->lut_bits = desc->lut_bits;
-    k->slot_bytes = (desc->max_words + 1) * 128;
-    const uint32_t checks_per_block = desc->lut_bits == 8 ? 6 : 8;
-    k->guard_bytes = 128 * (3 + checks_per_block * (desc->chunk_cols / kBlockCols));
+    k->slot_bytes = (desc->max_words + 1) * 256;
+    // a corrupt stream can advance its read pointer by one row per refill check and no further
+    const uint32_t checks_per_block = desc->lut_bits == 8 ? 3 : 4;
+    k->guard_bytes = 256 * (3 + checks_per_block * (desc->chunk_cols / kBlockCols));
     k->part_bytes = product ? 2 * 32 * 16 * batch * (uint32_t)sizeof(float) : 0;
     k->dyn_smem_bytes = (uint32_t)dev.smem_optin - kStaticSmem;
     k->batch = batch;
@@ -132,7 +134,6 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
         k.x = x + (uint64_t)b0 * desc->cols;
         k.y = y + (uint64_t)b0 * desc->rows;
         k.ws_ticket = (unsigned int *)workspace;
-        k.ws_rg = (int *)((uint8_t *)workspace + 256);
         k.ws_partial = (float *)((uint8_t *)workspace + ws_partial_offset());
         k.err = err_flag;
         cudaError_t e = launch_gemm(k, grid, (cudaStream_t)stream);

@@ -53,7 +53,7 @@ huffllm_status check_desc(const huffllm_desc *d) {
         d->n_chunks != (uint64_t)d->row_groups * d->col_chunks)
         return fail(HUFFLLM_ERR_CORRUPT, "chunk counts do not match the shape");
     if (d->lut_bits < kMinBudget || d->lut_bits > kMaxBudget) return fail(HUFFLLM_ERR_CORRUPT, "bad lut_bits");
-    uint32_t max_steps = d->chunk_cols / kBlockCols * 16;
+    uint32_t max_steps = d->chunk_cols / kBlockCols * 8;   // per bit sequence
     uint32_t w_bound = (kLagBits + max_steps * d->lut_bits + 31) / 32;
     if (d->max_words == 0 || d->max_words > w_bound) return fail(HUFFLLM_ERR_CORRUPT, "bad max_words");
     if (d->off_codebook % 256 || d->off_lut % 256 || d->off_index % 256 || d->off_payload % 256 ||
@@ -167,7 +167,7 @@ static void finish_codebook(huffllm_codebook *cb) {
         cb->len8[e] = (uint8_t)L;
         cb->bits8[e] = seq;
         for (uint32_t hi = 0; hi < (1u << (cb->budget - L)); ++hi)
-            cb->lut[seq | (hi << L)] = ((uint32_t)e << 23) | (uint32_t)L;
+            cb->lut[seq | (hi << L)] = ((uint32_t)L << 16) | ((uint32_t)e << 7);
     }
     int f[2];
     for (int k = 0; k < 2; ++k) {
@@ -289,10 +289,11 @@ inline uint32_t blocks_of(const Geometry &g, uint32_t kc) {
     return (uint32_t)((std::min<uint64_t>(left, g.Kc) + kBlockCols - 1) / kBlockCols);
 }
 
-// The weight at (chunk, lane, step) of the element map, or the pad word outside the tensor.
-inline uint16_t weight_at(const uint16_t *w, const Geometry &g, uint32_t rg, uint32_t kc, uint32_t lane, uint32_t step,
+// The weight at (chunk, sequence, step) of the element map, or the pad word outside the tensor.
+// Sequence s belongs to lane s % 32 and holds row g (s < 32) or row g + 8 (s >= 32) of the tile.
+inline uint16_t weight_at(const uint16_t *w, const Geometry &g, uint32_t rg, uint32_t kc, uint32_t seq, uint32_t step,
                           uint16_t pad) {
-    uint32_t gg = lane >> 2, t = lane & 3, kb = step >> 4, half = (step >> 3) & 1, i = step & 7;
+    uint32_t lane = seq & 31, half = seq >> 5, gg = lane >> 2, t = lane & 3, kb = step >> 3, i = step & 7;
     uint64_t r = (uint64_t)rg * 16 + gg + 8 * half;
     uint64_t c = (uint64_t)kc * g.Kc + (uint64_t)kb * 32 + t * 8 + i;
     return (r < g.rows && c < g.cols) ? w[r * g.cols + c] : pad;
@@ -329,8 +330,8 @@ huffllm_status huffllm_encode_bound(uint64_t rows, uint64_t cols, huffllm_dtype 
     uint64_t payload = 0;
     for (uint32_t kc = 0; kc < g.KC; ++kc) {
         uint32_t nkb = blocks_of(g, kc);
-        uint64_t w = (kLagBits + (uint64_t)nkb * 16 * kMaxBudget + 31) / 32;
-        payload += (uint64_t)g.RG * (nkb * 512ull + w * 128ull);
+        uint64_t w = (kLagBits + (uint64_t)nkb * 8 * kMaxBudget + 31) / 32;
+        payload += (uint64_t)g.RG * (nkb * 512ull + w * 256ull);
     }
     uint64_t n_chunks = (uint64_t)g.RG * g.KC;
     *max_bytes = (size_t)(256 + 256 + align_up(4ull << kMaxBudget, 256) + align_up(4 * (n_chunks + 1), 256) + payload + 256);
@@ -369,17 +370,17 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
     d.off_payload = d.off_index + align_up(4 * (n_chunks + 1), 256);
     if (blob_cap < d.off_payload) return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "blob capacity below the fixed sections");
 
-    // pass 1: words per lane row (W) of every chunk, from the code lengths alone
+    // pass 1: words per sequence (W) of every chunk, from the code lengths alone
     std::vector<uint32_t> words(n_chunks);
     std::vector<uint64_t> chunk_bits(n_chunks);
     std::atomic<int> bad{0};
     const uint8_t *len8 = cb->len8;
     const uint16_t pad = cb->pad_word;
     parallel_chunks(n_chunks, [&](uint64_t c) {
-        uint32_t rg = (uint32_t)(c / g.KC), kc = (uint32_t)(c % g.KC), steps = blocks_of(g, kc) * 16;
+        uint32_t rg = (uint32_t)(c / g.KC), kc = (uint32_t)(c % g.KC), steps = blocks_of(g, kc) * 8;
         uint32_t max_bits = 0;
         uint64_t sum = 0;
-        for (uint32_t lane = 0; lane < 32; ++lane) {
+        for (uint32_t lane = 0; lane < kSeqs; ++lane) {
             uint32_t bits = 0;
             for (uint32_t s = 0; s < steps; ++s) {
                 uint32_t l = len8[(weight_at(w, g, rg, kc, lane, s, pad) >> 7) & 0xFF];
@@ -400,7 +401,7 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
     uint64_t coded_bits = 0;
     for (uint64_t c = 0; c < n_chunks; ++c) {
         uint32_t nkb = blocks_of(g, (uint32_t)(c % g.KC));
-        rec[c + 1] = rec[c] + (nkb * 512ull + words[c] * 128ull) / kRecordUnit;
+        rec[c + 1] = rec[c] + (nkb * 512ull + words[c] * 256ull) / kRecordUnit;
         max_words = std::max(max_words, words[c]);
         coded_bits += chunk_bits[c];
     }
@@ -425,29 +426,29 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
     const uint32_t *bits8 = cb->bits8;
     std::atomic<uint64_t> checksum{0};
     parallel_chunks(n_chunks, [&](uint64_t c) {
-        uint32_t rg = (uint32_t)(c / g.KC), kc = (uint32_t)(c % g.KC), nkb = blocks_of(g, kc), steps = nkb * 16;
+        uint32_t rg = (uint32_t)(c / g.KC), kc = (uint32_t)(c % g.KC), nkb = blocks_of(g, kc), steps = nkb * 8;
         uint32_t W = words[c];
         uint8_t *raw = base + d.off_payload + rec[c] * kRecordUnit;
         uint32_t *coded = (uint32_t *)(raw + nkb * 512ull);
-        memset(coded, 0, (size_t)W * 128);
-        for (uint32_t lane = 0; lane < 32; ++lane) {
+        memset(coded, 0, (size_t)W * 256);
+        for (uint32_t lane = 0; lane < kSeqs; ++lane) {
             uint64_t acc = 0;
             uint32_t nacc = kLagBits, j = 0;
             for (uint32_t s = 0; s < steps; ++s) {
                 uint16_t v = weight_at(w, g, rg, kc, lane, s, pad);
-                raw[(s >> 4) * 512 + lane * 16 + (s & 15)] = (uint8_t)(((v >> 8) & 0x80) | (v & 0x7F));
+                raw[(s >> 3) * 512 + (lane & 31) * 16 + (lane >> 5) * 8 + (s & 7)] = (uint8_t)(((v >> 8) & 0x80) | (v & 0x7F));
                 uint32_t e = (v >> 7) & 0xFF;
                 acc |= (uint64_t)bits8[e] << nacc;
                 nacc += len8[e];
                 if (nacc >= 32) {
-                    coded[(size_t)j++ * 32 + lane] = (uint32_t)acc;
+                    coded[(size_t)j++ * kSeqs + lane] = (uint32_t)acc;
                     acc >>= 32;
                     nacc -= 32;
                 }
             }
-            if (nacc) coded[(size_t)j * 32 + lane] = (uint32_t)acc;
+            if (nacc) coded[(size_t)j * kSeqs + lane] = (uint32_t)acc;
         }
-        checksum.fetch_add(record_checksum(raw, nkb * 512ull + (uint64_t)W * 128, c));
+        checksum.fetch_add(record_checksum(raw, nkb * 512ull + (uint64_t)W * 256, c));
     });
     d.payload_checksum = checksum.load();
     memcpy(base, &d, sizeof(d));
@@ -506,31 +507,32 @@ huffllm_status huffllm_validate_blob(const void *blob, size_t bytes, huffllm_des
     std::atomic<uint32_t> max_words{0};
     const uint32_t mask = (1u << d.lut_bits) - 1;
     parallel_chunks(d.n_chunks, [&](uint64_t c) {
-        uint32_t kc = (uint32_t)(c % g.KC), rg = (uint32_t)(c / g.KC), nkb = blocks_of(g, kc), steps = nkb * 16;
+        uint32_t kc = (uint32_t)(c % g.KC), rg = (uint32_t)(c / g.KC), nkb = blocks_of(g, kc), steps = nkb * 8;
         if (index[c + 1] <= index[c]) { bad.store(1); return; }
         uint64_t size = (uint64_t)(index[c + 1] - index[c]) * kRecordUnit;
         if (size <= nkb * 512ull) { bad.store(2); return; }
-        uint32_t W = (uint32_t)((size - nkb * 512ull) / 128);
+        if ((size - nkb * 512ull) % 256) { bad.store(9); return; }
+        uint32_t W = (uint32_t)((size - nkb * 512ull) / 256);
         if (W > d.max_words) { bad.store(3); return; }
         uint32_t seen = max_words.load();
         while (W > seen && !max_words.compare_exchange_weak(seen, W)) {}
         const uint8_t *raw = base + d.off_payload + (uint64_t)index[c] * kRecordUnit;
         const uint32_t *coded = (const uint32_t *)(raw + nkb * 512ull);
         uint64_t sum = 0;
-        for (uint32_t lane = 0; lane < 32; ++lane) {
-            auto word = [&](uint32_t j) -> uint64_t { return j < W ? coded[(size_t)j * 32 + lane] : 0; };
+        for (uint32_t lane = 0; lane < kSeqs; ++lane) {
+            auto word = [&](uint32_t j) -> uint64_t { return j < W ? coded[(size_t)j * kSeqs + lane] : 0; };
             if (word(0) & ((1u << kLagBits) - 1)) { bad.store(4); return; }
             uint32_t pos = kLagBits;
             for (uint32_t s = 0; s < steps; ++s) {
                 uint64_t win = (word(pos >> 5) | (word((pos >> 5) + 1) << 32)) >> (pos & 31);
                 uint32_t e = cb.lut[(uint32_t)win & mask];
-                uint32_t l = e & 0x7FFFFF;
+                uint32_t l = e >> 16;
                 if (!l) { bad.store(5); return; }
-                uint32_t gg = lane >> 2, t = lane & 3, kb = s >> 4, half = (s >> 3) & 1, i = s & 7;
+                uint32_t ln = lane & 31, half = lane >> 5, gg = ln >> 2, t = ln & 3, kb = s >> 3, i = s & 7;
                 uint64_t r = (uint64_t)rg * 16 + gg + 8 * half, col = (uint64_t)kc * g.Kc + kb * 32ull + t * 8 + i;
                 if (r >= g.rows || col >= g.cols) {
-                    uint8_t rb = raw[(s >> 4) * 512 + lane * 16 + (s & 15)];
-                    if (rb != 0 || (e >> 23) != ((d.pad_word >> 7) & 0xFFu)) { bad.store(6); return; }
+                    uint8_t rb = raw[(s >> 3) * 512 + ln * 16 + half * 8 + (s & 7)];
+                    if (rb != 0 || ((e >> 7) & 0xFFu) != ((d.pad_word >> 7) & 0xFFu)) { bad.store(6); return; }
                 }
                 pos += l;
                 sum += l;

@@ -12,7 +12,8 @@ namespace huffllm {
 
 constexpr uint32_t kTileRows = 16;      // rows of a chunk tile
 constexpr uint32_t kBlockCols = 32;     // columns of one block (16 weights per lane)
-constexpr uint32_t kLagBits = 7;        // zero bits in front of every lane sequence
+constexpr uint32_t kLagBits = 7;        // zero bits in front of every bit sequence
+constexpr uint32_t kSeqs = 64;          // bit sequences per chunk: two per lane (rows g and g + 8)
 constexpr uint32_t kDefaultBudget = 8;  // default joint code-length bound
 constexpr uint32_t kMinBudget = 8, kMaxBudget = 12;
 constexpr uint32_t kRecordUnit = 128;   // record offsets are counted in this many bytes

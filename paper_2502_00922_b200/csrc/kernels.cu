@@ -10,7 +10,8 @@
 // weights never touch memory (Section 1).
 //
 // Mapping to the GPU
-//   * one warp decodes one chunk; lane l owns the bit sequence of lane l in the chunk record
+//   * one warp decodes one chunk; lane l owns the two bit sequences l and 32 + l of the chunk record
+//     and steps through them alternately, which gives every lane two independent dependency chains
 //   * the coded part of a record is brought into shared memory by one bulk-async copy per chunk
 //     (no multicast), completion on an mbarrier; two slots per warp, so the next chunk is in
 //     flight while this one is decoded
@@ -89,63 +90,77 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
 
 // ------------------------------------------------------------------------------ lane decoder
 
-// State of one lane's decoder.  (hi:lo) holds 64 stream bits; the current codeword starts at bit
-// pos + 7 of that window (the 7 bits in front are the lag that makes the table address fall out of
-// a single AND/OR); nxt is the shared-memory address of the lane's next 32-bit word.
+// State of the decoder of one bit sequence.  (hi:lo) holds 64 stream bits; the current codeword starts
+// at bit pos + 7 of that window (the 7 bits in front are the lag that makes the table address fall out
+// of a single AND/OR); nxt is the shared-memory address of the sequence's next 32-bit word.  Words of
+// one sequence are 256 bytes apart (a row of the record holds one word of each of the 64 sequences).
 struct LaneStream {
     uint32_t lo, hi, pos, nxt;
 };
 
 __device__ __forceinline__ void stream_open(LaneStream &s, uint32_t lane_word0) {
     s.lo = lds_stream(lane_word0);
-    s.hi = lds_stream(lane_word0 + 128);
-    s.nxt = lane_word0 + 256;
+    s.hi = lds_stream(lane_word0 + 256);
+    s.nxt = lane_word0 + 512;
     s.pos = 0;
 }
 
-// One decoder step: returns the table entry (exponent << 23 | length) and advances the start pointer.
+// One decoder step: returns the table entry (length << 16 | exponent << 7) and advances the start pointer.
 // The window is shifted as a 64-bit value, so the pointer may run past bit 32 between two refill
-// checks.  Only the entry's low byte (the length) is added to the pointer: dp4a with the byte
-// selector 1 does "pos += e & 0xFF" in one instruction, off the integer ALU pipe.
+// checks.  The table address is (window & index mask) | (table base + 4 * lane): one logic operation,
+// because the table sits on a boundary above the index bits.  Only byte 2 of the entry (the length)
+// is added to the pointer: dp4a with that byte selected does it in one instruction off the ALU pipe.
 __device__ __forceinline__ uint32_t stream_step(LaneStream &s, uint32_t idx_mask, uint32_t lut_lane) {
     uint64_t win = ((uint64_t)s.hi << 32) | s.lo;
-    uint32_t t = (uint32_t)(win >> s.pos);
-    uint32_t e = lds_lut((t & idx_mask) | lut_lane);
-    s.pos = __dp4a(e, 1u, s.pos);
+    uint32_t t = (uint32_t)(win >> s.pos), addr;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(addr) : "r"(t), "r"(idx_mask), "r"(lut_lane));
+    uint32_t e = lds_lut(addr);
+    s.pos = __dp4a(e, 0x00010000u, s.pos);
     return e;
 }
 
-// Refill: once 32 bits have been consumed, slide the window by one word.
+// Refill: once 32 bits have been consumed, slide the window by one word.  Written with predicated
+// instructions so that lanes which need a word and lanes which do not stay converged.
 __device__ __forceinline__ void stream_refill(LaneStream &s) {
-    if (s.pos & 32u) {
-        s.lo = s.hi;
-        s.hi = lds_stream(s.nxt);
-        s.nxt += 128;
-    }
-    s.pos &= 31u;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ge.u32 p, %2, 32;\n\t"
+        "@p mov.u32 %0, %1;\n\t"
+        "@p ld.shared.u32 %1, [%3];\n\t"
+        "@p add.u32 %3, %3, 256;\n\t"
+        "@p add.u32 %2, %2, -32;\n\t}"
+        : "+r"(s.lo), "+r"(s.hi), "+r"(s.pos), "+r"(s.nxt));
 }
 
 // Two table entries + two raw bytes -> two bf16 weights packed in one register.
-// SEL picks raw bytes (i, i+1) of `raw` as (byte, sign-replicated byte) pairs.
+// SEL picks raw bytes (i, i+1) of `raw` as (byte, sign-replicated byte) pairs.  The exponent of the
+// even weight is already in place (bits 7..14); the odd entry times 65536 puts its exponent at bits
+// 23..30 and pushes its length out of the word, so one multiply-add (FMA pipe) merges the two.
 template <uint32_t SEL>
 __device__ __forceinline__ uint32_t pack_pair(uint32_t e_even, uint32_t e_odd, uint32_t raw) {
-    uint32_t sm = prmt(raw, 0u, SEL);             // [sign1*0xFF, raw1, sign0*0xFF, raw0]
-    uint32_t ex = prmt(e_even, e_odd, 0x7632u);   // [E1 << 7 | E0 << 7] in the two halves
+    uint32_t sm = prmt(raw, 0u, SEL);   // [sign1*0xFF, raw1, sign0*0xFF, raw0]
+    uint32_t ex;
+    asm("mad.lo.u32 %0, %1, 65536, %2;" : "=r"(ex) : "r"(e_odd), "r"(e_even));
     return (sm & 0x807F807Fu) | (ex & 0x7F807F80u);
 }
 
 // Decode one block (16 weights of this lane) into 8 packed registers:
 // a[0..3] = row g, columns (0,1) (2,3) (4,5) (6,7);  a[4..7] = row g+8, same columns.
-// The window is checked for a refill before every R-th step: after a check at least 26 bits are
-// valid in front of the start pointer, enough for R codewords of at most 26/R bits.
+// The lane's two sequences are stepped alternately.  Each window is checked for a refill before every
+// R-th step: after a check at least 26 bits are valid in front of the start pointer, enough for R
+// codewords of at most 26/R bits.
 template <int R>
-__device__ __forceinline__ void decode_block(LaneStream &s, uint32_t idx_mask, uint32_t lut_lane, const uint4 &raw,
-                                             uint32_t (&a)[8]) {
+__device__ __forceinline__ void decode_block(LaneStream &sa, LaneStream &sb, uint32_t idx_mask, uint32_t lut_lane,
+                                             const uint4 &raw, uint32_t (&a)[8]) {
     uint32_t e[16];
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-        if (i % R == 0) stream_refill(s);
-        e[i] = stream_step(s, idx_mask, lut_lane);
+    for (int i = 0; i < 8; ++i) {
+        if (i % R == 0) {
+            stream_refill(sa);
+            stream_refill(sb);
+        }
+        e[i] = stream_step(sa, idx_mask, lut_lane);
+        e[8 + i] = stream_step(sb, idx_mask, lut_lane);
     }
     a[0] = pack_pair<0x9180u>(e[0], e[1], raw.x);
     a[1] = pack_pair<0xB3A2u>(e[2], e[3], raw.x);
@@ -193,43 +208,48 @@ __device__ __forceinline__ uint32_t slot_addr(const SmemPlan &p, uint32_t warp, 
 }
 
 constexpr int kMaxWarps = 32;
+// Experiment build only (-DHUFFLLM_TIMING): every warp writes nanosecond stamps of its phases into the
+// buffer passed as the error flag, [cta][warp][8].
+#ifdef HUFFLLM_TIMING
+__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define STAMP(i) do { if (lane == 0) ((unsigned long long *)k.err)[((size_t)blockIdx.x * 32 + warp) * 8 + (i)] = gtime(); } while (0)
+#else
+#define STAMP(i) do {} while (0)
+#endif
+#ifndef HUFFLLM_THREADS
+#define HUFFLLM_THREADS 1024
+#endif
+constexpr int kThreads = HUFFLLM_THREADS;   // threads per CTA of the decode kernels (one CTA per SM)
 constexpr uint32_t kWaitLimit = 1u << 22;
 
 // ------------------------------------------------------------------------------ the fused kernel
 
 // MODE 0: write the decoded weights.  MODE 1: y = W x for up to 8 activation vectors.
-// R = decoder steps between two refill checks (3 when codewords are at most 8 bits, else 2).
-template <int MODE, int R>
-__global__ void __launch_bounds__(1024, 1) huff_kernel(const KernelArgs k) {
+// LB = table index bits (the blob's lut_bits): 8 or 9.
+template <int MODE, int LB, int THREADS>
+__global__ void __launch_bounds__(THREADS, 1) huff_kernel(const KernelArgs k) {
+    constexpr int R = LB == 8 ? 3 : 2;                       // decoder steps between two refill checks
+    constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
     extern __shared__ __align__(128) uint8_t dyn_smem[];
     __shared__ __align__(8) uint64_t bars[kMaxWarps * 2];
     __shared__ int part_rg[kMaxWarps * 2];
-    __shared__ uint32_t s_last;
+    __shared__ int s_split_rg[2];        // row groups of this CTA that other CTAs also hold pieces of
+    __shared__ uint32_t s_split_info[2];
+    __shared__ uint32_t s_grp_first[kMaxWarps * 2 + 1], s_ngroups;
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps_launched = blockDim.x >> 5;
+    STAMP(0);
     const uint32_t smem_base = smem_u32(dyn_smem);
     const SmemPlan plan = plan_smem(smem_base, k, nwarps_launched);
     const uint32_t nw = plan.warps;
     const uint32_t vals = 16 * k.batch;
     float *part_val = (float *)(dyn_smem + k.dyn_smem_bytes - k.part_bytes);  // [2 * warps][16 * batch]
 
-    // ---- set-up: per-lane table, barriers
-    {
-        const uint32_t *lut_g = (const uint32_t *)(k.blob + k.off_lut);
-        uint32_t *lut_s = (uint32_t *)(dyn_smem + (plan.lut - smem_base));
-        for (uint32_t i = tid; i < (32u << k.lut_bits); i += blockDim.x) lut_s[i] = __ldg(lut_g + (i >> 5));
-        if (tid < kMaxWarps * 2) {
-            mbar_init(smem_u32(&bars[tid]), 1);
-            part_rg[tid] = -1;
-        }
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    __syncthreads();
-
     // ---- this warp's contiguous range of chunks
-    const uint64_t T = k.n_chunks;
-    const uint64_t cta_beg = T * blockIdx.x / gridDim.x, cta_end = T * (blockIdx.x + 1) / gridDim.x;
-    uint64_t c_beg = cta_beg, c_end = cta_beg;
+    const uint32_t T = (uint32_t)k.n_chunks;   // the entry points refuse tensors with 2^31 chunks or more
+    const uint32_t KC = k.col_chunks;
+    const uint32_t cta_beg = (uint32_t)((uint64_t)T * blockIdx.x / gridDim.x), cta_end = (uint32_t)((uint64_t)T * (blockIdx.x + 1) / gridDim.x);
+    uint32_t c_beg = cta_beg, c_end = cta_beg;
     if (warp < nw) {
         c_beg = cta_beg + (cta_end - cta_beg) * warp / nw;
         c_end = cta_beg + (cta_end - cta_beg) * (warp + 1) / nw;
@@ -237,41 +257,65 @@ __global__ void __launch_bounds__(1024, 1) huff_kernel(const KernelArgs k) {
 
     const uint32_t *index = (const uint32_t *)(k.blob + k.off_index);
     const uint8_t *payload = k.blob + k.off_payload;
-    const uint32_t idx_mask = ((1u << k.lut_bits) - 1u) << 7;
-    const uint32_t lut_lane = plan.lut | (lane << 2);
+    uint32_t lut_lane = plan.lut | (lane << 2);
+    asm volatile("mov.u32 %0, %0;" : "+r"(lut_lane));  // keep it in a register: it is an operand of every lookup
     const uint32_t g = lane >> 2, t = lane & 3;
+    const uint32_t bar0 = smem_u32(&bars[warp * 2]);
+    const uint32_t slot0 = slot_addr(plan, warp, 0, k.slot_bytes);
 
-    auto blocks_of = [&](uint64_t c) -> uint32_t {
-        uint32_t kc = (uint32_t)(c % k.col_chunks);
-        uint32_t left = (uint32_t)(k.cols - (uint64_t)kc * k.chunk_cols);
+    // blocks of 32 columns in column chunk kc
+    auto blocks_of = [&](uint32_t kc) -> uint32_t {
+        uint32_t left = (uint32_t)k.cols - kc * k.chunk_cols;
         return (min(left, k.chunk_cols) + 31u) >> 5;
     };
     // a record is usable if it lies inside the payload and its coded part fits a slot
     auto record_ok = [&](uint32_t r0, uint32_t r1, uint32_t nkb) -> bool {
         return r1 > r0 && r1 <= k.payload_units && (r1 - r0) * 128u > nkb * 512u &&
-               (r1 - r0) * 128u - nkb * 512u + 128u <= k.slot_bytes;
+               (r1 - r0) * 128u - nkb * 512u + 256u <= k.slot_bytes;
     };
-    // lane 0: start the bulk copy of chunk c's coded part into slot `which`
-    auto issue = [&](uint64_t c, uint32_t which) {
-        uint32_t nkb = blocks_of(c), r0 = __ldg(index + c), r1 = __ldg(index + c + 1);
-        uint32_t bar = smem_u32(&bars[warp * 2 + which]);
+    // lane 0: start the bulk copy of a chunk's coded part into slot `which`
+    auto issue = [&](uint32_t c, uint32_t which) {
+        uint32_t nkb = blocks_of(c % KC), r0 = __ldg(index + c), r1 = __ldg(index + c + 1);
+        uint32_t bar = bar0 + which * 8;
         if (record_ok(r0, r1, nkb)) {
             uint32_t bytes = (r1 - r0) * 128u - nkb * 512u;
             mbar_expect_tx(bar, bytes);
-            bulk_g2s(slot_addr(plan, warp, which, k.slot_bytes), payload + (uint64_t)r0 * 128u + nkb * 512u, bytes, bar);
+            bulk_g2s(slot0 + which * k.slot_bytes, payload + (uint64_t)r0 * 128u + nkb * 512u, bytes, bar);
         } else {
             mbar_expect_tx(bar, 0);  // completes the phase with nothing to wait for; the chunk is skipped below
         }
     };
 
+    // ---- set-up.  Every warp arms its own two barriers and starts its first copies at once, so the
+    // first compressed bytes are already on their way while the CTA builds the per-lane table.
+    if (lane == 0) {
+        mbar_init(bar0, 1);
+        mbar_init(bar0 + 8, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if (c_beg < c_end) {
+            issue(c_beg, 0);
+            if (c_beg + 1 < c_end) issue(c_beg + 1, 1);
+        }
+    }
+    {
+        const uint32_t *lut_g = (const uint32_t *)(k.blob + k.off_lut);
+        uint32_t *lut_s = (uint32_t *)(dyn_smem + (plan.lut - smem_base));
+        for (uint32_t i = tid; i < (32u << LB); i += THREADS) lut_s[i] = __ldg(lut_g + (i >> 5));
+        if (tid < kMaxWarps * 2) part_rg[tid] = -1;
+        if (tid < 2) s_split_rg[tid] = -1;
+    }
+    STAMP(1);
+    __syncthreads();
+    STAMP(2);
+
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
-    int64_t cur_rg = -1;
+    int cur_rg = -1;
     uint32_t n_partial = 0;
 
     // hand a finished row group to y (if this warp saw all of its chunks) or to the CTA's partial table
-    auto flush = [&](int64_t rg, uint64_t first_c, uint64_t last_c_excl) {
+    auto flush = [&](int rg, uint32_t first_c, uint32_t last_c_excl) {
         if (rg < 0) return;
-        bool complete = first_c <= (uint64_t)rg * k.col_chunks && last_c_excl >= (uint64_t)(rg + 1) * k.col_chunks;
+        bool complete = first_c <= (uint32_t)rg * KC && last_c_excl >= (uint32_t)(rg + 1) * KC;
         uint32_t ent = warp * 2 + min(n_partial, 1u);
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
@@ -292,35 +336,36 @@ __global__ void __launch_bounds__(1024, 1) huff_kernel(const KernelArgs k) {
     };
 
     if (c_beg < c_end) {
-        if (lane == 0) {
-            issue(c_beg, 0);
-            if (c_beg + 1 < c_end) issue(c_beg + 1, 1);
-        }
-        uint4 raw_next = make_uint4(0, 0, 0, 0);
-        {
-            uint32_t r0 = __ldg(index + c_beg);
-            if (r0 + 4u <= k.payload_units) raw_next = ldg_stream16(payload + (uint64_t)r0 * 128u + lane * 16u);
-        }
-        bool failed = false;
+        uint32_t rg = c_beg / KC, kc = c_beg - rg * KC;            // tracked incrementally from here on
+        uint32_t r0 = __ldg(index + c_beg), r1 = __ldg(index + c_beg + 1);
+        // raw sign/mantissa bytes travel one block ahead of the decoder, in two register sets used in turn
+        uint4 raw_a = make_uint4(0, 0, 0, 0), raw_b = make_uint4(0, 0, 0, 0);
+        bool primed = false, failed = false;
 
-        for (uint64_t c = c_beg; c < c_end; ++c) {
-            const uint32_t which = (uint32_t)(c - c_beg) & 1u, parity = (uint32_t)((c - c_beg) >> 1) & 1u;
-            const uint32_t rg = (uint32_t)(c / k.col_chunks), kc = (uint32_t)(c % k.col_chunks);
-            const uint32_t nkb = blocks_of(c);
-            const uint32_t r0 = __ldg(index + c), r1 = __ldg(index + c + 1);
+        for (uint32_t c = c_beg; c < c_end; ++c) {
+            const uint32_t which = (c - c_beg) & 1u, parity = ((c - c_beg) >> 1) & 1u;
+            const uint32_t nkb = blocks_of(kc);
             const bool ok = record_ok(r0, r1, nkb);
-            const uint8_t *raw_g = payload + (uint64_t)r0 * 128u + lane * 16u;
-            const bool next_ok = c + 1 < c_end && r1 + 4u <= k.payload_units;
-            const uint8_t *raw_g_next = payload + (uint64_t)r1 * 128u + lane * 16u;
+            // the chunk after this one: its first raw block is fetched from inside this chunk's loop
+            const bool has_next = c + 1 < c_end;
+            const uint32_t kc1 = kc + 1 == KC ? 0u : kc + 1;
+            const uint32_t r2 = has_next ? __ldg(index + c + 2) : r1;
+            const bool next_ok = has_next && record_ok(r1, r2, blocks_of(kc1));
 
-            if (MODE == 1 && (int64_t)rg != cur_rg) {
+            if (MODE == 1 && (int)rg != cur_rg) {
                 flush(cur_rg, c_beg, c);  // the previous row group ended with chunk c - 1
-                cur_rg = rg;
+                cur_rg = (int)rg;
             }
+
+            // records follow each other in memory: the block after this chunk's last one is the first block of
+            // the next record, `coded_bytes` further on
+            const uint8_t *raw_p = payload + (uint64_t)r0 * 128u + lane * 16u;   // raw bytes of block 0
+            const uint32_t coded_bytes = (r1 - r0) * 128u - nkb * 512u;
+            if (ok && !primed) raw_a = ldg_stream16(raw_p);
 
             // wait, with a limit, for the coded part; the outcome is made uniform across the warp
             {
-                uint32_t bar = smem_u32(&bars[warp * 2 + which]), spins = 0;
+                uint32_t bar = bar0 + which * 8, spins = 0;
                 bool done = mbar_try_wait(bar, parity);
                 while (!__all_sync(0xFFFFFFFFu, done)) {
                     if (++spins > kWaitLimit) { failed = true; break; }
@@ -332,124 +377,156 @@ __global__ void __launch_bounds__(1024, 1) huff_kernel(const KernelArgs k) {
                 }
             }
 
+            if (c == c_beg) STAMP(3);
             if (!ok) {  // record offsets out of range: report, produce nothing for this chunk, touch no memory
-                if (k.err && lane == 0) atomicExch(k.err, (int32_t)min(c + 1, (uint64_t)0x7FFFFFFF));
-                raw_next = next_ok ? ldg_stream16(raw_g_next) : make_uint4(0, 0, 0, 0);
+                if (k.err && lane == 0) atomicExch(k.err, (int32_t)min(c + 1, 0x7FFFFFFFu));
+                primed = false;
             } else {
-                LaneStream s;
-                stream_open(s, slot_addr(plan, warp, which, k.slot_bytes) + (lane << 2));
-                const uint64_t col0 = (uint64_t)kc * k.chunk_cols + t * 8u;
+                LaneStream sa, sb;
+                stream_open(sa, slot0 + which * k.slot_bytes + (lane << 2));
+                stream_open(sb, slot0 + which * k.slot_bytes + 128u + (lane << 2));
+                const uint32_t col0 = kc * k.chunk_cols + t * 8u;
+                // activations: lanes of unused output columns repeat the last vector; nx = blocks with a column in range
+                const uint16_t *xp = k.x + (MODE == 1 ? (uint64_t)min(g, k.batch - 1) * k.cols + col0 : 0);
+                const uint32_t nx = (MODE == 1 && col0 < (uint32_t)k.cols) ? min(nkb, ((uint32_t)k.cols - col0 + 31u) >> 5) : 0u;
+                uint16_t *out0 = MODE == 0 ? k.out + ((uint64_t)rg * 16 + g) * k.cols + col0 : nullptr;
 
-                for (uint32_t kb = 0; kb < nkb; ++kb) {
-                    const uint4 raw = raw_next;
-                    if (kb + 1 < nkb) raw_next = ldg_stream16(raw_g + (size_t)(kb + 1) * 512u);
-                    else if (next_ok) raw_next = ldg_stream16(raw_g_next);
-
-                    const uint64_t col = col0 + (uint64_t)kb * 32u;
+                // one block: start the fetch of the next block's raw bytes into `nxt`, decode with `cur`
+                auto block = [&](uint32_t kb, const uint4 &cur, uint4 &nxt) {
+                    raw_p += 512;
+                    if (kb + 1 < nkb) nxt = ldg_stream16(raw_p);
+                    else if (next_ok) nxt = ldg_stream16(raw_p + coded_bytes);
                     uint4 xv = make_uint4(0, 0, 0, 0);
-                    if (MODE == 1 && col < k.cols)  // lanes of unused output columns repeat the last vector
-                        xv = __ldg((const uint4 *)(k.x + (uint64_t)min(g, k.batch - 1) * k.cols + col));
+                    if (MODE == 1 && kb < nx) xv = __ldg((const uint4 *)(xp + kb * 32u));
 
                     uint32_t a[8];
-                    decode_block<R>(s, idx_mask, lut_lane, raw, a);
+                    decode_block<R>(sa, sb, kIdxMask, lut_lane, cur, a);
 
                     if (MODE == 1) {
                         mma_bf16_16816(acc, a[0], a[4], a[1], a[5], xv.x, xv.y);
                         mma_bf16_16816(acc, a[2], a[6], a[3], a[7], xv.z, xv.w);
                     } else {
+                        const uint32_t col = col0 + kb * 32u;
 #pragma unroll
                         for (int h = 0; h < 2; ++h) {
-                            uint64_t r = (uint64_t)rg * 16 + g + 8 * h;
-                            if (r >= k.rows || col >= k.cols) continue;
-                            uint16_t *dst = k.out + r * k.cols + col;
+                            if ((uint64_t)rg * 16 + g + 8 * h >= k.rows || col >= (uint32_t)k.cols) continue;
+                            uint16_t *dst = out0 + (uint64_t)(8 * h) * k.cols + kb * 32u;
                             if (k.cols % 8 == 0) {
                                 *(uint4 *)dst = make_uint4(a[4 * h], a[4 * h + 1], a[4 * h + 2], a[4 * h + 3]);
                             } else {
 #pragma unroll
                                 for (int i = 0; i < 8; ++i)
-                                    if (col + i < k.cols) dst[i] = (uint16_t)(a[4 * h + (i >> 1)] >> (16 * (i & 1)));
+                                    if (col + i < (uint32_t)k.cols) dst[i] = (uint16_t)(a[4 * h + (i >> 1)] >> (16 * (i & 1)));
                             }
                         }
                     }
+                };
+                for (uint32_t kb = 0; kb < nkb; kb += 2) {
+                    block(kb, raw_a, raw_b);
+                    if (kb + 1 < nkb) block(kb + 1, raw_b, raw_a);
                 }
+                if (nkb & 1u) raw_a = raw_b;     // the next chunk's first block always starts in raw_a
+                primed = next_ok;
             }
             __syncwarp();
             if (lane == 0 && c + 2 < c_end) issue(c + 2, which);
+            r0 = r1;
+            r1 = r2;
+            kc = kc1;
+            rg += kc1 == 0 ? 1u : 0u;
         }
         if (MODE == 1 && !failed) flush(cur_rg, c_beg, c_end);
     }
 
+    STAMP(4);
     if (MODE != 1) return;
 
-    // ---- combine inside the CTA, in warp order
+    // ---- combine inside the CTA, in warp order.  Entries (warp, slot) are ordered by chunk, so the pieces
+    // of one row group are neighbours; warp 0 finds the group boundaries with ballots, then each group is
+    // summed by its own set of threads, pieces taken in entry order.
     __syncthreads();
-    float *ws_val = k.ws_partial + (size_t)blockIdx.x * 2 * vals;
-    int *ws_rg = k.ws_rg + blockIdx.x * 2;
-    if (tid < vals) {
-        int cur = -1, n_out = 0;
-        float sum = 0.f;
-        auto emit = [&](int rg) {
-            bool complete = cta_beg <= (uint64_t)rg * k.col_chunks && cta_end >= (uint64_t)(rg + 1) * k.col_chunks;
-            if (complete) {
-                uint64_t r = (uint64_t)rg * 16 + (tid & 15);
-                if (r < k.rows) k.y[(uint64_t)(tid >> 4) * k.rows + r] = sum;
-            } else {
-                int slot = min(n_out, 1);
-                ws_val[(size_t)slot * vals + tid] = sum;
-                if (tid == 0) ws_rg[slot] = rg;
-                ++n_out;
-            }
-        };
-        for (uint32_t e = 0; e < nw * 2; ++e) {
-            int rg = part_rg[e];
-            if (rg < 0) continue;
-            if (rg != cur) {
-                if (cur >= 0) emit(cur);
-                cur = rg;
-                sum = 0.f;
-            }
-            sum += part_val[(size_t)e * vals + tid];
+    STAMP(5);
+    const uint32_t G = gridDim.x;
+    const uint32_t first_rg = cta_beg / KC;   // row group of this CTA's first chunk
+    if (warp == 0) {
+        const int t0 = part_rg[lane], t1 = part_rg[lane + 32];
+        const uint32_t v0 = __ballot_sync(0xFFFFFFFFu, t0 >= 0), v1 = __ballot_sync(0xFFFFFFFFu, t1 >= 0);
+        const uint32_t lt = (1u << lane) - 1u, le = lt | (1u << lane);
+        // tag of the nearest valid entry in front of each of this lane's two entries
+        const int p0 = (v0 & lt) ? 31 - __clz(v0 & lt) : 0, p1 = (v1 & lt) ? 31 - __clz(v1 & lt) : 0, pl = v0 ? 31 - __clz(v0) : 0;
+        const int q0 = __shfl_sync(0xFFFFFFFFu, t0, p0), q1 = __shfl_sync(0xFFFFFFFFu, t1, p1), ql = __shfl_sync(0xFFFFFFFFu, t0, pl);
+        const bool s0 = t0 >= 0 && (!(v0 & lt) || q0 != t0);
+        const bool s1 = t1 >= 0 && ((v1 & lt) ? q1 != t1 : (!v0 || ql != t1));
+        const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, s0), b1 = __ballot_sync(0xFFFFFFFFu, s1);
+        if (s0) { s_grp_first[__popc(b0 & le) - 1] = lane; }
+        if (s1) { s_grp_first[__popc(b0) + __popc(b1 & le) - 1] = lane + 32; }
+        if (lane == 0) {
+            s_ngroups = __popc(b0) + __popc(b1);
+            s_grp_first[__popc(b0) + __popc(b1)] = 64;
         }
-        if (cur >= 0) emit(cur);
-        if (tid == 0)
-            for (int sl = n_out; sl < 2; ++sl) ws_rg[sl] = -1;
     }
-
-    // ---- combine across CTAs: the last CTA to arrive adds the boundary partials in CTA order
-    __threadfence();
     __syncthreads();
-    if (tid == 0) s_last = (atomicAdd(k.ws_ticket, 1u) == gridDim.x - 1) ? 1u : 0u;
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    const uint32_t n_ent = gridDim.x * 2;
-    for (uint32_t e = warp; e < n_ent; e += nwarps_launched) {
-        int rg = __ldcg(k.ws_rg + e);
-        if (rg < 0) continue;
-        bool first = true;  // first valid entry of its row group?
-        for (int q = (int)e - 1; q >= 0; --q) {
-            int tag = __ldcg(k.ws_rg + q);
-            if (tag < 0) continue;
-            first = tag != rg;
-            break;
-        }
-        if (!first) continue;
-        for (uint32_t o = lane; o < vals; o += 32) {
-            float sum = 0.f;
-            for (uint32_t q = e; q < n_ent; ++q) {
-                int tag = __ldcg(k.ws_rg + q);
-                if (tag < 0) continue;
-                if (tag != rg) break;
-                sum += __ldcg(k.ws_partial + (size_t)q * vals + o);
-            }
+    for (uint32_t gi = tid / vals; gi < s_ngroups; gi += blockDim.x / vals) {
+        const uint32_t o = tid % vals, e0 = s_grp_first[gi], e1 = s_grp_first[gi + 1];
+        const int rg = part_rg[e0];
+        float sum = 0.f;
+        for (uint32_t e = e0; e < e1; ++e)
+            if (part_rg[e] == rg) sum += part_val[(size_t)e * vals + o];
+        const bool complete = cta_beg <= (uint32_t)rg * KC && cta_end >= (uint32_t)(rg + 1) * KC;
+        if (complete) {
             uint64_t r = (uint64_t)rg * 16 + (o & 15);
             if (r < k.rows) k.y[(uint64_t)(o >> 4) * k.rows + r] = sum;
+        } else {
+            // slot 0 holds the part of the CTA's first row group, slot 1 the part of its last one
+            uint32_t slot = (uint32_t)rg == first_rg ? 0u : 1u;
+            k.ws_partial[((size_t)blockIdx.x * 2 + slot) * vals + o] = sum;
+            if (o == 0) s_split_rg[slot] = rg;
+            __threadfence();
         }
     }
     __syncthreads();
-    // leave the scratch as it was found: all zero
-    for (uint32_t e = tid; e < n_ent; e += blockDim.x) k.ws_rg[e] = 0;
-    if (tid == 0) *k.ws_ticket = 0;
+
+    // ---- combine across CTAs.  A row group cut by CTA boundaries has one arrival counter (indexed by the
+    // first CTA that holds a piece of it); whoever arrives last adds the pieces in CTA order, so the sum
+    // does not depend on timing.  Nobody waits for anybody.
+    STAMP(6);
+    auto cta_of_chunk = [&](uint32_t ch) -> uint32_t {
+        uint32_t c = (uint32_t)((uint64_t)ch * G / T);
+        while (c + 1 < G && (uint32_t)((uint64_t)T * (c + 1) / G) <= ch) ++c;
+        while (c > 0 && (uint32_t)((uint64_t)T * c / G) > ch) --c;
+        return c;
+    };
+    if (tid < 2) {
+        int rg = s_split_rg[tid];
+        uint32_t info = 0;
+        if (rg >= 0) {
+            uint32_t c0 = cta_of_chunk((uint32_t)rg * k.col_chunks), c1 = cta_of_chunk((uint32_t)(rg + 1) * k.col_chunks - 1);
+            uint32_t old = atomicAdd(k.ws_ticket + c0, 1u);
+            if (old == c1 - c0) {          // every other holder has already published its piece
+                __threadfence();
+                k.ws_ticket[c0] = 0;       // leave the counter as it was found
+                info = 0x80000000u | (c0 << 12) | (c1 - c0);
+            }
+        }
+        s_split_info[tid] = info;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int sl = 0; sl < 2; ++sl) {
+        const uint32_t info = s_split_info[sl];
+        if (!(info & 0x80000000u) || tid >= vals) continue;
+        const int rg = s_split_rg[sl];
+        const uint32_t c0 = (info >> 12) & 0x7FFFFu, n = (info & 0xFFFu) + 1;
+        float sum = 0.f;
+        for (uint32_t q = 0; q < n; ++q) {
+            uint32_t c = c0 + q;
+            uint32_t slot = (uint32_t)((uint64_t)T * c / G) / k.col_chunks == (uint32_t)rg ? 0u : 1u;
+            sum += __ldcg(k.ws_partial + ((size_t)c * 2 + slot) * vals + tid);
+        }
+        uint64_t r = (uint64_t)rg * 16 + (tid & 15);
+        if (r < k.rows) k.y[(uint64_t)(tid >> 4) * k.rows + r] = sum;
+    }
+    STAMP(7);
 }
 
 // ------------------------------------------------------------------------------ plain bf16 GEMV
@@ -482,9 +559,9 @@ __global__ void __launch_bounds__(256) plain_gemv_kernel(const uint16_t *__restr
 
 // ------------------------------------------------------------------------------ launchers
 
-template <int MODE, int R>
+template <int MODE, int LB, int THREADS>
 static cudaError_t launch_one(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
-    auto fn = huff_kernel<MODE, R>;
+    auto fn = huff_kernel<MODE, LB, THREADS>;
     static bool attr_set[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
@@ -493,16 +570,16 @@ static cudaError_t launch_one(const KernelArgs &k, uint32_t grid, cudaStream_t s
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    fn<<<grid, 1024, k.dyn_smem_bytes, stream>>>(k);
+    fn<<<grid, THREADS, k.dyn_smem_bytes, stream>>>(k);
     return cudaGetLastError();
 }
 
 cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
-    return k.lut_bits == 8 ? launch_one<0, 3>(k, grid, stream) : launch_one<0, 2>(k, grid, stream);
+    return k.lut_bits == 8 ? launch_one<0, 8, kThreads>(k, grid, stream) : launch_one<0, 9, kThreads>(k, grid, stream);
 }
 
 cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
-    return k.lut_bits == 8 ? launch_one<1, 3>(k, grid, stream) : launch_one<1, 2>(k, grid, stream);
+    return k.lut_bits == 8 ? launch_one<1, 8, kThreads>(k, grid, stream) : launch_one<1, 9, kThreads>(k, grid, stream);
 }
 
 cudaError_t launch_plain_gemv(const uint16_t *w, uint64_t rows, uint64_t cols, const uint16_t *x, float *y, uint32_t sms,

@@ -11,7 +11,7 @@ struct KernelArgs {
     uint32_t payload_units;    // payload size in 128-byte units
     uint64_t rows, cols, n_chunks;
     uint32_t chunk_cols, col_chunks, lut_bits;
-    uint32_t slot_bytes;       // shared-memory bytes of one slot: (max_words + 1) * 128
+    uint32_t slot_bytes;       // shared-memory bytes of one slot: (max_words + 1) * 256
     uint32_t guard_bytes;      // readable bytes kept free behind the last slot
     uint32_t part_bytes;       // bytes at the end of dynamic shared memory for the CTA's partial sums
     uint32_t dyn_smem_bytes;
@@ -19,8 +19,7 @@ struct KernelArgs {
     float *y;                  // [batch][rows]
     uint32_t batch;            // 1..8
     float *ws_partial;         // [grid * 2][16 * batch]
-    int *ws_rg;                // [grid * 2]
-    unsigned int *ws_ticket;
+    unsigned int *ws_ticket;   // [grid] arrival counters, zero between calls
     uint16_t *out;             // decode output
     int32_t *err;              // may be null
 };

@@ -62,7 +62,7 @@ def gpu_gemm(hl, torch, up, x):
         hl.decode_gemm(up.desc, up.blob_dev, x_dev, batch, y, up.ws, up.ws_bytes, up.err)
     torch.cuda.synchronize()
     assert int(up.err.item()) == 0
-    assert int(up.ws[:256].count_nonzero().item()) == 0, "the scratch control words must be left zero"
+    assert int(up.ws[:4096].count_nonzero().item()) == 0, "the scratch control words must be left zero"
     res = y.cpu().numpy()
     assert np.all(np.isnan(res[batch * rows:]))
     return res[:batch * rows].reshape(batch, rows)

@@ -75,15 +75,16 @@ def test_blob_decodes_with_oracle_and_bits_match(rows, cols, ce, budget, gen):
     assert d.pad_word == orc.pad_word(lens)
     for chunk_ids, idx in orc.element_map(rows, cols, ce):
         n, _, steps = idx.shape
-        bits, off, raw = orc.encode_sequences(flat[idx.reshape(n * 32, steps)], lens, codes)
+        S = orc.SEQS
+        bits, off, raw = orc.encode_sequences(flat[idx.reshape(n * S, steps)], lens, codes)
         for a, cid in enumerate(chunk_ids):
             pbits, poff, praw = parsed["chunks"][int(cid)]
-            per = pbits.reshape(32, -1)
-            for l in range(32):
-                lo, hi = int(off[a * 32 + l]), int(off[a * 32 + l + 1])
+            per = pbits.reshape(S, -1)
+            for l in range(S):
+                lo, hi = int(off[a * S + l]), int(off[a * S + l + 1])
                 assert int(used[int(cid)][l]) == hi - lo
                 assert np.array_equal(per[l, :hi - lo], bits[lo:hi])
-            assert np.array_equal(praw, raw[a * 32:a * 32 + 32])
+            assert np.array_equal(praw, raw[a * S:a * S + S])
     # the LUT is what a bit-serial decode of every index gives
     assert np.array_equal(parsed["lut"], orc.lut_from_code(lens, codes, d.lut_bits))
     # accounting

@@ -227,8 +227,8 @@ def test_element_map_is_a_bijection(rows, cols, ce):
     for chunk_ids, idx in orc.element_map(rows, cols, ce):
         n_chunks += len(chunk_ids)
         np.add.at(seen, idx[idx >= 0], 1)
-        # a lane's 8 consecutive steps are 8 consecutive columns of one row
-        a = idx[0].reshape(32, -1, 2, 8)
+        # a sequence's 8 steps of one block are 8 consecutive columns of one row
+        a = idx[0].reshape(orc.SEQS, -1, 8)
         ok = a[..., 0] >= 0
         full = ok & (a[..., 7] >= 0)
         assert np.all((a[..., 7] - a[..., 0])[full] == 7)
