@@ -193,6 +193,30 @@ huffllm_status huffllm_decode_gemm_host(const huffllm_desc *desc, const void *bl
                                         huffllm_stream stream);
 
 /*
+ * (No counterpart in the paper: an engineering addition for callers that cannot allocate.)
+ *
+ * huffllm_decode_gemm for callers that have no device scratch buffer to hand over and no way to get
+ * one: code that runs inside a host application which has already claimed all of the GPU's memory
+ * for its own pools (a serving engine that reserved HBM for its KV cache, a plug-in that must not
+ * call cudaMalloc), or a latency-critical loop where an allocation, which synchronises the whole
+ * device, is not acceptable.  The call allocates nothing: its scratch is a fixed array inside the
+ * library's device image, HUFFLLM_STATIC_SCRATCH_BYTES long, which every GPU that loads the library
+ * holds until the process exits.
+ *
+ * Inputs and outputs are the caller's, exactly as in huffllm_decode_gemm; batch may be at most
+ * HUFFLLM_STATIC_MAX_BATCH — a larger batch is refused with HUFFLLM_ERR_BUFFER_TOO_SMALL and nothing
+ * is launched.  The first call on each device looks up the array's device address (with that device
+ * current) and remembers it; make that first call outside any stream capture.  Every call clears
+ * the scratch's control words on `stream` before the kernel runs, so a call never depends on what an
+ * earlier call left behind.  All calls on one GPU share the one array: two calls that can overlap on
+ * the GPU (different streams without an ordering between them) race on it and give wrong sums.
+ */
+#define HUFFLLM_STATIC_MAX_BATCH 8u
+#define HUFFLLM_STATIC_SCRATCH_BYTES (4096u + 512u * 2u * 16u * HUFFLLM_STATIC_MAX_BATCH * 4u)
+huffllm_status huffllm_decode_gemm_static(const huffllm_desc *desc, const void *blob_dev, const uint16_t *x_dev,
+                                          uint32_t batch, float *y_dev, int32_t *err_flag_dev, huffllm_stream stream);
+
+/*
  * Reference point for the compressed path: y = W x for an UNCOMPRESSED bf16 matrix (device,
  * row-major, 16-byte aligned rows, cols a multiple of 8), same fp32 accumulation.  This is the
  * dense product whose memory traffic the compression removes (Section 6).

@@ -48,6 +48,7 @@ _SIGNATURES = {
     "huffllm_decode_gemm": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemm_host": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
                                  C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
+    "huffllm_decode_gemm_static": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p],
     "huffllm_plain_gemv": [C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p],
     "huffllm_last_error": [],
 }
@@ -186,6 +187,15 @@ def decode_gemm_host(desc: Desc, blob_dev, x_host, batch: int, y_host, x_stage_d
     _check(lib().huffllm_decode_gemm_host(C.byref(desc), _ptr(blob_dev), _ptr(x_host), batch, _ptr(y_host),
                                           _ptr(x_stage_dev), _ptr(y_stage_dev), _ptr(workspace_dev), workspace_bytes_,
                                           _ptr(err_flag_dev), _stream(stream)))
+
+
+STATIC_MAX_BATCH = 8
+
+
+def decode_gemm_static(desc: Desc, blob_dev, x_dev, batch: int, y_dev, err_flag_dev=None, stream=None):
+    """huffllm_decode_gemm_static: the product with the library's built-in scratch (no workspace argument)."""
+    _check(lib().huffllm_decode_gemm_static(C.byref(desc), _ptr(blob_dev), _ptr(x_dev), batch, _ptr(y_dev),
+                                            _ptr(err_flag_dev), _stream(stream)))
 
 
 def plain_gemv(w_dev, rows: int, cols: int, x_dev, y_dev, stream=None):

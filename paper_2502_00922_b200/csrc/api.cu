@@ -163,6 +163,39 @@ huffllm_status huffllm_decode_gemm_host(const huffllm_desc *desc, const void *bl
     return HUFFLLM_OK;
 }
 
+}  // extern "C"
+
+// Scratch of huffllm_decode_gemm_static.  In host code this name is only a handle for the runtime, not a
+// device address: the address the kernels get comes from cudaGetSymbolAddress, once per device.
+static __device__ __align__(256) unsigned char g_static_scratch[HUFFLLM_STATIC_SCRATCH_BYTES];
+static void *g_static_scratch_addr[64] = {};
+
+extern "C" {
+
+huffllm_status huffllm_decode_gemm_static(const huffllm_desc *desc, const void *blob, const uint16_t *x, uint32_t batch,
+                                          float *y, int32_t *err_flag, huffllm_stream stream) {
+    clear_error();
+    if (batch == 0) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be at least 1");
+    if (batch > HUFFLLM_STATIC_MAX_BATCH || ws_bytes_for(batch) > sizeof(g_static_scratch))
+        return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "batch %u needs more than the %u-byte built-in scratch (at most %u vectors)",
+                    batch, (unsigned)HUFFLLM_STATIC_SCRATCH_BYTES, (unsigned)HUFFLLM_STATIC_MAX_BATCH);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
+    if (dev < 0 || dev >= 64) return fail(HUFFLLM_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
+    if (!g_static_scratch_addr[dev]) {   // set-up, once per device, with that device current
+        void *p = nullptr;
+        e = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (e != cudaSuccess || !p) return fail(HUFFLLM_ERR_CUDA, "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+        g_static_scratch_addr[dev] = p;
+    }
+    void *ws = g_static_scratch_addr[dev];
+    // the array keeps whatever the last call (finished or not) left: the control words must start at zero
+    e = cudaMemsetAsync(ws, 0, 4096, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "clearing the built-in scratch: %s", cudaGetErrorString(e));
+    return huffllm_decode_gemm(desc, blob, x, batch, y, ws, sizeof(g_static_scratch), err_flag, stream);
+}
+
 huffllm_status huffllm_plain_gemv(const uint16_t *w, uint64_t rows, uint64_t cols, const uint16_t *x, float *y, huffllm_stream stream) {
     clear_error();
     DeviceInfo *dev;
