@@ -167,7 +167,8 @@ huffllm_status huffllm_decode(const huffllm_desc *desc, const void *blob_dev, ui
  * y = W x with W taken straight from the compressed blob: weights are decoded in registers and
  * multiplied at once, so only compressed bytes cross the memory bus (Section 1: weights are
  * decompressed only when needed, to multiply with activations).  x: device, cols words of the
- * blob's dtype.  y: device, rows floats.  Products are exact, sums are accumulated in fp32.
+ * blob's dtype.  y: device, rows floats.  cols must be a multiple of 32 (UNSUPPORTED otherwise;
+ * huffllm_decode takes any shape).  Products are exact, sums are accumulated in fp32.
  * Results are bitwise reproducible from run to run.
  */
 huffllm_status huffllm_decode_gemv(const huffllm_desc *desc, const void *blob_dev, const uint16_t *x_dev, float *y_dev,

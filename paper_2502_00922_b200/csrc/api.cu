@@ -123,9 +123,7 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
     if (workspace_bytes < ws_bytes_for(batch)) return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "workspace too small");
     st = check_desc(desc);
     if (st != HUFFLLM_OK) return st;
-    if (desc->cols % 8) return fail(HUFFLLM_ERR_UNSUPPORTED, "fused products need cols to be a multiple of 8");
-    if (desc->cols % kBlockCols && ((desc->pad_word >> 7) & 0xFF) == 0xFF)
-        return fail(HUFFLLM_ERR_UNSUPPORTED, "pad weights are not finite for this tensor");
+    if (desc->cols % kBlockCols) return fail(HUFFLLM_ERR_UNSUPPORTED, "fused products need cols to be a multiple of 32");
     for (uint32_t b0 = 0; b0 < batch; b0 += kKernelBatch) {
         uint32_t nb = batch - b0 < kKernelBatch ? batch - b0 : kKernelBatch;
         KernelArgs k;

@@ -88,6 +88,16 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// Arrival counter bump that publishes this warp's earlier stores and acquires the other arrivals' stores.
+__device__ __forceinline__ uint32_t arrive_acq_rel(unsigned int *counter) {
+    uint32_t old;
+    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(counter) : "memory");
+    return old;
+}
+// Programmatic dependent launch: let the next kernel in the stream be scheduled early / wait for the previous one.
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait_prior_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // ------------------------------------------------------------------------------ lane decoder
 
 // State of the decoder of one bit sequence.  (hi:lo) holds 64 stream bits; the current codeword starts
@@ -141,7 +151,9 @@ __device__ __forceinline__ uint32_t pack_pair(uint32_t e_even, uint32_t e_odd, u
     uint32_t sm = prmt(raw, 0u, SEL);   // [sign1*0xFF, raw1, sign0*0xFF, raw0]
     uint32_t ex;
     asm("mad.lo.u32 %0, %1, 65536, %2;" : "=r"(ex) : "r"(e_odd), "r"(e_even));
-    return (sm & 0x807F807Fu) | (ex & 0x7F807F80u);
+    uint32_t w;   // sign and mantissa bits from sm, exponent bits from ex
+    asm("lop3.b32 %0, %1, %2, 0x807F807F, 0xE4;" : "=r"(w) : "r"(sm), "r"(ex));
+    return w;
 }
 
 // Decode one block (16 weights of this lane) into 8 packed registers:
@@ -232,13 +244,11 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const KernelArgs k) {
     constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
     extern __shared__ __align__(128) uint8_t dyn_smem[];
     __shared__ __align__(8) uint64_t bars[kMaxWarps * 2];
-    __shared__ int part_rg[kMaxWarps * 2];
-    __shared__ int s_split_rg[2];        // row groups of this CTA that other CTAs also hold pieces of
-    __shared__ uint32_t s_split_info[2];
-    __shared__ uint32_t s_grp_first[kMaxWarps * 2 + 1], s_ngroups;
+    __shared__ uint32_t s_arrive[kMaxWarps];   // arrival counters of row groups shared by several warps
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps_launched = blockDim.x >> 5;
     STAMP(0);
+    pdl_launch_dependents();   // the next kernel's set-up may overlap this kernel's tail
     const uint32_t smem_base = smem_u32(dyn_smem);
     const SmemPlan plan = plan_smem(smem_base, k, nwarps_launched);
     const uint32_t nw = plan.warps;
@@ -286,8 +296,19 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const KernelArgs k) {
         }
     };
 
-    // ---- set-up.  Every warp arms its own two barriers and starts its first copies at once, so the
-    // first compressed bytes are already on their way while the CTA builds the per-lane table.
+    // ---- set-up.  The table loads are started first, then every warp arms its own two barriers and starts
+    // its first copies, then the table is written to shared memory: the cold misses on the table, on the
+    // record index and on the first records overlap instead of following each other.
+    constexpr int kLutLoads = ((32 << LB) + THREADS - 1) / THREADS;
+    uint32_t lut_v[kLutLoads];
+    {
+        const uint32_t *lut_g = (const uint32_t *)(k.blob + k.off_lut);
+#pragma unroll
+        for (int i = 0; i < kLutLoads; ++i) {
+            uint32_t j = tid + i * THREADS;
+            lut_v[i] = j < (32u << LB) ? __ldg(lut_g + (j >> 5)) : 0u;
+        }
+    }
     if (lane == 0) {
         mbar_init(bar0, 1);
         mbar_init(bar0 + 8, 1);
@@ -298,11 +319,13 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const KernelArgs k) {
         }
     }
     {
-        const uint32_t *lut_g = (const uint32_t *)(k.blob + k.off_lut);
         uint32_t *lut_s = (uint32_t *)(dyn_smem + (plan.lut - smem_base));
-        for (uint32_t i = tid; i < (32u << LB); i += THREADS) lut_s[i] = __ldg(lut_g + (i >> 5));
-        if (tid < kMaxWarps * 2) part_rg[tid] = -1;
-        if (tid < 2) s_split_rg[tid] = -1;
+#pragma unroll
+        for (int i = 0; i < kLutLoads; ++i) {
+            uint32_t j = tid + i * THREADS;
+            if (j < (32u << LB)) lut_s[j] = lut_v[i];
+        }
+        if (tid < kMaxWarps) s_arrive[tid] = 0;
     }
     STAMP(1);
     __syncthreads();
@@ -310,29 +333,107 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const KernelArgs k) {
 
     float acc[4] = {0.f, 0.f, 0.f, 0.f};
     int cur_rg = -1;
-    uint32_t n_partial = 0;
 
-    // hand a finished row group to y (if this warp saw all of its chunks) or to the CTA's partial table
+    // ---- reduction of a finished row group, without any CTA-wide barrier.
+    // A row group whose chunks this warp decoded alone goes straight to y.  Otherwise the warp parks its
+    // piece in shared memory and bumps an arrival counter (indexed by the first warp that holds a piece);
+    // the warp that arrives last adds the pieces in warp order.  If other CTAs hold pieces too, the CTA's
+    // sum goes to the scratch buffer and the same game is played across CTAs with a counter in global
+    // memory.  Sums are always taken in the same order, and nobody waits for anybody.
+    const uint32_t G = gridDim.x;
+    const uint32_t cta_len = cta_end - cta_beg;
+    auto warp_beg = [&](uint32_t w) -> uint32_t { return cta_beg + cta_len * w / nw; };
+    auto cta_of_chunk = [&](uint32_t ch) -> uint32_t {
+        uint32_t c = (uint32_t)((uint64_t)ch * G / T);
+        while (c + 1 < G && (uint32_t)((uint64_t)T * (c + 1) / G) <= ch) ++c;
+        while (c > 0 && (uint32_t)((uint64_t)T * c / G) > ch) --c;
+        return c;
+    };
+    // lanes 0..vals-1 (looping if vals > 32) hold or produce the value of output o = column * 16 + row
+    auto finish_cta_sum = [&](int rg, float (&v)[4]) {       // v[i] = value of output o = lane + 32 i
+        const uint32_t g_lo = (uint32_t)rg * KC, g_hi = g_lo + KC;
+        if (cta_beg <= g_lo && cta_end >= g_hi) {             // the CTA held the whole row group
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                uint32_t o = lane + 32 * i;
+                uint64_t r = (uint64_t)rg * 16 + (o & 15);
+                if (o < vals && r < k.rows) k.y[(uint64_t)(o >> 4) * k.rows + r] = v[i];
+            }
+            return;
+        }
+        // slot 0 holds the piece of the CTA's first row group, slot 1 the piece of its last one
+        const uint32_t my_slot = (uint32_t)rg == cta_beg / KC ? 0u : 1u;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint32_t o = lane + 32 * i;
+            if (o < vals) k.ws_partial[((size_t)blockIdx.x * 2 + my_slot) * vals + o] = v[i];
+        }
+        __syncwarp();
+        const uint32_t c0 = cta_of_chunk(g_lo), c1 = cta_of_chunk(g_hi - 1);
+        uint32_t last = 0;
+        if (lane == 0) {
+            last = arrive_acq_rel(k.ws_ticket + c0) == c1 - c0 ? 1u : 0u;
+            if (last) k.ws_ticket[c0] = 0;                    // leave the counter as it was found
+        }
+        if (!__shfl_sync(0xFFFFFFFFu, last, 0)) return;       // somebody else will arrive later and add us in
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint32_t o = lane + 32 * i;
+            if (o >= vals) continue;
+            float sum = 0.f;
+            for (uint32_t c = c0; c <= c1; ++c) {
+                uint32_t slot = (uint32_t)((uint64_t)T * c / G) / KC == (uint32_t)rg ? 0u : 1u;
+                sum += __ldcg(k.ws_partial + ((size_t)c * 2 + slot) * vals + o);
+            }
+            uint64_t r = (uint64_t)rg * 16 + (o & 15);
+            if (r < k.rows) k.y[(uint64_t)(o >> 4) * k.rows + r] = sum;
+        }
+    };
     auto flush = [&](int rg, uint32_t first_c, uint32_t last_c_excl) {
         if (rg < 0) return;
-        bool complete = first_c <= (uint32_t)rg * KC && last_c_excl >= (uint32_t)(rg + 1) * KC;
-        uint32_t ent = warp * 2 + min(n_partial, 1u);
+        const uint32_t g_lo = max((uint32_t)rg * KC, cta_beg), g_hi = min((uint32_t)(rg + 1) * KC, cta_end);  // this CTA's part
+        const bool alone = first_c <= g_lo && last_c_excl >= g_hi;   // no other warp of this CTA holds a piece
+        // D fragment -> output order (o = column * 16 + row) through this warp's shared-memory entry
+        const uint32_t ent = warp * 2 + ((uint32_t)rg == c_beg / KC ? 0u : 1u);
+        float *mine = part_val + (size_t)ent * vals;
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
             uint32_t col = 2 * t + (j & 1), row = g + 8 * (j >> 1);
-            if (col >= k.batch) continue;
-            if (complete) {
-                uint64_t r = (uint64_t)rg * 16 + row;
-                if (r < k.rows) k.y[(uint64_t)col * k.rows + r] = acc[j];
-            } else {
-                part_val[(size_t)ent * vals + col * 16 + row] = acc[j];
-            }
-        }
-        if (!complete) {
-            if (lane == 0) part_rg[ent] = (int)rg;
-            ++n_partial;
+            if (col < k.batch) mine[col * 16 + row] = acc[j];
         }
         acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+        __syncwarp();
+        float v[4];
+        if (alone) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) v[i] = lane + 32 * i < vals ? mine[lane + 32 * i] : 0.f;
+            __syncwarp();
+            finish_cta_sum(rg, v);
+            return;
+        }
+        // which warps of this CTA hold a piece of this row group (lane l answers for warp l)
+        const uint32_t wb = warp_beg(lane), we = warp_beg(lane + 1);
+        const bool holds = lane < nw && wb < we && wb < g_hi && we > g_lo;
+        const uint32_t mask = __ballot_sync(0xFFFFFFFFu, holds);
+        const uint32_t w_first = __ffs(mask) - 1, n_hold = __popc(mask);
+        const uint32_t slot_of_lane = (uint32_t)rg == wb / KC ? 0u : 1u;
+        uint32_t last = 0;
+        if (lane == 0) {
+            __threadfence_block();
+            last = atomicAdd(&s_arrive[w_first], 1u) == n_hold - 1 ? 1u : 0u;
+            if (last) __threadfence_block();
+        }
+        if (!__shfl_sync(0xFFFFFFFFu, last, 0)) return;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v[i] = 0.f;
+        for (uint32_t m = mask; m; m &= m - 1) {              // pieces in warp order
+            const uint32_t w = __ffs(m) - 1;
+            const float *piece = part_val + (size_t)(w * 2 + __shfl_sync(0xFFFFFFFFu, slot_of_lane, w)) * vals;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (lane + 32 * i < vals) v[i] += piece[lane + 32 * i];
+        }
+        finish_cta_sum(rg, v);
     };
 
     if (c_beg < c_end) {
@@ -342,6 +443,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const KernelArgs k) {
         uint4 raw_a = make_uint4(0, 0, 0, 0), raw_b = make_uint4(0, 0, 0, 0);
         bool primed = false, failed = false;
 
+#pragma unroll 1
         for (uint32_t c = c_beg; c < c_end; ++c) {
             const uint32_t which = (c - c_beg) & 1u, parity = ((c - c_beg) >> 1) & 1u;
             const uint32_t nkb = blocks_of(kc);
@@ -377,7 +479,10 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const KernelArgs k) {
                 }
             }
 
-            if (c == c_beg) STAMP(3);
+            if (c == c_beg) {
+                STAMP(3);
+                pdl_wait_prior_grid();   // from here on this warp reads x and writes results: the previous kernel must be done
+            }
             if (!ok) {  // record offsets out of range: report, produce nothing for this chunk, touch no memory
                 if (k.err && lane == 0) atomicExch(k.err, (int32_t)min(c + 1, 0x7FFFFFFFu));
                 primed = false;
@@ -386,18 +491,22 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const KernelArgs k) {
                 stream_open(sa, slot0 + which * k.slot_bytes + (lane << 2));
                 stream_open(sb, slot0 + which * k.slot_bytes + 128u + (lane << 2));
                 const uint32_t col0 = kc * k.chunk_cols + t * 8u;
-                // activations: lanes of unused output columns repeat the last vector; nx = blocks with a column in range
-                const uint16_t *xp = k.x + (MODE == 1 ? (uint64_t)min(g, k.batch - 1) * k.cols + col0 : 0);
-                const uint32_t nx = (MODE == 1 && col0 < (uint32_t)k.cols) ? min(nkb, ((uint32_t)k.cols - col0 + 31u) >> 5) : 0u;
+                // activations: lanes of unused output columns repeat the last vector (cols is a multiple of 32 here,
+                // so every block of the chunk lies inside the row)
+                const uint16_t *xq = k.x + (MODE == 1 ? (uint64_t)min(g, k.batch - 1) * k.cols + col0 : 0);
                 uint16_t *out0 = MODE == 0 ? k.out + ((uint64_t)rg * 16 + g) * k.cols + col0 : nullptr;
+                const uint32_t last = nkb - 1;
 
                 // one block: start the fetch of the next block's raw bytes into `nxt`, decode with `cur`
                 auto block = [&](uint32_t kb, const uint4 &cur, uint4 &nxt) {
                     raw_p += 512;
-                    if (kb + 1 < nkb) nxt = ldg_stream16(raw_p);
-                    else if (next_ok) nxt = ldg_stream16(raw_p + coded_bytes);
-                    uint4 xv = make_uint4(0, 0, 0, 0);
-                    if (MODE == 1 && kb < nx) xv = __ldg((const uint4 *)(xp + kb * 32u));
+                    if (kb == last) raw_p += coded_bytes;           // the next record's first block
+                    if (kb != last || next_ok) nxt = ldg_stream16(raw_p);
+                    uint4 xv;
+                    if (MODE == 1) {
+                        xv = __ldg((const uint4 *)xq);
+                        xq += 32;
+                    }
 
                     uint32_t a[8];
                     decode_block<R>(sa, sb, kIdxMask, lut_lane, cur, a);
@@ -421,6 +530,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const KernelArgs k) {
                         }
                     }
                 };
+#pragma unroll 1
                 for (uint32_t kb = 0; kb < nkb; kb += 2) {
                     block(kb, raw_a, raw_b);
                     if (kb + 1 < nkb) block(kb + 1, raw_b, raw_a);
@@ -439,93 +549,6 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const KernelArgs k) {
     }
 
     STAMP(4);
-    if (MODE != 1) return;
-
-    // ---- combine inside the CTA, in warp order.  Entries (warp, slot) are ordered by chunk, so the pieces
-    // of one row group are neighbours; warp 0 finds the group boundaries with ballots, then each group is
-    // summed by its own set of threads, pieces taken in entry order.
-    __syncthreads();
-    STAMP(5);
-    const uint32_t G = gridDim.x;
-    const uint32_t first_rg = cta_beg / KC;   // row group of this CTA's first chunk
-    if (warp == 0) {
-        const int t0 = part_rg[lane], t1 = part_rg[lane + 32];
-        const uint32_t v0 = __ballot_sync(0xFFFFFFFFu, t0 >= 0), v1 = __ballot_sync(0xFFFFFFFFu, t1 >= 0);
-        const uint32_t lt = (1u << lane) - 1u, le = lt | (1u << lane);
-        // tag of the nearest valid entry in front of each of this lane's two entries
-        const int p0 = (v0 & lt) ? 31 - __clz(v0 & lt) : 0, p1 = (v1 & lt) ? 31 - __clz(v1 & lt) : 0, pl = v0 ? 31 - __clz(v0) : 0;
-        const int q0 = __shfl_sync(0xFFFFFFFFu, t0, p0), q1 = __shfl_sync(0xFFFFFFFFu, t1, p1), ql = __shfl_sync(0xFFFFFFFFu, t0, pl);
-        const bool s0 = t0 >= 0 && (!(v0 & lt) || q0 != t0);
-        const bool s1 = t1 >= 0 && ((v1 & lt) ? q1 != t1 : (!v0 || ql != t1));
-        const uint32_t b0 = __ballot_sync(0xFFFFFFFFu, s0), b1 = __ballot_sync(0xFFFFFFFFu, s1);
-        if (s0) { s_grp_first[__popc(b0 & le) - 1] = lane; }
-        if (s1) { s_grp_first[__popc(b0) + __popc(b1 & le) - 1] = lane + 32; }
-        if (lane == 0) {
-            s_ngroups = __popc(b0) + __popc(b1);
-            s_grp_first[__popc(b0) + __popc(b1)] = 64;
-        }
-    }
-    __syncthreads();
-    for (uint32_t gi = tid / vals; gi < s_ngroups; gi += blockDim.x / vals) {
-        const uint32_t o = tid % vals, e0 = s_grp_first[gi], e1 = s_grp_first[gi + 1];
-        const int rg = part_rg[e0];
-        float sum = 0.f;
-        for (uint32_t e = e0; e < e1; ++e)
-            if (part_rg[e] == rg) sum += part_val[(size_t)e * vals + o];
-        const bool complete = cta_beg <= (uint32_t)rg * KC && cta_end >= (uint32_t)(rg + 1) * KC;
-        if (complete) {
-            uint64_t r = (uint64_t)rg * 16 + (o & 15);
-            if (r < k.rows) k.y[(uint64_t)(o >> 4) * k.rows + r] = sum;
-        } else {
-            // slot 0 holds the part of the CTA's first row group, slot 1 the part of its last one
-            uint32_t slot = (uint32_t)rg == first_rg ? 0u : 1u;
-            k.ws_partial[((size_t)blockIdx.x * 2 + slot) * vals + o] = sum;
-            if (o == 0) s_split_rg[slot] = rg;
-            __threadfence();
-        }
-    }
-    __syncthreads();
-
-    // ---- combine across CTAs.  A row group cut by CTA boundaries has one arrival counter (indexed by the
-    // first CTA that holds a piece of it); whoever arrives last adds the pieces in CTA order, so the sum
-    // does not depend on timing.  Nobody waits for anybody.
-    STAMP(6);
-    auto cta_of_chunk = [&](uint32_t ch) -> uint32_t {
-        uint32_t c = (uint32_t)((uint64_t)ch * G / T);
-        while (c + 1 < G && (uint32_t)((uint64_t)T * (c + 1) / G) <= ch) ++c;
-        while (c > 0 && (uint32_t)((uint64_t)T * c / G) > ch) --c;
-        return c;
-    };
-    if (tid < 2) {
-        int rg = s_split_rg[tid];
-        uint32_t info = 0;
-        if (rg >= 0) {
-            uint32_t c0 = cta_of_chunk((uint32_t)rg * k.col_chunks), c1 = cta_of_chunk((uint32_t)(rg + 1) * k.col_chunks - 1);
-            uint32_t old = atomicAdd(k.ws_ticket + c0, 1u);
-            if (old == c1 - c0) {          // every other holder has already published its piece
-                __threadfence();
-                k.ws_ticket[c0] = 0;       // leave the counter as it was found
-                info = 0x80000000u | (c0 << 12) | (c1 - c0);
-            }
-        }
-        s_split_info[tid] = info;
-    }
-    __syncthreads();
-#pragma unroll
-    for (int sl = 0; sl < 2; ++sl) {
-        const uint32_t info = s_split_info[sl];
-        if (!(info & 0x80000000u) || tid >= vals) continue;
-        const int rg = s_split_rg[sl];
-        const uint32_t c0 = (info >> 12) & 0x7FFFFu, n = (info & 0xFFFu) + 1;
-        float sum = 0.f;
-        for (uint32_t q = 0; q < n; ++q) {
-            uint32_t c = c0 + q;
-            uint32_t slot = (uint32_t)((uint64_t)T * c / G) / k.col_chunks == (uint32_t)rg ? 0u : 1u;
-            sum += __ldcg(k.ws_partial + ((size_t)c * 2 + slot) * vals + tid);
-        }
-        uint64_t r = (uint64_t)rg * 16 + (tid & 15);
-        if (r < k.rows) k.y[(uint64_t)(tid >> 4) * k.rows + r] = sum;
-    }
     STAMP(7);
 }
 
@@ -570,8 +593,17 @@ static cudaError_t launch_one(const KernelArgs &k, uint32_t grid, cudaStream_t s
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    fn<<<grid, THREADS, k.dyn_smem_bytes, stream>>>(k);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(THREADS);
+    cfg.dynamicSmemBytes = k.dyn_smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // set-up overlaps the previous kernel's tail
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fn, k);
 }
 
 cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {

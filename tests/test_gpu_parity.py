@@ -115,7 +115,7 @@ GEMM_CASES = [
     (1024, 1024, 4096, 0, "gauss", 1),
     (16, 256, 4096, 0, "gauss", 1),
     (48, 1056, 4096, 0, "gauss", 1),
-    (40, 2056, 1024, 0, "student", 3),            # ragged rows, cols a multiple of 8 only
+    (40, 2080, 1024, 0, "student", 3),            # ragged rows, last column chunk holds a single block
     (16, 65536, 4096, 0, "gauss", 1),             # one row group split over every CTA
     (32, 32768, 4096, 0, "gauss", 8),
     (2368, 512, 512, 0, "gauss", 2),
@@ -201,9 +201,9 @@ def test_bad_record_offsets_are_reported_not_followed(hl, torch):
 
 
 def test_unsupported_requests_fail_before_launch(hl, torch):
-    w = wl.gaussian_weights(16, 516, 0.02, 14)     # cols not a multiple of 8
+    w = wl.gaussian_weights(16, 520, 0.02, 14)     # cols not a multiple of 32
     up = Uploaded(hl, torch, w, 512)
-    x = torch.zeros(516, dtype=torch.int16, device="cuda")
+    x = torch.zeros(520, dtype=torch.int16, device="cuda")
     y = torch.zeros(16, dtype=torch.float32, device="cuda")
     with pytest.raises(hl.HuffllmError) as e:
         hl.decode_gemv(up.desc, up.blob_dev, x, y, up.ws, up.ws_bytes, up.err)
