@@ -40,6 +40,18 @@ WORKLOADS = {
     "8b_layer": (wl.LAYER_8B, 0.02, 3000, "8B-shaped decoder layer (GQA k/v 1024x4096, FFN 14336), batch 1"),
     "ffn70b": (wl.FFN_70B, 0.015, 4000, "70B-FFN-shaped pair 28672x8192 / 8192x28672"),
 }
+# Which matrices of a layer table may run in one launch.  "deps": only matrices that a decoder layer can really
+# compute side by side (q,k,v read the same input; so do gate and up); "all": the whole table; "none": one each.
+def launch_groups(table, fuse: str):
+    n = len(table)
+    if fuse == "none" or n == 1:
+        return [[i] for i in range(n)]
+    if fuse == "all":
+        return [list(range(n))]
+    names = [t[0] for t in table]
+    if names[:7] == ["q", "k", "v", "o", "gate", "up", "down"]:
+        return [[0, 1, 2], [3], [4, 5], [6]]
+    return [[i] for i in range(n)]
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one fused-product launch over its algorithmic bytes, from the
 # ncu capture summarised in profiles/ (None until a capture exists); traffic = ratio * algorithmic bytes.
@@ -181,6 +193,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="llama7b_layer", choices=sorted(WORKLOADS))
     ap.add_argument("--chunk-elems", type=int, default=4096)
+    ap.add_argument("--fuse", default="deps", choices=["none", "deps", "all"],
+                    help="which matrices of the layer share a launch")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -208,9 +222,13 @@ def main():
     alg_bytes = sum(m["alg_bytes"] for m in mats)
     stream = torch.cuda.current_stream()
 
+    groups = launch_groups(WORKLOADS[args.workload][0], args.fuse)
+    calls = [dict(descs=[mats[i]["desc"] for i in g], blobs=[mats[i]["blob_dev"] for i in g], xs=[mats[i]["x_dev"] for i in g],
+                  ys=[mats[i]["y_dev"] for i in g], wss=[mats[i]["ws"] for i in g]) for g in groups]
+
     def step_device():
-        for m in mats:
-            hl.decode_gemv(m["desc"], m["blob_dev"], m["x_dev"], m["y_dev"], m["ws"], m["ws_bytes"], err, stream)
+        for c in calls:
+            hl.decode_gemm_multi(c["descs"], c["blobs"], c["xs"], 1, c["ys"], c["wss"], mats[0]["ws_bytes"], err, stream)
 
     def step_host():
         for m in mats:
@@ -327,10 +345,11 @@ def main():
                    "bits_per_param_payload": sum(m["coded_bits"] + m["raw_bits"] for m in mats) / n_weights,
                    "l2": "inputs larger than L2: the step streams %.0f MB of compressed weights, L2 is 126 MB" % (alg_bytes / 1e6),
                    "parallelism": "replicas only" if world > 1 else "single GPU",
+                   "launch_groups": [[mats[i]["name"] for i in g] for g in groups],
                    "tokens_per_s_equiv_one_layer": 1e3 / ms_step},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
-                     "traffic": None if NCU_TRAFFIC_RATIO is None else NCU_TRAFFIC_RATIO * alg_bytes / len(mats),
-                     "peak_source": peak_src, "kernel": "huff_kernel<product>", "launches_per_step": len(mats),
+                     "traffic": None if NCU_TRAFFIC_RATIO is None else NCU_TRAFFIC_RATIO * alg_bytes / len(groups),
+                     "peak_source": peak_src, "kernel": "huff_kernel<product>", "launches_per_step": len(groups), "fuse": args.fuse,
                      "algorithmic_bytes_per_step": alg_bytes, "kernel_ms_per_step": kernel_ms_step,
                      "frac_of_nominal_8TBs": achieved / 8000.0,
                      "per_matrix": [{"name": m["name"], "rows": m["rows"], "cols": m["cols"], "ms": t,
@@ -338,7 +357,7 @@ def main():
         "cpu_baseline": cpu,
         "e2e": {"value": world * unc_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": sum(2 * m["cols"] for m in mats), "d2h_bytes_per_step": sum(4 * m["rows"] for m in mats)},
-        "gpu_launches": len(mats) * args.steps,
+        "gpu_launches": len(groups) * args.steps,
         "clocks": clocks,
         "dense_bf16_gemv": {"own_kernel_ms_per_step": plain_ms, "cublas_mv_ms_per_step": cublas_ms,
                             "own_kernel_GBs": None if not plain_ms else unc_bytes / (plain_ms * 1e-3) / 1e9,

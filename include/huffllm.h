@@ -184,6 +184,19 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob_de
                                    huffllm_stream stream);
 
 /*
+ * Several products in ONE launch: y_i = W_i x_i for i < n (n <= 8, batch <= 8), e.g. the q, k and v
+ * projections of a decoder layer, or gate and up.  The chunks of all matrices are spread over the GPU
+ * together, so small matrices do not pay a launch, a set-up and a tail each.  Arrays are host arrays
+ * of n pointers; every matrix needs its own workspace (each workspace_bytes_each long, as reported by
+ * huffllm_workspace_bytes), its own x_i ([batch][cols_i]) and y_i ([batch][rows_i]).  All blobs must
+ * have been encoded with the same max_code_len.
+ */
+huffllm_status huffllm_decode_gemm_multi(uint32_t n, const huffllm_desc *const *descs, const void *const *blobs_dev,
+                                         const uint16_t *const *xs_dev, uint32_t batch, float *const *ys_dev,
+                                         void *const *workspaces_dev, size_t workspace_bytes_each, int32_t *err_flag_dev,
+                                         huffllm_stream stream);
+
+/*
  * The same product called with HOST activations and a HOST result: copies x to `x_stage_dev`
  * (device, batch*cols words), runs huffllm_decode_gemm, copies y from `y_stage_dev` (device,
  * batch*rows floats) to y_host and waits for the stream.  x_host / y_host should be pinned.

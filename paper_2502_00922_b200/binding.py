@@ -46,6 +46,8 @@ _SIGNATURES = {
     "huffllm_decode": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemv": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemm": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
+    "huffllm_decode_gemm_multi": [C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_size_t,
+                                  C.c_void_p, C.c_void_p],
     "huffllm_decode_gemm_host": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
                                  C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemm_static": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p],
@@ -180,6 +182,16 @@ def decode_gemm(desc: Desc, blob_dev, x_dev, batch: int, y_dev, workspace_dev, w
                 stream=None):
     _check(lib().huffllm_decode_gemm(C.byref(desc), _ptr(blob_dev), _ptr(x_dev), batch, _ptr(y_dev), _ptr(workspace_dev),
                                      workspace_bytes_, _ptr(err_flag_dev), _stream(stream)))
+
+
+def decode_gemm_multi(descs, blobs_dev, xs_dev, batch: int, ys_dev, workspaces_dev, workspace_bytes_each: int,
+                      err_flag_dev=None, stream=None):
+    """huffllm_decode_gemm_multi: lists of equal length, one entry per matrix."""
+    n = len(descs)
+    desc_arr = (C.POINTER(Desc) * n)(*[C.pointer(d) for d in descs])
+    ptrs = lambda seq: (C.c_void_p * n)(*[_ptr(t) for t in seq])
+    _check(lib().huffllm_decode_gemm_multi(n, desc_arr, ptrs(blobs_dev), ptrs(xs_dev), batch, ptrs(ys_dev), ptrs(workspaces_dev),
+                                           workspace_bytes_each, _ptr(err_flag_dev), _stream(stream)))
 
 
 def decode_gemm_host(desc: Desc, blob_dev, x_host, batch: int, y_host, x_stage_dev, y_stage_dev, workspace_dev,

@@ -44,38 +44,55 @@ size_t ws_bytes_for(uint32_t batch) {
     return ws_partial_offset() + (size_t)kMaxGrid * 2 * 16 * b * sizeof(float);
 }
 
-huffllm_status fill_args(const huffllm_desc *desc, const void *blob, uint32_t batch, bool product, const DeviceInfo &dev,
-                         KernelArgs *k, uint32_t *grid) {
+// Start a launch description.
+void begin_args(KernelArgs *k, uint32_t batch, const DeviceInfo &dev) {
+    memset(k, 0, sizeof(*k));
+    k->batch = batch;
+    k->dyn_smem_bytes = (uint32_t)dev.smem_optin - kStaticSmem;
+}
+
+// Append one matrix to a launch description (checks the descriptor and the blob pointer).
+huffllm_status add_matrix(KernelArgs *k, const huffllm_desc *desc, const void *blob) {
     huffllm_status st = check_desc(desc);
     if (st != HUFFLLM_OK) return st;
     if (!blob || ((uintptr_t)blob & 255)) return fail(HUFFLLM_ERR_INVALID_ARG, "blob must be a 256-byte aligned device pointer");
     if (desc->lut_bits > 9)
         return fail(HUFFLLM_ERR_UNSUPPORTED, "device kernels take max_code_len 8 or 9 (this blob: %u)", desc->lut_bits);
-    if (desc->n_chunks >= (1ull << 31)) return fail(HUFFLLM_ERR_UNSUPPORTED, "too many chunks for one launch");
-    memset(k, 0, sizeof(*k));
-    k->blob = (const uint8_t *)blob;
-    k->off_lut = desc->off_lut;
-    k->off_index = desc->off_index;
-    k->off_payload = desc->off_payload;
-    k->payload_units = (uint32_t)(desc->payload_bytes / kRecordUnit);
-    k->rows = desc->rows;
-    k->cols = desc->cols;
-    k->n_chunks = desc->n_chunks;
-    k->chunk_cols = desc->chunk_cols;
-    k->col_chunks = desc->col_chunks;
+    if (k->n_mats == kMaxMats) return fail(HUFFLLM_ERR_UNSUPPORTED, "at most %u matrices per call", kMaxMats);
+    if (k->n_mats && k->lut_bits != desc->lut_bits)
+        return fail(HUFFLLM_ERR_UNSUPPORTED, "matrices of one call must share max_code_len");
+    if (desc->n_chunks + k->total_chunks >= (1ull << 31)) return fail(HUFFLLM_ERR_UNSUPPORTED, "too many chunks for one launch");
+    MatArgs &m = k->m[k->n_mats++];
+    m.blob = (const uint8_t *)blob;
+    m.off_lut = desc->off_lut;
+    m.off_index = desc->off_index;
+    m.off_payload = desc->off_payload;
+    m.payload_units = (uint32_t)(desc->payload_bytes / kRecordUnit);
+    m.rows = desc->rows;
+    m.cols = desc->cols;
+    m.n_chunks = (uint32_t)desc->n_chunks;
+    m.chunk_cols = desc->chunk_cols;
+    m.col_chunks = desc->col_chunks;
+    m.chunk_base = k->total_chunks;
+    k->total_chunks += m.n_chunks;
     k->lut_bits = desc->lut_bits;
-    k->slot_bytes = (desc->max_words + 1) * 256;
+    uint32_t slot = (desc->max_words + 1) * 256;
     // a corrupt stream can advance its read pointer by one row per refill check and no further
     const uint32_t checks_per_block = desc->lut_bits == 8 ? 3 : 4;
-    k->guard_bytes = 256 * (3 + checks_per_block * (desc->chunk_cols / kBlockCols));
-    k->part_bytes = product ? 2 * 32 * 16 * batch * (uint32_t)sizeof(float) : 0;
-    k->dyn_smem_bytes = (uint32_t)dev.smem_optin - kStaticSmem;
-    k->batch = batch;
+    uint32_t guard = 256 * (3 + checks_per_block * (desc->chunk_cols / kBlockCols));
+    if (slot > k->slot_bytes) k->slot_bytes = slot;
+    if (guard > k->guard_bytes) k->guard_bytes = guard;
+    return HUFFLLM_OK;
+}
+
+// Close a launch description: shared-memory budget and grid size.
+huffllm_status finish_args(KernelArgs *k, bool product, const DeviceInfo &dev, uint32_t *grid) {
+    k->part_bytes = product ? 2 * 32 * 16 * k->batch * (uint32_t)sizeof(float) : 0;
     // worst case for the table's alignment gap is covered by assuming the window starts within 4 KB of zero
-    uint64_t fixed = (128ull << desc->lut_bits) + k->guard_bytes + k->part_bytes + 4096;
+    uint64_t fixed = (128ull << k->lut_bits) + k->guard_bytes + k->part_bytes + 4096;
     if (fixed + 2ull * k->slot_bytes > k->dyn_smem_bytes)
-        return fail(HUFFLLM_ERR_UNSUPPORTED, "chunk records too large for shared memory (max_words %u)", desc->max_words);
-    uint64_t g = desc->n_chunks < (uint64_t)dev.sms ? desc->n_chunks : (uint64_t)dev.sms;
+        return fail(HUFFLLM_ERR_UNSUPPORTED, "chunk records too large for shared memory (slot %u bytes)", k->slot_bytes);
+    uint64_t g = k->total_chunks < (uint64_t)dev.sms ? k->total_chunks : (uint64_t)dev.sms;
     *grid = (uint32_t)(g < kMaxGrid ? g : kMaxGrid);
     return HUFFLLM_OK;
 }
@@ -102,11 +119,57 @@ huffllm_status huffllm_decode(const huffllm_desc *desc, const void *blob, uint16
     if (!out || ((uintptr_t)out & 15)) return fail(HUFFLLM_ERR_INVALID_ARG, "out must be a 16-byte aligned device pointer");
     KernelArgs k;
     uint32_t grid;
-    if ((st = fill_args(desc, blob, 1, false, *dev, &k, &grid)) != HUFFLLM_OK) return st;
-    k.out = out;
+    begin_args(&k, 1, *dev);
+    if ((st = add_matrix(&k, desc, blob)) != HUFFLLM_OK) return st;
+    if ((st = finish_args(&k, false, *dev, &grid)) != HUFFLLM_OK) return st;
+    k.m[0].out = out;
     k.err = err_flag;
     cudaError_t e = launch_decode(k, grid, (cudaStream_t)stream);
     if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "decode launch: %s", cudaGetErrorString(e));
+    return HUFFLLM_OK;
+}
+
+// Checks shared by the product entry points for one matrix of a call.
+static huffllm_status check_product_args(const huffllm_desc *desc, const uint16_t *x, const float *y, const void *workspace,
+                                         size_t workspace_bytes, uint32_t batch) {
+    if (!x || !y || !workspace) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
+    if (((uintptr_t)x & 15) || ((uintptr_t)y & 3) || ((uintptr_t)workspace & 255))
+        return fail(HUFFLLM_ERR_INVALID_ARG, "x must be 16-byte, y 4-byte, workspace 256-byte aligned");
+    if (workspace_bytes < ws_bytes_for(batch)) return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "workspace too small");
+    huffllm_status st = check_desc(desc);
+    if (st != HUFFLLM_OK) return st;
+    if (desc->cols % kBlockCols) return fail(HUFFLLM_ERR_UNSUPPORTED, "fused products need cols to be a multiple of 32");
+    return HUFFLLM_OK;
+}
+
+huffllm_status huffllm_decode_gemm_multi(uint32_t n, const huffllm_desc *const *descs, const void *const *blobs,
+                                         const uint16_t *const *xs, uint32_t batch, float *const *ys, void *const *workspaces,
+                                         size_t workspace_bytes_each, int32_t *err_flag, huffllm_stream stream) {
+    clear_error();
+    DeviceInfo *dev;
+    huffllm_status st = device_info(&dev);
+    if (st != HUFFLLM_OK) return st;
+    if (!descs || !blobs || !xs || !ys || !workspaces) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
+    if (n == 0 || n > kMaxMats) return fail(HUFFLLM_ERR_INVALID_ARG, "between 1 and %u matrices per call", kMaxMats);
+    if (batch == 0 || batch > kKernelBatch) return fail(HUFFLLM_ERR_UNSUPPORTED, "batch must be in [1, %u] here", kKernelBatch);
+    KernelArgs k;
+    uint32_t grid;
+    begin_args(&k, batch, *dev);
+    for (uint32_t i = 0; i < n; ++i) {
+        if ((st = check_product_args(descs[i], xs[i], ys[i], workspaces[i], workspace_bytes_each, batch)) != HUFFLLM_OK) return st;
+        for (uint32_t j = 0; j < i; ++j)
+            if (workspaces[j] == workspaces[i]) return fail(HUFFLLM_ERR_INVALID_ARG, "matrices %u and %u share a workspace", j, i);
+        if ((st = add_matrix(&k, descs[i], blobs[i])) != HUFFLLM_OK) return st;
+        MatArgs &m = k.m[i];
+        m.x = xs[i];
+        m.y = ys[i];
+        m.ws_ticket = (unsigned int *)workspaces[i];
+        m.ws_partial = (float *)((uint8_t *)workspaces[i] + ws_partial_offset());
+    }
+    if ((st = finish_args(&k, true, *dev, &grid)) != HUFFLLM_OK) return st;
+    k.err = err_flag;
+    cudaError_t e = launch_gemm(k, grid, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "product launch: %s", cudaGetErrorString(e));
     return HUFFLLM_OK;
 }
 
@@ -116,23 +179,19 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
     DeviceInfo *dev;
     huffllm_status st = device_info(&dev);
     if (st != HUFFLLM_OK) return st;
-    if (!x || !y || !workspace) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
     if (batch == 0 || batch > 64) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be in [1, 64]");
-    if (((uintptr_t)x & 15) || ((uintptr_t)y & 3) || ((uintptr_t)workspace & 255))
-        return fail(HUFFLLM_ERR_INVALID_ARG, "x must be 16-byte, y 4-byte, workspace 256-byte aligned");
-    if (workspace_bytes < ws_bytes_for(batch)) return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "workspace too small");
-    st = check_desc(desc);
-    if (st != HUFFLLM_OK) return st;
-    if (desc->cols % kBlockCols) return fail(HUFFLLM_ERR_UNSUPPORTED, "fused products need cols to be a multiple of 32");
+    if ((st = check_product_args(desc, x, y, workspace, workspace_bytes, batch)) != HUFFLLM_OK) return st;
     for (uint32_t b0 = 0; b0 < batch; b0 += kKernelBatch) {
         uint32_t nb = batch - b0 < kKernelBatch ? batch - b0 : kKernelBatch;
         KernelArgs k;
         uint32_t grid;
-        if ((st = fill_args(desc, blob, nb, true, *dev, &k, &grid)) != HUFFLLM_OK) return st;
-        k.x = x + (uint64_t)b0 * desc->cols;
-        k.y = y + (uint64_t)b0 * desc->rows;
-        k.ws_ticket = (unsigned int *)workspace;
-        k.ws_partial = (float *)((uint8_t *)workspace + ws_partial_offset());
+        begin_args(&k, nb, *dev);
+        if ((st = add_matrix(&k, desc, blob)) != HUFFLLM_OK) return st;
+        if ((st = finish_args(&k, true, *dev, &grid)) != HUFFLLM_OK) return st;
+        k.m[0].x = x + (uint64_t)b0 * desc->cols;
+        k.m[0].y = y + (uint64_t)b0 * desc->rows;
+        k.m[0].ws_ticket = (unsigned int *)workspace;
+        k.m[0].ws_partial = (float *)((uint8_t *)workspace + ws_partial_offset());
         k.err = err_flag;
         cudaError_t e = launch_gemm(k, grid, (cudaStream_t)stream);
         if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "product launch: %s", cudaGetErrorString(e));

@@ -5,23 +5,32 @@
 
 namespace huffllm {
 
-struct KernelArgs {
+constexpr uint32_t kMaxMats = 8;   // matrices one launch can work through
+
+// One matrix of a launch.
+struct MatArgs {
     const uint8_t *blob;       // device
     uint64_t off_lut, off_index, off_payload;
+    uint64_t rows, cols;
     uint32_t payload_units;    // payload size in 128-byte units
-    uint64_t rows, cols, n_chunks;
-    uint32_t chunk_cols, col_chunks, lut_bits;
-    uint32_t slot_bytes;       // shared-memory bytes of one slot: (max_words + 1) * 256
-    uint32_t guard_bytes;      // readable bytes kept free behind the last slot
-    uint32_t part_bytes;       // bytes at the end of dynamic shared memory for the CTA's partial sums
-    uint32_t dyn_smem_bytes;
+    uint32_t n_chunks, chunk_cols, col_chunks;
+    uint32_t chunk_base;       // number of chunks of the matrices in front of this one
     const uint16_t *x;         // [batch][cols]
     float *y;                  // [batch][rows]
-    uint32_t batch;            // 1..8
     float *ws_partial;         // [grid * 2][16 * batch]
     unsigned int *ws_ticket;   // [grid] arrival counters, zero between calls
     uint16_t *out;             // decode output
+};
+
+struct KernelArgs {
+    uint32_t n_mats, total_chunks, lut_bits;
+    uint32_t slot_bytes;       // shared-memory bytes of one slot: (largest max_words + 1) * 256
+    uint32_t guard_bytes;      // readable bytes kept free behind the last slot
+    uint32_t part_bytes;       // bytes at the end of dynamic shared memory for the CTA's partial sums
+    uint32_t dyn_smem_bytes;
+    uint32_t batch;            // 1..8
     int32_t *err;              // may be null
+    MatArgs m[kMaxMats];
 };
 
 cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t stream);

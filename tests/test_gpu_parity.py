@@ -138,6 +138,31 @@ def test_fused_product_matches_oracle(hl, torch, rows, cols, ce, budget, gen, ba
     assert np.array_equal(y1, y2), "results must be bitwise reproducible"
 
 
+@pytest.mark.parametrize("batch", [1, 3])
+def test_several_matrices_in_one_launch(hl, torch, batch):
+    """Matrices of different shapes and chunk sizes through huffllm_decode_gemm_multi: every result against the
+    oracle, and the launch must leave every workspace's control words zero."""
+    shapes = [(256, 1024, 4096, "gauss"), (48, 2080, 1024, "student"), (1040, 512, 512, "gauss"), (16, 8192, 4096, "gauss"),
+              (2368, 256, 4096, "uniform")]
+    ups, xs, x_devs, ys = [], [], [], []
+    for i, (rows, cols, ce, gen) in enumerate(shapes):
+        w = make(gen, rows, cols, 900 + i)
+        ups.append(Uploaded(hl, torch, w, ce, 0, batch))
+        x = wl.activations(batch, cols, 950 + i)
+        xs.append(x)
+        x_devs.append(torch.from_numpy(x.view(np.int16)).cuda())
+        ys.append(torch.full((batch * rows,), float("nan"), dtype=torch.float32, device="cuda"))
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for rep in range(2):
+        hl.decode_gemm_multi([u.desc for u in ups], [u.blob_dev for u in ups], x_devs, batch, ys, [u.ws for u in ups],
+                             ups[0].ws_bytes, err)
+        torch.cuda.synchronize()
+        assert int(err.item()) == 0
+        for u, x, y in zip(ups, xs, ys):
+            check_product(y.cpu().numpy().reshape(batch, -1), u.w, x)
+            assert int(u.ws[:4096].count_nonzero().item()) == 0
+
+
 def test_product_closed_forms(hl, torch):
     rows, cols = 64, 1024
     ones = np.full((rows, cols), 0x3F80, dtype=np.uint16)
