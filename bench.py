@@ -55,7 +55,7 @@ def launch_groups(table, fuse: str):
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one fused-product launch over its algorithmic bytes, from the
 # ncu capture summarised in profiles/ (None until a capture exists); traffic = ratio * algorithmic bytes.
-NCU_TRAFFIC_RATIO = None
+NCU_TRAFFIC_RATIO = 1.03   # profiles/huff_kernel_product_llama7b_layer.md: 147.5 MB moved for 142.0 MB (gate+up), 72.3 for 71.0 (down)
 
 
 def measured_peak():
@@ -115,7 +115,7 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def prepare(workload: str, chunk_elems: int, hl, torch, dev):
+def prepare(workload: str, chunk_elems: int, hl, torch, dev, cpu_sample_mats: int = 0):
     """Generate, encode (host) and upload every matrix of the workload."""
     table, std, seed, _ = WORKLOADS[workload]
     mats = []
@@ -134,8 +134,8 @@ def prepare(workload: str, chunk_elems: int, hl, torch, dev):
                          y_dev=torch.zeros(rows, dtype=torch.float32, device=dev),
                          ws=torch.zeros(ws_bytes, dtype=torch.uint8, device=dev), ws_bytes=ws_bytes,
                          alg_bytes=int(alg_bytes), coded_bits=int(desc.coded_bits), raw_bits=int(desc.raw_bits),
-                         blob_bytes=int(desc.blob_bytes), w_sample=w[:512].copy() if i == 0 else None,
-                         x_np=x if i == 0 else None))
+                         blob_bytes=int(desc.blob_bytes), w_sample=w.copy() if i < cpu_sample_mats else None,
+                         x_np=x if i < cpu_sample_mats else None))
         del w
     return mats
 
@@ -166,9 +166,13 @@ def run_reference(args):
     import paper_2502_00922_b200 as hl   # host encoder only: it produces the blob the oracle decodes
     table, std, seed, desc_text = WORKLOADS[args.workload]
     name, rows, cols = table[0]
-    sample_rows = min(rows, 128)
-    w = wl.gaussian_weights(rows, cols, std, seed)[:sample_rows].copy()
+    w_full = wl.gaussian_weights(rows, cols, std, seed)
     x = wl.activations(1, cols, seed + 500)
+    # size the per-step sample so that warmup + K steps take about 90 s: probe 64 rows, then scale (16-row granularity)
+    probe = oracle_sample_time(hl, w_full[:64].copy(), x, args.chunk_elems)
+    budget_rows = 64 * 90.0 / (probe * (args.warmup + args.steps))
+    sample_rows = int(max(16, min(rows, budget_rows // 16 * 16)))
+    w = w_full[:sample_rows].copy()
     times = []
     for i in range(args.warmup + args.steps):
         dt = oracle_sample_time(hl, w, x, args.chunk_elems)
@@ -215,7 +219,8 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     args.warmup = max(args.warmup, 3)
 
-    mats = prepare(args.workload, args.chunk_elems, hl, torch, dev)
+    cpu_mats = 0 if (args.no_cpu_baseline or world > 1 or rank != 0) else 4      # whole matrices kept for the CPU-oracle leg
+    mats = prepare(args.workload, args.chunk_elems, hl, torch, dev, cpu_mats)
     err = torch.zeros(1, dtype=torch.int32, device=dev)
     n_weights = sum(m["rows"] * m["cols"] for m in mats)
     unc_bytes = 2 * n_weights
@@ -230,10 +235,13 @@ def main():
         for c in calls:
             hl.decode_gemm_multi(c["descs"], c["blobs"], c["xs"], 1, c["ys"], c["wss"], mats[0]["ws_bytes"], err, stream)
 
-    def step_host():
-        for m in mats:
-            hl.decode_gemm_host(m["desc"], m["blob_dev"], m["x_host"], 1, m["y_host"], m["x_dev"], m["y_dev"], m["ws"],
-                                m["ws_bytes"], err, stream)
+    for c, g in zip(calls, groups):
+        c["xh"], c["yh"] = [mats[i]["x_host"] for i in g], [mats[i]["y_host"] for i in g]
+
+    def step_host():      # host activations in, host results out, through the C-ABI's host-buffer call
+        for c in calls:
+            hl.decode_gemm_multi_host(c["descs"], c["blobs"], c["xh"], 1, c["yh"], c["xs"], c["ys"], c["wss"],
+                                      mats[0]["ws_bytes"], err, stream)
 
     def barrier():
         if dist is not None:
@@ -322,10 +330,11 @@ def main():
     # ---- the CPU oracle on a bounded sample of the same workload (rank 0, single GPU run only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        m0 = mats[0]
-        dt = oracle_sample_time(hl, m0["w_sample"], m0["x_np"], args.chunk_elems, repeats=1)
-        cpu = {"value": 2.0 * m0["w_sample"].size / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-               "sample": f"rows 0..{m0['w_sample'].shape[0] - 1} of matrix '{m0['name']}' ({m0['w_sample'].size} weights, "
+        sample = [m for m in mats if m["w_sample"] is not None]
+        dt = sum(oracle_sample_time(hl, m["w_sample"], m["x_np"], args.chunk_elems, repeats=1) for m in sample)
+        n_w = sum(m["w_sample"].size for m in sample)
+        cpu = {"value": 2.0 * n_w / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": f"matrices {[m['name'] for m in sample]} in full ({n_w} weights = {100.0 * n_w / n_weights:.0f} % of the step, "
                          f"{dt:.1f} s): bit-serial decode of the blob + fp64 product, one thread"}
 
     if rank != 0:

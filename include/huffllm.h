@@ -207,6 +207,16 @@ huffllm_status huffllm_decode_gemm_host(const huffllm_desc *desc, const void *bl
                                         huffllm_stream stream);
 
 /*
+ * huffllm_decode_gemm_multi with HOST activations and HOST results: copies every x_i to its staging
+ * buffer, runs the one launch, copies every y_i back and waits for the stream once.
+ */
+huffllm_status huffllm_decode_gemm_multi_host(uint32_t n, const huffllm_desc *const *descs, const void *const *blobs_dev,
+                                              const uint16_t *const *xs_host, uint32_t batch, float *const *ys_host,
+                                              uint16_t *const *x_stages_dev, float *const *y_stages_dev,
+                                              void *const *workspaces_dev, size_t workspace_bytes_each,
+                                              int32_t *err_flag_dev, huffllm_stream stream);
+
+/*
  * (No counterpart in the paper: an engineering addition for callers that cannot allocate.)
  *
  * huffllm_decode_gemm for callers that have no device scratch buffer to hand over and no way to get

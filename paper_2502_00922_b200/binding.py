@@ -48,6 +48,8 @@ _SIGNATURES = {
     "huffllm_decode_gemm": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemm_multi": [C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_size_t,
                                   C.c_void_p, C.c_void_p],
+    "huffllm_decode_gemm_multi_host": [C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
+                                       C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemm_host": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
                                  C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemm_static": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p],
@@ -192,6 +194,17 @@ def decode_gemm_multi(descs, blobs_dev, xs_dev, batch: int, ys_dev, workspaces_d
     ptrs = lambda seq: (C.c_void_p * n)(*[_ptr(t) for t in seq])
     _check(lib().huffllm_decode_gemm_multi(n, desc_arr, ptrs(blobs_dev), ptrs(xs_dev), batch, ptrs(ys_dev), ptrs(workspaces_dev),
                                            workspace_bytes_each, _ptr(err_flag_dev), _stream(stream)))
+
+
+def decode_gemm_multi_host(descs, blobs_dev, xs_host, batch: int, ys_host, x_stages_dev, y_stages_dev, workspaces_dev,
+                           workspace_bytes_each: int, err_flag_dev=None, stream=None):
+    """huffllm_decode_gemm_multi_host: host activations in, host results out, one wait for the stream."""
+    n = len(descs)
+    desc_arr = (C.POINTER(Desc) * n)(*[C.pointer(d) for d in descs])
+    ptrs = lambda seq: (C.c_void_p * n)(*[_ptr(t) for t in seq])
+    _check(lib().huffllm_decode_gemm_multi_host(n, desc_arr, ptrs(blobs_dev), ptrs(xs_host), batch, ptrs(ys_host),
+                                                ptrs(x_stages_dev), ptrs(y_stages_dev), ptrs(workspaces_dev),
+                                                workspace_bytes_each, _ptr(err_flag_dev), _stream(stream)))
 
 
 def decode_gemm_host(desc: Desc, blob_dev, x_host, batch: int, y_host, x_stage_dev, y_stage_dev, workspace_dev,

@@ -204,6 +204,31 @@ huffllm_status huffllm_decode_gemv(const huffllm_desc *desc, const void *blob, c
     return huffllm_decode_gemm(desc, blob, x, 1, y, workspace, workspace_bytes, err_flag, stream);
 }
 
+huffllm_status huffllm_decode_gemm_multi_host(uint32_t n, const huffllm_desc *const *descs, const void *const *blobs,
+                                              const uint16_t *const *xs_host, uint32_t batch, float *const *ys_host,
+                                              uint16_t *const *x_stages, float *const *y_stages, void *const *workspaces,
+                                              size_t workspace_bytes_each, int32_t *err_flag, huffllm_stream stream) {
+    clear_error();
+    if (!descs || !xs_host || !ys_host || !x_stages || !y_stages) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
+    if (n == 0 || n > kMaxMats) return fail(HUFFLLM_ERR_INVALID_ARG, "between 1 and %u matrices per call", kMaxMats);
+    cudaStream_t s = (cudaStream_t)stream;
+    for (uint32_t i = 0; i < n; ++i) {
+        if (!descs[i] || !xs_host[i] || !ys_host[i] || !x_stages[i] || !y_stages[i]) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
+        cudaError_t e = cudaMemcpyAsync(x_stages[i], xs_host[i], (size_t)batch * descs[i]->cols * 2, cudaMemcpyHostToDevice, s);
+        if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "copy of x: %s", cudaGetErrorString(e));
+    }
+    huffllm_status st = huffllm_decode_gemm_multi(n, descs, blobs, (const uint16_t *const *)x_stages, batch, y_stages, workspaces,
+                                                  workspace_bytes_each, err_flag, stream);
+    if (st != HUFFLLM_OK) return st;
+    for (uint32_t i = 0; i < n; ++i) {
+        cudaError_t e = cudaMemcpyAsync(ys_host[i], y_stages[i], (size_t)batch * descs[i]->rows * 4, cudaMemcpyDeviceToHost, s);
+        if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "copy of y: %s", cudaGetErrorString(e));
+    }
+    cudaError_t e = cudaStreamSynchronize(s);
+    if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "waiting for the stream: %s", cudaGetErrorString(e));
+    return HUFFLLM_OK;
+}
+
 huffllm_status huffllm_decode_gemm_host(const huffllm_desc *desc, const void *blob, const uint16_t *x_host, uint32_t batch,
                                         float *y_host, uint16_t *x_stage, float *y_stage, void *workspace,
                                         size_t workspace_bytes, int32_t *err_flag, huffllm_stream stream) {

@@ -161,6 +161,13 @@ def test_several_matrices_in_one_launch(hl, torch, batch):
         for u, x, y in zip(ups, xs, ys):
             check_product(y.cpu().numpy().reshape(batch, -1), u.w, x)
             assert int(u.ws[:4096].count_nonzero().item()) == 0
+    # the same call with host buffers
+    xh = [torch.from_numpy(x.view(np.int16).reshape(-1)).pin_memory() for x in xs]
+    yh = [torch.zeros(batch * u.w.shape[0], dtype=torch.float32).pin_memory() for u in ups]
+    hl.decode_gemm_multi_host([u.desc for u in ups], [u.blob_dev for u in ups], xh, batch, yh, x_devs, ys, [u.ws for u in ups],
+                              ups[0].ws_bytes, err)
+    for u, x, y in zip(ups, xs, yh):
+        check_product(y.numpy().reshape(batch, -1), u.w, x)
 
 
 def test_product_closed_forms(hl, torch):
