@@ -2,6 +2,7 @@
 // No allocation and no synchronisation here (huffllm_decode_gemm_host, which exists to be timed
 // end to end with host buffers, is the one call that waits for its stream).
 #include <cuda_runtime.h>
+#include <cstdlib>
 #include <cstring>
 
 #include "internal.h"
@@ -44,6 +45,39 @@ size_t ws_bytes_for(uint32_t batch) {
     return ws_partial_offset() + (size_t)kMaxGrid * 2 * 16 * b * sizeof(float);
 }
 
+// Geometry of the tensor-core small-batch path (batch 9..64): row tiles of 512 rows, column chunks cut into
+// `ksplit` ranges so that the work items fill the GPU's SMs in whole waves as well as they can.
+struct TcPlan {
+    uint32_t npad, tiles, m_tiles, ksplit, items;
+    size_t ticket_off, partial_off, bytes;
+};
+// Shared memory the tensor-core kernel needs with `tiles` 128-row tiles per CTA.
+uint64_t tc_smem_need(const huffllm_desc *d, uint32_t npad, uint32_t tiles) {
+    const uint32_t checks_per_block = d->lut_bits == 8 ? 3 : 4;
+    uint64_t guard = 256ull * (3 + checks_per_block * (d->chunk_cols / kBlockCols));
+    return (128ull << d->lut_bits) + guard + 4ull * npad * 64 + 4096 + 2ull * 8 * tiles * d->max_words * 256;
+}
+TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn_smem) {
+    TcPlan p;
+    p.npad = batch <= 16 ? 16 : (batch <= 32 ? 32 : 64);
+    p.tiles = 4;                                    // as many 8-warp tiles as the chunk slots leave room for
+    while (p.tiles > 1 && tc_smem_need(d, p.npad, p.tiles) > dyn_smem) --p.tiles;
+    p.m_tiles = (d->row_groups + 8 * p.tiles - 1) / (8 * p.tiles);
+    uint32_t best = 1;
+    double best_eff = 0;
+    for (uint32_t ks = 1; ks <= 16 && ks <= d->col_chunks; ++ks) {
+        uint64_t items = (uint64_t)p.m_tiles * ks, waves = (items + sms - 1) / sms;
+        double eff = (double)items / (double)(waves * sms);
+        if (eff > best_eff + 1e-9) { best_eff = eff; best = ks; }
+    }
+    p.ksplit = best;
+    p.items = p.m_tiles * best;
+    p.ticket_off = 4096;
+    p.partial_off = p.ticket_off + (((size_t)p.m_tiles * 32 * 4 + 255) / 256) * 256;
+    p.bytes = p.partial_off + (best > 1 ? (size_t)p.items * 32 * (p.npad / 2) * 32 * sizeof(float) : 0);
+    return p;
+}
+
 // Start a launch description.
 void begin_args(KernelArgs *k, uint32_t batch, const DeviceInfo &dev) {
     memset(k, 0, sizeof(*k));
@@ -76,7 +110,9 @@ huffllm_status add_matrix(KernelArgs *k, const huffllm_desc *desc, const void *b
     m.chunk_base = k->total_chunks;
     k->total_chunks += m.n_chunks;
     k->lut_bits = desc->lut_bits;
-    uint32_t slot = (desc->max_words + 1) * 256;
+    // a slot holds the W rows of a record; the window runs one row ahead of what it consumes, and that look-ahead
+    // past the last row lands in the next slot, the table or the guard area and is never used
+    uint32_t slot = desc->max_words * 256;
     // a corrupt stream can advance its read pointer by one row per refill check and no further
     const uint32_t checks_per_block = desc->lut_bits == 8 ? 3 : 4;
     uint32_t guard = 256 * (3 + checks_per_block * (desc->chunk_cols / kBlockCols));
@@ -108,6 +144,15 @@ huffllm_status huffllm_workspace_bytes(const huffllm_desc *desc, uint32_t batch,
     if (st != HUFFLLM_OK) return st;
     if (batch == 0 || batch > 64) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be in [1, 64]");
     *bytes = ws_bytes_for(batch);
+    if (batch > kKernelBatch) {      // the tensor-core path keeps partial tiles of its column ranges here
+        DeviceInfo *dev;
+        int sms = device_info(&dev) == HUFFLLM_OK ? dev->sms : 148;
+        clear_error();
+        uint32_t dyn = device_info(&dev) == HUFFLLM_OK ? (uint32_t)dev->smem_optin - kStaticSmem : 232448u - kStaticSmem;
+        clear_error();
+        size_t tc = tc_plan(desc, batch, (uint32_t)sms, dyn).bytes;
+        if (tc > *bytes) *bytes = tc;
+    }
     return HUFFLLM_OK;
 }
 
@@ -181,6 +226,33 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
     if (st != HUFFLLM_OK) return st;
     if (batch == 0 || batch > 64) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be in [1, 64]");
     if ((st = check_product_args(desc, x, y, workspace, workspace_bytes, batch)) != HUFFLLM_OK) return st;
+    if (batch > kKernelBatch) {
+        // tensor-core path: one pass over the compressed weights for the whole batch
+        const TcPlan tp = tc_plan(desc, batch, (uint32_t)dev->sms, (uint32_t)dev->smem_optin - kStaticSmem);
+        KernelArgs k;
+        uint32_t grid;
+        begin_args(&k, batch, *dev);
+        if ((st = add_matrix(&k, desc, blob)) != HUFFLLM_OK) return st;
+        k.part_bytes = 4 * tp.npad * 64;                       // four stages of activations
+        const uint64_t need = tc_smem_need(desc, tp.npad, tp.tiles);
+        if (need <= k.dyn_smem_bytes && workspace_bytes >= tp.bytes) {
+            k.m[0].x = x;
+            k.m[0].y = y;
+            k.tc_npad = tp.npad;
+            k.tc_tiles = tp.tiles;
+            k.tc_m_tiles = tp.m_tiles;
+            k.tc_ksplit = tp.ksplit;
+            k.tc_ticket = (unsigned int *)((uint8_t *)workspace + tp.ticket_off);
+            k.tc_partial = (float *)((uint8_t *)workspace + tp.partial_off);
+            k.err = err_flag;
+            grid = tp.items < (uint32_t)dev->sms ? tp.items : (uint32_t)dev->sms;
+            cudaError_t e = launch_gemm_tc(k, grid, (cudaStream_t)stream);
+            if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "tensor-core product launch: %s", cudaGetErrorString(e));
+            return HUFFLLM_OK;
+        }
+        if (workspace_bytes < tp.bytes) return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "workspace too small for batch %u", batch);
+        // chunk records too large for 32 warps' slots: fall through to passes of 8 vectors
+    }
     for (uint32_t b0 = 0; b0 < batch; b0 += kKernelBatch) {
         uint32_t nb = batch - b0 < kKernelBatch ? batch - b0 : kKernelBatch;
         KernelArgs k;

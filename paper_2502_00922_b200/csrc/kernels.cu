@@ -27,217 +27,9 @@
 #include <cuda_runtime.h>
 #include <cstdint>
 
-#include "kernels.h"
+#include "decode_common.cuh"
 
 namespace huffllm {
-
-// ------------------------------------------------------------------------------ PTX helpers
-
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ uint32_t lds_stream(uint32_t addr) {
-    uint32_t v;
-    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
-    return v;
-}
-// LUT reads: the table is constant once built, so the compiler may schedule these freely.
-__device__ __forceinline__ uint32_t lds_lut(uint32_t addr) {
-    uint32_t v;
-    asm("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ uint32_t prmt(uint32_t a, uint32_t b, uint32_t sel) {
-    uint32_t d;
-    asm("prmt.b32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(sel));
-    return d;
-}
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok != 0;
-}
-// Bulk asynchronous copy global -> this CTA's shared memory, completion counted on `bar`.
-__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
-    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
-                 "l"(src), "r"(bytes), "r"(bar)
-                 : "memory");
-}
-__device__ __forceinline__ uint4 ldg_stream16(const void *p) {
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
-}
-__device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
-                                               uint32_t b1) {
-    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
-                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
-                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
-}
-
-// Arrival counter bump that publishes this warp's earlier stores and acquires the other arrivals' stores.
-__device__ __forceinline__ uint32_t arrive_acq_rel(unsigned int *counter) {
-    uint32_t old;
-    asm volatile("atom.acq_rel.gpu.global.add.u32 %0, [%1], 1;" : "=r"(old) : "l"(counter) : "memory");
-    return old;
-}
-// Programmatic dependent launch: let the next kernel in the stream be scheduled early / wait for the previous one.
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
-__device__ __forceinline__ void pdl_wait_prior_grid() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-
-// ------------------------------------------------------------------------------ lane decoder
-
-// State of the decoder of one bit sequence.  (hi:lo) holds 64 stream bits; the current codeword starts
-// at bit pos + 7 of that window (the 7 bits in front are the lag that makes the table address fall out
-// of a single AND/OR); nxt is the shared-memory address of the sequence's next 32-bit word.  Words of
-// one sequence are 256 bytes apart (a row of the record holds one word of each of the 64 sequences).
-struct LaneStream {
-    uint32_t lo, hi, pos, nxt;
-};
-
-__device__ __forceinline__ void stream_open(LaneStream &s, uint32_t lane_word0) {
-    s.lo = lds_stream(lane_word0);
-    s.hi = lds_stream(lane_word0 + 256);
-    s.nxt = lane_word0 + 512;
-    s.pos = 0;
-}
-
-// One decoder step: returns the table entry (length << 16 | exponent << 7) and advances the start pointer.
-// The window is shifted as a 64-bit value, so the pointer may run past bit 32 between two refill
-// checks.  The table address is (window & index mask) | (table base + 4 * lane): one logic operation,
-// because the table sits on a boundary above the index bits.  Only byte 2 of the entry (the length)
-// is added to the pointer: dp4a with that byte selected does it in one instruction off the ALU pipe.
-__device__ __forceinline__ uint32_t stream_step(LaneStream &s, uint32_t idx_mask, uint32_t lut_lane) {
-    uint64_t win = ((uint64_t)s.hi << 32) | s.lo;
-    uint32_t t = (uint32_t)(win >> s.pos), addr;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(addr) : "r"(t), "r"(idx_mask), "r"(lut_lane));
-    uint32_t e = lds_lut(addr);
-    s.pos = __dp4a(e, 0x00010000u, s.pos);
-    return e;
-}
-
-// Refill: once 32 bits have been consumed, slide the window by one word.  Written with predicated
-// instructions so that lanes which need a word and lanes which do not stay converged.
-// The two additions are written as multiply-adds by a register holding 1 so that they run on the FMA pipe:
-// the 16-lane integer ALU pipe is the busiest unit of this kernel.
-__device__ __forceinline__ void stream_refill(LaneStream &s, uint32_t one) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ge.u32 p, %2, 32;\n\t"
-        "@p mov.u32 %0, %1;\n\t"
-        "@p ld.shared.u32 %1, [%3];\n\t"
-        "@p mad.lo.u32 %3, %4, 256, %3;\n\t"
-        "@p mad.lo.u32 %2, %4, 0xFFFFFFE0, %2;\n\t}"
-        : "+r"(s.lo), "+r"(s.hi), "+r"(s.pos), "+r"(s.nxt)
-        : "r"(one));
-}
-
-// Two table entries + two raw bytes -> two bf16 weights packed in one register.
-// SEL picks raw bytes (i, i+1) of `raw` as (byte, sign-replicated byte) pairs.  The exponent of the
-// even weight is already in place (bits 7..14); the odd entry times 65536 puts its exponent at bits
-// 23..30 and pushes its length out of the word, so one multiply-add (FMA pipe) merges the two.
-template <uint32_t SEL>
-__device__ __forceinline__ uint32_t pack_pair(uint32_t e_even, uint32_t e_odd, uint32_t raw) {
-    uint32_t sm = prmt(raw, 0u, SEL);   // [sign1*0xFF, raw1, sign0*0xFF, raw0]
-    uint32_t ex;
-    asm("mad.lo.u32 %0, %1, 65536, %2;" : "=r"(ex) : "r"(e_odd), "r"(e_even));
-    uint32_t w;   // sign and mantissa bits from sm, exponent bits from ex
-    asm("lop3.b32 %0, %1, %2, 0x807F807F, 0xE4;" : "=r"(w) : "r"(sm), "r"(ex));
-    return w;
-}
-
-// Decode one block (16 weights of this lane) into 8 packed registers:
-// a[0..3] = row g, columns (0,1) (2,3) (4,5) (6,7);  a[4..7] = row g+8, same columns.
-// The lane's two sequences are stepped alternately.  Each window is checked for a refill before every
-// R-th step: after a check at least 26 bits are valid in front of the start pointer, enough for R
-// codewords of at most 26/R bits.
-template <int R>
-__device__ __forceinline__ void decode_block(LaneStream &sa, LaneStream &sb, uint32_t idx_mask, uint32_t lut_lane, uint32_t one,
-                                             const uint4 &raw, uint32_t (&a)[8]) {
-    uint32_t e[16];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) {
-        if (i % R == 0) {
-            stream_refill(sa, one);
-            stream_refill(sb, one);
-        }
-        e[i] = stream_step(sa, idx_mask, lut_lane);
-        e[8 + i] = stream_step(sb, idx_mask, lut_lane);
-    }
-    a[0] = pack_pair<0x9180u>(e[0], e[1], raw.x);
-    a[1] = pack_pair<0xB3A2u>(e[2], e[3], raw.x);
-    a[2] = pack_pair<0x9180u>(e[4], e[5], raw.y);
-    a[3] = pack_pair<0xB3A2u>(e[6], e[7], raw.y);
-    a[4] = pack_pair<0x9180u>(e[8], e[9], raw.z);
-    a[5] = pack_pair<0xB3A2u>(e[10], e[11], raw.z);
-    a[6] = pack_pair<0x9180u>(e[12], e[13], raw.w);
-    a[7] = pack_pair<0xB3A2u>(e[14], e[15], raw.w);
-}
-
-// ------------------------------------------------------------------------------ shared memory plan
-
-// Dynamic shared memory, laid out at run time from the window's real start address:
-//   [base, lut)            slot pairs (as many as fit)
-//   [lut, lut + LUTSZ)     per-lane LUT; lut = base rounded up to a multiple of LUTSZ, so that the
-//                          index bits of a lookup address never overlap the table's base bits
-//   [lut + LUTSZ, ...)     more slot pairs, then a guard area no valid stream ever reads
-//   [end - part_bytes, end) the CTA's table of partial sums (fused product only)
-struct SmemPlan {
-    uint32_t lut;    // shared address of the table
-    uint32_t warps;  // warps that own a slot pair
-    uint32_t slotA;  // first slot pair before the table
-    uint32_t nA;     // slot pairs before the table
-    uint32_t slotB;  // first slot pair after it
-};
-
-__device__ __forceinline__ SmemPlan plan_smem(uint32_t base, const KernelArgs &k, uint32_t max_warps) {   // k: launch-wide fields only
-    SmemPlan p;
-    const uint32_t lut_bytes = 128u << k.lut_bits;
-    uint32_t a0 = (base + 127u) & ~127u;
-    p.lut = (base + lut_bytes - 1) / lut_bytes * lut_bytes;
-    p.slotA = a0;
-    p.nA = p.lut > a0 ? (p.lut - a0) / (2 * k.slot_bytes) : 0;  // a stream that overruns here reads the table: harmless
-    p.slotB = p.lut + lut_bytes;
-    uint32_t end = base + k.dyn_smem_bytes - k.part_bytes;
-    uint32_t roomB = end > p.slotB + k.guard_bytes ? end - p.slotB - k.guard_bytes : 0;
-    p.warps = min(max_warps, p.nA + roomB / (2 * k.slot_bytes));
-    return p;
-}
-
-__device__ __forceinline__ uint32_t slot_addr(const SmemPlan &p, uint32_t warp, uint32_t which, uint32_t slot_bytes) {
-    uint32_t pair = warp < p.nA ? p.slotA + warp * 2 * slot_bytes : p.slotB + (warp - p.nA) * 2 * slot_bytes;
-    return pair + which * slot_bytes;
-}
-
-constexpr int kMaxWarps = 32;
-// Experiment build only (-DHUFFLLM_TIMING): every warp writes nanosecond stamps of its phases into the
-// buffer passed as the error flag, [cta][warp][8].
-#ifdef HUFFLLM_TIMING
-__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define STAMP(i) do { if (lane == 0) ((unsigned long long *)A.err)[((size_t)blockIdx.x * 32 + warp) * 8 + (i)] = gtime(); } while (0)
-#define BLOCKSTAMP(n, phase) do { if (lane == 0 && blockIdx.x == 3 && (n) < 64) ((unsigned long long *)A.err)[148 * 32 * 8 + (warp * 64 + (n)) * 4 + (phase)] = clock64(); } while (0)
-#else
-#define STAMP(i) do {} while (0)
-#define BLOCKSTAMP(n, phase) do {} while (0)
-#endif
-#ifndef HUFFLLM_THREADS
-#define HUFFLLM_THREADS 1024
-#endif
-constexpr int kThreads = HUFFLLM_THREADS;   // threads per CTA of the decode kernels (one CTA per SM)
-constexpr uint32_t kWaitLimit = 1u << 22;
 
 // ------------------------------------------------------------------------------ the fused kernel
 
@@ -310,7 +102,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         // a record is usable if it lies inside the payload and its coded part fits a slot
         auto record_ok = [&](uint32_t r0, uint32_t r1, uint32_t nkb) -> bool {
             return r1 > r0 && r1 <= k.payload_units && (r1 - r0) * 128u > nkb * 512u &&
-                   (r1 - r0) * 128u - nkb * 512u + 256u <= A.slot_bytes;
+                   (r1 - r0) * 128u - nkb * 512u <= A.slot_bytes;
         };
         // lane 0: start the bulk copy of a chunk's coded part into slot `which`
         auto issue = [&](uint32_t c, uint32_t which) {

@@ -24,17 +24,25 @@ struct MatArgs {
 
 struct KernelArgs {
     uint32_t n_mats, total_chunks, lut_bits;
-    uint32_t slot_bytes;       // shared-memory bytes of one slot: (largest max_words + 1) * 256
+    uint32_t slot_bytes;       // shared-memory bytes of one slot: largest max_words * 256
     uint32_t guard_bytes;      // readable bytes kept free behind the last slot
     uint32_t part_bytes;       // bytes at the end of dynamic shared memory for the CTA's partial sums
     uint32_t dyn_smem_bytes;
     uint32_t batch;            // 1..8
     int32_t *err;              // may be null
+    // tensor-core small-batch path only
+    uint32_t tc_npad;          // batch rounded up to 16, 32 or 64
+    uint32_t tc_tiles;         // 128-row tiles a CTA decodes side by side (8 warps each): 1..4
+    uint32_t tc_m_tiles;       // row tiles of 128 * tc_tiles rows
+    uint32_t tc_ksplit;        // ranges the column chunks are cut into
+    float *tc_partial;         // [m_tiles * ksplit][32 warps][npad / 2][32]
+    unsigned int *tc_ticket;   // [m_tiles][32], zero between calls
     MatArgs m[kMaxMats];
 };
 
 cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t stream);
 cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream);
+cudaError_t launch_gemm_tc(const KernelArgs &k, uint32_t grid, cudaStream_t stream);
 cudaError_t launch_plain_gemv(const uint16_t *w, uint64_t rows, uint64_t cols, const uint16_t *x, float *y, uint32_t sms,
                               cudaStream_t stream);
 

@@ -1,0 +1,395 @@
+// Small-batch product on the 5th-generation tensor cores (tcgen05), batch 16..64.
+//
+// Same decoder as the matrix-vector kernel (one table lookup per weight, two bit sequences per lane), but the
+// decoded bf16 weights are not multiplied from registers: every warp stores its 16 rows x 32 columns of a
+// block into TENSOR MEMORY as the A operand of a 128-row tile, the activations of the same 32 columns go to
+// shared memory as the B operand, and one thread issues tcgen05.mma (M = 128, N = padded batch, K = 16)
+// whose fp32 accumulator also lives in tensor memory.  The decoded weights are consumed where they are
+// produced (Section 1 of the paper: decompress only to multiply) and one pass over the compressed bytes
+// serves the whole batch; the tensor pipe only takes the batch-fold of multiply-adds off the issue slots.
+//
+// Geometry of a CTA: 32 decoder warps = 4 tiles of 8 warps; a tile is 128 rows (8 row groups of 16), warp
+// (q = warp % 4, h = warp / 4 % 2) of a tile owns tensor-memory lanes 32 q + 16 h .. + 15, which is what the
+// 16x256b store shape of a warp can reach.  Tensor memory (512 columns): 4 accumulators of N columns, then
+// 4 tiles x 4 stages x 16 columns of A (a stage = one block of 32 weight columns = two K = 16 steps).
+// A work item is (512 rows) x (a range of column chunks); partial results of the ranges of one row tile are
+// added in a fixed order by whoever finishes last (per-warp arrival counters, nobody waits).
+//
+// Stage protocol: every warp fills its share of stage s (A rows, a slice of B), then bumps a shared-memory
+// counter; the 32nd arrival issues the 8 MMAs of the stage and a tcgen05.commit onto the stage's "empty"
+// mbarrier, which the warps wait on (with a limit) before they reuse the stage four blocks later.
+#include "decode_common.cuh"
+
+namespace huffllm {
+
+constexpr int kTcStages = 4;
+constexpr int kTcTiles = 4;
+
+__device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_dst), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish() {
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols) {
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+// 16 lanes x 512 bits: thread (g = lane / 4, t = lane % 4) supplies, for rows g and g + 8, the 32-bit columns
+// 2t, 2t+1 (r0, r1 | r2, r3) and 8 + 2t, 8 + 2t + 1 (r4, r5 | r6, r7).
+__device__ __forceinline__ void tc_st_16x256b_x2(uint32_t taddr, const uint32_t (&r)[8]) {
+    asm volatile("tcgen05.st.sync.aligned.16x256b.x2.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};" ::"r"(taddr), "r"(r[0]),
+                 "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7])
+                 : "memory");
+}
+__device__ __forceinline__ void tc_mma_f16_tmem_a(uint32_t d, uint32_t a, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}" ::"r"(d),
+        "r"(a), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+template <int N>
+__device__ __forceinline__ void tc_ld_32x32b(uint32_t taddr, uint32_t (&v)[N]);
+template <>
+__device__ __forceinline__ void tc_ld_32x32b<8>(uint32_t taddr, uint32_t (&v)[8]) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x8.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+                 : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7])
+                 : "r"(taddr)
+                 : "memory");
+}
+template <>
+__device__ __forceinline__ void tc_ld_32x32b<16>(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]),
+          "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+template <>
+__device__ __forceinline__ void tc_ld_32x32b<32>(uint32_t taddr, uint32_t (&v)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, %17, "
+        "%18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]), "=r"(v[9]),
+          "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]), "=r"(v[17]), "=r"(v[18]),
+          "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]),
+          "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr)
+        : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major operand without swizzle: 8-row x 16-byte core matrices,
+// `lbo` bytes between core matrices along K, `sbo` bytes between 8-row groups.
+__device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t addr, uint32_t lbo, uint32_t sbo) {
+    return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46);
+}
+
+// LB = table index bits; NPAD = batch rounded up to 16, 32 or 64 (the MMA's N).
+template <int LB, int NPAD>
+__global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_constant__ KernelArgs A) {
+    constexpr int R = LB == 8 ? 3 : 2;
+    constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
+    constexpr int S = kTcStages;
+    constexpr uint32_t kBStage = NPAD * 64;                 // bytes of B per stage: NPAD rows x 32 columns of bf16
+    constexpr uint32_t kLbo = 128, kSbo = 512;              // core matrices: 4 along K side by side, then the next 8 rows
+    constexpr uint32_t kACol0 = kTcTiles * NPAD;            // first tensor-memory column of the A stages
+    // instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, N = NPAD, M = 128
+    constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NPAD >> 3) << 17) | ((128u >> 4) << 24);
+
+    extern __shared__ __align__(128) uint8_t dyn_smem[];
+    __shared__ __align__(8) uint64_t bars[kMaxWarps * 2];   // per warp: its two coded-copy barriers
+    __shared__ __align__(8) uint64_t empty_bar[S];          // stage may be refilled (arrived on by tcgen05.commit)
+    __shared__ uint32_t full_cnt[S];                        // warps that have filled the stage
+    __shared__ uint32_t s_tmem_base;
+
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const MatArgs &k = A.m[0];
+    const uint32_t smem_base = smem_u32(dyn_smem);
+    const uint32_t n_tiles = A.tc_tiles, n_dec = n_tiles * 8;          // decoder warps; the others leave at once
+    const SmemPlan plan = plan_smem(smem_base, A, n_dec);
+    if (plan.warps < n_dec) {                                   // the entry point sizes shared memory so that this cannot happen
+        if (tid == 0 && A.err) atomicExch(A.err, -3);
+        return;
+    }
+    const uint32_t b_base = smem_base + A.dyn_smem_bytes - A.part_bytes;   // S stages of B behind everything else
+    uint32_t lut_lane = plan.lut | (lane << 2);
+    asm volatile("mov.u32 %0, %0;" : "+r"(lut_lane));
+    const uint32_t bar0 = smem_u32(&bars[warp * 2]);
+    const uint32_t slot0 = slot_addr(plan, warp, 0, A.slot_bytes);
+
+    // ---- set-up: table, barriers, tensor memory
+    {
+        const uint32_t *lut_g = (const uint32_t *)(k.blob + k.off_lut);
+        uint32_t *lut_s = (uint32_t *)(dyn_smem + (plan.lut - smem_base));
+        for (uint32_t i = tid; i < (32u << LB); i += 1024) lut_s[i] = __ldg(lut_g + (i >> 5));
+    }
+    if (lane == 0) {
+        mbar_init(bar0, 1);
+        mbar_init(bar0 + 8, 1);
+    }
+    if (tid < S) {
+        mbar_init(smem_u32(&empty_bar[tid]), 1);
+        full_cnt[tid] = 0;
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    if (warp == 0) {
+        tmem_alloc(smem_u32(&s_tmem_base), 512);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = s_tmem_base;
+    if (warp >= n_dec) {                 // not a decoder warp in this configuration: only the teardown barrier is left
+        tc_fence_before();
+        __syncthreads();
+        return;
+    }
+
+    // ---- roles
+    const uint32_t tile = warp >> 3, q = warp & 3, h = (warp >> 2) & 1;
+    const uint32_t rgi = tile * 8 + q * 2 + h;                              // row group of the CTA's 32 that this warp decodes
+    const uint32_t a_lane = (32u * q + 16u * h) << 16;
+    const uint32_t KC = k.col_chunks, RG = (uint32_t)((k.rows + 15) / 16);
+    const uint32_t *index = (const uint32_t *)(k.blob + k.off_index);
+    const uint8_t *payload = k.blob + k.off_payload;
+    const uint32_t ksplit = A.tc_ksplit, n_items = A.tc_m_tiles * ksplit;
+    uint32_t phase = 0, gb = 0;          // coded-copy barrier parities; blocks this CTA has gone through so far
+    bool failed = false;                 // a wait ran out: stop waiting, keep moving, report
+
+    auto blocks_of = [&](uint32_t kc) -> uint32_t {
+        uint32_t left = (uint32_t)k.cols - kc * k.chunk_cols;
+        return (min(left, k.chunk_cols) + 31u) >> 5;
+    };
+    auto record_ok = [&](uint32_t r0, uint32_t r1, uint32_t nkb) -> bool {
+        return r1 > r0 && r1 <= k.payload_units && (r1 - r0) * 128u > nkb * 512u &&
+               (r1 - r0) * 128u - nkb * 512u <= A.slot_bytes;
+    };
+    auto issue = [&](uint32_t c, uint32_t which) {
+        uint32_t nkb = blocks_of(c % KC), r0 = __ldg(index + c), r1 = __ldg(index + c + 1);
+        uint32_t bar = bar0 + which * 8;
+        if (record_ok(r0, r1, nkb)) {
+            uint32_t bytes = (r1 - r0) * 128u - nkb * 512u;
+            mbar_expect_tx(bar, bytes);
+            bulk_g2s(slot0 + which * A.slot_bytes, payload + (uint64_t)r0 * 128u + nkb * 512u, bytes, bar);
+        } else {
+            mbar_expect_tx(bar, 0);
+        }
+    };
+    auto bounded_wait = [&](uint32_t bar, uint32_t parity) {
+        if (failed) return;
+        uint32_t spins = 0;
+        bool done = mbar_try_wait(bar, parity);
+        while (!__all_sync(0xFFFFFFFFu, done)) {
+            if (++spins > kWaitLimit) {
+                failed = true;
+                if (A.err && lane == 0) atomicExch(A.err, -2);
+                return;
+            }
+            done = mbar_try_wait(bar, parity);
+        }
+    };
+
+    // The activations of a block are NPAD * 4 pieces of 16 bytes, 32 per warp, carried by the first warps.  A warp's
+    // piece u = 32 warp + lane belongs to vector n = u / 4 and K positions 8 kap .. 8 kap + 7 (kap = u % 4) of the
+    // tile, which hold columns base .. base + 3 and base + 8 .. base + 11 of the block, base = 16 (kap & 1) + 4 (kap >> 1).
+    const bool x_carrier = warp * 32 + lane < NPAD * 4;
+    const uint32_t x_n = (warp * 32 + lane) >> 2, x_kap = lane & 3;
+    const uint16_t *x_src = k.x + (uint64_t)x_n * k.cols + (x_kap & 1) * 16 + (x_kap >> 1) * 4;
+    auto load_x = [&](uint4 &v, uint32_t col_block) {        // fetched one block ahead of its use
+        if (x_carrier && x_n < A.batch) {
+            uint2 lo = __ldg((const uint2 *)(x_src + col_block)), hi = __ldg((const uint2 *)(x_src + col_block + 8));
+            v = make_uint4(lo.x, lo.y, hi.x, hi.y);
+        }
+    };
+
+    // One block of the stage protocol.  `a` = this warp's decoded 16 rows x 32 columns (null if the warp has no rows).
+    auto stage_block = [&](const uint32_t *a, const uint4 &xv, bool first_of_item) {
+        const uint32_t s = gb % S, use = gb / S;
+        if (use > 0) bounded_wait(smem_u32(&empty_bar[s]), (use - 1) & 1u);
+        tc_fence_after();
+        if (a) {
+            // lane (g, t): row g's weights 0..3 -> 32-bit columns 2t, 2t+1; weights 4..7 -> columns 8 + 2t, 8 + 2t + 1
+            const uint32_t r[8] = {a[0], a[1], a[4], a[5], a[2], a[3], a[6], a[7]};
+            tc_st_16x256b_x2(tmem + a_lane + kACol0 + (tile * S + s) * 16, r);
+        }
+        if (x_carrier) {
+            const uint32_t dst = b_base + s * kBStage + (x_n >> 3) * kSbo + x_kap * kLbo + (x_n & 7) * 16;
+            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(xv.x), "r"(xv.y), "r"(xv.z), "r"(xv.w) : "memory");
+        }
+        tc_wait_st();
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the B slice must be visible to the tensor core's reads
+        tc_fence_before();
+        __syncwarp();
+        uint32_t last = 0;
+        if (lane == 0) {
+            __threadfence_block();
+            last = atomicAdd(&full_cnt[s], 1u) == n_dec - 1 ? 1u : 0u;
+            if (last) {
+                full_cnt[s] = 0;
+                __threadfence_block();
+                tc_fence_after();
+                const uint32_t bst = b_base + s * kBStage;
+                for (uint32_t tl = 0; tl < n_tiles; ++tl) {
+#pragma unroll
+                    for (uint32_t j = 0; j < 2; ++j)      // two K = 16 steps per stage
+                        tc_mma_f16_tmem_a(tmem + tl * NPAD, tmem + kACol0 + (tl * S + s) * 16 + j * 8,
+                                          smem_desc_kmajor(bst + j * 2 * kLbo, kLbo, kSbo), kIdesc, (first_of_item && j == 0) ? 0u : 1u);
+                }
+                tc_commit(smem_u32(&empty_bar[s]));
+            }
+        }
+        __syncwarp();
+        ++gb;
+    };
+
+#pragma unroll 1
+    for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+        const uint32_t mt = item / ksplit, ks = item % ksplit;
+        const uint32_t rg = mt * n_dec + rgi;
+        const bool active = rg < RG;
+        const uint32_t kc0 = (uint32_t)((uint64_t)KC * ks / ksplit), kc1 = (uint32_t)((uint64_t)KC * (ks + 1) / ksplit);
+        const uint32_t gb_item = gb;
+        // the item's blocks are consecutive 32-column blocks of the matrix, from col_lo up to col_hi
+        const uint32_t col_lo = kc0 * k.chunk_cols, col_hi = min(kc1 * k.chunk_cols, (uint32_t)k.cols);
+        uint32_t col_blk = col_lo;
+        uint4 x_cur = make_uint4(0, 0, 0, 0), x_nxt = make_uint4(0, 0, 0, 0);
+        load_x(x_cur, col_lo);
+
+        if (active) {
+            const uint32_t c_beg = rg * KC + kc0, c_end = rg * KC + kc1;
+            if (lane == 0) {
+                issue(c_beg, 0);
+                if (c_beg + 1 < c_end) issue(c_beg + 1, 1);
+            }
+            uint32_t kc = kc0;
+            uint32_t r0 = __ldg(index + c_beg), r1 = __ldg(index + c_beg + 1);
+#pragma unroll 1
+            for (uint32_t c = c_beg; c < c_end; ++c, ++kc) {
+                const uint32_t which = (c - c_beg) & 1u;
+                const uint32_t nkb = blocks_of(kc);
+                const bool ok = record_ok(r0, r1, nkb);
+                const uint32_t r2 = c + 1 < c_end ? __ldg(index + c + 2) : r1;
+                const uint8_t *raw_p = payload + (uint64_t)r0 * 128u + lane * 16u;
+                uint4 raw_cur = make_uint4(0, 0, 0, 0);
+                if (ok) raw_cur = ldg_stream16(raw_p);
+                bounded_wait(bar0 + which * 8, (phase >> which) & 1u);
+                phase ^= 1u << which;
+                if (!ok && A.err && lane == 0) atomicExch(A.err, (int32_t)min(c + 1, 0x7FFFFFFFu));
+                LaneStream sa, sb;
+                stream_open(sa, slot0 + which * A.slot_bytes + (lane << 2));
+                stream_open(sb, slot0 + which * A.slot_bytes + 128u + (lane << 2));
+#pragma unroll 1
+                for (uint32_t kb = 0; kb < nkb; ++kb) {
+                    uint4 raw_next = raw_cur;
+                    if (ok && kb + 1 < nkb) raw_next = ldg_stream16(raw_p + (size_t)(kb + 1) * 512u);
+                    if (col_blk + 32 < col_hi) load_x(x_nxt, col_blk + 32);
+                    uint32_t a[8];
+                    decode_block<R>(sa, sb, kIdxMask, lut_lane, 1u, raw_cur, a);   // a chunk that is not ok decodes garbage, never out of range
+                    stage_block(a, x_cur, gb == gb_item);
+                    raw_cur = raw_next;
+                    x_cur = x_nxt;
+                    col_blk += 32;
+                }
+                __syncwarp();
+                if (lane == 0 && c + 2 < c_end) issue(c + 2, which);
+                r0 = r1;
+                r1 = r2;
+            }
+        } else {
+            // no rows of the matrix for this warp: it still carries its slice of the activations and its arrivals
+            for (; col_blk < col_hi; col_blk += 32) {
+                if (col_blk + 32 < col_hi) load_x(x_nxt, col_blk + 32);
+                stage_block(nullptr, x_cur, gb == gb_item);
+                x_cur = x_nxt;
+            }
+        }
+
+        // ---- epilogue of the item: wait for the last stage's MMAs, read this warp's 32 rows x NPAD/2 columns
+        {
+            const uint32_t gl = gb - 1;
+            bounded_wait(smem_u32(&empty_bar[gl % S]), (gl / S) & 1u);
+            tc_fence_after();
+            uint32_t v[NPAD / 2];
+            tc_ld_32x32b<NPAD / 2>(tmem + ((32u * q) << 16) + tile * NPAD + h * (NPAD / 2), v);
+            tc_wait_ld();
+            tc_fence_before();
+            // thread `lane` holds row 32 q + lane of the tile, columns n = h * NPAD/2 + i
+            const uint64_t row = (uint64_t)(mt * n_dec + tile * 8) * 16 + 32u * q + lane;
+            const uint32_t n0 = h * (NPAD / 2);
+            if (ksplit == 1) {
+#pragma unroll
+                for (int i = 0; i < NPAD / 2; ++i)
+                    if (n0 + i < A.batch && row < k.rows) k.y[(uint64_t)(n0 + i) * k.rows + row] = __uint_as_float(v[i]);
+            } else {
+                // piece of (item, warp): [NPAD/2][32] floats; the last range to arrive adds the pieces in range order
+                float *piece = A.tc_partial + ((size_t)item * 32 + warp) * (NPAD / 2) * 32;   // 32 piece slots per item, n_dec used
+#pragma unroll
+                for (int i = 0; i < NPAD / 2; ++i) piece[i * 32 + lane] = __uint_as_float(v[i]);
+                __syncwarp();
+                uint32_t last = 0;
+                if (lane == 0) {
+                    unsigned int *ctr = A.tc_ticket + mt * 32 + warp;
+                    last = arrive_acq_rel(ctr) == ksplit - 1 ? 1u : 0u;
+                    if (last) *ctr = 0;
+                }
+                if (__shfl_sync(0xFFFFFFFFu, last, 0)) {
+                    // range after range, NPAD/2 independent loads in flight each time; every output adds its pieces in range order
+                    float sum[NPAD / 2];
+#pragma unroll
+                    for (int i = 0; i < NPAD / 2; ++i) sum[i] = 0.f;
+                    for (uint32_t s2 = 0; s2 < ksplit; ++s2) {
+                        const float *pc = A.tc_partial + ((size_t)(mt * ksplit + s2) * 32 + warp) * (NPAD / 2) * 32 + lane;
+#pragma unroll
+                        for (int i = 0; i < NPAD / 2; ++i) sum[i] += __ldcg(pc + i * 32);
+                    }
+#pragma unroll
+                    for (int i = 0; i < NPAD / 2; ++i)
+                        if (n0 + i < A.batch && row < k.rows) k.y[(uint64_t)(n0 + i) * k.rows + row] = sum[i];
+                }
+            }
+        }
+    }
+
+    // ---- teardown
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem, 512);
+}
+
+template <int LB, int NPAD>
+static cudaError_t launch_tc_one(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
+    auto fn = huff_gemm_tc_kernel<LB, NPAD>;
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)k.dyn_smem_bytes);
+        if (e != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    fn<<<grid, 1024, k.dyn_smem_bytes, stream>>>(k);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_gemm_tc(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
+    if (k.lut_bits == 8) {
+        if (k.tc_npad == 16) return launch_tc_one<8, 16>(k, grid, stream);
+        if (k.tc_npad == 32) return launch_tc_one<8, 32>(k, grid, stream);
+        return launch_tc_one<8, 64>(k, grid, stream);
+    }
+    if (k.tc_npad == 16) return launch_tc_one<9, 16>(k, grid, stream);
+    if (k.tc_npad == 32) return launch_tc_one<9, 32>(k, grid, stream);
+    return launch_tc_one<9, 64>(k, grid, stream);
+}
+
+}  // namespace huffllm

@@ -122,8 +122,13 @@ GEMM_CASES = [
     (272, 2080, 16384, 0, "gauss", 4),
     (512, 4096, 4096, 9, "student", 5),
     (256, 2048, 4096, 0, "uniform", 8),
-    (128, 1024, 1024, 0, "gauss", 16),            # two passes of 8
+    (128, 1024, 1024, 0, "gauss", 16),            # batch 9..64 runs on the tcgen05 path
     (64, 1024, 4096, 0, "gauss", 23),
+    (40, 2080, 1024, 0, "student", 9),            # ragged rows, padded batch
+    (1040, 4096, 4096, 0, "gauss", 64),           # three row tiles, column chunks cut into ranges
+    (16, 65536, 4096, 0, "gauss", 16),            # one row group, 16 column ranges
+    (2368, 512, 512, 0, "uniform", 48),           # several work items per CTA
+    (528, 2048, 4096, 9, "student", 32),          # 512-entry table
 ]
 
 
