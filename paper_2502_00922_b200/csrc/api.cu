@@ -72,8 +72,11 @@ TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn
     }
     p.ksplit = best;
     p.items = p.m_tiles * best;
-    p.ticket_off = 4096;
-    p.partial_off = p.ticket_off + (((size_t)p.m_tiles * 32 * 4 + 255) / 256) * 256;
+    p.ticket_off = ws_bytes_for(kKernelBatch);      // behind everything the register-path kernels may write
+    // the counters' region is sized for the smallest tile (most row tiles), so that plans for different batch sizes
+    // sharing one workspace never put partial sums where another plan keeps counters
+    const size_t max_m_tiles = (d->row_groups + 7) / 8;
+    p.partial_off = p.ticket_off + ((max_m_tiles * 32 * 4 + 255) / 256) * 256;
     p.bytes = p.partial_off + (best > 1 ? (size_t)p.items * 32 * (p.npad / 2) * 32 * sizeof(float) : 0);
     return p;
 }

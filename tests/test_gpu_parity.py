@@ -271,3 +271,42 @@ def test_full_size_layer_matrix_sampled(hl, torch):
     # a property that holds at any size: y(-x) = -y exactly (sign flips commute with every rounding)
     yn = gpu_gemm(hl, torch, up, x ^ np.uint16(0x8000))
     assert np.array_equal(yn, -y)
+
+
+STRESS = [
+    # generator, chunk_elems — the distribution stress configuration at 4096 x 14336
+    ("student", 4096), ("uniform", 4096), ("patterns", 4096), ("gauss", 1024), ("gauss", 16384),
+]
+
+
+@pytest.mark.parametrize("gen,ce", STRESS)
+def test_distribution_stress_full_size(hl, torch, gen, ce):
+    """4096 x 14336 bf16: heavy tails with outlier rows, uniform exponents (worst compression), every bit pattern,
+    and the smallest / largest benchmark chunk sizes.  Decode is compared everywhere with the original tensor;
+    the fused product (finite inputs only) on sampled rows with the oracle."""
+    rows, cols = 4096, 14336
+    w = make(gen, rows, cols, 3000 + ce)
+    up = Uploaded(hl, torch, w, ce)
+    got = gpu_decode(hl, torch, up)
+    assert np.array_equal(got, w)
+    del got
+    if gen == "patterns":
+        return                                     # NaN / Inf weights: decode only
+    x = wl.activations(1, cols, 3500)
+    y = gpu_gemm(hl, torch, up, x)
+    rs = np.random.default_rng(1).choice(rows, 48, replace=False)
+    yo, d = orc.matmul(w[rs], x)
+    assert np.all(np.abs(y[0, rs] - yo[0]) <= TOL * d[0])
+
+
+@pytest.mark.parametrize("rows,cols", [(28672, 8192), (8192, 28672)])
+def test_ffn70b_shapes_small_batch_sampled(hl, torch, rows, cols):
+    """70B-FFN shapes at full size, batch 1 / 4 (register path) and 16 / 64 (tensor-core path), sampled rows."""
+    w = wl.gaussian_weights(rows, cols, 0.015, 4000 + rows)
+    rs = np.random.default_rng(2).choice(rows, 24, replace=False)
+    up = Uploaded(hl, torch, w, 4096, 0, 64)
+    for batch in (1, 4, 16, 64):
+        x = wl.activations(batch, cols, 4500 + batch)
+        y = gpu_gemm(hl, torch, up, x)
+        yo, d = orc.matmul(w[rs], x)
+        assert np.all(np.abs(y[:, rs] - yo) <= TOL * d), f"batch {batch}"
