@@ -110,7 +110,6 @@ huffllm_status add_matrix(KernelArgs *k, const huffllm_desc *desc, const void *b
     m.n_chunks = (uint32_t)desc->n_chunks;
     m.chunk_cols = desc->chunk_cols;
     m.col_chunks = desc->col_chunks;
-    m.chunk_base = k->total_chunks;
     k->total_chunks += m.n_chunks;
     k->lut_bits = desc->lut_bits;
     // a slot holds the W rows of a record; the window runs one row ahead of what it consumes, and that look-ahead
@@ -133,6 +132,27 @@ huffllm_status finish_args(KernelArgs *k, bool product, const DeviceInfo &dev, u
         return fail(HUFFLLM_ERR_UNSUPPORTED, "chunk records too large for shared memory (slot %u bytes)", k->slot_bytes);
     uint64_t g = k->total_chunks < (uint64_t)dev.sms ? k->total_chunks : (uint64_t)dev.sms;
     *grid = (uint32_t)(g < kMaxGrid ? g : kMaxGrid);
+    // deal the CTAs out to the matrices: one each, then always to the matrix with the most chunks per CTA, so that
+    // the largest piece is as small as it can be and no CTA works in two matrices
+    if (*grid < k->n_mats) return fail(HUFFLLM_ERR_UNSUPPORTED, "more matrices than SMs");
+    uint32_t cnt[kMaxMats];
+    for (uint32_t i = 0; i < k->n_mats; ++i) cnt[i] = 1;
+    for (uint32_t left = *grid - k->n_mats; left; --left) {
+        uint32_t best = k->n_mats;
+        for (uint32_t i = 0; i < k->n_mats; ++i) {
+            if (cnt[i] >= k->m[i].n_chunks) continue;
+            if (best == k->n_mats || (uint64_t)k->m[i].n_chunks * cnt[best] > (uint64_t)k->m[best].n_chunks * cnt[i]) best = i;
+        }
+        if (best == k->n_mats) break;
+        ++cnt[best];
+    }
+    uint32_t first = 0;
+    for (uint32_t i = 0; i < k->n_mats; ++i) {
+        k->m[i].cta_first = first;
+        k->m[i].cta_count = cnt[i];
+        first += cnt[i];
+    }
+    *grid = first;
     return HUFFLLM_OK;
 }
 

@@ -37,9 +37,8 @@ namespace huffllm {
 // LB = table index bits (the blobs' lut_bits): 8 or 9.
 //
 // One launch works through a LIST of matrices (A.n_mats, usually the matrices of one decoder layer that
-// may run together).  The chunks of all matrices form one long list that is cut into equal pieces, one
-// per CTA, so almost every CTA lies inside a single matrix and builds a single table; the few CTAs whose
-// piece crosses from one matrix into the next rebuild the table once, behind a CTA-wide barrier.
+// may run together).  The CTAs are dealt out to the matrices in proportion to their chunks, so every CTA
+// lies inside a single matrix, builds a single table and meets no CTA-wide barrier after set-up.
 template <int MODE, int LB, int THREADS>
 __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant__ KernelArgs A) {
     constexpr int R = LB == 8 ? 3 : 2;                       // decoder steps between two refill checks
@@ -72,19 +71,14 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     uint32_t phase = 0;            // bit s = parity of the next completion of this warp's barrier s
     bool waited_prior = false, failed = false;
 
-    // this CTA's piece of the list of all chunks
-    const uint32_t G = gridDim.x, TT = A.total_chunks;
-    auto cta_cut = [&](uint32_t c) -> uint32_t { return (uint32_t)((uint64_t)TT * c / G); };
-    const uint32_t piece_beg = cta_cut(blockIdx.x), piece_end = cta_cut(blockIdx.x + 1);
-    bool first_segment = true;
-
-#pragma unroll 1
-    for (uint32_t mi = 0; mi < A.n_mats; ++mi) {
+    // the matrix this CTA works in, and the CTA's piece of that matrix's chunks
+    uint32_t mi = 0;
+    while (mi + 1 < A.n_mats && blockIdx.x >= A.m[mi + 1].cta_first) ++mi;
+    {
         const MatArgs &k = A.m[mi];
-        if (piece_end <= k.chunk_base || piece_beg >= k.chunk_base + k.n_chunks) continue;
-        // ---- the part of matrix mi that this CTA works on, in the matrix's own chunk numbers
-        const uint32_t cta_beg = max(piece_beg, k.chunk_base) - k.chunk_base;
-        const uint32_t cta_end = min(piece_end, k.chunk_base + k.n_chunks) - k.chunk_base;
+        const uint32_t G = k.cta_count, J = blockIdx.x - k.cta_first;       // CTAs of this matrix, this CTA's number among them
+        auto cta_cut = [&](uint32_t j) -> uint32_t { return (uint32_t)((uint64_t)k.n_chunks * j / G); };
+        const uint32_t cta_beg = cta_cut(J), cta_end = cta_cut(J + 1);
         const uint32_t KC = k.col_chunks;
         uint32_t c_beg = cta_beg, c_end = cta_beg;
         if (warp < nw) {
@@ -134,8 +128,6 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
             issue(c_beg, 0);
             if (c_beg + 1 < c_end) issue(c_beg + 1, 1);
         }
-        if (!first_segment) __syncthreads();      // everybody is done with the previous matrix's table and counters
-        first_segment = false;
         {
             uint32_t *lut_s = (uint32_t *)(dyn_smem + (plan.lut - smem_base));
 #pragma unroll
@@ -160,15 +152,12 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         // memory.  Sums are always taken in the same order, and nobody waits for anybody.
         const uint32_t cta_len = cta_end - cta_beg;
         auto warp_beg = [&](uint32_t w) -> uint32_t { return cta_beg + cta_len * w / nw; };
-        auto cta_of_chunk = [&](uint32_t ch) -> uint32_t {     // ch = chunk number inside this matrix
-            const uint32_t gch = ch + k.chunk_base;
-            uint32_t c = (uint32_t)((uint64_t)gch * G / TT);
-            while (c + 1 < G && cta_cut(c + 1) <= gch) ++c;
-            while (c > 0 && cta_cut(c) > gch) --c;
+        auto cta_of_chunk = [&](uint32_t ch) -> uint32_t {     // which of the matrix's CTAs works on chunk ch
+            uint32_t c = (uint32_t)((uint64_t)ch * G / k.n_chunks);
+            while (c + 1 < G && cta_cut(c + 1) <= ch) ++c;
+            while (c > 0 && cta_cut(c) > ch) --c;
             return c;
         };
-        // first chunk of this matrix that CTA c works on
-        auto cta_first_chunk = [&](uint32_t c) -> uint32_t { return max(cta_cut(c), k.chunk_base) - k.chunk_base; };
         // lanes 0..vals-1 (looping if vals > 32) hold or produce the value of output o = column * 16 + row
         auto finish_cta_sum = [&](int rg, float (&v)[4]) {       // v[i] = value of output o = lane + 32 i
             const uint32_t g_lo = (uint32_t)rg * KC, g_hi = g_lo + KC;
@@ -186,7 +175,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 uint32_t o = lane + 32 * i;
-                if (o < vals) k.ws_partial[((size_t)blockIdx.x * 2 + my_slot) * vals + o] = v[i];
+                if (o < vals) k.ws_partial[((size_t)J * 2 + my_slot) * vals + o] = v[i];
             }
             __syncwarp();
             const uint32_t c0 = cta_of_chunk(g_lo), c1 = cta_of_chunk(g_hi - 1);
@@ -202,7 +191,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                 if (o >= vals) continue;
                 float sum = 0.f;
                 for (uint32_t c = c0; c <= c1; ++c) {
-                    uint32_t slot = cta_first_chunk(c) / KC == (uint32_t)rg ? 0u : 1u;
+                    uint32_t slot = cta_cut(c) / KC == (uint32_t)rg ? 0u : 1u;
                     sum += __ldcg(k.ws_partial + ((size_t)c * 2 + slot) * vals + o);
                 }
                 uint64_t r = (uint64_t)rg * 16 + (o & 15);

@@ -14,11 +14,11 @@ struct MatArgs {
     uint64_t rows, cols;
     uint32_t payload_units;    // payload size in 128-byte units
     uint32_t n_chunks, chunk_cols, col_chunks;
-    uint32_t chunk_base;       // number of chunks of the matrices in front of this one
+    uint32_t cta_first, cta_count;   // the CTAs of the launch that work on this matrix (each at least one chunk)
     const uint16_t *x;         // [batch][cols]
     float *y;                  // [batch][rows]
-    float *ws_partial;         // [grid * 2][16 * batch]
-    unsigned int *ws_ticket;   // [grid] arrival counters, zero between calls
+    float *ws_partial;         // [cta_count * 2][16 * batch]
+    unsigned int *ws_ticket;   // [cta_count] arrival counters, zero between calls
     uint16_t *out;             // decode output
 };
 
