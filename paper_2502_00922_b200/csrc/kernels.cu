@@ -26,6 +26,7 @@
 //     (shared memory inside a CTA, a scratch buffer plus a last-CTA pass across CTAs)
 #include <cuda_runtime.h>
 #include <cstdint>
+#include <type_traits>
 
 #include "decode_common.cuh"
 
@@ -310,11 +311,16 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                     const uint32_t last = nkb - 1;
 
                     // one block: start the fetch of the next block's raw bytes into `nxt`, decode with `cur`
-                    auto block = [&](uint32_t kb, const uint4 &cur, uint4 &nxt) {
+                    // (may_be_last = false: the caller knows that another block of this chunk follows)
+                    auto block = [&](uint32_t kb, const uint4 &cur, uint4 &nxt, auto may_be_last) {
                         BLOCKSTAMP((c - c_beg) * 8 + kb, 0);
                         raw_p += 512;
-                        if (kb == last) raw_p += coded_bytes;           // the next record's first block
-                        if (kb != last || next_ok) nxt = ldg_stream16(raw_p);
+                        if (decltype(may_be_last)::value) {
+                            if (kb == last) raw_p += coded_bytes;       // the next record's first block
+                            if (kb != last || next_ok) nxt = ldg_stream16(raw_p);
+                        } else {
+                            nxt = ldg_stream16(raw_p);
+                        }
                         uint4 xv;
                         if (MODE == 1) {
                             xv = __ldg((const uint4 *)xq);
@@ -345,10 +351,20 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                             }
                         }
                     };
+                    constexpr std::integral_constant<bool, false> inner{};
+                    constexpr std::integral_constant<bool, true> maybe_last{};
+                    uint32_t kb = 0;
 #pragma unroll 1
-                    for (uint32_t kb = 0; kb < nkb; kb += 2) {
-                        block(kb, raw_a, raw_b);
-                        if (kb + 1 < nkb) block(kb + 1, raw_b, raw_a);
+                    for (; kb + 4 <= nkb; kb += 4) {                    // the usual case: groups of four blocks
+                        block(kb, raw_a, raw_b, inner);
+                        block(kb + 1, raw_b, raw_a, inner);
+                        block(kb + 2, raw_a, raw_b, inner);
+                        block(kb + 3, raw_b, raw_a, maybe_last);
+                    }
+#pragma unroll 1
+                    for (; kb < nkb; kb += 2) {
+                        block(kb, raw_a, raw_b, maybe_last);
+                        if (kb + 1 < nkb) block(kb + 1, raw_b, raw_a, maybe_last);
                     }
                     if (nkb & 1u) raw_a = raw_b;     // the next chunk's first block always starts in raw_a
                     primed = next_ok;
