@@ -99,18 +99,18 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
             return r1 > r0 && r1 <= k.payload_units && (r1 - r0) * 128u > nkb * 512u &&
                    (r1 - r0) * 128u - nkb * 512u <= A.slot_bytes;
         };
-        // lane 0: start the bulk copy of a chunk's coded part into slot `which`
-        auto issue = [&](uint32_t c, uint32_t which) {
-            uint32_t nkb = blocks_of(c % KC), r0 = __ldg(index + c), r1 = __ldg(index + c + 1);
-            uint32_t bar = bar0 + which * 8;
-            if (record_ok(r0, r1, nkb)) {
-                uint32_t bytes = (r1 - r0) * 128u - nkb * 512u;
+        // lane 0: start the bulk copy of the coded part of a chunk (column chunk kc_c, record [ra, rb)) into slot `which`
+        auto issue_known = [&](uint32_t kc_c, uint32_t ra, uint32_t rb, uint32_t which) {
+            const uint32_t nkb = blocks_of(kc_c), bar = bar0 + which * 8;
+            if (record_ok(ra, rb, nkb)) {
+                uint32_t bytes = (rb - ra) * 128u - nkb * 512u;
                 mbar_expect_tx(bar, bytes);
-                bulk_g2s(slot0 + which * A.slot_bytes, payload + (uint64_t)r0 * 128u + nkb * 512u, bytes, bar);
+                bulk_g2s(slot0 + which * A.slot_bytes, payload + (uint64_t)ra * 128u + nkb * 512u, bytes, bar);
             } else {
                 mbar_expect_tx(bar, 0);  // completes the phase with nothing to wait for; the chunk is skipped below
             }
         };
+        auto issue = [&](uint32_t c, uint32_t which) { issue_known(c % KC, __ldg(index + c), __ldg(index + c + 1), which); };
 
         // ---- set-up of a segment.  The table loads are started first, then every warp starts its first
         // copies, then the table is written to shared memory: the cold misses on the table, on the record
@@ -370,7 +370,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                     primed = next_ok;
                 }
                 __syncwarp();
-                if (lane == 0 && c + 2 < c_end) issue(c + 2, which);
+                if (lane == 0 && c + 2 < c_end) issue_known(kc1 + 1 == KC ? 0u : kc1 + 1, r2, __ldg(index + c + 3), which);
                 r0 = r1;
                 r1 = r2;
                 kc = kc1;
