@@ -115,13 +115,13 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def prepare(workload: str, chunk_elems: int, hl, torch, dev, cpu_sample_mats: int = 0):
+def prepare(workload: str, chunk_elems: int, hl, torch, dev, cpu_sample_mats: int = 0, split: int = 0):
     """Generate, encode (host) and upload every matrix of the workload."""
     table, std, seed, _ = WORKLOADS[workload]
     mats = []
     for i, (name, rows, cols) in enumerate(table):
         w = wl.gaussian_weights(rows, cols, std, seed + i)
-        cb = hl.build_codebook(w)
+        cb = hl.build_codebook(w, hl.BF16, 0, split)
         blob, desc = hl.encode(cb, w, chunk_elems)
         cb.free()
         x = wl.activations(1, cols, seed + 500 + i)
@@ -199,6 +199,8 @@ def main():
     ap.add_argument("--chunk-elems", type=int, default=4096)
     ap.add_argument("--fuse", default="deps", choices=["none", "deps", "all"],
                     help="which matrices of the layer share a launch")
+    ap.add_argument("--split", default="paper", choices=["paper", "whole-exponent"],
+                    help="field split of the blobs: the paper's BF16 {1,4,4,7} or {1,8,7} (one 256-symbol exponent code)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -220,7 +222,8 @@ def main():
     args.warmup = max(args.warmup, 3)
 
     cpu_mats = 0 if (args.no_cpu_baseline or world > 1 or rank != 0) else 4      # whole matrices kept for the CPU-oracle leg
-    mats = prepare(args.workload, args.chunk_elems, hl, torch, dev, cpu_mats)
+    split = 0 if args.split == "paper" else 1
+    mats = prepare(args.workload, args.chunk_elems, hl, torch, dev, cpu_mats, split)
     err = torch.zeros(1, dtype=torch.int32, device=dev)
     n_weights = sum(m["rows"] * m["cols"] for m in mats)
     unc_bytes = 2 * n_weights
@@ -347,6 +350,7 @@ def main():
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
         "config": {"workload": args.workload, "what": WORKLOADS[args.workload][3], "chunk_elems": args.chunk_elems,
+                   "split": "bf16 {1,4,4,7}" if args.split == "paper" else "bf16 {1,8,7} (whole exponent)",
                    "max_code_len": int(mats[0]["desc"].lut_bits), "weights_per_step": n_weights,
                    "uncompressed_bytes": unc_bytes, "compressed_bytes": sum(m["blob_bytes"] for m in mats),
                    "compression_ratio_total": unc_bytes / sum(m["blob_bytes"] for m in mats),

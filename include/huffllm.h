@@ -40,6 +40,15 @@ typedef enum {
 
 typedef enum { HUFFLLM_BF16 = 0, HUFFLLM_FP16 = 1 } huffllm_dtype;
 
+/* How a weight's bits are grouped into coded fields.
+ *   HUFFLLM_SPLIT_PAPER           the paper's hardware-friendly splits: BF16 {1,4,4,7} (Section 5.1)
+ *   HUFFLLM_SPLIT_WHOLE_EXPONENT  BF16 {1,8,7}: the 8-bit exponent is one symbol of a 256-symbol code.  The
+ *                                 paper's entropy table lists this split and Section 3.1 sets it aside because a
+ *                                 256-entry CAM is too costly in its hardware decoder; a lookup table in GPU
+ *                                 shared memory has no such cost, so the split is offered here.  The device
+ *                                 kernels are the same: they see only the table.                              */
+typedef enum { HUFFLLM_SPLIT_PAPER = 0, HUFFLLM_SPLIT_WHOLE_EXPONENT = 1 } huffllm_split;
+
 /* A CUDA stream handle (cudaStream_t), spelled without the CUDA headers. */
 typedef struct CUstream_st *huffllm_stream;
 
@@ -52,12 +61,14 @@ typedef struct huffllm_codebook huffllm_codebook;
  *
  * Blob layout (every section starts on a 256-byte boundary):
  *   header    this struct
- *   codebook  uint8 lengths[3][32]; 0 = symbol unused; codewords are canonical: symbols ordered by
+ *   codebook  n_fields == 2: uint8 lengths[3][32] (hi-nibble code, lo-nibble code, zeros);
+ *             n_fields == 1: uint8 lengths[256] of the whole-exponent code.
+ *             0 = symbol unused; codewords are canonical: symbols ordered by
  *             (length, symbol), first codeword 0, next = (previous + 1) << (length growth); a
  *             codeword's most significant bit comes first in the stream
  *   LUT       uint32[1 << lut_bits], indexed by the next lut_bits stream bits (first bit = bit 0);
- *             BF16 entry = (length of hi-nibble code + length of lo-nibble code) << 16 | exponent << 7,
- *             i.e. the exponent already sits where a bf16 word has it
+ *             BF16 entry = (code length of the weight: hi-nibble + lo-nibble code, or the whole-exponent
+ *             code) << 16 | exponent << 7, i.e. the exponent already sits where a bf16 word has it
  *   index     uint32[n_chunks + 1]: record offsets from off_payload, in units of 128 bytes
  *   payload   one record per chunk, chunk id = row_group * col_chunks + col_chunk
  *
@@ -70,7 +81,8 @@ typedef struct huffllm_codebook huffllm_codebook;
  * mantissa; a lane's 16 bytes are row g's eight weights, then row g + 8's), then W rows of 64
  * little-endian uint32 (row j, sequence s): the sequence's bits, bit i in word i / 32 at bit
  * i % 32.  A sequence starts with `lag_bits` zero bits, then for every weight
- * code(exponent >> 4) code(exponent & 15); bits after the last codeword are zero.  W is the
+ * code(exponent >> 4) code(exponent & 15) (n_fields == 2) or code(exponent) (n_fields == 1); bits after
+ * the last codeword are zero.  W is the
  * longest sequence of the chunk in words (all 64 are padded to it).
  */
 typedef struct huffllm_desc {
@@ -86,7 +98,7 @@ typedef struct huffllm_desc {
     uint64_t n_chunks;        /* row_groups * col_chunks                                   */
     uint32_t lut_bits;        /* L_max of one weight's coded fields together (8 .. 12)     */
     uint32_t lag_bits;        /* 7                                                         */
-    uint32_t n_fields;        /* coded fields per weight: 2 (BF16)                         */
+    uint32_t n_fields;        /* coded fields per weight: 2 (BF16 {1,4,4,7}) or 1 ({1,8,7}) */
     uint8_t  caps[4];         /* per-field maximum code length chosen under lut_bits       */
     uint16_t pad_word;        /* weight stored at positions outside the tensor            */
     uint16_t reserved0;
@@ -114,6 +126,20 @@ typedef struct huffllm_desc {
  */
 huffllm_status huffllm_build_codebook(const uint16_t *w_host, uint64_t rows, uint64_t cols, huffllm_dtype dtype,
                                       uint32_t max_code_len, huffllm_codebook **out);
+
+/*
+ * The same for a chosen field split.  HUFFLLM_SPLIT_PAPER is huffllm_build_codebook.  With
+ * HUFFLLM_SPLIT_WHOLE_EXPONENT (BF16 only) the exponent byte is coded by one Huffman code of at most
+ * max_code_len bits (0 = 8; range 8..12; the optimal length-limited code when plain Huffman is longer);
+ * blobs encoded with it have n_fields == 1 and run through the same device calls.
+ */
+huffllm_status huffllm_build_codebook_split(const uint16_t *w_host, uint64_t rows, uint64_t cols, huffllm_dtype dtype,
+                                            huffllm_split split, uint32_t max_code_len, huffllm_codebook **out);
+
+/* Read the code of a whole-exponent codebook: per exponent value its count, code length (0 = unused) and
+ * canonical codeword.  Arrays hold 256 entries.  INVALID_ARG for a codebook of another split.        */
+huffllm_status huffllm_codebook_get_exponent(const huffllm_codebook *cb, uint64_t counts[256], uint8_t lengths[256],
+                                             uint32_t codes[256]);
 
 /* Read one field of a codebook: number of symbols of the field's alphabet, and per symbol its
  * count, code length (0 = unused) and canonical codeword.  Arrays hold 32 entries.            */

@@ -13,6 +13,9 @@
  *     mantissa bits each coded by its own Huffman code      (Section 3.1)
  *   - field split BF16 {1,4,4,7}: sign and the seven mantissa bits raw; the
  *     8-bit exponent is coded as two 4-bit groups            (Section 5.1)
+ *   - BF16 with the exponent coded whole, {1,8,7}: one 256-symbol code; the
+ *     split the paper's entropy table lists and sets aside because a 256-entry
+ *     CAM is too large for its hardware decoder              (Section 3.1, entropy table)
  *   - decoder: compare the bits at the start pointer with every stored codeword,
  *     emit the matching symbol, advance the pointer by that codeword's length
  *                                                           (Section 3.2, decoder figure)
@@ -37,24 +40,30 @@
 #include <string.h>
 #include <math.h>
 
-#define ORC_MAXSYM 32
-#define ORC_BF16 0
-#define ORC_FP16 1
+#define ORC_MAXSYM 256
+#define ORC_BF16 0      /* {1,4,4,7} */
+#define ORC_FP16 1      /* {1,5,5,5} */
+#define ORC_BF16_E8 2   /* {1,8,7}: BF16 numbers, exponent coded as one 8-bit symbol */
 
 /* ------------------------------------------------------------------ fields */
 
-int orc_num_fields(int dtype) { return dtype == ORC_BF16 ? 2 : 3; }
-int orc_field_symbols(int dtype) { return dtype == ORC_BF16 ? 16 : 32; }
-int orc_raw_bits(int dtype) { return dtype == ORC_BF16 ? 8 : 1; }
+int orc_num_fields(int dtype) { return dtype == ORC_BF16 ? 2 : dtype == ORC_FP16 ? 3 : 1; }
+int orc_field_symbols(int dtype) { return dtype == ORC_BF16 ? 16 : dtype == ORC_FP16 ? 32 : 256; }
+int orc_raw_bits(int dtype) { return dtype == ORC_FP16 ? 1 : 8; }
 
 /* Split one 16-bit word into its coded fields f[] and its raw (uncoded) bits.
  * BF16: word = s(1) E(8) m(7);  f0 = E>>4, f1 = E&15, raw = s<<7 | m.
- * FP16: word = s(1) E(5) M(10); f0 = E, f1 = M>>5, f2 = M&31, raw = s.      */
+ * FP16: word = s(1) E(5) M(10); f0 = E, f1 = M>>5, f2 = M&31, raw = s.
+ * BF16 whole exponent: f0 = E, raw = s<<7 | m.                               */
 void orc_split(int dtype, uint16_t b, uint8_t f[3], uint8_t *raw)
 {
     if (dtype == ORC_BF16) {
         unsigned s = b >> 15, e = (b >> 7) & 0xFF, m = b & 0x7F;
         f[0] = (uint8_t)(e >> 4); f[1] = (uint8_t)(e & 15); f[2] = 0;
+        *raw = (uint8_t)((s << 7) | m);
+    } else if (dtype == ORC_BF16_E8) {
+        unsigned s = b >> 15, e = (b >> 7) & 0xFF, m = b & 0x7F;
+        f[0] = (uint8_t)e; f[1] = 0; f[2] = 0;
         *raw = (uint8_t)((s << 7) | m);
     } else {
         unsigned s = b >> 15, e = (b >> 10) & 31, m = b & 0x3FF;
@@ -68,6 +77,9 @@ uint16_t orc_join(int dtype, const uint8_t f[3], uint8_t raw)
     if (dtype == ORC_BF16) {
         unsigned s = raw >> 7, m = raw & 0x7F, e = ((unsigned)f[0] << 4) | f[1];
         return (uint16_t)((s << 15) | (e << 7) | m);
+    } else if (dtype == ORC_BF16_E8) {
+        unsigned s = raw >> 7, m = raw & 0x7F;
+        return (uint16_t)((s << 15) | ((unsigned)f[0] << 7) | m);
     } else {
         unsigned s = raw & 1, m = ((unsigned)f[1] << 5) | f[2];
         return (uint16_t)((s << 15) | ((unsigned)f[0] << 10) | m);
@@ -184,7 +196,7 @@ uint64_t orc_code_cost(const uint64_t *counts, const uint8_t *len, int nsym)
 
 /* Code lengths for all coded fields of a tensor under a length budget.
  * budget == 0: unrestricted Huffman for every field.
- * FP16: every field is limited to `budget` on its own.
+ * FP16 and BF16 whole exponent: every field is limited to `budget` on its own.
  * BF16: the two exponent nibbles of one weight are decoded together, so the
  *       budget bounds the SUM of the two fields' maximum lengths: choose caps
  *       (c0, c1), c0 + c1 <= budget, minimising the total coded bits; ties go to
@@ -200,7 +212,7 @@ int orc_build_lengths(int dtype, const uint64_t counts[3][ORC_MAXSYM], int budge
         for (int k = 0; k < nf; ++k) if (orc_huffman_lengths(counts[k], ns, len[k]) == 0) return -1;
         return 0;
     }
-    if (dtype == ORC_FP16) {
+    if (dtype != ORC_BF16) {
         for (int k = 0; k < nf; ++k) {
             if (orc_limited_lengths(counts[k], ns, budget, len[k]) <= 0) return -1;
             caps[k] = budget;
@@ -316,7 +328,7 @@ int64_t orc_decode_sequences(int dtype, const uint8_t *bits, const uint64_t *bit
  * with the IEEE conventions for E == 0 and E == all ones).                    */
 double orc_value(int dtype, uint16_t b)
 {
-    int ebits = dtype == ORC_BF16 ? 8 : 5, mbits = dtype == ORC_BF16 ? 7 : 10;
+    int ebits = dtype == ORC_FP16 ? 5 : 8, mbits = dtype == ORC_FP16 ? 10 : 7;
     int bias = (1 << (ebits - 1)) - 1, emax = (1 << ebits) - 1;
     int s = b >> 15, e = (b >> mbits) & emax, m = b & ((1 << mbits) - 1);
     double sign = s ? -1.0 : 1.0, frac = (double)m / (double)(1 << mbits);

@@ -23,8 +23,8 @@ import subprocess
 
 import numpy as np
 
-BF16, FP16 = 0, 1
-MAXSYM = 32
+BF16, FP16, BF16_E8 = 0, 1, 2     # BF16_E8: bf16 numbers with the exponent coded whole (one 256-symbol field)
+MAXSYM = 256
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "huffllm_oracle.c")
 _SO = os.path.join(_HERE, "liboracle.so")
@@ -68,11 +68,11 @@ def _p(a, t):
 # ----------------------------------------------------------------- codebooks
 
 def num_fields(dtype):
-    return 2 if dtype == BF16 else 3
+    return {BF16: 2, FP16: 3, BF16_E8: 1}[dtype]
 
 
 def field_symbols(dtype):
-    return 16 if dtype == BF16 else 32
+    return {BF16: 16, FP16: 32, BF16_E8: 256}[dtype]
 
 
 def histogram(w: np.ndarray, dtype=BF16) -> np.ndarray:
@@ -101,7 +101,7 @@ def code_cost(counts, lengths) -> int:
 
 
 def build_lengths(counts: np.ndarray, dtype=BF16, budget: int = 0):
-    """Code lengths [3][32] and the per-field caps chosen under `budget` (0 = unrestricted)."""
+    """Code lengths [3][MAXSYM] and the per-field caps chosen under `budget` (0 = unrestricted)."""
     counts = np.ascontiguousarray(counts, dtype=np.uint64)
     lens = np.zeros((3, MAXSYM), dtype=np.uint8)
     caps = (C.c_int * 3)()
@@ -231,12 +231,13 @@ def element_map(rows: int, cols: int, chunk_elems: int):
 def pad_word(lens: np.ndarray, dtype=BF16) -> int:
     """The weight written at positions outside the tensor: every coded field takes its shortest codeword
     (ties: smallest symbol), raw bits zero."""
-    assert dtype == BF16
+    assert dtype in (BF16, BF16_E8)
     f = []
-    for k in range(2):
-        used = [(int(lens[k][s]), s) for s in range(16) if lens[k][s]]
+    for k in range(num_fields(dtype)):
+        used = [(int(lens[k][s]), s) for s in range(field_symbols(dtype)) if lens[k][s]]
         f.append(min(used)[1])
-    return ((f[0] << 4 | f[1]) << 7) & 0xFFFF
+    e = (f[0] << 4 | f[1]) if dtype == BF16 else f[0]
+    return (e << 7) & 0xFFFF
 
 
 def encode_tensor(w: np.ndarray, chunk_elems: int = 4096, budget: int = 8, dtype=BF16):
@@ -280,8 +281,9 @@ def decode_tensor(enc) -> np.ndarray:
 #   56 u32 lut_bits | 60 u32 lag_bits | 64 u32 n_fields | 68 u8 caps[4] | 72 u16 pad_word | 74 u16 0
 #   76 u32 max_words | 80 u64 off_codebook | 88 u64 off_lut | 96 u64 off_index | 104 u64 off_payload
 #   112 u64 payload_bytes | 120 u64 blob_bytes | 128 u64 coded_bits | 136 u64 raw_bits | 144 u64 checksum
-# codebook: u8 lengths[3][32].  LUT: u32[1 << lut_bits], entry = (len0 + len1) << 16 | E << 7, indexed by the
-# next lut_bits stream bits (first bit = bit 0).  index: u32[n_chunks + 1], record offsets in 128-byte
+# codebook: n_fields == 2: u8 lengths[3][32] (two nibble codes, third row zero); n_fields == 1: u8 lengths[256]
+# of the whole-exponent code.  LUT: u32[1 << lut_bits], entry = (code length of the weight) << 16 | E << 7,
+# indexed by the next lut_bits stream bits (first bit = bit 0).  index: u32[n_chunks + 1], record offsets in 128-byte
 # units from off_payload.  Record of a chunk with nkb blocks: raw bytes [nkb][32 lanes][16] (a lane's 16
 # bytes: row g's eight weights, then row g+8's), then W rows of 64 little-endian u32 (row j, sequence s):
 # the sequence's bits, bit i in word i // 32 at bit i % 32, starting with LAG_BITS zero bits; unused bits
@@ -308,13 +310,19 @@ def parse_blob(blob) -> dict:
     h = parse_header(blob)
     rows, cols, ce, dtype = h["rows"], h["cols"], h["chunk_elems"], h["dtype"]
     assert dtype == BF16, "reader covers bf16 blobs"
+    assert h["n_fields"] in (1, 2)
+    scheme = BF16 if h["n_fields"] == 2 else BF16_E8          # how the exponent is coded
     geo = geometry(rows, cols, ce)
     assert (h["tile_rows"], h["chunk_cols"], h["row_groups"], h["col_chunks"]) == (16, geo["Kc"], geo["RG"], geo["KC"])
-    assert h["n_chunks"] == geo["RG"] * geo["KC"] and h["lag_bits"] == LAG_BITS and h["n_fields"] == 2
+    assert h["n_chunks"] == geo["RG"] * geo["KC"] and h["lag_bits"] == LAG_BITS
     assert h["blob_bytes"] == len(blob)
     for k in ("off_codebook", "off_lut", "off_index", "off_payload"):
         assert h[k] % 256 == 0
-    lens = np.frombuffer(blob, dtype=np.uint8, count=96, offset=h["off_codebook"]).reshape(3, 32).copy()
+    lens = np.zeros((3, MAXSYM), dtype=np.uint8)
+    if scheme == BF16:
+        lens[:, :32] = np.frombuffer(blob, dtype=np.uint8, count=96, offset=h["off_codebook"]).reshape(3, 32)
+    else:
+        lens[0] = np.frombuffer(blob, dtype=np.uint8, count=256, offset=h["off_codebook"])
     codes = codes_for(lens)
     lut = np.frombuffer(blob, dtype=np.uint32, count=1 << h["lut_bits"], offset=h["off_lut"]).copy()
     index = np.frombuffer(blob, dtype=np.uint32, count=h["n_chunks"] + 1, offset=h["off_index"]).astype(np.int64)
@@ -338,7 +346,7 @@ def parse_blob(blob) -> dict:
             body = np.ascontiguousarray(seq_bits[:, LAG_BITS:])
             off = (np.arange(SEQS + 1, dtype=np.uint64) * np.uint64(body.shape[1]))
             chunks[int(cid)] = (body.ravel(), off, raw)
-    enc = dict(rows=rows, cols=cols, chunk_elems=ce, dtype=dtype, lens=lens, codes=codes, caps=list(h["caps"][:3]),
+    enc = dict(rows=rows, cols=cols, chunk_elems=ce, dtype=scheme, lens=lens, codes=codes, caps=list(h["caps"][:3]),
                pad=h["pad_word"], chunks=chunks, header=h, lut=lut)
     assert max_words == h["max_words"]
     return enc
@@ -367,9 +375,9 @@ def decode_blob(blob):
     return out[:-1].reshape(rows, cols), used_all
 
 
-def lut_from_code(lens, codes, lut_bits: int) -> np.ndarray:
+def lut_from_code(lens, codes, lut_bits: int, dtype=BF16) -> np.ndarray:
     """What the blob's LUT must contain, found the slow way: for every index, write its bits out as a
-    stream and run one bit-serial decode of a single weight (both nibble fields) on it."""
+    stream and run one bit-serial decode of a single weight (all its coded fields) on it."""
     n = 1 << lut_bits
     idx_bits = ((np.arange(n, dtype=np.uint32)[:, None] >> np.arange(lut_bits, dtype=np.uint32)) & 1).astype(np.uint8)
     out = np.zeros(n, dtype=np.uint32)
@@ -377,7 +385,7 @@ def lut_from_code(lens, codes, lut_bits: int) -> np.ndarray:
     for i in range(n):
         off = np.array([0, lut_bits], dtype=np.uint64)
         try:
-            seq, used = decode_sequences(idx_bits[i], off, raw, lens, codes, BF16)
+            seq, used = decode_sequences(idx_bits[i], off, raw, lens, codes, dtype)
         except ValueError:
             continue                                   # no codeword pair is a prefix of this index
         out[i] = (int(used[0]) << 16) | (((int(seq[0, 0]) >> 7) & 0xFF) << 7)

@@ -7,6 +7,7 @@ import os
 import numpy as np
 
 BF16, FP16 = 0, 1
+SPLIT_PAPER, SPLIT_WHOLE_EXPONENT = 0, 1
 _SO = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libhuffllm.so")
 _lib = None
 
@@ -37,6 +38,8 @@ assert C.sizeof(Desc) == 256
 
 _SIGNATURES = {
     "huffllm_build_codebook": [C.c_void_p, C.c_uint64, C.c_uint64, C.c_int, C.c_uint32, C.POINTER(C.c_void_p)],
+    "huffllm_build_codebook_split": [C.c_void_p, C.c_uint64, C.c_uint64, C.c_int, C.c_int, C.c_uint32, C.POINTER(C.c_void_p)],
+    "huffllm_codebook_get_exponent": [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
     "huffllm_codebook_get": [C.c_void_p, C.c_uint32, C.POINTER(C.c_uint32), C.c_void_p, C.c_void_p, C.c_void_p],
     "huffllm_codebook_free": [C.c_void_p],
     "huffllm_encode_bound": [C.c_uint64, C.c_uint64, C.c_int, C.c_uint32, C.POINTER(C.c_size_t)],
@@ -121,6 +124,14 @@ class Codebook:
         _check(lib().huffllm_codebook_get(self._h, field, C.byref(n), counts.ctypes.data, lengths.ctypes.data, codes.ctypes.data))
         return n.value, counts, lengths, codes
 
+    def get_exponent(self):
+        """Whole-exponent codebooks: (counts, lengths, codes), 256 entries each."""
+        counts = np.zeros(256, np.uint64)
+        lengths = np.zeros(256, np.uint8)
+        codes = np.zeros(256, np.uint32)
+        _check(lib().huffllm_codebook_get_exponent(self._h, counts.ctypes.data, lengths.ctypes.data, codes.ctypes.data))
+        return counts, lengths, codes
+
     def free(self):
         if self._h:
             lib().huffllm_codebook_free(self._h)
@@ -133,11 +144,14 @@ class Codebook:
             pass
 
 
-def build_codebook(w: np.ndarray, dtype: int = BF16, max_code_len: int = 0) -> Codebook:
+def build_codebook(w: np.ndarray, dtype: int = BF16, max_code_len: int = 0, split: int = SPLIT_PAPER) -> Codebook:
     w = np.ascontiguousarray(w, dtype=np.uint16)
     rows, cols = w.shape if w.ndim == 2 else (1, w.size)
     h = C.c_void_p()
-    _check(lib().huffllm_build_codebook(w.ctypes.data, rows, cols, dtype, max_code_len, C.byref(h)))
+    if split == SPLIT_PAPER:
+        _check(lib().huffllm_build_codebook(w.ctypes.data, rows, cols, dtype, max_code_len, C.byref(h)))
+    else:
+        _check(lib().huffllm_build_codebook_split(w.ctypes.data, rows, cols, dtype, split, max_code_len, C.byref(h)))
     return Codebook(h)
 
 

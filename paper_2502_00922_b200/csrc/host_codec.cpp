@@ -46,7 +46,7 @@ huffllm_status check_desc(const huffllm_desc *d) {
     if (d->chunk_elems % (kTileRows * kBlockCols) || d->chunk_elems < 512 || d->chunk_elems > 16384)
         return fail(HUFFLLM_ERR_CORRUPT, "bad chunk_elems");
     if (d->tile_rows != kTileRows || d->chunk_cols != d->chunk_elems / kTileRows || d->lag_bits != kLagBits ||
-        d->n_fields != 2)
+        (d->n_fields != 2 && d->n_fields != 1))
         return fail(HUFFLLM_ERR_CORRUPT, "bad tile geometry");
     if (d->row_groups != (d->rows + kTileRows - 1) / kTileRows ||
         d->col_chunks != (d->cols + d->chunk_cols - 1) / d->chunk_cols ||
@@ -57,7 +57,7 @@ huffllm_status check_desc(const huffllm_desc *d) {
     uint32_t w_bound = (kLagBits + max_steps * d->lut_bits + 31) / 32;
     if (d->max_words == 0 || d->max_words > w_bound) return fail(HUFFLLM_ERR_CORRUPT, "bad max_words");
     if (d->off_codebook % 256 || d->off_lut % 256 || d->off_index % 256 || d->off_payload % 256 ||
-        d->off_codebook < 256 || d->off_lut < d->off_codebook + 96 ||
+        d->off_codebook < 256 || d->off_lut < d->off_codebook + (d->n_fields == 1 ? 256u : 96u) ||
         d->off_index < d->off_lut + (4ull << d->lut_bits) || d->off_payload < d->off_index + 4 * (d->n_chunks + 1) ||
         d->payload_bytes % kRecordUnit || d->blob_bytes < d->off_payload + d->payload_bytes ||
         d->payload_bytes / kRecordUnit > 0xFFFFFFFFull)
@@ -143,9 +143,13 @@ using namespace huffllm;
 
 struct huffllm_codebook {
     uint32_t dtype, budget;
+    uint32_t n_fields;       // 2: hi/lo nibble codes (len, code);  1: one code for the exponent byte (len_e, code_e)
     uint64_t counts[3][32];
     uint8_t len[3][32];
     uint32_t code[3][32];
+    uint64_t counts_e[256];
+    uint8_t len_e[256];
+    uint32_t code_e[256];
     uint8_t caps[4];
     uint16_t pad_word;
     uint8_t len8[256];    // code length of a whole exponent byte (hi + lo), 0 = no codeword
@@ -159,24 +163,58 @@ static void finish_codebook(huffllm_codebook *cb) {
     memset(cb->bits8, 0, sizeof(cb->bits8));
     cb->lut.assign((size_t)1 << cb->budget, 0u);
     for (int e = 0; e < 256; ++e) {
-        int h = e >> 4, l = e & 15;
-        int lh = cb->len[0][h], ll = cb->len[1][l];
-        if (!lh || !ll) continue;
-        uint32_t seq = reverse_bits(cb->code[0][h], lh) | (reverse_bits(cb->code[1][l], ll) << lh);
-        int L = lh + ll;
+        uint32_t seq;
+        int L;
+        if (cb->n_fields == 2) {
+            int h = e >> 4, l = e & 15;
+            int lh = cb->len[0][h], ll = cb->len[1][l];
+            if (!lh || !ll) continue;
+            seq = reverse_bits(cb->code[0][h], lh) | (reverse_bits(cb->code[1][l], ll) << lh);
+            L = lh + ll;
+        } else {
+            L = cb->len_e[e];
+            if (!L) continue;
+            seq = reverse_bits(cb->code_e[e], L);
+        }
         cb->len8[e] = (uint8_t)L;
         cb->bits8[e] = seq;
         for (uint32_t hi = 0; hi < (1u << (cb->budget - L)); ++hi)
             cb->lut[seq | (hi << L)] = ((uint32_t)L << 16) | ((uint32_t)e << 7);
     }
-    int f[2];
-    for (int k = 0; k < 2; ++k) {
+    // pad word: every coded field takes its shortest codeword (ties: the smallest symbol)
+    if (cb->n_fields == 2) {
+        int f[2];
+        for (int k = 0; k < 2; ++k) {
+            int best = -1;
+            for (int s = 0; s < 16; ++s)
+                if (cb->len[k][s] && (best < 0 || cb->len[k][s] < cb->len[k][best])) best = s;
+            f[k] = best;
+        }
+        cb->pad_word = (uint16_t)(((f[0] << 4) | f[1]) << 7);
+    } else {
         int best = -1;
-        for (int s = 0; s < 16; ++s)
-            if (cb->len[k][s] && (best < 0 || cb->len[k][s] < cb->len[k][best])) best = s;
-        f[k] = best;
+        for (int e = 0; e < 256; ++e)
+            if (cb->len_e[e] && (best < 0 || cb->len_e[e] < cb->len_e[best])) best = e;
+        cb->pad_word = (uint16_t)(best << 7);
     }
-    cb->pad_word = (uint16_t)(((f[0] << 4) | f[1]) << 7);
+}
+
+// Histogram of the exponent byte of a bf16 tensor, threaded over slices.
+static void exponent_histogram(const uint16_t *w, uint64_t n, uint64_t hist[256]) {
+    unsigned nt = std::max(1u, std::min(16u, std::thread::hardware_concurrency()));
+    if (n < (1u << 20)) nt = 1;
+    std::vector<std::vector<uint64_t>> part(nt, std::vector<uint64_t>(256, 0));
+    std::vector<std::thread> th;
+    for (unsigned t = 0; t < nt; ++t)
+        th.emplace_back([&, t] {
+            uint64_t a = n * t / nt, b = n * (t + 1) / nt;
+            uint64_t *h = part[t].data();
+            for (uint64_t i = a; i < b; ++i) h[(w[i] >> 7) & 0xFF]++;
+        });
+    for (auto &x : th) x.join();
+    memset(hist, 0, 256 * sizeof(uint64_t));
+    for (unsigned t = 0; t < nt; ++t)
+        for (int e = 0; e < 256; ++e) hist[e] += part[t][e];
 }
 
 extern "C" {
@@ -201,24 +239,13 @@ huffllm_status huffllm_build_codebook(const uint16_t *w, uint64_t rows, uint64_t
     memset(cb->code, 0, sizeof(cb->code));
     memset(cb->caps, 0, sizeof(cb->caps));
 
-    // histogram of the exponent byte, threaded over slices, then folded into the two nibble fields
-    const uint64_t n = rows * cols;
-    unsigned nt = std::max(1u, std::min(16u, std::thread::hardware_concurrency()));
-    if (n < (1u << 20)) nt = 1;
-    std::vector<std::vector<uint64_t>> part(nt, std::vector<uint64_t>(256, 0));
-    std::vector<std::thread> th;
-    for (unsigned t = 0; t < nt; ++t)
-        th.emplace_back([&, t] {
-            uint64_t a = n * t / nt, b = n * (t + 1) / nt;
-            uint64_t *h = part[t].data();
-            for (uint64_t i = a; i < b; ++i) h[(w[i] >> 7) & 0xFF]++;
-        });
-    for (auto &x : th) x.join();
-    for (unsigned t = 0; t < nt; ++t)
-        for (int e = 0; e < 256; ++e) {
-            cb->counts[0][e >> 4] += part[t][e];
-            cb->counts[1][e & 15] += part[t][e];
-        }
+    // histogram of the exponent byte, folded into the two nibble fields
+    cb->n_fields = 2;
+    exponent_histogram(w, rows * cols, cb->counts_e);
+    for (int e = 0; e < 256; ++e) {
+        cb->counts[0][e >> 4] += cb->counts_e[e];
+        cb->counts[1][e & 15] += cb->counts_e[e];
+    }
 
     bool have = false;
     uint64_t best = 0;
@@ -247,10 +274,53 @@ huffllm_status huffllm_build_codebook(const uint16_t *w, uint64_t rows, uint64_t
     return HUFFLLM_OK;
 }
 
+huffllm_status huffllm_build_codebook_split(const uint16_t *w, uint64_t rows, uint64_t cols, huffllm_dtype dtype,
+                                            huffllm_split split, uint32_t max_code_len, huffllm_codebook **out) {
+    if (split == HUFFLLM_SPLIT_PAPER) return huffllm_build_codebook(w, rows, cols, dtype, max_code_len, out);
+    clear_error();
+    if (split != HUFFLLM_SPLIT_WHOLE_EXPONENT) return fail(HUFFLLM_ERR_INVALID_ARG, "bad split");
+    if (!w || !out || rows == 0 || cols == 0) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer or empty tensor");
+    if (dtype != HUFFLLM_BF16) return fail(HUFFLLM_ERR_UNSUPPORTED, "the whole-exponent split is for bf16");
+    uint32_t budget = max_code_len ? max_code_len : kDefaultBudget;
+    if (budget < kMinBudget || budget > kMaxBudget)
+        return fail(HUFFLLM_ERR_UNSUPPORTED, "max_code_len must be 0 or in [%u, %u]", kMinBudget, kMaxBudget);
+    huffllm_codebook *cb = new (std::nothrow) huffllm_codebook();
+    if (!cb) return fail(HUFFLLM_ERR_NOMEM, "out of host memory");
+    cb->dtype = dtype;
+    cb->budget = budget;
+    cb->n_fields = 1;
+    memset(cb->counts, 0, sizeof(cb->counts));
+    memset(cb->len, 0, sizeof(cb->len));
+    memset(cb->code, 0, sizeof(cb->code));
+    memset(cb->caps, 0, sizeof(cb->caps));
+    exponent_histogram(w, rows * cols, cb->counts_e);
+    if (!limited_lengths(cb->counts_e, 256, (int)budget, cb->len_e)) {
+        delete cb;
+        return fail(HUFFLLM_ERR_INVALID_ARG, "no code fits max_code_len");
+    }
+    cb->caps[0] = (uint8_t)budget;
+    canonical_codes(cb->len_e, 256, cb->code_e);
+    finish_codebook(cb);
+    *out = cb;
+    return HUFFLLM_OK;
+}
+
+huffllm_status huffllm_codebook_get_exponent(const huffllm_codebook *cb, uint64_t counts[256], uint8_t lengths[256],
+                                             uint32_t codes[256]) {
+    clear_error();
+    if (!cb || cb->n_fields != 1) return fail(HUFFLLM_ERR_INVALID_ARG, "not a whole-exponent codebook");
+    for (int e = 0; e < 256; ++e) {
+        if (counts) counts[e] = cb->counts_e[e];
+        if (lengths) lengths[e] = cb->len_e[e];
+        if (codes) codes[e] = cb->code_e[e];
+    }
+    return HUFFLLM_OK;
+}
+
 huffllm_status huffllm_codebook_get(const huffllm_codebook *cb, uint32_t field, uint32_t *n_symbols, uint64_t counts[32],
                                     uint8_t lengths[32], uint32_t codes[32]) {
     clear_error();
-    if (!cb || field >= 2) return fail(HUFFLLM_ERR_INVALID_ARG, "bad codebook or field");
+    if (!cb || cb->n_fields != 2 || field >= 2) return fail(HUFFLLM_ERR_INVALID_ARG, "bad codebook or field");
     if (n_symbols) *n_symbols = 16;
     for (int s = 0; s < 32; ++s) {
         if (counts) counts[s] = cb->counts[field][s];
@@ -361,7 +431,7 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
     d.n_chunks = n_chunks;
     d.lut_bits = cb->budget;
     d.lag_bits = kLagBits;
-    d.n_fields = 2;
+    d.n_fields = cb->n_fields;
     memcpy(d.caps, cb->caps, 4);
     d.pad_word = cb->pad_word;
     d.off_codebook = 256;
@@ -417,7 +487,11 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
 
     memset(base, 0, d.off_payload);
     memcpy(base, &d, sizeof(d));
-    for (int k = 0; k < 3; ++k) memcpy(base + d.off_codebook + 32 * k, cb->len[k], 32);
+    if (cb->n_fields == 2) {
+        for (int k = 0; k < 3; ++k) memcpy(base + d.off_codebook + 32 * k, cb->len[k], 32);
+    } else {
+        memcpy(base + d.off_codebook, cb->len_e, 256);
+    }
     memcpy(base + d.off_lut, cb->lut.data(), 4ull << cb->budget);
     uint32_t *index = (uint32_t *)(base + d.off_index);
     for (uint64_t c = 0; c <= n_chunks; ++c) index[c] = (uint32_t)rec[c];
@@ -472,27 +546,42 @@ huffllm_status huffllm_validate_blob(const void *blob, size_t bytes, huffllm_des
     memset(cb.code, 0, sizeof(cb.code));
     cb.dtype = d.dtype;
     cb.budget = d.lut_bits;
-    for (int k = 0; k < 3; ++k) memcpy(cb.len[k], base + d.off_codebook + 32 * k, 32);
-    for (int k = 0; k < 2; ++k) {
+    cb.n_fields = d.n_fields;
+    memset(cb.len, 0, sizeof(cb.len));
+    memset(cb.len_e, 0, sizeof(cb.len_e));
+    memset(cb.code_e, 0, sizeof(cb.code_e));
+    // Kraft sum of one stored code: complete, or the single 1-bit code
+    auto check_code = [&](const uint8_t *len, int slots, int nsym, int cap, int k) -> bool {
         uint64_t kraft = 0;
         int used = 0, mx = 0;
-        for (int s = 0; s < 32; ++s) {
-            int l = cb.len[k][s];
+        for (int s = 0; s < slots; ++s) {
+            int l = len[s];
             if (!l) continue;
-            if (s >= 16 || l > 15) return fail(HUFFLLM_ERR_CORRUPT, "code length out of range");
+            if (s >= nsym || l > 15) { fail(HUFFLLM_ERR_CORRUPT, "code length out of range"); return false; }
             kraft += 1ull << (16 - l);
             ++used;
             mx = std::max(mx, l);
         }
-        if (used == 0) return fail(HUFFLLM_ERR_CORRUPT, "field %d has no codewords", k);
-        if (!(kraft == (1ull << 16) || (used == 1 && mx == 1))) return fail(HUFFLLM_ERR_CORRUPT, "field %d is not a complete prefix code", k);
-        if (mx > d.caps[k]) return fail(HUFFLLM_ERR_CORRUPT, "field %d exceeds its cap", k);
+        if (used == 0) { fail(HUFFLLM_ERR_CORRUPT, "field %d has no codewords", k); return false; }
+        if (!(kraft == (1ull << 16) || (used == 1 && mx == 1))) { fail(HUFFLLM_ERR_CORRUPT, "field %d is not a complete prefix code", k); return false; }
+        if (mx > cap) { fail(HUFFLLM_ERR_CORRUPT, "field %d exceeds its cap", k); return false; }
+        return true;
+    };
+    if (d.n_fields == 2) {
+        for (int k = 0; k < 3; ++k) memcpy(cb.len[k], base + d.off_codebook + 32 * k, 32);
+        for (int k = 0; k < 2; ++k)
+            if (!check_code(cb.len[k], 32, 16, d.caps[k], k)) return HUFFLLM_ERR_CORRUPT;
+        for (int s = 0; s < 32; ++s)
+            if (cb.len[2][s]) return fail(HUFFLLM_ERR_CORRUPT, "unexpected third field");
+        if (d.caps[0] + d.caps[1] > (int)d.lut_bits) return fail(HUFFLLM_ERR_CORRUPT, "caps exceed lut_bits");
+        canonical_codes(cb.len[0], 16, cb.code[0]);
+        canonical_codes(cb.len[1], 16, cb.code[1]);
+    } else {
+        memcpy(cb.len_e, base + d.off_codebook, 256);
+        if (!check_code(cb.len_e, 256, 256, d.caps[0], 0)) return HUFFLLM_ERR_CORRUPT;
+        if (d.caps[0] > d.lut_bits || d.caps[1]) return fail(HUFFLLM_ERR_CORRUPT, "caps exceed lut_bits");
+        canonical_codes(cb.len_e, 256, cb.code_e);
     }
-    for (int s = 0; s < 32; ++s)
-        if (cb.len[2][s]) return fail(HUFFLLM_ERR_CORRUPT, "unexpected third field");
-    if (d.caps[0] + d.caps[1] > (int)d.lut_bits) return fail(HUFFLLM_ERR_CORRUPT, "caps exceed lut_bits");
-    canonical_codes(cb.len[0], 16, cb.code[0]);
-    canonical_codes(cb.len[1], 16, cb.code[1]);
     finish_codebook(&cb);
     if (memcmp(cb.lut.data(), base + d.off_lut, 4ull << d.lut_bits) != 0) return fail(HUFFLLM_ERR_CORRUPT, "LUT does not match the codebook");
     if (cb.pad_word != d.pad_word) return fail(HUFFLLM_ERR_CORRUPT, "pad_word does not match the codebook");

@@ -27,9 +27,9 @@ def torch():
 class Uploaded:
     """A tensor encoded on the host and resident on the device, with its scratch buffers."""
 
-    def __init__(self, hl, torch, w, chunk_elems=4096, budget=0, batch=1):
+    def __init__(self, hl, torch, w, chunk_elems=4096, budget=0, batch=1, split=0):
         self.w = w
-        cb = hl.build_codebook(w, hl.BF16, budget)
+        cb = hl.build_codebook(w, hl.BF16, budget, split)
         self.blob, self.desc = hl.encode(cb, w, chunk_elems)
         cb.free()
         hl.validate_blob(self.blob)
@@ -109,6 +109,24 @@ def test_decode_is_bit_exact(hl, torch, rows, cols, ce, budget, gen):
         ref, _ = orc.decode_blob(up.blob)          # the oracle's bit-serial decode of the same blob
         assert np.array_equal(ref, w)
     assert np.array_equal(got, w)                  # lossless: the oracle's result is the original tensor
+
+
+@pytest.mark.parametrize("rows,cols,ce,budget,gen,batch", [
+    (1024, 1024, 4096, 0, "gauss", 1), (37, 300, 1024, 0, "student", 0), (256, 2048, 4096, 0, "patterns", 0),
+    (512, 4096, 4096, 9, "student", 5), (272, 2080, 16384, 0, "gauss", 4), (16, 512, 512, 0, "constant", 2),
+    (1040, 4096, 4096, 0, "gauss", 33), (256, 2048, 4096, 0, "uniform", 8)])
+def test_whole_exponent_split_decode_and_product(hl, torch, rows, cols, ce, budget, gen, batch):
+    """Blobs of the {1,8,7} split (one 256-symbol exponent code) run through the same kernels: only the table differs."""
+    w = make(gen, rows, cols, 700 + rows)
+    up = Uploaded(hl, torch, w, ce, budget, max(batch, 1), split=hl.SPLIT_WHOLE_EXPONENT)
+    assert up.desc.n_fields == 1
+    assert np.array_equal(gpu_decode(hl, torch, up), w)
+    if rows * cols <= 300_000:
+        ref, _ = orc.decode_blob(up.blob)
+        assert np.array_equal(ref, w)
+    if batch:
+        x = wl.activations(batch, cols, 800 + cols)
+        check_product(gpu_gemm(hl, torch, up, x), w, x)
 
 
 GEMM_CASES = [

@@ -53,30 +53,55 @@ def test_codebook_cost_matches_oracle(name, budget):
     cb.free()
 
 
-@pytest.mark.parametrize("rows,cols,ce,budget,gen", [
-    (48, 1056, 4096, 8, "gauss"), (37, 300, 1024, 8, "student"), (16, 256, 4096, 9, "gauss"),
-    (5, 31, 512, 8, "patterns"), (33, 2080, 16384, 8, "gauss"), (64, 1024, 4096, 12, "uniform"),
-    (20, 520, 1024, 10, "patterns"), (1, 8, 512, 8, "gauss")])
-def test_blob_decodes_with_oracle_and_bits_match(rows, cols, ce, budget, gen):
+@pytest.mark.parametrize("name", sorted(DATASETS))
+@pytest.mark.parametrize("budget", [0, 8, 9, 12])
+def test_whole_exponent_codebook_cost_matches_oracle(name, budget):
+    w = DATASETS[name]()
+    cb = hl.build_codebook(w, hl.BF16, budget, hl.SPLIT_WHOLE_EXPONENT)
+    counts = orc.histogram(w, orc.BF16_E8)
+    olens, ocaps = orc.build_lengths(counts, orc.BF16_E8, budget or 8)
+    c, lens, codes = cb.get_exponent()
+    assert np.array_equal(c, counts[0])
+    assert kraft_ok(lens) and max(lens) <= (budget or 8)
+    assert np.array_equal(codes, orc.canonical_codes(lens))
+    assert orc.code_cost(c, lens) == orc.code_cost(counts[0], olens[0])
+    with pytest.raises(hl.HuffllmError):
+        cb.get(0)                                       # the nibble accessor does not apply
+    cb.free()
+    cb2 = hl.build_codebook(w, hl.BF16, budget)
+    with pytest.raises(hl.HuffllmError):
+        cb2.get_exponent()
+    cb2.free()
+
+
+@pytest.mark.parametrize("rows,cols,ce,budget,gen,split", [
+    (48, 1056, 4096, 8, "gauss", 0), (37, 300, 1024, 8, "student", 0), (16, 256, 4096, 9, "gauss", 0),
+    (5, 31, 512, 8, "patterns", 0), (33, 2080, 16384, 8, "gauss", 0), (64, 1024, 4096, 12, "uniform", 0),
+    (20, 520, 1024, 10, "patterns", 0), (1, 8, 512, 8, "gauss", 0),
+    (48, 1056, 4096, 8, "gauss", 1), (37, 300, 1024, 9, "student", 1), (5, 31, 512, 8, "patterns", 1),
+    (64, 1024, 4096, 12, "uniform", 1), (33, 2080, 16384, 8, "gauss", 1)])
+def test_blob_decodes_with_oracle_and_bits_match(rows, cols, ce, budget, gen, split):
     w = {"gauss": lambda: wl.gaussian_weights(rows, cols, 0.02, 31),
          "student": lambda: wl.student_t_weights(rows, cols, 32),
          "uniform": lambda: wl.uniform_exponent_weights(rows, cols, 33),
          "patterns": lambda: wl.all_patterns_weights(rows, cols, 34)}[gen]()
-    cb = hl.build_codebook(w, hl.BF16, budget)
+    cb = hl.build_codebook(w, hl.BF16, budget, split)
     blob, d = hl.encode(cb, w, ce)
+    assert d.n_fields == (2 if split == 0 else 1)
     assert d.blob_bytes == blob.size <= hl.encode_bound(rows, cols, hl.BF16, ce)
     hl.validate_blob(blob)
     back, used = orc.decode_blob(blob)                  # slow reader + bit-serial decoder; checks lag/tail/pad bits
     assert np.array_equal(back, w)
     # the oracle's own encoding with the blob's code lengths gives the same bits, lane by lane
     parsed = orc.parse_blob(blob)
-    lens, codes = parsed["lens"], parsed["codes"]
+    lens, codes, scheme = parsed["lens"], parsed["codes"], parsed["dtype"]
+    assert scheme == (orc.BF16 if split == 0 else orc.BF16_E8)
     flat = np.append(w.ravel(), np.uint16(d.pad_word))
-    assert d.pad_word == orc.pad_word(lens)
+    assert d.pad_word == orc.pad_word(lens, scheme)
     for chunk_ids, idx in orc.element_map(rows, cols, ce):
         n, _, steps = idx.shape
         S = orc.SEQS
-        bits, off, raw = orc.encode_sequences(flat[idx.reshape(n * S, steps)], lens, codes)
+        bits, off, raw = orc.encode_sequences(flat[idx.reshape(n * S, steps)], lens, codes, scheme)
         for a, cid in enumerate(chunk_ids):
             pbits, poff, praw = parsed["chunks"][int(cid)]
             per = pbits.reshape(S, -1)
@@ -86,15 +111,16 @@ def test_blob_decodes_with_oracle_and_bits_match(rows, cols, ce, budget, gen):
                 assert np.array_equal(per[l, :hi - lo], bits[lo:hi])
             assert np.array_equal(praw, raw[a * S:a * S + S])
     # the LUT is what a bit-serial decode of every index gives
-    assert np.array_equal(parsed["lut"], orc.lut_from_code(lens, codes, d.lut_bits))
+    assert np.array_equal(parsed["lut"], orc.lut_from_code(lens, codes, d.lut_bits, scheme))
     # accounting
     assert d.coded_bits == sum(int(u.sum()) for u in used.values()) and d.raw_bits == 8 * rows * cols
     cb.free()
 
 
-def test_validator_rejects_damaged_blobs():
+@pytest.mark.parametrize("split", [0, 1])
+def test_validator_rejects_damaged_blobs(split):
     w = wl.gaussian_weights(48, 1056, 0.02, 41)
-    cb = hl.build_codebook(w)
+    cb = hl.build_codebook(w, hl.BF16, 0, split)
     blob, d = hl.encode(cb, w, 4096)
     hl.validate_blob(blob)
 
@@ -109,7 +135,7 @@ def test_validator_rejects_damaged_blobs():
     damaged(16, 1)                               # rows
     damaged(56, 1)                               # lut_bits
     damaged(76, 1)                               # max_words
-    damaged(d.off_codebook + 6, 1)               # a code length
+    damaged(d.off_codebook + (6 if split == 0 else int(np.argmax(blob[d.off_codebook:d.off_codebook + 256] > 0))), 1)   # a code length
     damaged(d.off_lut + 40, 1)                   # a LUT entry
     damaged(d.off_index + 4, 1)                  # record index
     damaged(d.off_payload + 8 * 512 + 0, 1)      # lag bit of chunk 0 lane 0

@@ -129,7 +129,7 @@ def test_canonical_codes_prefix_free_and_ordered():
 def test_joint_budget_is_best_split_bf16():
     rng = np.random.default_rng(5)
     for trial in range(10):
-        counts = np.zeros((3, 32), dtype=np.uint64)
+        counts = np.zeros((3, orc.MAXSYM), dtype=np.uint64)
         n0, n1 = int(rng.integers(1, 5)), int(rng.integers(2, 7))
         counts[0, rng.choice(16, n0, replace=False)] = rng.integers(1, 50, n0)
         counts[1, rng.choice(16, n1, replace=False)] = rng.integers(1, 50, n1)
@@ -186,13 +186,57 @@ def test_worked_example_bf16():
     assert y[0, 0] == float(g["y"][0]) and d[0, 0] == float(g["abs_sum"][0])
 
 
+def test_worked_example_bf16_whole_exponent():
+    g = read_golden("worked_example_bf16_whole_exponent.txt")
+    w = np.array([int(x, 16) for x in g["weights_hex"]], dtype=np.uint16)
+    counts = orc.histogram(w, orc.BF16_E8)
+    lens, _ = orc.build_lengths(counts, orc.BF16_E8, 0)
+    codes = orc.codes_for(lens)
+    syms = [int(s, 16) for s in g["exp_symbols"]]
+    assert [int(lens[0][s]) for s in syms] == [int(x) for x in g["exp_lengths"]]
+    assert [format(int(codes[0][s]), "0{}b".format(int(lens[0][s]))) for s in syms] == g["exp_codes"]
+    assert int((lens[0] > 0).sum()) == len(syms) and not lens[1:].any()
+    bits, off, raw = orc.encode_sequences(w[None, :], lens, codes, orc.BF16_E8)
+    assert "".join(map(str, bits)) == g["bitstream"][0]
+    assert [int(x) for x in raw[0]] == [int(x, 16) for x in g["raw_hex"]]
+    assert len(bits) + 8 * 8 == int(g["payload_bits"][0])
+    back, used = orc.decode_sequences(bits, off, raw, lens, codes, orc.BF16_E8)
+    assert np.array_equal(back[0], w) and int(used[0]) == len(bits)
+
+
+def test_whole_exponent_split_against_the_nibble_split():
+    """{1,8,7} codes the same exponent byte as {1,4,4,7}: same raw bytes, same decoded words, and its entropy is at
+    most the sum of the nibble entropies, so its Huffman cost is below the nibble cost + 1 bit per weight."""
+    w = wl.gaussian_weights(256, 1024, 0.02, 11)
+    c2, c1 = orc.histogram(w, orc.BF16), orc.histogram(w, orc.BF16_E8)
+    assert int(c1[0].sum()) == w.size and not c1[1:].any()
+    # the byte histogram folds into the two nibble histograms
+    assert np.array_equal(c1[0].reshape(16, 16).sum(axis=1), c2[0][:16])
+    assert np.array_equal(c1[0].reshape(16, 16).sum(axis=0), c2[1][:16])
+    l2, _ = orc.build_lengths(c2, orc.BF16, 0)
+    l1, _ = orc.build_lengths(c1, orc.BF16_E8, 0)
+    p = c1[0][c1[0] > 0].astype(np.float64) / w.size
+    H = float(-(p * np.log2(p)).sum())
+    avg1 = orc.code_cost(c1[0], l1[0]) / w.size
+    avg2 = (orc.code_cost(c2[0], l2[0]) + orc.code_cost(c2[1], l2[1])) / w.size
+    assert H <= avg1 < H + 1 and avg1 < avg2
+    assert abs((8 + avg1) - 10.7) < 0.2                    # about one bit per weight below the nibble split's 11.7
+    for budget in (8, 9, 12):
+        lb, caps = orc.build_lengths(c1, orc.BF16_E8, budget)
+        assert max(lb[0]) <= budget and caps[0] == budget and kraft_num(lb[0]) == 1 << 32
+        assert orc.code_cost(c1[0], lb[0]) >= orc.code_cost(c1[0], l1[0])
+    bits, off, raw = orc.encode_sequences(w.reshape(64, -1), l1, orc.codes_for(l1), orc.BF16_E8)
+    _, _, raw2 = orc.encode_sequences(w.reshape(64, -1), l2, orc.codes_for(l2), orc.BF16)
+    assert np.array_equal(raw, raw2)
+
+
 # ----------------------------------------------------------------- lossless
 
-@pytest.mark.parametrize("dtype", [orc.BF16, orc.FP16])
+@pytest.mark.parametrize("dtype", [orc.BF16, orc.FP16, orc.BF16_E8])
 def test_every_pattern_round_trips(dtype):
     w = wl.all_patterns_weights(64, 2048, seed=7)                                # 2 x all 65536 patterns
     counts = orc.histogram(w, dtype)
-    for budget in (0, 12) if dtype == orc.FP16 else (0, 8, 10, 12):
+    for budget in (0, 12) if dtype != orc.BF16 else (0, 8, 10, 12):
         lens, caps = orc.build_lengths(counts, dtype, budget)
         codes = orc.codes_for(lens)
         bits, off, raw = orc.encode_sequences(w.reshape(16, -1), lens, codes, dtype)
