@@ -115,7 +115,7 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def prepare(workload: str, chunk_elems: int, hl, torch, dev, cpu_sample_mats: int = 0, split: int = 0):
+def prepare(workload: str, chunk_elems: int, hl, torch, dev, cpu_sample_mats: int = 0, split: int = 0, batch: int = 1):
     """Generate, encode (host) and upload every matrix of the workload."""
     table, std, seed, _ = WORKLOADS[workload]
     mats = []
@@ -124,18 +124,18 @@ def prepare(workload: str, chunk_elems: int, hl, torch, dev, cpu_sample_mats: in
         cb = hl.build_codebook(w, hl.BF16, 0, split)
         blob, desc = hl.encode(cb, w, chunk_elems)
         cb.free()
-        x = wl.activations(1, cols, seed + 500 + i)
-        ws_bytes = hl.workspace_bytes(desc, 1)
-        alg_bytes = (desc.payload_bytes + 4 * (desc.n_chunks + 1) + (4 << desc.lut_bits) + 2 * cols + 4 * rows)
+        x = wl.activations(batch, cols, seed + 500 + i)
+        ws_bytes = hl.workspace_bytes(desc, batch)
+        alg_bytes = (desc.payload_bytes + 4 * (desc.n_chunks + 1) + (4 << desc.lut_bits) + batch * (2 * cols + 4 * rows))
         mats.append(dict(name=name, rows=rows, cols=cols, desc=desc, blob_dev=torch.from_numpy(blob).to(dev),
                          x_host=torch.from_numpy(x.view(np.int16).reshape(-1)).pin_memory(),
-                         y_host=torch.zeros(rows, dtype=torch.float32).pin_memory(),
+                         y_host=torch.zeros(batch * rows, dtype=torch.float32).pin_memory(),
                          x_dev=torch.from_numpy(x.view(np.int16).reshape(-1)).to(dev),
-                         y_dev=torch.zeros(rows, dtype=torch.float32, device=dev),
+                         y_dev=torch.zeros(batch * rows, dtype=torch.float32, device=dev),
                          ws=torch.zeros(ws_bytes, dtype=torch.uint8, device=dev), ws_bytes=ws_bytes,
                          alg_bytes=int(alg_bytes), coded_bits=int(desc.coded_bits), raw_bits=int(desc.raw_bits),
                          blob_bytes=int(desc.blob_bytes), w_sample=w.copy() if i < cpu_sample_mats else None,
-                         x_np=x if i < cpu_sample_mats else None))
+                         x_np=x[:1] if i < cpu_sample_mats else None))
         del w
     return mats
 
@@ -201,6 +201,8 @@ def main():
                     help="which matrices of the layer share a launch")
     ap.add_argument("--split", default="paper", choices=["paper", "whole-exponent"],
                     help="field split of the blobs: the paper's BF16 {1,4,4,7} or {1,8,7} (one 256-symbol exponent code)")
+    ap.add_argument("--batch", type=int, default=1,
+                    help="activation vectors per product (1..64; above 8 every matrix is its own launch on the tcgen05 path)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -221,9 +223,14 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
     args.warmup = max(args.warmup, 3)
 
-    cpu_mats = 0 if (args.no_cpu_baseline or world > 1 or rank != 0) else 4      # whole matrices kept for the CPU-oracle leg
+    cpu_mats = 0 if (args.no_cpu_baseline or world > 1 or rank != 0) else 7      # whole matrices kept for the CPU-oracle leg (about 20 s)
     split = 0 if args.split == "paper" else 1
-    mats = prepare(args.workload, args.chunk_elems, hl, torch, dev, cpu_mats, split)
+    B = args.batch
+    if not 1 <= B <= 64:
+        raise SystemExit("--batch must be in [1, 64]")
+    if B > 8:
+        args.fuse = "none"           # the tensor-core path takes one matrix per launch
+    mats = prepare(args.workload, args.chunk_elems, hl, torch, dev, cpu_mats, split, B)
     err = torch.zeros(1, dtype=torch.int32, device=dev)
     n_weights = sum(m["rows"] * m["cols"] for m in mats)
     unc_bytes = 2 * n_weights
@@ -234,17 +241,28 @@ def main():
     calls = [dict(descs=[mats[i]["desc"] for i in g], blobs=[mats[i]["blob_dev"] for i in g], xs=[mats[i]["x_dev"] for i in g],
                   ys=[mats[i]["y_dev"] for i in g], wss=[mats[i]["ws"] for i in g]) for g in groups]
 
+    ws_each = min(m["ws_bytes"] for m in mats)
+
     def step_device():
+        if B > 8:
+            for m in mats:
+                hl.decode_gemm(m["desc"], m["blob_dev"], m["x_dev"], B, m["y_dev"], m["ws"], m["ws_bytes"], err, stream)
+            return
         for c in calls:
-            hl.decode_gemm_multi(c["descs"], c["blobs"], c["xs"], 1, c["ys"], c["wss"], mats[0]["ws_bytes"], err, stream)
+            hl.decode_gemm_multi(c["descs"], c["blobs"], c["xs"], B, c["ys"], c["wss"], ws_each, err, stream)
 
     for c, g in zip(calls, groups):
         c["xh"], c["yh"] = [mats[i]["x_host"] for i in g], [mats[i]["y_host"] for i in g]
 
     def step_host():      # host activations in, host results out, through the C-ABI's host-buffer call
+        if B > 8:
+            for m in mats:
+                hl.decode_gemm_host(m["desc"], m["blob_dev"], m["x_host"], B, m["y_host"], m["x_dev"], m["y_dev"], m["ws"],
+                                    m["ws_bytes"], err, stream)
+            return
         for c in calls:
-            hl.decode_gemm_multi_host(c["descs"], c["blobs"], c["xh"], 1, c["yh"], c["xs"], c["ys"], c["wss"],
-                                      mats[0]["ws_bytes"], err, stream)
+            hl.decode_gemm_multi_host(c["descs"], c["blobs"], c["xh"], B, c["yh"], c["xs"], c["ys"], c["wss"],
+                                      ws_each, err, stream)
 
     def barrier():
         if dist is not None:
@@ -283,7 +301,7 @@ def main():
     for s in range(n_b):
         ev[s][0].record(stream)
         for i, m in enumerate(mats):
-            hl.decode_gemv(m["desc"], m["blob_dev"], m["x_dev"], m["y_dev"], m["ws"], m["ws_bytes"], err, stream)
+            hl.decode_gemm(m["desc"], m["blob_dev"], m["x_dev"], B, m["y_dev"], m["ws"], m["ws_bytes"], err, stream)
             ev[s][i + 1].record(stream)
     barrier()
     per_mat_ms = [statistics.median(ev[s][i].elapsed_time(ev[s][i + 1]) for s in range(n_b)) for i in range(len(mats))]
@@ -308,10 +326,10 @@ def main():
                 w_dev.view(torch.bfloat16).normal_(0, 0.02)
             def plain():
                 for w_dev, m in dense:
-                    hl.plain_gemv(w_dev, m["rows"], m["cols"], m["x_dev"], m["y_dev"], stream)
+                    hl.plain_gemv(w_dev, m["rows"], m["cols"], m["x_dev"], m["y_dev"], stream)     # one vector: the batch-1 cost
             def cublas():
                 for w_dev, m in dense:
-                    torch.mv(w_dev.view(torch.bfloat16), m["x_dev"].view(torch.bfloat16))
+                    torch.mv(w_dev.view(torch.bfloat16), m["x_dev"][:m["cols"]].view(torch.bfloat16))
             for fn, key in ((plain, "plain"), (cublas, "cublas")):
                 for _ in range(args.warmup):
                     fn()
@@ -349,7 +367,7 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
         "data": "synthetic",
-        "config": {"workload": args.workload, "what": WORKLOADS[args.workload][3], "chunk_elems": args.chunk_elems,
+        "config": {"workload": args.workload, "what": WORKLOADS[args.workload][3], "chunk_elems": args.chunk_elems, "batch": B,
                    "split": "bf16 {1,4,4,7}" if args.split == "paper" else "bf16 {1,8,7} (whole exponent)",
                    "max_code_len": int(mats[0]["desc"].lut_bits), "weights_per_step": n_weights,
                    "uncompressed_bytes": unc_bytes, "compressed_bytes": sum(m["blob_bytes"] for m in mats),
@@ -362,14 +380,14 @@ def main():
                    "tokens_per_s_equiv_one_layer": 1e3 / ms_step},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": None if NCU_TRAFFIC_RATIO is None else NCU_TRAFFIC_RATIO * alg_bytes / len(groups),
-                     "peak_source": peak_src, "kernel": "huff_kernel<product>", "launches_per_step": len(groups), "fuse": args.fuse,
+                     "peak_source": peak_src, "kernel": "huff_kernel<product>" if B <= 8 else "huff_gemm_tc_kernel", "launches_per_step": len(groups), "fuse": args.fuse,
                      "algorithmic_bytes_per_step": alg_bytes, "kernel_ms_per_step": kernel_ms_step,
                      "frac_of_nominal_8TBs": achieved / 8000.0,
                      "per_matrix": [{"name": m["name"], "rows": m["rows"], "cols": m["cols"], "ms": t,
                                      "comp_GBs": m["alg_bytes"] / (t * 1e-3) / 1e9} for m, t in zip(mats, per_mat_ms)]},
         "cpu_baseline": cpu,
         "e2e": {"value": world * unc_bytes / (e2e_ms * 1e-3) / 1e9, "unit": UNIT, "ms_per_step": e2e_ms,
-                "h2d_bytes_per_step": sum(2 * m["cols"] for m in mats), "d2h_bytes_per_step": sum(4 * m["rows"] for m in mats)},
+                "h2d_bytes_per_step": B * sum(2 * m["cols"] for m in mats), "d2h_bytes_per_step": B * sum(4 * m["rows"] for m in mats)},
         "gpu_launches": len(groups) * args.steps,
         "clocks": clocks,
         "dense_bf16_gemv": {"own_kernel_ms_per_step": plain_ms, "cublas_mv_ms_per_step": cublas_ms,
