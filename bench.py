@@ -55,7 +55,7 @@ def launch_groups(table, fuse: str):
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one fused-product launch over its algorithmic bytes, from the
 # ncu capture summarised in profiles/ (None until a capture exists); traffic = ratio * algorithmic bytes.
-NCU_TRAFFIC_RATIO = 1.03   # profiles/huff_kernel_product_llama7b_layer.md: 147.5 MB moved for 142.0 MB (gate+up), 72.3 for 71.0 (down)
+NCU_TRAFFIC_RATIO = 1.02   # profiles/huff_kernel_product_llama7b_layer.md: 145.7 MB moved for 142.0 MB (gate+up), 71.8 for 71.0 (down)
 
 
 def measured_peak():
