@@ -62,13 +62,17 @@ typedef struct huffllm_codebook huffllm_codebook;
  * Blob layout (every section starts on a 256-byte boundary):
  *   header    this struct
  *   codebook  n_fields == 2: uint8 lengths[3][32] (hi-nibble code, lo-nibble code, zeros);
- *             n_fields == 1: uint8 lengths[256] of the whole-exponent code.
+ *             n_fields == 1: uint8 lengths[256] of the whole-exponent code;
+ *             n_fields == 3 (FP16): uint8 lengths[3][32] (exponent, upper five, lower five mantissa bits).
  *             0 = symbol unused; codewords are canonical: symbols ordered by
  *             (length, symbol), first codeword 0, next = (previous + 1) << (length growth); a
  *             codeword's most significant bit comes first in the stream
  *   LUT       uint32[1 << lut_bits], indexed by the next lut_bits stream bits (first bit = bit 0);
  *             BF16 entry = (code length of the weight: hi-nibble + lo-nibble code, or the whole-exponent
- *             code) << 16 | exponent << 7, i.e. the exponent already sits where a bf16 word has it
+ *             code) << 16 | exponent << 7, i.e. the exponent already sits where a bf16 word has it.
+ *             FP16: three such tables back to back, one per field, indexed by the next lut_bits bits at that
+ *             field's position; entry = code length << 16 | symbol << (10, 5, 0): the three entries of a
+ *             weight OR-ed together give its 15 low bits
  *   index     uint32[n_chunks + 1]: record offsets from off_payload, in units of 128 bytes
  *   payload   one record per chunk, chunk id = row_group * col_chunks + col_chunk
  *
@@ -82,7 +86,11 @@ typedef struct huffllm_codebook huffllm_codebook;
  * little-endian uint32 (row j, sequence s): the sequence's bits, bit i in word i / 32 at bit
  * i % 32.  A sequence starts with `lag_bits` zero bits, then for every weight
  * code(exponent >> 4) code(exponent & 15) (n_fields == 2) or code(exponent) (n_fields == 1); bits after
- * the last codeword are zero.  W is the
+ * the last codeword are zero.
+ * FP16 blobs: per weight code(exponent) code(mantissa >> 5) code(mantissa & 31); the raw part of a record is
+ * [block][lane] uint16 (padded to a multiple of 128 bytes) holding the signs of the lane's 16 weights of the block:
+ * the lane's weights form eight pairs (row g: columns (0,1) (2,3) (4,5) (6,7) of its eight, then row g + 8 likewise);
+ * bit p is the sign of the first weight of pair p, bit 8 + p the sign of its second weight.  W is the
  * longest sequence of the chunk in words (all 64 are padded to it).
  */
 typedef struct huffllm_desc {
@@ -96,9 +104,9 @@ typedef struct huffllm_desc {
     uint32_t row_groups;      /* ceil(rows / 16)                                           */
     uint32_t col_chunks;      /* ceil(cols / chunk_cols)                                   */
     uint64_t n_chunks;        /* row_groups * col_chunks                                   */
-    uint32_t lut_bits;        /* L_max of one weight's coded fields together (8 .. 12)     */
-    uint32_t lag_bits;        /* 7                                                         */
-    uint32_t n_fields;        /* coded fields per weight: 2 (BF16 {1,4,4,7}) or 1 ({1,8,7}) */
+    uint32_t lut_bits;        /* L_max: BF16: of one weight's coded fields together; FP16: of each field (8 .. 12) */
+    uint32_t lag_bits;        /* 7 (BF16 blobs), 5 (FP16 blobs)                            */
+    uint32_t n_fields;        /* coded fields per weight: 2 (BF16 {1,4,4,7}), 1 ({1,8,7}), 3 (FP16 {1,5,5,5}) */
     uint8_t  caps[4];         /* per-field maximum code length chosen under lut_bits       */
     uint16_t pad_word;        /* weight stored at positions outside the tensor            */
     uint16_t reserved0;
@@ -122,7 +130,9 @@ typedef struct huffllm_desc {
  * being the optimal length-limited prefix code for its cap; where plain Huffman already fits,
  * the result is plain Huffman.  0 selects the default (8); supported range 8..12.
  * A field with a single used symbol gets a 1-bit code.  An empty tensor is INVALID_ARG.
- * On success *out owns a new codebook.  HUFFLLM_FP16 returns UNSUPPORTED in this build.
+ * HUFFLLM_FP16 is the paper's {1,5,5,5} split (Section 3.1): sign raw, exponent and the two mantissa halves each
+ * with its own code, each limited to max_code_len on its own (Section 3.2 quotes 12 for these 5-bit fields; the
+ * device kernels take 8).  On success *out owns a new codebook.
  */
 huffllm_status huffllm_build_codebook(const uint16_t *w_host, uint64_t rows, uint64_t cols, huffllm_dtype dtype,
                                       uint32_t max_code_len, huffllm_codebook **out);

@@ -188,7 +188,10 @@ def matmul(w: np.ndarray, x: np.ndarray, dtype=BF16):
 
 TILE_ROWS = 16
 BLOCK_COLS = 32
-LAG_BITS = 7
+def lag_bits(dtype: int) -> int:
+    """Zero bits in front of every bit sequence of a blob: 7 for bf16 blobs, 5 for fp16 blobs."""
+    return 5 if dtype == FP16 else 7
+
 SEQS = 64          # bit sequences per chunk
 
 
@@ -231,11 +234,12 @@ def element_map(rows: int, cols: int, chunk_elems: int):
 def pad_word(lens: np.ndarray, dtype=BF16) -> int:
     """The weight written at positions outside the tensor: every coded field takes its shortest codeword
     (ties: smallest symbol), raw bits zero."""
-    assert dtype in (BF16, BF16_E8)
     f = []
     for k in range(num_fields(dtype)):
         used = [(int(lens[k][s]), s) for s in range(field_symbols(dtype)) if lens[k][s]]
         f.append(min(used)[1])
+    if dtype == FP16:
+        return (f[0] << 10 | f[1] << 5 | f[2]) & 0xFFFF
     e = (f[0] << 4 | f[1]) if dtype == BF16 else f[0]
     return (e << 7) & 0xFFFF
 
@@ -286,7 +290,7 @@ def decode_tensor(enc) -> np.ndarray:
 # indexed by the next lut_bits stream bits (first bit = bit 0).  index: u32[n_chunks + 1], record offsets in 128-byte
 # units from off_payload.  Record of a chunk with nkb blocks: raw bytes [nkb][32 lanes][16] (a lane's 16
 # bytes: row g's eight weights, then row g+8's), then W rows of 64 little-endian u32 (row j, sequence s):
-# the sequence's bits, bit i in word i // 32 at bit i % 32, starting with LAG_BITS zero bits; unused bits
+# the sequence's bits, bit i in word i // 32 at bit i % 32, starting with lag_bits zero bits (7 for bf16 blobs, 5 for fp16); unused bits
 # after the last codeword are zero.
 
 HEADER = struct.Struct("<4sIIIQQIIIIQIII4sHHIQQQQQQQQ")
@@ -309,22 +313,22 @@ def parse_blob(blob) -> dict:
     blob = bytes(blob)
     h = parse_header(blob)
     rows, cols, ce, dtype = h["rows"], h["cols"], h["chunk_elems"], h["dtype"]
-    assert dtype == BF16, "reader covers bf16 blobs"
-    assert h["n_fields"] in (1, 2)
-    scheme = BF16 if h["n_fields"] == 2 else BF16_E8          # how the exponent is coded
+    assert (dtype, h["n_fields"]) in ((BF16, 1), (BF16, 2), (FP16, 3))
+    scheme = FP16 if dtype == FP16 else (BF16 if h["n_fields"] == 2 else BF16_E8)      # which fields are coded
     geo = geometry(rows, cols, ce)
     assert (h["tile_rows"], h["chunk_cols"], h["row_groups"], h["col_chunks"]) == (16, geo["Kc"], geo["RG"], geo["KC"])
-    assert h["n_chunks"] == geo["RG"] * geo["KC"] and h["lag_bits"] == LAG_BITS
+    assert h["n_chunks"] == geo["RG"] * geo["KC"] and h["lag_bits"] == lag_bits(dtype)
     assert h["blob_bytes"] == len(blob)
     for k in ("off_codebook", "off_lut", "off_index", "off_payload"):
         assert h[k] % 256 == 0
     lens = np.zeros((3, MAXSYM), dtype=np.uint8)
-    if scheme == BF16:
+    if scheme in (BF16, FP16):
         lens[:, :32] = np.frombuffer(blob, dtype=np.uint8, count=96, offset=h["off_codebook"]).reshape(3, 32)
     else:
         lens[0] = np.frombuffer(blob, dtype=np.uint8, count=256, offset=h["off_codebook"])
     codes = codes_for(lens)
-    lut = np.frombuffer(blob, dtype=np.uint32, count=1 << h["lut_bits"], offset=h["off_lut"]).copy()
+    n_tables = 3 if scheme == FP16 else 1
+    lut = np.frombuffer(blob, dtype=np.uint32, count=n_tables << h["lut_bits"], offset=h["off_lut"]).copy()
     index = np.frombuffer(blob, dtype=np.uint32, count=h["n_chunks"] + 1, offset=h["off_index"]).astype(np.int64)
     assert index[0] == 0 and np.all(np.diff(index) > 0) and index[-1] * 128 == h["payload_bytes"]
     assert h["off_payload"] + h["payload_bytes"] <= len(blob)
@@ -335,15 +339,28 @@ def parse_blob(blob) -> dict:
         for a, cid in enumerate(chunk_ids):
             beg = h["off_payload"] + int(index[cid]) * 128
             size = int(index[cid + 1] - index[cid]) * 128
-            W = (size - nkb * 512) // 256
-            assert W >= 1 and nkb * 512 + W * 256 == size
+            raw_bytes = nkb * 512 if scheme != FP16 else -(-nkb * 64 // 128) * 128
+            W = (size - raw_bytes) // 256
+            assert W >= 1 and raw_bytes + W * 256 == size
             max_words = max(max_words, W)
-            raw = np.frombuffer(blob, dtype=np.uint8, count=nkb * 512, offset=beg).reshape(nkb, 32, 2, 8)
-            raw = raw.transpose(2, 1, 0, 3).reshape(SEQS, steps).copy()        # [half][lane] -> sequence
-            words = np.frombuffer(blob, dtype="<u4", count=W * SEQS, offset=beg + nkb * 512).reshape(W, SEQS)
+            if scheme != FP16:
+                raw = np.frombuffer(blob, dtype=np.uint8, count=nkb * 512, offset=beg).reshape(nkb, 32, 2, 8)
+                raw = raw.transpose(2, 1, 0, 3).reshape(SEQS, steps).copy()        # [half][lane] -> sequence
+            else:
+                # one uint16 per (block, lane): bit p = sign of the first weight of pair p, bit 8 + p of its second;
+                # pairs 0..3 are row g's weights (0,1) (2,3) (4,5) (6,7), pairs 4..7 row g+8's
+                sg = np.frombuffer(blob, dtype="<u2", count=nkb * 32, offset=beg).reshape(nkb, 32)
+                assert not np.frombuffer(blob, dtype=np.uint8, count=raw_bytes - nkb * 64, offset=beg + nkb * 64).any()
+                raw = np.zeros((SEQS, steps), dtype=np.uint8)
+                for half in range(2):
+                    for i in range(8):
+                        bit = (i // 2 + 4 * half) + 8 * (i % 2)
+                        raw[half * 32:half * 32 + 32, i::8] = ((sg >> bit) & 1).T
+            words = np.frombuffer(blob, dtype="<u4", count=W * SEQS, offset=beg + raw_bytes).reshape(W, SEQS)
             seq_bits = ((words.T[:, :, None] >> np.arange(32, dtype=np.uint32)) & 1).astype(np.uint8).reshape(SEQS, W * 32)
-            assert not seq_bits[:, :LAG_BITS].any(), "lag bits must be zero"
-            body = np.ascontiguousarray(seq_bits[:, LAG_BITS:])
+            lag = h["lag_bits"]
+            assert not seq_bits[:, :lag].any(), "lag bits must be zero"
+            body = np.ascontiguousarray(seq_bits[:, lag:])
             off = (np.arange(SEQS + 1, dtype=np.uint64) * np.uint64(body.shape[1]))
             chunks[int(cid)] = (body.ravel(), off, raw)
     enc = dict(rows=rows, cols=cols, chunk_elems=ce, dtype=scheme, lens=lens, codes=codes, caps=list(h["caps"][:3]),
@@ -377,7 +394,17 @@ def decode_blob(blob):
 
 def lut_from_code(lens, codes, lut_bits: int, dtype=BF16) -> np.ndarray:
     """What the blob's LUT must contain, found the slow way: for every index, write its bits out as a
-    stream and run one bit-serial decode of a single weight (all its coded fields) on it."""
+    stream and run one bit-serial decode of a single weight (all its coded fields) on it.
+    FP16 blobs hold one table per field: entry = length << 16 | symbol << (10, 5, 0); each is found by decoding
+    a single symbol of that field alone (the one-field scheme's decoder, given that field's code)."""
+    if dtype == FP16:
+        tables = []
+        for k in range(3):
+            l1, c1 = np.zeros_like(lens), np.zeros_like(codes)
+            l1[0], c1[0] = lens[k], codes[k]
+            t = lut_from_code(l1, c1, lut_bits, BF16_E8)           # entry = length << 16 | symbol << 7
+            tables.append((t & np.uint32(0xFFFF0000)) | (((t >> np.uint32(7)) & np.uint32(0xFF)) << np.uint32(10 - 5 * k)))
+        return np.concatenate(tables)
     n = 1 << lut_bits
     idx_bits = ((np.arange(n, dtype=np.uint32)[:, None] >> np.arange(lut_bits, dtype=np.uint32)) & 1).astype(np.uint8)
     out = np.zeros(n, dtype=np.uint32)

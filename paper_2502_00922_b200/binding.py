@@ -113,8 +113,9 @@ def _stream(stream):
 class Codebook:
     """Owner of a huffllm_codebook*."""
 
-    def __init__(self, handle):
+    def __init__(self, handle, dtype: int = BF16):
         self._h = handle
+        self.dtype = dtype
 
     def get(self, field: int):
         n = C.c_uint32()
@@ -152,7 +153,7 @@ def build_codebook(w: np.ndarray, dtype: int = BF16, max_code_len: int = 0, spli
         _check(lib().huffllm_build_codebook(w.ctypes.data, rows, cols, dtype, max_code_len, C.byref(h)))
     else:
         _check(lib().huffllm_build_codebook_split(w.ctypes.data, rows, cols, dtype, split, max_code_len, C.byref(h)))
-    return Codebook(h)
+    return Codebook(h, dtype)
 
 
 def encode_bound(rows: int, cols: int, dtype: int = BF16, chunk_elems: int = 4096) -> int:
@@ -165,7 +166,7 @@ def encode(cb: Codebook, w: np.ndarray, chunk_elems: int = 4096):
     """Returns (blob as a numpy uint8 array trimmed to its size, Desc)."""
     w = np.ascontiguousarray(w, dtype=np.uint16)
     rows, cols = w.shape
-    cap = encode_bound(rows, cols, BF16, chunk_elems)
+    cap = encode_bound(rows, cols, cb.dtype, chunk_elems)
     buf = np.empty(cap, dtype=np.uint8)
     d = Desc()
     _check(lib().huffllm_encode(cb._h, w.ctypes.data, rows, cols, chunk_elems, buf.ctypes.data, cap, C.byref(d)))

@@ -40,13 +40,13 @@ static inline uint64_t record_checksum(const uint8_t *p, uint64_t n, uint64_t ch
 huffllm_status check_desc(const huffllm_desc *d) {
     if (!d) return fail(HUFFLLM_ERR_INVALID_ARG, "descriptor is null");
     if (memcmp(d->magic, "HFLM", 4) != 0 || d->version != 1) return fail(HUFFLLM_ERR_CORRUPT, "bad magic or version");
-    if (d->dtype != HUFFLLM_BF16) return fail(HUFFLLM_ERR_UNSUPPORTED, "only bf16 blobs are supported");
+    if (d->dtype != HUFFLLM_BF16 && d->dtype != HUFFLLM_FP16) return fail(HUFFLLM_ERR_CORRUPT, "bad dtype");
     if (d->rows == 0 || d->cols == 0 || d->rows > (1ull << 31) || d->cols > (1ull << 31))
         return fail(HUFFLLM_ERR_CORRUPT, "bad shape");
     if (d->chunk_elems % (kTileRows * kBlockCols) || d->chunk_elems < 512 || d->chunk_elems > 16384)
         return fail(HUFFLLM_ERR_CORRUPT, "bad chunk_elems");
-    if (d->tile_rows != kTileRows || d->chunk_cols != d->chunk_elems / kTileRows || d->lag_bits != kLagBits ||
-        (d->n_fields != 2 && d->n_fields != 1))
+    if (d->tile_rows != kTileRows || d->chunk_cols != d->chunk_elems / kTileRows || d->lag_bits != lag_bits_for(d->dtype) ||
+        (d->dtype == HUFFLLM_BF16 && d->n_fields != 2 && d->n_fields != 1) || (d->dtype == HUFFLLM_FP16 && d->n_fields != 3))
         return fail(HUFFLLM_ERR_CORRUPT, "bad tile geometry");
     if (d->row_groups != (d->rows + kTileRows - 1) / kTileRows ||
         d->col_chunks != (d->cols + d->chunk_cols - 1) / d->chunk_cols ||
@@ -54,11 +54,11 @@ huffllm_status check_desc(const huffllm_desc *d) {
         return fail(HUFFLLM_ERR_CORRUPT, "chunk counts do not match the shape");
     if (d->lut_bits < kMinBudget || d->lut_bits > kMaxBudget) return fail(HUFFLLM_ERR_CORRUPT, "bad lut_bits");
     uint32_t max_steps = d->chunk_cols / kBlockCols * 8;   // per bit sequence
-    uint32_t w_bound = (kLagBits + max_steps * d->lut_bits + 31) / 32;
+    uint32_t w_bound = (d->lag_bits + max_steps * d->lut_bits * (d->dtype == HUFFLLM_FP16 ? 3 : 1) + 31) / 32;
     if (d->max_words == 0 || d->max_words > w_bound) return fail(HUFFLLM_ERR_CORRUPT, "bad max_words");
     if (d->off_codebook % 256 || d->off_lut % 256 || d->off_index % 256 || d->off_payload % 256 ||
         d->off_codebook < 256 || d->off_lut < d->off_codebook + (d->n_fields == 1 ? 256u : 96u) ||
-        d->off_index < d->off_lut + (4ull << d->lut_bits) || d->off_payload < d->off_index + 4 * (d->n_chunks + 1) ||
+        d->off_index < d->off_lut + (d->dtype == HUFFLLM_FP16 ? 3 : 1) * (4ull << d->lut_bits) || d->off_payload < d->off_index + 4 * (d->n_chunks + 1) ||
         d->payload_bytes % kRecordUnit || d->blob_bytes < d->off_payload + d->payload_bytes ||
         d->payload_bytes / kRecordUnit > 0xFFFFFFFFull)
         return fail(HUFFLLM_ERR_CORRUPT, "bad section offsets");
@@ -150,6 +150,7 @@ struct huffllm_codebook {
     uint64_t counts_e[256];
     uint8_t len_e[256];
     uint32_t code_e[256];
+    uint32_t bits5[3][32];   // FP16: stream bits of a field's codeword, first bit in bit 0
     uint8_t caps[4];
     uint16_t pad_word;
     uint8_t len8[256];    // code length of a whole exponent byte (hi + lo), 0 = no codeword
@@ -159,6 +160,29 @@ struct huffllm_codebook {
 
 // Fill len8 / bits8 / lut / pad_word from len[] and code[].
 static void finish_codebook(huffllm_codebook *cb) {
+    if (cb->dtype == HUFFLLM_FP16) {
+        // three tables, one per field; entry = length << 16 | symbol << (10, 5, 0)
+        const uint32_t n = 1u << cb->budget;
+        cb->lut.assign((size_t)3 * n, 0u);
+        uint32_t pad = 0;
+        for (int k = 0; k < 3; ++k) {
+            const int shift = 10 - 5 * k;
+            int best = -1;
+            for (int s = 0; s < 32; ++s) {
+                int L = cb->len[k][s];
+                cb->bits5[k][s] = 0;
+                if (!L) continue;
+                if (best < 0 || L < cb->len[k][best]) best = s;
+                uint32_t seq = reverse_bits(cb->code[k][s], L);
+                cb->bits5[k][s] = seq;
+                for (uint32_t hi = 0; hi < (1u << (cb->budget - L)); ++hi)
+                    cb->lut[(size_t)k * n + (seq | (hi << L))] = ((uint32_t)L << 16) | ((uint32_t)s << shift);
+            }
+            pad |= (uint32_t)best << shift;
+        }
+        cb->pad_word = (uint16_t)pad;
+        return;
+    }
     memset(cb->len8, 0, sizeof(cb->len8));
     memset(cb->bits8, 0, sizeof(cb->bits8));
     cb->lut.assign((size_t)1 << cb->budget, 0u);
@@ -225,8 +249,7 @@ huffllm_status huffllm_build_codebook(const uint16_t *w, uint64_t rows, uint64_t
                                       uint32_t max_code_len, huffllm_codebook **out) {
     clear_error();
     if (!w || !out || rows == 0 || cols == 0) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer or empty tensor");
-    if (dtype == HUFFLLM_FP16) return fail(HUFFLLM_ERR_UNSUPPORTED, "fp16 {1,5,5,5} is not built yet");
-    if (dtype != HUFFLLM_BF16) return fail(HUFFLLM_ERR_INVALID_ARG, "bad dtype");
+    if (dtype != HUFFLLM_BF16 && dtype != HUFFLLM_FP16) return fail(HUFFLLM_ERR_INVALID_ARG, "bad dtype");
     uint32_t budget = max_code_len ? max_code_len : kDefaultBudget;
     if (budget < kMinBudget || budget > kMaxBudget)
         return fail(HUFFLLM_ERR_UNSUPPORTED, "max_code_len must be 0 or in [%u, %u]", kMinBudget, kMaxBudget);
@@ -239,6 +262,28 @@ huffllm_status huffllm_build_codebook(const uint16_t *w, uint64_t rows, uint64_t
     memset(cb->code, 0, sizeof(cb->code));
     memset(cb->caps, 0, sizeof(cb->caps));
 
+    if (dtype == HUFFLLM_FP16) {
+        // {1,5,5,5}: exponent, upper and lower mantissa half, each with its own code limited to `budget`
+        cb->n_fields = 3;
+        const uint64_t n = rows * cols;
+        for (uint64_t i = 0; i < n; ++i) {
+            uint16_t v = w[i];
+            cb->counts[0][(v >> 10) & 31]++;
+            cb->counts[1][(v >> 5) & 31]++;
+            cb->counts[2][v & 31]++;
+        }
+        for (int k = 0; k < 3; ++k) {
+            if (!limited_lengths(cb->counts[k], 32, (int)budget, cb->len[k])) {
+                delete cb;
+                return fail(HUFFLLM_ERR_INVALID_ARG, "no code fits max_code_len");
+            }
+            cb->caps[k] = (uint8_t)budget;
+            canonical_codes(cb->len[k], 32, cb->code[k]);
+        }
+        finish_codebook(cb);
+        *out = cb;
+        return HUFFLLM_OK;
+    }
     // histogram of the exponent byte, folded into the two nibble fields
     cb->n_fields = 2;
     exponent_histogram(w, rows * cols, cb->counts_e);
@@ -320,8 +365,8 @@ huffllm_status huffllm_codebook_get_exponent(const huffllm_codebook *cb, uint64_
 huffllm_status huffllm_codebook_get(const huffllm_codebook *cb, uint32_t field, uint32_t *n_symbols, uint64_t counts[32],
                                     uint8_t lengths[32], uint32_t codes[32]) {
     clear_error();
-    if (!cb || cb->n_fields != 2 || field >= 2) return fail(HUFFLLM_ERR_INVALID_ARG, "bad codebook or field");
-    if (n_symbols) *n_symbols = 16;
+    if (!cb || cb->n_fields < 2 || field >= cb->n_fields) return fail(HUFFLLM_ERR_INVALID_ARG, "bad codebook or field");
+    if (n_symbols) *n_symbols = cb->n_fields == 2 ? 16 : 32;
     for (int s = 0; s < 32; ++s) {
         if (counts) counts[s] = cb->counts[field][s];
         if (lengths) lengths[s] = cb->len[field][s];
@@ -395,16 +440,17 @@ huffllm_status huffllm_encode_bound(uint64_t rows, uint64_t cols, huffllm_dtype 
     clear_error();
     Geometry g;
     if (!max_bytes) return fail(HUFFLLM_ERR_INVALID_ARG, "max_bytes is null");
-    if (dtype != HUFFLLM_BF16) return fail(HUFFLLM_ERR_UNSUPPORTED, "only bf16 is supported");
+    if (dtype != HUFFLLM_BF16 && dtype != HUFFLLM_FP16) return fail(HUFFLLM_ERR_INVALID_ARG, "bad dtype");
     if (!make_geometry(rows, cols, chunk_elems, &g)) return fail(HUFFLLM_ERR_INVALID_ARG, "bad shape or chunk_elems");
+    const uint64_t fields = dtype == HUFFLLM_FP16 ? 3 : 1;
     uint64_t payload = 0;
     for (uint32_t kc = 0; kc < g.KC; ++kc) {
         uint32_t nkb = blocks_of(g, kc);
-        uint64_t w = (kLagBits + (uint64_t)nkb * 8 * kMaxBudget + 31) / 32;
-        payload += (uint64_t)g.RG * (nkb * 512ull + w * 256ull);
+        uint64_t w = (lag_bits_for(dtype) + (uint64_t)nkb * 8 * kMaxBudget * fields + 31) / 32;
+        payload += (uint64_t)g.RG * (raw_part_bytes(dtype, nkb) + w * 256ull);
     }
     uint64_t n_chunks = (uint64_t)g.RG * g.KC;
-    *max_bytes = (size_t)(256 + 256 + align_up(4ull << kMaxBudget, 256) + align_up(4 * (n_chunks + 1), 256) + payload + 256);
+    *max_bytes = (size_t)(256 + 256 + align_up(fields * (4ull << kMaxBudget), 256) + align_up(4 * (n_chunks + 1), 256) + payload + 256);
     return HUFFLLM_OK;
 }
 
@@ -430,13 +476,14 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
     d.col_chunks = g.KC;
     d.n_chunks = n_chunks;
     d.lut_bits = cb->budget;
-    d.lag_bits = kLagBits;
+    d.lag_bits = lag_bits_for(cb->dtype);
     d.n_fields = cb->n_fields;
     memcpy(d.caps, cb->caps, 4);
     d.pad_word = cb->pad_word;
     d.off_codebook = 256;
     d.off_lut = 512;
-    d.off_index = d.off_lut + align_up(4ull << cb->budget, 256);
+    const bool fp16 = cb->dtype == HUFFLLM_FP16;
+    d.off_index = d.off_lut + align_up((fp16 ? 3 : 1) * (4ull << cb->budget), 256);
     d.off_payload = d.off_index + align_up(4 * (n_chunks + 1), 256);
     if (blob_cap < d.off_payload) return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "blob capacity below the fixed sections");
 
@@ -453,12 +500,19 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
         for (uint32_t lane = 0; lane < kSeqs; ++lane) {
             uint32_t bits = 0;
             for (uint32_t s = 0; s < steps; ++s) {
-                uint32_t l = len8[(weight_at(w, g, rg, kc, lane, s, pad) >> 7) & 0xFF];
-                if (!l) bad.store(1);
-                bits += l;
+                const uint16_t v = weight_at(w, g, rg, kc, lane, s, pad);
+                if (fp16) {
+                    uint32_t l0 = cb->len[0][(v >> 10) & 31], l1 = cb->len[1][(v >> 5) & 31], l2 = cb->len[2][v & 31];
+                    if (!l0 || !l1 || !l2) bad.store(1);
+                    bits += l0 + l1 + l2;
+                } else {
+                    uint32_t l = len8[(v >> 7) & 0xFF];
+                    if (!l) bad.store(1);
+                    bits += l;
+                }
             }
             sum += bits;
-            max_bits = std::max(max_bits, bits + kLagBits);
+            max_bits = std::max(max_bits, bits + d.lag_bits);
         }
         words[c] = std::max(1u, (max_bits + 31) / 32);
         chunk_bits[c] = sum;
@@ -471,7 +525,7 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
     uint64_t coded_bits = 0;
     for (uint64_t c = 0; c < n_chunks; ++c) {
         uint32_t nkb = blocks_of(g, (uint32_t)(c % g.KC));
-        rec[c + 1] = rec[c] + (nkb * 512ull + words[c] * 256ull) / kRecordUnit;
+        rec[c + 1] = rec[c] + (raw_part_bytes(cb->dtype, nkb) + words[c] * 256ull) / kRecordUnit;
         max_words = std::max(max_words, words[c]);
         coded_bits += chunk_bits[c];
     }
@@ -479,7 +533,7 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
     d.payload_bytes = rec[n_chunks] * kRecordUnit;
     d.blob_bytes = d.off_payload + d.payload_bytes;
     d.coded_bits = coded_bits;
-    d.raw_bits = 8 * rows * cols;
+    d.raw_bits = (fp16 ? 1 : 8) * rows * cols;
     if (rec[n_chunks] > 0xFFFFFFFFull) return fail(HUFFLLM_ERR_UNSUPPORTED, "payload exceeds the 32-bit record index");
     if (blob_cap < d.blob_bytes)
         return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "blob needs %llu bytes, capacity is %llu", (unsigned long long)d.blob_bytes,
@@ -487,12 +541,12 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
 
     memset(base, 0, d.off_payload);
     memcpy(base, &d, sizeof(d));
-    if (cb->n_fields == 2) {
+    if (cb->n_fields >= 2) {
         for (int k = 0; k < 3; ++k) memcpy(base + d.off_codebook + 32 * k, cb->len[k], 32);
     } else {
         memcpy(base + d.off_codebook, cb->len_e, 256);
     }
-    memcpy(base + d.off_lut, cb->lut.data(), 4ull << cb->budget);
+    memcpy(base + d.off_lut, cb->lut.data(), cb->lut.size() * sizeof(uint32_t));
     uint32_t *index = (uint32_t *)(base + d.off_index);
     for (uint64_t c = 0; c <= n_chunks; ++c) index[c] = (uint32_t)rec[c];
 
@@ -503,26 +557,40 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
         uint32_t rg = (uint32_t)(c / g.KC), kc = (uint32_t)(c % g.KC), nkb = blocks_of(g, kc), steps = nkb * 8;
         uint32_t W = words[c];
         uint8_t *raw = base + d.off_payload + rec[c] * kRecordUnit;
-        uint32_t *coded = (uint32_t *)(raw + nkb * 512ull);
+        const uint32_t raw_bytes = raw_part_bytes(cb->dtype, nkb);
+        uint32_t *coded = (uint32_t *)(raw + raw_bytes);
         memset(coded, 0, (size_t)W * 256);
+        if (fp16) memset(raw, 0, raw_bytes);
         for (uint32_t lane = 0; lane < kSeqs; ++lane) {
             uint64_t acc = 0;
-            uint32_t nacc = kLagBits, j = 0;
-            for (uint32_t s = 0; s < steps; ++s) {
-                uint16_t v = weight_at(w, g, rg, kc, lane, s, pad);
-                raw[(s >> 3) * 512 + (lane & 31) * 16 + (lane >> 5) * 8 + (s & 7)] = (uint8_t)(((v >> 8) & 0x80) | (v & 0x7F));
-                uint32_t e = (v >> 7) & 0xFF;
-                acc |= (uint64_t)bits8[e] << nacc;
-                nacc += len8[e];
+            uint32_t nacc = d.lag_bits, j = 0;
+            auto append = [&](uint32_t bits, uint32_t len) {      // len <= 16, nacc < 32
+                acc |= (uint64_t)bits << nacc;
+                nacc += len;
                 if (nacc >= 32) {
                     coded[(size_t)j++ * kSeqs + lane] = (uint32_t)acc;
                     acc >>= 32;
                     nacc -= 32;
                 }
+            };
+            for (uint32_t s = 0; s < steps; ++s) {
+                uint16_t v = weight_at(w, g, rg, kc, lane, s, pad);
+                if (fp16) {
+                    // sign bit of weight i of the sequence: pair p = i / 2 (+ 4 for the row g + 8 sequence), bit p (+ 8 if odd)
+                    uint32_t i = s & 7, p = (i >> 1) + 4 * (lane >> 5), bit = p + 8 * (i & 1);
+                    uint16_t *sg = (uint16_t *)(raw + (s >> 3) * 64 + (lane & 31) * 2);
+                    *sg = (uint16_t)(*sg | ((v >> 15) << bit));
+                    uint32_t f[3] = {(uint32_t)(v >> 10) & 31, (uint32_t)(v >> 5) & 31, (uint32_t)v & 31};
+                    for (int k = 0; k < 3; ++k) append(cb->bits5[k][f[k]], cb->len[k][f[k]]);
+                } else {
+                    raw[(s >> 3) * 512 + (lane & 31) * 16 + (lane >> 5) * 8 + (s & 7)] = (uint8_t)(((v >> 8) & 0x80) | (v & 0x7F));
+                    uint32_t e = (v >> 7) & 0xFF;
+                    append(bits8[e], len8[e]);
+                }
             }
             if (nacc) coded[(size_t)j * kSeqs + lane] = (uint32_t)acc;
         }
-        checksum.fetch_add(record_checksum(raw, nkb * 512ull + (uint64_t)W * 256, c));
+        checksum.fetch_add(record_checksum(raw, raw_bytes + (uint64_t)W * 256, c));
     });
     d.payload_checksum = checksum.load();
     memcpy(base, &d, sizeof(d));
@@ -567,7 +635,15 @@ huffllm_status huffllm_validate_blob(const void *blob, size_t bytes, huffllm_des
         if (mx > cap) { fail(HUFFLLM_ERR_CORRUPT, "field %d exceeds its cap", k); return false; }
         return true;
     };
-    if (d.n_fields == 2) {
+    const bool fp16 = d.dtype == HUFFLLM_FP16;
+    if (fp16) {
+        for (int k = 0; k < 3; ++k) {
+            memcpy(cb.len[k], base + d.off_codebook + 32 * k, 32);
+            if (!check_code(cb.len[k], 32, 32, d.caps[k], k)) return HUFFLLM_ERR_CORRUPT;
+            if (d.caps[k] > d.lut_bits) return fail(HUFFLLM_ERR_CORRUPT, "caps exceed lut_bits");
+            canonical_codes(cb.len[k], 32, cb.code[k]);
+        }
+    } else if (d.n_fields == 2) {
         for (int k = 0; k < 3; ++k) memcpy(cb.len[k], base + d.off_codebook + 32 * k, 32);
         for (int k = 0; k < 2; ++k)
             if (!check_code(cb.len[k], 32, 16, d.caps[k], k)) return HUFFLLM_ERR_CORRUPT;
@@ -583,7 +659,7 @@ huffllm_status huffllm_validate_blob(const void *blob, size_t bytes, huffllm_des
         canonical_codes(cb.len_e, 256, cb.code_e);
     }
     finish_codebook(&cb);
-    if (memcmp(cb.lut.data(), base + d.off_lut, 4ull << d.lut_bits) != 0) return fail(HUFFLLM_ERR_CORRUPT, "LUT does not match the codebook");
+    if (memcmp(cb.lut.data(), base + d.off_lut, cb.lut.size() * sizeof(uint32_t)) != 0) return fail(HUFFLLM_ERR_CORRUPT, "LUT does not match the codebook");
     if (cb.pad_word != d.pad_word) return fail(HUFFLLM_ERR_CORRUPT, "pad_word does not match the codebook");
 
     Geometry g;
@@ -599,27 +675,50 @@ huffllm_status huffllm_validate_blob(const void *blob, size_t bytes, huffllm_des
         uint32_t kc = (uint32_t)(c % g.KC), rg = (uint32_t)(c / g.KC), nkb = blocks_of(g, kc), steps = nkb * 8;
         if (index[c + 1] <= index[c]) { bad.store(1); return; }
         uint64_t size = (uint64_t)(index[c + 1] - index[c]) * kRecordUnit;
-        if (size <= nkb * 512ull) { bad.store(2); return; }
-        if ((size - nkb * 512ull) % 256) { bad.store(9); return; }
-        uint32_t W = (uint32_t)((size - nkb * 512ull) / 256);
+        const uint64_t raw_bytes = raw_part_bytes(d.dtype, nkb);
+        if (size <= raw_bytes) { bad.store(2); return; }
+        if ((size - raw_bytes) % 256) { bad.store(9); return; }
+        uint32_t W = (uint32_t)((size - raw_bytes) / 256);
         if (W > d.max_words) { bad.store(3); return; }
         uint32_t seen = max_words.load();
         while (W > seen && !max_words.compare_exchange_weak(seen, W)) {}
         const uint8_t *raw = base + d.off_payload + (uint64_t)index[c] * kRecordUnit;
-        const uint32_t *coded = (const uint32_t *)(raw + nkb * 512ull);
+        const uint32_t *coded = (const uint32_t *)(raw + raw_bytes);
         uint64_t sum = 0;
+        if (fp16)
+            for (uint64_t b = nkb * 64ull; b < raw_bytes; ++b)
+                if (raw[b]) { bad.store(10); return; }          // padding behind the sign bits
         for (uint32_t lane = 0; lane < kSeqs; ++lane) {
             auto word = [&](uint32_t j) -> uint64_t { return j < W ? coded[(size_t)j * kSeqs + lane] : 0; };
-            if (word(0) & ((1u << kLagBits) - 1)) { bad.store(4); return; }
-            uint32_t pos = kLagBits;
+            if (word(0) & ((1u << d.lag_bits) - 1)) { bad.store(4); return; }
+            uint32_t pos = d.lag_bits;
             for (uint32_t s = 0; s < steps; ++s) {
+                uint32_t ln = lane & 31, half = lane >> 5, gg = ln >> 2, t = ln & 3, kb = s >> 3, i = s & 7;
+                uint64_t r = (uint64_t)rg * 16 + gg + 8 * half, col = (uint64_t)kc * g.Kc + kb * 32ull + t * 8 + i;
+                const bool outside = r >= g.rows || col >= g.cols;
+                if (fp16) {
+                    uint32_t word15 = 0;
+                    for (uint32_t k = 0; k < 3; ++k) {
+                        uint64_t win = (word(pos >> 5) | (word((pos >> 5) + 1) << 32)) >> (pos & 31);
+                        uint32_t e = cb.lut[((size_t)k << d.lut_bits) + ((uint32_t)win & mask)];
+                        uint32_t l = e >> 16;
+                        if (!l) { bad.store(5); return; }
+                        word15 |= e & 0x7FFFu;
+                        pos += l;
+                        sum += l;
+                    }
+                    if (outside) {
+                        uint32_t bit = ((i >> 1) + 4 * half) + 8 * (i & 1);
+                        uint16_t sg = *(const uint16_t *)(raw + kb * 64 + ln * 2);
+                        if (((sg >> bit) & 1) || word15 != d.pad_word) { bad.store(6); return; }
+                    }
+                    continue;
+                }
                 uint64_t win = (word(pos >> 5) | (word((pos >> 5) + 1) << 32)) >> (pos & 31);
                 uint32_t e = cb.lut[(uint32_t)win & mask];
                 uint32_t l = e >> 16;
                 if (!l) { bad.store(5); return; }
-                uint32_t ln = lane & 31, half = lane >> 5, gg = ln >> 2, t = ln & 3, kb = s >> 3, i = s & 7;
-                uint64_t r = (uint64_t)rg * 16 + gg + 8 * half, col = (uint64_t)kc * g.Kc + kb * 32ull + t * 8 + i;
-                if (r >= g.rows || col >= g.cols) {
+                if (outside) {
                     uint8_t rb = raw[(s >> 3) * 512 + ln * 16 + half * 8 + (s & 7)];
                     if (rb != 0 || ((e >> 7) & 0xFFu) != ((d.pad_word >> 7) & 0xFFu)) { bad.store(6); return; }
                 }
@@ -637,7 +736,7 @@ huffllm_status huffllm_validate_blob(const void *blob, size_t bytes, huffllm_des
     if (total_bits.load() != d.coded_bits) return fail(HUFFLLM_ERR_CORRUPT, "coded_bits does not match the payload");
     if (max_words.load() != d.max_words) return fail(HUFFLLM_ERR_CORRUPT, "max_words does not match the payload");
     if (checksum.load() != d.payload_checksum) return fail(HUFFLLM_ERR_CORRUPT, "payload checksum mismatch");
-    if (d.raw_bits != 8 * d.rows * d.cols) return fail(HUFFLLM_ERR_CORRUPT, "raw_bits does not match the shape");
+    if (d.raw_bits != (fp16 ? 1 : 8) * d.rows * d.cols) return fail(HUFFLLM_ERR_CORRUPT, "raw_bits does not match the shape");
     if (desc_out) *desc_out = d;
     return HUFFLLM_OK;
 }

@@ -12,7 +12,9 @@ namespace huffllm {
 
 constexpr uint32_t kTileRows = 16;      // rows of a chunk tile
 constexpr uint32_t kBlockCols = 32;     // columns of one block (16 weights per lane)
-constexpr uint32_t kLagBits = 7;        // zero bits in front of every bit sequence
+// Zero bits in front of every bit sequence: they put the table index where the device forms a table address from the
+// shifted window with one logic operation (BF16: one table, 128 bytes per entry; FP16: 32 bytes per entry).
+inline uint32_t lag_bits_for(uint32_t dtype) { return dtype == HUFFLLM_FP16 ? 5u : 7u; }
 constexpr uint32_t kSeqs = 64;          // bit sequences per chunk: two per lane (rows g and g + 8)
 constexpr uint32_t kDefaultBudget = 8;  // default joint code-length bound
 constexpr uint32_t kMinBudget = 8, kMaxBudget = 12;
@@ -23,6 +25,12 @@ void clear_error();
 
 // Geometry checks common to host and device calls; returns OK or sets the error.
 huffllm_status check_desc(const huffllm_desc *d);
+
+// Bytes of the raw part of a record with nkb blocks: BF16 one byte per weight; FP16 one sign bit per weight
+// ([block][lane] uint16), padded to the record unit.
+inline uint32_t raw_part_bytes(uint32_t dtype, uint32_t nkb) {
+    return dtype == HUFFLLM_FP16 ? (nkb * 64u + kRecordUnit - 1) / kRecordUnit * kRecordUnit : nkb * 512u;
+}
 
 inline uint32_t blocks_in_chunk(const huffllm_desc &d, uint32_t kc) {
     uint64_t left = d.cols - (uint64_t)kc * d.chunk_cols;

@@ -148,7 +148,10 @@ def test_validator_rejects_damaged_blobs(split):
 def test_argument_errors():
     w = wl.gaussian_weights(16, 64, 0.02, 51)
     with pytest.raises(hl.HuffllmError) as e:
-        hl.build_codebook(w, hl.FP16)
+        hl.build_codebook(w, 7)
+    assert e.value.status_name == "INVALID_ARG"
+    with pytest.raises(hl.HuffllmError) as e:
+        hl.build_codebook(w, hl.FP16, 0, hl.SPLIT_WHOLE_EXPONENT)
     assert e.value.status_name == "UNSUPPORTED"
     with pytest.raises(hl.HuffllmError) as e:
         hl.build_codebook(w, hl.BF16, 5)
@@ -165,6 +168,96 @@ def test_argument_errors():
     assert hl.workspace_bytes(d, 1) > 0
     with pytest.raises(hl.HuffllmError):
         hl.workspace_bytes(d, 65)
+
+
+FP16_SETS = {
+    "fp16": lambda r, c: wl.gaussian_weights(r, c, 0.02, 71, "fp16"),
+    "fp16_from_bf16": lambda r, c: wl.gaussian_weights(r, c, 0.02, 72, "fp16_from_bf16"),
+    "patterns": lambda r, c: wl.all_patterns_weights(r, c, 73),
+    "constant": lambda r, c: np.full((r, c), 0x2E66, dtype=np.uint16),
+}
+
+
+@pytest.mark.parametrize("name", sorted(FP16_SETS))
+@pytest.mark.parametrize("budget", [0, 8, 12])
+def test_fp16_codebook_cost_matches_oracle(name, budget):
+    """FP16 {1,5,5,5}: three codes, each limited on its own."""
+    w = FP16_SETS[name](64, 1024)
+    cb = hl.build_codebook(w, hl.FP16, budget)
+    counts = orc.histogram(w, orc.FP16)
+    olens, ocaps = orc.build_lengths(counts, orc.FP16, budget or 8)
+    for f in range(3):
+        n, c, lens, codes = cb.get(f)
+        assert n == 32 and np.array_equal(c, counts[f][:32])
+        assert kraft_ok(lens) and max(lens) <= (budget or 8)
+        assert np.array_equal(codes, orc.canonical_codes(lens))
+        assert orc.code_cost(c, lens) == orc.code_cost(counts[f], olens[f])
+    cb.free()
+
+
+@pytest.mark.parametrize("rows,cols,ce,budget,gen", [
+    (48, 1056, 1024, 8, "fp16"), (37, 300, 1024, 8, "fp16_from_bf16"), (5, 31, 512, 8, "patterns"),
+    (33, 2080, 4096, 12, "fp16"), (16, 512, 512, 8, "constant"), (64, 1024, 2048, 9, "fp16_from_bf16")])
+def test_fp16_blob_decodes_with_oracle_and_bits_match(rows, cols, ce, budget, gen):
+    w = FP16_SETS[gen](rows, cols)
+    cb = hl.build_codebook(w, hl.FP16, budget)
+    blob, d = hl.encode(cb, w, ce)
+    assert (d.dtype, d.n_fields, d.lag_bits) == (hl.FP16, 3, 5)
+    assert d.blob_bytes == blob.size <= hl.encode_bound(rows, cols, hl.FP16, ce)
+    hl.validate_blob(blob)
+    back, used = orc.decode_blob(blob)
+    assert np.array_equal(back, w)
+    parsed = orc.parse_blob(blob)
+    lens, codes = parsed["lens"], parsed["codes"]
+    assert parsed["dtype"] == orc.FP16 and d.pad_word == orc.pad_word(lens, orc.FP16)
+    flat = np.append(w.ravel(), np.uint16(d.pad_word))
+    for chunk_ids, idx in orc.element_map(rows, cols, ce):
+        n, _, steps = idx.shape
+        S = orc.SEQS
+        bits, off, raw = orc.encode_sequences(flat[idx.reshape(n * S, steps)], lens, codes, orc.FP16)
+        for a, cid in enumerate(chunk_ids):
+            pbits, poff, praw = parsed["chunks"][int(cid)]
+            per = pbits.reshape(S, -1)
+            for l in range(S):
+                lo, hi = int(off[a * S + l]), int(off[a * S + l + 1])
+                assert int(used[int(cid)][l]) == hi - lo
+                assert np.array_equal(per[l, :hi - lo], bits[lo:hi])
+            assert np.array_equal(praw, raw[a * S:a * S + S])          # sign bits, sequence by sequence
+    assert np.array_equal(parsed["lut"], orc.lut_from_code(lens, codes, d.lut_bits, orc.FP16))
+    assert d.coded_bits == sum(int(u.sum()) for u in used.values()) and d.raw_bits == rows * cols
+    cb.free()
+
+
+def test_fp16_validator_rejects_damaged_blobs():
+    w = wl.gaussian_weights(48, 1056, 0.02, 74, "fp16")
+    cb = hl.build_codebook(w, hl.FP16)
+    blob, d = hl.encode(cb, w, 1024)
+    hl.validate_blob(blob)
+    first = int(np.frombuffer(blob.tobytes(), dtype="<u4", count=2, offset=d.off_index)[1]) * 128   # size of record 0
+
+    def damaged(offset, xor=0xFF):
+        b = blob.copy()
+        b[offset] ^= xor
+        with pytest.raises(hl.HuffllmError):
+            hl.validate_blob(b)
+
+    damaged(8, 3)                                # dtype
+    damaged(60, 2)                               # lag_bits
+    damaged(d.off_codebook + 40, 1)              # a code length of the second field
+    damaged(d.off_lut + 4 * 300, 1)              # an entry of the second table
+    damaged(d.off_payload + 128, 0x01)           # a lag bit of record 0 (its raw part is 2 blocks * 64 bytes)
+    damaged(d.off_payload + 128 + 300)           # coded bits
+    damaged(d.off_payload + first - 1, 0x80)     # tail padding of record 0
+
+
+def test_fp16_lands_on_the_papers_bits_per_param():
+    # entropy table and Section 5: true fp16 weights ~13.7 bits/param, bf16-origin weights stored as fp16 ~10.96
+    for gen, lo, hi in (("fp16", 13.55, 13.9), ("fp16_from_bf16", 10.8, 11.15)):
+        w = wl.gaussian_weights(256, 4096, 0.02, 75, gen)
+        cb = hl.build_codebook(w, hl.FP16)
+        blob, d = hl.encode(cb, w, 4096)
+        assert lo <= (d.coded_bits + d.raw_bits) / w.size <= hi
+        cb.free()
 
 
 def test_compression_accounting_on_paper_shaped_weights():
