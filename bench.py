@@ -130,18 +130,20 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def prepare(workload: str, chunk_elems: int, hl, torch, dev, cpu_sample_mats: int = 0, split: int = 0, batch: int = 1):
+def prepare(workload: str, chunk_elems: int, hl, torch, dev, cpu_sample_mats: int = 0, split: int = 0, batch: int = 1,
+            wdtype: str = "bf16"):
     """Generate, encode (host) and upload every matrix of the workload."""
     table, std, seed, _ = WORKLOADS[workload]
     mats = []
     for i, (name, rows, cols) in enumerate(table):
-        w = wl.gaussian_weights(rows, cols, std, seed + i)
-        cb = hl.build_codebook(w, hl.BF16, 0, split)
+        w = wl.gaussian_weights(rows, cols, std, seed + i, wdtype)
+        cb = hl.build_codebook(w, hl.BF16 if wdtype == "bf16" else hl.FP16, 0, split)
         blob, desc = hl.encode(cb, w, chunk_elems)
         cb.free()
-        x = wl.activations(batch, cols, seed + 500 + i)
+        x = wl.activations(batch, cols, seed + 500 + i, "bf16" if wdtype == "bf16" else "fp16")
         ws_bytes = hl.workspace_bytes(desc, batch)
-        alg_bytes = (desc.payload_bytes + 4 * (desc.n_chunks + 1) + (4 << desc.lut_bits) + batch * (2 * cols + 4 * rows))
+        alg_bytes = (desc.payload_bytes + 4 * (desc.n_chunks + 1) + (1 if wdtype == "bf16" else 3) * (4 << desc.lut_bits)
+                     + batch * (2 * cols + 4 * rows))
         mats.append(dict(name=name, rows=rows, cols=cols, desc=desc, blob_dev=torch.from_numpy(blob).to(dev),
                          x_host=torch.from_numpy(x.view(np.int16).reshape(-1)).pin_memory(),
                          y_host=torch.zeros(batch * rows, dtype=torch.float32).pin_memory(),
@@ -155,10 +157,10 @@ def prepare(workload: str, chunk_elems: int, hl, torch, dev, cpu_sample_mats: in
     return mats
 
 
-def oracle_sample_time(hl, w_sample, x_np, chunk_elems: int, repeats: int = 1):
+def oracle_sample_time(hl, w_sample, x_np, chunk_elems: int, repeats: int = 1, fp16: bool = False):
     """Time the CPU oracle (bit-serial decode of the library's blob + fp64 product) on a sample tensor."""
     from oracle import oracle as orc
-    cb = hl.build_codebook(w_sample)
+    cb = hl.build_codebook(w_sample, hl.FP16 if fp16 else hl.BF16)
     blob, _ = hl.encode(cb, w_sample, chunk_elems)
     cb.free()
     orc.lib()
@@ -166,7 +168,7 @@ def oracle_sample_time(hl, w_sample, x_np, chunk_elems: int, repeats: int = 1):
     for _ in range(repeats):
         t0 = time.perf_counter()
         back, _ = orc.decode_blob(blob)
-        y, _ = orc.matmul(back, x_np)
+        y, _ = orc.matmul(back, x_np, orc.FP16 if fp16 else orc.BF16)
         dt = time.perf_counter() - t0
         best = dt if best is None else min(best, dt)
     assert np.array_equal(back, w_sample)
@@ -216,6 +218,9 @@ def main():
                     help="which matrices of the layer share a launch")
     ap.add_argument("--split", default="paper", choices=["paper", "whole-exponent"],
                     help="field split of the blobs: the paper's BF16 {1,4,4,7} or {1,8,7} (one 256-symbol exponent code)")
+    ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16", "fp16_from_bf16"],
+                    help="weight format: bf16 {1,4,4,7} blobs, or fp16 {1,5,5,5} blobs of true fp16 weights / of bf16 weights "
+                         "stored as fp16 (use --chunk-elems 1024 for fp16: larger records do not fit 32 warps' slots)")
     ap.add_argument("--batch", type=int, default=1,
                     help="activation vectors per product (1..64; above 8 every matrix is its own launch on the tcgen05 path)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -245,7 +250,10 @@ def main():
         raise SystemExit("--batch must be in [1, 64]")
     if B > 8:
         args.fuse = "none"           # the tensor-core path takes one matrix per launch
-    mats = prepare(args.workload, args.chunk_elems, hl, torch, dev, cpu_mats, split, B)
+    fp16 = args.dtype != "bf16"
+    if fp16 and B > 8:
+        raise SystemExit("--dtype fp16 takes --batch up to 8 here")
+    mats = prepare(args.workload, args.chunk_elems, hl, torch, dev, cpu_mats, split, B, args.dtype)
     err = torch.zeros(1, dtype=torch.int32, device=dev)
     n_weights = sum(m["rows"] * m["cols"] for m in mats)
     unc_bytes = 2 * n_weights
@@ -327,7 +335,7 @@ def main():
 
     # ---- the dense product the compression competes with: same layer, uncompressed bf16, own kernel and cuBLAS
     plain_ms = cublas_ms = None
-    if rank == 0:
+    if rank == 0 and not fp16:
         try:
             dense = [(torch.randint(-2**15, 2**15, (m["rows"], m["cols"]), dtype=torch.int16, device=dev), m) for m in mats]
             for w_dev, m in dense:
@@ -360,7 +368,7 @@ def main():
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         sample = [m for m in mats if m["w_sample"] is not None]
-        dt = sum(oracle_sample_time(hl, m["w_sample"], m["x_np"], args.chunk_elems, repeats=1) for m in sample)
+        dt = sum(oracle_sample_time(hl, m["w_sample"], m["x_np"], args.chunk_elems, repeats=1, fp16=fp16) for m in sample)
         n_w = sum(m["w_sample"].size for m in sample)
         cpu = {"value": 2.0 * n_w / dt / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
                "sample": f"matrices {[m['name'] for m in sample]} in full ({n_w} weights = {100.0 * n_w / n_weights:.0f} % of the step, "
@@ -373,10 +381,11 @@ def main():
     achieved = alg_bytes / (kernel_ms_step * 1e-3) / 1e9
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "bf16",
+        "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp16" if fp16 else "bf16",
         "data": "synthetic",
         "config": {"workload": args.workload, "what": WORKLOADS[args.workload][3], "chunk_elems": args.chunk_elems, "batch": B,
-                   "split": "bf16 {1,4,4,7}" if args.split == "paper" else "bf16 {1,8,7} (whole exponent)",
+                   "split": ("fp16 {1,5,5,5}" + (" of bf16-origin weights" if args.dtype == "fp16_from_bf16" else "")) if fp16 else
+                            ("bf16 {1,4,4,7}" if args.split == "paper" else "bf16 {1,8,7} (whole exponent)"),
                    "max_code_len": int(mats[0]["desc"].lut_bits), "weights_per_step": n_weights,
                    "uncompressed_bytes": unc_bytes, "compressed_bytes": sum(m["blob_bytes"] for m in mats),
                    "compression_ratio_total": unc_bytes / sum(m["blob_bytes"] for m in mats),

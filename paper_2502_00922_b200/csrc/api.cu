@@ -93,8 +93,11 @@ huffllm_status add_matrix(KernelArgs *k, const huffllm_desc *desc, const void *b
     huffllm_status st = check_desc(desc);
     if (st != HUFFLLM_OK) return st;
     if (!blob || ((uintptr_t)blob & 255)) return fail(HUFFLLM_ERR_INVALID_ARG, "blob must be a 256-byte aligned device pointer");
-    if (desc->lut_bits > 9)
-        return fail(HUFFLLM_ERR_UNSUPPORTED, "device kernels take max_code_len 8 or 9 (this blob: %u)", desc->lut_bits);
+    const uint32_t fmt = desc->dtype == HUFFLLM_FP16 ? 1u : 0u;
+    if (desc->lut_bits > (fmt ? 8u : 9u))
+        return fail(HUFFLLM_ERR_UNSUPPORTED, "device kernels take max_code_len 8%s (this blob: %u)", fmt ? "" : " or 9", desc->lut_bits);
+    if (k->n_mats && k->fmt != fmt) return fail(HUFFLLM_ERR_UNSUPPORTED, "matrices of one call must share the dtype");
+    k->fmt = fmt;
     if (k->n_mats == kMaxMats) return fail(HUFFLLM_ERR_UNSUPPORTED, "at most %u matrices per call", kMaxMats);
     if (k->n_mats && k->lut_bits != desc->lut_bits)
         return fail(HUFFLLM_ERR_UNSUPPORTED, "matrices of one call must share max_code_len");
@@ -116,7 +119,7 @@ huffllm_status add_matrix(KernelArgs *k, const huffllm_desc *desc, const void *b
     // past the last row lands in the next slot, the table or the guard area and is never used
     uint32_t slot = desc->max_words * 256;
     // a corrupt stream can advance its read pointer by one row per refill check and no further
-    const uint32_t checks_per_block = desc->lut_bits == 8 ? 3 : 4;
+    const uint32_t checks_per_block = fmt ? 8 : (desc->lut_bits == 8 ? 3 : 4);
     uint32_t guard = 256 * (3 + checks_per_block * (desc->chunk_cols / kBlockCols));
     if (slot > k->slot_bytes) k->slot_bytes = slot;
     if (guard > k->guard_bytes) k->guard_bytes = guard;
@@ -249,7 +252,7 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
     if (st != HUFFLLM_OK) return st;
     if (batch == 0 || batch > 64) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be in [1, 64]");
     if ((st = check_product_args(desc, x, y, workspace, workspace_bytes, batch)) != HUFFLLM_OK) return st;
-    if (batch > kKernelBatch) {
+    if (batch > kKernelBatch && desc->dtype == HUFFLLM_BF16) {
         // tensor-core path: one pass over the compressed weights for the whole batch
         const TcPlan tp = tc_plan(desc, batch, (uint32_t)dev->sms, (uint32_t)dev->smem_optin - kStaticSmem);
         KernelArgs k;

@@ -57,6 +57,17 @@ __device__ __forceinline__ uint4 ldg_stream16(const void *p) {
                  : "l"(p));
     return v;
 }
+__device__ __forceinline__ uint32_t ldg_stream2(const void *p) {
+    uint16_t v;
+    asm volatile("ld.global.nc.L1::no_allocate.u16 %0, [%1];" : "=h"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void mma_f16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                              uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
 __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
                                                uint32_t b1) {
     asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
@@ -161,6 +172,48 @@ __device__ __forceinline__ void decode_block(LaneStream &sa, LaneStream &sb, uin
     a[5] = pack_pair<0xB3A2u>(e[10], e[11], raw.z);
     a[6] = pack_pair<0x9180u>(e[12], e[13], raw.w);
     a[7] = pack_pair<0xB3A2u>(e[14], e[15], raw.w);
+}
+
+// ------------------------------------------------------------------------------ FP16 {1,5,5,5}
+
+// FP16 blobs code three fields per weight (exponent, upper and lower mantissa half: Section 3.1), each with its own
+// 256-entry table.  The tables sit 8 KB apart, each replicated eight times (entry i of copy c at word 8 i + c; a lane
+// uses copy lane % 8), so the index bits of a lookup address are bits 5..12 and the lag of the stream is 5 bits.
+// A table entry is length << 16 | symbol << (10, 5, 0): the three entries of a weight OR-ed together are its low
+// 15 bits.  One refill check per weight: after it the pointer is below 32, three codewords of at most 8 bits and the
+// lag of the last lookup end at bit 31 + 16 + 13 = 60 of the 64-bit window.
+__device__ __forceinline__ uint32_t fp16_field(LaneStream &s, uint32_t lut_lane, uint32_t table_off) {
+    uint64_t win = ((uint64_t)s.hi << 32) | s.lo;
+    uint32_t t = (uint32_t)(win >> s.pos), addr, e;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(addr) : "r"(t), "r"(0xFFu << 5), "r"(lut_lane));
+    asm("ld.shared.u32 %0, [%1];" : "=r"(e) : "r"(addr + table_off));
+    s.pos = __dp4a(e, 0x00010000u, s.pos);
+    return e;
+}
+__device__ __forceinline__ uint32_t fp16_weight(LaneStream &s, uint32_t lut_lane) {
+    uint32_t e0 = fp16_field(s, lut_lane, 0), e1 = fp16_field(s, lut_lane, 8192), e2 = fp16_field(s, lut_lane, 16384), w;
+    asm("lop3.b32 %0, %1, %2, %3, 0xFE;" : "=r"(w) : "r"(e0), "r"(e1), "r"(e2));
+    return w;                                      // low 16 bits: exponent and mantissa; above: the three lengths mixed
+}
+// Decode one block of an FP16 chunk into 8 packed registers (same order as decode_block).  `signs` is the lane's
+// uint16 of the block: bit p = sign of the first weight of pair p, bit 8 + p = sign of its second weight.
+__device__ __forceinline__ void decode_block_fp16(LaneStream &sa, LaneStream &sb, uint32_t lut_lane, uint32_t one, uint32_t signs,
+                                                  uint32_t (&a)[8]) {
+    uint32_t w[16];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        stream_refill(sa, one);
+        stream_refill(sb, one);
+        w[i] = fp16_weight(sa, lut_lane);
+        w[8 + i] = fp16_weight(sb, lut_lane);
+    }
+    const uint32_t s32 = prmt(signs, 0u, 0x4140u);     // first-weight signs in bits 0..7, second-weight signs in bits 16..23
+#pragma unroll
+    for (int p = 0; p < 8; ++p) {
+        uint32_t pair = prmt(w[2 * p], w[2 * p + 1], 0x5410u);   // low halves of the two weights
+        uint32_t sh = s32 << (15 - p);                            // their sign bits at bits 15 and 31
+        asm("lop3.b32 %0, %1, %2, 0x7FFF7FFF, 0xE4;" : "=r"(a[p]) : "r"(pair), "r"(sh));   // mask bit set: pair, else sign
+    }
 }
 
 // ------------------------------------------------------------------------------ shared memory plan

@@ -40,8 +40,13 @@ namespace huffllm {
 // One launch works through a LIST of matrices (A.n_mats, usually the matrices of one decoder layer that
 // may run together).  The CTAs are dealt out to the matrices in proportion to their chunks, so every CTA
 // lies inside a single matrix, builds a single table and meets no CTA-wide barrier after set-up.
-template <int MODE, int LB, int THREADS>
+// FMT = 0: BF16 blobs; FMT = 1: FP16 {1,5,5,5} blobs (three lookups per weight, sign bits as the raw part).
+template <int MODE, int LB, int THREADS, int FMT>
 __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant__ KernelArgs A) {
+    constexpr uint32_t kRawBlock = FMT ? 64u : 512u;          // raw bytes of one block of a record
+    constexpr uint32_t kRawLane = FMT ? 2u : 16u;             // of which one lane's share
+    // raw part of a record with nkb blocks (FP16: padded to the 128-byte record unit)
+    auto raw_part = [](uint32_t nkb) -> uint32_t { return FMT ? (nkb * 64u + 127u) & ~127u : nkb * 512u; };
     constexpr int R = LB == 8 ? 3 : 2;                       // decoder steps between two refill checks
     constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
     extern __shared__ __align__(128) uint8_t dyn_smem[];
@@ -57,7 +62,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     const uint32_t vals = 16 * A.batch;
     float *part_val = (float *)(dyn_smem + A.dyn_smem_bytes - A.part_bytes);  // [2 * warps][16 * batch]
 
-    uint32_t lut_lane = plan.lut | (lane << 2);
+    uint32_t lut_lane = plan.lut | ((FMT ? lane & 7u : lane) << 2);
     asm volatile("mov.u32 %0, %0;" : "+r"(lut_lane));  // keep it in a register: it is an operand of every lookup
     uint32_t one = 1;
     asm volatile("mov.u32 %0, %0;" : "+r"(one));       // a 1 the compiler cannot see through (see stream_refill)
@@ -96,16 +101,16 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         };
         // a record is usable if it lies inside the payload and its coded part fits a slot
         auto record_ok = [&](uint32_t r0, uint32_t r1, uint32_t nkb) -> bool {
-            return r1 > r0 && r1 <= k.payload_units && (r1 - r0) * 128u > nkb * 512u &&
-                   (r1 - r0) * 128u - nkb * 512u <= A.slot_bytes;
+            return r1 > r0 && r1 <= k.payload_units && (r1 - r0) * 128u > raw_part(nkb) &&
+                   (r1 - r0) * 128u - raw_part(nkb) <= A.slot_bytes;
         };
         // lane 0: start the bulk copy of the coded part of a chunk (column chunk kc_c, record [ra, rb)) into slot `which`
         auto issue_known = [&](uint32_t kc_c, uint32_t ra, uint32_t rb, uint32_t which) {
             const uint32_t nkb = blocks_of(kc_c), bar = bar0 + which * 8;
             if (record_ok(ra, rb, nkb)) {
-                uint32_t bytes = (rb - ra) * 128u - nkb * 512u;
+                uint32_t bytes = (rb - ra) * 128u - raw_part(nkb);
                 mbar_expect_tx(bar, bytes);
-                bulk_g2s(slot0 + which * A.slot_bytes, payload + (uint64_t)ra * 128u + nkb * 512u, bytes, bar);
+                bulk_g2s(slot0 + which * A.slot_bytes, payload + (uint64_t)ra * 128u + raw_part(nkb), bytes, bar);
             } else {
                 mbar_expect_tx(bar, 0);  // completes the phase with nothing to wait for; the chunk is skipped below
             }
@@ -115,14 +120,17 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         // ---- set-up of a segment.  The table loads are started first, then every warp starts its first
         // copies, then the table is written to shared memory: the cold misses on the table, on the record
         // index and on the first records overlap instead of following each other.
-        constexpr int kLutLoads = ((32 << LB) + THREADS - 1) / THREADS;
+        // (FP16: three tables of 256 entries, eight copies each: word j holds entry j / 8 of its table)
+        constexpr uint32_t kLutWords = FMT ? 3u * 8u * 256u : 32u << LB;
+        constexpr uint32_t kLutRep = FMT ? 3u : 5u;            // log2 of the copies per entry
+        constexpr int kLutLoads = (kLutWords + THREADS - 1) / THREADS;
         uint32_t lut_v[kLutLoads];
         {
             const uint32_t *lut_g = (const uint32_t *)(k.blob + k.off_lut);
 #pragma unroll
             for (int i = 0; i < kLutLoads; ++i) {
                 uint32_t j = tid + i * THREADS;
-                lut_v[i] = j < (32u << LB) ? __ldg(lut_g + (j >> 5)) : 0u;
+                lut_v[i] = j < kLutWords ? __ldg(lut_g + (j >> kLutRep)) : 0u;
             }
         }
         if (lane == 0 && c_beg < c_end) {
@@ -134,7 +142,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
 #pragma unroll
             for (int i = 0; i < kLutLoads; ++i) {
                 uint32_t j = tid + i * THREADS;
-                if (j < (32u << LB)) lut_s[j] = lut_v[i];
+                if (j < kLutWords) lut_s[j] = lut_v[i];
             }
             if (tid < kMaxWarps) s_arrive[tid] = 0;
         }
@@ -271,9 +279,13 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
 
                 // records follow each other in memory: the block after this chunk's last one is the first block
                 // of the next record, `coded_bytes` further on
-                const uint8_t *raw_p = payload + (uint64_t)r0 * 128u + lane * 16u;   // raw bytes of block 0
-                const uint32_t coded_bytes = (r1 - r0) * 128u - nkb * 512u;
-                if (ok && !primed) raw_a = ldg_stream16(raw_p);
+                const uint8_t *raw_p = payload + (uint64_t)r0 * 128u + lane * kRawLane;   // raw bytes of block 0
+                const uint32_t coded_bytes = (r1 - r0) * 128u - nkb * kRawBlock;           // from behind the last block to the next record
+                auto load_raw = [](const uint8_t *p) -> uint4 {
+                    if (FMT) return make_uint4(ldg_stream2(p), 0, 0, 0);
+                    return ldg_stream16(p);
+                };
+                if (ok && !primed) raw_a = load_raw(raw_p);
 
                 // wait, with a limit, for the coded part; the outcome is made uniform across the warp
                 {
@@ -314,12 +326,12 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                     // (may_be_last = false: the caller knows that another block of this chunk follows)
                     auto block = [&](uint32_t kb, const uint4 &cur, uint4 &nxt, auto may_be_last) {
                         BLOCKSTAMP((c - c_beg) * 8 + kb, 0);
-                        raw_p += 512;
+                        raw_p += kRawBlock;
                         if (decltype(may_be_last)::value) {
                             if (kb == last) raw_p += coded_bytes;       // the next record's first block
-                            if (kb != last || next_ok) nxt = ldg_stream16(raw_p);
+                            if (kb != last || next_ok) nxt = load_raw(raw_p);
                         } else {
-                            nxt = ldg_stream16(raw_p);
+                            nxt = load_raw(raw_p);
                         }
                         uint4 xv;
                         if (MODE == 1) {
@@ -328,12 +340,18 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                         }
 
                         uint32_t a[8];
-                        decode_block<R>(sa, sb, kIdxMask, lut_lane, one, cur, a);
+                        if (FMT) decode_block_fp16(sa, sb, lut_lane, one, cur.x, a);
+                        else decode_block<R>(sa, sb, kIdxMask, lut_lane, one, cur, a);
                         BLOCKSTAMP((c - c_beg) * 8 + kb, 1);
 
                         if (MODE == 1) {
-                            mma_bf16_16816(acc, a[0], a[4], a[1], a[5], xv.x, xv.y);
-                            mma_bf16_16816(acc, a[2], a[6], a[3], a[7], xv.z, xv.w);
+                            if (FMT) {
+                                mma_f16_16816(acc, a[0], a[4], a[1], a[5], xv.x, xv.y);
+                                mma_f16_16816(acc, a[2], a[6], a[3], a[7], xv.z, xv.w);
+                            } else {
+                                mma_bf16_16816(acc, a[0], a[4], a[1], a[5], xv.x, xv.y);
+                                mma_bf16_16816(acc, a[2], a[6], a[3], a[7], xv.z, xv.w);
+                            }
                             BLOCKSTAMP((c - c_beg) * 8 + kb, 2);
                         } else {
                             const uint32_t col = col0 + kb * 32u;
@@ -413,9 +431,9 @@ __global__ void __launch_bounds__(256) plain_gemv_kernel(const uint16_t *__restr
 
 // ------------------------------------------------------------------------------ launchers
 
-template <int MODE, int LB, int THREADS>
+template <int MODE, int LB, int THREADS, int FMT>
 static cudaError_t launch_one(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
-    auto fn = huff_kernel<MODE, LB, THREADS>;
+    auto fn = huff_kernel<MODE, LB, THREADS, FMT>;
     static bool attr_set[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
@@ -438,11 +456,13 @@ static cudaError_t launch_one(const KernelArgs &k, uint32_t grid, cudaStream_t s
 }
 
 cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
-    return k.lut_bits == 8 ? launch_one<0, 8, kThreads>(k, grid, stream) : launch_one<0, 9, kThreads>(k, grid, stream);
+    if (k.fmt) return launch_one<0, 8, kThreads, 1>(k, grid, stream);
+    return k.lut_bits == 8 ? launch_one<0, 8, kThreads, 0>(k, grid, stream) : launch_one<0, 9, kThreads, 0>(k, grid, stream);
 }
 
 cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
-    return k.lut_bits == 8 ? launch_one<1, 8, kThreads>(k, grid, stream) : launch_one<1, 9, kThreads>(k, grid, stream);
+    if (k.fmt) return launch_one<1, 8, kThreads, 1>(k, grid, stream);
+    return k.lut_bits == 8 ? launch_one<1, 8, kThreads, 0>(k, grid, stream) : launch_one<1, 9, kThreads, 0>(k, grid, stream);
 }
 
 cudaError_t launch_plain_gemv(const uint16_t *w, uint64_t rows, uint64_t cols, const uint16_t *x, float *y, uint32_t sms,

@@ -27,9 +27,9 @@ def torch():
 class Uploaded:
     """A tensor encoded on the host and resident on the device, with its scratch buffers."""
 
-    def __init__(self, hl, torch, w, chunk_elems=4096, budget=0, batch=1, split=0):
+    def __init__(self, hl, torch, w, chunk_elems=4096, budget=0, batch=1, split=0, dtype=0):
         self.w = w
-        cb = hl.build_codebook(w, hl.BF16, budget, split)
+        cb = hl.build_codebook(w, dtype, budget, split)
         self.blob, self.desc = hl.encode(cb, w, chunk_elems)
         cb.free()
         hl.validate_blob(self.blob)
@@ -68,8 +68,8 @@ def gpu_gemm(hl, torch, up, x):
     return res[:batch * rows].reshape(batch, rows)
 
 
-def check_product(y_gpu, w, x):
-    y, d = orc.matmul(w, x)
+def check_product(y_gpu, w, x, dtype=orc.BF16):
+    y, d = orc.matmul(w, x, dtype)
     err = np.abs(y_gpu.astype(np.float64) - y)
     assert np.all(err <= TOL * d + 1e-30), f"max err/bound = {np.max(err / (TOL * d + 1e-30))}"
     assert np.all(y_gpu[d == 0] == 0)
@@ -127,6 +127,47 @@ def test_whole_exponent_split_decode_and_product(hl, torch, rows, cols, ce, budg
     if batch:
         x = wl.activations(batch, cols, 800 + cols)
         check_product(gpu_gemm(hl, torch, up, x), w, x)
+
+
+FP16_GENS = {"fp16": lambda r, c, seed: wl.gaussian_weights(r, c, 0.02, seed, "fp16"),
+             "fp16_from_bf16": lambda r, c, seed: wl.gaussian_weights(r, c, 0.02, seed, "fp16_from_bf16"),
+             "patterns": lambda r, c, seed: wl.all_patterns_weights(r, c, seed),
+             "constant": lambda r, c, seed: np.full((r, c), 0xAE66, dtype=np.uint16)}
+
+
+@pytest.mark.parametrize("rows,cols,ce,gen,batch", [
+    (1024, 1024, 1024, "fp16", 1),                # true fp16 weights: 13.7 bits per weight
+    (37, 300, 512, "fp16_from_bf16", 0),          # ragged rows and columns (decode only)
+    (256, 2048, 1024, "patterns", 0),             # every bit pattern incl. NaN / Inf / denormals (decode only)
+    (5, 31, 512, "patterns", 0),
+    (16, 512, 512, "constant", 2),                # single-symbol codes in all three fields
+    (40, 2080, 1024, "fp16_from_bf16", 3),        # ragged rows, odd number of blocks in the last column chunk
+    (512, 4096, 2048, "fp16_from_bf16", 8),       # larger chunks fit when the weights came from bf16 (10.9 bits per weight)
+    (2368, 512, 512, "fp16", 5),                  # many chunks per warp
+    (272, 2048, 1024, "fp16", 16),                # batch above 8: passes of 8 vectors
+])
+def test_fp16_decode_and_product(hl, torch, rows, cols, ce, gen, batch):
+    """FP16 {1,5,5,5} blobs: bit-exact decode and products within the tolerance, against the oracle."""
+    w = FP16_GENS[gen](rows, cols, 900 + rows)
+    up = Uploaded(hl, torch, w, ce, 0, max(batch, 1), dtype=hl.FP16)
+    assert (up.desc.dtype, up.desc.n_fields) == (hl.FP16, 3)
+    assert np.array_equal(gpu_decode(hl, torch, up), w)
+    if rows * cols <= 300_000:
+        ref, _ = orc.decode_blob(up.blob)
+        assert np.array_equal(ref, w)
+    if batch:
+        x = wl.activations(batch, cols, 950 + cols, "fp16")
+        check_product(gpu_gemm(hl, torch, up, x), w, x, orc.FP16)
+
+
+def test_fp16_large_chunks_run_with_fewer_warps(hl, torch):
+    """Records too large for 32 pairs of shared-memory slots are decoded by as many warps as have room."""
+    w = wl.gaussian_weights(64, 4096, 0.02, 990, "fp16")
+    up = Uploaded(hl, torch, w, 16384, 0, 1, dtype=hl.FP16)
+    assert up.desc.max_words > 64
+    assert np.array_equal(gpu_decode(hl, torch, up), w)
+    x = wl.activations(1, 4096, 991, "fp16")
+    check_product(gpu_gemm(hl, torch, up, x), w, x, orc.FP16)
 
 
 GEMM_CASES = [
