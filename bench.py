@@ -131,13 +131,13 @@ class ClockSampler:
 
 
 def prepare(workload: str, chunk_elems: int, hl, torch, dev, cpu_sample_mats: int = 0, split: int = 0, batch: int = 1,
-            wdtype: str = "bf16"):
+            wdtype: str = "bf16", max_code_len: int = 0):
     """Generate, encode (host) and upload every matrix of the workload."""
     table, std, seed, _ = WORKLOADS[workload]
     mats = []
     for i, (name, rows, cols) in enumerate(table):
         w = wl.gaussian_weights(rows, cols, std, seed + i, wdtype)
-        cb = hl.build_codebook(w, hl.BF16 if wdtype == "bf16" else hl.FP16, 0, split)
+        cb = hl.build_codebook(w, hl.BF16 if wdtype == "bf16" else hl.FP16, max_code_len, split)
         blob, desc = hl.encode(cb, w, chunk_elems)
         cb.free()
         x = wl.activations(batch, cols, seed + 500 + i, "bf16" if wdtype == "bf16" else "fp16")
@@ -218,6 +218,7 @@ def main():
                     help="which matrices of the layer share a launch")
     ap.add_argument("--split", default="paper", choices=["paper", "whole-exponent"],
                     help="field split of the blobs: the paper's BF16 {1,4,4,7} or {1,8,7} (one 256-symbol exponent code)")
+    ap.add_argument("--max-code-len", type=int, default=0, help="L_max of the codebooks (0 = the library's default, 8; the kernels take 8 or 9)")
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16", "fp16_from_bf16"],
                     help="weight format: bf16 {1,4,4,7} blobs, or fp16 {1,5,5,5} blobs of true fp16 weights / of bf16 weights "
                          "stored as fp16 (use --chunk-elems 1024 for fp16: larger records do not fit 32 warps' slots)")
@@ -253,7 +254,7 @@ def main():
     fp16 = args.dtype != "bf16"
     if fp16 and B > 8:
         raise SystemExit("--dtype fp16 takes --batch up to 8 here")
-    mats = prepare(args.workload, args.chunk_elems, hl, torch, dev, cpu_mats, split, B, args.dtype)
+    mats = prepare(args.workload, args.chunk_elems, hl, torch, dev, cpu_mats, split, B, args.dtype, args.max_code_len)
     err = torch.zeros(1, dtype=torch.int32, device=dev)
     n_weights = sum(m["rows"] * m["cols"] for m in mats)
     unc_bytes = 2 * n_weights
