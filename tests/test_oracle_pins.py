@@ -186,6 +186,27 @@ def test_worked_example_bf16():
     assert y[0, 0] == float(g["y"][0]) and d[0, 0] == float(g["abs_sum"][0])
 
 
+def test_worked_example_fp16():
+    g = read_golden("worked_example_fp16.txt")
+    w = np.array([int(x, 16) for x in g["weights_hex"]], dtype=np.uint16)
+    counts = orc.histogram(w, orc.FP16)
+    lens, _ = orc.build_lengths(counts, orc.FP16, 0)
+    codes = orc.codes_for(lens)
+    for field, key in ((0, "exp"), (1, "mhi"), (2, "mlo")):
+        syms = [int(s, 16) for s in g[key + "_symbols"]]
+        assert [int(lens[field][s]) for s in syms] == [int(x) for x in g[key + "_lengths"]]
+        assert [format(int(codes[field][s]), "0{}b".format(int(lens[field][s]))) for s in syms] == g[key + "_codes"]
+        assert int((lens[field] > 0).sum()) == len(syms)
+    bits, off, raw = orc.encode_sequences(w[None, :], lens, codes, orc.FP16)
+    assert "".join(map(str, bits)) == g["bitstream"][0]
+    assert [int(x) for x in raw[0]] == [int(x) for x in g["raw_bits"]]
+    assert len(bits) + 8 == int(g["payload_bits"][0])
+    back, used = orc.decode_sequences(bits, off, raw, lens, codes, orc.FP16)
+    assert np.array_equal(back[0], w) and int(used[0]) == len(bits)
+    y, d = orc.matmul(w[None, :], np.full((1, 8), 0x3C00, dtype=np.uint16), orc.FP16)
+    assert y[0, 0] == float(g["y"][0]) and d[0, 0] == float(g["abs_sum"][0])
+
+
 def test_worked_example_bf16_whole_exponent():
     g = read_golden("worked_example_bf16_whole_exponent.txt")
     w = np.array([int(x, 16) for x in g["weights_hex"]], dtype=np.uint16)
