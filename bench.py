@@ -266,6 +266,10 @@ def main():
                   ys=[mats[i]["y_dev"] for i in g], wss=[mats[i]["ws"] for i in g]) for g in groups]
 
     ws_each = min(m["ws_bytes"] for m in mats)
+    raw_stream = stream.cuda_stream
+    for c, g in zip(calls, groups):      # argument arrays marshalled once per launch group
+        c["prep"] = hl.PreparedMulti(c["descs"], c["blobs"], c["xs"], min(B, 8), c["ys"], c["wss"], ws_each, err,
+                                     [mats[i]["x_host"] for i in g], [mats[i]["y_host"] for i in g])
 
     def step_device():
         if B > 8:
@@ -273,7 +277,7 @@ def main():
                 hl.decode_gemm(m["desc"], m["blob_dev"], m["x_dev"], B, m["y_dev"], m["ws"], m["ws_bytes"], err, stream)
             return
         for c in calls:
-            hl.decode_gemm_multi(c["descs"], c["blobs"], c["xs"], B, c["ys"], c["wss"], ws_each, err, stream)
+            c["prep"].run(raw_stream)
 
     for c, g in zip(calls, groups):
         c["xh"], c["yh"] = [mats[i]["x_host"] for i in g], [mats[i]["y_host"] for i in g]
@@ -285,8 +289,7 @@ def main():
                                     m["ws_bytes"], err, stream)
             return
         for c in calls:
-            hl.decode_gemm_multi_host(c["descs"], c["blobs"], c["xh"], B, c["yh"], c["xs"], c["ys"], c["wss"],
-                                      ws_each, err, stream)
+            c["prep"].run_host(raw_stream)
 
     def barrier():
         if dist is not None:

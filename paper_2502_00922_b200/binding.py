@@ -222,6 +222,37 @@ def decode_gemm_multi_host(descs, blobs_dev, xs_host, batch: int, ys_host, x_sta
                                                 workspace_bytes_each, _ptr(err_flag_dev), _stream(stream)))
 
 
+class PreparedMulti:
+    """The argument arrays of a huffllm_decode_gemm_multi / _multi_host call, marshalled once.  A caller that issues
+    the same launch every step (a decoder layer) pays one foreign call per step instead of rebuilding the arrays.
+    The tensors must stay alive and in place for as long as the object is used."""
+
+    def __init__(self, descs, blobs_dev, xs_dev, batch: int, ys_dev, workspaces_dev, workspace_bytes_each: int,
+                 err_flag_dev=None, xs_host=None, ys_host=None):
+        n = self.n = len(descs)
+        self._keep = (descs, blobs_dev, xs_dev, ys_dev, workspaces_dev, err_flag_dev, xs_host, ys_host)
+        self.descs = (C.POINTER(Desc) * n)(*[C.pointer(d) for d in descs])
+        ptrs = lambda seq: (C.c_void_p * n)(*[_ptr(t) for t in seq])
+        self.blobs, self.xs, self.ys, self.wss = ptrs(blobs_dev), ptrs(xs_dev), ptrs(ys_dev), ptrs(workspaces_dev)
+        self.xh = ptrs(xs_host) if xs_host is not None else None
+        self.yh = ptrs(ys_host) if ys_host is not None else None
+        self.batch, self.ws_each, self.err = batch, workspace_bytes_each, _ptr(err_flag_dev)
+        self._fn, self._fn_host = lib().huffllm_decode_gemm_multi, lib().huffllm_decode_gemm_multi_host
+
+    def run(self, stream: int):
+        """Device-resident activations and results; `stream` is the raw cudaStream_t value."""
+        st = self._fn(self.n, self.descs, self.blobs, self.xs, self.batch, self.ys, self.wss, self.ws_each, self.err, stream)
+        if st:
+            _check(st)
+
+    def run_host(self, stream: int):
+        """Host activations in, host results out (returns when the results are on the host)."""
+        st = self._fn_host(self.n, self.descs, self.blobs, self.xh, self.batch, self.yh, self.xs, self.ys, self.wss,
+                           self.ws_each, self.err, stream)
+        if st:
+            _check(st)
+
+
 def decode_gemm_host(desc: Desc, blob_dev, x_host, batch: int, y_host, x_stage_dev, y_stage_dev, workspace_dev,
                      workspace_bytes_: int, err_flag_dev=None, stream=None):
     _check(lib().huffllm_decode_gemm_host(C.byref(desc), _ptr(blob_dev), _ptr(x_host), batch, _ptr(y_host),
