@@ -332,6 +332,39 @@ def test_full_size_layer_matrix_sampled(hl, torch):
     assert np.array_equal(yn, -y)
 
 
+@pytest.mark.parametrize("fuse", ["deps", "all"])
+def test_full_layer_in_the_benchmarks_launch_groups_sampled(hl, torch, fuse):
+    """The whole Llama-7B-shaped layer exactly as bench.py runs it (same generators, same launch groups, the prepared
+    multi-matrix call): sampled rows of all seven products against the oracle, twice (results are reproducible)."""
+    import bench
+    dev = torch.device("cuda", 0)
+    mats = bench.prepare("llama7b_layer", 4096, hl, torch, dev, cpu_sample_mats=7)
+    groups = bench.launch_groups(wl.LAYER_LLAMA7B, fuse)
+    err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.current_stream().cuda_stream
+    preps = [hl.PreparedMulti([mats[i]["desc"] for i in g], [mats[i]["blob_dev"] for i in g], [mats[i]["x_dev"] for i in g], 1,
+                              [mats[i]["y_dev"] for i in g], [mats[i]["ws"] for i in g], mats[0]["ws_bytes"], err) for g in groups]
+    first = None
+    for rep in range(2):
+        for m in mats:
+            m["y_dev"].fill_(float("nan"))
+        for p in preps:
+            p.run(stream)
+        torch.cuda.synchronize()
+        assert int(err.item()) == 0
+        ys = [m["y_dev"].cpu().numpy() for m in mats]
+        if first is None:
+            first = ys
+        else:
+            assert all(np.array_equal(a, b) for a, b in zip(first, ys))
+    rng = np.random.default_rng(5)
+    for m, y in zip(mats, first):
+        rs = rng.choice(m["rows"], 32, replace=False)
+        yo, d = orc.matmul(m["w_sample"][rs], m["x_np"])
+        assert np.all(np.abs(y[rs] - yo[0]) <= TOL * d[0]), m["name"]
+        assert int(m["ws"][:4096].count_nonzero().item()) == 0
+
+
 STRESS = [
     # generator, chunk_elems — the distribution stress configuration at 4096 x 14336
     ("student", 4096), ("uniform", 4096), ("patterns", 4096), ("gauss", 1024), ("gauss", 16384),
