@@ -55,6 +55,13 @@ def launch_groups(table, fuse: str):
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one fused-product launch over its algorithmic bytes, from the
 # ncu capture summarised in profiles/ (None until a capture exists); traffic = ratio * algorithmic bytes.
+# Integer instructions per weight of the bf16 fused kernel (per lane): what the decoder formulation needs (window shift,
+# table address, pointer advance; 1.5 for the pack; 4 per refill check, 3 checks per 8 weights) and what the kernel
+# executes (per-opcode counters of the ncu capture summarised in profiles/: LOP3, SHF, IDP, IMAD, VIADD, ISETP, PRMT, SEL,
+# IADD3, LEA, MOV, PLOP3).  B200 issues 64 32-bit integer lane-operations per clock and SM (16 lanes per scheduler).
+INT_OPS_ALGORITHMIC = 6.0
+INT_OPS_EXECUTED = 7.83
+INT_LANES_PER_CLK_PER_SM = 64
 NCU_TRAFFIC_RATIO = 1.02   # profiles/huff_kernel_product_llama7b_layer.md: 145.7 MB moved for 142.0 MB (gate+up), 71.8 for 71.0 (down)
 
 
@@ -381,6 +388,7 @@ def main():
     if rank != 0:
         return
     peak, peak_src = measured_peak()
+    n_sms = torch.cuda.get_device_properties(dev).multi_processor_count
     value = whole_job_value(unc_bytes, world, ms_step)
     achieved = alg_bytes / (kernel_ms_step * 1e-3) / 1e9
     out = {
@@ -406,6 +414,16 @@ def main():
                      "frac_of_nominal_8TBs": achieved / 8000.0,
                      "per_matrix": [{"name": m["name"], "rows": m["rows"], "cols": m["cols"], "ms": t,
                                      "comp_GBs": m["alg_bytes"] / (t * 1e-3) / 1e9} for m, t in zip(mats, per_mat_ms)]},
+        # what actually binds the bf16 kernel: 32-bit integer issue; peak = SMs x 64 lane-ops x SM clock
+        "alu_roofline": None if (fp16 or B > 8) else {
+            "bound": "alu", "unit": "Gop/s",
+            "peak": n_sms * INT_LANES_PER_CLK_PER_SM * (clocks.get("sm_mhz") or 1965.0) * 1e6 / 1e9,
+            "achieved": n_weights * INT_OPS_ALGORITHMIC / (kernel_ms_step * 1e-3) / 1e9,
+            "frac": n_weights * INT_OPS_ALGORITHMIC / (kernel_ms_step * 1e-3) /
+                    (n_sms * INT_LANES_PER_CLK_PER_SM * (clocks.get("sm_mhz") or 1965.0) * 1e6),
+            "int_ops_per_weight_algorithmic": INT_OPS_ALGORITHMIC, "int_ops_per_weight_executed": INT_OPS_EXECUTED,
+            "frac_executed": n_weights * INT_OPS_EXECUTED / (kernel_ms_step * 1e-3) /
+                             (n_sms * INT_LANES_PER_CLK_PER_SM * (clocks.get("sm_mhz") or 1965.0) * 1e6)},
         "cpu_baseline": cpu,
         "e2e": {"value": whole_job_value(unc_bytes, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": B * sum(2 * m["cols"] for m in mats), "d2h_bytes_per_step": B * sum(4 * m["rows"] for m in mats)},
