@@ -117,14 +117,16 @@ __device__ __forceinline__ uint32_t stream_step(LaneStream &s, uint32_t idx_mask
 }
 
 // Refill: once 32 bits have been consumed, slide the window by one word.  Written with predicated
-// instructions so that lanes which need a word and lanes which do not stay converged.
+// instructions so that lanes which need a word and lanes which do not stay converged.  The low word is
+// reloaded from shared memory rather than copied from the high word: a load is not an integer
+// instruction, and 32-bit integer issue is what bounds this kernel.
 // The two additions are written as multiply-adds by a register holding 1 so that they run on the FMA pipe:
 // the 16-lane integer ALU pipe is the busiest unit of this kernel.
 __device__ __forceinline__ void stream_refill(LaneStream &s, uint32_t one) {
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
         "setp.ge.u32 p, %2, 32;\n\t"
-        "@p mov.u32 %0, %1;\n\t"
+        "@p ld.shared.u32 %0, [%3+-256];\n\t"
         "@p ld.shared.u32 %1, [%3];\n\t"
         "@p mad.lo.u32 %3, %4, 256, %3;\n\t"
         "@p mad.lo.u32 %2, %4, 0xFFFFFFE0, %2;\n\t}"
