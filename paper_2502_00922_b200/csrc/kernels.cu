@@ -94,11 +94,9 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         const uint32_t *index = (const uint32_t *)(k.blob + k.off_index);
         const uint8_t *payload = k.blob + k.off_payload;
 
-        // blocks of 32 columns in column chunk kc
-        auto blocks_of = [&](uint32_t kc) -> uint32_t {
-            uint32_t left = (uint32_t)k.cols - kc * k.chunk_cols;
-            return (min(left, k.chunk_cols) + 31u) >> 5;
-        };
+        // blocks of 32 columns in column chunk kc: every chunk is full except, possibly, the last one of a row
+        const uint32_t nkb_tail = ((uint32_t)k.cols - (KC - 1) * k.chunk_cols + 31u) >> 5;
+        auto blocks_of = [&](uint32_t kc) -> uint32_t { return kc + 1 == KC ? nkb_tail : k.chunk_cols >> 5; };
         // a record is usable if it lies inside the payload and its coded part fits a slot
         auto record_ok = [&](uint32_t r0, uint32_t r1, uint32_t nkb) -> bool {
             return r1 > r0 && r1 <= k.payload_units && (r1 - r0) * 128u > raw_part(nkb) &&
@@ -260,12 +258,20 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
             // raw sign/mantissa bytes travel one block ahead of the decoder, in two register sets used in turn
             uint4 raw_a = make_uint4(0, 0, 0, 0), raw_b = make_uint4(0, 0, 0, 0);
             bool primed = false;
+            bool ok = record_ok(r0, r1, blocks_of(kc));               // carried along: every record is checked once
+            // Running pointers.  Records follow each other in memory and so do the columns of a row group's chunks,
+            // so the raw-byte pointer and the activation pointer simply run on from chunk to chunk.
+            const uint8_t *raw_p = payload + (uint64_t)r0 * 128u + lane * kRawLane;
+            const uint16_t *xq = k.x + (MODE == 1 ? (uint64_t)min(g, A.batch - 1) * k.cols + kc * k.chunk_cols + t * 8u : 0);
+            uint32_t which = 0;
+            auto load_raw = [](const uint8_t *p) -> uint4 {
+                if (FMT) return make_uint4(ldg_stream2(p), 0, 0, 0);
+                return ldg_stream16(p);
+            };
 
 #pragma unroll 1
             for (uint32_t c = c_beg; c < c_end; ++c) {
-                const uint32_t which = (c - c_beg) & 1u;
                 const uint32_t nkb = blocks_of(kc);
-                const bool ok = record_ok(r0, r1, nkb);
                 // the chunk after this one: its first raw block is fetched from inside this chunk's loop
                 const bool has_next = c + 1 < c_end;
                 const uint32_t kc1 = kc + 1 == KC ? 0u : kc + 1;
@@ -277,14 +283,8 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                     cur_rg = (int)rg;
                 }
 
-                // records follow each other in memory: the block after this chunk's last one is the first block
-                // of the next record, `coded_bytes` further on
-                const uint8_t *raw_p = payload + (uint64_t)r0 * 128u + lane * kRawLane;   // raw bytes of block 0
-                const uint32_t coded_bytes = (r1 - r0) * 128u - nkb * kRawBlock;           // from behind the last block to the next record
-                auto load_raw = [](const uint8_t *p) -> uint4 {
-                    if (FMT) return make_uint4(ldg_stream2(p), 0, 0, 0);
-                    return ldg_stream16(p);
-                };
+                // the block after this chunk's last one is the first block of the next record, `coded_bytes` further on
+                const uint32_t coded_bytes = (r1 - r0) * 128u - nkb * kRawBlock;
                 if (ok && !primed) raw_a = load_raw(raw_p);
 
                 // wait, with a limit, for the coded part; the outcome is made uniform across the warp
@@ -311,14 +311,15 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                 if (!ok) {  // record offsets out of range: report, produce nothing for this chunk, touch no memory
                     if (A.err && lane == 0) atomicExch(A.err, (int32_t)min(c + 1, 0x7FFFFFFFu));
                     primed = false;
+                    raw_p = payload + (uint64_t)r1 * 128u + lane * kRawLane;      // where the next record would start
+                    if (MODE == 1) xq += nkb * 32u;
                 } else {
                     LaneStream sa, sb;
                     stream_open(sa, slot0 + which * A.slot_bytes + (lane << 2));
                     stream_open(sb, slot0 + which * A.slot_bytes + 128u + (lane << 2));
                     const uint32_t col0 = kc * k.chunk_cols + t * 8u;
-                    // activations: lanes of unused output columns repeat the last vector (cols is a multiple of 32
-                    // here, so every block of the chunk lies inside the row)
-                    const uint16_t *xq = k.x + (MODE == 1 ? (uint64_t)min(g, A.batch - 1) * k.cols + col0 : 0);
+                    // (activations: lanes of unused output columns repeat the last vector; cols is a multiple of 32
+                    // here, so every block of the chunk lies inside the row and xq ends the chunk where the next begins)
                     uint16_t *out0 = MODE == 0 ? k.out + ((uint64_t)rg * 16 + g) * k.cols + col0 : nullptr;
                     const uint32_t last = nkb - 1;
 
@@ -391,6 +392,9 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                 if (lane == 0 && c + 2 < c_end) issue_known(kc1 + 1 == KC ? 0u : kc1 + 1, r2, __ldg(index + c + 3), which);
                 r0 = r1;
                 r1 = r2;
+                ok = next_ok;
+                which ^= 1u;
+                if (MODE == 1 && kc1 == 0) xq -= k.cols;              // the next chunk starts the next row group: back to column 0
                 kc = kc1;
                 rg += kc1 == 0 ? 1u : 0u;
             }
