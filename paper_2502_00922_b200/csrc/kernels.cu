@@ -50,7 +50,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     constexpr int R = LB == 8 ? 3 : 2;                       // decoder steps between two refill checks
     constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
     extern __shared__ __align__(128) uint8_t dyn_smem[];
-    __shared__ __align__(8) uint64_t bars[kMaxWarps * 2];
+    __shared__ __align__(16) uint64_t bars[kMaxWarps * 2];     // a warp's two barriers differ in address bit 3 only
     __shared__ uint32_t s_arrive[kMaxWarps];   // arrival counters of row groups shared by several warps
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps_launched = blockDim.x >> 5;
@@ -74,7 +74,6 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         mbar_init(bar0 + 8, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    uint32_t phase = 0;            // bit s = parity of the next completion of this warp's barrier s
     bool waited_prior = false, failed = false;
 
     // the matrix this CTA works in, and the CTA's piece of that matrix's chunks
@@ -264,6 +263,10 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
             const uint8_t *raw_p = payload + (uint64_t)r0 * 128u + lane * kRawLane;
             const uint16_t *xq = k.x + (MODE == 1 ? (uint64_t)min(g, A.batch - 1) * k.cols + kc * k.chunk_cols + t * 8u : 0);
             uint32_t which = 0;
+            // this chunk's slot (the lane's column of it) and barrier, toggled by XOR from chunk to chunk; parity of the
+            // barrier's next completion (each of the two barriers completes every second chunk)
+            uint32_t slot_cur = slot0 + (lane << 2), bar_cur = bar0, par = 0;
+            const uint32_t slot_tog = slot_cur ^ (slot_cur + A.slot_bytes);
             auto load_raw = [](const uint8_t *p) -> uint4 {
                 if (FMT) return make_uint4(ldg_stream2(p), 0, 0, 0);
                 return ldg_stream16(p);
@@ -289,18 +292,16 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
 
                 // wait, with a limit, for the coded part; the outcome is made uniform across the warp
                 {
-                    const uint32_t bar = bar0 + which * 8, parity = (phase >> which) & 1u;
                     uint32_t spins = 0;
-                    bool done = mbar_try_wait(bar, parity);
+                    bool done = mbar_try_wait(bar_cur, par);
                     while (!__all_sync(0xFFFFFFFFu, done)) {
                         if (++spins > kWaitLimit) { failed = true; break; }
-                        done = mbar_try_wait(bar, parity);
+                        done = mbar_try_wait(bar_cur, par);
                     }
                     if (failed) {
                         if (A.err && lane == 0) atomicExch(A.err, -1);
                         break;
                     }
-                    phase ^= 1u << which;
                 }
 
                 if (!waited_prior) {
@@ -315,8 +316,8 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                     if (MODE == 1) xq += nkb * 32u;
                 } else {
                     LaneStream sa, sb;
-                    stream_open(sa, slot0 + which * A.slot_bytes + (lane << 2));
-                    stream_open(sb, slot0 + which * A.slot_bytes + 128u + (lane << 2));
+                    stream_open(sa, slot_cur);
+                    stream_open(sb, slot_cur + 128u);
                     const uint32_t col0 = kc * k.chunk_cols + t * 8u;
                     // (activations: lanes of unused output columns repeat the last vector; cols is a multiple of 32
                     // here, so every block of the chunk lies inside the row and xq ends the chunk where the next begins)
@@ -393,7 +394,10 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                 r0 = r1;
                 r1 = r2;
                 ok = next_ok;
+                par ^= which;                                         // 0, 0, 1, 1, 0, 0, ...
                 which ^= 1u;
+                slot_cur ^= slot_tog;
+                bar_cur ^= 8u;
                 if (MODE == 1 && kc1 == 0) xq -= k.cols;              // the next chunk starts the next row group: back to column 0
                 kc = kc1;
                 rg += kc1 == 0 ? 1u : 0u;
