@@ -55,13 +55,14 @@ def launch_groups(table, fuse: str):
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one fused-product launch over its algorithmic bytes, from the
 # ncu capture summarised in profiles/ (None until a capture exists); traffic = ratio * algorithmic bytes.
-# Integer instructions per weight of the bf16 fused kernel (per lane): what the decoder formulation needs (window shift,
-# table address, pointer advance; 1.5 for the pack; 4 per refill check, 3 checks per 8 weights) and what the kernel
-# executes (per-opcode counters of the ncu capture summarised in profiles/: LOP3, SHF, IDP, IMAD, VIADD, ISETP, PRMT, SEL,
-# IADD3, LEA, MOV, PLOP3).  B200 issues 64 32-bit integer lane-operations per clock and SM (16 lanes per scheduler).
-INT_OPS_ALGORITHMIC = 6.0
-INT_OPS_EXECUTED = 7.83
-INT_LANES_PER_CLK_PER_SM = 64
+# What binds the bf16 fused kernel is instruction dispatch.  A one-off probe on the B200 (8 warps per scheduler, independent
+# chains) gave 2.0 cycles per warp instruction and scheduler for LOP3, SHF, PRMT, IDP4A, ISETP and SEL, and 1.1-1.2 for IMAD,
+# FADD and conflict-free LDS; the kernel's time is the sum of these over its instruction mix.  Per weight-lane step the
+# formulation needs 12.0 dispatch cycles (decoder step: shift 2 + address 2 + lookup 1 + pointer advance 2; pack 2.6; refill
+# check 6.4 x 3/8) and the kernel executes 15.2 (per-opcode counters of the ncu capture in profiles/: 5.56 two-cycle and 4.07 one-cycle instructions).
+DISPATCH_CYCLES_ALGORITHMIC = 12.0
+DISPATCH_CYCLES_EXECUTED = 15.2
+SCHEDULERS_PER_SM = 4
 NCU_TRAFFIC_RATIO = 1.02   # profiles/huff_kernel_product_llama7b_layer.md: 145.7 MB moved for 142.0 MB (gate+up), 71.8 for 71.0 (down)
 
 
@@ -414,16 +415,17 @@ def main():
                      "frac_of_nominal_8TBs": achieved / 8000.0,
                      "per_matrix": [{"name": m["name"], "rows": m["rows"], "cols": m["cols"], "ms": t,
                                      "comp_GBs": m["alg_bytes"] / (t * 1e-3) / 1e9} for m, t in zip(mats, per_mat_ms)]},
-        # what actually binds the bf16 kernel: 32-bit integer issue; peak = SMs x 64 lane-ops x SM clock
+        # what actually binds the bf16 kernel: instruction dispatch; peak = dispatch cycles the GPU has per
+        # second (SMs x 4 schedulers x SM clock), achieved = dispatch cycles the decoder formulation needs for the step's weights
         "alu_roofline": None if (fp16 or B > 8) else {
-            "bound": "alu", "unit": "Gop/s",
-            "peak": n_sms * INT_LANES_PER_CLK_PER_SM * (clocks.get("sm_mhz") or 1965.0) * 1e6 / 1e9,
-            "achieved": n_weights * INT_OPS_ALGORITHMIC / (kernel_ms_step * 1e-3) / 1e9,
-            "frac": n_weights * INT_OPS_ALGORITHMIC / (kernel_ms_step * 1e-3) /
-                    (n_sms * INT_LANES_PER_CLK_PER_SM * (clocks.get("sm_mhz") or 1965.0) * 1e6),
-            "int_ops_per_weight_algorithmic": INT_OPS_ALGORITHMIC, "int_ops_per_weight_executed": INT_OPS_EXECUTED,
-            "frac_executed": n_weights * INT_OPS_EXECUTED / (kernel_ms_step * 1e-3) /
-                             (n_sms * INT_LANES_PER_CLK_PER_SM * (clocks.get("sm_mhz") or 1965.0) * 1e6)},
+            "bound": "alu", "unit": "G dispatch cycles/s",
+            "peak": n_sms * SCHEDULERS_PER_SM * (clocks.get("sm_mhz") or 1965.0) * 1e6 / 1e9,
+            "achieved": n_weights / 32 * DISPATCH_CYCLES_ALGORITHMIC / (kernel_ms_step * 1e-3) / 1e9,
+            "frac": n_weights / 32 * DISPATCH_CYCLES_ALGORITHMIC / (kernel_ms_step * 1e-3) /
+                    (n_sms * SCHEDULERS_PER_SM * (clocks.get("sm_mhz") or 1965.0) * 1e6),
+            "cycles_per_32_weights_algorithmic": DISPATCH_CYCLES_ALGORITHMIC, "cycles_per_32_weights_executed": DISPATCH_CYCLES_EXECUTED,
+            "frac_executed": n_weights / 32 * DISPATCH_CYCLES_EXECUTED / (kernel_ms_step * 1e-3) /
+                             (n_sms * SCHEDULERS_PER_SM * (clocks.get("sm_mhz") or 1965.0) * 1e6)},
         "cpu_baseline": cpu,
         "e2e": {"value": whole_job_value(unc_bytes, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": B * sum(2 * m["cols"] for m in mats), "d2h_bytes_per_step": B * sum(4 * m["rows"] for m in mats)},
