@@ -105,7 +105,7 @@ typedef struct huffllm_desc {
     uint32_t col_chunks;      /* ceil(cols / chunk_cols)                                   */
     uint64_t n_chunks;        /* row_groups * col_chunks                                   */
     uint32_t lut_bits;        /* L_max: BF16: of one weight's coded fields together; FP16: of each field (8 .. 12) */
-    uint32_t lag_bits;        /* 7 (BF16 blobs), 5 (FP16 blobs)                            */
+    uint32_t lag_bits;        /* 7 (BF16 blobs), 6 (FP16 blobs)                            */
     uint32_t n_fields;        /* coded fields per weight: 2 (BF16 {1,4,4,7}), 1 ({1,8,7}), 3 (FP16 {1,5,5,5}) */
     uint8_t  caps[4];         /* per-field maximum code length chosen under lut_bits       */
     uint16_t pad_word;        /* weight stored at positions outside the tensor            */

@@ -189,8 +189,8 @@ def matmul(w: np.ndarray, x: np.ndarray, dtype=BF16):
 TILE_ROWS = 16
 BLOCK_COLS = 32
 def lag_bits(dtype: int) -> int:
-    """Zero bits in front of every bit sequence of a blob: 7 for bf16 blobs, 5 for fp16 blobs."""
-    return 5 if dtype == FP16 else 7
+    """Zero bits in front of every bit sequence of a blob: 7 for bf16 blobs, 6 for fp16 blobs."""
+    return 6 if dtype == FP16 else 7
 
 SEQS = 64          # bit sequences per chunk
 
@@ -290,7 +290,7 @@ def decode_tensor(enc) -> np.ndarray:
 # indexed by the next lut_bits stream bits (first bit = bit 0).  index: u32[n_chunks + 1], record offsets in 128-byte
 # units from off_payload.  Record of a chunk with nkb blocks: raw bytes [nkb][32 lanes][16] (a lane's 16
 # bytes: row g's eight weights, then row g+8's), then W rows of 64 little-endian u32 (row j, sequence s):
-# the sequence's bits, bit i in word i // 32 at bit i % 32, starting with lag_bits zero bits (7 for bf16 blobs, 5 for fp16); unused bits
+# the sequence's bits, bit i in word i // 32 at bit i % 32, starting with lag_bits zero bits (7 for bf16 blobs, 6 for fp16); unused bits
 # after the last codeword are zero.
 
 HEADER = struct.Struct("<4sIIIQQIIIIQIII4sHHIQQQQQQQQ")

@@ -115,6 +115,8 @@ huffllm_status add_matrix(KernelArgs *k, const huffllm_desc *desc, const void *b
     m.col_chunks = desc->col_chunks;
     k->total_chunks += m.n_chunks;
     k->lut_bits = desc->lut_bits;
+    k->lut_align = fmt ? 16384u : 128u << desc->lut_bits;
+    k->lut_size = fmt ? 49152u : 128u << desc->lut_bits;
     // a slot holds the W rows of a record; the window runs one row ahead of what it consumes, and that look-ahead
     // past the last row lands in the next slot, the table or the guard area and is never used
     uint32_t slot = desc->max_words * 256;
@@ -130,7 +132,7 @@ huffllm_status add_matrix(KernelArgs *k, const huffllm_desc *desc, const void *b
 huffllm_status finish_args(KernelArgs *k, bool product, const DeviceInfo &dev, uint32_t *grid) {
     k->part_bytes = product ? 2 * 32 * 16 * k->batch * (uint32_t)sizeof(float) : 0;
     // worst case for the table's alignment gap is covered by assuming the window starts within 4 KB of zero
-    uint64_t fixed = (128ull << k->lut_bits) + k->guard_bytes + k->part_bytes + 4096;
+    uint64_t fixed = (uint64_t)k->lut_size + k->guard_bytes + k->part_bytes + 4096;
     if (fixed + 2ull * k->slot_bytes > k->dyn_smem_bytes)
         return fail(HUFFLLM_ERR_UNSUPPORTED, "chunk records too large for shared memory (slot %u bytes)", k->slot_bytes);
     uint64_t g = k->total_chunks < (uint64_t)dev.sms ? k->total_chunks : (uint64_t)dev.sms;

@@ -122,16 +122,29 @@ __device__ __forceinline__ uint32_t stream_step(LaneStream &s, uint32_t idx_mask
 // instruction, and 32-bit integer issue is what bounds this kernel.
 // The two additions are written as multiply-adds by a register holding 1 so that they run on the FMA pipe:
 // the 16-lane integer ALU pipe is the busiest unit of this kernel.
+template <bool RELOAD = true>
 __device__ __forceinline__ void stream_refill(LaneStream &s, uint32_t one) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ge.u32 p, %2, 32;\n\t"
-        "@p ld.shared.u32 %0, [%3+-256];\n\t"
-        "@p ld.shared.u32 %1, [%3];\n\t"
-        "@p mad.lo.u32 %3, %4, 256, %3;\n\t"
-        "@p mad.lo.u32 %2, %4, 0xFFFFFFE0, %2;\n\t}"
-        : "+r"(s.lo), "+r"(s.hi), "+r"(s.pos), "+r"(s.nxt)
-        : "r"(one));
+    if (RELOAD) {
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ge.u32 p, %2, 32;\n\t"
+            "@p ld.shared.u32 %0, [%3+-256];\n\t"
+            "@p ld.shared.u32 %1, [%3];\n\t"
+            "@p mad.lo.u32 %3, %4, 256, %3;\n\t"
+            "@p mad.lo.u32 %2, %4, 0xFFFFFFE0, %2;\n\t}"
+            : "+r"(s.lo), "+r"(s.hi), "+r"(s.pos), "+r"(s.nxt)
+            : "r"(one));
+    } else {   // where shared-memory bandwidth is the scarcer resource (FP16 blobs): copy the register instead
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "setp.ge.u32 p, %2, 32;\n\t"
+            "@p mov.u32 %0, %1;\n\t"
+            "@p ld.shared.u32 %1, [%3];\n\t"
+            "@p mad.lo.u32 %3, %4, 256, %3;\n\t"
+            "@p mad.lo.u32 %2, %4, 0xFFFFFFE0, %2;\n\t}"
+            : "+r"(s.lo), "+r"(s.hi), "+r"(s.pos), "+r"(s.nxt)
+            : "r"(one));
+    }
 }
 
 // Two table entries + two raw bytes -> two bf16 weights packed in one register.
@@ -179,21 +192,23 @@ __device__ __forceinline__ void decode_block(LaneStream &sa, LaneStream &sb, uin
 // ------------------------------------------------------------------------------ FP16 {1,5,5,5}
 
 // FP16 blobs code three fields per weight (exponent, upper and lower mantissa half: Section 3.1), each with its own
-// 256-entry table.  The tables sit 8 KB apart, each replicated eight times (entry i of copy c at word 8 i + c; a lane
-// uses copy lane % 8), so the index bits of a lookup address are bits 5..12 and the lag of the stream is 5 bits.
+// 256-entry table.  The tables sit 16 KB apart, each replicated sixteen times (entry i of copy c at word 16 i + c; a
+// lane uses copy lane % 16: two lanes share a copy and collide when their entries fall into the same bank, which the
+// measured 86 % shared-memory pipe load of an eight-fold version made worth halving), so the index bits of a lookup
+// address are bits 6..13 and the lag of the stream is 6 bits.
 // A table entry is length << 16 | symbol << (10, 5, 0): the three entries of a weight OR-ed together are its low
 // 15 bits.  One refill check per weight: after it the pointer is below 32, three codewords of at most 8 bits and the
-// lag of the last lookup end at bit 31 + 16 + 13 = 60 of the 64-bit window.
+// lag of the last lookup end at bit 31 + 16 + 14 = 61 of the 64-bit window.
 __device__ __forceinline__ uint32_t fp16_field(LaneStream &s, uint32_t lut_lane, uint32_t table_off) {
     uint64_t win = ((uint64_t)s.hi << 32) | s.lo;
     uint32_t t = (uint32_t)(win >> s.pos), addr, e;
-    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(addr) : "r"(t), "r"(0xFFu << 5), "r"(lut_lane));
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(addr) : "r"(t), "r"(0xFFu << 6), "r"(lut_lane));
     asm("ld.shared.u32 %0, [%1];" : "=r"(e) : "r"(addr + table_off));
     s.pos = __dp4a(e, 0x00010000u, s.pos);
     return e;
 }
 __device__ __forceinline__ uint32_t fp16_weight(LaneStream &s, uint32_t lut_lane) {
-    uint32_t e0 = fp16_field(s, lut_lane, 0), e1 = fp16_field(s, lut_lane, 8192), e2 = fp16_field(s, lut_lane, 16384), w;
+    uint32_t e0 = fp16_field(s, lut_lane, 0), e1 = fp16_field(s, lut_lane, 16384), e2 = fp16_field(s, lut_lane, 32768), w;
     asm("lop3.b32 %0, %1, %2, %3, 0xFE;" : "=r"(w) : "r"(e0), "r"(e1), "r"(e2));
     return w;                                      // low 16 bits: exponent and mantissa; above: the three lengths mixed
 }
@@ -204,8 +219,8 @@ __device__ __forceinline__ void decode_block_fp16(LaneStream &sa, LaneStream &sb
     uint32_t w[16];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        stream_refill(sa, one);
-        stream_refill(sb, one);
+        stream_refill<false>(sa, one);
+        stream_refill<false>(sb, one);
         w[i] = fp16_weight(sa, lut_lane);
         w[8 + i] = fp16_weight(sb, lut_lane);
     }
@@ -236,12 +251,12 @@ struct SmemPlan {
 
 __device__ __forceinline__ SmemPlan plan_smem(uint32_t base, const KernelArgs &k, uint32_t max_warps) {   // k: launch-wide fields only
     SmemPlan p;
-    const uint32_t lut_bytes = 128u << k.lut_bits;
+    const uint32_t lut_bytes = k.lut_align;
     uint32_t a0 = (base + 127u) & ~127u;
     p.lut = (base + lut_bytes - 1) / lut_bytes * lut_bytes;
     p.slotA = a0;
     p.nA = p.lut > a0 ? (p.lut - a0) / (2 * k.slot_bytes) : 0;  // a stream that overruns here reads the table: harmless
-    p.slotB = p.lut + lut_bytes;
+    p.slotB = p.lut + k.lut_size;
     uint32_t end = base + k.dyn_smem_bytes - k.part_bytes;
     uint32_t roomB = end > p.slotB + k.guard_bytes ? end - p.slotB - k.guard_bytes : 0;
     p.warps = min(max_warps, p.nA + roomB / (2 * k.slot_bytes));

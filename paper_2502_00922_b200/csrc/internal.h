@@ -13,8 +13,8 @@ namespace huffllm {
 constexpr uint32_t kTileRows = 16;      // rows of a chunk tile
 constexpr uint32_t kBlockCols = 32;     // columns of one block (16 weights per lane)
 // Zero bits in front of every bit sequence: they put the table index where the device forms a table address from the
-// shifted window with one logic operation (BF16: one table, 128 bytes per entry; FP16: 32 bytes per entry).
-inline uint32_t lag_bits_for(uint32_t dtype) { return dtype == HUFFLLM_FP16 ? 5u : 7u; }
+// shifted window with one logic operation (BF16: one table, 128 bytes per entry; FP16: 64 bytes per entry).
+inline uint32_t lag_bits_for(uint32_t dtype) { return dtype == HUFFLLM_FP16 ? 6u : 7u; }
 constexpr uint32_t kSeqs = 64;          // bit sequences per chunk: two per lane (rows g and g + 8)
 constexpr uint32_t kDefaultBudget = 8;  // default joint code-length bound
 constexpr uint32_t kMinBudget = 8, kMaxBudget = 12;

@@ -62,7 +62,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     const uint32_t vals = 16 * A.batch;
     float *part_val = (float *)(dyn_smem + A.dyn_smem_bytes - A.part_bytes);  // [2 * warps][16 * batch]
 
-    uint32_t lut_lane = plan.lut | ((FMT ? lane & 7u : lane) << 2);
+    uint32_t lut_lane = plan.lut | ((FMT ? lane & 15u : lane) << 2);
     asm volatile("mov.u32 %0, %0;" : "+r"(lut_lane));  // keep it in a register: it is an operand of every lookup
     uint32_t one = 1;
     asm volatile("mov.u32 %0, %0;" : "+r"(one));       // a 1 the compiler cannot see through (see stream_refill)
@@ -117,9 +117,9 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         // ---- set-up of a segment.  The table loads are started first, then every warp starts its first
         // copies, then the table is written to shared memory: the cold misses on the table, on the record
         // index and on the first records overlap instead of following each other.
-        // (FP16: three tables of 256 entries, eight copies each: word j holds entry j / 8 of its table)
-        constexpr uint32_t kLutWords = FMT ? 3u * 8u * 256u : 32u << LB;
-        constexpr uint32_t kLutRep = FMT ? 3u : 5u;            // log2 of the copies per entry
+        // (FP16: three tables of 256 entries, sixteen copies each: word j holds entry j / 16 of its table)
+        constexpr uint32_t kLutWords = FMT ? 3u * 16u * 256u : 32u << LB;
+        constexpr uint32_t kLutRep = FMT ? 4u : 5u;            // log2 of the copies per entry
         constexpr int kLutLoads = (kLutWords + THREADS - 1) / THREADS;
         uint32_t lut_v[kLutLoads];
         {

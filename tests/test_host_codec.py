@@ -202,7 +202,7 @@ def test_fp16_blob_decodes_with_oracle_and_bits_match(rows, cols, ce, budget, ge
     w = FP16_SETS[gen](rows, cols)
     cb = hl.build_codebook(w, hl.FP16, budget)
     blob, d = hl.encode(cb, w, ce)
-    assert (d.dtype, d.n_fields, d.lag_bits) == (hl.FP16, 3, 5)
+    assert (d.dtype, d.n_fields, d.lag_bits) == (hl.FP16, 3, 6)
     assert d.blob_bytes == blob.size <= hl.encode_bound(rows, cols, hl.FP16, ce)
     hl.validate_blob(blob)
     back, used = orc.decode_blob(blob)
