@@ -253,6 +253,16 @@ huffllm_status huffllm_decode_gemm_multi_host(uint32_t n, const huffllm_desc *co
                                               int32_t *err_flag_dev, huffllm_stream stream);
 
 /*
+ * The same without the wait: copies, launch and copies back are only enqueued on `stream`; the caller waits for the
+ * stream before it reads ys_host.  Lets the launches of one decoder layer follow each other without a host round trip.
+ */
+huffllm_status huffllm_decode_gemm_multi_host_async(uint32_t n, const huffllm_desc *const *descs, const void *const *blobs_dev,
+                                                    const uint16_t *const *xs_host, uint32_t batch, float *const *ys_host,
+                                                    uint16_t *const *x_stages_dev, float *const *y_stages_dev,
+                                                    void *const *workspaces_dev, size_t workspace_bytes_each,
+                                                    int32_t *err_flag_dev, huffllm_stream stream);
+
+/*
  * (No counterpart in the paper: an engineering addition for callers that cannot allocate.)
  *
  * huffllm_decode_gemm for callers that have no device scratch buffer to hand over and no way to get

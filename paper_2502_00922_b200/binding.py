@@ -49,6 +49,8 @@ _SIGNATURES = {
     "huffllm_decode": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemv": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemm": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
+    "huffllm_decode_gemm_multi_host_async": [C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p,
+                                             C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemm_multi": [C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_size_t,
                                   C.c_void_p, C.c_void_p],
     "huffllm_decode_gemm_multi_host": [C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
@@ -238,10 +240,18 @@ class PreparedMulti:
         self.yh = ptrs(ys_host) if ys_host is not None else None
         self.batch, self.ws_each, self.err = batch, workspace_bytes_each, _ptr(err_flag_dev)
         self._fn, self._fn_host = lib().huffllm_decode_gemm_multi, lib().huffllm_decode_gemm_multi_host
+        self._fn_host_async = lib().huffllm_decode_gemm_multi_host_async
 
     def run(self, stream: int):
         """Device-resident activations and results; `stream` is the raw cudaStream_t value."""
         st = self._fn(self.n, self.descs, self.blobs, self.xs, self.batch, self.ys, self.wss, self.ws_each, self.err, stream)
+        if st:
+            _check(st)
+
+    def run_host_async(self, stream: int):
+        """Host activations in, host results out, enqueued only: wait for the stream before reading the results."""
+        st = self._fn_host_async(self.n, self.descs, self.blobs, self.xh, self.batch, self.yh, self.xs, self.ys, self.wss,
+                                 self.ws_each, self.err, stream)
         if st:
             _check(st)
 

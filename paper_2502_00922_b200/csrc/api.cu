@@ -304,10 +304,10 @@ huffllm_status huffllm_decode_gemv(const huffllm_desc *desc, const void *blob, c
     return huffllm_decode_gemm(desc, blob, x, 1, y, workspace, workspace_bytes, err_flag, stream);
 }
 
-huffllm_status huffllm_decode_gemm_multi_host(uint32_t n, const huffllm_desc *const *descs, const void *const *blobs,
-                                              const uint16_t *const *xs_host, uint32_t batch, float *const *ys_host,
-                                              uint16_t *const *x_stages, float *const *y_stages, void *const *workspaces,
-                                              size_t workspace_bytes_each, int32_t *err_flag, huffllm_stream stream) {
+huffllm_status huffllm_decode_gemm_multi_host_async(uint32_t n, const huffllm_desc *const *descs, const void *const *blobs,
+                                                    const uint16_t *const *xs_host, uint32_t batch, float *const *ys_host,
+                                                    uint16_t *const *x_stages, float *const *y_stages, void *const *workspaces,
+                                                    size_t workspace_bytes_each, int32_t *err_flag, huffllm_stream stream) {
     clear_error();
     if (!descs || !xs_host || !ys_host || !x_stages || !y_stages) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
     if (n == 0 || n > kMaxMats) return fail(HUFFLLM_ERR_INVALID_ARG, "between 1 and %u matrices per call", kMaxMats);
@@ -324,7 +324,17 @@ huffllm_status huffllm_decode_gemm_multi_host(uint32_t n, const huffllm_desc *co
         cudaError_t e = cudaMemcpyAsync(ys_host[i], y_stages[i], (size_t)batch * descs[i]->rows * 4, cudaMemcpyDeviceToHost, s);
         if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "copy of y: %s", cudaGetErrorString(e));
     }
-    cudaError_t e = cudaStreamSynchronize(s);
+    return HUFFLLM_OK;
+}
+
+huffllm_status huffllm_decode_gemm_multi_host(uint32_t n, const huffllm_desc *const *descs, const void *const *blobs,
+                                              const uint16_t *const *xs_host, uint32_t batch, float *const *ys_host,
+                                              uint16_t *const *x_stages, float *const *y_stages, void *const *workspaces,
+                                              size_t workspace_bytes_each, int32_t *err_flag, huffllm_stream stream) {
+    huffllm_status st = huffllm_decode_gemm_multi_host_async(n, descs, blobs, xs_host, batch, ys_host, x_stages, y_stages, workspaces,
+                                                             workspace_bytes_each, err_flag, stream);
+    if (st != HUFFLLM_OK) return st;
+    cudaError_t e = cudaStreamSynchronize((cudaStream_t)stream);
     if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "waiting for the stream: %s", cudaGetErrorString(e));
     return HUFFLLM_OK;
 }

@@ -232,6 +232,15 @@ def test_several_matrices_in_one_launch(hl, torch, batch):
                               ups[0].ws_bytes, err)
     for u, x, y in zip(ups, xs, yh):
         check_product(y.numpy().reshape(batch, -1), u.w, x)
+    # and enqueued only, through the prepared call: the caller waits for the stream
+    for y in yh:
+        y.fill_(float("nan"))
+    prep = hl.PreparedMulti([u.desc for u in ups], [u.blob_dev for u in ups], x_devs, batch, ys, [u.ws for u in ups],
+                            ups[0].ws_bytes, err, xh, yh)
+    prep.run_host_async(torch.cuda.current_stream().cuda_stream)
+    torch.cuda.current_stream().synchronize()
+    for u, x, y in zip(ups, xs, yh):
+        check_product(y.numpy().reshape(batch, -1), u.w, x)
 
 
 def test_product_closed_forms(hl, torch):
