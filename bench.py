@@ -355,6 +355,23 @@ def main():
     per_mat_ms = [statistics.median(ev[s][i].elapsed_time(ev[s][i + 1]) for s in range(n_b)) for i in range(len(mats))]
     kernel_ms_step = ms_step              # launches run back to back: average launch duration = step time / launches
 
+    # ---- the same step as ONE launch over all matrices (valid where the products are independent, as they are here; a
+    # decoder layer's data dependencies allow only the default grouping): reported beside the headline, not as it
+    one_launch_ms = None
+    if B <= 8 and len(mats) > 1 and len(groups) > 1 and len(mats) <= 8:
+        allp = hl.PreparedMulti([m["desc"] for m in mats], [m["blob_dev"] for m in mats], [m["x_dev"] for m in mats], B,
+                                [m["y_dev"] for m in mats], [m["ws"] for m in mats], ws_each, err)
+        for _ in range(args.warmup):
+            allp.run(raw_stream)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        a.record(stream)
+        for _ in range(args.steps):
+            allp.run(raw_stream)
+        b.record(stream)
+        barrier()
+        one_launch_ms = max_over_ranks(a.elapsed_time(b) / args.steps, dist, dev)
+
     # ---- end to end through the host-buffer call: x from pinned host memory, y back to the host, every launch
     for _ in range(args.warmup):
         step_host()
@@ -433,6 +450,10 @@ def main():
                      "peak_source": peak_src, "kernel": "huff_kernel<product>" if B <= 8 else "huff_gemm_tc_kernel", "launches_per_step": len(groups), "fuse": args.fuse,
                      "algorithmic_bytes_per_step": alg_bytes, "kernel_ms_per_step": kernel_ms_step,
                      "frac_of_nominal_8TBs": achieved / 8000.0,
+                     "one_launch": None if not one_launch_ms else {
+                         "ms_per_step": one_launch_ms, "value": whole_job_value(unc_bytes, world, one_launch_ms),
+                         "frac": alg_bytes / (one_launch_ms * 1e-3) / 1e9 / peak,
+                         "note": "all matrices of the step in one launch: only valid where their inputs are independent"},
                      "per_matrix": [{"name": m["name"], "rows": m["rows"], "cols": m["cols"], "ms": t,
                                      "comp_GBs": m["alg_bytes"] / (t * 1e-3) / 1e9} for m, t in zip(mats, per_mat_ms)]},
         # what actually binds the bf16 kernel: instruction dispatch; peak = dispatch cycles the GPU has per
