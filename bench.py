@@ -372,6 +372,24 @@ def main():
         barrier()
         one_launch_ms = max_over_ranks(a.elapsed_time(b) / args.steps, dist, dev)
 
+    # ---- plain decompression of the same blobs to 16-bit weights (huffllm_decode): reads the blobs, writes 2 bytes per weight
+    decode_ms = None
+    if rank == 0:
+        big = max(mats, key=lambda m: m["rows"] * m["cols"])
+        out_dev = torch.empty(big["rows"] * big["cols"], dtype=torch.int16, device=dev)
+        n_d = min(args.steps, 100)
+        for it in range(3 + n_d):
+            if it == 3:
+                torch.cuda.synchronize()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(stream)
+            for m in mats:
+                hl.decode(m["desc"], m["blob_dev"], out_dev, err, stream)
+        b.record(stream)
+        torch.cuda.synchronize()
+        decode_ms = a.elapsed_time(b) / n_d
+        del out_dev
+
     # ---- end to end through the host-buffer call: x from pinned host memory, y back to the host, every launch
     for _ in range(args.warmup):
         step_host()
@@ -470,6 +488,10 @@ def main():
         "cpu_baseline": cpu,
         "e2e": {"value": whole_job_value(unc_bytes, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": B * sum(2 * m["cols"] for m in mats), "d2h_bytes_per_step": B * sum(4 * m["rows"] for m in mats)},
+        "decode_only": None if not decode_ms else {
+            "ms_per_step": decode_ms, "uncompressed_GBs": unc_bytes / (decode_ms * 1e-3) / 1e9,
+            "hbm_GBs_read_plus_written": (sum(m["blob_bytes"] for m in mats) + unc_bytes) / (decode_ms * 1e-3) / 1e9,
+            "note": "huffllm_decode of every matrix of the step, one launch each, into a device buffer"},
         "gpu_launches": len(groups) * args.steps,
         "clocks": clocks,
         "dense_bf16_gemv": {"own_kernel_ms_per_step": plain_ms, "cublas_mv_ms_per_step": cublas_ms,
