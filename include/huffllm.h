@@ -81,8 +81,11 @@ typedef struct huffllm_codebook huffllm_codebook;
  * l = 4 g + t (g < 8, t < 4) owns rows g and g + 8 of the tile and columns 8t .. 8t+7 of every
  * block, as two independent bit sequences: sequence l holds row g's weights, sequence 32 + l
  * holds row g + 8's, block after block (eight weights per block each).  Positions outside the
- * tensor hold `pad_word`.  Record = raw bytes [block][lane][16] (BF16 raw byte = sign << 7 |
- * mantissa; a lane's 16 bytes are row g's eight weights, then row g + 8's), then W rows of 64
+ * tensor hold `pad_word`.  Record = raw bytes [block][lane][16] (a lane's 16 bytes are row g's eight
+ * weights, then row g + 8's, in groups of four weights per little-endian 32-bit word: weight j of a
+ * group has its seven mantissa bits in the low bits of byte (0, 2, 1, 3)[j] of the word and its sign in
+ * bit 7 of byte (1, 3, 2, 0)[j], which puts the first pair's bits, and after a rotation by one byte the
+ * second pair's, where a packed pair of bf16 words has them), then W rows of 64
  * little-endian uint32 (row j, sequence s): the sequence's bits, bit i in word i / 32 at bit
  * i % 32.  A sequence starts with `lag_bits` zero bits, then for every weight
  * code(exponent >> 4) code(exponent & 15) (n_fields == 2) or code(exponent) (n_fields == 1); bits after

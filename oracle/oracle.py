@@ -344,7 +344,13 @@ def parse_blob(blob) -> dict:
             assert W >= 1 and raw_bytes + W * 256 == size
             max_words = max(max_words, W)
             if scheme != FP16:
-                raw = np.frombuffer(blob, dtype=np.uint8, count=nkb * 512, offset=beg).reshape(nkb, 32, 2, 8)
+                # a lane's 16 bytes: row g's eight weights, then row g+8's, in groups of four weights per 32-bit word:
+                # weight j of a group has its mantissa in the low 7 bits of byte (0, 2, 1, 3)[j] and its sign in bit 7
+                # of byte (1, 3, 2, 0)[j]
+                by = np.frombuffer(blob, dtype=np.uint8, count=nkb * 512, offset=beg).reshape(nkb, 32, 2, 2, 4)
+                mant = by[..., [0, 2, 1, 3]] & np.uint8(0x7F)
+                sign = by[..., [1, 3, 2, 0]] & np.uint8(0x80)
+                raw = (mant | sign).reshape(nkb, 32, 2, 8)
                 raw = raw.transpose(2, 1, 0, 3).reshape(SEQS, steps).copy()        # [half][lane] -> sequence
             else:
                 # one uint16 per (block, lane): bit p = sign of the first weight of pair p, bit 8 + p of its second;

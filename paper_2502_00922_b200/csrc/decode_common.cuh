@@ -147,19 +147,21 @@ __device__ __forceinline__ void stream_refill(LaneStream &s, uint32_t one) {
     }
 }
 
-// Two table entries + two raw bytes -> two bf16 weights packed in one register.
-// SEL picks raw bytes (i, i+1) of `raw` as (byte, sign-replicated byte) pairs.  The exponent of the
-// even weight is already in place (bits 7..14); the odd entry times 65536 puts its exponent at bits
-// 23..30 and pushes its length out of the word, so one multiply-add (FMA pipe) merges the two.
-template <uint32_t SEL>
-__device__ __forceinline__ uint32_t pack_pair(uint32_t e_even, uint32_t e_odd, uint32_t raw) {
-    uint32_t sm = prmt(raw, 0u, SEL);   // [sign1*0xFF, raw1, sign0*0xFF, raw0]
+// Two table entries + the raw word of their group -> two bf16 weights packed in one register.
+// A raw word holds the sign and mantissa bits of four consecutive weights of a row, laid out so that the first pair's
+// bits already sit where a packed pair of bf16 words has them (mantissas at bits 0..6 and 16..22, signs at 15 and 31)
+// and the second pair's do after a rotation by one byte; the other pair's bits lie in the exponent positions, which
+// the select below takes from the table entries.  The exponent of the even weight is already in place (bits 7..14);
+// the odd entry times 65536 puts its exponent at bits 23..30 and pushes its length out of the word, so one
+// multiply-add merges the two.
+__device__ __forceinline__ uint32_t pack_pair(uint32_t e_even, uint32_t e_odd, uint32_t sm) {
     uint32_t ex;
     asm("mad.lo.u32 %0, %1, 65536, %2;" : "=r"(ex) : "r"(e_odd), "r"(e_even));
     uint32_t w;   // sign and mantissa bits from sm, exponent bits from ex
     asm("lop3.b32 %0, %1, %2, 0x807F807F, 0xE4;" : "=r"(w) : "r"(sm), "r"(ex));
     return w;
 }
+__device__ __forceinline__ uint32_t rotr8(uint32_t v) { return prmt(v, v, 0x0321u); }
 
 // Decode one block (16 weights of this lane) into 8 packed registers:
 // a[0..3] = row g, columns (0,1) (2,3) (4,5) (6,7);  a[4..7] = row g+8, same columns.
@@ -179,14 +181,14 @@ __device__ __forceinline__ void decode_block(LaneStream &sa, LaneStream &sb, uin
         e[i] = stream_step(sa, idx_mask, lut_lane);
         e[8 + i] = stream_step(sb, idx_mask, lut_lane);
     }
-    a[0] = pack_pair<0x9180u>(e[0], e[1], raw.x);
-    a[1] = pack_pair<0xB3A2u>(e[2], e[3], raw.x);
-    a[2] = pack_pair<0x9180u>(e[4], e[5], raw.y);
-    a[3] = pack_pair<0xB3A2u>(e[6], e[7], raw.y);
-    a[4] = pack_pair<0x9180u>(e[8], e[9], raw.z);
-    a[5] = pack_pair<0xB3A2u>(e[10], e[11], raw.z);
-    a[6] = pack_pair<0x9180u>(e[12], e[13], raw.w);
-    a[7] = pack_pair<0xB3A2u>(e[14], e[15], raw.w);
+    a[0] = pack_pair(e[0], e[1], raw.x);
+    a[1] = pack_pair(e[2], e[3], rotr8(raw.x));
+    a[2] = pack_pair(e[4], e[5], raw.y);
+    a[3] = pack_pair(e[6], e[7], rotr8(raw.y));
+    a[4] = pack_pair(e[8], e[9], raw.z);
+    a[5] = pack_pair(e[10], e[11], rotr8(raw.z));
+    a[6] = pack_pair(e[12], e[13], raw.w);
+    a[7] = pack_pair(e[14], e[15], rotr8(raw.w));
 }
 
 // ------------------------------------------------------------------------------ FP16 {1,5,5,5}

@@ -560,7 +560,7 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
         const uint32_t raw_bytes = raw_part_bytes(cb->dtype, nkb);
         uint32_t *coded = (uint32_t *)(raw + raw_bytes);
         memset(coded, 0, (size_t)W * 256);
-        if (fp16) memset(raw, 0, raw_bytes);
+        memset(raw, 0, raw_bytes);
         for (uint32_t lane = 0; lane < kSeqs; ++lane) {
             uint64_t acc = 0;
             uint32_t nacc = d.lag_bits, j = 0;
@@ -583,7 +583,9 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
                     uint32_t f[3] = {(uint32_t)(v >> 10) & 31, (uint32_t)(v >> 5) & 31, (uint32_t)v & 31};
                     for (int k = 0; k < 3; ++k) append(cb->bits5[k][f[k]], cb->len[k][f[k]]);
                 } else {
-                    raw[(s >> 3) * 512 + (lane & 31) * 16 + (lane >> 5) * 8 + (s & 7)] = (uint8_t)(((v >> 8) & 0x80) | (v & 0x7F));
+                    uint8_t *grp = raw + (s >> 3) * 512 + (lane & 31) * 16 + (lane >> 5) * 8 + (s & 4);    // the weight's group of four
+                    grp[kRawMantByte[s & 3]] |= (uint8_t)(v & 0x7F);
+                    grp[kRawSignByte[s & 3]] |= (uint8_t)((v >> 8) & 0x80);
                     uint32_t e = (v >> 7) & 0xFF;
                     append(bits8[e], len8[e]);
                 }
@@ -719,7 +721,8 @@ huffllm_status huffllm_validate_blob(const void *blob, size_t bytes, huffllm_des
                 uint32_t l = e >> 16;
                 if (!l) { bad.store(5); return; }
                 if (outside) {
-                    uint8_t rb = raw[(s >> 3) * 512 + ln * 16 + half * 8 + (s & 7)];
+                    const uint8_t *grp = raw + (s >> 3) * 512 + ln * 16 + half * 8 + (s & 4);
+                    uint8_t rb = (uint8_t)((grp[kRawMantByte[s & 3]] & 0x7F) | (grp[kRawSignByte[s & 3]] & 0x80));
                     if (rb != 0 || ((e >> 7) & 0xFFu) != ((d.pad_word >> 7) & 0xFFu)) { bad.store(6); return; }
                 }
                 pos += l;

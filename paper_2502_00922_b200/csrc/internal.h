@@ -32,6 +32,11 @@ inline uint32_t raw_part_bytes(uint32_t dtype, uint32_t nkb) {
     return dtype == HUFFLLM_FP16 ? (nkb * 64u + kRecordUnit - 1) / kRecordUnit * kRecordUnit : nkb * 512u;
 }
 
+// BF16 raw bytes: the four weights i = 4 q + j of a group share a 32-bit word; weight j's seven mantissa bits go to the
+// low bits of byte kRawMantByte[j] of the word and its sign to bit 7 of byte kRawSignByte[j].
+constexpr uint32_t kRawMantByte[4] = {0, 2, 1, 3};
+constexpr uint32_t kRawSignByte[4] = {1, 3, 2, 0};
+
 inline uint32_t blocks_in_chunk(const huffllm_desc &d, uint32_t kc) {
     uint64_t left = d.cols - (uint64_t)kc * d.chunk_cols;
     uint64_t c = left < d.chunk_cols ? left : d.chunk_cols;
