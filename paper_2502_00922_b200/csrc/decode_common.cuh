@@ -120,30 +120,29 @@ __device__ __forceinline__ uint32_t stream_step(LaneStream &s, uint32_t idx_mask
 // instructions so that lanes which need a word and lanes which do not stay converged.  The low word is
 // reloaded from shared memory rather than copied from the high word: a load is not an integer
 // instruction, and 32-bit integer issue is what bounds this kernel.
-// The two additions are written as multiply-adds by a register holding 1 so that they run on the FMA pipe:
-// the 16-lane integer ALU pipe is the busiest unit of this kernel.
+// (A plain 32-bit addition costs one dispatch cycle; logic, shift, compare, select and byte-permute instructions two.
+// Adding the entry's length by multiply-high with a register holding 65536 is cheap in isolation, 1.35 cycles, but
+// made this kernel 20 % slower: the pointer advance sits on the decoder's dependency chain.)
 template <bool RELOAD = true>
-__device__ __forceinline__ void stream_refill(LaneStream &s, uint32_t one) {
+__device__ __forceinline__ void stream_refill(LaneStream &s) {
     if (RELOAD) {
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
             "setp.ge.u32 p, %2, 32;\n\t"
             "@p ld.shared.u32 %0, [%3+-256];\n\t"
             "@p ld.shared.u32 %1, [%3];\n\t"
-            "@p mad.lo.u32 %3, %4, 256, %3;\n\t"
-            "@p mad.lo.u32 %2, %4, 0xFFFFFFE0, %2;\n\t}"
-            : "+r"(s.lo), "+r"(s.hi), "+r"(s.pos), "+r"(s.nxt)
-            : "r"(one));
+            "@p add.u32 %3, %3, 256;\n\t"
+            "@p add.u32 %2, %2, 0xFFFFFFE0;\n\t}"
+            : "+r"(s.lo), "+r"(s.hi), "+r"(s.pos), "+r"(s.nxt));
     } else {   // where shared-memory bandwidth is the scarcer resource (FP16 blobs): copy the register instead
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
             "setp.ge.u32 p, %2, 32;\n\t"
             "@p mov.u32 %0, %1;\n\t"
             "@p ld.shared.u32 %1, [%3];\n\t"
-            "@p mad.lo.u32 %3, %4, 256, %3;\n\t"
-            "@p mad.lo.u32 %2, %4, 0xFFFFFFE0, %2;\n\t}"
-            : "+r"(s.lo), "+r"(s.hi), "+r"(s.pos), "+r"(s.nxt)
-            : "r"(one));
+            "@p add.u32 %3, %3, 256;\n\t"
+            "@p add.u32 %2, %2, 0xFFFFFFE0;\n\t}"
+            : "+r"(s.lo), "+r"(s.hi), "+r"(s.pos), "+r"(s.nxt));
     }
 }
 
@@ -169,14 +168,14 @@ __device__ __forceinline__ uint32_t rotr8(uint32_t v) { return prmt(v, v, 0x0321
 // R-th step: after a check at least 26 bits are valid in front of the start pointer, enough for R
 // codewords of at most 26/R bits.
 template <int R>
-__device__ __forceinline__ void decode_block(LaneStream &sa, LaneStream &sb, uint32_t idx_mask, uint32_t lut_lane, uint32_t one,
+__device__ __forceinline__ void decode_block(LaneStream &sa, LaneStream &sb, uint32_t idx_mask, uint32_t lut_lane,
                                              const uint4 &raw, uint32_t (&a)[8]) {
     uint32_t e[16];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         if (i % R == 0) {
-            stream_refill(sa, one);
-            stream_refill(sb, one);
+            stream_refill(sa);
+            stream_refill(sb);
         }
         e[i] = stream_step(sa, idx_mask, lut_lane);
         e[8 + i] = stream_step(sb, idx_mask, lut_lane);
@@ -216,13 +215,13 @@ __device__ __forceinline__ uint32_t fp16_weight(LaneStream &s, uint32_t lut_lane
 }
 // Decode one block of an FP16 chunk into 8 packed registers (same order as decode_block).  `signs` is the lane's
 // uint16 of the block: bit p = sign of the first weight of pair p, bit 8 + p = sign of its second weight.
-__device__ __forceinline__ void decode_block_fp16(LaneStream &sa, LaneStream &sb, uint32_t lut_lane, uint32_t one, uint32_t signs,
+__device__ __forceinline__ void decode_block_fp16(LaneStream &sa, LaneStream &sb, uint32_t lut_lane, uint32_t signs,
                                                   uint32_t (&a)[8]) {
     uint32_t w[16];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        stream_refill<false>(sa, one);
-        stream_refill<false>(sb, one);
+        stream_refill<false>(sa);
+        stream_refill<false>(sb);
         w[i] = fp16_weight(sa, lut_lane);
         w[8 + i] = fp16_weight(sb, lut_lane);
     }

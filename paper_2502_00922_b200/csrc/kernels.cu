@@ -64,8 +64,6 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
 
     uint32_t lut_lane = plan.lut | ((FMT ? lane & 15u : lane) << 2);
     asm volatile("mov.u32 %0, %0;" : "+r"(lut_lane));  // keep it in a register: it is an operand of every lookup
-    uint32_t one = 1;
-    asm volatile("mov.u32 %0, %0;" : "+r"(one));       // a 1 the compiler cannot see through (see stream_refill)
     const uint32_t g = lane >> 2, t = lane & 3;
     const uint32_t bar0 = smem_u32(&bars[warp * 2]);
     const uint32_t slot0 = slot_addr(plan, warp, 0, A.slot_bytes);
@@ -342,8 +340,8 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                         }
 
                         uint32_t a[8];
-                        if (FMT) decode_block_fp16(sa, sb, lut_lane, one, cur.x, a);
-                        else decode_block<R>(sa, sb, kIdxMask, lut_lane, one, cur, a);
+                        if (FMT) decode_block_fp16(sa, sb, lut_lane, cur.x, a);
+                        else decode_block<R>(sa, sb, kIdxMask, lut_lane, cur, a);
                         BLOCKSTAMP((c - c_beg) * 8 + kb, 1);
 
                         if (MODE == 1) {

@@ -294,7 +294,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                     if (ok && kb + 1 < nkb) raw_next = ldg_stream16(raw_p + (size_t)(kb + 1) * 512u);
                     if (col_blk + 32 < col_hi) load_x(x_nxt, col_blk + 32);
                     uint32_t a[8];
-                    decode_block<R>(sa, sb, kIdxMask, lut_lane, 1u, raw_cur, a);   // a chunk that is not ok decodes garbage, never out of range
+                    decode_block<R>(sa, sb, kIdxMask, lut_lane, raw_cur, a);   // a chunk that is not ok decodes garbage, never out of range
                     stage_block(a, x_cur, gb == gb_item);
                     raw_cur = raw_next;
                     x_cur = x_nxt;
