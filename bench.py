@@ -56,12 +56,13 @@ FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of one fused-product launch over its algorithmic bytes, from the
 # ncu capture summarised in profiles/ (None until a capture exists); traffic = ratio * algorithmic bytes.
 # What binds the bf16 fused kernel is instruction dispatch.  A one-off probe on the B200 (8 warps per scheduler, independent
-# chains) gave 2.0 cycles per warp instruction and scheduler for LOP3, SHF, PRMT, IDP4A, ISETP and SEL, and 1.1-1.2 for IMAD,
-# FADD and conflict-free LDS; the kernel's time is the sum of these over its instruction mix.  Per weight-lane step the
-# formulation needs 12.0 dispatch cycles (decoder step: shift 2 + address 2 + lookup 1 + pointer advance 2; pack 2.6; refill
-# check 6.4 x 3/8) and the kernel executes 15.2 (per-opcode counters of the ncu capture in profiles/: 5.56 two-cycle and 4.07 one-cycle instructions).
-DISPATCH_CYCLES_ALGORITHMIC = 12.0
-DISPATCH_CYCLES_EXECUTED = 15.2
+# chains) gave 2.0 cycles per warp instruction and scheduler for LOP3, SHF, PRMT, IDP4A, ISETP and SEL, and 1.0-1.2 for integer
+# additions, IMAD with an immediate, FADD and conflict-free LDS; the kernel's time is the sum of these over its instruction
+# mix.  Per weight-lane step the formulation needs 11.4 dispatch cycles (decoder step: shift 2 + address 2 + lookup 1 + pointer
+# advance 2; pack 2.1; refill check 6 x 3/8) and the kernel executes 14.2 (per-opcode counters of the ncu capture in profiles/:
+# 4.89 two-cycle and 4.43 one-cycle instructions).
+DISPATCH_CYCLES_ALGORITHMIC = 11.4
+DISPATCH_CYCLES_EXECUTED = 14.2
 SCHEDULERS_PER_SM = 4
 NCU_TRAFFIC_RATIO = 1.02   # profiles/huff_kernel_product_llama7b_layer.md: 145.7 MB moved for 142.0 MB (gate+up), 71.8 for 71.0 (down)
 
