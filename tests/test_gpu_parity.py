@@ -374,6 +374,36 @@ def test_full_layer_in_the_benchmarks_launch_groups_sampled(hl, torch, fuse):
         assert int(m["ws"][:4096].count_nonzero().item()) == 0
 
 
+def test_launches_can_be_captured_in_a_cuda_graph(hl, torch):
+    """The device calls only enqueue work on the stream they are given (no allocation, no synchronisation), so a
+    step can be captured once and replayed; replays with new activations give the oracle's products."""
+    rows, cols = 512, 4096
+    w = wl.gaussian_weights(rows, cols, 0.02, 77)
+    up = Uploaded(hl, torch, w)
+    x0 = wl.activations(1, cols, 78)
+    x_dev = torch.from_numpy(x0.view(np.int16).reshape(-1)).cuda()
+    y_dev = torch.zeros(rows, dtype=torch.float32, device="cuda")
+    hl.decode_gemv(up.desc, up.blob_dev, x_dev, y_dev, up.ws, up.ws_bytes, up.err)      # first call outside the capture
+    torch.cuda.synchronize()
+    side = torch.cuda.Stream()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        side.wait_stream(torch.cuda.current_stream())
+        with torch.cuda.graph(graph, stream=side):
+            hl.decode_gemv(up.desc, up.blob_dev, x_dev, y_dev, up.ws, up.ws_bytes, up.err, side)
+            hl.decode_gemv(up.desc, up.blob_dev, x_dev, y_dev, up.ws, up.ws_bytes, up.err, side)
+    for seed in (79, 80):
+        x = wl.activations(1, cols, seed)
+        x_dev.copy_(torch.from_numpy(x.view(np.int16).reshape(-1)))
+        y_dev.fill_(float("nan"))
+        torch.cuda.synchronize()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert int(up.err.item()) == 0
+        check_product(y_dev.cpu().numpy()[None, :], w, x)
+        assert int(up.ws[:4096].count_nonzero().item()) == 0
+
+
 STRESS = [
     # generator, chunk_elems — the distribution stress configuration at 4096 x 14336
     ("student", 4096), ("uniform", 4096), ("patterns", 4096), ("gauss", 1024), ("gauss", 16384),
