@@ -248,6 +248,9 @@ def main():
                          "stored as fp16 (use --chunk-elems 1024 for fp16: larger records do not fit 32 warps' slots)")
     ap.add_argument("--batch", type=int, default=1,
                     help="activation vectors per product (1..64; above 8 every matrix is its own launch on the tcgen05 path)")
+    ap.add_argument("--layers", type=int, default=1,
+                    help="sweep through this many decoder layers per step (each layer has its own copy of the blobs in HBM): "
+                         "the per-token pass over a whole model, e.g. --workload 8b_layer --layers 32")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -280,14 +283,20 @@ def main():
         raise SystemExit("--dtype fp16 takes --batch up to 8 here")
     mats = prepare(args.workload, args.chunk_elems, hl, torch, dev, cpu_mats, split, B, args.dtype, args.max_code_len)
     err = torch.zeros(1, dtype=torch.int32, device=dev)
-    n_weights = sum(m["rows"] * m["cols"] for m in mats)
+    L = args.layers
+    if L < 1 or (L > 1 and B > 8):
+        raise SystemExit("--layers must be at least 1 (and takes --batch up to 8)")
+    n_weights = L * sum(m["rows"] * m["cols"] for m in mats)
     unc_bytes = 2 * n_weights
-    alg_bytes = sum(m["alg_bytes"] for m in mats)
+    alg_bytes = L * sum(m["alg_bytes"] for m in mats)
     stream = torch.cuda.current_stream()
 
+    # every layer of the sweep streams its own copy of the blobs from HBM (same content, distinct memory)
+    layer_blobs = [[m["blob_dev"] for m in mats]] + [[m["blob_dev"].clone() for m in mats] for _ in range(L - 1)]
     groups = launch_groups(WORKLOADS[args.workload][0], args.fuse)
-    calls = [dict(descs=[mats[i]["desc"] for i in g], blobs=[mats[i]["blob_dev"] for i in g], xs=[mats[i]["x_dev"] for i in g],
-                  ys=[mats[i]["y_dev"] for i in g], wss=[mats[i]["ws"] for i in g]) for g in groups]
+    calls = [dict(descs=[mats[i]["desc"] for i in g], blobs=[blobs[i] for i in g], xs=[mats[i]["x_dev"] for i in g],
+                  ys=[mats[i]["y_dev"] for i in g], wss=[mats[i]["ws"] for i in g]) for blobs in layer_blobs for g in groups]
+    groups = groups * L              # one entry per launch of the step
 
     ws_each = min(m["ws_bytes"] for m in mats)
     raw_stream = stream.cuda_stream
@@ -359,7 +368,7 @@ def main():
     # ---- the same step as ONE launch over all matrices (valid where the products are independent, as they are here; a
     # decoder layer's data dependencies allow only the default grouping): reported beside the headline, not as it
     one_launch_ms = None
-    if B <= 8 and len(mats) > 1 and len(groups) > 1 and len(mats) <= 8:
+    if L == 1 and B <= 8 and len(mats) > 1 and len(groups) > 1 and len(mats) <= 8:
         allp = hl.PreparedMulti([m["desc"] for m in mats], [m["blob_dev"] for m in mats], [m["x_dev"] for m in mats], B,
                                 [m["y_dev"] for m in mats], [m["ws"] for m in mats], ws_each, err)
         for _ in range(args.warmup):
@@ -375,7 +384,7 @@ def main():
 
     # ---- plain decompression of the same blobs to 16-bit weights (huffllm_decode): reads the blobs, writes 2 bytes per weight
     decode_ms = None
-    if rank == 0:
+    if rank == 0 and L == 1:
         big = max(mats, key=lambda m: m["rows"] * m["cols"])
         out_dev = torch.empty(big["rows"] * big["cols"], dtype=torch.int16, device=dev)
         n_d = min(args.steps, 100)
@@ -435,7 +444,7 @@ def main():
     plain_ms = cublas_ms = None
     if rank == 0 and not fp16:
         try:
-            dense = [(torch.randint(-2**15, 2**15, (m["rows"], m["cols"]), dtype=torch.int16, device=dev), m) for m in mats]
+            dense = [(torch.randint(-2**15, 2**15, (m["rows"], m["cols"]), dtype=torch.int16, device=dev), m) for _ in range(L) for m in mats]
             for w_dev, m in dense:
                 w_dev.view(torch.bfloat16).normal_(0, 0.02)
             def plain():
@@ -482,18 +491,18 @@ def main():
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "fp16" if fp16 else "bf16",
         "data": "synthetic",
-        "config": {"workload": args.workload, "what": WORKLOADS[args.workload][3], "chunk_elems": args.chunk_elems, "batch": B,
+        "config": {"workload": args.workload, "what": WORKLOADS[args.workload][3], "chunk_elems": args.chunk_elems, "batch": B, "layers": L,
                    "split": ("fp16 {1,5,5,5}" + (" of bf16-origin weights" if args.dtype == "fp16_from_bf16" else "")) if fp16 else
                             ("bf16 {1,4,4,7}" if args.split == "paper" else "bf16 {1,8,7} (whole exponent)"),
                    "max_code_len": int(mats[0]["desc"].lut_bits), "weights_per_step": n_weights,
-                   "uncompressed_bytes": unc_bytes, "compressed_bytes": sum(m["blob_bytes"] for m in mats),
-                   "compression_ratio_total": unc_bytes / sum(m["blob_bytes"] for m in mats),
-                   "compression_ratio_payload": 16.0 * n_weights / sum(m["coded_bits"] + m["raw_bits"] for m in mats),
-                   "bits_per_param_payload": sum(m["coded_bits"] + m["raw_bits"] for m in mats) / n_weights,
+                   "uncompressed_bytes": unc_bytes, "compressed_bytes": L * sum(m["blob_bytes"] for m in mats),
+                   "compression_ratio_total": unc_bytes / (L * sum(m["blob_bytes"] for m in mats)),
+                   "compression_ratio_payload": 16.0 * n_weights / (L * sum(m["coded_bits"] + m["raw_bits"] for m in mats)),
+                   "bits_per_param_payload": L * sum(m["coded_bits"] + m["raw_bits"] for m in mats) / n_weights,
                    "l2": "inputs larger than L2: the step streams %.0f MB of compressed weights, L2 is 126 MB" % (alg_bytes / 1e6),
                    "parallelism": "replicas only" if world > 1 else "single GPU",
-                   "launch_groups": [[mats[i]["name"] for i in g] for g in groups],
-                   "tokens_per_s_equiv_one_layer": 1e3 / ms_step},
+                   "launch_groups": [[mats[i]["name"] for i in g] for g in groups[:len(groups) // L]],
+                   "ms_per_layer": ms_step / L, "tokens_per_s_equiv": 1e3 / ms_step},
         "roofline": {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak,
                      "traffic": None if NCU_TRAFFIC_RATIO is None else NCU_TRAFFIC_RATIO * alg_bytes / len(groups),
                      "peak_source": peak_src, "kernel": "huff_kernel<product>" if B <= 8 else "huff_gemm_tc_kernel", "launches_per_step": len(groups), "fuse": args.fuse,
@@ -518,7 +527,8 @@ def main():
                              (n_sms * SCHEDULERS_PER_SM * (clocks.get("sm_mhz") or 1965.0) * 1e6)},
         "cpu_baseline": cpu,
         "e2e": {"value": whole_job_value(unc_bytes, world, e2e_ms), "unit": UNIT, "ms_per_step": e2e_ms, "submission": e2e_mode,
-                "h2d_bytes_per_step": B * sum(2 * m["cols"] for m in mats), "d2h_bytes_per_step": B * sum(4 * m["rows"] for m in mats)},
+                "h2d_bytes_per_step": B * sum(2 * m["cols"] for m in mats), "d2h_bytes_per_step": B * sum(4 * m["rows"] for m in mats),
+                "note": None if L == 1 else "one copy of the activations in, every layer's launches, one copy of the last layer's results out"},
         "decode_only": None if not decode_ms else {
             "ms_per_step": decode_ms, "uncompressed_GBs": unc_bytes / (decode_ms * 1e-3) / 1e9,
             "hbm_GBs_read_plus_written": (sum(m["blob_bytes"] for m in mats) + unc_bytes) / (decode_ms * 1e-3) / 1e9,
