@@ -423,3 +423,41 @@ def lut_from_code(lens, codes, lut_bits: int, dtype=BF16) -> np.ndarray:
             continue                                   # no codeword pair is a prefix of this index
         out[i] = (int(used[0]) << 16) | (((int(seq[0, 0]) >> 7) & 0xFF) << 7)
     return out
+
+
+# ----------------------------------------------------------------- bit-field splits (Section 3.1, entropy table)
+
+def split_fields(w: np.ndarray, widths) -> list:
+    """The fields of every 16-bit word under a split: ``widths`` lists the field widths from the most significant
+    bit down (the table's "1-5-5-5" is [1, 5, 5, 5], "8-8" is [8, 8], "16" is [16]) and must add up to 16."""
+    widths = [int(x) for x in widths]
+    if sum(widths) != 16 or any(x < 1 for x in widths):
+        raise ValueError("field widths must be positive and add up to 16")
+    w = np.ascontiguousarray(w, dtype=np.uint16).ravel().astype(np.uint32)
+    out, hi = [], 16
+    for width in widths:
+        lo = hi - width
+        out.append((w >> np.uint32(lo)) & np.uint32((1 << width) - 1))
+        hi = lo
+    return out
+
+
+def split_histograms(w: np.ndarray, widths) -> list:
+    """Per field, how often each of its 2^width values occurs."""
+    return [np.bincount(f, minlength=1 << int(width)).astype(np.uint64) for f, width in zip(split_fields(w, widths), widths)]
+
+
+def shannon_entropy(counts) -> float:
+    """- sum p log2 p over the symbols that occur, in double precision (bits per symbol)."""
+    c = np.asarray(counts, dtype=np.float64)
+    total = c.sum()
+    if total == 0:
+        return 0.0
+    p = c[c > 0] / total
+    return float(-(p * np.log2(p)).sum())
+
+
+def split_entropy(w: np.ndarray, widths):
+    """One row of the entropy table: the entropy of each field, and their sum = bits per parameter of the split."""
+    per_field = [shannon_entropy(h) for h in split_histograms(w, widths)]
+    return per_field, float(sum(per_field))

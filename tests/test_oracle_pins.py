@@ -384,3 +384,77 @@ def test_matmul_closed_forms():
     p = np.array([[0x4000, 0x3F00, 0x3E80, 0xBF80]], dtype=np.uint16)           # 2, .5, .25, -1
     y, d = orc.matmul(p, np.array([[0x3F80, 0x4000, 0x4080, 0x3F80]], dtype=np.uint16))  # 1 2 4 1
     assert y[0, 0] == 2 + 1 + 1 - 1 and d[0, 0] == 5
+
+
+# ------------------------------------------------------------------ bit-field splits (Section 3.1 entropy table)
+
+def test_split_entropy_hand_sample():
+    g = read_golden("entropy_table_section3_1.txt")
+    w = np.array([int(x, 16) for x in g["sample_hex"]], dtype=np.uint16)
+    widths = [int(x) for x in g["sample_widths"]]
+    per_field, total = orc.split_entropy(w, widths)
+    want = [float(x) for x in g["sample_entropy"]]
+    assert per_field == pytest.approx(want, abs=1e-12) and total == pytest.approx(sum(want), abs=1e-12)
+    h = orc.split_histograms(w, widths)
+    assert [int(h[0][1]), int(h[0][2]), int(h[1][2]), int(h[1][3])] == [6, 2, 4, 4]
+    assert [int(x) for x in h[2][:4]] == [4, 2, 1, 1] and all(int(x.sum()) == 8 for x in h)
+
+
+def test_split_entropy_closed_forms():
+    every = np.arange(65536, dtype=np.uint16)                 # each 16-bit pattern once: every field is uniform
+    for widths in ([16], [8, 8], [1, 5, 5, 5], [4, 4, 4, 4], [1, 4, 4, 7], [3, 13], [1] * 16):
+        per_field, total = orc.split_entropy(every, widths)
+        assert per_field == pytest.approx([float(x) for x in widths], abs=1e-12) and total == pytest.approx(16.0, abs=1e-12)
+    assert orc.split_entropy(np.full(1000, 0x3C00, dtype=np.uint16), [1, 5, 5, 5]) == ([0.0] * 4, 0.0)
+    # a product set (each combination of a field-0 value and a field-1 value exactly once): the fields are
+    # independent, so the sum of the field entropies equals the entropy of the whole word
+    a, b = np.array([3, 77, 200], dtype=np.uint16), np.array([0, 1, 2, 3, 250], dtype=np.uint16)
+    w = ((a[:, None] << 8) | b[None, :]).ravel()
+    per_field, total = orc.split_entropy(w, [8, 8])
+    assert per_field == pytest.approx([math.log2(3), math.log2(5)], abs=1e-12)
+    assert total == pytest.approx(orc.split_entropy(w, [16])[1], abs=1e-12)
+
+
+def test_split_field_order_is_most_significant_first():
+    w = np.array([0x8000, 0x7C00, 0x03E0, 0x001F], dtype=np.uint16)      # one field of {1,5,5,5} all ones, in turn
+    f = orc.split_fields(w, [1, 5, 5, 5])
+    assert [list(map(int, x)) for x in f] == [[1, 0, 0, 0], [0, 31, 0, 0], [0, 0, 31, 0], [0, 0, 0, 31]]
+    with pytest.raises(ValueError):
+        orc.split_fields(w, [8, 7])
+
+
+def test_refining_a_split_never_lowers_its_total():
+    # entropy is subadditive: cutting a field in two can only raise the sum, and no split beats the whole word
+    w = wl.gaussian_weights(256, 4096, 0.02, 5, "fp16_from_bf16")
+    t16 = orc.split_entropy(w, [16])[1]
+    t88 = orc.split_entropy(w, [8, 8])[1]
+    t4444 = orc.split_entropy(w, [4, 4, 4, 4])[1]
+    t1555 = orc.split_entropy(w, [1, 5, 5, 5])[1]
+    t1x16 = orc.split_entropy(w, [1] * 16)[1]
+    assert t16 <= t88 + 1e-9 <= t4444 + 2e-9 <= t1x16 + 3e-9 and t16 <= t1555 + 1e-9 <= t1x16 + 2e-9
+    # and the field histogram of {1,5,5,5} is the one the codebook builder counts
+    counts = orc.histogram(w, orc.FP16)
+    h = orc.split_histograms(w, [1, 5, 5, 5])
+    for k in range(3):
+        assert np.array_equal(h[k + 1], counts[k][:32])
+    # a Huffman code of a field spends between H and H + 1 bits per symbol
+    for k in range(3):
+        lens = orc.huffman_lengths(counts[k][:32])
+        avg = orc.code_cost(counts[k][:32], lens) / w.size
+        H = orc.shannon_entropy(h[k + 1])
+        assert H - 1e-9 <= avg < H + 1
+
+
+def test_synthetic_fp16_weights_land_on_the_papers_entropy_table():
+    # Real checkpoints are unavailable: a soft pin of the synthetic stand-in against the printed rows.
+    g = read_golden("entropy_table_section3_1.txt")
+    w = wl.gaussian_weights(1024, 4096, 0.02, 11, "fp16_from_bf16")
+    for name, widths, tol in (("16", [16], 0.15), ("8_8", [8, 8], 0.15), ("1_5_5_5", [1, 5, 5, 5], 0.15), ("4_4_4_4", [4, 4, 4, 4], 0.35)):
+        per_field, total = orc.split_entropy(w, widths)
+        want = [float(x) for x in g["split_" + name]]
+        assert np.abs(np.array(per_field) - np.array(want)).max() < tol, (name, per_field)
+        if name != "4_4_4_4":
+            assert abs(total - float(g["total_" + name][0])) < tol
+    # the ordering the section argues from: 16 < 8-8 < 1-5-5-5 < 4-4-4-4
+    tot = [orc.split_entropy(w, s)[1] for s in ([16], [8, 8], [1, 5, 5, 5], [4, 4, 4, 4])]
+    assert tot == sorted(tot)
