@@ -252,6 +252,8 @@ def main():
                     help="sweep through this many decoder layers per step (each layer has its own copy of the blobs in HBM): "
                          "the per-token pass over a whole model, e.g. --workload 8b_layer --layers 32")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--explore-splits", action="store_true",
+                    help="also count and report the entropy of other bit-field splits of the workload's largest matrix (Section 3.1 table)")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
@@ -471,6 +473,33 @@ def main():
         except Exception as ex:   # the comparison point must never take the benchmark down
             print(f"[bench] dense comparison skipped: {ex}", file=sys.stderr)
 
+    # ---- the entropy table of Section 3.1 on the workload's largest matrix: device counting pass + host entropies
+    explorer = None
+    if rank == 0 and args.explore_splits:
+        table, std, seed, _ = WORKLOADS[args.workload]
+        i_big = max(range(len(table)), key=lambda i: table[i][1] * table[i][2])
+        name, rows, cols = table[i_big]
+        w_dev = torch.from_numpy(wl.gaussian_weights(rows, cols, std, seed + i_big, args.dtype).view(np.int16)).to(dev)
+        splits = [[16], [8, 8], [1, 5, 5, 5], [4, 4, 4, 4]] if fp16 else [[16], [8, 8], [1, 8, 7], [1, 4, 4, 7]]
+        explorer = {"matrix": name, "weights": rows * cols, "rows": []}
+        for widths in splits:
+            counts = torch.zeros(hl.split_counts_size(widths), dtype=torch.int64, device=dev)
+            for _ in range(3):
+                hl.split_histogram(w_dev, rows * cols, widths, counts, stream)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record(stream)
+            for _ in range(20):
+                hl.split_histogram(w_dev, rows * cols, widths, counts, stream)
+            b.record(stream)
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / 20
+            ent, huf = hl.split_entropy(counts.cpu().numpy().view(np.uint64), widths)
+            explorer["rows"].append({"split": "-".join(map(str, widths)), "entropy_bits": [round(float(x), 4) for x in ent],
+                                     "total_bits_per_param": round(float(ent.sum()), 4), "huffman_bits_per_param": round(float(huf.sum()), 4),
+                                     "ms": ms, "GBs_read": 2 * rows * cols * (2 if widths == [16] else 1) / (ms * 1e-3) / 1e9})
+        del w_dev
+
     # ---- the CPU oracle on a bounded sample of the same workload (rank 0, single GPU run only)
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -535,6 +564,7 @@ def main():
             "note": "huffllm_decode of every matrix of the step, one launch each, into a device buffer"},
         "gpu_launches": len(groups) * args.steps,
         "clocks": clocks,
+        "split_explorer": explorer,
         "dense_bf16_gemv": {"own_kernel_ms_per_step": plain_ms, "cublas_mv_ms_per_step": cublas_ms,
                             "own_kernel_GBs": None if not plain_ms else unc_bytes / (plain_ms * 1e-3) / 1e9,
                             "speedup_vs_own_dense": None if not plain_ms else plain_ms / ms_step},

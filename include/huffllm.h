@@ -297,6 +297,31 @@ huffllm_status huffllm_decode_gemm_static(const huffllm_desc *desc, const void *
 huffllm_status huffllm_plain_gemv(const uint16_t *w_dev, uint64_t rows, uint64_t cols, const uint16_t *x_dev,
                                   float *y_dev, huffllm_stream stream);
 
+/*
+ * Bit-field split explorer (Section 3.1, entropy table): what would it cost, in bits per parameter, to cut the
+ * 16-bit weights into fields some other way and code each field on its own?
+ *
+ * A split is a list of field widths from the most significant bit down: {1,5,5,5} = sign, exponent, upper and lower
+ * mantissa half of an FP16 number; {8,8}; {4,4,4,4}; {16} (the whole word as one symbol).  1 <= n_fields <=
+ * HUFFLLM_MAX_FIELDS, every width 1..16, the widths add up to 16.
+ *
+ * huffllm_split_counts_size: number of counters of a split = sum over the fields of 2^width.
+ * huffllm_split_histogram: one streaming pass (two for a 16-bit field) over n_weights 16-bit words in DEVICE memory
+ *   (16-byte aligned) that counts, per field, how often each value occurs.  counts_dev (device, 8-byte aligned,
+ *   huffllm_split_counts_size entries) is overwritten: field 0's 2^width counters first, then field 1's, ...
+ *   Asynchronous on `stream`; no allocation; at most 2^38 weights per call.
+ * huffllm_split_entropy (host only): from such counters (HOST memory) the Shannon entropy of each field in bits per
+ *   parameter (entropy_bits[n_fields]); their sum is the split's "Total Bits/Param" of the table.  If huffman_bits
+ *   is not NULL it receives, per field, the average codeword length of an unrestricted Huffman code for the counts
+ *   (a field with a single value in use costs 1 bit, as in the blob format).
+ */
+#define HUFFLLM_MAX_FIELDS 16
+huffllm_status huffllm_split_counts_size(const uint8_t *widths, uint32_t n_fields, size_t *n_counts);
+huffllm_status huffllm_split_histogram(const uint16_t *w_dev, uint64_t n_weights, const uint8_t *widths, uint32_t n_fields,
+                                       uint64_t *counts_dev, huffllm_stream stream);
+huffllm_status huffllm_split_entropy(const uint64_t *counts_host, const uint8_t *widths, uint32_t n_fields,
+                                     double *entropy_bits, double *huffman_bits);
+
 /* Message of the last failing call on this thread ("" if none). */
 const char *huffllm_last_error(void);
 

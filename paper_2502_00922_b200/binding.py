@@ -59,6 +59,9 @@ _SIGNATURES = {
                                  C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemm_static": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p],
     "huffllm_plain_gemv": [C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p],
+    "huffllm_split_counts_size": [C.c_void_p, C.c_uint32, C.POINTER(C.c_size_t)],
+    "huffllm_split_histogram": [C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p],
+    "huffllm_split_entropy": [C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p],
     "huffllm_last_error": [],
 }
 
@@ -281,3 +284,32 @@ def decode_gemm_static(desc: Desc, blob_dev, x_dev, batch: int, y_dev, err_flag_
 
 def plain_gemv(w_dev, rows: int, cols: int, x_dev, y_dev, stream=None):
     _check(lib().huffllm_plain_gemv(_ptr(w_dev), rows, cols, _ptr(x_dev), _ptr(y_dev), _stream(stream)))
+
+
+def _widths(widths) -> np.ndarray:
+    return np.ascontiguousarray(list(widths), dtype=np.uint8)
+
+
+def split_counts_size(widths) -> int:
+    """huffllm_split_counts_size: counters of a split (sum of 2^width over its fields)."""
+    wd, n = _widths(widths), C.c_size_t(0)
+    _check(lib().huffllm_split_counts_size(wd.ctypes.data, wd.size, C.byref(n)))
+    return n.value
+
+
+def split_histogram(w_dev, n_weights: int, widths, counts_dev, stream=None):
+    """huffllm_split_histogram: per-field value counts of 16-bit words in device memory (counts_dev: uint64, device)."""
+    wd = _widths(widths)
+    _check(lib().huffllm_split_histogram(_ptr(w_dev), n_weights, wd.ctypes.data, wd.size, _ptr(counts_dev), _stream(stream)))
+
+
+def split_entropy(counts_host: np.ndarray, widths, huffman: bool = True):
+    """huffllm_split_entropy: (entropy per field, Huffman bits per field or None) from host counters."""
+    wd = _widths(widths)
+    counts = np.ascontiguousarray(counts_host, dtype=np.uint64)
+    if counts.size != sum(1 << int(x) for x in wd):
+        raise ValueError("counter array does not match the split")
+    ent = np.zeros(wd.size, dtype=np.float64)
+    huf = np.zeros(wd.size, dtype=np.float64) if huffman else None
+    _check(lib().huffllm_split_entropy(counts.ctypes.data, wd.ctypes.data, wd.size, ent.ctypes.data, _ptr(huf)))
+    return ent, huf
