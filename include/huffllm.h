@@ -175,6 +175,26 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w_host
                               uint32_t chunk_elems, void *blob_host, size_t blob_cap, huffllm_desc *desc);
 
 /*
+ * The same steps for weights that already sit in DEVICE memory (a model being loaded): count on the device, build the
+ * codebook from the counts, encode on the device.  The blob is, byte for byte, the one huffllm_encode writes.
+ *
+ * huffllm_build_codebook_from_counts: counts (host) = BF16: the 256 counters of the exponent byte, i.e. field 1 of
+ *   huffllm_split_histogram with widths {1,8,7}; FP16: the 96 counters of exponent, upper and lower mantissa half,
+ *   i.e. fields 1..3 of widths {1,5,5,5}.  Same result as huffllm_build_codebook_split on the tensor itself.
+ * huffllm_encode_device: w_dev (device, row-major; the fast path wants 16-byte alignment and cols % 8 == 0, anything
+ *   else works too), blob_dev and scratch_dev (device, 256-byte aligned; capacities as for huffllm_encode /
+ *   huffllm_encode_device_scratch_bytes).  Launches on `stream` and WAITS for it (the descriptor depends on the
+ *   payload size and checksum, which only the device knows): this is an offline call, not part of the decode path.
+ *   Errors as huffllm_encode; on error the blob's content is unspecified.
+ */
+huffllm_status huffllm_build_codebook_from_counts(const uint64_t *counts_host, huffllm_dtype dtype, huffllm_split split,
+                                                  uint32_t max_code_len, huffllm_codebook **out);
+huffllm_status huffllm_encode_device_scratch_bytes(uint64_t rows, uint64_t cols, uint32_t chunk_elems, size_t *bytes);
+huffllm_status huffllm_encode_device(const huffllm_codebook *cb, const uint16_t *w_dev, uint64_t rows, uint64_t cols,
+                                     uint32_t chunk_elems, void *blob_dev, size_t blob_cap, void *scratch_dev,
+                                     size_t scratch_bytes, huffllm_desc *desc, huffllm_stream stream);
+
+/*
  * Check a blob held in host memory before it is uploaded: header fields and geometry, section
  * bounds, Kraft sums of the stored code lengths, the LUT against the codebook, a monotone record
  * index, record sizes, and a walk over every lane's bits (each lane must hold exactly its number

@@ -59,6 +59,10 @@ _SIGNATURES = {
                                  C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemm_static": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p],
     "huffllm_plain_gemv": [C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p],
+    "huffllm_build_codebook_from_counts": [C.c_void_p, C.c_int, C.c_int, C.c_uint32, C.POINTER(C.c_void_p)],
+    "huffllm_encode_device_scratch_bytes": [C.c_uint64, C.c_uint64, C.c_uint32, C.POINTER(C.c_size_t)],
+    "huffllm_encode_device": [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t,
+                              C.POINTER(Desc), C.c_void_p],
     "huffllm_split_counts_size": [C.c_void_p, C.c_uint32, C.POINTER(C.c_size_t)],
     "huffllm_split_histogram": [C.c_void_p, C.c_uint64, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p],
     "huffllm_split_entropy": [C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p],
@@ -313,3 +317,28 @@ def split_entropy(counts_host: np.ndarray, widths, huffman: bool = True):
     huf = np.zeros(wd.size, dtype=np.float64) if huffman else None
     _check(lib().huffllm_split_entropy(counts.ctypes.data, wd.ctypes.data, wd.size, ent.ctypes.data, _ptr(huf)))
     return ent, huf
+
+
+def build_codebook_from_counts(counts_host: np.ndarray, dtype: int = BF16, max_code_len: int = 0, split: int = SPLIT_PAPER) -> Codebook:
+    """huffllm_build_codebook_from_counts: BF16: 256 exponent-byte counters; FP16: 96 counters (exponent, upper, lower mantissa half)."""
+    counts = np.ascontiguousarray(counts_host, dtype=np.uint64)
+    if counts.size != (96 if dtype == FP16 else 256):
+        raise ValueError("counter array does not match the dtype")
+    h = C.c_void_p()
+    _check(lib().huffllm_build_codebook_from_counts(counts.ctypes.data, dtype, split, max_code_len, C.byref(h)))
+    return Codebook(h, dtype)
+
+
+def encode_device_scratch_bytes(rows: int, cols: int, chunk_elems: int = 4096) -> int:
+    n = C.c_size_t(0)
+    _check(lib().huffllm_encode_device_scratch_bytes(rows, cols, chunk_elems, C.byref(n)))
+    return n.value
+
+
+def encode_device(cb: Codebook, w_dev, rows: int, cols: int, chunk_elems, blob_dev, blob_cap: int, scratch_dev, scratch_bytes: int,
+                  stream=None) -> Desc:
+    """huffllm_encode_device: encode weights resident on the device into blob_dev; returns the descriptor."""
+    desc = Desc()
+    _check(lib().huffllm_encode_device(cb._h, _ptr(w_dev), rows, cols, chunk_elems, _ptr(blob_dev), blob_cap, _ptr(scratch_dev),
+                                       scratch_bytes, C.byref(desc), _stream(stream)))
+    return desc

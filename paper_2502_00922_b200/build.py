@@ -8,7 +8,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 INCLUDE = os.path.join(os.path.dirname(PKG), "include")
 SO = os.path.join(PKG, "libhuffllm.so")
-SOURCES = ["host_codec.cpp", "api.cu", "kernels.cu", "kernels_tc.cu", "split_explorer.cu"]
+SOURCES = ["host_codec.cpp", "api.cu", "kernels.cu", "kernels_tc.cu", "split_explorer.cu", "encode_device.cu"]
 
 
 def needs_build() -> bool:

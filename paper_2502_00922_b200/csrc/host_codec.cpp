@@ -245,11 +245,13 @@ extern "C" {
 
 const char *huffllm_last_error(void) { return g_err; }
 
-huffllm_status huffllm_build_codebook(const uint16_t *w, uint64_t rows, uint64_t cols, huffllm_dtype dtype,
-                                      uint32_t max_code_len, huffllm_codebook **out) {
-    clear_error();
-    if (!w || !out || rows == 0 || cols == 0) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer or empty tensor");
+// The codebook of a tensor from its symbol counts.  FP16: counts3 = the 3 x 32 counters of exponent, upper and lower
+// mantissa half.  BF16: counts_e = the 256 counters of the exponent byte (both BF16 splits start from them).
+static huffllm_status codebook_from_counts(huffllm_dtype dtype, huffllm_split split, uint32_t max_code_len, const uint64_t *counts3,
+                                           const uint64_t *counts_e, huffllm_codebook **out) {
     if (dtype != HUFFLLM_BF16 && dtype != HUFFLLM_FP16) return fail(HUFFLLM_ERR_INVALID_ARG, "bad dtype");
+    if (split != HUFFLLM_SPLIT_PAPER && split != HUFFLLM_SPLIT_WHOLE_EXPONENT) return fail(HUFFLLM_ERR_INVALID_ARG, "bad split");
+    if (split == HUFFLLM_SPLIT_WHOLE_EXPONENT && dtype != HUFFLLM_BF16) return fail(HUFFLLM_ERR_UNSUPPORTED, "the whole-exponent split is for bf16");
     uint32_t budget = max_code_len ? max_code_len : kDefaultBudget;
     if (budget < kMinBudget || budget > kMaxBudget)
         return fail(HUFFLLM_ERR_UNSUPPORTED, "max_code_len must be 0 or in [%u, %u]", kMinBudget, kMaxBudget);
@@ -258,6 +260,7 @@ huffllm_status huffllm_build_codebook(const uint16_t *w, uint64_t rows, uint64_t
     cb->dtype = dtype;
     cb->budget = budget;
     memset(cb->counts, 0, sizeof(cb->counts));
+    memset(cb->counts_e, 0, sizeof(cb->counts_e));
     memset(cb->len, 0, sizeof(cb->len));
     memset(cb->code, 0, sizeof(cb->code));
     memset(cb->caps, 0, sizeof(cb->caps));
@@ -265,14 +268,8 @@ huffllm_status huffllm_build_codebook(const uint16_t *w, uint64_t rows, uint64_t
     if (dtype == HUFFLLM_FP16) {
         // {1,5,5,5}: exponent, upper and lower mantissa half, each with its own code limited to `budget`
         cb->n_fields = 3;
-        const uint64_t n = rows * cols;
-        for (uint64_t i = 0; i < n; ++i) {
-            uint16_t v = w[i];
-            cb->counts[0][(v >> 10) & 31]++;
-            cb->counts[1][(v >> 5) & 31]++;
-            cb->counts[2][v & 31]++;
-        }
         for (int k = 0; k < 3; ++k) {
+            memcpy(cb->counts[k], counts3 + 32 * k, 32 * sizeof(uint64_t));
             if (!limited_lengths(cb->counts[k], 32, (int)budget, cb->len[k])) {
                 delete cb;
                 return fail(HUFFLLM_ERR_INVALID_ARG, "no code fits max_code_len");
@@ -284,9 +281,21 @@ huffllm_status huffllm_build_codebook(const uint16_t *w, uint64_t rows, uint64_t
         *out = cb;
         return HUFFLLM_OK;
     }
+    memcpy(cb->counts_e, counts_e, sizeof(cb->counts_e));
+    if (split == HUFFLLM_SPLIT_WHOLE_EXPONENT) {
+        cb->n_fields = 1;
+        if (!limited_lengths(cb->counts_e, 256, (int)budget, cb->len_e)) {
+            delete cb;
+            return fail(HUFFLLM_ERR_INVALID_ARG, "no code fits max_code_len");
+        }
+        cb->caps[0] = (uint8_t)budget;
+        canonical_codes(cb->len_e, 256, cb->code_e);
+        finish_codebook(cb);
+        *out = cb;
+        return HUFFLLM_OK;
+    }
     // histogram of the exponent byte, folded into the two nibble fields
     cb->n_fields = 2;
-    exponent_histogram(w, rows * cols, cb->counts_e);
     for (int e = 0; e < 256; ++e) {
         cb->counts[0][e >> 4] += cb->counts_e[e];
         cb->counts[1][e & 15] += cb->counts_e[e];
@@ -321,33 +330,37 @@ huffllm_status huffllm_build_codebook(const uint16_t *w, uint64_t rows, uint64_t
 
 huffllm_status huffllm_build_codebook_split(const uint16_t *w, uint64_t rows, uint64_t cols, huffllm_dtype dtype,
                                             huffllm_split split, uint32_t max_code_len, huffllm_codebook **out) {
-    if (split == HUFFLLM_SPLIT_PAPER) return huffllm_build_codebook(w, rows, cols, dtype, max_code_len, out);
     clear_error();
-    if (split != HUFFLLM_SPLIT_WHOLE_EXPONENT) return fail(HUFFLLM_ERR_INVALID_ARG, "bad split");
     if (!w || !out || rows == 0 || cols == 0) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer or empty tensor");
-    if (dtype != HUFFLLM_BF16) return fail(HUFFLLM_ERR_UNSUPPORTED, "the whole-exponent split is for bf16");
-    uint32_t budget = max_code_len ? max_code_len : kDefaultBudget;
-    if (budget < kMinBudget || budget > kMaxBudget)
-        return fail(HUFFLLM_ERR_UNSUPPORTED, "max_code_len must be 0 or in [%u, %u]", kMinBudget, kMaxBudget);
-    huffllm_codebook *cb = new (std::nothrow) huffllm_codebook();
-    if (!cb) return fail(HUFFLLM_ERR_NOMEM, "out of host memory");
-    cb->dtype = dtype;
-    cb->budget = budget;
-    cb->n_fields = 1;
-    memset(cb->counts, 0, sizeof(cb->counts));
-    memset(cb->len, 0, sizeof(cb->len));
-    memset(cb->code, 0, sizeof(cb->code));
-    memset(cb->caps, 0, sizeof(cb->caps));
-    exponent_histogram(w, rows * cols, cb->counts_e);
-    if (!limited_lengths(cb->counts_e, 256, (int)budget, cb->len_e)) {
-        delete cb;
-        return fail(HUFFLLM_ERR_INVALID_ARG, "no code fits max_code_len");
+    if (dtype == HUFFLLM_FP16) {
+        uint64_t counts3[3 * 32] = {};
+        const uint64_t n = rows * cols;
+        for (uint64_t i = 0; i < n; ++i) {
+            uint16_t v = w[i];
+            counts3[(v >> 10) & 31]++;
+            counts3[32 + ((v >> 5) & 31)]++;
+            counts3[64 + (v & 31)]++;
+        }
+        return codebook_from_counts(dtype, split, max_code_len, counts3, nullptr, out);
     }
-    cb->caps[0] = (uint8_t)budget;
-    canonical_codes(cb->len_e, 256, cb->code_e);
-    finish_codebook(cb);
-    *out = cb;
-    return HUFFLLM_OK;
+    uint64_t counts_e[256];
+    exponent_histogram(w, rows * cols, counts_e);
+    return codebook_from_counts(dtype, split, max_code_len, nullptr, counts_e, out);
+}
+
+huffllm_status huffllm_build_codebook(const uint16_t *w, uint64_t rows, uint64_t cols, huffllm_dtype dtype,
+                                      uint32_t max_code_len, huffllm_codebook **out) {
+    return huffllm_build_codebook_split(w, rows, cols, dtype, HUFFLLM_SPLIT_PAPER, max_code_len, out);
+}
+
+huffllm_status huffllm_build_codebook_from_counts(const uint64_t *counts, huffllm_dtype dtype, huffllm_split split,
+                                                  uint32_t max_code_len, huffllm_codebook **out) {
+    clear_error();
+    if (!counts || !out) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
+    uint64_t total = 0;
+    for (int i = 0; i < (dtype == HUFFLLM_FP16 ? 32 : 256); ++i) total += counts[i];
+    if (total == 0) return fail(HUFFLLM_ERR_INVALID_ARG, "empty tensor");
+    return codebook_from_counts(dtype, split, max_code_len, counts, counts, out);
 }
 
 huffllm_status huffllm_codebook_get_exponent(const huffllm_codebook *cb, uint64_t counts[256], uint8_t lengths[256],
@@ -433,6 +446,69 @@ void parallel_chunks(uint64_t n, F f) {
 
 }  // namespace
 
+namespace huffllm {
+
+// Everything of a blob's descriptor that does not depend on the payload.
+void fill_desc_fixed(const huffllm_codebook *cb, uint64_t rows, uint64_t cols, uint32_t chunk_elems, uint32_t Kc, uint32_t RG,
+                     uint32_t KC, huffllm_desc *out) {
+    huffllm_desc d;
+    memset(&d, 0, sizeof(d));
+    memcpy(d.magic, "HFLM", 4);
+    d.version = 1;
+    d.dtype = cb->dtype;
+    d.chunk_elems = chunk_elems;
+    d.rows = rows;
+    d.cols = cols;
+    d.tile_rows = kTileRows;
+    d.chunk_cols = Kc;
+    d.row_groups = RG;
+    d.col_chunks = KC;
+    d.n_chunks = (uint64_t)RG * KC;
+    d.lut_bits = cb->budget;
+    d.lag_bits = lag_bits_for(cb->dtype);
+    d.n_fields = cb->n_fields;
+    memcpy(d.caps, cb->caps, 4);
+    d.pad_word = cb->pad_word;
+    d.off_codebook = 256;
+    d.off_lut = 512;
+    d.off_index = d.off_lut + align_up((cb->dtype == HUFFLLM_FP16 ? 3 : 1) * (4ull << cb->budget), 256);
+    d.off_payload = d.off_index + align_up(4 * (d.n_chunks + 1), 256);
+    d.raw_bits = (cb->dtype == HUFFLLM_FP16 ? 1 : 8) * rows * cols;
+    *out = d;
+}
+
+// Header, code lengths and decode table: bytes [0, off_index) of the blob (the caller has zeroed them).
+void write_fixed_sections(const huffllm_codebook *cb, const huffllm_desc &d, uint8_t *base) {
+    memcpy(base, &d, sizeof(d));
+    if (cb->n_fields >= 2) {
+        for (int k = 0; k < 3; ++k) memcpy(base + d.off_codebook + 32 * k, cb->len[k], 32);
+    } else {
+        memcpy(base + d.off_codebook, cb->len_e, 256);
+    }
+    memcpy(base + d.off_lut, cb->lut.data(), cb->lut.size() * sizeof(uint32_t));
+}
+
+// The encoder's view of a codebook: per symbol the code length (0 = no codeword) and the stream bits, first bit in
+// bit 0.  BF16: indexed by the exponent byte.  FP16: field k's symbol s at index 32 k + s.
+void encoder_tables(const huffllm_codebook *cb, uint8_t len[256], uint32_t bits[256]) {
+    memset(len, 0, 256);
+    memset(bits, 0, 256 * sizeof(uint32_t));
+    if (cb->dtype == HUFFLLM_FP16) {
+        for (int k = 0; k < 3; ++k)
+            for (int s = 0; s < 32; ++s) {
+                len[32 * k + s] = cb->len[k][s];
+                bits[32 * k + s] = cb->bits5[k][s];
+            }
+    } else {
+        memcpy(len, cb->len8, 256);
+        memcpy(bits, cb->bits8, 256 * sizeof(uint32_t));
+    }
+}
+
+uint32_t codebook_dtype(const huffllm_codebook *cb) { return cb->dtype; }
+
+}  // namespace huffllm
+
 extern "C" {
 
 huffllm_status huffllm_encode_bound(uint64_t rows, uint64_t cols, huffllm_dtype dtype, uint32_t chunk_elems,
@@ -463,28 +539,8 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
     const uint64_t n_chunks = (uint64_t)g.RG * g.KC;
 
     huffllm_desc d;
-    memset(&d, 0, sizeof(d));
-    memcpy(d.magic, "HFLM", 4);
-    d.version = 1;
-    d.dtype = cb->dtype;
-    d.chunk_elems = chunk_elems;
-    d.rows = rows;
-    d.cols = cols;
-    d.tile_rows = kTileRows;
-    d.chunk_cols = g.Kc;
-    d.row_groups = g.RG;
-    d.col_chunks = g.KC;
-    d.n_chunks = n_chunks;
-    d.lut_bits = cb->budget;
-    d.lag_bits = lag_bits_for(cb->dtype);
-    d.n_fields = cb->n_fields;
-    memcpy(d.caps, cb->caps, 4);
-    d.pad_word = cb->pad_word;
-    d.off_codebook = 256;
-    d.off_lut = 512;
+    fill_desc_fixed(cb, rows, cols, chunk_elems, g.Kc, g.RG, g.KC, &d);
     const bool fp16 = cb->dtype == HUFFLLM_FP16;
-    d.off_index = d.off_lut + align_up((fp16 ? 3 : 1) * (4ull << cb->budget), 256);
-    d.off_payload = d.off_index + align_up(4 * (n_chunks + 1), 256);
     if (blob_cap < d.off_payload) return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "blob capacity below the fixed sections");
 
     // pass 1: words per sequence (W) of every chunk, from the code lengths alone
@@ -540,13 +596,7 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
                     (unsigned long long)blob_cap);
 
     memset(base, 0, d.off_payload);
-    memcpy(base, &d, sizeof(d));
-    if (cb->n_fields >= 2) {
-        for (int k = 0; k < 3; ++k) memcpy(base + d.off_codebook + 32 * k, cb->len[k], 32);
-    } else {
-        memcpy(base + d.off_codebook, cb->len_e, 256);
-    }
-    memcpy(base + d.off_lut, cb->lut.data(), cb->lut.size() * sizeof(uint32_t));
+    write_fixed_sections(cb, d, base);
     uint32_t *index = (uint32_t *)(base + d.off_index);
     for (uint64_t c = 0; c <= n_chunks; ++c) index[c] = (uint32_t)rec[c];
 

@@ -37,6 +37,13 @@ inline uint32_t raw_part_bytes(uint32_t dtype, uint32_t nkb) {
 constexpr uint32_t kRawMantByte[4] = {0, 2, 1, 3};
 constexpr uint32_t kRawSignByte[4] = {1, 3, 2, 0};
 
+// Pieces of the host encoder that the device encoder shares (defined with the codebook, in the host codec).
+void fill_desc_fixed(const huffllm_codebook *cb, uint64_t rows, uint64_t cols, uint32_t chunk_elems, uint32_t Kc, uint32_t RG,
+                     uint32_t KC, huffllm_desc *out);
+void write_fixed_sections(const huffllm_codebook *cb, const huffllm_desc &d, uint8_t *base);
+void encoder_tables(const huffllm_codebook *cb, uint8_t len[256], uint32_t bits[256]);
+uint32_t codebook_dtype(const huffllm_codebook *cb);
+
 inline uint32_t blocks_in_chunk(const huffllm_desc &d, uint32_t kc) {
     uint64_t left = d.cols - (uint64_t)kc * d.chunk_cols;
     uint64_t c = left < d.chunk_cols ? left : d.chunk_cols;
