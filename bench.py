@@ -498,7 +498,38 @@ def main():
             explorer["rows"].append({"split": "-".join(map(str, widths)), "entropy_bits": [round(float(x), 4) for x in ent],
                                      "total_bits_per_param": round(float(ent.sum()), 4), "huffman_bits_per_param": round(float(huf.sum()), 4),
                                      "ms": ms, "GBs_read": 2 * rows * cols * (2 if widths == [16] else 1) / (ms * 1e-3) / 1e9})
-        del w_dev
+        # compression of that matrix where it sits: counts (above), codebook from the counts, encoder on the device
+        hd = hl.FP16 if fp16 else hl.BF16
+        widths = [1, 5, 5, 5] if fp16 else [1, 8, 7]
+        counts = torch.zeros(hl.split_counts_size(widths), dtype=torch.int64, device=dev)
+        cap = hl.encode_bound(rows, cols, hd, args.chunk_elems)
+        blob_dev = torch.zeros(cap, dtype=torch.uint8, device=dev)
+        n_scr = hl.encode_device_scratch_bytes(rows, cols, args.chunk_elems)
+        scr = torch.zeros(n_scr, dtype=torch.uint8, device=dev)
+        def compress():
+            hl.split_histogram(w_dev, rows * cols, widths, counts, stream)
+            c = counts.cpu().numpy().view(np.uint64)
+            cb = hl.build_codebook_from_counts(c[2:98] if fp16 else c[2:258], hd, args.max_code_len, split)
+            d = hl.encode_device(cb, w_dev, rows, cols, args.chunk_elems, blob_dev, cap, scr, n_scr, stream)
+            cb.free()
+            return d
+        compress()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        for _ in range(5):
+            d_enc = compress()
+        torch.cuda.synchronize()
+        dev_ms = (time.perf_counter() - t0) * 1e3 / 5
+        w_host = w_dev.cpu().numpy().view(np.uint16)
+        t0 = time.perf_counter()
+        cb = hl.build_codebook(w_host, hd, args.max_code_len, split)
+        blob_h, _ = hl.encode(cb, w_host, args.chunk_elems)
+        host_ms = (time.perf_counter() - t0) * 1e3
+        cb.free()
+        explorer["compress"] = {"device_ms": dev_ms, "host_ms": host_ms, "same_blob": bool(np.array_equal(blob_dev[:d_enc.blob_bytes].cpu().numpy(), blob_h)),
+                                "device_GBs_of_weights": 2 * rows * cols / (dev_ms * 1e-3) / 1e9,
+                                "note": "counting pass + codebook from the counts + device encoder, wall clock including its two waits; host: codebook + encoder on the host cores"}
+        del w_dev, blob_dev
 
     # ---- the CPU oracle on a bounded sample of the same workload (rank 0, single GPU run only)
     cpu = None

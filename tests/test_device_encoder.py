@@ -105,6 +105,28 @@ def test_device_encoder_writes_the_host_encoders_blob(hl, rows, cols, ce, kind, 
 
 
 @pytest.mark.gpu
+def test_full_size_matrix_on_the_device_equals_the_host_blob(hl):
+    """A full-size FFN matrix of the benchmark's layer (45 M weights, 11008 chunks)."""
+    import torch
+    rows, cols, ce = 11008, 4096, 4096
+    w = wl.gaussian_weights(rows, cols, 0.02, 1003)
+    w_dev = torch.from_numpy(w.view(np.int16)).cuda()
+    counts = torch.zeros(hl.split_counts_size([1, 8, 7]), dtype=torch.int64, device="cuda")
+    hl.split_histogram(w_dev, rows * cols, [1, 8, 7], counts)
+    cb = hl.build_codebook_from_counts(counts.cpu().numpy().view(np.uint64)[2:258], 0)
+    cap = hl.encode_bound(rows, cols, 0, ce)
+    blob_dev = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+    n_scr = hl.encode_device_scratch_bytes(rows, cols, ce)
+    desc = hl.encode_device(cb, w_dev, rows, cols, ce, blob_dev, cap, torch.zeros(n_scr, dtype=torch.uint8, device="cuda"), n_scr)
+    cb_host = hl.build_codebook(w, 0)
+    want, desc_host = hl.encode(cb_host, w, ce)
+    assert bytes(desc) == bytes(desc_host)
+    assert np.array_equal(blob_dev[:desc.blob_bytes].cpu().numpy(), want)
+    cb.free()
+    cb_host.free()
+
+
+@pytest.mark.gpu
 def test_device_encoded_blob_feeds_the_product_kernel(hl):
     import torch
     rows, cols = 256, 2048
