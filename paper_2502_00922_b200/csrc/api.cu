@@ -155,6 +155,8 @@ huffllm_status finish_args(KernelArgs *k, bool product, const DeviceInfo &dev, u
     for (uint32_t i = 0; i < k->n_mats; ++i) {
         k->m[i].cta_first = first;
         k->m[i].cta_count = cnt[i];
+        k->m[i].cta_chunks = k->m[i].n_chunks / cnt[i];
+        k->m[i].cta_extra = k->m[i].n_chunks % cnt[i];
         first += cnt[i];
     }
     *grid = first;

@@ -254,7 +254,7 @@ __device__ __forceinline__ SmemPlan plan_smem(uint32_t base, const KernelArgs &k
     SmemPlan p;
     const uint32_t lut_bytes = k.lut_align;
     uint32_t a0 = (base + 127u) & ~127u;
-    p.lut = (base + lut_bytes - 1) / lut_bytes * lut_bytes;
+    p.lut = (base + lut_bytes - 1) & ~(lut_bytes - 1);        // lut_align is a power of two
     p.slotA = a0;
     p.nA = p.lut > a0 ? (p.lut - a0) / (2 * k.slot_bytes) : 0;  // a stream that overruns here reads the table: harmless
     p.slotB = p.lut + k.lut_size;

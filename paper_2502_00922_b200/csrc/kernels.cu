@@ -80,13 +80,17 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     {
         const MatArgs &k = A.m[mi];
         const uint32_t G = k.cta_count, J = blockIdx.x - k.cta_first;       // CTAs of this matrix, this CTA's number among them
-        auto cta_cut = [&](uint32_t j) -> uint32_t { return (uint32_t)((uint64_t)k.n_chunks * j / G); };
+        // (the set-up runs in all 32 warps at once and is bound by instruction issue: no 64-bit divisions here)
+        auto cta_cut = [&](uint32_t j) -> uint32_t { return j * k.cta_chunks + min(j, k.cta_extra); };   // first chunk of the matrix's CTA j
         const uint32_t cta_beg = cta_cut(J), cta_end = cta_cut(J + 1);
         const uint32_t KC = k.col_chunks;
+        // the CTA's chunks are dealt to its warps the same way: wq each, the first wr warps one more
+        const uint32_t cta_len = cta_end - cta_beg, wq = cta_len / nw, wr = cta_len - wq * nw;
+        auto warp_beg = [&](uint32_t w) -> uint32_t { return cta_beg + w * wq + min(w, wr); };
         uint32_t c_beg = cta_beg, c_end = cta_beg;
         if (warp < nw) {
-            c_beg = cta_beg + (cta_end - cta_beg) * warp / nw;
-            c_end = cta_beg + (cta_end - cta_beg) * (warp + 1) / nw;
+            c_beg = warp_beg(warp);
+            c_end = warp_beg(warp + 1);
         }
         const uint32_t *index = (const uint32_t *)(k.blob + k.off_index);
         const uint8_t *payload = k.blob + k.off_payload;
@@ -154,13 +158,9 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         // the warp that arrives last adds the pieces in warp order.  If other CTAs hold pieces too, the CTA's
         // sum goes to the scratch buffer and the same game is played across CTAs with a counter in global
         // memory.  Sums are always taken in the same order, and nobody waits for anybody.
-        const uint32_t cta_len = cta_end - cta_beg;
-        auto warp_beg = [&](uint32_t w) -> uint32_t { return cta_beg + cta_len * w / nw; };
         auto cta_of_chunk = [&](uint32_t ch) -> uint32_t {     // which of the matrix's CTAs works on chunk ch
-            uint32_t c = (uint32_t)((uint64_t)ch * G / k.n_chunks);
-            while (c + 1 < G && cta_cut(c + 1) <= ch) ++c;
-            while (c > 0 && cta_cut(c) > ch) --c;
-            return c;
+            const uint32_t big = k.cta_extra * (k.cta_chunks + 1);
+            return ch < big ? ch / (k.cta_chunks + 1) : k.cta_extra + (ch - big) / k.cta_chunks;
         };
         // lanes 0..vals-1 (looping if vals > 32) hold or produce the value of output o = column * 16 + row
         auto finish_cta_sum = [&](int rg, float (&v)[4]) {       // v[i] = value of output o = lane + 32 i

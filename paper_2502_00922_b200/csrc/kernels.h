@@ -15,6 +15,7 @@ struct MatArgs {
     uint32_t payload_units;    // payload size in 128-byte units
     uint32_t n_chunks, chunk_cols, col_chunks;
     uint32_t cta_first, cta_count;   // the CTAs of the launch that work on this matrix (each at least one chunk)
+    uint32_t cta_chunks, cta_extra;  // n_chunks / cta_count and n_chunks % cta_count: the first cta_extra CTAs take one chunk more
     const uint16_t *x;         // [batch][cols]
     float *y;                  // [batch][rows]
     float *ws_partial;         // [cta_count * 2][16 * batch]
