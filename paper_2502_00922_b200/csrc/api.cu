@@ -124,6 +124,7 @@ huffllm_status add_matrix(KernelArgs *k, const huffllm_desc *desc, const void *b
     const uint32_t checks_per_block = fmt ? 8 : (desc->lut_bits == 8 ? 3 : 4);
     uint32_t guard = 256 * (3 + checks_per_block * (desc->chunk_cols / kBlockCols));
     if (slot > k->slot_bytes) k->slot_bytes = slot;
+    k->pair_recip = (uint32_t)(0x100000000ull / (2ull * k->slot_bytes));
     if (guard > k->guard_bytes) k->guard_bytes = guard;
     return HUFFLLM_OK;
 }

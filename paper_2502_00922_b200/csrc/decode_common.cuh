@@ -256,11 +256,18 @@ __device__ __forceinline__ SmemPlan plan_smem(uint32_t base, const KernelArgs &k
     uint32_t a0 = (base + 127u) & ~127u;
     p.lut = (base + lut_bytes - 1) & ~(lut_bytes - 1);        // lut_align is a power of two
     p.slotA = a0;
-    p.nA = p.lut > a0 ? (p.lut - a0) / (2 * k.slot_bytes) : 0;  // a stream that overruns here reads the table: harmless
+    // (divisions by the slot pair's size as a multiplication by its rounded-down reciprocal and one correction: this
+    // runs in every warp of a launch's set-up, which is bound by instruction issue)
+    const uint32_t pair = 2 * k.slot_bytes;
+    auto div_pair = [&](uint32_t x) -> uint32_t {
+        uint32_t q = __umulhi(x, k.pair_recip);
+        return x - q * pair >= pair ? q + 1 : q;
+    };
+    p.nA = p.lut > a0 ? div_pair(p.lut - a0) : 0;  // a stream that overruns here reads the table: harmless
     p.slotB = p.lut + k.lut_size;
     uint32_t end = base + k.dyn_smem_bytes - k.part_bytes;
     uint32_t roomB = end > p.slotB + k.guard_bytes ? end - p.slotB - k.guard_bytes : 0;
-    p.warps = min(max_warps, p.nA + roomB / (2 * k.slot_bytes));
+    p.warps = min(max_warps, p.nA + div_pair(roomB));
     return p;
 }
 

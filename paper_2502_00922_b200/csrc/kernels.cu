@@ -85,7 +85,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         const uint32_t cta_beg = cta_cut(J), cta_end = cta_cut(J + 1);
         const uint32_t KC = k.col_chunks;
         // the CTA's chunks are dealt to its warps the same way: wq each, the first wr warps one more
-        const uint32_t cta_len = cta_end - cta_beg, wq = cta_len / nw, wr = cta_len - wq * nw;
+        const uint32_t cta_len = cta_end - cta_beg, wq = nw == 32 ? cta_len >> 5 : cta_len / nw, wr = cta_len - wq * nw;
         auto warp_beg = [&](uint32_t w) -> uint32_t { return cta_beg + w * wq + min(w, wr); };
         uint32_t c_beg = cta_beg, c_end = cta_beg;
         if (warp < nw) {
@@ -94,6 +94,15 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         }
         const uint32_t *index = (const uint32_t *)(k.blob + k.off_index);
         const uint8_t *payload = k.blob + k.off_payload;
+        // the offsets of the warp's first two records: asked for before anything else of the set-up, whose
+        // instructions then run while the loads are under way
+        const uint32_t rg_first = c_beg / KC, kc_first = c_beg - rg_first * KC;
+        uint32_t idx0 = 0, idx1 = 0, idx2 = 0;
+        if (lane == 0 && c_beg < c_end) {
+            idx0 = __ldg(index + c_beg);
+            idx1 = __ldg(index + c_beg + 1);
+            idx2 = c_beg + 1 < c_end ? __ldg(index + c_beg + 2) : 0u;
+        }
 
         // blocks of 32 columns in column chunk kc: every chunk is full except, possibly, the last one of a row
         const uint32_t nkb_tail = ((uint32_t)k.cols - (KC - 1) * k.chunk_cols + 31u) >> 5;
@@ -114,7 +123,6 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                 mbar_expect_tx(bar, 0);  // completes the phase with nothing to wait for; the chunk is skipped below
             }
         };
-        auto issue = [&](uint32_t c, uint32_t which) { issue_known(c % KC, __ldg(index + c), __ldg(index + c + 1), which); };
 
         // ---- set-up of a segment.  The table loads are started first, then every warp starts its first
         // copies, then the table is written to shared memory: the cold misses on the table, on the record
@@ -133,8 +141,8 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
             }
         }
         if (lane == 0 && c_beg < c_end) {
-            issue(c_beg, 0);
-            if (c_beg + 1 < c_end) issue(c_beg + 1, 1);
+            issue_known(kc_first, idx0, idx1, 0);
+            if (c_beg + 1 < c_end) issue_known(kc_first + 1 == KC ? 0u : kc_first + 1, idx1, idx2, 1);
         }
         {
             uint32_t *lut_s = (uint32_t *)(dyn_smem + (plan.lut - smem_base));
@@ -250,7 +258,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         };
 
         if (c_beg < c_end && !failed) {
-            uint32_t rg = c_beg / KC, kc = c_beg - rg * KC;            // tracked incrementally from here on
+            uint32_t rg = rg_first, kc = kc_first;                    // tracked incrementally from here on
             uint32_t r0 = __ldg(index + c_beg), r1 = __ldg(index + c_beg + 1);
             // raw sign/mantissa bytes travel one block ahead of the decoder, in two register sets used in turn
             uint4 raw_a = make_uint4(0, 0, 0, 0), raw_b = make_uint4(0, 0, 0, 0);

@@ -28,6 +28,7 @@ struct KernelArgs {
     uint32_t fmt;              // 0: BF16 blobs (one table), 1: FP16 blobs (three tables)
     uint32_t lut_align, lut_size;   // shared-memory window of the table(s): a power-of-two alignment above the index bits, and its bytes
     uint32_t slot_bytes;       // shared-memory bytes of one slot: largest max_words * 256
+    uint32_t pair_recip;       // floor(2^32 / (2 * slot_bytes)): umulhi(x, pair_recip) is x / (2 * slot_bytes) or one less
     uint32_t guard_bytes;      // readable bytes kept free behind the last slot
     uint32_t part_bytes;       // bytes at the end of dynamic shared memory for the CTA's partial sums
     uint32_t dyn_smem_bytes;
