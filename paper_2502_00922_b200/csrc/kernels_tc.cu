@@ -108,7 +108,6 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     extern __shared__ __align__(128) uint8_t dyn_smem[];
     __shared__ __align__(8) uint64_t bars[kMaxWarps * 2];   // per warp: its two coded-copy barriers
     __shared__ __align__(8) uint64_t empty_bar[S];          // stage may be refilled (arrived on by tcgen05.commit)
-    __shared__ uint32_t full_cnt[S];                        // warps that have filled the stage
     __shared__ uint32_t s_tmem_base;
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -138,7 +137,6 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     }
     if (tid < S) {
         mbar_init(smem_u32(&empty_bar[tid]), 1);
-        full_cnt[tid] = 0;
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     if (warp == 0) {
@@ -205,12 +203,16 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     const bool x_carrier = warp * 32 + lane < NPAD * 4;
     const uint32_t x_n = (warp * 32 + lane) >> 2, x_kap = lane & 3;
     const uint16_t *x_src = k.x + (uint64_t)x_n * k.cols + (x_kap & 1) * 16 + (x_kap >> 1) * 4;
-    auto load_x = [&](uint4 &v, uint32_t col_block) {        // fetched one block ahead of its use
-        if (x_carrier && x_n < A.batch) {
-            uint2 lo = __ldg((const uint2 *)(x_src + col_block)), hi = __ldg((const uint2 *)(x_src + col_block + 8));
+    const bool x_loads = x_carrier && x_n < A.batch;         // carriers of padding vectors stage zeros
+    auto load_x = [&](uint4 &v, const uint16_t *p) {         // fetched one block ahead of its use
+        if (x_loads) {
+            uint2 lo = __ldg((const uint2 *)p), hi = __ldg((const uint2 *)(p + 8));
             v = make_uint4(lo.x, lo.y, hi.x, hi.y);
         }
     };
+    // addresses that change only with the stage: this warp's rows of the A operand, its piece of the B slice
+    const uint32_t a_dst0 = tmem + a_lane + kACol0 + tile * S * 16;
+    const uint32_t x_dst0 = b_base + (x_n >> 3) * kSbo + x_kap * kLbo + (x_n & 7) * 16;
 
     // One block of the stage protocol.  `a` = this warp's decoded 16 rows x 32 columns (null if the warp has no rows).
     auto stage_block = [&](const uint32_t *a, const uint4 &xv, bool first_of_item) {
@@ -220,35 +222,28 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
         if (a) {
             // lane (g, t): row g's weights 0..3 -> 32-bit columns 2t, 2t+1; weights 4..7 -> columns 8 + 2t, 8 + 2t + 1
             const uint32_t r[8] = {a[0], a[1], a[4], a[5], a[2], a[3], a[6], a[7]};
-            tc_st_16x256b_x2(tmem + a_lane + kACol0 + (tile * S + s) * 16, r);
+            tc_st_16x256b_x2(a_dst0 + s * 16, r);
         }
-        if (x_carrier) {
-            const uint32_t dst = b_base + s * kBStage + (x_n >> 3) * kSbo + x_kap * kLbo + (x_n & 7) * 16;
-            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(dst), "r"(xv.x), "r"(xv.y), "r"(xv.z), "r"(xv.w) : "memory");
-        }
+        if (x_carrier)
+            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(x_dst0 + s * kBStage), "r"(xv.x), "r"(xv.y), "r"(xv.z), "r"(xv.w) : "memory");
         tc_wait_st();
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the B slice must be visible to the tensor core's reads
         tc_fence_before();
-        __syncwarp();
-        uint32_t last = 0;
-        if (lane == 0) {
-            __threadfence_block();
-            last = atomicAdd(&full_cnt[s], 1u) == n_dec - 1 ? 1u : 0u;
-            if (last) {
-                full_cnt[s] = 0;
-                __threadfence_block();
-                tc_fence_after();
-                const uint32_t bst = b_base + s * kBStage;
-                for (uint32_t tl = 0; tl < n_tiles; ++tl) {
+        // every decoder warp's rows and the activations of this block are in place: a hardware barrier, so that a warp
+        // that waits costs no issue slots (the decoders are bound by instruction issue; a polling loop would take
+        // slots from the warps that still decode)
+        asm volatile("bar.sync 1, %0;" ::"r"(n_dec * 32u) : "memory");
+        if (warp == (gb & 7u) && lane == 0) {                   // the first tile's warps take turns in issuing the block's MMAs
+            tc_fence_after();
+            const uint32_t bst = b_base + s * kBStage;
+            for (uint32_t tl = 0; tl < n_tiles; ++tl) {
 #pragma unroll
-                    for (uint32_t j = 0; j < 2; ++j)      // two K = 16 steps per stage
-                        tc_mma_f16_tmem_a(tmem + tl * NPAD, tmem + kACol0 + (tl * S + s) * 16 + j * 8,
-                                          smem_desc_kmajor(bst + j * 2 * kLbo, kLbo, kSbo), kIdesc, (first_of_item && j == 0) ? 0u : 1u);
-                }
-                tc_commit(smem_u32(&empty_bar[s]));
+                for (uint32_t j = 0; j < 2; ++j)      // two K = 16 steps per stage
+                    tc_mma_f16_tmem_a(tmem + tl * NPAD, tmem + kACol0 + (tl * S + s) * 16 + j * 8,
+                                      smem_desc_kmajor(bst + j * 2 * kLbo, kLbo, kSbo), kIdesc, (first_of_item && j == 0) ? 0u : 1u);
             }
+            tc_commit(smem_u32(&empty_bar[s]));
         }
-        __syncwarp();
         ++gb;
     };
 
@@ -261,9 +256,10 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
         const uint32_t gb_item = gb;
         // the item's blocks are consecutive 32-column blocks of the matrix, from col_lo up to col_hi
         const uint32_t col_lo = kc0 * k.chunk_cols, col_hi = min(kc1 * k.chunk_cols, (uint32_t)k.cols);
-        uint32_t col_blk = col_lo;
-        uint4 x_cur = make_uint4(0, 0, 0, 0), x_nxt = make_uint4(0, 0, 0, 0);
-        load_x(x_cur, col_lo);
+        // activations: x_a holds the current block's piece at the top of every chunk; the pointer names the block after it
+        const uint16_t *x_p = x_src + col_lo + 32, *const x_end = x_src + col_hi;
+        uint4 x_a = make_uint4(0, 0, 0, 0), x_b = make_uint4(0, 0, 0, 0);
+        load_x(x_a, x_src + col_lo);
 
         if (active) {
             const uint32_t c_beg = rg * KC + kc0, c_end = rg * KC + kc1;
@@ -288,17 +284,27 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                 LaneStream sa, sb;
                 stream_open(sa, slot0 + which * A.slot_bytes + (lane << 2));
                 stream_open(sb, slot0 + which * A.slot_bytes + 128u + (lane << 2));
-#pragma unroll 1
-                for (uint32_t kb = 0; kb < nkb; ++kb) {
-                    uint4 raw_next = raw_cur;
-                    if (ok && kb + 1 < nkb) raw_next = ldg_stream16(raw_p + (size_t)(kb + 1) * 512u);
-                    if (col_blk + 32 < col_hi) load_x(x_nxt, col_blk + 32);
+                // one block: fetch the next block's raw bytes and activations into the other register set, decode
+                // this one, hand it to the tensor core
+                auto block = [&](const uint4 &raw_c, uint4 &raw_n, const uint4 &x_c, uint4 &x_n2, bool more) {
+                    raw_p += 512;
+                    if (more && ok) raw_n = ldg_stream16(raw_p);
+                    if (x_p < x_end) load_x(x_n2, x_p);
+                    x_p += 32;
                     uint32_t a[8];
-                    decode_block<R>(sa, sb, kIdxMask, lut_lane, raw_cur, a);   // a chunk that is not ok decodes garbage, never out of range
-                    stage_block(a, x_cur, gb == gb_item);
-                    raw_cur = raw_next;
-                    x_cur = x_nxt;
-                    col_blk += 32;
+                    decode_block<R>(sa, sb, kIdxMask, lut_lane, raw_c, a);   // a chunk that is not ok decodes garbage, never out of range
+                    stage_block(a, x_c, gb == gb_item);
+                };
+                uint4 raw_b = make_uint4(0, 0, 0, 0);
+                uint32_t kb = 0;
+#pragma unroll 1
+                for (; kb + 2 <= nkb; kb += 2) {                  // the usual case: pairs of blocks, two register sets in turn
+                    block(raw_cur, raw_b, x_a, x_b, true);
+                    block(raw_b, raw_cur, x_b, x_a, kb + 2 < nkb);
+                }
+                if (kb < nkb) {                                   // odd block count (a ragged last chunk)
+                    block(raw_cur, raw_b, x_a, x_b, false);
+                    x_a = x_b;
                 }
                 __syncwarp();
                 if (lane == 0 && c + 2 < c_end) issue(c + 2, which);
@@ -307,10 +313,11 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
             }
         } else {
             // no rows of the matrix for this warp: it still carries its slice of the activations and its arrivals
-            for (; col_blk < col_hi; col_blk += 32) {
-                if (col_blk + 32 < col_hi) load_x(x_nxt, col_blk + 32);
-                stage_block(nullptr, x_cur, gb == gb_item);
-                x_cur = x_nxt;
+            for (uint32_t col_blk = col_lo; col_blk < col_hi; col_blk += 32) {
+                if (x_p < x_end) load_x(x_b, x_p);
+                x_p += 32;
+                stage_block(nullptr, x_a, gb == gb_item);
+                x_a = x_b;
             }
         }
 
