@@ -84,9 +84,12 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         auto cta_cut = [&](uint32_t j) -> uint32_t { return j * k.cta_chunks + min(j, k.cta_extra); };   // first chunk of the matrix's CTA j
         const uint32_t cta_beg = cta_cut(J), cta_end = cta_cut(J + 1);
         const uint32_t KC = k.col_chunks;
-        // the CTA's chunks are dealt to its warps the same way: wq each, the first wr warps one more
+        // the CTA's chunks are dealt to its warps: wq each, and wr warps in the MIDDLE of the range one more.  The warps
+        // with the extra chunk finish last; in the middle their row groups belong to this CTA alone, so what runs at
+        // the very end of the launch is a reduction in shared memory, not the one across CTAs with its global round trips
         const uint32_t cta_len = cta_end - cta_beg, wq = nw == 32 ? cta_len >> 5 : cta_len / nw, wr = cta_len - wq * nw;
-        auto warp_beg = [&](uint32_t w) -> uint32_t { return cta_beg + w * wq + min(w, wr); };
+        const uint32_t w_mid = (nw - wr) >> 1;
+        auto warp_beg = [&](uint32_t w) -> uint32_t { return cta_beg + w * wq + min(w > w_mid ? w - w_mid : 0u, wr); };
         uint32_t c_beg = cta_beg, c_end = cta_beg;
         if (warp < nw) {
             c_beg = warp_beg(warp);
