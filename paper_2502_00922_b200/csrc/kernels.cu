@@ -79,7 +79,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     while (mi + 1 < A.n_mats && blockIdx.x >= A.m[mi + 1].cta_first) ++mi;
     {
         const MatArgs &k = A.m[mi];
-        const uint32_t G = k.cta_count, J = blockIdx.x - k.cta_first;       // CTAs of this matrix, this CTA's number among them
+        const uint32_t J = blockIdx.x - k.cta_first;                        // this CTA's number among the CTAs of its matrix
         // (the set-up runs in all 32 warps at once and is bound by instruction issue: no 64-bit divisions here)
         auto cta_cut = [&](uint32_t j) -> uint32_t { return j * k.cta_chunks + min(j, k.cta_extra); };   // first chunk of the matrix's CTA j
         const uint32_t cta_beg = cta_cut(J), cta_end = cta_cut(J + 1);
