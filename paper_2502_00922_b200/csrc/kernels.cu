@@ -131,16 +131,18 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         // copies, then the table is written to shared memory: the cold misses on the table, on the record
         // index and on the first records overlap instead of following each other.
         // (FP16: three tables of 256 entries, sixteen copies each: word j holds entry j / 16 of its table)
+        // The table goes to shared memory in 16-byte pieces: four neighbouring copies of one entry per piece.
         constexpr uint32_t kLutWords = FMT ? 3u * 16u * 256u : 32u << LB;
         constexpr uint32_t kLutRep = FMT ? 4u : 5u;            // log2 of the copies per entry
-        constexpr int kLutLoads = (kLutWords + THREADS - 1) / THREADS;
+        constexpr uint32_t kLutVecs = kLutWords / 4;
+        constexpr int kLutLoads = (kLutVecs + THREADS - 1) / THREADS;
         uint32_t lut_v[kLutLoads];
         {
             const uint32_t *lut_g = (const uint32_t *)(k.blob + k.off_lut);
 #pragma unroll
             for (int i = 0; i < kLutLoads; ++i) {
-                uint32_t j = tid + i * THREADS;
-                lut_v[i] = j < kLutWords ? __ldg(lut_g + (j >> kLutRep)) : 0u;
+                uint32_t v = tid + i * THREADS;
+                lut_v[i] = (kLutVecs % THREADS == 0 || v < kLutVecs) ? __ldg(lut_g + (v >> (kLutRep - 2))) : 0u;
             }
         }
         if (lane == 0 && c_beg < c_end) {
@@ -148,11 +150,11 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
             if (c_beg + 1 < c_end) issue_known(kc_first + 1 == KC ? 0u : kc_first + 1, idx1, idx2, 1);
         }
         {
-            uint32_t *lut_s = (uint32_t *)(dyn_smem + (plan.lut - smem_base));
+            uint4 *lut_s = (uint4 *)(dyn_smem + (plan.lut - smem_base));
 #pragma unroll
             for (int i = 0; i < kLutLoads; ++i) {
-                uint32_t j = tid + i * THREADS;
-                if (j < kLutWords) lut_s[j] = lut_v[i];
+                uint32_t v = tid + i * THREADS;
+                if (kLutVecs % THREADS == 0 || v < kLutVecs) lut_s[v] = make_uint4(lut_v[i], lut_v[i], lut_v[i], lut_v[i]);
             }
             if (tid < kMaxWarps) s_arrive[tid] = 0;
         }
