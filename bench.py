@@ -281,8 +281,6 @@ def main():
     if B > 8:
         args.fuse = "none"           # the tensor-core path takes one matrix per launch
     fp16 = args.dtype != "bf16"
-    if fp16 and B > 8:
-        raise SystemExit("--dtype fp16 takes --batch up to 8 here")
     mats = prepare(args.workload, args.chunk_elems, hl, torch, dev, cpu_mats, split, B, args.dtype, args.max_code_len)
     err = torch.zeros(1, dtype=torch.int32, device=dev)
     L = args.layers

@@ -53,9 +53,11 @@ struct TcPlan {
 };
 // Shared memory the tensor-core kernel needs with `tiles` 128-row tiles per CTA.
 uint64_t tc_smem_need(const huffllm_desc *d, uint32_t npad, uint32_t tiles) {
-    const uint32_t checks_per_block = d->lut_bits == 8 ? 3 : 4;
+    const bool fp16 = d->dtype == HUFFLLM_FP16;
+    const uint32_t checks_per_block = fp16 ? 8 : (d->lut_bits == 8 ? 3 : 4);
     uint64_t guard = 256ull * (3 + checks_per_block * (d->chunk_cols / kBlockCols));
-    return (128ull << d->lut_bits) + guard + 4ull * npad * 64 + 4096 + 2ull * 8 * tiles * d->max_words * 256;
+    const uint64_t lut = fp16 ? 49152ull : 128ull << d->lut_bits;
+    return lut + guard + 4ull * npad * 64 + 4096 + 2ull * 8 * tiles * d->max_words * 256;
 }
 TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn_smem) {
     TcPlan p;
@@ -257,7 +259,7 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
     if (st != HUFFLLM_OK) return st;
     if (batch == 0 || batch > 64) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be in [1, 64]");
     if ((st = check_product_args(desc, x, y, workspace, workspace_bytes, batch)) != HUFFLLM_OK) return st;
-    if (batch > kKernelBatch && desc->dtype == HUFFLLM_BF16) {
+    if (batch > kKernelBatch) {
         // tensor-core path: one pass over the compressed weights for the whole batch
         const TcPlan tp = tc_plan(desc, batch, (uint32_t)dev->sms, (uint32_t)dev->smem_optin - kStaticSmem);
         KernelArgs k;

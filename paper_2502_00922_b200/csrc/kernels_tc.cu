@@ -93,9 +93,17 @@ __device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t addr, uint32_t lbo
     return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46);
 }
 
-// LB = table index bits; NPAD = batch rounded up to 16, 32 or 64 (the MMA's N).
-template <int LB, int NPAD>
+// LB = table index bits; NPAD = batch rounded up to 16, 32 or 64 (the MMA's N); FMT = 0: BF16 blobs, 1: FP16 {1,5,5,5} blobs
+// (three tables, sign words as the raw part, f16 operands).
+template <int LB, int NPAD, int FMT>
 __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_constant__ KernelArgs A) {
+    constexpr uint32_t kRawBlock = FMT ? 64u : 512u;          // raw bytes of one block of a record
+    constexpr uint32_t kRawLane = FMT ? 2u : 16u;             // of which one lane's share
+    auto raw_part = [](uint32_t nkb) -> uint32_t { return FMT ? (nkb * 64u + 127u) & ~127u : nkb * 512u; };
+    auto load_raw = [](const uint8_t *p) -> uint4 {
+        if (FMT) return make_uint4(ldg_stream2(p), 0, 0, 0);
+        return ldg_stream16(p);
+    };
     constexpr int R = LB == 8 ? 3 : 2;
     constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
     constexpr int S = kTcStages;
@@ -103,7 +111,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     constexpr uint32_t kLbo = 128, kSbo = 512;              // core matrices: 4 along K side by side, then the next 8 rows
     constexpr uint32_t kACol0 = kTcTiles * NPAD;            // first tensor-memory column of the A stages
     // instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, N = NPAD, M = 128
-    constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NPAD >> 3) << 17) | ((128u >> 4) << 24);
+    constexpr uint32_t kIdesc = (1u << 4) | (FMT ? 0u : (1u << 7) | (1u << 10)) | ((uint32_t)(NPAD >> 3) << 17) | ((128u >> 4) << 24);
 
     extern __shared__ __align__(128) uint8_t dyn_smem[];
     __shared__ __align__(8) uint64_t bars[kMaxWarps * 2];   // per warp: its two coded-copy barriers
@@ -120,7 +128,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
         return;
     }
     const uint32_t b_base = smem_base + A.dyn_smem_bytes - A.part_bytes;   // S stages of B behind everything else
-    uint32_t lut_lane = plan.lut | (lane << 2);
+    uint32_t lut_lane = plan.lut | ((FMT ? lane & 15u : lane) << 2);
     asm volatile("mov.u32 %0, %0;" : "+r"(lut_lane));
     const uint32_t bar0 = smem_u32(&bars[warp * 2]);
     const uint32_t slot0 = slot_addr(plan, warp, 0, A.slot_bytes);
@@ -129,7 +137,9 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     {
         const uint32_t *lut_g = (const uint32_t *)(k.blob + k.off_lut);
         uint32_t *lut_s = (uint32_t *)(dyn_smem + (plan.lut - smem_base));
-        for (uint32_t i = tid; i < (32u << LB); i += 1024) lut_s[i] = __ldg(lut_g + (i >> 5));
+        // (FP16: three tables of 256 entries, sixteen copies each: word j holds entry j / 16)
+        constexpr uint32_t kLutWords = FMT ? 3u * 16u * 256u : 32u << LB;
+        for (uint32_t i = tid; i < kLutWords; i += 1024) lut_s[i] = __ldg(lut_g + (i >> (FMT ? 4 : 5)));
     }
     if (lane == 0) {
         mbar_init(bar0, 1);
@@ -169,16 +179,16 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
         return (min(left, k.chunk_cols) + 31u) >> 5;
     };
     auto record_ok = [&](uint32_t r0, uint32_t r1, uint32_t nkb) -> bool {
-        return r1 > r0 && r1 <= k.payload_units && (r1 - r0) * 128u > nkb * 512u &&
-               (r1 - r0) * 128u - nkb * 512u <= A.slot_bytes;
+        return r1 > r0 && r1 <= k.payload_units && (r1 - r0) * 128u > raw_part(nkb) &&
+               (r1 - r0) * 128u - raw_part(nkb) <= A.slot_bytes;
     };
     auto issue = [&](uint32_t c, uint32_t which) {
         uint32_t nkb = blocks_of(c % KC), r0 = __ldg(index + c), r1 = __ldg(index + c + 1);
         uint32_t bar = bar0 + which * 8;
         if (record_ok(r0, r1, nkb)) {
-            uint32_t bytes = (r1 - r0) * 128u - nkb * 512u;
+            uint32_t bytes = (r1 - r0) * 128u - raw_part(nkb);
             mbar_expect_tx(bar, bytes);
-            bulk_g2s(slot0 + which * A.slot_bytes, payload + (uint64_t)r0 * 128u + nkb * 512u, bytes, bar);
+            bulk_g2s(slot0 + which * A.slot_bytes, payload + (uint64_t)r0 * 128u + raw_part(nkb), bytes, bar);
         } else {
             mbar_expect_tx(bar, 0);
         }
@@ -275,9 +285,9 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                 const uint32_t nkb = blocks_of(kc);
                 const bool ok = record_ok(r0, r1, nkb);
                 const uint32_t r2 = c + 1 < c_end ? __ldg(index + c + 2) : r1;
-                const uint8_t *raw_p = payload + (uint64_t)r0 * 128u + lane * 16u;
+                const uint8_t *raw_p = payload + (uint64_t)r0 * 128u + lane * kRawLane;
                 uint4 raw_cur = make_uint4(0, 0, 0, 0);
-                if (ok) raw_cur = ldg_stream16(raw_p);
+                if (ok) raw_cur = load_raw(raw_p);
                 bounded_wait(bar0 + which * 8, (phase >> which) & 1u);
                 phase ^= 1u << which;
                 if (!ok && A.err && lane == 0) atomicExch(A.err, (int32_t)min(c + 1, 0x7FFFFFFFu));
@@ -287,12 +297,13 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                 // one block: fetch the next block's raw bytes and activations into the other register set, decode
                 // this one, hand it to the tensor core
                 auto block = [&](const uint4 &raw_c, uint4 &raw_n, const uint4 &x_c, uint4 &x_n2, bool more) {
-                    raw_p += 512;
-                    if (more && ok) raw_n = ldg_stream16(raw_p);
+                    raw_p += kRawBlock;
+                    if (more && ok) raw_n = load_raw(raw_p);
                     if (x_p < x_end) load_x(x_n2, x_p);
                     x_p += 32;
                     uint32_t a[8];
-                    decode_block<R>(sa, sb, kIdxMask, lut_lane, raw_c, a);   // a chunk that is not ok decodes garbage, never out of range
+                    if (FMT) decode_block_fp16(sa, sb, lut_lane, raw_c.x, a);   // a chunk that is not ok decodes garbage, never out of range
+                    else decode_block<R>(sa, sb, kIdxMask, lut_lane, raw_c, a);
                     stage_block(a, x_c, gb == gb_item);
                 };
                 uint4 raw_b = make_uint4(0, 0, 0, 0);
@@ -373,9 +384,9 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
-template <int LB, int NPAD>
+template <int LB, int NPAD, int FMT>
 static cudaError_t launch_tc_one(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
-    auto fn = huff_gemm_tc_kernel<LB, NPAD>;
+    auto fn = huff_gemm_tc_kernel<LB, NPAD, FMT>;
     static bool attr_set[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
@@ -389,14 +400,19 @@ static cudaError_t launch_tc_one(const KernelArgs &k, uint32_t grid, cudaStream_
 }
 
 cudaError_t launch_gemm_tc(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
-    if (k.lut_bits == 8) {
-        if (k.tc_npad == 16) return launch_tc_one<8, 16>(k, grid, stream);
-        if (k.tc_npad == 32) return launch_tc_one<8, 32>(k, grid, stream);
-        return launch_tc_one<8, 64>(k, grid, stream);
+    if (k.fmt) {
+        if (k.tc_npad == 16) return launch_tc_one<8, 16, 1>(k, grid, stream);
+        if (k.tc_npad == 32) return launch_tc_one<8, 32, 1>(k, grid, stream);
+        return launch_tc_one<8, 64, 1>(k, grid, stream);
     }
-    if (k.tc_npad == 16) return launch_tc_one<9, 16>(k, grid, stream);
-    if (k.tc_npad == 32) return launch_tc_one<9, 32>(k, grid, stream);
-    return launch_tc_one<9, 64>(k, grid, stream);
+    if (k.lut_bits == 8) {
+        if (k.tc_npad == 16) return launch_tc_one<8, 16, 0>(k, grid, stream);
+        if (k.tc_npad == 32) return launch_tc_one<8, 32, 0>(k, grid, stream);
+        return launch_tc_one<8, 64, 0>(k, grid, stream);
+    }
+    if (k.tc_npad == 16) return launch_tc_one<9, 16, 0>(k, grid, stream);
+    if (k.tc_npad == 32) return launch_tc_one<9, 32, 0>(k, grid, stream);
+    return launch_tc_one<9, 64, 0>(k, grid, stream);
 }
 
 }  // namespace huffllm

@@ -144,7 +144,10 @@ FP16_GENS = {"fp16": lambda r, c, seed: wl.gaussian_weights(r, c, 0.02, seed, "f
     (40, 2080, 1024, "fp16_from_bf16", 3),        # ragged rows, odd number of blocks in the last column chunk
     (512, 4096, 2048, "fp16_from_bf16", 8),       # larger chunks fit when the weights came from bf16 (10.9 bits per weight)
     (2368, 512, 512, "fp16", 5),                  # many chunks per warp
-    (272, 2048, 1024, "fp16", 16),                # batch above 8: passes of 8 vectors
+    (272, 2048, 1024, "fp16", 16),                # batch above 8: the tensor-core path with f16 operands
+    (1000, 4096, 1024, "fp16", 33),               # ragged row tiles, batch padded to 64, several column ranges
+    (600, 2080, 1024, "fp16_from_bf16", 9),       # odd block count in the last chunk, batch padded to 16
+    (64, 4096, 4096, "fp16", 12),                 # records too large for the tensor-core kernel's slots: passes of 8 vectors
 ])
 def test_fp16_decode_and_product(hl, torch, rows, cols, ce, gen, batch):
     """FP16 {1,5,5,5} blobs: bit-exact decode and products within the tolerance, against the oracle."""
