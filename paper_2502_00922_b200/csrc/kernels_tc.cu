@@ -1,7 +1,7 @@
-// Small-batch product on the 5th-generation tensor cores (tcgen05), batch 16..64.
+// Small-batch product on the 5th-generation tensor cores (tcgen05), batch 9..64.
 //
 // Same decoder as the matrix-vector kernel (one table lookup per weight, two bit sequences per lane), but the
-// decoded bf16 weights are not multiplied from registers: every warp stores its 16 rows x 32 columns of a
+// decoded 16-bit weights are not multiplied from registers: every warp stores its 16 rows x 32 columns of a
 // block into TENSOR MEMORY as the A operand of a 128-row tile, the activations of the same 32 columns go to
 // shared memory as the B operand, and one thread issues tcgen05.mma (M = 128, N = padded batch, K = 16)
 // whose fp32 accumulator also lives in tensor memory.  The decoded weights are consumed where they are
@@ -15,9 +15,10 @@
 // A work item is (512 rows) x (a range of column chunks); partial results of the ranges of one row tile are
 // added in a fixed order by whoever finishes last (per-warp arrival counters, nobody waits).
 //
-// Stage protocol: every warp fills its share of stage s (A rows, a slice of B), then bumps a shared-memory
-// counter; the 32nd arrival issues the 8 MMAs of the stage and a tcgen05.commit onto the stage's "empty"
-// mbarrier, which the warps wait on (with a limit) before they reuse the stage four blocks later.
+// Stage protocol: every warp fills its share of stage s (A rows, a slice of B) and meets the other decoder warps at
+// a hardware barrier; one of them (they take turns) then issues the 8 MMAs of the stage and a tcgen05.commit onto
+// the stage's "empty" mbarrier, which the warps wait on (with a limit) before they reuse the stage four blocks later.
+// BF16 and FP16 {1,5,5,5} blobs share the kernel (template parameter FMT): tables, raw part and operand format differ.
 #include "decode_common.cuh"
 
 namespace huffllm {
