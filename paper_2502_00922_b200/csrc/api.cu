@@ -52,12 +52,15 @@ struct TcPlan {
     size_t ticket_off, partial_off, bytes;
 };
 // Shared memory the tensor-core kernel needs with `tiles` 128-row tiles per CTA.
+// Stages of the tensor-core kernel: four, two at the widest batch padding, where shared memory is short.
+uint32_t tc_stages(uint32_t npad) { return npad == 64 ? 2u : 4u; }
 uint64_t tc_smem_need(const huffllm_desc *d, uint32_t npad, uint32_t tiles) {
     const bool fp16 = d->dtype == HUFFLLM_FP16;
     const uint32_t checks_per_block = fp16 ? 8 : (d->lut_bits == 8 ? 3 : 4);
     uint64_t guard = 256ull * (3 + checks_per_block * (d->chunk_cols / kBlockCols));
     const uint64_t lut = fp16 ? 49152ull : 128ull << d->lut_bits;
-    return lut + guard + 4ull * npad * 64 + 4096 + 2ull * 8 * tiles * d->max_words * 256;
+    const uint64_t b_stages = (uint64_t)tc_stages(npad) * npad * 64;          // the guard area may lie over them
+    return lut + (guard > b_stages ? guard - b_stages : 0) + b_stages + 4096 + 2ull * 8 * tiles * d->max_words * 256;
 }
 TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn_smem) {
     TcPlan p;
@@ -135,7 +138,7 @@ huffllm_status add_matrix(KernelArgs *k, const huffllm_desc *desc, const void *b
 huffllm_status finish_args(KernelArgs *k, bool product, const DeviceInfo &dev, uint32_t *grid) {
     k->part_bytes = product ? 2 * 32 * 16 * k->batch * (uint32_t)sizeof(float) : 0;
     // worst case for the table's alignment gap is covered by assuming the window starts within 4 KB of zero
-    uint64_t fixed = (uint64_t)k->lut_size + k->guard_bytes + k->part_bytes + 4096;
+    uint64_t fixed = (uint64_t)k->lut_size + (k->guard_bytes > k->part_bytes ? k->guard_bytes - k->part_bytes : 0) + k->part_bytes + 4096;
     if (fixed + 2ull * k->slot_bytes > k->dyn_smem_bytes)
         return fail(HUFFLLM_ERR_UNSUPPORTED, "chunk records too large for shared memory (slot %u bytes)", k->slot_bytes);
     uint64_t g = k->total_chunks < (uint64_t)dev.sms ? k->total_chunks : (uint64_t)dev.sms;
@@ -266,7 +269,7 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
         uint32_t grid;
         begin_args(&k, batch, *dev);
         if ((st = add_matrix(&k, desc, blob)) != HUFFLLM_OK) return st;
-        k.part_bytes = 4 * tp.npad * 64;                       // four stages of activations
+        k.part_bytes = tc_stages(tp.npad) * tp.npad * 64;      // the stages of activations
         const uint64_t need = tc_smem_need(desc, tp.npad, tp.tiles);
         if (need <= k.dyn_smem_bytes && workspace_bytes >= tp.bytes) {
             k.m[0].x = x;

@@ -240,7 +240,7 @@ __device__ __forceinline__ void decode_block_fp16(LaneStream &sa, LaneStream &sb
 //   [base, lut)            slot pairs (as many as fit)
 //   [lut, lut + LUTSZ)     per-lane LUT; lut = base rounded up to a multiple of LUTSZ, so that the
 //                          index bits of a lookup address never overlap the table's base bits
-//   [lut + LUTSZ, ...)     more slot pairs, then a guard area no valid stream ever reads
+//   [lut + LUTSZ, ...)     more slot pairs, then a guard area no valid stream ever reads (it may overlap the next area)
 //   [end - part_bytes, end) the CTA's table of partial sums (fused product only)
 struct SmemPlan {
     uint32_t lut;    // shared address of the table
@@ -266,7 +266,9 @@ __device__ __forceinline__ SmemPlan plan_smem(uint32_t base, const KernelArgs &k
     p.nA = p.lut > a0 ? div_pair(p.lut - a0) : 0;  // a stream that overruns here reads the table: harmless
     p.slotB = p.lut + k.lut_size;
     uint32_t end = base + k.dyn_smem_bytes - k.part_bytes;
-    uint32_t roomB = end > p.slotB + k.guard_bytes ? end - p.slotB - k.guard_bytes : 0;
+    // the guard area (read only, and only by a corrupt stream) may lie over what follows the slots; what it needs beyond that stays free
+    const uint32_t guard_extra = k.guard_bytes > k.part_bytes ? k.guard_bytes - k.part_bytes : 0;
+    uint32_t roomB = end > p.slotB + guard_extra ? end - p.slotB - guard_extra : 0;
     p.warps = min(max_warps, p.nA + div_pair(roomB));
     return p;
 }

@@ -107,7 +107,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     };
     constexpr int R = LB == 8 ? 3 : 2;
     constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
-    constexpr int S = kTcStages;
+    constexpr int S = NPAD == 64 ? 2 : kTcStages;          // the host's tc_stages(): shared memory is short at the widest padding
     constexpr uint32_t kBStage = NPAD * 64;                 // bytes of B per stage: NPAD rows x 32 columns of bf16
     constexpr uint32_t kLbo = 128, kSbo = 512;              // core matrices: 4 along K side by side, then the next 8 rows
     constexpr uint32_t kACol0 = kTcTiles * NPAD;            // first tensor-memory column of the A stages
