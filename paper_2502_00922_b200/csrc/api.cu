@@ -68,12 +68,24 @@ TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn
     p.tiles = 4;                                    // as many 8-warp tiles as the chunk slots leave room for
     while (p.tiles > 1 && tc_smem_need(d, p.npad, p.tiles) > dyn_smem) --p.tiles;
     p.m_tiles = (d->row_groups + 8 * p.tiles - 1) / (8 * p.tiles);
+    // Column ranges: the one with the shortest finish time.  A CTA takes items b, b + grid, ... in turn; an item costs its
+    // column chunks (ranges of one matrix differ by a chunk when ksplit does not divide the chunk count) plus an epilogue
+    // worth about a quarter of a chunk.  Counting whole waves alone would pick many short, unequal ranges.
     uint32_t best = 1;
-    double best_eff = 0;
+    uint64_t best_span = ~0ull;
     for (uint32_t ks = 1; ks <= 16 && ks <= d->col_chunks; ++ks) {
-        uint64_t items = (uint64_t)p.m_tiles * ks, waves = (items + sms - 1) / sms;
-        double eff = (double)items / (double)(waves * sms);
-        if (eff > best_eff + 1e-9) { best_eff = eff; best = ks; }
+        const uint64_t items = (uint64_t)p.m_tiles * ks, grid = items < sms ? items : sms;
+        uint64_t span = 0;
+        for (uint64_t b = 0; b < grid; ++b) {
+            uint64_t t = 0;
+            for (uint64_t it = b; it < items; it += grid) {
+                const uint32_t r = (uint32_t)(it % ks);
+                const uint32_t len = (uint32_t)((uint64_t)d->col_chunks * (r + 1) / ks) - (uint32_t)((uint64_t)d->col_chunks * r / ks);
+                t += 4ull * len + 1;
+            }
+            if (t > span) span = t;
+        }
+        if (span < best_span) { best_span = span; best = ks; }
     }
     p.ksplit = best;
     p.items = p.m_tiles * best;
