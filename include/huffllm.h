@@ -226,7 +226,8 @@ huffllm_status huffllm_decode(const huffllm_desc *desc, const void *blob_dev, ui
  * y = W x with W taken straight from the compressed blob: weights are decoded in registers and
  * multiplied at once, so only compressed bytes cross the memory bus (Section 1: weights are
  * decompressed only when needed, to multiply with activations).  x: device, cols words of the
- * blob's dtype.  y: device, rows floats.  cols must be a multiple of 32 (UNSUPPORTED otherwise;
+ * blob's dtype.  y: rows floats in device memory, or in pinned host memory the device can address (the results
+ * then go to the host as the kernels produce them; y is only ever written).  cols must be a multiple of 32 (UNSUPPORTED otherwise;
  * huffllm_decode takes any shape).  Products are exact, sums are accumulated in fp32.
  * Results are bitwise reproducible from run to run.
  */
@@ -341,6 +342,17 @@ huffllm_status huffllm_split_histogram(const uint16_t *w_dev, uint64_t n_weights
                                        uint64_t *counts_dev, huffllm_stream stream);
 huffllm_status huffllm_split_entropy(const uint64_t *counts_host, const uint8_t *widths, uint32_t n_fields,
                                      double *entropy_bits, double *huffman_bits);
+
+/*
+ * Copy `bytes` (a multiple of 16; both pointers 16-byte aligned) between two buffers the device can address —
+ * device memory, or pinned host memory (cudaHostAlloc / cudaHostRegister: with unified addressing the device reaches
+ * it through the same pointer) — with a small kernel on `stream`.  Meant for the activations and results of a decode
+ * step (tens of kilobytes per token, Section 1: end-to-end latency): between kernels, and above all inside a CUDA graph,
+ * a kernel copy costs a few microseconds where a DMA copy costs about ten.  The product calls also accept such pinned host
+ * memory as their y, in which case the results are written to the host by the kernels themselves (x should be
+ * staged into device memory: every CTA reads it).  Asynchronous; wait for the stream before reading a host destination.
+ */
+huffllm_status huffllm_stage_copy(void *dst, const void *src, size_t bytes, huffllm_stream stream);
 
 /* Message of the last failing call on this thread ("" if none). */
 const char *huffllm_last_error(void);

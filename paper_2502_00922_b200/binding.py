@@ -58,6 +58,7 @@ _SIGNATURES = {
     "huffllm_decode_gemm_host": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p,
                                  C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemm_static": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p],
+    "huffllm_stage_copy": [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p],
     "huffllm_plain_gemv": [C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p],
     "huffllm_build_codebook_from_counts": [C.c_void_p, C.c_int, C.c_int, C.c_uint32, C.POINTER(C.c_void_p)],
     "huffllm_encode_device_scratch_bytes": [C.c_uint64, C.c_uint64, C.c_uint32, C.POINTER(C.c_size_t)],
@@ -342,3 +343,8 @@ def encode_device(cb: Codebook, w_dev, rows: int, cols: int, chunk_elems, blob_d
     _check(lib().huffllm_encode_device(cb._h, _ptr(w_dev), rows, cols, chunk_elems, _ptr(blob_dev), blob_cap, _ptr(scratch_dev),
                                        scratch_bytes, C.byref(desc), _stream(stream)))
     return desc
+
+
+def stage_copy(dst, src, nbytes: int, stream=None):
+    """huffllm_stage_copy: a small copy by a kernel between device-accessible buffers (device or pinned host memory)."""
+    _check(lib().huffllm_stage_copy(_ptr(dst), _ptr(src), nbytes, _stream(stream)))

@@ -408,6 +408,18 @@ huffllm_status huffllm_decode_gemm_static(const huffllm_desc *desc, const void *
     return huffllm_decode_gemm(desc, blob, x, batch, y, ws, sizeof(g_static_scratch), err_flag, stream);
 }
 
+huffllm_status huffllm_stage_copy(void *dst, const void *src, size_t bytes, huffllm_stream stream) {
+    clear_error();
+    DeviceInfo *dev;
+    huffllm_status st = device_info(&dev);
+    if (st != HUFFLLM_OK) return st;
+    if (!dst || !src) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
+    if (bytes % 16 || ((uintptr_t)dst & 15) || ((uintptr_t)src & 15)) return fail(HUFFLLM_ERR_INVALID_ARG, "size and pointers must be multiples of 16 bytes");
+    cudaError_t e = launch_stage_copy(dst, src, bytes, (uint32_t)dev->sms, (cudaStream_t)stream);
+    if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "copy launch: %s", cudaGetErrorString(e));
+    return HUFFLLM_OK;
+}
+
 huffllm_status huffllm_plain_gemv(const uint16_t *w, uint64_t rows, uint64_t cols, const uint16_t *x, float *y, huffllm_stream stream) {
     clear_error();
     DeviceInfo *dev;

@@ -47,6 +47,7 @@ struct KernelArgs {
 cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t stream);
 cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream);
 cudaError_t launch_gemm_tc(const KernelArgs &k, uint32_t grid, cudaStream_t stream);
+cudaError_t launch_stage_copy(void *dst, const void *src, uint64_t bytes, uint32_t sms, cudaStream_t stream);
 cudaError_t launch_plain_gemv(const uint16_t *w, uint64_t rows, uint64_t cols, const uint16_t *x, float *y, uint32_t sms,
                               cudaStream_t stream);
 

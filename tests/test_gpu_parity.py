@@ -444,3 +444,27 @@ def test_ffn70b_shapes_small_batch_sampled(hl, torch, rows, cols):
         y = gpu_gemm(hl, torch, up, x)
         yo, d = orc.matmul(w[rs], x)
         assert np.all(np.abs(y[:, rs] - yo) <= TOL * d), f"batch {batch}"
+
+
+def test_results_straight_to_pinned_host_memory_and_kernel_copy(hl, torch):
+    """y may be pinned host memory (the kernels write the results to the host themselves), and huffllm_stage_copy moves
+    small buffers between pinned host memory and the device with a kernel."""
+    rows, cols = 1040, 2048
+    w = wl.gaussian_weights(rows, cols, 0.02, 77)
+    up = Uploaded(hl, torch, w, 4096, 0, 3)
+    x = wl.activations(3, cols, 78)
+    x_host = torch.from_numpy(x.view(np.int16).reshape(-1).copy()).pin_memory()
+    x_dev = torch.zeros(x_host.numel() + 8, dtype=torch.int16, device="cuda")
+    y_host = torch.full((3 * rows + 4,), float("nan"), dtype=torch.float32).pin_memory()
+    hl.stage_copy(x_dev, x_host, x_host.numel() * 2)
+    hl.decode_gemm(up.desc, up.blob_dev, x_dev, 3, y_host, up.ws, up.ws_bytes, up.err)
+    torch.cuda.synchronize()
+    assert int(up.err.item()) == 0
+    assert np.array_equal(x_dev.cpu().numpy()[:x_host.numel()], x_host.numpy()) and not x_dev[x_host.numel():].any()
+    y = y_host.numpy()
+    assert np.all(np.isnan(y[3 * rows:]))
+    check_product(y[:3 * rows].reshape(3, rows), w, x)
+    # the same results as through device memory, bit for bit
+    assert np.array_equal(gpu_gemm(hl, torch, up, x), y[:3 * rows].reshape(3, rows))
+    with pytest.raises(hl.HuffllmError):
+        hl.stage_copy(x_dev, x_host, 24)                      # not a multiple of 16
