@@ -584,7 +584,7 @@ def main():
                          "note": "all matrices of the step in one launch: only valid where their inputs are independent"},
                      "per_matrix": [{"name": m["name"], "rows": m["rows"], "cols": m["cols"], "ms": t,
                                      "comp_GBs": m["alg_bytes"] / (t * 1e-3) / 1e9} for m, t in zip(mats, per_mat_ms)]},
-        # what actually binds the bf16 kernel: instruction dispatch (see DESIGN.md); peak = dispatch cycles the GPU has per
+        # what actually binds the bf16 kernel: instruction dispatch; peak = dispatch cycles the GPU has per
         # second (SMs x 4 schedulers x SM clock), achieved = dispatch cycles the decoder formulation needs for the step's weights
         "alu_roofline": None if (fp16 or B > 8) else {
             "bound": "alu", "unit": "G dispatch cycles/s",
