@@ -60,11 +60,11 @@ FALLBACK_HBM_GBS = 6650.0
 # additions, IMAD with an immediate, FADD and conflict-free LDS; the kernel's time is the sum of these over its instruction
 # mix.  Per weight-lane step the formulation needs 11.4 dispatch cycles (decoder step: shift 2 + address 2 + lookup 1 + pointer
 # advance 2; pack 2.1; refill check 6 x 3/8) and the kernel executes 14.2 (per-opcode counters of the ncu capture in profiles/:
-# 4.89 two-cycle and 4.43 one-cycle instructions).
+# 4.76 two-cycle and 4.68 one-cycle instructions).
 DISPATCH_CYCLES_ALGORITHMIC = 11.4
 DISPATCH_CYCLES_EXECUTED = 14.2
 SCHEDULERS_PER_SM = 4
-NCU_TRAFFIC_RATIO = 1.03   # profiles/huff_kernel_product_llama7b_layer.md: 145.7 MB moved for 142.0 MB (gate+up), 71.8 for 71.0 (down)
+NCU_TRAFFIC_RATIO = 1.03   # profiles/huff_kernel_product_llama7b_layer.md: 146.9 MB moved for 142.1 MB (gate+up), 71.9 for 71.0 (down)
 
 
 def max_over_ranks(v: float, dist, device) -> float:
