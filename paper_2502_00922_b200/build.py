@@ -30,6 +30,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
         cmd.insert(1, "-DHUFFLLM_TIMING")
     if os.environ.get("HUFFLLM_THREADS"):          # experiment knob: threads per CTA of the decode kernels
         cmd.insert(1, "-DHUFFLLM_THREADS=" + os.environ["HUFFLLM_THREADS"])
+    for d in os.environ.get("HUFFLLM_DEFS", "").split():   # experiment knob: extra -D definitions
+        cmd.insert(1, "-D" + d)
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     subprocess.check_call(cmd)

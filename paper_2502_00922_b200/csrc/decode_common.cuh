@@ -95,11 +95,11 @@ struct LaneStream {
     uint32_t lo, hi, pos, nxt;
 };
 
-__device__ __forceinline__ void stream_open(LaneStream &s, uint32_t lane_word0) {
+__device__ __forceinline__ void stream_open(LaneStream &s, uint32_t lane_word0, uint32_t pos0 = 0) {
     s.lo = lds_stream(lane_word0);
     s.hi = lds_stream(lane_word0 + 256);
     s.nxt = lane_word0 + 512;
-    s.pos = 0;
+    s.pos = pos0;
 }
 
 // One decoder step: returns the table entry (length << 16 | exponent << 7) and advances the start pointer.
@@ -111,6 +111,18 @@ __device__ __forceinline__ uint32_t stream_step(LaneStream &s, uint32_t idx_mask
     uint64_t win = ((uint64_t)s.hi << 32) | s.lo;
     uint32_t t = (uint32_t)(win >> s.pos), addr;
     asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(addr) : "r"(t), "r"(idx_mask), "r"(lut_lane));
+    uint32_t e = lds_lut(addr);
+    s.pos = __dp4a(e, 0x00010000u, s.pos);
+    return e;
+}
+
+// The same step for a pointer that stands on the codeword itself (the sequence's leading zero bits already skipped):
+// the 8-bit table index is then byte 0 of the shifted window, and index * 128 + table base is one byte dot product.
+// Nothing is kept in front of the pointer, so a window holds 33 valid bits after a refill check: four codewords.
+__device__ __forceinline__ uint32_t stream_step_skip(LaneStream &s, uint32_t lut_lane) {
+    uint64_t win = ((uint64_t)s.hi << 32) | s.lo;
+    uint32_t t = (uint32_t)(win >> s.pos);
+    uint32_t addr = __dp4a(t, 0x00000080u, lut_lane);
     uint32_t e = lds_lut(addr);
     s.pos = __dp4a(e, 0x00010000u, s.pos);
     return e;
@@ -167,7 +179,7 @@ __device__ __forceinline__ uint32_t rotr8(uint32_t v) { return prmt(v, v, 0x0321
 // The lane's two sequences are stepped alternately.  Each window is checked for a refill before every
 // R-th step: after a check at least 26 bits are valid in front of the start pointer, enough for R
 // codewords of at most 26/R bits.
-template <int R>
+template <int R, bool SKIP = false>
 __device__ __forceinline__ void decode_block(LaneStream &sa, LaneStream &sb, uint32_t idx_mask, uint32_t lut_lane,
                                              const uint4 &raw, uint32_t (&a)[8]) {
     uint32_t e[16];
@@ -177,8 +189,8 @@ __device__ __forceinline__ void decode_block(LaneStream &sa, LaneStream &sb, uin
             stream_refill(sa);
             stream_refill(sb);
         }
-        e[i] = stream_step(sa, idx_mask, lut_lane);
-        e[8 + i] = stream_step(sb, idx_mask, lut_lane);
+        e[i] = SKIP ? stream_step_skip(sa, lut_lane) : stream_step(sa, idx_mask, lut_lane);
+        e[8 + i] = SKIP ? stream_step_skip(sb, lut_lane) : stream_step(sb, idx_mask, lut_lane);
     }
     a[0] = pack_pair(e[0], e[1], raw.x);
     a[1] = pack_pair(e[2], e[3], rotr8(raw.x));

@@ -47,7 +47,10 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     constexpr uint32_t kRawLane = FMT ? 2u : 16u;             // of which one lane's share
     // raw part of a record with nkb blocks (FP16: padded to the 128-byte record unit)
     auto raw_part = [](uint32_t nkb) -> uint32_t { return FMT ? (nkb * 64u + 127u) & ~127u : nkb * 512u; };
-    constexpr int R = LB == 8 ? 3 : 2;                       // decoder steps between two refill checks
+    // 8-bit BF16 tables: the decoder starts behind the sequences' leading zero bits and forms the table address from
+    // byte 0 of the shifted window (stream_step_skip), which leaves room for four codewords between two refill checks
+    constexpr bool SKIP = LB == 8 && FMT == 0;
+    constexpr int R = SKIP ? 4 : LB == 8 ? 3 : 2;            // decoder steps between two refill checks
     constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
     extern __shared__ __align__(128) uint8_t dyn_smem[];
     __shared__ __align__(16) uint64_t bars[kMaxWarps * 2];     // a warp's two barriers differ in address bit 3 only
@@ -327,8 +330,8 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                     if (MODE == 1) xq += nkb * 32u;
                 } else {
                     LaneStream sa, sb;
-                    stream_open(sa, slot_cur);
-                    stream_open(sb, slot_cur + 128u);
+                    stream_open(sa, slot_cur, SKIP ? 7u : 0u);
+                    stream_open(sb, slot_cur + 128u, SKIP ? 7u : 0u);
                     const uint32_t col0 = kc * k.chunk_cols + t * 8u;
                     // (activations: lanes of unused output columns repeat the last vector; cols is a multiple of 32
                     // here, so every block of the chunk lies inside the row and xq ends the chunk where the next begins)
@@ -354,7 +357,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
 
                         uint32_t a[8];
                         if (FMT) decode_block_fp16(sa, sb, lut_lane, cur.x, a);
-                        else decode_block<R>(sa, sb, kIdxMask, lut_lane, cur, a);
+                        else decode_block<R, SKIP>(sa, sb, kIdxMask, lut_lane, cur, a);
                         BLOCKSTAMP((c - c_beg) * 8 + kb, 1);
 
                         if (MODE == 1) {

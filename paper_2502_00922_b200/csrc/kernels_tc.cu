@@ -96,6 +96,9 @@ __device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t addr, uint32_t lbo
 
 // LB = table index bits; NPAD = batch rounded up to 16, 32 or 64 (the MMA's N); FMT = 0: BF16 blobs, 1: FP16 {1,5,5,5} blobs
 // (three tables, sign words as the raw part, f16 operands).
+#ifndef HUFFLLM_TC_SKIP_BELOW
+#define HUFFLLM_TC_SKIP_BELOW 64
+#endif
 template <int LB, int NPAD, int FMT>
 __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_constant__ KernelArgs A) {
     constexpr uint32_t kRawBlock = FMT ? 64u : 512u;          // raw bytes of one block of a record
@@ -105,7 +108,10 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
         if (FMT) return make_uint4(ldg_stream2(p), 0, 0, 0);
         return ldg_stream16(p);
     };
-    constexpr int R = LB == 8 ? 3 : 2;
+    // the decoder that starts behind the leading zero bits (see huff_kernel); at the widest padding, where a block's
+    // time is set by the two-stage hand-over, it measured 1.4 % slower and is left out
+    constexpr bool SKIP = LB == 8 && FMT == 0 && NPAD < HUFFLLM_TC_SKIP_BELOW;
+    constexpr int R = SKIP ? 4 : LB == 8 ? 3 : 2;
     constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
     constexpr int S = NPAD == 64 ? 2 : kTcStages;          // the host's tc_stages(): shared memory is short at the widest padding
     constexpr uint32_t kBStage = NPAD * 64;                 // bytes of B per stage: NPAD rows x 32 columns of bf16
@@ -293,8 +299,8 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                 phase ^= 1u << which;
                 if (!ok && A.err && lane == 0) atomicExch(A.err, (int32_t)min(c + 1, 0x7FFFFFFFu));
                 LaneStream sa, sb;
-                stream_open(sa, slot0 + which * A.slot_bytes + (lane << 2));
-                stream_open(sb, slot0 + which * A.slot_bytes + 128u + (lane << 2));
+                stream_open(sa, slot0 + which * A.slot_bytes + (lane << 2), SKIP ? 7u : 0u);
+                stream_open(sb, slot0 + which * A.slot_bytes + 128u + (lane << 2), SKIP ? 7u : 0u);
                 // one block: fetch the next block's raw bytes and activations into the other register set, decode
                 // this one, hand it to the tensor core
                 auto block = [&](const uint4 &raw_c, uint4 &raw_n, const uint4 &x_c, uint4 &x_n2, bool more) {
@@ -304,7 +310,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                     x_p += 32;
                     uint32_t a[8];
                     if (FMT) decode_block_fp16(sa, sb, lut_lane, raw_c.x, a);   // a chunk that is not ok decodes garbage, never out of range
-                    else decode_block<R>(sa, sb, kIdxMask, lut_lane, raw_c, a);
+                    else decode_block<R, SKIP>(sa, sb, kIdxMask, lut_lane, raw_c, a);
                     stage_block(a, x_c, gb == gb_item);
                 };
                 uint4 raw_b = make_uint4(0, 0, 0, 0);
