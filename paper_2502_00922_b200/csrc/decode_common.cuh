@@ -116,16 +116,59 @@ __device__ __forceinline__ uint32_t stream_step(LaneStream &s, uint32_t idx_mask
     return e;
 }
 
-// The same step for a pointer that stands on the codeword itself (the sequence's leading zero bits already skipped):
-// the 8-bit table index is then byte 0 of the shifted window, and index * 128 + table base is one byte dot product.
-// Nothing is kept in front of the pointer, so a window holds 33 valid bits after a refill check: four codewords.
-__device__ __forceinline__ uint32_t stream_step_skip(LaneStream &s, uint32_t lut_lane) {
-    uint64_t win = ((uint64_t)s.hi << 32) | s.lo;
-    uint32_t t = (uint32_t)(win >> s.pos);
-    uint32_t addr = __dp4a(t, 0x00000080u, lut_lane);
-    uint32_t e = lds_lut(addr);
-    s.pos = __dp4a(e, 0x00010000u, s.pos);
-    return e;
+// The decoder of 8-bit BF16 tables works on four codewords at a time.  Its pointer stands on the codeword itself (the
+// sequence's leading zero bits are skipped when the sequence is opened), so after a refill check, with the pointer
+// below 32, the low 32 bits of the shifted window are all valid: room for four codewords of at most 8 bits.
+//   * The 32 bits are taken out of the window once (one 64-bit shift) and then shifted in place by each codeword's
+//     length: the shared-memory copy of the table repeats the length in an entry's low 5 bits (lut_entry_inplace), and a
+//     wrapping shift reads just those.  The pointer is not on the chain from one lookup to the next.
+//   * The table index is byte 0 of that word, and index * 128 + table base is one byte dot product.
+//   * The pointer is advanced once per four codewords by two three-input additions of the whole entries.  Only its low
+//     6 bits mean anything (pointer + lengths <= 31 + 32; bits 5 and 6 of an entry are zero, the exponent starts at
+//     bit 7, so nothing carries into them and bit 6 stays zero); whatever piles up above bit 6 is never read: the
+//     refill check tests bit 5 and the funnel shift reads bits 0..4.
+__device__ __forceinline__ uint32_t lut_entry_inplace(uint32_t e) { return e | (e >> 16); }
+
+__device__ __forceinline__ void stream_refill4(LaneStream &s) {
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b32 b;\n\t"
+        "setp.ne.u32 q, 0, 0;\n\t"
+        "lop3.or.b32 b|p, %2, 32, 0, 0xC0, q;\n\t"          // p = bit 5 of the pointer: 32 or more bits consumed
+        "@p ld.shared.u32 %0, [%3+-256];\n\t"
+        "@p ld.shared.u32 %1, [%3];\n\t"
+        "@p add.u32 %3, %3, 256;\n\t"
+        "@p add.u32 %2, %2, 0xFFFFFFE0;\n\t}"
+        : "+r"(s.lo), "+r"(s.hi), "+r"(s.pos), "+r"(s.nxt));
+}
+// The 32 window bits at the pointer, right after a refill check (pointer below 32: a 32-bit funnel shift is enough,
+// and it reads only the pointer's low 5 bits).
+__device__ __forceinline__ uint32_t window_at(const LaneStream &s) {
+    uint32_t t;
+    asm("shf.r.wrap.b32 %0, %1, %2, %3;" : "=r"(t) : "r"(s.lo), "r"(s.hi), "r"(s.pos));
+    return t;
+}
+__device__ __forceinline__ uint32_t lookup_byte0(uint32_t t, uint32_t lut_lane) { return lds_lut(__dp4a(t, 0x00000080u, lut_lane)); }
+__device__ __forceinline__ uint32_t shift_by_entry(uint32_t t, uint32_t e) {
+    uint32_t d;
+    asm("shf.r.wrap.b32 %0, %1, 0, %2;" : "=r"(d) : "r"(t), "r"(e));
+    return d;
+}
+// Four codewords of each of a lane's two sequences, the two chains interleaved.
+__device__ __forceinline__ void stream_step4x2(LaneStream &sa, LaneStream &sb, uint32_t lut_lane, uint32_t *ea, uint32_t *eb) {
+    stream_refill4(sa);
+    stream_refill4(sb);
+    uint32_t ta = window_at(sa), tb = window_at(sb);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        ea[k] = lookup_byte0(ta, lut_lane);
+        eb[k] = lookup_byte0(tb, lut_lane);
+        if (k < 3) {
+            ta = shift_by_entry(ta, ea[k]);
+            tb = shift_by_entry(tb, eb[k]);
+        }
+    }
+    sa.pos = (sa.pos + ea[0] + ea[1]) + (ea[2] + ea[3]);
+    sb.pos = (sb.pos + eb[0] + eb[1]) + (eb[2] + eb[3]);
 }
 
 // Refill: once 32 bits have been consumed, slide the window by one word.  Written with predicated
@@ -183,14 +226,18 @@ template <int R, bool SKIP = false>
 __device__ __forceinline__ void decode_block(LaneStream &sa, LaneStream &sb, uint32_t idx_mask, uint32_t lut_lane,
                                              const uint4 &raw, uint32_t (&a)[8]) {
     uint32_t e[16];
+    if (SKIP) {
+        stream_step4x2(sa, sb, lut_lane, e, e + 8);
+        stream_step4x2(sa, sb, lut_lane, e + 4, e + 12);
+    } else
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
         if (i % R == 0) {
             stream_refill(sa);
             stream_refill(sb);
         }
-        e[i] = SKIP ? stream_step_skip(sa, lut_lane) : stream_step(sa, idx_mask, lut_lane);
-        e[8 + i] = SKIP ? stream_step_skip(sb, lut_lane) : stream_step(sb, idx_mask, lut_lane);
+        e[i] = stream_step(sa, idx_mask, lut_lane);
+        e[8 + i] = stream_step(sb, idx_mask, lut_lane);
     }
     a[0] = pack_pair(e[0], e[1], raw.x);
     a[1] = pack_pair(e[2], e[3], rotr8(raw.x));

@@ -47,8 +47,8 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     constexpr uint32_t kRawLane = FMT ? 2u : 16u;             // of which one lane's share
     // raw part of a record with nkb blocks (FP16: padded to the 128-byte record unit)
     auto raw_part = [](uint32_t nkb) -> uint32_t { return FMT ? (nkb * 64u + 127u) & ~127u : nkb * 512u; };
-    // 8-bit BF16 tables: the decoder starts behind the sequences' leading zero bits and forms the table address from
-    // byte 0 of the shifted window (stream_step_skip), which leaves room for four codewords between two refill checks
+    // 8-bit BF16 tables: the decoder starts behind the sequences' leading zero bits and works on four codewords at a
+    // time (stream_step4x2)
     constexpr bool SKIP = LB == 8 && FMT == 0;
     constexpr int R = SKIP ? 4 : LB == 8 ? 3 : 2;            // decoder steps between two refill checks
     constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
@@ -146,6 +146,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
             for (int i = 0; i < kLutLoads; ++i) {
                 uint32_t v = tid + i * THREADS;
                 lut_v[i] = (kLutVecs % THREADS == 0 || v < kLutVecs) ? __ldg(lut_g + (v >> (kLutRep - 2))) : 0u;
+                if (SKIP) lut_v[i] = lut_entry_inplace(lut_v[i]);   // the length once more, where an in-place shift reads it
             }
         }
         if (lane == 0 && c_beg < c_end) {
