@@ -295,6 +295,12 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                 const uint32_t kc1 = kc + 1 == KC ? 0u : kc + 1;
                 const uint32_t r2 = has_next ? __ldg(index + c + 2) : r1;
                 const bool next_ok = has_next && record_ok(r1, r2, blocks_of(kc1));
+#ifdef HUFFLLM_PFC
+                // the raw part of the next record (one 128-byte line per lane) is asked into L2 a whole chunk ahead: the
+                // loads that bring it to registers run only one block ahead of the decoder, too short for a DRAM miss
+                if (next_ok && lane * 128u < raw_part(blocks_of(kc1)))
+                    asm volatile("prefetch.global.L2 [%0];" ::"l"(payload + (uint64_t)r1 * 128u + lane * 128u));
+#endif
 
                 if (MODE == 1 && (int)rg != cur_rg) {
                     flush(cur_rg, c_beg, c);  // the previous row group ended with chunk c - 1
@@ -341,14 +347,27 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
 
                     // one block: start the fetch of the next block's raw bytes into `nxt`, decode with `cur`
                     // (may_be_last = false: the caller knows that another block of this chunk follows)
+                    // Every block asks L2 for the 16 bytes per lane that lie four blocks further on in the record stream (the
+                    // loads that bring raw bytes to registers run one block ahead of the decoder, too short for a miss in
+                    // DRAM).  In a record's first half that is the raw part of its second half; in the second half it is the
+                    // coded part and, at its end, the start of the next record.  Measured: this plain form is the fastest;
+                    // asking only for raw bytes, or for the next record's first blocks, gains a third of it or nothing.
+                    // Not done where it could reach past the payload (the last records).
+                    // (products of BF16 blobs only: the decode-only kernel has no register to spare for it, and an FP16 record's
+                    // raw part is a sixteenth of its bytes)
+                    constexpr bool kPrefetchRaw = MODE == 1 && FMT == 0;
+                    const bool pf_safe = r1 + 4u * kRawBlock / 128u <= k.payload_units;
                     auto block = [&](uint32_t kb, const uint4 &cur, uint4 &nxt, auto may_be_last) {
                         BLOCKSTAMP((c - c_beg) * 8 + kb, 0);
                         raw_p += kRawBlock;
+                        if (kPrefetchRaw && pf_safe) asm volatile("prefetch.global.L2 [%0];" ::"l"(raw_p + 3u * kRawBlock));
                         if (decltype(may_be_last)::value) {
                             if (kb == last) raw_p += coded_bytes;       // the next record's first block
                             if (kb != last || next_ok) nxt = load_raw(raw_p);
                         } else {
+#ifndef HUFFLLM_NORAW
                             nxt = load_raw(raw_p);
+#endif
                         }
                         uint4 xv;
                         if (MODE == 1) {
