@@ -58,13 +58,13 @@ FALLBACK_HBM_GBS = 6650.0
 # What binds the bf16 fused kernel is instruction dispatch.  A one-off probe on the B200 (8 warps per scheduler, independent
 # chains) gave 2.0 cycles per warp instruction and scheduler for LOP3, SHF, PRMT, IDP4A, ISETP and SEL, and 1.0-1.2 for integer
 # additions, IMAD with an immediate, FADD and conflict-free LDS; the kernel's time is the sum of these over its instruction
-# mix.  Per weight-lane step the formulation needs 11.4 dispatch cycles (decoder step: shift 2 + address 2 + lookup 1 + pointer
-# advance 2; pack 2.1; refill check 6 x 3/8) and the kernel executes 14.2 (per-opcode counters of the ncu capture in profiles/:
-# 4.76 two-cycle and 4.68 one-cycle instructions).
-DISPATCH_CYCLES_ALGORITHMIC = 11.4
-DISPATCH_CYCLES_EXECUTED = 14.2
+# mix.  Per weight-lane step the formulation needs 9.1 dispatch cycles (per four codewords of a sequence: window extraction 2,
+# four times address 2 + lookup 1, three in-place shifts of 2, pointer advance 2, refill check 6; pack 2.1 per weight) and the
+# kernel executes 12.1 (per-opcode counters of the ncu capture in profiles/: 3.65 two-cycle and 4.83 one-cycle instructions).
+DISPATCH_CYCLES_ALGORITHMIC = 9.1
+DISPATCH_CYCLES_EXECUTED = 12.1
 SCHEDULERS_PER_SM = 4
-NCU_TRAFFIC_RATIO = 1.03   # profiles/huff_kernel_product_llama7b_layer.md: 146.9 MB moved for 142.1 MB (gate+up), 71.9 for 71.0 (down)
+NCU_TRAFFIC_RATIO = 1.03   # profiles/huff_kernel_product_llama7b_layer.md: 147.0 MB moved for 142.1 MB (gate+up), 72.4 for 71.0 (down)
 
 
 def max_over_ranks(v: float, dist, device) -> float:
