@@ -95,6 +95,8 @@ typedef struct huffllm_codebook huffllm_codebook;
  * the lane's weights form eight pairs (row g: columns (0,1) (2,3) (4,5) (6,7) of its eight, then row g + 8 likewise);
  * bit p is the sign of the first weight of pair p, bit 8 + p the sign of its second weight.  W is the
  * longest sequence of the chunk in words (all 64 are padded to it).
+ * Behind the last record the blob holds 4096 zero bytes (part of blob_bytes): the product kernels ask the cache for
+ * bytes up to 2 KB past the record they work on, and with this slack such a request never leaves the blob.
  */
 typedef struct huffllm_desc {
     char     magic[4];        /* "HFLM"                                                    */
@@ -116,7 +118,7 @@ typedef struct huffllm_desc {
     uint32_t max_words;       /* largest W over all chunks                                 */
     uint64_t off_codebook, off_lut, off_index, off_payload;   /* byte offsets in the blob */
     uint64_t payload_bytes;   /* 128 * index[n_chunks]                                     */
-    uint64_t blob_bytes;      /* total size: what the device kernels stream from HBM       */
+    uint64_t blob_bytes;      /* total size: off_payload + payload_bytes + 4096 zero bytes  */
     uint64_t coded_bits;      /* sum of codeword lengths over all stored weights           */
     uint64_t raw_bits;        /* raw bits of the rows*cols real weights                    */
     uint64_t payload_checksum;/* sum over chunks of (2 id + 1) * FNV-1a-64(record bytes)   */

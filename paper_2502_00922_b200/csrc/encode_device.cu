@@ -333,11 +333,12 @@ extern "C" huffllm_status huffllm_encode_device(const huffllm_codebook *cb, cons
     if (tot.bad & 2u) return fail(HUFFLLM_ERR_UNSUPPORTED, "payload exceeds the 32-bit record index");
     d.max_words = tot.max_words;
     d.payload_bytes = tot.payload_units * kRecordUnit;
-    d.blob_bytes = d.off_payload + d.payload_bytes;
+    d.blob_bytes = d.off_payload + d.payload_bytes + kTailSlack;
     d.coded_bits = tot.coded_bits;
     if (blob_cap < d.blob_bytes)
         return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "blob needs %llu bytes, capacity is %llu", (unsigned long long)d.blob_bytes, (unsigned long long)blob_cap);
 
+    if ((e = cudaMemsetAsync((uint8_t *)blob + d.off_payload + d.payload_bytes, 0, kTailSlack, s)) != cudaSuccess) return cuda_fail("clearing the tail");
     encode_write_kernel<<<grid, kEncThreads, 0, s>>>(A);
     encode_checksum_kernel<<<(uint32_t)((d.n_chunks + 127) / 128), 128, 0, s>>>(A);
     if ((e = cudaGetLastError()) != cudaSuccess) return cuda_fail("encode write pass");

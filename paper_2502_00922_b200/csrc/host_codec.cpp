@@ -59,7 +59,7 @@ huffllm_status check_desc(const huffllm_desc *d) {
     if (d->off_codebook % 256 || d->off_lut % 256 || d->off_index % 256 || d->off_payload % 256 ||
         d->off_codebook < 256 || d->off_lut < d->off_codebook + (d->n_fields == 1 ? 256u : 96u) ||
         d->off_index < d->off_lut + (d->dtype == HUFFLLM_FP16 ? 3 : 1) * (4ull << d->lut_bits) || d->off_payload < d->off_index + 4 * (d->n_chunks + 1) ||
-        d->payload_bytes % kRecordUnit || d->blob_bytes < d->off_payload + d->payload_bytes ||
+        d->payload_bytes % kRecordUnit || d->blob_bytes < d->off_payload + d->payload_bytes + kTailSlack ||
         d->payload_bytes / kRecordUnit > 0xFFFFFFFFull)
         return fail(HUFFLLM_ERR_CORRUPT, "bad section offsets");
     return HUFFLLM_OK;
@@ -526,7 +526,7 @@ huffllm_status huffllm_encode_bound(uint64_t rows, uint64_t cols, huffllm_dtype 
         payload += (uint64_t)g.RG * (raw_part_bytes(dtype, nkb) + w * 256ull);
     }
     uint64_t n_chunks = (uint64_t)g.RG * g.KC;
-    *max_bytes = (size_t)(256 + 256 + align_up(fields * (4ull << kMaxBudget), 256) + align_up(4 * (n_chunks + 1), 256) + payload + 256);
+    *max_bytes = (size_t)(256 + 256 + align_up(fields * (4ull << kMaxBudget), 256) + align_up(4 * (n_chunks + 1), 256) + payload + 256 + kTailSlack);
     return HUFFLLM_OK;
 }
 
@@ -587,7 +587,7 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
     }
     d.max_words = max_words;
     d.payload_bytes = rec[n_chunks] * kRecordUnit;
-    d.blob_bytes = d.off_payload + d.payload_bytes;
+    d.blob_bytes = d.off_payload + d.payload_bytes + kTailSlack;
     d.coded_bits = coded_bits;
     d.raw_bits = (fp16 ? 1 : 8) * rows * cols;
     if (rec[n_chunks] > 0xFFFFFFFFull) return fail(HUFFLLM_ERR_UNSUPPORTED, "payload exceeds the 32-bit record index");
@@ -596,6 +596,7 @@ huffllm_status huffllm_encode(const huffllm_codebook *cb, const uint16_t *w, uin
                     (unsigned long long)blob_cap);
 
     memset(base, 0, d.off_payload);
+    memset(base + d.off_payload + d.payload_bytes, 0, kTailSlack);
     write_fixed_sections(cb, d, base);
     uint32_t *index = (uint32_t *)(base + d.off_index);
     for (uint64_t c = 0; c <= n_chunks; ++c) index[c] = (uint32_t)rec[c];

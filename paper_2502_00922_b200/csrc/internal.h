@@ -19,6 +19,9 @@ constexpr uint32_t kSeqs = 64;          // bit sequences per chunk: two per lane
 constexpr uint32_t kDefaultBudget = 8;  // default joint code-length bound
 constexpr uint32_t kMinBudget = 8, kMaxBudget = 12;
 constexpr uint32_t kRecordUnit = 128;   // record offsets are counted in this many bytes
+// Zero bytes behind the payload, part of the blob: the product kernel's requests into L2 run up to 2 KB past the record
+// they are issued in, and with this slack they never leave the blob.
+constexpr uint64_t kTailSlack = 4096;
 
 huffllm_status fail(huffllm_status st, const char *fmt, ...);
 void clear_error();

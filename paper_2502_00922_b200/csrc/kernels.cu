@@ -352,15 +352,15 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                     // DRAM).  In a record's first half that is the raw part of its second half; in the second half it is the
                     // coded part and, at its end, the start of the next record.  Measured: this plain form is the fastest;
                     // asking only for raw bytes, or for the next record's first blocks, gains a third of it or nothing.
-                    // Not done where it could reach past the payload (the last records).
+                    // The request ends at most 2 KB behind the record it is issued in: inside the blob, whose format keeps 4 KB of
+                    // zero bytes behind the payload for this.
                     // (products of BF16 blobs only: the decode-only kernel has no register to spare for it, and an FP16 record's
                     // raw part is a sixteenth of its bytes)
                     constexpr bool kPrefetchRaw = MODE == 1 && FMT == 0;
-                    const bool pf_safe = r1 + 4u * kRawBlock / 128u <= k.payload_units;
                     auto block = [&](uint32_t kb, const uint4 &cur, uint4 &nxt, auto may_be_last) {
                         BLOCKSTAMP((c - c_beg) * 8 + kb, 0);
                         raw_p += kRawBlock;
-                        if (kPrefetchRaw && pf_safe) asm volatile("prefetch.global.L2 [%0];" ::"l"(raw_p + 3u * kRawBlock));
+                        if (kPrefetchRaw) asm volatile("prefetch.global.L2 [%0];" ::"l"(raw_p + 3u * kRawBlock));
                         if (decltype(may_be_last)::value) {
                             if (kb == last) raw_p += coded_bytes;       // the next record's first block
                             if (kb != last || next_ok) nxt = load_raw(raw_p);
