@@ -114,6 +114,16 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append(line.strip())
 
+    def wait_first(self, limit_s: float):
+        """Wait until the sampler has delivered its first line (or the limit has passed)."""
+        t0 = time.time()
+        while self.proc and not self.lines and time.time() - t0 < limit_s:
+            time.sleep(0.02)
+
+    def mark(self):
+        """Only samples that arrive after this call count (if any do)."""
+        self.first = len(self.lines)
+
     def stop(self):
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
@@ -124,7 +134,8 @@ class ClockSampler:
             self.proc.kill()
         sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        first = getattr(self, "first", 0)
+        for ln in (self.lines[first:] if len(self.lines) > first else self.lines):
             f = [x.strip() for x in ln.split(",")]
             if len(f) < 7:
                 continue
@@ -343,9 +354,10 @@ def main():
     sampler = ClockSampler(uuid if uuid.startswith("GPU-") or uuid.isdigit() else "GPU-" + uuid)
     barrier()
     sampler.start()
-    time.sleep(0.3)                       # let the sampler come up before the timed region starts
+    sampler.wait_first(3.0)               # let the sampler come up before the timed region starts
     t_beg, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     barrier()
+    sampler.mark()                        # samples from here on were taken under load
     t_beg.record(stream)
     for s in range(args.steps):
         step_device()
