@@ -174,6 +174,9 @@ def prepare(workload: str, chunk_elems: int, hl, torch, dev, cpu_sample_mats: in
                          blob_bytes=int(desc.blob_bytes), w_sample=w.copy() if i < cpu_sample_mats else None,
                          x_np=x[:1] if i < cpu_sample_mats else None))
         del w
+    ws_each = max(m["ws_bytes"] for m in mats)       # a multi-matrix call states one size that every workspace must have
+    for m in mats:
+        m["ws"], m["ws_bytes"] = torch.zeros(ws_each, dtype=torch.uint8, device=dev), ws_each
     # activations and results of the whole step live in one host buffer and one device buffer each (the matrices'
     # tensors are views), so that a step's inputs go in with one copy and its results come out with one
     nx, ny = sum(m["x_dev"].numel() for m in mats), sum(m["y_dev"].numel() for m in mats)
@@ -309,7 +312,7 @@ def main():
                   ys=[mats[i]["y_dev"] for i in g], wss=[mats[i]["ws"] for i in g]) for blobs in layer_blobs for g in groups]
     groups = groups * L              # one entry per launch of the step
 
-    ws_each = min(m["ws_bytes"] for m in mats)
+    ws_each = max(m["ws_bytes"] for m in mats)
     raw_stream = stream.cuda_stream
     for c, g in zip(calls, groups):      # argument arrays marshalled once per launch group
         c["prep"] = hl.PreparedMulti(c["descs"], c["blobs"], c["xs"], min(B, 8), c["ys"], c["wss"], ws_each, err,
@@ -471,9 +474,14 @@ def main():
             dense = [(torch.randint(-2**15, 2**15, (m["rows"], m["cols"]), dtype=torch.int16, device=dev), m) for _ in range(L) for m in mats]
             for w_dev, m in dense:
                 w_dev.view(torch.bfloat16).normal_(0, 0.02)
+            # the dense layer in the same launch groups as the compressed one
+            n_g = len(groups) // L
+            dense_preps = [hl.PreparedPlainMulti([dense[l * len(mats) + i][0] for i in g], [mats[i]["rows"] for i in g],
+                                                 [mats[i]["cols"] for i in g], [mats[i]["x_dev"] for i in g],
+                                                 [mats[i]["y_dev"] for i in g]) for l in range(L) for g in groups[:n_g]]
             def plain():
-                for w_dev, m in dense:
-                    hl.plain_gemv(w_dev, m["rows"], m["cols"], m["x_dev"], m["y_dev"], stream)     # one vector: the batch-1 cost
+                for p in dense_preps:
+                    p.run(raw_stream)
             def cublas():
                 for w_dev, m in dense:
                     torch.mv(w_dev.view(torch.bfloat16), m["x_dev"][:m["cols"]].view(torch.bfloat16))

@@ -15,6 +15,12 @@
  *     (create with huffllm_build_codebook, release with huffllm_codebook_free).
  *   - Weights are row-major [rows = out_features][cols = in_features], as 16-bit patterns.
  *   - Device calls are asynchronous on `stream`, never synchronise, never allocate.
+ *   - The decode and product kernels are launched so that their set-up may overlap the tail of the kernel in
+ *     front of them on the stream: they read the BLOB (table, record index, first records) before that kernel
+ *     has finished, and everything else (x, workspace, y, out) only after it has.  A blob must therefore be
+ *     complete in device memory before the kernel that precedes the call on the stream starts; a blob written
+ *     by that very kernel (a device-side copy or encoder right in front of the call) needs a stream
+ *     synchronisation or an event in between.
  *   - Every call returns a huffllm_status; huffllm_last_error() gives a thread-local message.
  *     Nothing aborts, throws, or traps on the device.
  */
@@ -208,12 +214,14 @@ huffllm_status huffllm_validate_blob(const void *blob_host, size_t bytes, huffll
 /* --------------------------------------------------------- device: decode, and decode fused with products */
 
 /*
- * Scratch bytes the fused products need for `batch` activation vectors.  The workspace must be
- * zero-filled once after allocation; its first 4096 bytes are control words that every call
- * leaves zero again, the rest is overwritten freely.  Calls that share a workspace must not
- * overlap on the GPU.
+ * Scratch bytes the fused products need for this matrix and `batch` activation vectors.  The workspace must be
+ * zero-filled once after allocation.  Its first huffllm_workspace_control_bytes(desc) bytes are arrival counters:
+ * every call that completes leaves them zero again; the rest holds partial sums and is overwritten freely.
+ * After a call that set the error flag, clear those leading bytes before the workspace is used again.
+ * Calls that share a workspace must not overlap on the GPU.
  */
 huffllm_status huffllm_workspace_bytes(const huffllm_desc *desc, uint32_t batch, size_t *bytes);
+huffllm_status huffllm_workspace_control_bytes(const huffllm_desc *desc, size_t *bytes);
 
 /*
  * Decompress a blob (device, 256-byte aligned) to its original 16-bit weights, bit for bit
@@ -249,9 +257,9 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob_de
  * Several products in ONE launch: y_i = W_i x_i for i < n (n <= 8, batch <= 8), e.g. the q, k and v
  * projections of a decoder layer, or gate and up.  The chunks of all matrices are spread over the GPU
  * together, so small matrices do not pay a launch, a set-up and a tail each.  Arrays are host arrays
- * of n pointers; every matrix needs its own workspace (each workspace_bytes_each long, as reported by
- * huffllm_workspace_bytes), its own x_i ([batch][cols_i]) and y_i ([batch][rows_i]).  All blobs must
- * have been encoded with the same max_code_len.
+ * of n pointers; every matrix needs its own workspace (each at least workspace_bytes_each long, which must
+ * cover huffllm_workspace_bytes of every matrix of the call), its own x_i ([batch][cols_i]) and y_i
+ * ([batch][rows_i]).  All blobs must have been encoded with the same max_code_len.
  */
 huffllm_status huffllm_decode_gemm_multi(uint32_t n, const huffllm_desc *const *descs, const void *const *blobs_dev,
                                          const uint16_t *const *xs_dev, uint32_t batch, float *const *ys_dev,
@@ -300,25 +308,32 @@ huffllm_status huffllm_decode_gemm_multi_host_async(uint32_t n, const huffllm_de
  * holds until the process exits.
  *
  * Inputs and outputs are the caller's, exactly as in huffllm_decode_gemm; batch may be at most
- * HUFFLLM_STATIC_MAX_BATCH — a larger batch is refused with HUFFLLM_ERR_BUFFER_TOO_SMALL and nothing
- * is launched.  The first call on each device looks up the array's device address (with that device
+ * HUFFLLM_STATIC_MAX_BATCH, and huffllm_workspace_bytes(desc, batch) at most HUFFLLM_STATIC_SCRATCH_BYTES
+ * (true for any matrix of up to about half a million rows) — anything larger is refused with
+ * HUFFLLM_ERR_BUFFER_TOO_SMALL.  A call that is refused, for this or any other reason, enqueues nothing and
+ * leaves the array untouched.  The first call on each device looks up the array's device address (with that device
  * current) and remembers it; make that first call outside any stream capture.  Every call clears
  * the scratch's control words on `stream` before the kernel runs, so a call never depends on what an
  * earlier call left behind.  All calls on one GPU share the one array: two calls that can overlap on
  * the GPU (different streams without an ordering between them) race on it and give wrong sums.
  */
 #define HUFFLLM_STATIC_MAX_BATCH 8u
-#define HUFFLLM_STATIC_SCRATCH_BYTES (4096u + 512u * 2u * 16u * HUFFLLM_STATIC_MAX_BATCH * 4u)
+#define HUFFLLM_STATIC_SCRATCH_BYTES (1u << 20)
 huffllm_status huffllm_decode_gemm_static(const huffllm_desc *desc, const void *blob_dev, const uint16_t *x_dev,
                                           uint32_t batch, float *y_dev, int32_t *err_flag_dev, huffllm_stream stream);
 
 /*
  * Reference point for the compressed path: y = W x for an UNCOMPRESSED bf16 matrix (device,
- * row-major, 16-byte aligned rows, cols a multiple of 8), same fp32 accumulation.  This is the
- * dense product whose memory traffic the compression removes (Section 6).
+ * row-major, 16-byte aligned rows, cols a multiple of 8), same fp32 accumulation, written as a
+ * streaming kernel (many independent 16-byte loads in flight per lane).  This is the dense product
+ * whose memory traffic the compression removes (Section 6: compression pays while weight movement
+ * binds).  huffllm_plain_gemv_multi runs up to 8 such products (host arrays of n pointers / sizes)
+ * in one launch, so that the dense layer can be timed in the same launch groups as the compressed one.
  */
 huffllm_status huffllm_plain_gemv(const uint16_t *w_dev, uint64_t rows, uint64_t cols, const uint16_t *x_dev,
                                   float *y_dev, huffllm_stream stream);
+huffllm_status huffllm_plain_gemv_multi(uint32_t n, const uint16_t *const *ws_dev, const uint64_t *rows, const uint64_t *cols,
+                                        const uint16_t *const *xs_dev, float *const *ys_dev, huffllm_stream stream);
 
 /*
  * Bit-field split explorer (Section 3.1, entropy table): what would it cost, in bits per parameter, to cut the

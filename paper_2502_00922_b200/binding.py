@@ -46,6 +46,7 @@ _SIGNATURES = {
     "huffllm_encode": [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint32, C.c_void_p, C.c_size_t, C.POINTER(Desc)],
     "huffllm_validate_blob": [C.c_void_p, C.c_size_t, C.POINTER(Desc)],
     "huffllm_workspace_bytes": [C.POINTER(Desc), C.c_uint32, C.POINTER(C.c_size_t)],
+    "huffllm_workspace_control_bytes": [C.POINTER(Desc), C.POINTER(C.c_size_t)],
     "huffllm_decode": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemv": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemm": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
@@ -60,6 +61,7 @@ _SIGNATURES = {
     "huffllm_decode_gemm_static": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p],
     "huffllm_stage_copy": [C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p],
     "huffllm_plain_gemv": [C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p, C.c_void_p, C.c_void_p],
+    "huffllm_plain_gemv_multi": [C.c_uint32, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
     "huffllm_build_codebook_from_counts": [C.c_void_p, C.c_int, C.c_int, C.c_uint32, C.POINTER(C.c_void_p)],
     "huffllm_encode_device_scratch_bytes": [C.c_uint64, C.c_uint64, C.c_uint32, C.POINTER(C.c_size_t)],
     "huffllm_encode_device": [C.c_void_p, C.c_void_p, C.c_uint64, C.c_uint64, C.c_uint32, C.c_void_p, C.c_size_t, C.c_void_p, C.c_size_t,
@@ -196,6 +198,13 @@ def workspace_bytes(desc: Desc, batch: int = 1) -> int:
     return n.value
 
 
+def workspace_control_bytes(desc: Desc) -> int:
+    """huffllm_workspace_control_bytes: the leading bytes of a workspace that are zero between calls."""
+    n = C.c_size_t()
+    _check(lib().huffllm_workspace_control_bytes(C.byref(desc), C.byref(n)))
+    return n.value
+
+
 def decode(desc: Desc, blob_dev, out_dev, err_flag_dev=None, stream=None):
     _check(lib().huffllm_decode(C.byref(desc), _ptr(blob_dev), _ptr(out_dev), _ptr(err_flag_dev), _stream(stream)))
 
@@ -289,6 +298,28 @@ def decode_gemm_static(desc: Desc, blob_dev, x_dev, batch: int, y_dev, err_flag_
 
 def plain_gemv(w_dev, rows: int, cols: int, x_dev, y_dev, stream=None):
     _check(lib().huffllm_plain_gemv(_ptr(w_dev), rows, cols, _ptr(x_dev), _ptr(y_dev), _stream(stream)))
+
+
+class PreparedPlainMulti:
+    """The argument arrays of a huffllm_plain_gemv_multi call, marshalled once (the tensors must stay alive and in place)."""
+
+    def __init__(self, ws_dev, rows, cols, xs_dev, ys_dev):
+        n = self.n = len(ws_dev)
+        self._keep = (ws_dev, xs_dev, ys_dev)
+        ptrs = lambda seq: (C.c_void_p * n)(*[_ptr(t) for t in seq])
+        self.ws, self.xs, self.ys = ptrs(ws_dev), ptrs(xs_dev), ptrs(ys_dev)
+        self.rows, self.cols = (C.c_uint64 * n)(*rows), (C.c_uint64 * n)(*cols)
+        self._fn = lib().huffllm_plain_gemv_multi
+
+    def run(self, stream: int):
+        st = self._fn(self.n, self.ws, self.rows, self.cols, self.xs, self.ys, stream)
+        if st:
+            _check(st)
+
+
+def plain_gemv_multi(ws_dev, rows, cols, xs_dev, ys_dev, stream=None):
+    """huffllm_plain_gemv_multi: several dense bf16 products in one launch (lists of equal length)."""
+    PreparedPlainMulti(ws_dev, rows, cols, xs_dev, ys_dev).run(_stream(stream))
 
 
 def _widths(widths) -> np.ndarray:

@@ -26,12 +26,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-I" + INCLUDE, "-shared", "-Xcompiler", "-fPIC", "-o", SO] + [os.path.join(CSRC, s) for s in SOURCES]
     cmd += ["-lpthread"]
-    if os.environ.get("HUFFLLM_TIMING"):           # experiment knob: per-warp phase stamps
-        cmd.insert(1, "-DHUFFLLM_TIMING")
-    if os.environ.get("HUFFLLM_THREADS"):          # experiment knob: threads per CTA of the decode kernels
-        cmd.insert(1, "-DHUFFLLM_THREADS=" + os.environ["HUFFLLM_THREADS"])
-    for d in os.environ.get("HUFFLLM_DEFS", "").split():   # experiment knob: extra -D definitions
-        cmd.insert(1, "-D" + d)
     if verbose:
         cmd.insert(1, "-Xptxas=-v")
     subprocess.check_call(cmd)

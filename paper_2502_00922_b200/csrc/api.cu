@@ -2,6 +2,7 @@
 // No allocation and no synchronisation here (huffllm_decode_gemm_host, which exists to be timed
 // end to end with host buffers, is the one call that waits for its stream).
 #include <cuda_runtime.h>
+#include <atomic>
 #include <cstdlib>
 #include <cstring>
 
@@ -16,33 +17,50 @@ constexpr uint32_t kMaxGrid = 512;        // CTAs the scratch layout provides fo
 constexpr uint32_t kKernelBatch = 8;      // activation vectors one launch multiplies
 constexpr uint32_t kStaticSmem = 2048;    // barriers and tables the kernel declares statically (rounded up)
 
+// Per-device facts, looked up once.  Threads may race to fill an entry: they write the same values, and `known` is
+// published last.
+struct DeviceSlot {
+    std::atomic<bool> known{false};
+    std::atomic<int> sms{0}, smem_optin{0};
+};
+DeviceSlot g_dev[64];
 struct DeviceInfo {
-    bool known = false;
     int sms = 0, smem_optin = 0;
 };
-DeviceInfo g_dev[64];
 
-huffllm_status device_info(DeviceInfo **out) {
+huffllm_status device_info(DeviceInfo *out) {
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
     if (dev < 0 || dev >= 64) return fail(HUFFLLM_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
-    DeviceInfo &d = g_dev[dev];
-    if (!d.known) {
-        if ((e = cudaDeviceGetAttribute(&d.sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess ||
-            (e = cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess)
+    DeviceSlot &d = g_dev[dev];
+    if (!d.known.load(std::memory_order_acquire)) {
+        int sms = 0, smem = 0;
+        if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess ||
+            (e = cudaDeviceGetAttribute(&smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev)) != cudaSuccess)
             return fail(HUFFLLM_ERR_CUDA, "cudaDeviceGetAttribute: %s", cudaGetErrorString(e));
-        d.known = true;
+        d.sms.store(sms, std::memory_order_relaxed);
+        d.smem_optin.store(smem, std::memory_order_relaxed);
+        d.known.store(true, std::memory_order_release);
     }
-    *out = &d;
+    out->sms = d.sms.load(std::memory_order_relaxed);
+    out->smem_optin = d.smem_optin.load(std::memory_order_relaxed);
     return HUFFLLM_OK;
 }
 
-// Scratch layout: [0, 4096) arrival counters (one per CTA, zero between calls) | partial sums
-size_t ws_partial_offset() { return 4096; }
-size_t ws_bytes_for(uint32_t batch) {
+// Scratch layout of one matrix's workspace:
+//   [0, 4096)            arrival counters of the register-path kernel (one per CTA)
+//   [4096, partial_off)  arrival counters of the tensor-core kernel, sized for its smallest tile
+//   [partial_off, ...)   partial sums: of the register path's CTAs, or of the tensor-core path's work items
+// Everything in front of partial_off is zero between calls; what lies behind it is overwritten freely by either path.
+size_t ws_ctrl_bytes(const huffllm_desc *) { return 4096; }
+size_t ws_partial_offset(const huffllm_desc *d) {
+    const size_t max_m_tiles = (d->row_groups + 7) / 8;      // tensor-core row tiles at their smallest (128 rows)
+    return ws_ctrl_bytes(d) + (max_m_tiles * 32 * 4 + 255) / 256 * 256;
+}
+size_t ws_bytes_for(const huffllm_desc *d, uint32_t batch) {
     uint32_t b = batch < kKernelBatch ? batch : kKernelBatch;
-    return ws_partial_offset() + (size_t)kMaxGrid * 2 * 16 * b * sizeof(float);
+    return ws_partial_offset(d) + (size_t)kMaxGrid * 2 * 16 * b * sizeof(float);
 }
 
 // Geometry of the tensor-core small-batch path (batch 9..64): row tiles of 512 rows, column chunks cut into
@@ -89,11 +107,10 @@ TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn
     }
     p.ksplit = best;
     p.items = p.m_tiles * best;
-    p.ticket_off = ws_bytes_for(kKernelBatch);      // behind everything the register-path kernels may write
     // the counters' region is sized for the smallest tile (most row tiles), so that plans for different batch sizes
     // sharing one workspace never put partial sums where another plan keeps counters
-    const size_t max_m_tiles = (d->row_groups + 7) / 8;
-    p.partial_off = p.ticket_off + ((max_m_tiles * 32 * 4 + 255) / 256) * 256;
+    p.ticket_off = ws_ctrl_bytes(d);
+    p.partial_off = ws_partial_offset(d);
     p.bytes = p.partial_off + (best > 1 ? (size_t)p.items * 32 * (p.npad / 2) * 32 * sizeof(float) : 0);
     return p;
 }
@@ -191,30 +208,39 @@ huffllm_status huffllm_workspace_bytes(const huffllm_desc *desc, uint32_t batch,
     huffllm_status st = check_desc(desc);
     if (st != HUFFLLM_OK) return st;
     if (batch == 0 || batch > 64) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be in [1, 64]");
-    *bytes = ws_bytes_for(batch);
+    *bytes = ws_bytes_for(desc, batch);     // (above 8 vectors: what passes of 8 need, should the tensor-core kernel not fit)
     if (batch > kKernelBatch) {      // the tensor-core path keeps partial tiles of its column ranges here
-        DeviceInfo *dev;
-        int sms = device_info(&dev) == HUFFLLM_OK ? dev->sms : 148;
+        DeviceInfo dev;       // without a device (a host-only caller sizing buffers): the B200's figures
+        const bool have = device_info(&dev) == HUFFLLM_OK;
         clear_error();
-        uint32_t dyn = device_info(&dev) == HUFFLLM_OK ? (uint32_t)dev->smem_optin - kStaticSmem : 232448u - kStaticSmem;
-        clear_error();
+        const int sms = have ? dev.sms : 148;
+        const uint32_t dyn = (have ? (uint32_t)dev.smem_optin : 232448u) - kStaticSmem;
         size_t tc = tc_plan(desc, batch, (uint32_t)sms, dyn).bytes;
         if (tc > *bytes) *bytes = tc;
     }
     return HUFFLLM_OK;
 }
 
+huffllm_status huffllm_workspace_control_bytes(const huffllm_desc *desc, size_t *bytes) {
+    clear_error();
+    if (!bytes) return fail(HUFFLLM_ERR_INVALID_ARG, "bytes is null");
+    huffllm_status st = check_desc(desc);
+    if (st != HUFFLLM_OK) return st;
+    *bytes = ws_partial_offset(desc);
+    return HUFFLLM_OK;
+}
+
 huffllm_status huffllm_decode(const huffllm_desc *desc, const void *blob, uint16_t *out, int32_t *err_flag, huffllm_stream stream) {
     clear_error();
-    DeviceInfo *dev;
+    DeviceInfo dev;
     huffllm_status st = device_info(&dev);
     if (st != HUFFLLM_OK) return st;
     if (!out || ((uintptr_t)out & 15)) return fail(HUFFLLM_ERR_INVALID_ARG, "out must be a 16-byte aligned device pointer");
     KernelArgs k;
     uint32_t grid;
-    begin_args(&k, 1, *dev);
+    begin_args(&k, 1, dev);
     if ((st = add_matrix(&k, desc, blob)) != HUFFLLM_OK) return st;
-    if ((st = finish_args(&k, false, *dev, &grid)) != HUFFLLM_OK) return st;
+    if ((st = finish_args(&k, false, dev, &grid)) != HUFFLLM_OK) return st;
     k.m[0].out = out;
     k.err = err_flag;
     cudaError_t e = launch_decode(k, grid, (cudaStream_t)stream);
@@ -228,9 +254,9 @@ static huffllm_status check_product_args(const huffllm_desc *desc, const uint16_
     if (!x || !y || !workspace) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
     if (((uintptr_t)x & 15) || ((uintptr_t)y & 3) || ((uintptr_t)workspace & 255))
         return fail(HUFFLLM_ERR_INVALID_ARG, "x must be 16-byte, y 4-byte, workspace 256-byte aligned");
-    if (workspace_bytes < ws_bytes_for(batch)) return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "workspace too small");
     huffllm_status st = check_desc(desc);
     if (st != HUFFLLM_OK) return st;
+    if (workspace_bytes < ws_bytes_for(desc, batch)) return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "workspace too small");
     if (desc->cols % kBlockCols) return fail(HUFFLLM_ERR_UNSUPPORTED, "fused products need cols to be a multiple of 32");
     return HUFFLLM_OK;
 }
@@ -239,7 +265,7 @@ huffllm_status huffllm_decode_gemm_multi(uint32_t n, const huffllm_desc *const *
                                          const uint16_t *const *xs, uint32_t batch, float *const *ys, void *const *workspaces,
                                          size_t workspace_bytes_each, int32_t *err_flag, huffllm_stream stream) {
     clear_error();
-    DeviceInfo *dev;
+    DeviceInfo dev;
     huffllm_status st = device_info(&dev);
     if (st != HUFFLLM_OK) return st;
     if (!descs || !blobs || !xs || !ys || !workspaces) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
@@ -247,7 +273,7 @@ huffllm_status huffllm_decode_gemm_multi(uint32_t n, const huffllm_desc *const *
     if (batch == 0 || batch > kKernelBatch) return fail(HUFFLLM_ERR_UNSUPPORTED, "batch must be in [1, %u] here", kKernelBatch);
     KernelArgs k;
     uint32_t grid;
-    begin_args(&k, batch, *dev);
+    begin_args(&k, batch, dev);
     for (uint32_t i = 0; i < n; ++i) {
         if ((st = check_product_args(descs[i], xs[i], ys[i], workspaces[i], workspace_bytes_each, batch)) != HUFFLLM_OK) return st;
         for (uint32_t j = 0; j < i; ++j)
@@ -257,9 +283,9 @@ huffllm_status huffllm_decode_gemm_multi(uint32_t n, const huffllm_desc *const *
         m.x = xs[i];
         m.y = ys[i];
         m.ws_ticket = (unsigned int *)workspaces[i];
-        m.ws_partial = (float *)((uint8_t *)workspaces[i] + ws_partial_offset());
+        m.ws_partial = (float *)((uint8_t *)workspaces[i] + ws_partial_offset(descs[i]));
     }
-    if ((st = finish_args(&k, true, *dev, &grid)) != HUFFLLM_OK) return st;
+    if ((st = finish_args(&k, true, dev, &grid)) != HUFFLLM_OK) return st;
     k.err = err_flag;
     cudaError_t e = launch_gemm(k, grid, (cudaStream_t)stream);
     if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "product launch: %s", cudaGetErrorString(e));
@@ -269,17 +295,17 @@ huffllm_status huffllm_decode_gemm_multi(uint32_t n, const huffllm_desc *const *
 huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, const uint16_t *x, uint32_t batch, float *y,
                                    void *workspace, size_t workspace_bytes, int32_t *err_flag, huffllm_stream stream) {
     clear_error();
-    DeviceInfo *dev;
+    DeviceInfo dev;
     huffllm_status st = device_info(&dev);
     if (st != HUFFLLM_OK) return st;
     if (batch == 0 || batch > 64) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be in [1, 64]");
     if ((st = check_product_args(desc, x, y, workspace, workspace_bytes, batch)) != HUFFLLM_OK) return st;
     if (batch > kKernelBatch) {
         // tensor-core path: one pass over the compressed weights for the whole batch
-        const TcPlan tp = tc_plan(desc, batch, (uint32_t)dev->sms, (uint32_t)dev->smem_optin - kStaticSmem);
+        const TcPlan tp = tc_plan(desc, batch, (uint32_t)dev.sms, (uint32_t)dev.smem_optin - kStaticSmem);
         KernelArgs k;
         uint32_t grid;
-        begin_args(&k, batch, *dev);
+        begin_args(&k, batch, dev);
         if ((st = add_matrix(&k, desc, blob)) != HUFFLLM_OK) return st;
         k.part_bytes = tc_stages(tp.npad) * tp.npad * 64;      // the stages of activations
         const uint64_t need = tc_smem_need(desc, tp.npad, tp.tiles);
@@ -293,7 +319,7 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
             k.tc_ticket = (unsigned int *)((uint8_t *)workspace + tp.ticket_off);
             k.tc_partial = (float *)((uint8_t *)workspace + tp.partial_off);
             k.err = err_flag;
-            grid = tp.items < (uint32_t)dev->sms ? tp.items : (uint32_t)dev->sms;
+            grid = tp.items < (uint32_t)dev.sms ? tp.items : (uint32_t)dev.sms;
             cudaError_t e = launch_gemm_tc(k, grid, (cudaStream_t)stream);
             if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "tensor-core product launch: %s", cudaGetErrorString(e));
             return HUFFLLM_OK;
@@ -305,13 +331,13 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
         uint32_t nb = batch - b0 < kKernelBatch ? batch - b0 : kKernelBatch;
         KernelArgs k;
         uint32_t grid;
-        begin_args(&k, nb, *dev);
+        begin_args(&k, nb, dev);
         if ((st = add_matrix(&k, desc, blob)) != HUFFLLM_OK) return st;
-        if ((st = finish_args(&k, true, *dev, &grid)) != HUFFLLM_OK) return st;
+        if ((st = finish_args(&k, true, dev, &grid)) != HUFFLLM_OK) return st;
         k.m[0].x = x + (uint64_t)b0 * desc->cols;
         k.m[0].y = y + (uint64_t)b0 * desc->rows;
         k.m[0].ws_ticket = (unsigned int *)workspace;
-        k.m[0].ws_partial = (float *)((uint8_t *)workspace + ws_partial_offset());
+        k.m[0].ws_partial = (float *)((uint8_t *)workspace + ws_partial_offset(desc));
         k.err = err_flag;
         cudaError_t e = launch_gemm(k, grid, (cudaStream_t)stream);
         if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "product launch: %s", cudaGetErrorString(e));
@@ -331,9 +357,14 @@ huffllm_status huffllm_decode_gemm_multi_host_async(uint32_t n, const huffllm_de
     clear_error();
     if (!descs || !xs_host || !ys_host || !x_stages || !y_stages) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
     if (n == 0 || n > kMaxMats) return fail(HUFFLLM_ERR_INVALID_ARG, "between 1 and %u matrices per call", kMaxMats);
+    if (batch == 0 || batch > kKernelBatch) return fail(HUFFLLM_ERR_UNSUPPORTED, "batch must be in [1, %u] here", kKernelBatch);
     cudaStream_t s = (cudaStream_t)stream;
-    for (uint32_t i = 0; i < n; ++i) {
+    for (uint32_t i = 0; i < n; ++i) {     // nothing is enqueued before every argument has been looked at
         if (!descs[i] || !xs_host[i] || !ys_host[i] || !x_stages[i] || !y_stages[i]) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
+        huffllm_status st = check_desc(descs[i]);
+        if (st != HUFFLLM_OK) return st;
+    }
+    for (uint32_t i = 0; i < n; ++i) {
         cudaError_t e = cudaMemcpyAsync(x_stages[i], xs_host[i], (size_t)batch * descs[i]->cols * 2, cudaMemcpyHostToDevice, s);
         if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "copy of x: %s", cudaGetErrorString(e));
     }
@@ -364,6 +395,9 @@ huffllm_status huffllm_decode_gemm_host(const huffllm_desc *desc, const void *bl
                                         size_t workspace_bytes, int32_t *err_flag, huffllm_stream stream) {
     clear_error();
     if (!desc || !x_host || !y_host || !x_stage || !y_stage) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
+    if (batch == 0 || batch > 64) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be in [1, 64]");
+    huffllm_status st0 = check_product_args(desc, x_stage, y_stage, workspace, workspace_bytes, batch);
+    if (st0 != HUFFLLM_OK) return st0;       // nothing is enqueued for a call that will be refused
     cudaStream_t s = (cudaStream_t)stream;
     cudaError_t e = cudaMemcpyAsync(x_stage, x_host, (size_t)batch * desc->cols * 2, cudaMemcpyHostToDevice, s);
     if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "copy of x: %s", cudaGetErrorString(e));
@@ -380,7 +414,7 @@ huffllm_status huffllm_decode_gemm_host(const huffllm_desc *desc, const void *bl
 // Scratch of huffllm_decode_gemm_static.  In host code this name is only a handle for the runtime, not a
 // device address: the address the kernels get comes from cudaGetSymbolAddress, once per device.
 static __device__ __align__(256) unsigned char g_static_scratch[HUFFLLM_STATIC_SCRATCH_BYTES];
-static void *g_static_scratch_addr[64] = {};
+static std::atomic<void *> g_static_scratch_addr[64];
 
 extern "C" {
 
@@ -388,48 +422,84 @@ huffllm_status huffllm_decode_gemm_static(const huffllm_desc *desc, const void *
                                           float *y, int32_t *err_flag, huffllm_stream stream) {
     clear_error();
     if (batch == 0) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be at least 1");
-    if (batch > HUFFLLM_STATIC_MAX_BATCH || ws_bytes_for(batch) > sizeof(g_static_scratch))
-        return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "batch %u needs more than the %u-byte built-in scratch (at most %u vectors)",
-                    batch, (unsigned)HUFFLLM_STATIC_SCRATCH_BYTES, (unsigned)HUFFLLM_STATIC_MAX_BATCH);
+    huffllm_status st = check_desc(desc);
+    if (st != HUFFLLM_OK) return st;
+    if (batch > HUFFLLM_STATIC_MAX_BATCH || ws_bytes_for(desc, batch) > sizeof(g_static_scratch))
+        return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL,
+                    "this matrix with %u vectors needs %zu bytes of scratch; the built-in array has %u (and takes at most %u vectors)",
+                    batch, ws_bytes_for(desc, batch), (unsigned)HUFFLLM_STATIC_SCRATCH_BYTES, (unsigned)HUFFLLM_STATIC_MAX_BATCH);
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "cudaGetDevice: %s", cudaGetErrorString(e));
     if (dev < 0 || dev >= 64) return fail(HUFFLLM_ERR_UNSUPPORTED, "device ordinal %d out of range", dev);
-    if (!g_static_scratch_addr[dev]) {   // set-up, once per device, with that device current
-        void *p = nullptr;
-        e = cudaGetSymbolAddress(&p, g_static_scratch);
-        if (e != cudaSuccess || !p) return fail(HUFFLLM_ERR_CUDA, "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
-        g_static_scratch_addr[dev] = p;
+    void *ws = g_static_scratch_addr[dev].load(std::memory_order_acquire);
+    if (!ws) {   // set-up, once per device, with that device current (racing threads look up the same address)
+        e = cudaGetSymbolAddress(&ws, g_static_scratch);
+        if (e != cudaSuccess || !ws) return fail(HUFFLLM_ERR_CUDA, "cudaGetSymbolAddress: %s", cudaGetErrorString(e));
+        g_static_scratch_addr[dev].store(ws, std::memory_order_release);
     }
-    void *ws = g_static_scratch_addr[dev];
+    // Everything that can refuse the call is checked before anything is enqueued: a refused call leaves the array alone.
+    DeviceInfo info;
+    if ((st = device_info(&info)) != HUFFLLM_OK) return st;
+    if ((st = check_product_args(desc, x, y, ws, sizeof(g_static_scratch), batch)) != HUFFLLM_OK) return st;
+    {
+        KernelArgs k;
+        uint32_t grid;
+        begin_args(&k, batch, info);
+        if ((st = add_matrix(&k, desc, blob)) != HUFFLLM_OK) return st;
+        if ((st = finish_args(&k, true, info, &grid)) != HUFFLLM_OK) return st;
+    }
     // the array keeps whatever the last call (finished or not) left: the control words must start at zero
-    e = cudaMemsetAsync(ws, 0, 4096, (cudaStream_t)stream);
+    e = cudaMemsetAsync(ws, 0, ws_partial_offset(desc), (cudaStream_t)stream);
     if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "clearing the built-in scratch: %s", cudaGetErrorString(e));
     return huffllm_decode_gemm(desc, blob, x, batch, y, ws, sizeof(g_static_scratch), err_flag, stream);
 }
 
 huffllm_status huffllm_stage_copy(void *dst, const void *src, size_t bytes, huffllm_stream stream) {
     clear_error();
-    DeviceInfo *dev;
+    DeviceInfo dev;
     huffllm_status st = device_info(&dev);
     if (st != HUFFLLM_OK) return st;
     if (!dst || !src) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
     if (bytes % 16 || ((uintptr_t)dst & 15) || ((uintptr_t)src & 15)) return fail(HUFFLLM_ERR_INVALID_ARG, "size and pointers must be multiples of 16 bytes");
-    cudaError_t e = launch_stage_copy(dst, src, bytes, (uint32_t)dev->sms, (cudaStream_t)stream);
+    cudaError_t e = launch_stage_copy(dst, src, bytes, (uint32_t)dev.sms, (cudaStream_t)stream);
     if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "copy launch: %s", cudaGetErrorString(e));
     return HUFFLLM_OK;
 }
 
-huffllm_status huffllm_plain_gemv(const uint16_t *w, uint64_t rows, uint64_t cols, const uint16_t *x, float *y, huffllm_stream stream) {
+huffllm_status huffllm_plain_gemv_multi(uint32_t n, const uint16_t *const *ws, const uint64_t *rows, const uint64_t *cols,
+                                        const uint16_t *const *xs, float *const *ys, huffllm_stream stream) {
     clear_error();
-    DeviceInfo *dev;
+    DeviceInfo dev;
     huffllm_status st = device_info(&dev);
     if (st != HUFFLLM_OK) return st;
-    if (!w || !x || !y || rows == 0 || cols == 0) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer or empty matrix");
-    if (cols % 8 || ((uintptr_t)w & 15) || ((uintptr_t)x & 15)) return fail(HUFFLLM_ERR_UNSUPPORTED, "cols must be a multiple of 8 and pointers 16-byte aligned");
-    cudaError_t e = launch_plain_gemv(w, rows, cols, x, y, (uint32_t)dev->sms, (cudaStream_t)stream);
+    if (!ws || !rows || !cols || !xs || !ys) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
+    if (n == 0 || n > kMaxMats) return fail(HUFFLLM_ERR_INVALID_ARG, "between 1 and %u matrices per call", kMaxMats);
+    PlainArgs a;
+    memset(&a, 0, sizeof(a));
+    a.n_mats = n;
+    uint64_t pairs = 0;
+    for (uint32_t i = 0; i < n; ++i) {
+        if (!ws[i] || !xs[i] || !ys[i] || rows[i] == 0 || cols[i] == 0) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer or empty matrix");
+        if (cols[i] % 8 || ((uintptr_t)ws[i] & 15) || ((uintptr_t)xs[i] & 15))
+            return fail(HUFFLLM_ERR_UNSUPPORTED, "cols must be a multiple of 8 and pointers 16-byte aligned");
+        a.m[i].w = ws[i];
+        a.m[i].x = xs[i];
+        a.m[i].y = ys[i];
+        a.m[i].rows = rows[i];
+        a.m[i].cols = cols[i];
+        a.m[i].pair_first = (uint32_t)pairs;
+        pairs += (rows[i] + 1) / 2;
+        if (pairs >= (1ull << 31)) return fail(HUFFLLM_ERR_UNSUPPORTED, "too many rows for one launch");
+    }
+    a.total_pairs = (uint32_t)pairs;
+    cudaError_t e = launch_plain_gemv(a, (uint32_t)dev.sms, (cudaStream_t)stream);
     if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "plain gemv launch: %s", cudaGetErrorString(e));
     return HUFFLLM_OK;
+}
+
+huffllm_status huffllm_plain_gemv(const uint16_t *w, uint64_t rows, uint64_t cols, const uint16_t *x, float *y, huffllm_stream stream) {
+    return huffllm_plain_gemv_multi(1, &w, &rows, &cols, &x, &y, stream);
 }
 
 }  // extern "C"

@@ -338,20 +338,7 @@ __device__ __forceinline__ uint32_t slot_addr(const SmemPlan &p, uint32_t warp, 
 }
 
 constexpr int kMaxWarps = 32;
-// Experiment build only (-DHUFFLLM_TIMING): every warp writes nanosecond stamps of its phases into the
-// buffer passed as the error flag, [cta][warp][8].
-#ifdef HUFFLLM_TIMING
-__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define STAMP(i) do { if (lane == 0) ((unsigned long long *)A.err)[((size_t)blockIdx.x * 32 + warp) * 8 + (i)] = gtime(); } while (0)
-#define BLOCKSTAMP(n, phase) do { if (lane == 0 && blockIdx.x == 3 && (n) < 64) ((unsigned long long *)A.err)[148 * 32 * 8 + (warp * 64 + (n)) * 4 + (phase)] = clock64(); } while (0)
-#else
-#define STAMP(i) do {} while (0)
-#define BLOCKSTAMP(n, phase) do {} while (0)
-#endif
-#ifndef HUFFLLM_THREADS
-#define HUFFLLM_THREADS 1024
-#endif
-constexpr int kThreads = HUFFLLM_THREADS;   // threads per CTA of the decode kernels (one CTA per SM)
+constexpr int kThreads = 1024;   // threads per CTA of the decode kernels (one CTA per SM)
 constexpr uint32_t kWaitLimit = 1u << 22;
 
 }  // namespace huffllm

@@ -25,6 +25,7 @@
 //   * partial sums of a row group that is split over warps or CTAs are combined in a fixed order
 //     (shared memory inside a CTA, a scratch buffer plus a last-CTA pass across CTAs)
 #include <cuda_runtime.h>
+#include <atomic>
 #include <cstdint>
 #include <type_traits>
 
@@ -57,7 +58,6 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     __shared__ uint32_t s_arrive[kMaxWarps];   // arrival counters of row groups shared by several warps
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps_launched = blockDim.x >> 5;
-    STAMP(0);
     pdl_launch_dependents();   // the next kernel's set-up may overlap this kernel's tail
     const uint32_t smem_base = smem_u32(dyn_smem);
     const SmemPlan plan = plan_smem(smem_base, A, nwarps_launched);
@@ -162,9 +162,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
             }
             if (tid < kMaxWarps) s_arrive[tid] = 0;
         }
-        STAMP(1);
         __syncthreads();
-        STAMP(2);
 
         float acc[4] = {0.f, 0.f, 0.f, 0.f};
         int cur_rg = -1;
@@ -295,12 +293,6 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                 const uint32_t kc1 = kc + 1 == KC ? 0u : kc + 1;
                 const uint32_t r2 = has_next ? __ldg(index + c + 2) : r1;
                 const bool next_ok = has_next && record_ok(r1, r2, blocks_of(kc1));
-#ifdef HUFFLLM_PFC
-                // the raw part of the next record (one 128-byte line per lane) is asked into L2 a whole chunk ahead: the
-                // loads that bring it to registers run only one block ahead of the decoder, too short for a DRAM miss
-                if (next_ok && lane * 128u < raw_part(blocks_of(kc1)))
-                    asm volatile("prefetch.global.L2 [%0];" ::"l"(payload + (uint64_t)r1 * 128u + lane * 128u));
-#endif
 
                 if (MODE == 1 && (int)rg != cur_rg) {
                     flush(cur_rg, c_beg, c);  // the previous row group ended with chunk c - 1
@@ -326,7 +318,6 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                 }
 
                 if (!waited_prior) {
-                    STAMP(3);
                     pdl_wait_prior_grid();   // from here on this warp reads x and writes results: the previous kernel must be done
                     waited_prior = true;
                 }
@@ -358,16 +349,13 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                     // raw part is a sixteenth of its bytes)
                     constexpr bool kPrefetchRaw = MODE == 1 && FMT == 0;
                     auto block = [&](uint32_t kb, const uint4 &cur, uint4 &nxt, auto may_be_last) {
-                        BLOCKSTAMP((c - c_beg) * 8 + kb, 0);
                         raw_p += kRawBlock;
                         if (kPrefetchRaw) asm volatile("prefetch.global.L2 [%0];" ::"l"(raw_p + 3u * kRawBlock));
                         if (decltype(may_be_last)::value) {
                             if (kb == last) raw_p += coded_bytes;       // the next record's first block
                             if (kb != last || next_ok) nxt = load_raw(raw_p);
                         } else {
-#ifndef HUFFLLM_NORAW
                             nxt = load_raw(raw_p);
-#endif
                         }
                         uint4 xv;
                         if (MODE == 1) {
@@ -378,7 +366,6 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                         uint32_t a[8];
                         if (FMT) decode_block_fp16(sa, sb, lut_lane, cur.x, a);
                         else decode_block<R, SKIP>(sa, sb, kIdxMask, lut_lane, cur, a);
-                        BLOCKSTAMP((c - c_beg) * 8 + kb, 1);
 
                         if (MODE == 1) {
                             if (FMT) {
@@ -388,7 +375,6 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                                 mma_bf16_16816(acc, a[0], a[4], a[1], a[5], xv.x, xv.y);
                                 mma_bf16_16816(acc, a[2], a[6], a[3], a[7], xv.z, xv.w);
                             }
-                            BLOCKSTAMP((c - c_beg) * 8 + kb, 2);
                         } else {
                             const uint32_t col = col0 + kb * 32u;
 #pragma unroll
@@ -438,36 +424,69 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
             }
             if (MODE == 1 && !failed) flush(cur_rg, c_beg, c_end);
         }
-        STAMP(4);
     }
-    STAMP(7);
 }
 
 // ------------------------------------------------------------------------------ plain bf16 GEMV
 
-// One warp per row, 16-byte loads, fp32 accumulation, shuffle reduction.
-__global__ void __launch_bounds__(256) plain_gemv_kernel(const uint16_t *__restrict__ w, uint64_t rows, uint64_t cols,
-                                                         const uint16_t *__restrict__ x, float *__restrict__ y) {
+// The dense product the compressed path competes with: y = W x for uncompressed bf16 matrices, written as a streaming
+// kernel so that it is a fair opponent.  One launch takes a list of matrices (the same launch groups as the compressed
+// path).  A warp takes two rows at a time and walks them 2 KB per step: eight independent 16-byte loads per lane are in
+// flight before the first is used (32 warps per SM: about 128 KB per SM on its way, several times what the memory
+// latency times an SM's share of the bandwidth asks for); x comes from L1 and is shared by the two rows; products in
+// fp32, shuffle reduction.  Row pairs are dealt round-robin to the warps of the grid.
+__device__ __forceinline__ void fma_bf16x8(float &lo, float &hi, const uint4 &w, const uint4 &x) {
+    const uint32_t wv[4] = {w.x, w.y, w.z, w.w}, xv[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        lo = fmaf(__uint_as_float(wv[j] << 16), __uint_as_float(xv[j] << 16), lo);
+        hi = fmaf(__uint_as_float(wv[j] & 0xFFFF0000u), __uint_as_float(xv[j] & 0xFFFF0000u), hi);
+    }
+}
+
+__global__ void __launch_bounds__(256, 4) plain_gemv_kernel(const __grid_constant__ PlainArgs A) {
     const uint32_t lane = threadIdx.x & 31;
-    const uint64_t warp = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = ((uint64_t)gridDim.x * blockDim.x) >> 5;
-    for (uint64_t r = warp; r < rows; r += nwarps) {
-        const uint4 *wr = (const uint4 *)(w + r * cols);
-        const uint4 *xr = (const uint4 *)x;
-        float acc0 = 0.f, acc1 = 0.f;
-        for (uint64_t i = lane; i < cols / 8; i += 32) {
-            uint4 a = ldg_stream16(wr + i);
-            uint4 b = __ldg(xr + i);
-            const uint32_t av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    uint32_t mi = 0;
+    for (uint32_t u = warp; u < A.total_pairs; u += nwarps) {
+        while (mi + 1 < A.n_mats && u >= A.m[mi + 1].pair_first) ++mi;
+        const PlainMat &m = A.m[mi];
+        const uint64_t r = 2ull * (u - m.pair_first);
+        const bool two = r + 1 < m.rows;
+        const uint32_t nv = (uint32_t)(m.cols >> 3);                       // 16-byte pieces of a row
+        const uint4 *w0 = (const uint4 *)(m.w + r * m.cols), *w1 = two ? w0 + nv : w0;
+        const uint4 *xr = (const uint4 *)m.x;
+        float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
+        uint32_t i = lane;
+        for (; i + 96 < nv; i += 128) {                                    // four pieces of each row per lane and step
+            uint4 p[4], q[4], xv[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) p[j] = ldg_stream16(w0 + i + 32 * j);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) q[j] = ldg_stream16(w1 + i + 32 * j);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) xv[j] = __ldg(xr + i + 32 * j);
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                acc0 = fmaf(__uint_as_float(av[j] << 16), __uint_as_float(bv[j] << 16), acc0);
-                acc1 = fmaf(__uint_as_float(av[j] & 0xFFFF0000u), __uint_as_float(bv[j] & 0xFFFF0000u), acc1);
+                fma_bf16x8(a0, a1, p[j], xv[j]);
+                fma_bf16x8(b0, b1, q[j], xv[j]);
             }
         }
-        float acc = acc0 + acc1;
+        for (; i < nv; i += 32) {
+            const uint4 p = ldg_stream16(w0 + i), q = ldg_stream16(w1 + i), xv = __ldg(xr + i);
+            fma_bf16x8(a0, a1, p, xv);
+            fma_bf16x8(b0, b1, q, xv);
+        }
+        float sa = a0 + a1, sb = b0 + b1;
 #pragma unroll
-        for (int o = 16; o; o >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, o);
-        if (lane == 0) y[r] = acc;
+        for (int o = 16; o; o >>= 1) {
+            sa += __shfl_xor_sync(0xFFFFFFFFu, sa, o);
+            sb += __shfl_xor_sync(0xFFFFFFFFu, sb, o);
+        }
+        if (lane == 0) {
+            m.y[r] = sa;
+            if (two) m.y[r + 1] = sb;
+        }
     }
 }
 
@@ -494,13 +513,13 @@ cudaError_t launch_stage_copy(void *dst, const void *src, uint64_t bytes, uint32
 template <int MODE, int LB, int THREADS, int FMT>
 static cudaError_t launch_one(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
     auto fn = huff_kernel<MODE, LB, THREADS, FMT>;
-    static bool attr_set[64] = {};
+    static std::atomic<bool> attr_set[64];   // set twice by racing threads at worst: the call is idempotent
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    if (dev < 0 || dev >= 64 || !attr_set[dev].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)k.dyn_smem_bytes);
         if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+        if (dev >= 0 && dev < 64) attr_set[dev].store(true, std::memory_order_release);
     }
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(grid);
@@ -525,11 +544,10 @@ cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream)
     return k.lut_bits == 8 ? launch_one<1, 8, kThreads, 0>(k, grid, stream) : launch_one<1, 9, kThreads, 0>(k, grid, stream);
 }
 
-cudaError_t launch_plain_gemv(const uint16_t *w, uint64_t rows, uint64_t cols, const uint16_t *x, float *y, uint32_t sms,
-                              cudaStream_t stream) {
-    uint64_t blocks = (rows + 7) / 8;
-    uint32_t grid = (uint32_t)(blocks < (uint64_t)sms * 8 ? blocks : (uint64_t)sms * 8);
-    plain_gemv_kernel<<<grid, 256, 0, stream>>>(w, rows, cols, x, y);
+cudaError_t launch_plain_gemv(const PlainArgs &a, uint32_t sms, cudaStream_t stream) {
+    const uint64_t blocks = ((uint64_t)a.total_pairs + 7) / 8;              // 8 warps per CTA, a row pair per warp and turn
+    const uint32_t grid = (uint32_t)(blocks < (uint64_t)sms * 4 ? blocks : (uint64_t)sms * 4);
+    plain_gemv_kernel<<<grid, 256, 0, stream>>>(a);
     return cudaGetLastError();
 }
 

@@ -30,7 +30,7 @@ struct KernelArgs {
     uint32_t slot_bytes;       // shared-memory bytes of one slot: largest max_words * 256
     uint32_t pair_recip;       // floor(2^32 / (2 * slot_bytes)): umulhi(x, pair_recip) is x / (2 * slot_bytes) or one less
     uint32_t guard_bytes;      // readable bytes kept free behind the last slot
-    uint32_t part_bytes;       // bytes at the end of dynamic shared memory for the CTA's partial sums
+    uint32_t part_bytes;       // bytes at the end of dynamic shared memory for the CTA's partial sums (tensor-core path: the stages of activations)
     uint32_t dyn_smem_bytes;
     uint32_t batch;            // 1..8
     int32_t *err;              // may be null
@@ -48,7 +48,18 @@ cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t strea
 cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream);
 cudaError_t launch_gemm_tc(const KernelArgs &k, uint32_t grid, cudaStream_t stream);
 cudaError_t launch_stage_copy(void *dst, const void *src, uint64_t bytes, uint32_t sms, cudaStream_t stream);
-cudaError_t launch_plain_gemv(const uint16_t *w, uint64_t rows, uint64_t cols, const uint16_t *x, float *y, uint32_t sms,
-                              cudaStream_t stream);
+// The dense bf16 comparison product: up to kMaxMats matrices per launch, rows dealt to the warps in pairs.
+struct PlainMat {
+    const uint16_t *w;         // [rows][cols] bf16, device
+    const uint16_t *x;         // [cols]
+    float *y;                  // [rows]
+    uint64_t rows, cols;
+    uint32_t pair_first;       // number of the matrix's first row pair among the launch's row pairs
+};
+struct PlainArgs {
+    uint32_t n_mats, total_pairs;
+    PlainMat m[kMaxMats];
+};
+cudaError_t launch_plain_gemv(const PlainArgs &a, uint32_t sms, cudaStream_t stream);
 
 }  // namespace huffllm

@@ -19,6 +19,8 @@
 // a hardware barrier; one of them (they take turns) then issues the 8 MMAs of the stage and a tcgen05.commit onto
 // the stage's "empty" mbarrier, which the warps wait on (with a limit) before they reuse the stage four blocks later.
 // BF16 and FP16 {1,5,5,5} blobs share the kernel (template parameter FMT): tables, raw part and operand format differ.
+#include <atomic>
+
 #include "decode_common.cuh"
 
 namespace huffllm {
@@ -96,9 +98,6 @@ __device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t addr, uint32_t lbo
 
 // LB = table index bits; NPAD = batch rounded up to 16, 32 or 64 (the MMA's N); FMT = 0: BF16 blobs, 1: FP16 {1,5,5,5} blobs
 // (three tables, sign words as the raw part, f16 operands).
-#ifndef HUFFLLM_TC_SKIP_BELOW
-#define HUFFLLM_TC_SKIP_BELOW 64
-#endif
 template <int LB, int NPAD, int FMT>
 __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_constant__ KernelArgs A) {
     constexpr uint32_t kRawBlock = FMT ? 64u : 512u;          // raw bytes of one block of a record
@@ -110,7 +109,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     };
     // the decoder that starts behind the leading zero bits (see huff_kernel); at the widest padding, where a block's
     // time is set by the two-stage hand-over, it measured 1.4 % slower and is left out
-    constexpr bool SKIP = LB == 8 && FMT == 0 && NPAD < HUFFLLM_TC_SKIP_BELOW;
+    constexpr bool SKIP = LB == 8 && FMT == 0 && NPAD < 64;
     constexpr int R = SKIP ? 4 : LB == 8 ? 3 : 2;
     constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
     constexpr int S = NPAD == 64 ? 2 : kTcStages;          // the host's tc_stages(): shared memory is short at the widest padding
@@ -397,13 +396,13 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
 template <int LB, int NPAD, int FMT>
 static cudaError_t launch_tc_one(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
     auto fn = huff_gemm_tc_kernel<LB, NPAD, FMT>;
-    static bool attr_set[64] = {};
+    static std::atomic<bool> attr_set[64];   // set twice by racing threads at worst: the call is idempotent
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    if (dev < 0 || dev >= 64 || !attr_set[dev].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)k.dyn_smem_bytes);
         if (e != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+        if (dev >= 0 && dev < 64) attr_set[dev].store(true, std::memory_order_release);
     }
     fn<<<grid, 1024, k.dyn_smem_bytes, stream>>>(k);
     return cudaGetLastError();

@@ -62,7 +62,7 @@ def gpu_gemm(hl, torch, up, x):
         hl.decode_gemm(up.desc, up.blob_dev, x_dev, batch, y, up.ws, up.ws_bytes, up.err)
     torch.cuda.synchronize()
     assert int(up.err.item()) == 0
-    assert int(up.ws[:4096].count_nonzero().item()) == 0, "the scratch control words must be left zero"
+    assert int(up.ws[:hl.workspace_control_bytes(up.desc)].count_nonzero().item()) == 0, "the scratch control words must be left zero"
     res = y.cpu().numpy()
     assert np.all(np.isnan(res[batch * rows:]))
     return res[:batch * rows].reshape(batch, rows)
@@ -220,26 +220,29 @@ def test_several_matrices_in_one_launch(hl, torch, batch):
         x_devs.append(torch.from_numpy(x.view(np.int16)).cuda())
         ys.append(torch.full((batch * rows,), float("nan"), dtype=torch.float32, device="cuda"))
     err = torch.zeros(1, dtype=torch.int32, device="cuda")
+    ws_each = max(u.ws_bytes for u in ups)         # every workspace of a call has at least the largest matrix's size
+    for u in ups:
+        u.ws = torch.zeros(ws_each, dtype=torch.uint8, device="cuda")
     for rep in range(2):
         hl.decode_gemm_multi([u.desc for u in ups], [u.blob_dev for u in ups], x_devs, batch, ys, [u.ws for u in ups],
-                             ups[0].ws_bytes, err)
+                             ws_each, err)
         torch.cuda.synchronize()
         assert int(err.item()) == 0
         for u, x, y in zip(ups, xs, ys):
             check_product(y.cpu().numpy().reshape(batch, -1), u.w, x)
-            assert int(u.ws[:4096].count_nonzero().item()) == 0
+            assert int(u.ws[:hl.workspace_control_bytes(u.desc)].count_nonzero().item()) == 0
     # the same call with host buffers
     xh = [torch.from_numpy(x.view(np.int16).reshape(-1)).pin_memory() for x in xs]
     yh = [torch.zeros(batch * u.w.shape[0], dtype=torch.float32).pin_memory() for u in ups]
     hl.decode_gemm_multi_host([u.desc for u in ups], [u.blob_dev for u in ups], xh, batch, yh, x_devs, ys, [u.ws for u in ups],
-                              ups[0].ws_bytes, err)
+                              ws_each, err)
     for u, x, y in zip(ups, xs, yh):
         check_product(y.numpy().reshape(batch, -1), u.w, x)
     # and enqueued only, through the prepared call: the caller waits for the stream
     for y in yh:
         y.fill_(float("nan"))
     prep = hl.PreparedMulti([u.desc for u in ups], [u.blob_dev for u in ups], x_devs, batch, ys, [u.ws for u in ups],
-                            ups[0].ws_bytes, err, xh, yh)
+                            ws_each, err, xh, yh)
     prep.run_host_async(torch.cuda.current_stream().cuda_stream)
     torch.cuda.current_stream().synchronize()
     for u, x, y in zip(ups, xs, yh):
@@ -355,7 +358,7 @@ def test_full_layer_in_the_benchmarks_launch_groups_sampled(hl, torch, fuse):
     err = torch.zeros(1, dtype=torch.int32, device="cuda")
     stream = torch.cuda.current_stream().cuda_stream
     preps = [hl.PreparedMulti([mats[i]["desc"] for i in g], [mats[i]["blob_dev"] for i in g], [mats[i]["x_dev"] for i in g], 1,
-                              [mats[i]["y_dev"] for i in g], [mats[i]["ws"] for i in g], mats[0]["ws_bytes"], err) for g in groups]
+                              [mats[i]["y_dev"] for i in g], [mats[i]["ws"] for i in g], max(m["ws_bytes"] for m in mats), err) for g in groups]
     first = None
     for rep in range(2):
         for m in mats:
@@ -374,7 +377,7 @@ def test_full_layer_in_the_benchmarks_launch_groups_sampled(hl, torch, fuse):
         rs = rng.choice(m["rows"], 32, replace=False)
         yo, d = orc.matmul(m["w_sample"][rs], m["x_np"])
         assert np.all(np.abs(y[rs] - yo[0]) <= TOL * d[0]), m["name"]
-        assert int(m["ws"][:4096].count_nonzero().item()) == 0
+        assert int(m["ws"][:hl.workspace_control_bytes(m["desc"])].count_nonzero().item()) == 0
 
 
 def test_launches_can_be_captured_in_a_cuda_graph(hl, torch):
@@ -404,7 +407,7 @@ def test_launches_can_be_captured_in_a_cuda_graph(hl, torch):
         torch.cuda.synchronize()
         assert int(up.err.item()) == 0
         check_product(y_dev.cpu().numpy()[None, :], w, x)
-        assert int(up.ws[:4096].count_nonzero().item()) == 0
+        assert int(up.ws[:hl.workspace_control_bytes(up.desc)].count_nonzero().item()) == 0
 
 
 STRESS = [
