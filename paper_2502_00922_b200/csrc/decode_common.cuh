@@ -44,6 +44,22 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
+// Arrival without a transaction count (a consumer hands a slot back).
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// One look at a barrier's phase, without waiting.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
 // Bulk asynchronous copy global -> this CTA's shared memory, completion counted on `bar`.
 __device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(dst),
@@ -340,5 +356,6 @@ __device__ __forceinline__ uint32_t slot_addr(const SmemPlan &p, uint32_t warp, 
 constexpr int kMaxWarps = 32;
 constexpr int kThreads = 1024;   // threads per CTA of the decode kernels (one CTA per SM)
 constexpr uint32_t kWaitLimit = 1u << 22;
+constexpr uint32_t kFeederIdleLimit = 1u << 22;   // polls of 100 ns without any slot coming back before the feeder gives up
 
 }  // namespace huffllm

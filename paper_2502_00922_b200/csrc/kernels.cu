@@ -12,18 +12,18 @@
 // Mapping to the GPU
 //   * one warp decodes one chunk; lane l owns the two bit sequences l and 32 + l of the chunk record
 //     and steps through them alternately, which gives every lane two independent dependency chains
-//   * the coded part of a record is brought into shared memory by one bulk-async copy per chunk
-//     (no multicast), completion on an mbarrier; two slots per warp, so the next chunk is in
-//     flight while this one is decoded
-//   * the raw sign/mantissa bytes go straight from global memory to registers, 16 bytes per lane
-//     per block of 32 columns, one block ahead
+//   * one warp of the CTA (the feeder) does the bookkeeping of all the others: per decoder warp it reads the
+//     record index, checks the offsets and starts one bulk-async copy per chunk (no multicast) of the coded
+//     part into one of the warp's two shared-memory slots, completion on an mbarrier; a second mbarrier per
+//     slot brings the slot back.  It also asks L2 for the raw part of a record with one bulk prefetch
+//   * the raw sign/mantissa bytes go straight from global memory to the decoders' registers, 16 bytes per
+//     lane per block of 32 columns, one block ahead
 //   * the LUT is replicated per lane in shared memory (entry i of lane l at word 32 i + l), so a
-//     warp-wide lookup never has a bank conflict; it is placed on an address boundary that lets
-//     the lookup address be formed with a single logic operation
+//     warp-wide lookup never has a bank conflict
 //   * a lane's 16 weights of a block are exactly its share of two m16n8k16 tensor-core operand
 //     tiles, so the product needs no shuffles: decode, pack to bf16x2, mma
 //   * partial sums of a row group that is split over warps or CTAs are combined in a fixed order
-//     (shared memory inside a CTA, a scratch buffer plus a last-CTA pass across CTAs)
+//     (shared memory inside a CTA, arrival counters and a scratch buffer across CTAs); nobody waits for anybody
 #include <cuda_runtime.h>
 #include <atomic>
 #include <cstdint>
@@ -37,393 +37,432 @@ namespace huffllm {
 
 // MODE 0: write the decoded weights.  MODE 1: y = W x for up to 8 activation vectors.
 // LB = table index bits (the blobs' lut_bits): 8 or 9.
+// FMT = 0: BF16 blobs; FMT = 1: FP16 {1,5,5,5} blobs (three lookups per weight, sign bits as the raw part).
 //
 // One launch works through a LIST of matrices (A.n_mats, usually the matrices of one decoder layer that
 // may run together).  The CTAs are dealt out to the matrices in proportion to their chunks, so every CTA
 // lies inside a single matrix, builds a single table and meets no CTA-wide barrier after set-up.
-// FMT = 0: BF16 blobs; FMT = 1: FP16 {1,5,5,5} blobs (three lookups per weight, sign bits as the raw part).
+//
+// Roles.  The last warp of the CTA is the FEEDER: lane w looks after decoder warp w.  It reads the record index,
+// checks the offsets, starts the bulk copy of a chunk's coded part into one of the warp's two slots and leaves
+// a two-word note (the record's offsets) beside it; the copy's barrier carries the note to the decoder.  When a
+// decoder has finished with a slot it says so on a second barrier, which the feeder polls.  All bookkeeping of a
+// chunk is thus one lane's work instead of a whole warp's: the decoder warps, whose issue slots bound the kernel,
+// spend theirs on decoding.
 template <int MODE, int LB, int THREADS, int FMT>
 __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant__ KernelArgs A) {
     constexpr uint32_t kRawBlock = FMT ? 64u : 512u;          // raw bytes of one block of a record
     constexpr uint32_t kRawLane = FMT ? 2u : 16u;             // of which one lane's share
-    // raw part of a record with nkb blocks (FP16: padded to the 128-byte record unit)
-    auto raw_part = [](uint32_t nkb) -> uint32_t { return FMT ? (nkb * 64u + 127u) & ~127u : nkb * 512u; };
+    // raw part of a record with nkb blocks, in record units of 128 bytes (FP16: rounded up to whole units)
+    auto raw_units = [](uint32_t nkb) -> uint32_t { return FMT ? (nkb + 1u) >> 1 : nkb * 4u; };
     // 8-bit BF16 tables: the decoder starts behind the sequences' leading zero bits and works on four codewords at a
     // time (stream_step4x2)
     constexpr bool SKIP = LB == 8 && FMT == 0;
     constexpr int R = SKIP ? 4 : LB == 8 ? 3 : 2;            // decoder steps between two refill checks
     constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
     extern __shared__ __align__(128) uint8_t dyn_smem[];
-    __shared__ __align__(16) uint64_t bars[kMaxWarps * 2];     // a warp's two barriers differ in address bit 3 only
+    // per decoder warp: "full" barriers of its two slots (the copy has landed), then the two "empty" ones (the decoder is done)
+    __shared__ __align__(16) uint64_t bars[kMaxWarps * 4];
+    __shared__ __align__(16) uint2 notes[kMaxWarps * 2];       // per slot: the record's first and last offset, or kBadRecord
     __shared__ uint32_t s_arrive[kMaxWarps];   // arrival counters of row groups shared by several warps
+    __shared__ uint32_t s_stop;                // a decoder gave up waiting: the feeder stops too
+    constexpr uint32_t kBadRecord = 0xFFFFFFFFu;
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps_launched = blockDim.x >> 5;
     pdl_launch_dependents();   // the next kernel's set-up may overlap this kernel's tail
     const uint32_t smem_base = smem_u32(dyn_smem);
-    const SmemPlan plan = plan_smem(smem_base, A, nwarps_launched);
-    const uint32_t nw = plan.warps;
+    const uint32_t feeder = nwarps_launched - 1;
+    const SmemPlan plan = plan_smem(smem_base, A, feeder);
+    const uint32_t nw = plan.warps;                            // decoder warps
     const uint32_t vals = 16 * A.batch;
     float *part_val = (float *)(dyn_smem + A.dyn_smem_bytes - A.part_bytes);  // [2 * warps][16 * batch]
-
-    uint32_t lut_lane = plan.lut | ((FMT ? lane & 15u : lane) << 2);
-    asm volatile("mov.u32 %0, %0;" : "+r"(lut_lane));  // keep it in a register: it is an operand of every lookup
-    const uint32_t g = lane >> 2, t = lane & 3;
-    const uint32_t bar0 = smem_u32(&bars[warp * 2]);
-    const uint32_t slot0 = slot_addr(plan, warp, 0, A.slot_bytes);
-    if (lane == 0) {
-        mbar_init(bar0, 1);
-        mbar_init(bar0 + 8, 1);
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    }
-    bool waited_prior = false, failed = false;
 
     // the matrix this CTA works in, and the CTA's piece of that matrix's chunks
     uint32_t mi = 0;
     while (mi + 1 < A.n_mats && blockIdx.x >= A.m[mi + 1].cta_first) ++mi;
-    {
-        const MatArgs &k = A.m[mi];
-        const uint32_t J = blockIdx.x - k.cta_first;                        // this CTA's number among the CTAs of its matrix
-        // (the set-up runs in all 32 warps at once and is bound by instruction issue: no 64-bit divisions here)
-        auto cta_cut = [&](uint32_t j) -> uint32_t { return j * k.cta_chunks + min(j, k.cta_extra); };   // first chunk of the matrix's CTA j
-        const uint32_t cta_beg = cta_cut(J), cta_end = cta_cut(J + 1);
-        const uint32_t KC = k.col_chunks;
-        // the CTA's chunks are dealt to its warps: wq each, and wr warps in the MIDDLE of the range one more.  The warps
-        // with the extra chunk finish last; in the middle their row groups belong to this CTA alone, so what runs at
-        // the very end of the launch is a reduction in shared memory, not the one across CTAs with its global round trips
-        const uint32_t cta_len = cta_end - cta_beg, wq = nw == 32 ? cta_len >> 5 : cta_len / nw, wr = cta_len - wq * nw;
-        const uint32_t w_mid = (nw - wr) >> 1;
-        auto warp_beg = [&](uint32_t w) -> uint32_t { return cta_beg + w * wq + min(w > w_mid ? w - w_mid : 0u, wr); };
-        uint32_t c_beg = cta_beg, c_end = cta_beg;
-        if (warp < nw) {
-            c_beg = warp_beg(warp);
-            c_end = warp_beg(warp + 1);
-        }
-        const uint32_t *index = (const uint32_t *)(k.blob + k.off_index);
-        const uint8_t *payload = k.blob + k.off_payload;
-        // the offsets of the warp's first two records: asked for before anything else of the set-up, whose
-        // instructions then run while the loads are under way
-        const uint32_t rg_first = c_beg / KC, kc_first = c_beg - rg_first * KC;
-        uint32_t idx0 = 0, idx1 = 0, idx2 = 0;
-        if (lane == 0 && c_beg < c_end) {
-            idx0 = __ldg(index + c_beg);
-            idx1 = __ldg(index + c_beg + 1);
-            idx2 = c_beg + 1 < c_end ? __ldg(index + c_beg + 2) : 0u;
-        }
+    const MatArgs &k = A.m[mi];
+    const uint32_t J = blockIdx.x - k.cta_first;                        // this CTA's number among the CTAs of its matrix
+    auto cta_cut = [&](uint32_t j) -> uint32_t { return j * k.cta_chunks + min(j, k.cta_extra); };   // first chunk of the matrix's CTA j
+    const uint32_t cta_beg = cta_cut(J), cta_end = cta_cut(J + 1);
+    const uint32_t KC = k.col_chunks;
+    // the CTA's chunks are dealt to its decoder warps: wq each, and wr warps in the MIDDLE of the range one more.  The
+    // warps with the extra chunk finish last; in the middle their row groups belong to this CTA alone, so what runs at
+    // the very end of the launch is a reduction in shared memory, not the one across CTAs with its global round trips
+    const uint32_t cta_len = cta_end - cta_beg, wq = nw == 31 ? cta_len / 31u : cta_len / nw, wr = cta_len - wq * nw;
+    const uint32_t w_mid = (nw - wr) >> 1;
+    auto warp_beg = [&](uint32_t w) -> uint32_t { return cta_beg + w * wq + min(w > w_mid ? w - w_mid : 0u, wr); };
+    const uint32_t *index = (const uint32_t *)(k.blob + k.off_index);
+    const uint8_t *payload = k.blob + k.off_payload;
+    // blocks of 32 columns in column chunk kc: every chunk is full except, possibly, the last one of a row
+    const uint32_t nkb_full = k.chunk_cols >> 5, nkb_tail = ((uint32_t)k.cols - (KC - 1) * k.chunk_cols + 31u) >> 5;
 
-        // blocks of 32 columns in column chunk kc: every chunk is full except, possibly, the last one of a row
-        const uint32_t nkb_tail = ((uint32_t)k.cols - (KC - 1) * k.chunk_cols + 31u) >> 5;
-        auto blocks_of = [&](uint32_t kc) -> uint32_t { return kc + 1 == KC ? nkb_tail : k.chunk_cols >> 5; };
-        // a record is usable if it lies inside the payload and its coded part fits a slot
-        auto record_ok = [&](uint32_t r0, uint32_t r1, uint32_t nkb) -> bool {
-            return r1 > r0 && r1 <= k.payload_units && (r1 - r0) * 128u > raw_part(nkb) &&
-                   (r1 - r0) * 128u - raw_part(nkb) <= A.slot_bytes;
-        };
-        // lane 0: start the bulk copy of the coded part of a chunk (column chunk kc_c, record [ra, rb)) into slot `which`
-        auto issue_known = [&](uint32_t kc_c, uint32_t ra, uint32_t rb, uint32_t which) {
-            const uint32_t nkb = blocks_of(kc_c), bar = bar0 + which * 8;
-            if (record_ok(ra, rb, nkb)) {
-                uint32_t bytes = (rb - ra) * 128u - raw_part(nkb);
-                mbar_expect_tx(bar, bytes);
-                bulk_g2s(slot0 + which * A.slot_bytes, payload + (uint64_t)ra * 128u + raw_part(nkb), bytes, bar);
+    const uint32_t bar_w = smem_u32(&bars[(warp == feeder ? lane : warp) * 4]);   // the four barriers of "my" decoder warp
+    constexpr uint32_t kSetupBarrier = 1;       // hardware barrier of the set-up: the decoders wait at it, the feeder only arrives
+
+    if (warp == feeder) {
+        // ================================================================== the feeder
+        // lane w: next chunk and end of decoder warp w's range, that chunk's column chunk, chunks issued so far, and the
+        // offsets of the record to issue next
+        uint32_t f_ci = 0, f_ce = 0, f_issued = 0, f_ra = 0, f_rb = 0;
+        if (lane < nw) {
+            f_ci = warp_beg(lane);
+            f_ce = warp_beg(lane + 1);
+            if (f_ci < f_ce) {                       // asked for first: the set-up below runs while the answers are under way
+                f_ra = __ldg(index + f_ci);
+                f_rb = __ldg(index + f_ci + 1);
+            }
+#pragma unroll
+            for (int i = 0; i < 4; ++i) mbar_init(bar_w + 8 * i, 1);
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        if (lane == 0) *(volatile uint32_t *)&s_stop = 0;
+        __syncwarp();
+        // the barriers exist: the decoders may go on as soon as their table is built; the feeder does not wait for them
+        asm volatile("bar.arrive %0, %1;" ::"r"(kSetupBarrier), "r"(THREADS) : "memory");
+        uint32_t f_kc = f_ci % KC;
+        const uint32_t slot_units = A.slot_bytes >> 7, slot_w = slot_addr(plan, lane < nw ? lane : 0u, 0, A.slot_bytes);
+        const uint32_t note_w = smem_u32(&notes[lane * 2]);
+        uint32_t idle = 0;
+        while (__any_sync(0xFFFFFFFFu, f_ci < f_ce)) {
+            const uint32_t which = f_issued & 1u;
+            // a slot is free for its first chunk, and later once the decoder has handed it back
+            const bool ready = f_ci < f_ce && (f_issued < 2 || mbar_test_wait(bar_w + 16 + 8 * which, ((f_issued >> 1) - 1u) & 1u));
+            if (ready) {
+                const uint32_t full = bar_w + 8 * which, nkb = f_kc + 1 == KC ? nkb_tail : nkb_full;
+                // a record is usable if it lies inside the payload, is longer than its raw part and its coded part fits a slot
+                const bool ok = f_rb <= k.payload_units && f_rb - f_ra - raw_units(nkb) - 1u < slot_units;
+                asm volatile("st.shared.v2.u32 [%0], {%1, %2};" ::"r"(note_w + 8 * which), "r"(ok ? f_ra : kBadRecord), "r"(f_rb) : "memory");
+                if (ok) {
+                    const uint32_t bytes = (f_rb - f_ra - raw_units(nkb)) << 7;
+                    mbar_expect_tx(full, bytes);
+                    bulk_g2s(slot_w + which * A.slot_bytes, payload + ((uint64_t)(f_ra + raw_units(nkb)) << 7), bytes, full);
+                    // the raw part of the record is asked into L2 with one request (not for a warp's first two chunks: at the
+                    // start of a launch every warp's copies are under way at once, and only the decoders' own loads matter)
+                    if (f_issued >= 2)
+                        asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(payload + ((uint64_t)f_ra << 7)), "r"(raw_units(nkb) << 7) : "memory");
+                } else {
+                    mbar_expect_tx(full, 0);  // completes the phase with nothing to wait for; the decoder skips the chunk
+                }
+                ++f_ci;
+                ++f_issued;
+                f_kc = f_kc + 1 == KC ? 0u : f_kc + 1;
+                f_ra = f_rb;
+                if (f_ci < f_ce) f_rb = __ldg(index + f_ci + 1);
+            }
+            if (__any_sync(0xFFFFFFFFu, ready)) {
+                idle = 0;
             } else {
-                mbar_expect_tx(bar, 0);  // completes the phase with nothing to wait for; the chunk is skipped below
-            }
-        };
-
-        // ---- set-up of a segment.  The table loads are started first, then every warp starts its first
-        // copies, then the table is written to shared memory: the cold misses on the table, on the record
-        // index and on the first records overlap instead of following each other.
-        // (FP16: three tables of 256 entries, sixteen copies each: word j holds entry j / 16 of its table)
-        // The table goes to shared memory in 16-byte pieces: four neighbouring copies of one entry per piece.
-        constexpr uint32_t kLutWords = FMT ? 3u * 16u * 256u : 32u << LB;
-        constexpr uint32_t kLutRep = FMT ? 4u : 5u;            // log2 of the copies per entry
-        constexpr uint32_t kLutVecs = kLutWords / 4;
-        constexpr int kLutLoads = (kLutVecs + THREADS - 1) / THREADS;
-        uint32_t lut_v[kLutLoads];
-        {
-            const uint32_t *lut_g = (const uint32_t *)(k.blob + k.off_lut);
-#pragma unroll
-            for (int i = 0; i < kLutLoads; ++i) {
-                uint32_t v = tid + i * THREADS;
-                lut_v[i] = (kLutVecs % THREADS == 0 || v < kLutVecs) ? __ldg(lut_g + (v >> (kLutRep - 2))) : 0u;
-                if (SKIP) lut_v[i] = lut_entry_inplace(lut_v[i]);   // the length once more, where an in-place shift reads it
+                __nanosleep(100);
+                if (++idle > kFeederIdleLimit || *(volatile uint32_t *)&s_stop) break;   // (a decoder that stopped never hands slots back)
             }
         }
-        if (lane == 0 && c_beg < c_end) {
-            issue_known(kc_first, idx0, idx1, 0);
-            if (c_beg + 1 < c_end) issue_known(kc_first + 1 == KC ? 0u : kc_first + 1, idx1, idx2, 1);
-        }
-        {
-            uint4 *lut_s = (uint4 *)(dyn_smem + (plan.lut - smem_base));
-#pragma unroll
-            for (int i = 0; i < kLutLoads; ++i) {
-                uint32_t v = tid + i * THREADS;
-                if (kLutVecs % THREADS == 0 || v < kLutVecs) lut_s[v] = make_uint4(lut_v[i], lut_v[i], lut_v[i], lut_v[i]);
-            }
-            if (tid < kMaxWarps) s_arrive[tid] = 0;
-        }
-        __syncthreads();
+        return;
+    }
 
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        int cur_rg = -1;
-
-        // ---- reduction of a finished row group, without any CTA-wide barrier.
-        // A row group whose chunks this warp decoded alone goes straight to y.  Otherwise the warp parks its
-        // piece in shared memory and bumps an arrival counter (indexed by the first warp that holds a piece);
-        // the warp that arrives last adds the pieces in warp order.  If other CTAs hold pieces too, the CTA's
-        // sum goes to the scratch buffer and the same game is played across CTAs with a counter in global
-        // memory.  Sums are always taken in the same order, and nobody waits for anybody.
-        auto cta_of_chunk = [&](uint32_t ch) -> uint32_t {     // which of the matrix's CTAs works on chunk ch
-            const uint32_t big = k.cta_extra * (k.cta_chunks + 1);
-            return ch < big ? ch / (k.cta_chunks + 1) : k.cta_extra + (ch - big) / k.cta_chunks;
-        };
-        // lanes 0..vals-1 (looping if vals > 32) hold or produce the value of output o = column * 16 + row
-        auto finish_cta_sum = [&](int rg, float (&v)[4]) {       // v[i] = value of output o = lane + 32 i
-            const uint32_t g_lo = (uint32_t)rg * KC, g_hi = g_lo + KC;
-            if (cta_beg <= g_lo && cta_end >= g_hi) {             // the CTA held the whole row group
+    // ====================================================================== the decoder warps
+    // ---- set-up: the table loads are started first, then this warp's own values are worked out, then the table is
+    // written to shared memory (by the decoder warps alone: the feeder is already asking for records)
+    // (FP16: three tables of 256 entries, sixteen copies each: word j holds entry j / 16 of its table)
+    // The table goes to shared memory in 16-byte pieces: four neighbouring copies of one entry per piece.
+    constexpr uint32_t kLutWords = FMT ? 3u * 16u * 256u : 32u << LB;
+    constexpr uint32_t kLutRep = FMT ? 4u : 5u;            // log2 of the copies per entry
+    constexpr uint32_t kLutVecs = kLutWords / 4;
+    constexpr uint32_t kLutThreads = THREADS - 32;
+    constexpr int kLutLoads = (kLutVecs + kLutThreads - 1) / kLutThreads;
+    uint32_t lut_v[kLutLoads];
+    {
+        const uint32_t *lut_g = (const uint32_t *)(k.blob + k.off_lut);
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    uint32_t o = lane + 32 * i;
-                    uint64_t r = (uint64_t)rg * 16 + (o & 15);
-                    if (o < vals && r < k.rows) k.y[(uint64_t)(o >> 4) * k.rows + r] = v[i];
-                }
-                return;
-            }
-            // slot 0 holds the piece of the CTA's first row group in this matrix, slot 1 the piece of its last one
-            const uint32_t my_slot = (uint32_t)rg == cta_beg / KC ? 0u : 1u;
+        for (int i = 0; i < kLutLoads; ++i) {
+            uint32_t v = tid + i * kLutThreads;
+            lut_v[i] = v < kLutVecs ? __ldg(lut_g + (v >> (kLutRep - 2))) : 0u;
+            if (SKIP) lut_v[i] = lut_entry_inplace(lut_v[i]);   // the length once more, where an in-place shift reads it
+        }
+    }
+    uint32_t lut_lane = plan.lut | ((FMT ? lane & 15u : lane) << 2);
+    asm volatile("mov.u32 %0, %0;" : "+r"(lut_lane));  // keep it in a register: it is an operand of every lookup
+    const uint32_t g = lane >> 2, t = lane & 3;
+    uint32_t c_beg = 0, c_end = 0;
+    if (warp < nw) {
+        c_beg = warp_beg(warp);
+        c_end = warp_beg(warp + 1);
+    }
+    // the warp's first record: its raw bytes are asked for before the table is finished
+    uint32_t r_first = c_beg < c_end ? __ldg(index + c_beg) : 0xFFFFFFFFu;
+    // raw sign/mantissa bytes travel one block ahead of the decoder, in two register sets used in turn
+    uint4 raw_a = make_uint4(0, 0, 0, 0), raw_b = make_uint4(0, 0, 0, 0);
+    bool primed = false;
+    auto load_raw = [](const uint8_t *p) -> uint4 {
+        if (FMT) return make_uint4(ldg_stream2(p), 0, 0, 0);
+        return ldg_stream16(p);
+    };
+    const uint8_t *raw_p = payload;
+    {
+        uint4 *lut_s = (uint4 *)(dyn_smem + (plan.lut - smem_base));
+#pragma unroll
+        for (int i = 0; i < kLutLoads; ++i) {
+            uint32_t v = tid + i * kLutThreads;
+            if (v < kLutVecs) lut_s[v] = make_uint4(lut_v[i], lut_v[i], lut_v[i], lut_v[i]);
+        }
+        if (tid < kMaxWarps) s_arrive[tid] = 0;
+    }
+    if (r_first < k.payload_units) {        // (the blob keeps 4 KB behind the payload: a block's read stays inside it)
+        raw_p = payload + ((uint64_t)r_first << 7) + lane * kRawLane;
+        raw_a = load_raw(raw_p);
+        primed = true;
+    }
+    asm volatile("bar.sync %0, %1;" ::"r"(kSetupBarrier), "r"(THREADS) : "memory");
+    if (warp >= nw) return;
+
+    bool waited_prior = false, failed = false;
+
+    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    int cur_rg = -1;
+
+    // ---- reduction of a finished row group, without any CTA-wide barrier.
+    // A row group whose chunks this warp decoded alone goes straight to y.  Otherwise the warp parks its
+    // piece in shared memory and bumps an arrival counter (indexed by the first warp that holds a piece);
+    // the warp that arrives last adds the pieces in warp order.  If other CTAs hold pieces too, the CTA's
+    // sum goes to the scratch buffer and the same game is played across CTAs with a counter in global
+    // memory.  Sums are always taken in the same order, and nobody waits for anybody.
+    auto cta_of_chunk = [&](uint32_t ch) -> uint32_t {     // which of the matrix's CTAs works on chunk ch
+        const uint32_t big = k.cta_extra * (k.cta_chunks + 1);
+        return ch < big ? ch / (k.cta_chunks + 1) : k.cta_extra + (ch - big) / k.cta_chunks;
+    };
+    // lanes 0..vals-1 (looping if vals > 32) hold or produce the value of output o = column * 16 + row
+    auto finish_cta_sum = [&](int rg, float (&v)[4]) {       // v[i] = value of output o = lane + 32 i
+        const uint32_t g_lo = (uint32_t)rg * KC, g_hi = g_lo + KC;
+        if (cta_beg <= g_lo && cta_end >= g_hi) {             // the CTA held the whole row group
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
                 uint32_t o = lane + 32 * i;
-                if (o < vals) k.ws_partial[((size_t)J * 2 + my_slot) * vals + o] = v[i];
-            }
-            __syncwarp();
-            const uint32_t c0 = cta_of_chunk(g_lo), c1 = cta_of_chunk(g_hi - 1);
-            uint32_t last = 0;
-            if (lane == 0) {
-                last = arrive_acq_rel(k.ws_ticket + c0) == c1 - c0 ? 1u : 0u;
-                if (last) k.ws_ticket[c0] = 0;                    // leave the counter as it was found
-            }
-            if (!__shfl_sync(0xFFFFFFFFu, last, 0)) return;       // somebody else will arrive later and add us in
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                uint32_t o = lane + 32 * i;
-                if (o >= vals) continue;
-                float sum = 0.f;
-                for (uint32_t c = c0; c <= c1; ++c) {
-                    uint32_t slot = cta_cut(c) / KC == (uint32_t)rg ? 0u : 1u;
-                    sum += __ldcg(k.ws_partial + ((size_t)c * 2 + slot) * vals + o);
-                }
                 uint64_t r = (uint64_t)rg * 16 + (o & 15);
-                if (r < k.rows) k.y[(uint64_t)(o >> 4) * k.rows + r] = sum;
+                if (o < vals && r < k.rows) k.y[(uint64_t)(o >> 4) * k.rows + r] = v[i];
             }
-        };
-        auto flush = [&](int rg, uint32_t first_c, uint32_t last_c_excl) {
-            if (rg < 0) return;
-            const uint32_t g_lo = max((uint32_t)rg * KC, cta_beg), g_hi = min((uint32_t)(rg + 1) * KC, cta_end);  // this CTA's part
-            const bool alone = first_c <= g_lo && last_c_excl >= g_hi;   // no other warp of this CTA holds a piece
-            // D fragment -> output order (o = column * 16 + row) through this warp's shared-memory entry
-            const uint32_t ent = warp * 2 + ((uint32_t)rg == c_beg / KC ? 0u : 1u);
-            float *mine = part_val + (size_t)ent * vals;
+            return;
+        }
+        // slot 0 holds the piece of the CTA's first row group in this matrix, slot 1 the piece of its last one
+        const uint32_t my_slot = (uint32_t)rg == cta_beg / KC ? 0u : 1u;
 #pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                uint32_t col = 2 * t + (j & 1), row = g + 8 * (j >> 1);
-                if (col < A.batch) mine[col * 16 + row] = acc[j];
+        for (int i = 0; i < 4; ++i) {
+            uint32_t o = lane + 32 * i;
+            if (o < vals) k.ws_partial[((size_t)J * 2 + my_slot) * vals + o] = v[i];
+        }
+        __syncwarp();
+        const uint32_t c0 = cta_of_chunk(g_lo), c1 = cta_of_chunk(g_hi - 1);
+        uint32_t last = 0;
+        if (lane == 0) {
+            last = arrive_acq_rel(k.ws_ticket + c0) == c1 - c0 ? 1u : 0u;
+            if (last) k.ws_ticket[c0] = 0;                    // leave the counter as it was found
+        }
+        if (!__shfl_sync(0xFFFFFFFFu, last, 0)) return;       // somebody else will arrive later and add us in
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            uint32_t o = lane + 32 * i;
+            if (o >= vals) continue;
+            float sum = 0.f;
+            for (uint32_t c = c0; c <= c1; ++c) {
+                uint32_t slot = cta_cut(c) / KC == (uint32_t)rg ? 0u : 1u;
+                sum += __ldcg(k.ws_partial + ((size_t)c * 2 + slot) * vals + o);
             }
-            acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+            uint64_t r = (uint64_t)rg * 16 + (o & 15);
+            if (r < k.rows) k.y[(uint64_t)(o >> 4) * k.rows + r] = sum;
+        }
+    };
+    auto flush = [&](int rg, uint32_t first_c, uint32_t last_c_excl) {
+        if (rg < 0) return;
+        const uint32_t g_lo = max((uint32_t)rg * KC, cta_beg), g_hi = min((uint32_t)(rg + 1) * KC, cta_end);  // this CTA's part
+        const bool alone = first_c <= g_lo && last_c_excl >= g_hi;   // no other warp of this CTA holds a piece
+        // D fragment -> output order (o = column * 16 + row) through this warp's shared-memory entry
+        const uint32_t ent = warp * 2 + ((uint32_t)rg == c_beg / KC ? 0u : 1u);
+        float *mine = part_val + (size_t)ent * vals;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            uint32_t col = 2 * t + (j & 1), row = g + 8 * (j >> 1);
+            if (col < A.batch) mine[col * 16 + row] = acc[j];
+        }
+        acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+        __syncwarp();
+        float v[4];
+        if (alone) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) v[i] = lane + 32 * i < vals ? mine[lane + 32 * i] : 0.f;
             __syncwarp();
-            float v[4];
-            if (alone) {
-#pragma unroll
-                for (int i = 0; i < 4; ++i) v[i] = lane + 32 * i < vals ? mine[lane + 32 * i] : 0.f;
-                __syncwarp();
-                finish_cta_sum(rg, v);
-                return;
-            }
-            // which warps of this CTA hold a piece of this row group (lane l answers for warp l)
-            const uint32_t wb = warp_beg(lane), we = warp_beg(lane + 1);
-            const bool holds = lane < nw && wb < we && wb < g_hi && we > g_lo;
-            const uint32_t mask = __ballot_sync(0xFFFFFFFFu, holds);
-            const uint32_t w_first = __ffs(mask) - 1, n_hold = __popc(mask);
-            const uint32_t slot_of_lane = (uint32_t)rg == wb / KC ? 0u : 1u;
-            uint32_t last = 0;
-            if (lane == 0) {
-                __threadfence_block();
-                last = atomicAdd(&s_arrive[w_first], 1u) == n_hold - 1 ? 1u : 0u;
-                if (last) __threadfence_block();
-            }
-            if (!__shfl_sync(0xFFFFFFFFu, last, 0)) return;
-#pragma unroll
-            for (int i = 0; i < 4; ++i) v[i] = 0.f;
-            for (uint32_t m = mask; m; m &= m - 1) {              // pieces in warp order
-                const uint32_t w = __ffs(m) - 1;
-                const float *piece = part_val + (size_t)(w * 2 + __shfl_sync(0xFFFFFFFFu, slot_of_lane, w)) * vals;
-#pragma unroll
-                for (int i = 0; i < 4; ++i)
-                    if (lane + 32 * i < vals) v[i] += piece[lane + 32 * i];
-            }
             finish_cta_sum(rg, v);
-        };
+            return;
+        }
+        // which warps of this CTA hold a piece of this row group (lane l answers for warp l)
+        const uint32_t wb = warp_beg(lane), we = warp_beg(lane + 1);
+        const bool holds = lane < nw && wb < we && wb < g_hi && we > g_lo;
+        const uint32_t mask = __ballot_sync(0xFFFFFFFFu, holds);
+        const uint32_t w_first = __ffs(mask) - 1, n_hold = __popc(mask);
+        const uint32_t slot_of_lane = (uint32_t)rg == wb / KC ? 0u : 1u;
+        uint32_t last = 0;
+        if (lane == 0) {
+            __threadfence_block();
+            last = atomicAdd(&s_arrive[w_first], 1u) == n_hold - 1 ? 1u : 0u;
+            if (last) __threadfence_block();
+        }
+        if (!__shfl_sync(0xFFFFFFFFu, last, 0)) return;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) v[i] = 0.f;
+        for (uint32_t m = mask; m; m &= m - 1) {              // pieces in warp order
+            const uint32_t w = __ffs(m) - 1;
+            const float *piece = part_val + (size_t)(w * 2 + __shfl_sync(0xFFFFFFFFu, slot_of_lane, w)) * vals;
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+                if (lane + 32 * i < vals) v[i] += piece[lane + 32 * i];
+        }
+        finish_cta_sum(rg, v);
+    };
 
-        if (c_beg < c_end && !failed) {
-            uint32_t rg = rg_first, kc = kc_first;                    // tracked incrementally from here on
-            uint32_t r0 = __ldg(index + c_beg), r1 = __ldg(index + c_beg + 1);
-            // raw sign/mantissa bytes travel one block ahead of the decoder, in two register sets used in turn
-            uint4 raw_a = make_uint4(0, 0, 0, 0), raw_b = make_uint4(0, 0, 0, 0);
-            bool primed = false;
-            bool ok = record_ok(r0, r1, blocks_of(kc));               // carried along: every record is checked once
-            // Running pointers.  Records follow each other in memory and so do the columns of a row group's chunks,
-            // so the raw-byte pointer and the activation pointer simply run on from chunk to chunk.
-            const uint8_t *raw_p = payload + (uint64_t)r0 * 128u + lane * kRawLane;
-            const uint16_t *xq = k.x + (MODE == 1 ? (uint64_t)min(g, A.batch - 1) * k.cols + kc * k.chunk_cols + t * 8u : 0);
-            uint32_t which = 0;
-            // this chunk's slot (the lane's column of it) and barrier, toggled by XOR from chunk to chunk; parity of the
-            // barrier's next completion (each of the two barriers completes every second chunk)
-            uint32_t slot_cur = slot0 + (lane << 2), bar_cur = bar0, par = 0;
-            const uint32_t slot_tog = slot_cur ^ (slot_cur + A.slot_bytes);
-            auto load_raw = [](const uint8_t *p) -> uint4 {
-                if (FMT) return make_uint4(ldg_stream2(p), 0, 0, 0);
-                return ldg_stream16(p);
-            };
+    if (c_beg < c_end) {
+        uint32_t rg = c_beg / KC, kc = c_beg - rg * KC;               // tracked incrementally from here on
+        // The activation pointer runs on from chunk to chunk: the columns of a row group's chunks follow each other.
+        const uint16_t *xq = k.x + (MODE == 1 ? (uint64_t)min(g, A.batch - 1) * k.cols + kc * k.chunk_cols + t * 8u : 0);
+        // this chunk's slot (the lane's column of it), its barrier and its note, toggled by XOR from chunk to chunk; parity
+        // of the barrier's next completion (each of the two "full" barriers completes every second chunk)
+        uint32_t slot_cur = slot_addr(plan, warp, 0, A.slot_bytes) + (lane << 2), bar_cur = bar_w, par = 0, which = 0;
+        const uint32_t slot_tog = slot_cur ^ (slot_cur + A.slot_bytes);
+        uint32_t note_cur = smem_u32(&notes[warp * 2]);
 
 #pragma unroll 1
-            for (uint32_t c = c_beg; c < c_end; ++c) {
-                const uint32_t nkb = blocks_of(kc);
-                // the chunk after this one: its first raw block is fetched from inside this chunk's loop
-                const bool has_next = c + 1 < c_end;
-                const uint32_t kc1 = kc + 1 == KC ? 0u : kc + 1;
-                const uint32_t r2 = has_next ? __ldg(index + c + 2) : r1;
-                const bool next_ok = has_next && record_ok(r1, r2, blocks_of(kc1));
+        for (uint32_t c = c_beg; c < c_end; ++c) {
+            const uint32_t nkb = kc + 1 == KC ? nkb_tail : nkb_full;
+            if (MODE == 1 && (int)rg != cur_rg) {
+                flush(cur_rg, c_beg, c);  // the previous row group ended with chunk c - 1
+                cur_rg = (int)rg;
+            }
 
-                if (MODE == 1 && (int)rg != cur_rg) {
-                    flush(cur_rg, c_beg, c);  // the previous row group ended with chunk c - 1
-                    cur_rg = (int)rg;
-                }
-
-                // the block after this chunk's last one is the first block of the next record, `coded_bytes` further on
-                const uint32_t coded_bytes = (r1 - r0) * 128u - nkb * kRawBlock;
-                if (ok && !primed) raw_a = load_raw(raw_p);
-
-                // wait, with a limit, for the coded part; the outcome is made uniform across the warp
-                {
-                    uint32_t spins = 0;
-                    bool done = mbar_try_wait(bar_cur, par);
-                    while (!__all_sync(0xFFFFFFFFu, done)) {
-                        if (++spins > kWaitLimit) { failed = true; break; }
-                        done = mbar_try_wait(bar_cur, par);
-                    }
-                    if (failed) {
-                        if (A.err && lane == 0) atomicExch(A.err, -1);
+            // wait, with a limit, for the coded part; the outcome is made uniform across the warp
+            if (!failed) {
+                uint32_t spins = 0;
+                bool done = mbar_try_wait(bar_cur, par);
+                while (!__all_sync(0xFFFFFFFFu, done)) {
+                    if (++spins > kWaitLimit) {
+                        failed = true;      // this chunk and the warp's later ones add nothing; the row groups are still closed
+                        if (lane == 0) {
+                            if (A.err) atomicExch(A.err, -1);
+                            *(volatile uint32_t *)&s_stop = 1;
+                        }
                         break;
                     }
+                    done = mbar_try_wait(bar_cur, par);
                 }
-
-                if (!waited_prior) {
-                    pdl_wait_prior_grid();   // from here on this warp reads x and writes results: the previous kernel must be done
-                    waited_prior = true;
-                }
-                if (!ok) {  // record offsets out of range: report, produce nothing for this chunk, touch no memory
-                    if (A.err && lane == 0) atomicExch(A.err, (int32_t)min(c + 1, 0x7FFFFFFFu));
-                    primed = false;
-                    raw_p = payload + (uint64_t)r1 * 128u + lane * kRawLane;      // where the next record would start
-                    if (MODE == 1) xq += nkb * 32u;
-                } else {
-                    LaneStream sa, sb;
-                    stream_open(sa, slot_cur, SKIP ? 7u : 0u);
-                    stream_open(sb, slot_cur + 128u, SKIP ? 7u : 0u);
-                    const uint32_t col0 = kc * k.chunk_cols + t * 8u;
-                    // (activations: lanes of unused output columns repeat the last vector; cols is a multiple of 32
-                    // here, so every block of the chunk lies inside the row and xq ends the chunk where the next begins)
-                    uint16_t *out0 = MODE == 0 ? k.out + ((uint64_t)rg * 16 + g) * k.cols + col0 : nullptr;
-                    const uint32_t last = nkb - 1;
-
-                    // one block: start the fetch of the next block's raw bytes into `nxt`, decode with `cur`
-                    // (may_be_last = false: the caller knows that another block of this chunk follows)
-                    // Every block asks L2 for the 16 bytes per lane that lie four blocks further on in the record stream (the
-                    // loads that bring raw bytes to registers run one block ahead of the decoder, too short for a miss in
-                    // DRAM).  In a record's first half that is the raw part of its second half; in the second half it is the
-                    // coded part and, at its end, the start of the next record.  Measured: this plain form is the fastest;
-                    // asking only for raw bytes, or for the next record's first blocks, gains a third of it or nothing.
-                    // The request ends at most 2 KB behind the record it is issued in: inside the blob, whose format keeps 4 KB of
-                    // zero bytes behind the payload for this.
-                    // (products of BF16 blobs only: the decode-only kernel has no register to spare for it, and an FP16 record's
-                    // raw part is a sixteenth of its bytes)
-                    constexpr bool kPrefetchRaw = MODE == 1 && FMT == 0;
-                    auto block = [&](uint32_t kb, const uint4 &cur, uint4 &nxt, auto may_be_last) {
-                        raw_p += kRawBlock;
-                        if (kPrefetchRaw) asm volatile("prefetch.global.L2 [%0];" ::"l"(raw_p + 3u * kRawBlock));
-                        if (decltype(may_be_last)::value) {
-                            if (kb == last) raw_p += coded_bytes;       // the next record's first block
-                            if (kb != last || next_ok) nxt = load_raw(raw_p);
-                        } else {
-                            nxt = load_raw(raw_p);
-                        }
-                        uint4 xv;
-                        if (MODE == 1) {
-                            xv = __ldg((const uint4 *)xq);
-                            xq += 32;
-                        }
-
-                        uint32_t a[8];
-                        if (FMT) decode_block_fp16(sa, sb, lut_lane, cur.x, a);
-                        else decode_block<R, SKIP>(sa, sb, kIdxMask, lut_lane, cur, a);
-
-                        if (MODE == 1) {
-                            if (FMT) {
-                                mma_f16_16816(acc, a[0], a[4], a[1], a[5], xv.x, xv.y);
-                                mma_f16_16816(acc, a[2], a[6], a[3], a[7], xv.z, xv.w);
-                            } else {
-                                mma_bf16_16816(acc, a[0], a[4], a[1], a[5], xv.x, xv.y);
-                                mma_bf16_16816(acc, a[2], a[6], a[3], a[7], xv.z, xv.w);
-                            }
-                        } else {
-                            const uint32_t col = col0 + kb * 32u;
-#pragma unroll
-                            for (int h = 0; h < 2; ++h) {
-                                if ((uint64_t)rg * 16 + g + 8 * h >= k.rows || col >= (uint32_t)k.cols) continue;
-                                uint16_t *dst = out0 + (uint64_t)(8 * h) * k.cols + kb * 32u;
-                                if (k.cols % 8 == 0) {
-                                    *(uint4 *)dst = make_uint4(a[4 * h], a[4 * h + 1], a[4 * h + 2], a[4 * h + 3]);
-                                } else {
-#pragma unroll
-                                    for (int i = 0; i < 8; ++i)
-                                        if (col + i < (uint32_t)k.cols) dst[i] = (uint16_t)(a[4 * h + (i >> 1)] >> (16 * (i & 1)));
-                                }
-                            }
-                        }
-                    };
-                    constexpr std::integral_constant<bool, false> inner{};
-                    constexpr std::integral_constant<bool, true> maybe_last{};
-                    uint32_t kb = 0;
-#pragma unroll 1
-                    for (; kb + 4 <= nkb; kb += 4) {                    // the usual case: groups of four blocks
-                        block(kb, raw_a, raw_b, inner);
-                        block(kb + 1, raw_b, raw_a, inner);
-                        block(kb + 2, raw_a, raw_b, inner);
-                        block(kb + 3, raw_b, raw_a, maybe_last);
-                    }
-#pragma unroll 1
-                    for (; kb < nkb; kb += 2) {
-                        block(kb, raw_a, raw_b, maybe_last);
-                        if (kb + 1 < nkb) block(kb + 1, raw_b, raw_a, maybe_last);
-                    }
-                    if (nkb & 1u) raw_a = raw_b;     // the next chunk's first block always starts in raw_a
-                    primed = next_ok;
-                }
-                __syncwarp();
-                if (lane == 0 && c + 2 < c_end) issue_known(kc1 + 1 == KC ? 0u : kc1 + 1, r2, __ldg(index + c + 3), which);
-                r0 = r1;
-                r1 = r2;
-                ok = next_ok;
-                par ^= which;                                         // 0, 0, 1, 1, 0, 0, ...
-                which ^= 1u;
-                slot_cur ^= slot_tog;
-                bar_cur ^= 8u;
-                if (MODE == 1 && kc1 == 0) xq -= k.cols;              // the next chunk starts the next row group: back to column 0
-                kc = kc1;
-                rg += kc1 == 0 ? 1u : 0u;
             }
-            if (MODE == 1 && !failed) flush(cur_rg, c_beg, c_end);
+            if (!waited_prior) {
+                pdl_wait_prior_grid();   // from here on this warp reads x and writes results: the previous kernel must be done
+                waited_prior = true;
+            }
+            uint32_t r0, r1;            // the feeder's note: the record's first and last offset
+            asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(note_cur));
+            if (failed || r0 == kBadRecord) {  // record offsets out of range: report, produce nothing for this chunk, touch no memory
+                if (!failed && A.err && lane == 0) atomicExch(A.err, (int32_t)min(c + 1, 0x7FFFFFFFu));
+                primed = false;
+                if (MODE == 1) xq += nkb * 32u;
+            } else {
+                if (!primed) {
+                    raw_p = payload + ((uint64_t)r0 << 7) + lane * kRawLane;
+                    raw_a = load_raw(raw_p);
+                }
+                // the record behind this one is the next chunk's: its first raw block is fetched from inside this chunk's last
+                // block (the address lies inside the blob whatever that record's offsets turn out to be)
+                const bool has_next = c + 1 < c_end;
+                const uint32_t coded_bytes = (r1 - r0 - raw_units(nkb)) << 7;
+                LaneStream sa, sb;
+                stream_open(sa, slot_cur, SKIP ? 7u : 0u);
+                stream_open(sb, slot_cur + 128u, SKIP ? 7u : 0u);
+                const uint32_t col0 = kc * k.chunk_cols + t * 8u;
+                // (activations: lanes of unused output columns repeat the last vector; cols is a multiple of 32
+                // here, so every block of the chunk lies inside the row and xq ends the chunk where the next begins)
+                uint16_t *out0 = MODE == 0 ? k.out + ((uint64_t)rg * 16 + g) * k.cols + col0 : nullptr;
+                const uint32_t last = nkb - 1;
+
+                // one block: start the fetch of the next block's raw bytes into `nxt`, decode with `cur`
+                // (may_be_last = false: the caller knows that another block of this chunk follows)
+                // Every block asks L2 for the 16 bytes per lane that lie four blocks further on in the record stream (the
+                // loads that bring raw bytes to registers run one block ahead of the decoder, too short for a miss in
+                // DRAM).  In a record's first half that is the raw part of its second half; in the second half it is the
+                // coded part and, at its end, the start of the next record.  The request ends at most 2 KB behind the
+                // record it is issued in: inside the blob, whose format keeps 4 KB of zero bytes behind the payload for this.
+                // (products of BF16 blobs only: the decode-only kernel has no register to spare for it, and an FP16 record's
+                // raw part is a sixteenth of its bytes)
+                constexpr bool kPrefetchRaw = false;
+                auto block = [&](uint32_t kb, const uint4 &cur, uint4 &nxt, auto may_be_last) {
+                    raw_p += kRawBlock;
+                    if (kPrefetchRaw) asm volatile("prefetch.global.L2 [%0];" ::"l"(raw_p + 3u * kRawBlock));
+                    if (decltype(may_be_last)::value) {
+                        if (kb == last) raw_p += coded_bytes;       // the next record's first block
+                        if (kb != last || has_next) nxt = load_raw(raw_p);
+                    } else {
+                        nxt = load_raw(raw_p);
+                    }
+                    uint4 xv;
+                    if (MODE == 1) {
+                        xv = __ldg((const uint4 *)xq);
+                        xq += 32;
+                    }
+
+                    uint32_t a[8];
+                    if (FMT) decode_block_fp16(sa, sb, lut_lane, cur.x, a);
+                    else decode_block<R, SKIP>(sa, sb, kIdxMask, lut_lane, cur, a);
+
+                    if (MODE == 1) {
+                        if (FMT) {
+                            mma_f16_16816(acc, a[0], a[4], a[1], a[5], xv.x, xv.y);
+                            mma_f16_16816(acc, a[2], a[6], a[3], a[7], xv.z, xv.w);
+                        } else {
+                            mma_bf16_16816(acc, a[0], a[4], a[1], a[5], xv.x, xv.y);
+                            mma_bf16_16816(acc, a[2], a[6], a[3], a[7], xv.z, xv.w);
+                        }
+                    } else {
+                        const uint32_t col = col0 + kb * 32u;
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            if ((uint64_t)rg * 16 + g + 8 * h >= k.rows || col >= (uint32_t)k.cols) continue;
+                            uint16_t *dst = out0 + (uint64_t)(8 * h) * k.cols + kb * 32u;
+                            if (k.cols % 8 == 0) {
+                                *(uint4 *)dst = make_uint4(a[4 * h], a[4 * h + 1], a[4 * h + 2], a[4 * h + 3]);
+                            } else {
+#pragma unroll
+                                for (int i = 0; i < 8; ++i)
+                                    if (col + i < (uint32_t)k.cols) dst[i] = (uint16_t)(a[4 * h + (i >> 1)] >> (16 * (i & 1)));
+                            }
+                        }
+                    }
+                };
+                constexpr std::integral_constant<bool, false> inner{};
+                constexpr std::integral_constant<bool, true> maybe_last{};
+                uint32_t kb = 0;
+#pragma unroll 1
+                for (; kb + 4 <= nkb; kb += 4) {                    // the usual case: groups of four blocks
+                    block(kb, raw_a, raw_b, inner);
+                    block(kb + 1, raw_b, raw_a, inner);
+                    block(kb + 2, raw_a, raw_b, inner);
+                    block(kb + 3, raw_b, raw_a, maybe_last);
+                }
+#pragma unroll 1
+                for (; kb < nkb; kb += 2) {
+                    block(kb, raw_a, raw_b, maybe_last);
+                    if (kb + 1 < nkb) block(kb + 1, raw_b, raw_a, maybe_last);
+                }
+                if (nkb & 1u) raw_a = raw_b;     // the next chunk's first block always starts in raw_a
+                primed = has_next;
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar_cur + 16);                 // the slot goes back to the feeder
+            par ^= which;                                         // 0, 0, 1, 1, 0, 0, ...
+            which ^= 1u;
+            slot_cur ^= slot_tog;
+            bar_cur ^= 8u;
+            note_cur ^= 8u;
+            kc = kc + 1 == KC ? 0u : kc + 1;
+            if (kc == 0) {                                        // the next chunk starts the next row group: back to column 0
+                ++rg;
+                if (MODE == 1) xq -= k.cols;
+            }
         }
+        if (MODE == 1) flush(cur_rg, c_beg, c_end);
     }
 }
 
