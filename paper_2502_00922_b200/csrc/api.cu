@@ -478,7 +478,7 @@ huffllm_status huffllm_plain_gemv_multi(uint32_t n, const uint16_t *const *ws, c
     PlainArgs a;
     memset(&a, 0, sizeof(a));
     a.n_mats = n;
-    uint64_t pairs = 0;
+    uint64_t total = 0;
     for (uint32_t i = 0; i < n; ++i) {
         if (!ws[i] || !xs[i] || !ys[i] || rows[i] == 0 || cols[i] == 0) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer or empty matrix");
         if (cols[i] % 8 || ((uintptr_t)ws[i] & 15) || ((uintptr_t)xs[i] & 15))
@@ -488,11 +488,11 @@ huffllm_status huffllm_plain_gemv_multi(uint32_t n, const uint16_t *const *ws, c
         a.m[i].y = ys[i];
         a.m[i].rows = rows[i];
         a.m[i].cols = cols[i];
-        a.m[i].pair_first = (uint32_t)pairs;
-        pairs += (rows[i] + 1) / 2;
-        if (pairs >= (1ull << 31)) return fail(HUFFLLM_ERR_UNSUPPORTED, "too many rows for one launch");
+        a.m[i].row_first = (uint32_t)total;
+        total += rows[i];
+        if (total >= (1ull << 31)) return fail(HUFFLLM_ERR_UNSUPPORTED, "too many rows for one launch");
     }
-    a.total_pairs = (uint32_t)pairs;
+    a.total_rows = (uint32_t)total;
     cudaError_t e = launch_plain_gemv(a, (uint32_t)dev.sms, (cudaStream_t)stream);
     if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "plain gemv launch: %s", cudaGetErrorString(e));
     return HUFFLLM_OK;

@@ -470,10 +470,10 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
 
 // The dense product the compressed path competes with: y = W x for uncompressed bf16 matrices, written as a streaming
 // kernel so that it is a fair opponent.  One launch takes a list of matrices (the same launch groups as the compressed
-// path).  A warp takes two rows at a time and walks them 2 KB per step: eight independent 16-byte loads per lane are in
-// flight before the first is used (32 warps per SM: about 128 KB per SM on its way, several times what the memory
-// latency times an SM's share of the bandwidth asks for); x comes from L1 and is shared by the two rows; products in
-// fp32, shuffle reduction.  Row pairs are dealt round-robin to the warps of the grid.
+// path).  A warp takes one row at a time and walks it 4 KB per step: eight independent 16-byte loads per lane are in
+// flight before the first is used (32 warps per SM: 128 KB per SM on its way, several times what the memory latency
+// times an SM's share of the bandwidth asks for); x comes from L1; products in fp32, shuffle reduction.  Rows are dealt
+// round-robin to the warps of the grid, so every SM keeps loads in flight until the launch ends.
 __device__ __forceinline__ void fma_bf16x8(float &lo, float &hi, const uint4 &w, const uint4 &x) {
     const uint32_t wv[4] = {w.x, w.y, w.z, w.w}, xv[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
@@ -487,45 +487,28 @@ __global__ void __launch_bounds__(256, 4) plain_gemv_kernel(const __grid_constan
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
     uint32_t mi = 0;
-    for (uint32_t u = warp; u < A.total_pairs; u += nwarps) {
-        while (mi + 1 < A.n_mats && u >= A.m[mi + 1].pair_first) ++mi;
+    for (uint32_t u = warp; u < A.total_rows; u += nwarps) {
+        while (mi + 1 < A.n_mats && u >= A.m[mi + 1].row_first) ++mi;
         const PlainMat &m = A.m[mi];
-        const uint64_t r = 2ull * (u - m.pair_first);
-        const bool two = r + 1 < m.rows;
+        const uint64_t r = u - m.row_first;
         const uint32_t nv = (uint32_t)(m.cols >> 3);                       // 16-byte pieces of a row
-        const uint4 *w0 = (const uint4 *)(m.w + r * m.cols), *w1 = two ? w0 + nv : w0;
-        const uint4 *xr = (const uint4 *)m.x;
+        const uint4 *wr = (const uint4 *)(m.w + r * m.cols), *xr = (const uint4 *)m.x;
         float a0 = 0.f, a1 = 0.f, b0 = 0.f, b1 = 0.f;
-        uint32_t i = lane;
-        for (; i + 96 < nv; i += 128) {                                    // four pieces of each row per lane and step
-            uint4 p[4], q[4], xv[4];
+        for (uint32_t i = lane; i < nv; i += 256) {                        // eight pieces per lane and step
+            uint4 p[8];
 #pragma unroll
-            for (int j = 0; j < 4; ++j) p[j] = ldg_stream16(w0 + i + 32 * j);
+            for (int j = 0; j < 8; ++j) p[j] = i + 32 * j < nv ? ldg_stream16(wr + i + 32 * j) : make_uint4(0, 0, 0, 0);
 #pragma unroll
-            for (int j = 0; j < 4; ++j) q[j] = ldg_stream16(w1 + i + 32 * j);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) xv[j] = __ldg(xr + i + 32 * j);
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                fma_bf16x8(a0, a1, p[j], xv[j]);
-                fma_bf16x8(b0, b1, q[j], xv[j]);
+            for (int j = 0; j < 8; ++j) {
+                const uint4 xv = i + 32 * j < nv ? __ldg(xr + i + 32 * j) : make_uint4(0, 0, 0, 0);
+                if (j & 1) fma_bf16x8(b0, b1, p[j], xv);
+                else fma_bf16x8(a0, a1, p[j], xv);
             }
         }
-        for (; i < nv; i += 32) {
-            const uint4 p = ldg_stream16(w0 + i), q = ldg_stream16(w1 + i), xv = __ldg(xr + i);
-            fma_bf16x8(a0, a1, p, xv);
-            fma_bf16x8(b0, b1, q, xv);
-        }
-        float sa = a0 + a1, sb = b0 + b1;
+        float sum = (a0 + a1) + (b0 + b1);
 #pragma unroll
-        for (int o = 16; o; o >>= 1) {
-            sa += __shfl_xor_sync(0xFFFFFFFFu, sa, o);
-            sb += __shfl_xor_sync(0xFFFFFFFFu, sb, o);
-        }
-        if (lane == 0) {
-            m.y[r] = sa;
-            if (two) m.y[r + 1] = sb;
-        }
+        for (int o = 16; o; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+        if (lane == 0) m.y[r] = sum;
     }
 }
 
@@ -584,7 +567,7 @@ cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream)
 }
 
 cudaError_t launch_plain_gemv(const PlainArgs &a, uint32_t sms, cudaStream_t stream) {
-    const uint64_t blocks = ((uint64_t)a.total_pairs + 7) / 8;              // 8 warps per CTA, a row pair per warp and turn
+    const uint64_t blocks = ((uint64_t)a.total_rows + 7) / 8;               // 8 warps per CTA, a row per warp and turn
     const uint32_t grid = (uint32_t)(blocks < (uint64_t)sms * 4 ? blocks : (uint64_t)sms * 4);
     plain_gemv_kernel<<<grid, 256, 0, stream>>>(a);
     return cudaGetLastError();

@@ -48,16 +48,16 @@ cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t strea
 cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream);
 cudaError_t launch_gemm_tc(const KernelArgs &k, uint32_t grid, cudaStream_t stream);
 cudaError_t launch_stage_copy(void *dst, const void *src, uint64_t bytes, uint32_t sms, cudaStream_t stream);
-// The dense bf16 comparison product: up to kMaxMats matrices per launch, rows dealt to the warps in pairs.
+// The dense bf16 comparison product: up to kMaxMats matrices per launch, rows dealt to the warps round-robin.
 struct PlainMat {
     const uint16_t *w;         // [rows][cols] bf16, device
     const uint16_t *x;         // [cols]
     float *y;                  // [rows]
     uint64_t rows, cols;
-    uint32_t pair_first;       // number of the matrix's first row pair among the launch's row pairs
+    uint32_t row_first;        // number of the matrix's first row among the launch's rows
 };
 struct PlainArgs {
-    uint32_t n_mats, total_pairs;
+    uint32_t n_mats, total_rows;
     PlainMat m[kMaxMats];
 };
 cudaError_t launch_plain_gemv(const PlainArgs &a, uint32_t sms, cudaStream_t stream);
