@@ -346,7 +346,7 @@ def main():
                     help="which matrices of the layer share a launch")
     ap.add_argument("--split", default="paper", choices=["paper", "whole-exponent"],
                     help="field split of the blobs: the paper's BF16 {1,4,4,7} or {1,8,7} (one 256-symbol exponent code)")
-    ap.add_argument("--max-code-len", type=int, default=0, help="L_max of the codebooks (0 = the library's default, 8; the kernels take 8 or 9)")
+    ap.add_argument("--max-code-len", type=int, default=0, help="L_max of the codebooks (0 = the library's default, 8; range 8..12, Section 3.2 quotes 12; above 9 the kernels look long codewords up in two levels)")
     ap.add_argument("--dtype", default="bf16", choices=["bf16", "fp16", "fp16_from_bf16"],
                     help="weight format: bf16 {1,4,4,7} blobs, or fp16 {1,5,5,5} blobs of true fp16 weights / of bf16 weights "
                          "stored as fp16 (use --chunk-elems 1024 for fp16: larger records do not fit 32 warps' slots)")

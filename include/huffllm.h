@@ -142,8 +142,11 @@ typedef struct huffllm_desc {
  * the result is plain Huffman.  0 selects the default (8); supported range 8..12.
  * A field with a single used symbol gets a 1-bit code.  An empty tensor is INVALID_ARG.
  * HUFFLLM_FP16 is the paper's {1,5,5,5} split (Section 3.1): sign raw, exponent and the two mantissa halves each
- * with its own code, each limited to max_code_len on its own (Section 3.2 quotes 12 for these 5-bit fields; the
- * device kernels take 8).  On success *out owns a new codebook.
+ * with its own code, each limited to max_code_len on its own (Section 3.2 quotes 12 for these 5-bit fields).
+ * The device kernels decode every limit from 8 to 12: up to 8 bits per field (FP16) or 9 bits per weight (BF16)
+ * with one table lookup per codeword, longer codes with a second lookup for the codewords that exceed 8 bits
+ * (slower by the extra instructions; small batches above 8 vectors then run as passes of 8).
+ * On success *out owns a new codebook.
  */
 huffllm_status huffllm_build_codebook(const uint16_t *w_host, uint64_t rows, uint64_t cols, huffllm_dtype dtype,
                                       uint32_t max_code_len, huffllm_codebook **out);

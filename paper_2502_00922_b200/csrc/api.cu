@@ -128,8 +128,7 @@ huffllm_status add_matrix(KernelArgs *k, const huffllm_desc *desc, const void *b
     if (st != HUFFLLM_OK) return st;
     if (!blob || ((uintptr_t)blob & 255)) return fail(HUFFLLM_ERR_INVALID_ARG, "blob must be a 256-byte aligned device pointer");
     const uint32_t fmt = desc->dtype == HUFFLLM_FP16 ? 1u : 0u;
-    if (desc->lut_bits > (fmt ? 8u : 9u))
-        return fail(HUFFLLM_ERR_UNSUPPORTED, "device kernels take max_code_len 8%s (this blob: %u)", fmt ? "" : " or 9", desc->lut_bits);
+
     if (k->n_mats && k->fmt != fmt) return fail(HUFFLLM_ERR_UNSUPPORTED, "matrices of one call must share the dtype");
     k->fmt = fmt;
     if (k->n_mats == kMaxMats) return fail(HUFFLLM_ERR_UNSUPPORTED, "at most %u matrices per call", kMaxMats);
@@ -149,13 +148,18 @@ huffllm_status add_matrix(KernelArgs *k, const huffllm_desc *desc, const void *b
     m.col_chunks = desc->col_chunks;
     k->total_chunks += m.n_chunks;
     k->lut_bits = desc->lut_bits;
-    k->lut_align = fmt ? 16384u : 128u << desc->lut_bits;
-    k->lut_size = fmt ? 49152u : 128u << desc->lut_bits;
+    // BF16 tables of up to 9 bits are replicated per lane; longer ones are looked up in two levels: a per-lane table of the
+    // first 8 bits, then one copy of the whole table behind it
+    // (FP16: three sixteen-fold tables of 8 bits; fields of 9 bits and more take the second level too)
+    const bool two_level = desc->lut_bits > (fmt ? 8u : 9u);
+    k->lut_align = fmt ? 16384u : 128u << (two_level ? 8u : desc->lut_bits);
+    k->lut_size = fmt ? 49152u + (two_level ? 3u * (4u << desc->lut_bits) : 0u)
+                      : (two_level ? (128u << 8) + (4u << desc->lut_bits) : 128u << desc->lut_bits);
     // a slot holds the W rows of a record; the window runs one row ahead of what it consumes, and that look-ahead
     // past the last row lands in the next slot, the table or the guard area and is never used
     uint32_t slot = desc->max_words * 256;
     // a corrupt stream can advance its read pointer by one row per refill check and no further
-    const uint32_t checks_per_block = fmt ? 8 : (desc->lut_bits == 8 ? 3 : 4);
+    const uint32_t checks_per_block = fmt ? (two_level ? 24 : 8) : (desc->lut_bits == 8 ? 3 : 4);
     uint32_t guard = 256 * (3 + checks_per_block * (desc->chunk_cols / kBlockCols));
     if (slot > k->slot_bytes) k->slot_bytes = slot;
     k->pair_recip = (uint32_t)(0x100000000ull / (2ull * k->slot_bytes));
@@ -300,8 +304,9 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
     if (st != HUFFLLM_OK) return st;
     if (batch == 0 || batch > 64) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be in [1, 64]");
     if ((st = check_product_args(desc, x, y, workspace, workspace_bytes, batch)) != HUFFLLM_OK) return st;
-    if (batch > kKernelBatch) {
-        // tensor-core path: one pass over the compressed weights for the whole batch
+    if (batch > kKernelBatch && desc->lut_bits <= (desc->dtype == HUFFLLM_FP16 ? 8u : 9u)) {
+        // tensor-core path: one pass over the compressed weights for the whole batch (tables of up to 9 bits; longer
+        // codes take passes of 8 vectors through the register-path kernel and its two-level lookup)
         const TcPlan tp = tc_plan(desc, batch, (uint32_t)dev.sms, (uint32_t)dev.smem_optin - kStaticSmem);
         KernelArgs k;
         uint32_t grid;

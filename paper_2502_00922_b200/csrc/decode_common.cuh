@@ -132,6 +132,22 @@ __device__ __forceinline__ uint32_t stream_step(LaneStream &s, uint32_t idx_mask
     return e;
 }
 
+// Tables of 10 to 12 index bits (Section 3.2 quotes L_max = 12) are looked up in two levels.  The first level is the
+// 256-entry table of the first 8 stream bits, replicated per lane like the 8-bit table; an entry whose codeword is longer
+// than 8 bits carries a mark (bit 31) instead of a result, and the lane then reads the entry from the whole table
+// (one copy in shared memory, indexed by all lut_bits bits; bank conflicts there do not matter: long codewords are
+// rare).  full_mask = ((1 << lut_bits) - 1) << 2 turns the shifted window into that table's byte offset.
+constexpr uint32_t kLongMark = 0x80000000u;
+__device__ __forceinline__ uint32_t stream_step_long(LaneStream &s, uint32_t lut_lane, uint32_t full_base, uint32_t full_mask) {
+    uint64_t win = ((uint64_t)s.hi << 32) | s.lo;
+    uint32_t t = (uint32_t)(win >> s.pos), addr;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(addr) : "r"(t), "r"(0xFFu << 7), "r"(lut_lane));
+    uint32_t e = lds_lut(addr);
+    if (e & kLongMark) e = lds_lut(full_base + ((t >> 5) & full_mask));   // (t >> 7) is the index: times 4 bytes
+    s.pos = __dp4a(e, 0x00010000u, s.pos);
+    return e;
+}
+
 // The decoder of 8-bit BF16 tables works on four codewords at a time.  Its pointer stands on the codeword itself (the
 // sequence's leading zero bits are skipped when the sequence is opened), so after a refill check, with the pointer
 // below 32, the low 32 bits of the shifted window are all valid: room for four codewords of at most 8 bits.
@@ -238,9 +254,9 @@ __device__ __forceinline__ uint32_t rotr8(uint32_t v) { return prmt(v, v, 0x0321
 // The lane's two sequences are stepped alternately.  Each window is checked for a refill before every
 // R-th step: after a check at least 26 bits are valid in front of the start pointer, enough for R
 // codewords of at most 26/R bits.
-template <int R, bool SKIP = false>
+template <int R, bool SKIP = false, bool LONG = false>
 __device__ __forceinline__ void decode_block(LaneStream &sa, LaneStream &sb, uint32_t idx_mask, uint32_t lut_lane,
-                                             const uint4 &raw, uint32_t (&a)[8]) {
+                                             const uint4 &raw, uint32_t (&a)[8], uint32_t full_base = 0, uint32_t full_mask = 0) {
     uint32_t e[16];
     if (SKIP) {
         stream_step4x2(sa, sb, lut_lane, e, e + 8);
@@ -252,8 +268,13 @@ __device__ __forceinline__ void decode_block(LaneStream &sa, LaneStream &sb, uin
             stream_refill(sa);
             stream_refill(sb);
         }
-        e[i] = stream_step(sa, idx_mask, lut_lane);
-        e[8 + i] = stream_step(sb, idx_mask, lut_lane);
+        if (LONG) {
+            e[i] = stream_step_long(sa, lut_lane, full_base, full_mask);
+            e[8 + i] = stream_step_long(sb, lut_lane, full_base, full_mask);
+        } else {
+            e[i] = stream_step(sa, idx_mask, lut_lane);
+            e[8 + i] = stream_step(sb, idx_mask, lut_lane);
+        }
     }
     a[0] = pack_pair(e[0], e[1], raw.x);
     a[1] = pack_pair(e[2], e[3], rotr8(raw.x));
@@ -288,17 +309,46 @@ __device__ __forceinline__ uint32_t fp16_weight(LaneStream &s, uint32_t lut_lane
     asm("lop3.b32 %0, %1, %2, %3, 0xFE;" : "=r"(w) : "r"(e0), "r"(e1), "r"(e2));
     return w;                                      // low 16 bits: exponent and mantissa; above: the three lengths mixed
 }
+// Field codes of 9 to 12 bits (Section 3.2: L_max = 12 for the 5-bit fields): two levels, as for BF16.  The first level is
+// the field's sixteen-fold table of the first 8 bits; a marked entry sends the lane to the field's whole table
+// (1 << lut_bits entries, one copy; the three follow each other from full_base).  A codeword may now take 12 bits, so the
+// window is checked before every field (pointer below 32: lag 6 + 12 bits end inside the 64-bit window).
+__device__ __forceinline__ uint32_t fp16_field_long(LaneStream &s, uint32_t lut_lane, uint32_t table_off, uint32_t full_addr,
+                                                    uint32_t full_mask) {
+    stream_refill<false>(s);
+    uint64_t win = ((uint64_t)s.hi << 32) | s.lo;
+    uint32_t t = (uint32_t)(win >> s.pos), addr, e;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(addr) : "r"(t), "r"(0xFFu << 6), "r"(lut_lane));
+    asm("ld.shared.u32 %0, [%1];" : "=r"(e) : "r"(addr + table_off));
+    if (e & kLongMark) e = lds_lut(full_addr + ((t >> 4) & full_mask));     // (t >> 6) is the index: times 4 bytes
+    s.pos = __dp4a(e, 0x00010000u, s.pos);
+    return e;
+}
+__device__ __forceinline__ uint32_t fp16_weight_long(LaneStream &s, uint32_t lut_lane, uint32_t full_base, uint32_t full_mask) {
+    const uint32_t table_bytes = full_mask + 4u;                            // bytes of one field's whole table
+    uint32_t e0 = fp16_field_long(s, lut_lane, 0, full_base, full_mask);
+    uint32_t e1 = fp16_field_long(s, lut_lane, 16384, full_base + table_bytes, full_mask);
+    uint32_t e2 = fp16_field_long(s, lut_lane, 32768, full_base + 2u * table_bytes, full_mask), w;
+    asm("lop3.b32 %0, %1, %2, %3, 0xFE;" : "=r"(w) : "r"(e0), "r"(e1), "r"(e2));
+    return w;
+}
 // Decode one block of an FP16 chunk into 8 packed registers (same order as decode_block).  `signs` is the lane's
 // uint16 of the block: bit p = sign of the first weight of pair p, bit 8 + p = sign of its second weight.
+template <bool LONG = false>
 __device__ __forceinline__ void decode_block_fp16(LaneStream &sa, LaneStream &sb, uint32_t lut_lane, uint32_t signs,
-                                                  uint32_t (&a)[8]) {
+                                                  uint32_t (&a)[8], uint32_t full_base = 0, uint32_t full_mask = 0) {
     uint32_t w[16];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        stream_refill<false>(sa);
-        stream_refill<false>(sb);
-        w[i] = fp16_weight(sa, lut_lane);
-        w[8 + i] = fp16_weight(sb, lut_lane);
+        if (LONG) {
+            w[i] = fp16_weight_long(sa, lut_lane, full_base, full_mask);
+            w[8 + i] = fp16_weight_long(sb, lut_lane, full_base, full_mask);
+        } else {
+            stream_refill<false>(sa);
+            stream_refill<false>(sb);
+            w[i] = fp16_weight(sa, lut_lane);
+            w[8 + i] = fp16_weight(sb, lut_lane);
+        }
     }
     const uint32_t s32 = prmt(signs, 0u, 0x4140u);     // first-weight signs in bits 0..7, second-weight signs in bits 16..23
 #pragma unroll

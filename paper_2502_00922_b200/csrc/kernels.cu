@@ -36,7 +36,8 @@ namespace huffllm {
 // ------------------------------------------------------------------------------ the fused kernel
 
 // MODE 0: write the decoded weights.  MODE 1: y = W x for up to 8 activation vectors.
-// LB = table index bits (the blobs' lut_bits): 8 or 9.
+// LB = table index bits (the blobs' lut_bits): 8 or 9; LB = 12 stands for every longer limit up to 12 (BF16: 10..12,
+// FP16: 9..12): two-level lookup, the number of bits is A.lut_bits.
 // FMT = 0: BF16 blobs; FMT = 1: FP16 {1,5,5,5} blobs (three lookups per weight, sign bits as the raw part).
 //
 // One launch works through a LIST of matrices (A.n_mats, usually the matrices of one decoder layer that
@@ -58,8 +59,10 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     // 8-bit BF16 tables: the decoder starts behind the sequences' leading zero bits and works on four codewords at a
     // time (stream_step4x2)
     constexpr bool SKIP = LB == 8 && FMT == 0;
+    constexpr bool LONG = LB > 9;                            // first level of 8 bits, then the whole table (FP16: lut_bits 9..12)
+    constexpr uint32_t kLB1 = LONG ? 8u : (uint32_t)LB;      // index bits of the per-lane table
     constexpr int R = SKIP ? 4 : LB == 8 ? 3 : 2;            // decoder steps between two refill checks
-    constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
+    constexpr uint32_t kIdxMask = ((1u << kLB1) - 1u) << 7;
     extern __shared__ __align__(128) uint8_t dyn_smem[];
     // per decoder warp: "full" barriers of its two slots (the copy has landed), then the two "empty" ones (the decoder is done)
     __shared__ __align__(16) uint64_t bars[kMaxWarps * 4];
@@ -164,7 +167,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     // written to shared memory (by the decoder warps alone: the feeder is already asking for records)
     // (FP16: three tables of 256 entries, sixteen copies each: word j holds entry j / 16 of its table)
     // The table goes to shared memory in 16-byte pieces: four neighbouring copies of one entry per piece.
-    constexpr uint32_t kLutWords = FMT ? 3u * 16u * 256u : 32u << LB;
+    constexpr uint32_t kLutWords = FMT ? 3u * 16u * 256u : 32u << kLB1;
     constexpr uint32_t kLutRep = FMT ? 4u : 5u;            // log2 of the copies per entry
     constexpr uint32_t kLutVecs = kLutWords / 4;
     constexpr uint32_t kLutThreads = THREADS - 32;
@@ -175,10 +178,15 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
 #pragma unroll
         for (int i = 0; i < kLutLoads; ++i) {
             uint32_t v = tid + i * kLutThreads;
-            lut_v[i] = v < kLutVecs ? __ldg(lut_g + (v >> (kLutRep - 2))) : 0u;
+            // (entry of vector v: BF16 v / 8; FP16 field v / 1024, entry v / 4 % 256 of that field's table of 1 << lut_bits)
+            const uint32_t src = FMT ? ((v >> 10) << A.lut_bits) + ((v >> 2) & 255u) : v >> (kLutRep - 2);
+            lut_v[i] = v < kLutVecs ? __ldg(lut_g + src) : 0u;
             if (SKIP) lut_v[i] = lut_entry_inplace(lut_v[i]);   // the length once more, where an in-place shift reads it
+            if (LONG && (lut_v[i] >> 16) > 8u) lut_v[i] |= kLongMark;   // a codeword longer than the first level resolves
         }
     }
+    // two-level lookup: the whole table (1 << lut_bits entries, one copy) sits behind the per-lane first level
+    const uint32_t full_base = plan.lut + (FMT ? 49152u : 128u << kLB1), full_mask = ((1u << A.lut_bits) - 1u) << 2;
     uint32_t lut_lane = plan.lut | ((FMT ? lane & 15u : lane) << 2);
     asm volatile("mov.u32 %0, %0;" : "+r"(lut_lane));  // keep it in a register: it is an operand of every lookup
     const uint32_t g = lane >> 2, t = lane & 3;
@@ -205,6 +213,11 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
             if (v < kLutVecs) lut_s[v] = make_uint4(lut_v[i], lut_v[i], lut_v[i], lut_v[i]);
         }
         if (tid < kMaxWarps) s_arrive[tid] = 0;
+        if (LONG) {
+            const uint32_t *lut_g = (const uint32_t *)(k.blob + k.off_lut);
+            uint32_t *full_s = (uint32_t *)(dyn_smem + (full_base - smem_base));
+            for (uint32_t i = tid; i < (FMT ? 3u : 1u) << A.lut_bits; i += kLutThreads) full_s[i] = __ldg(lut_g + i);
+        }
     }
     if (r_first < k.payload_units) {        // (the blob keeps 4 KB behind the payload: a block's read stays inside it)
         raw_p = payload + ((uint64_t)r_first << 7) + lane * kRawLane;
@@ -404,8 +417,8 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                     }
 
                     uint32_t a[8];
-                    if (FMT) decode_block_fp16(sa, sb, lut_lane, cur.x, a);
-                    else decode_block<R, SKIP>(sa, sb, kIdxMask, lut_lane, cur, a);
+                    if (FMT) decode_block_fp16<LONG>(sa, sb, lut_lane, cur.x, a, full_base, full_mask);
+                    else decode_block<R, SKIP, LONG>(sa, sb, kIdxMask, lut_lane, cur, a, full_base, full_mask);
 
                     if (MODE == 1) {
                         if (FMT) {
@@ -557,12 +570,14 @@ static cudaError_t launch_one(const KernelArgs &k, uint32_t grid, cudaStream_t s
 }
 
 cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
-    if (k.fmt) return launch_one<0, 8, kThreads, 1>(k, grid, stream);
+    if (k.fmt) return k.lut_bits > 8 ? launch_one<0, 12, kThreads, 1>(k, grid, stream) : launch_one<0, 8, kThreads, 1>(k, grid, stream);
+    if (k.lut_bits > 9) return launch_one<0, 12, kThreads, 0>(k, grid, stream);
     return k.lut_bits == 8 ? launch_one<0, 8, kThreads, 0>(k, grid, stream) : launch_one<0, 9, kThreads, 0>(k, grid, stream);
 }
 
 cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
-    if (k.fmt) return launch_one<1, 8, kThreads, 1>(k, grid, stream);
+    if (k.fmt) return k.lut_bits > 8 ? launch_one<1, 12, kThreads, 1>(k, grid, stream) : launch_one<1, 8, kThreads, 1>(k, grid, stream);
+    if (k.lut_bits > 9) return launch_one<1, 12, kThreads, 0>(k, grid, stream);
     return k.lut_bits == 8 ? launch_one<1, 8, kThreads, 0>(k, grid, stream) : launch_one<1, 9, kThreads, 0>(k, grid, stream);
 }
 

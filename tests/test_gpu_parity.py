@@ -97,6 +97,7 @@ def make(gen, rows, cols, seed):
             "student": lambda: wl.student_t_weights(rows, cols, seed),
             "uniform": lambda: wl.uniform_exponent_weights(rows, cols, seed),
             "patterns": lambda: wl.all_patterns_weights(rows, cols, seed),
+            "skewed": lambda: wl.skewed_exponent_weights(rows, cols, seed),
             "constant": lambda: np.full((rows, cols), 0xBD33, dtype=np.uint16)}[gen]()
 
 
@@ -132,7 +133,8 @@ def test_whole_exponent_split_decode_and_product(hl, torch, rows, cols, ce, budg
 FP16_GENS = {"fp16": lambda r, c, seed: wl.gaussian_weights(r, c, 0.02, seed, "fp16"),
              "fp16_from_bf16": lambda r, c, seed: wl.gaussian_weights(r, c, 0.02, seed, "fp16_from_bf16"),
              "patterns": lambda r, c, seed: wl.all_patterns_weights(r, c, seed),
-             "constant": lambda r, c, seed: np.full((r, c), 0xAE66, dtype=np.uint16)}
+             "constant": lambda r, c, seed: np.full((r, c), 0xAE66, dtype=np.uint16),
+             "skewed": lambda r, c, seed: wl.skewed_exponent_weights(r, c, seed, dtype="fp16")}
 
 
 @pytest.mark.parametrize("rows,cols,ce,gen,batch", [
@@ -160,6 +162,31 @@ def test_fp16_decode_and_product(hl, torch, rows, cols, ce, gen, batch):
         assert np.array_equal(ref, w)
     if batch:
         x = wl.activations(batch, cols, 950 + cols, "fp16")
+        check_product(gpu_gemm(hl, torch, up, x), w, x, orc.FP16)
+
+
+@pytest.mark.parametrize("rows,cols,ce,budget,gen,batch", [
+    (256, 1024, 1024, 12, "skewed", 1),           # Section 3.2's L_max = 12: geometric laws in all three fields, long codewords occur
+    (128, 2048, 512, 10, "skewed", 5),
+    (1024, 1024, 1024, 12, "fp16", 3),            # true fp16 weights under the longer limit
+    (37, 300, 512, 9, "skewed", 0),               # ragged, 9 bits (decode only)
+    (256, 2048, 1024, 12, "patterns", 0),         # every bit pattern (decode only)
+    (64, 1024, 1024, 12, "skewed", 16),           # batch above 8: passes of 8 vectors
+])
+def test_fp16_long_field_codes_decode_and_product(hl, torch, rows, cols, ce, budget, gen, batch):
+    """FP16 {1,5,5,5} blobs whose field codes are limited to 9..12 bits: two-level lookup on the device."""
+    w = FP16_GENS[gen](rows, cols, 1400 + rows + budget)
+    up = Uploaded(hl, torch, w, ce, budget, max(batch, 1), dtype=hl.FP16)
+    assert (up.desc.dtype, up.desc.lut_bits) == (hl.FP16, budget)
+    if gen == "skewed":
+        lut = up.blob[up.desc.off_lut:up.desc.off_lut + 3 * (4 << budget)].view(np.uint32)
+        assert int(((lut >> 16) > 8).sum()) > 0, "the case should contain codewords longer than the first level"
+    assert np.array_equal(gpu_decode(hl, torch, up), w)
+    if rows * cols <= 600_000:
+        ref, _ = orc.decode_blob(up.blob)
+        assert np.array_equal(ref, w)
+    if batch:
+        x = wl.activations(batch, cols, 1450 + cols, "fp16")
         check_product(gpu_gemm(hl, torch, up, x), w, x, orc.FP16)
 
 
@@ -203,6 +230,37 @@ def test_fused_product_matches_oracle(hl, torch, rows, cols, ce, budget, gen, ba
     check_product(y1, w, x)
     y2 = gpu_gemm(hl, torch, up, x)
     assert np.array_equal(y1, y2), "results must be bitwise reproducible"
+
+
+@pytest.mark.parametrize("rows,cols,ce,budget,gen,batch,split", [
+    (1024, 1024, 4096, 12, "gauss", 1, 0),        # the small benchmark configuration with the paper's L_max
+    (256, 2048, 4096, 10, "skewed", 5, 0),        # geometric exponents: codewords of 9 and 10 bits do occur
+    (256, 2048, 4096, 12, "skewed", 1, 0),        # ... and of 11 and 12
+    (96, 4096, 4096, 11, "student", 3, 0),
+    (256, 2048, 4096, 12, "patterns", 0, 0),      # every bit pattern (decode only)
+    (37, 300, 1024, 12, "skewed", 0, 0),          # ragged rows and columns (decode only)
+    (272, 2080, 16384, 12, "skewed", 8, 0),       # largest chunks, ragged last column chunk
+    (512, 4096, 4096, 12, "skewed", 4, 1),        # one 256-symbol exponent code of up to 12 bits
+    (128, 1024, 1024, 12, "skewed", 16, 0),       # batch above 8: passes of 8 vectors through the two-level kernel
+])
+def test_long_code_tables_decode_and_product(hl, torch, rows, cols, ce, budget, gen, batch, split):
+    """max_code_len 10..12 (Section 3.2 quotes L_max = 12): the device looks codewords up in two levels.  Decode is
+    bit-exact and products stay within the tolerance, against the oracle."""
+    w = make(gen, rows, cols, 1200 + rows + budget)
+    up = Uploaded(hl, torch, w, ce, budget, max(batch, 1), split=split)
+    assert up.desc.lut_bits == budget
+    if gen == "skewed":                            # the case is only worth its name if long codewords are really there
+        lut = up.blob[up.desc.off_lut:up.desc.off_lut + (4 << budget)].view(np.uint32)
+        assert int(((lut >> 16) > 8).sum()) > 0
+    assert np.array_equal(gpu_decode(hl, torch, up), w)
+    if rows * cols <= 600_000:
+        ref, _ = orc.decode_blob(up.blob)
+        assert np.array_equal(ref, w)
+    if batch:
+        x = wl.activations(batch, cols, 1300 + cols)
+        y1 = gpu_gemm(hl, torch, up, x)
+        check_product(y1, w, x)
+        assert np.array_equal(y1, gpu_gemm(hl, torch, up, x)), "results must be bitwise reproducible"
 
 
 @pytest.mark.parametrize("batch", [1, 3])
@@ -320,10 +378,7 @@ def test_unsupported_requests_fail_before_launch(hl, torch):
         hl.decode_gemv(up.desc, up.blob_dev, x, y, up.ws, up.ws_bytes, up.err)
     assert e.value.status_name == "UNSUPPORTED"
     w = wl.gaussian_weights(16, 512, 0.02, 15)
-    up = Uploaded(hl, torch, w, 512, budget=12)    # larger codes than the device table handles
-    with pytest.raises(hl.HuffllmError) as e:
-        hl.decode(up.desc, up.blob_dev, torch.zeros(16 * 512, dtype=torch.int16, device="cuda"), up.err)
-    assert e.value.status_name == "UNSUPPORTED"
+    up = Uploaded(hl, torch, w, 512)
     with pytest.raises(hl.HuffllmError) as e:      # misaligned blob pointer
         hl.decode(up.desc, up.blob_dev.data_ptr() + 8, torch.zeros(16 * 512, dtype=torch.int16, device="cuda"), up.err)
     assert e.value.status_name == "INVALID_ARG"

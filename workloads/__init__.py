@@ -24,6 +24,7 @@ __all__ = [
     "student_t_weights",
     "uniform_exponent_weights",
     "all_patterns_weights",
+    "skewed_exponent_weights",
     "activations",
     "LAYER_LLAMA7B",
     "LAYER_8B",
@@ -94,6 +95,25 @@ def all_patterns_weights(rows: int, cols: int, seed: int) -> np.ndarray:
         v = rng.integers(0, 65536, size=n, dtype=np.uint32).astype(np.uint16)
     rng.shuffle(v)
     return v.reshape(rows, cols)
+
+
+def skewed_exponent_weights(rows: int, cols: int, seed: int, e_top: int = 130, span: int = 28, dtype: str = "bf16") -> np.ndarray:
+    """Exponents with a geometric law: exponent e_top - j has probability proportional to 2^-j (j < span), sign and
+    mantissa uniform.  Such a field has Huffman codewords of every length up to about `span` bits, so every
+    length limit from 8 to 12 bites and long codewords do occur: the stress case for the longer decode tables.
+    Values stay finite and moderate.  dtype "fp16": the same law on the 5-bit exponent (e_top and span are clipped)."""
+    rng = np.random.default_rng(seed)
+    j = np.minimum(rng.geometric(0.5, size=(rows, cols)) - 1, span - 1).astype(np.int64)
+    s = rng.integers(0, 2, size=(rows, cols), dtype=np.uint16)
+    if dtype == "bf16":
+        e = (e_top - j).astype(np.uint16)
+        m = rng.integers(0, 128, size=(rows, cols), dtype=np.uint16)
+        return ((s << 15) | (e << 7) | m).astype(np.uint16)
+    e = np.clip(min(e_top, 17) - j, 1, 30).astype(np.uint16)
+    # the mantissa halves follow the same kind of law, so that their codes grow long too
+    mh = np.minimum(rng.geometric(0.5, size=(rows, cols)) - 1, 31).astype(np.uint16)
+    ml = np.minimum(rng.geometric(0.5, size=(rows, cols)) - 1, 31).astype(np.uint16)
+    return ((s << 15) | (e << 10) | (mh << 5) | ml).astype(np.uint16)
 
 
 def activations(batch: int, cols: int, seed: int, dtype: str = "bf16") -> np.ndarray:
