@@ -229,11 +229,25 @@ huffllm_status huffllm_workspace_control_bytes(const huffllm_desc *desc, size_t 
 /*
  * Decompress a blob (device, 256-byte aligned) to its original 16-bit weights, bit for bit
  * (Section 3.2: sign, exponent and mantissa are concatenated back into the 16-bit weight).
- * `out` (device) receives rows*cols words, row-major.  `err_flag` (device int32, may be null) is
- * set non-zero if the kernel met an out-of-range record offset or a copy that never arrived.
+ * `out` (device) receives rows*cols words, row-major.  `err_flag` (device int32, may be null; the same in the
+ * product calls) is left alone by a sound blob and otherwise set to: c + 1 if chunk c's record offsets point outside
+ * the payload or do not fit (that chunk is skipped, nothing is read through them); 0x40000000 + c + 1 if chunk c's bits
+ * made the decoder run past the end of its record (a damaged coded part: the chunk's output is wrong, but no read left
+ * the CTA's shared memory: a sequence moves on by at most one row per refill check, and room for that is kept, see
+ * huffllm_decode_smem_plan); -1 if a copy never arrived within the wait limit.  A damaged coded part that still ends
+ * inside its record is not detectable here: huffllm_validate_blob (host, checksum) is the check for that.
  */
 huffllm_status huffllm_decode(const huffllm_desc *desc, const void *blob_dev, uint16_t *out_dev,
                               int32_t *err_flag_dev, huffllm_stream stream);
+
+/*
+ * The shared-memory budget a decoder CTA keeps for this blob (host call, no device needed; any pointer may be null):
+ * bytes of the decode table(s), bytes of one slot (the coded rows of the largest record: max_words * 256), the number
+ * of refill checks per bit sequence and block of 32 columns, and the readable bytes kept behind the last slot,
+ * 256 * (3 + checks * blocks per chunk): the furthest row any stream, sound or not, can make the decoder touch.
+ */
+huffllm_status huffllm_decode_smem_plan(const huffllm_desc *desc, uint32_t *table_bytes, uint32_t *slot_bytes,
+                                        uint32_t *refill_checks_per_block, uint32_t *guard_bytes);
 
 /*
  * y = W x with W taken straight from the compressed blob: weights are decoded in registers and

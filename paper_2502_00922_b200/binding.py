@@ -47,6 +47,7 @@ _SIGNATURES = {
     "huffllm_validate_blob": [C.c_void_p, C.c_size_t, C.POINTER(Desc)],
     "huffllm_workspace_bytes": [C.POINTER(Desc), C.c_uint32, C.POINTER(C.c_size_t)],
     "huffllm_workspace_control_bytes": [C.POINTER(Desc), C.POINTER(C.c_size_t)],
+    "huffllm_decode_smem_plan": [C.POINTER(Desc), C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)],
     "huffllm_decode": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemv": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemm": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
@@ -203,6 +204,13 @@ def workspace_control_bytes(desc: Desc) -> int:
     n = C.c_size_t()
     _check(lib().huffllm_workspace_control_bytes(C.byref(desc), C.byref(n)))
     return n.value
+
+
+def decode_smem_plan(desc: Desc) -> dict:
+    """huffllm_decode_smem_plan: table bytes, slot bytes, refill checks per block and guard bytes of a decoder CTA."""
+    t, sl, ch, g = C.c_uint32(), C.c_uint32(), C.c_uint32(), C.c_uint32()
+    _check(lib().huffllm_decode_smem_plan(C.byref(desc), C.byref(t), C.byref(sl), C.byref(ch), C.byref(g)))
+    return {"table_bytes": t.value, "slot_bytes": sl.value, "refill_checks_per_block": ch.value, "guard_bytes": g.value}
 
 
 def decode(desc: Desc, blob_dev, out_dev, err_flag_dev=None, stream=None):

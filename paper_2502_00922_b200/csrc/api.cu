@@ -115,6 +115,35 @@ TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn
     return p;
 }
 
+// What a blob asks of a decoder CTA's shared memory.
+struct SmemNeeds {
+    uint32_t table_align, table_bytes;   // window of the decode table(s)
+    uint32_t slot_bytes;                 // one slot: the W rows of the largest record
+    uint32_t checks_per_block;           // refill checks per bit sequence and block of 32 columns
+    uint32_t guard_bytes;                // readable bytes kept behind the last slot
+};
+SmemNeeds smem_needs(const huffllm_desc *desc) {
+    SmemNeeds n;
+    const bool fmt = desc->dtype == HUFFLLM_FP16;
+    // BF16 tables of up to 9 bits are replicated per lane; longer ones are looked up in two levels: a per-lane table of the
+    // first 8 bits, then one copy of the whole table behind it
+    // (FP16: three sixteen-fold tables of 8 bits; fields of 9 bits and more take the second level too)
+    const bool two_level = desc->lut_bits > (fmt ? 8u : 9u);
+    n.table_align = fmt ? 16384u : 128u << (two_level ? 8u : desc->lut_bits);
+    n.table_bytes = fmt ? 49152u + (two_level ? 3u * (4u << desc->lut_bits) : 0u)
+                        : (two_level ? (128u << 8) + (4u << desc->lut_bits) : 128u << desc->lut_bits);
+    // a slot holds the W rows of a record; the window runs one row ahead of what it consumes, and that look-ahead
+    // past the last row lands in the next slot, the table or the guard area and is never used
+    n.slot_bytes = desc->max_words * 256;
+    // A stream can move its read pointer by one row per refill check and no further, whatever its bits and whatever the
+    // table says: a sequence opens on rows 0 and 1, and every check loads at most the next row.  The furthest row a
+    // chunk's decoder can touch is therefore 1 + checks, counted from the slot's first row, and the bytes kept readable
+    // behind the last slot cover that for a slot of any size.
+    n.checks_per_block = fmt ? (two_level ? 24 : 8) : (desc->lut_bits == 8 ? 3 : 4);
+    n.guard_bytes = 256 * (3 + n.checks_per_block * (desc->chunk_cols / kBlockCols));
+    return n;
+}
+
 // Start a launch description.
 void begin_args(KernelArgs *k, uint32_t batch, const DeviceInfo &dev) {
     memset(k, 0, sizeof(*k));
@@ -148,22 +177,12 @@ huffllm_status add_matrix(KernelArgs *k, const huffllm_desc *desc, const void *b
     m.col_chunks = desc->col_chunks;
     k->total_chunks += m.n_chunks;
     k->lut_bits = desc->lut_bits;
-    // BF16 tables of up to 9 bits are replicated per lane; longer ones are looked up in two levels: a per-lane table of the
-    // first 8 bits, then one copy of the whole table behind it
-    // (FP16: three sixteen-fold tables of 8 bits; fields of 9 bits and more take the second level too)
-    const bool two_level = desc->lut_bits > (fmt ? 8u : 9u);
-    k->lut_align = fmt ? 16384u : 128u << (two_level ? 8u : desc->lut_bits);
-    k->lut_size = fmt ? 49152u + (two_level ? 3u * (4u << desc->lut_bits) : 0u)
-                      : (two_level ? (128u << 8) + (4u << desc->lut_bits) : 128u << desc->lut_bits);
-    // a slot holds the W rows of a record; the window runs one row ahead of what it consumes, and that look-ahead
-    // past the last row lands in the next slot, the table or the guard area and is never used
-    uint32_t slot = desc->max_words * 256;
-    // a corrupt stream can advance its read pointer by one row per refill check and no further
-    const uint32_t checks_per_block = fmt ? (two_level ? 24 : 8) : (desc->lut_bits == 8 ? 3 : 4);
-    uint32_t guard = 256 * (3 + checks_per_block * (desc->chunk_cols / kBlockCols));
-    if (slot > k->slot_bytes) k->slot_bytes = slot;
+    const SmemNeeds need = smem_needs(desc);
+    k->lut_align = need.table_align;
+    k->lut_size = need.table_bytes;
+    if (need.slot_bytes > k->slot_bytes) k->slot_bytes = need.slot_bytes;
     k->pair_recip = (uint32_t)(0x100000000ull / (2ull * k->slot_bytes));
-    if (guard > k->guard_bytes) k->guard_bytes = guard;
+    if (need.guard_bytes > k->guard_bytes) k->guard_bytes = need.guard_bytes;
     return HUFFLLM_OK;
 }
 
@@ -231,6 +250,19 @@ huffllm_status huffllm_workspace_control_bytes(const huffllm_desc *desc, size_t 
     huffllm_status st = check_desc(desc);
     if (st != HUFFLLM_OK) return st;
     *bytes = ws_partial_offset(desc);
+    return HUFFLLM_OK;
+}
+
+huffllm_status huffllm_decode_smem_plan(const huffllm_desc *desc, uint32_t *table_bytes, uint32_t *slot_bytes,
+                                        uint32_t *refill_checks_per_block, uint32_t *guard_bytes) {
+    clear_error();
+    huffllm_status st = check_desc(desc);
+    if (st != HUFFLLM_OK) return st;
+    const SmemNeeds n = smem_needs(desc);
+    if (table_bytes) *table_bytes = n.table_bytes;
+    if (slot_bytes) *slot_bytes = n.slot_bytes;
+    if (refill_checks_per_block) *refill_checks_per_block = n.checks_per_block;
+    if (guard_bytes) *guard_bytes = n.guard_bytes;
     return HUFFLLM_OK;
 }
 

@@ -406,6 +406,7 @@ __device__ __forceinline__ uint32_t slot_addr(const SmemPlan &p, uint32_t warp, 
 constexpr int kMaxWarps = 32;
 constexpr int kThreads = 1024;   // threads per CTA of the decode kernels (one CTA per SM)
 constexpr uint32_t kWaitLimit = 1u << 22;
+constexpr uint32_t kErrOverrun = 0x40000000u;     // error flag: this bit + (chunk + 1): the chunk's bits ran past its record
 constexpr uint32_t kFeederIdleLimit = 1u << 22;   // polls of 100 ns without any slot coming back before the feeder gives up
 
 }  // namespace huffllm

@@ -461,6 +461,13 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                 }
                 if (nkb & 1u) raw_a = raw_b;     // the next chunk's first block always starts in raw_a
                 primed = has_next;
+                // A sequence of a sound record ends inside the record's W rows, so its next-row pointer stands at most two
+                // rows behind them.  Bits that made the decoder run further (a damaged coded part) are reported; what was
+                // decoded from them is wrong, but every read stayed inside shared memory (one row per refill check at most).
+                const uint32_t row_limit = slot_cur + 512u + coded_bytes;
+                if (__any_sync(0xFFFFFFFFu, sa.nxt > row_limit || sb.nxt > row_limit + 128u)) {
+                    if (A.err && lane == 0) atomicExch(A.err, (int32_t)(kErrOverrun | min(c + 1, kErrOverrun - 1u)));
+                }
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(bar_cur + 16);                 // the slot goes back to the feeder

@@ -369,6 +369,52 @@ def test_bad_record_offsets_are_reported_not_followed(hl, torch):
     assert np.array_equal(got[good], w[good])
 
 
+def test_damaged_coded_part_is_reported_and_contained(hl, torch):
+    """The coded rows of one chunk are overwritten (on the host) with the longest codeword over and over, so that the
+    chunk's sequences run far past their record.  The kernels must say so in the error flag, stay inside their shared
+    memory (the read pointer moves one row per refill check at most, and room for that is kept), and decode every
+    other chunk as before."""
+    rows, cols = 64, 2048
+    w = wl.gaussian_weights(rows, cols, 0.02, 21)
+    up = Uploaded(hl, torch, w)
+    d = up.desc
+    blob = up.blob.copy()
+    lut = blob[d.off_lut:d.off_lut + (4 << d.lut_bits)].view(np.uint32)
+    longest = int(((lut >> 16) & 0xFF).max())
+    q = int(np.argmax((lut >> 16) & 0xFF))                       # eight stream bits that start a longest codeword
+    assert longest == 8                                            # (so the same byte follows it again)
+    idx = blob[d.off_index:d.off_index + 4 * (d.n_chunks + 1)].view(np.uint32)
+    victim = 5
+    nkb = d.chunk_cols // 32
+    beg, end = d.off_payload + 128 * int(idx[victim]) + 512 * nkb, d.off_payload + 128 * int(idx[victim + 1])
+    n_words = (end - beg) // 256                                   # W rows of 64 words
+    bits = np.zeros(32 * n_words, dtype=np.uint64)
+    i = np.arange(7, bits.size)
+    bits[7:] = (q >> ((i - 7) % 8)) & 1                            # 7 leading zero bits, then the byte for ever
+    words = (bits.reshape(n_words, 32) << np.arange(32, dtype=np.uint64)).sum(axis=1).astype(np.uint32)
+    blob[beg:end].view(np.uint32).reshape(n_words, 64)[:] = words[:, None]
+    with pytest.raises(hl.HuffllmError):
+        hl.validate_blob(blob)                                     # the host check (checksum, bit walk) refuses it
+    dev = torch.from_numpy(blob).cuda()
+    out = torch.zeros(rows * cols, dtype=torch.int16, device="cuda")
+    hl.decode(d, dev, out, up.err)
+    torch.cuda.synchronize()
+    assert int(up.err.item()) == 0x40000000 + victim + 1
+    got = out.cpu().numpy().view(np.uint16).reshape(rows, cols)
+    good = np.ones((rows, cols), dtype=bool)
+    rg, kc = divmod(victim, d.col_chunks)
+    good[rg * 16:(rg + 1) * 16, kc * d.chunk_cols:(kc + 1) * d.chunk_cols] = False
+    assert np.array_equal(got[good], w[good])
+    # the fused product reports it too and leaves its workspace usable
+    up.err.zero_()
+    x_dev = torch.from_numpy(wl.activations(1, cols, 22).view(np.int16)).cuda()
+    y = torch.zeros(rows, dtype=torch.float32, device="cuda")
+    hl.decode_gemv(d, dev, x_dev, y, up.ws, up.ws_bytes, up.err)
+    torch.cuda.synchronize()
+    assert int(up.err.item()) == 0x40000000 + victim + 1
+    assert int(up.ws[:hl.workspace_control_bytes(d)].count_nonzero().item()) == 0
+
+
 def test_unsupported_requests_fail_before_launch(hl, torch):
     w = wl.gaussian_weights(16, 520, 0.02, 14)     # cols not a multiple of 32
     up = Uploaded(hl, torch, w, 512)
