@@ -334,6 +334,58 @@ def small_batch_leg(hl, torch, dev, stream, chunk_elems: int, peak_for_small: fl
     return out
 
 
+def sweep_8b_leg(hl, torch, dev, stream, chunk_elems: int, peak: float, layers: int = 32):
+    """The per-token pass over an 8B-shaped model: `layers` decoder layers, every layer with its own copy of the seven
+    blobs in HBM (same content, distinct memory), four launches per layer, batch 1; beside it the dense bf16 sweep of the
+    same shapes in the same launch groups."""
+    mats = prepare("8b_layer", chunk_elems, hl, torch, dev)
+    table = WORKLOADS["8b_layer"][0]
+    groups = launch_groups(table, "deps")
+    err = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws_each = max(m["ws_bytes"] for m in mats)
+    blobs = [[m["blob_dev"] for m in mats]] + [[m["blob_dev"].clone() for m in mats] for _ in range(layers - 1)]
+    preps = [hl.PreparedMulti([mats[i]["desc"] for i in g], [bl[i] for i in g], [mats[i]["x_dev"] for i in g], 1,
+                              [mats[i]["y_dev"] for i in g], [mats[i]["ws"] for i in g], ws_each, err) for bl in blobs for g in groups]
+    raw = stream.cuda_stream
+
+    def timed(fn, n):
+        for _ in range(3):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record(stream)
+        for _ in range(n):
+            fn()
+        b.record(stream)
+        torch.cuda.synchronize()
+        return a.elapsed_time(b) / n
+
+    ms = timed(lambda: [p.run(raw) for p in preps], 30)
+    assert int(err.item()) == 0
+    n_w = layers * sum(r * c for _, r, c in table)
+    alg = layers * sum(m["alg_bytes"] for m in mats)
+    out = {"workload": f"8B-shaped model, {layers} layers, batch 1, {len(preps)} launches per token", "weights": n_w,
+           "compressed_bytes_resident": layers * sum(m["blob_bytes"] for m in mats), "ms_per_token": ms, "ms_per_layer": ms / layers,
+           "tokens_per_s_equiv": 1e3 / ms, "uncompressed_GBs": 2.0 * n_w / (ms * 1e-3) / 1e9,
+           "frac_of_hbm_peak_on_compressed_bytes": alg / (ms * 1e-3) / 1e9 / peak}
+    del preps, blobs
+    try:
+        dense = [[torch.empty((r, c), dtype=torch.int16, device=dev) for _, r, c in table] for _ in range(layers)]
+        for lw in dense:
+            for w_dev in lw:
+                w_dev.view(torch.bfloat16).normal_(0, 0.02)
+        dpreps = [hl.PreparedPlainMulti([lw[i] for i in g], [table[i][1] for i in g], [table[i][2] for i in g],
+                                        [mats[i]["x_dev"] for i in g], [mats[i]["y_dev"] for i in g]) for lw in dense for g in groups]
+        dms = timed(lambda: [p.run(raw) for p in dpreps], 30)
+        out["dense_bf16_ms_per_token"] = dms
+        out["speedup_vs_dense"] = dms / ms
+        del dense, dpreps
+    except Exception as ex:
+        print(f"[bench] dense sweep skipped: {ex}", file=sys.stderr)
+    torch.cuda.empty_cache()
+    return out
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -358,6 +410,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-small-batch", action="store_true",
                     help="skip the extra leg that times one 70B-FFN-shaped matrix at batch 1 / 16 / 64")
+    ap.add_argument("--no-sweep", action="store_true",
+                    help="skip the extra leg that sweeps 32 layers of the 8B-shaped model (11 GB of blobs resident)")
     ap.add_argument("--repeats", type=int, default=0,
                     help="timed regions of exactly --steps steps each (0: as many as fill about 0.8 s, so that the clock "
                          "sampler sees the GPU under load); the line's ms_per_step is the median region, min and max are reported")
@@ -688,6 +742,9 @@ def main():
     small_batch = None
     if rank == 0 and world == 1 and not args.no_small_batch and not fp16 and args.workload == "llama7b_layer" and L == 1:
         small_batch = small_batch_leg(hl, torch, dev, stream, args.chunk_elems, peak_for_small=measured_peak()[0])
+    sweep_8b = None
+    if rank == 0 and world == 1 and not args.no_sweep and not fp16 and args.workload == "llama7b_layer" and L == 1 and B == 1:
+        sweep_8b = sweep_8b_leg(hl, torch, dev, stream, args.chunk_elems, measured_peak()[0])
 
     if rank != 0:
         return
@@ -745,6 +802,7 @@ def main():
                             "note": "own streaming kernel in the same launch groups as the compressed path; the north star asks for "
                                     "speedup_vs_own_dense >= compression_ratio_total"},
         "small_batch": small_batch,
+        "sweep_8b_32_layers": sweep_8b,
         "cpu_baseline_all_cores": cpu_all,
         "timing": {"regions": R, "steps_per_region": args.steps, "ms_per_step_min": ms_min, "ms_per_step_median": ms_step,
                    "ms_per_step_max": ms_max, "note": "every region is exactly --steps steps between two CUDA events; the line's "
