@@ -299,7 +299,7 @@ def run_reference(args):
 
 
 def small_batch_leg(hl, torch, dev, stream, chunk_elems: int, peak_for_small: float):
-    """One 70B-FFN-shaped matrix (28672 x 8192) at batch 1, 16 and 64: ms per product, fraction of the HBM peak on the
+    """One 70B-FFN-shaped matrix (28672 x 8192) at batch 1, 16, 32 and 64: ms per product, fraction of the HBM peak on the
     compressed bytes, and which kernel ran."""
     name, rows, cols = wl.FFN_70B[0]
     w = wl.gaussian_weights(rows, cols, 0.015, 4000)
@@ -312,7 +312,7 @@ def small_batch_leg(hl, torch, dev, stream, chunk_elems: int, peak_for_small: fl
     ws_bytes = hl.workspace_bytes(desc, 64)
     ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
     out = {"matrix": f"{rows}x{cols}", "chunk_elems": chunk_elems, "compressed_bytes": int(desc.blob_bytes), "batches": []}
-    for batch in (1, 16, 64):
+    for batch in (1, 16, 32, 64):
         x = torch.from_numpy(wl.activations(batch, cols, 4500 + batch).view(np.int16).reshape(-1)).to(dev)
         y = torch.zeros(batch * rows, dtype=torch.float32, device=dev)
         for _ in range(5):
@@ -329,7 +329,9 @@ def small_batch_leg(hl, torch, dev, stream, chunk_elems: int, peak_for_small: fl
         alg = desc.payload_bytes + 4 * (desc.n_chunks + 1) + (4 << desc.lut_bits) + batch * (2 * cols + 4 * rows)
         out["batches"].append({"batch": batch, "ms": ms, "frac_of_hbm_peak": alg / (ms * 1e-3) / 1e9 / peak_for_small,
                                "uncompressed_GBs": 2.0 * rows * cols / (ms * 1e-3) / 1e9,
-                               "kernel": "huff_kernel<product> (mma.sync, registers)" if batch <= 8 else "huff_gemm_tc_kernel (tcgen05)"})
+                               "kernel": "huff_kernel<product> (mma.sync on the decoded registers)" if batch <= 8 else
+                                         ("huff_kernel<product, two tiles of activations> (mma.sync on the decoded registers)" if batch <= 16
+                                          else "huff_gemm_tc_kernel (tcgen05)")})
     assert int(err.item()) == 0
     return out
 
@@ -403,7 +405,8 @@ def main():
                     help="weight format: bf16 {1,4,4,7} blobs, or fp16 {1,5,5,5} blobs of true fp16 weights / of bf16 weights "
                          "stored as fp16 (use --chunk-elems 1024 for fp16: larger records do not fit 32 warps' slots)")
     ap.add_argument("--batch", type=int, default=1,
-                    help="activation vectors per product (1..64; above 8 every matrix is its own launch on the tcgen05 path)")
+                    help="activation vectors per product (1..64; above 8 every matrix is its own launch: 9..16 on the register "
+                         "path with two tiles of activations, above that on the tcgen05 path)")
     ap.add_argument("--layers", type=int, default=1,
                     help="sweep through this many decoder layers per step (each layer has its own copy of the blobs in HBM): "
                          "the per-token pass over a whole model, e.g. --workload 8b_layer --layers 32")

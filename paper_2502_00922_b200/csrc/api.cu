@@ -58,9 +58,19 @@ size_t ws_partial_offset(const huffllm_desc *d) {
     const size_t max_m_tiles = (d->row_groups + 7) / 8;      // tensor-core row tiles at their smallest (128 rows)
     return ws_ctrl_bytes(d) + (max_m_tiles * 32 * 4 + 255) / 256 * 256;
 }
+// Partial sums of the register path: [kMaxGrid * 2][16 * b] CTA pieces, and, with two tiles of activations (batch
+// 9..16), [kMaxGrid][2 * 32][16 * b] pieces that the warps of one CTA exchange (shared memory has no room for them).
+constexpr uint32_t kTwoTileBatch = 16;    // most activation vectors of the register path with two tiles
+bool two_tile_blob(const huffllm_desc *d) { return d->dtype == HUFFLLM_BF16 && d->lut_bits == 8; }
+size_t ws_cta_pieces_bytes(uint32_t b) { return (size_t)kMaxGrid * 2 * 16 * b * sizeof(float); }
+// (a workspace sized for `batch` vectors serves every smaller batch too)
 size_t ws_bytes_for(const huffllm_desc *d, uint32_t batch) {
-    uint32_t b = batch < kKernelBatch ? batch : kKernelBatch;
-    return ws_partial_offset(d) + (size_t)kMaxGrid * 2 * 16 * b * sizeof(float);
+    size_t need = ws_cta_pieces_bytes(batch < kKernelBatch ? batch : kKernelBatch);
+    if (batch > kKernelBatch && two_tile_blob(d)) {
+        const uint32_t b = batch < kTwoTileBatch ? batch : kTwoTileBatch;
+        need = ws_cta_pieces_bytes(b) + (size_t)kMaxGrid * 2 * 32 * 16 * b * sizeof(float);
+    }
+    return ws_partial_offset(d) + need;
 }
 
 // Geometry of the tensor-core small-batch path (batch 9..64): row tiles of 512 rows, column chunks cut into
@@ -188,7 +198,8 @@ huffllm_status add_matrix(KernelArgs *k, const huffllm_desc *desc, const void *b
 
 // Close a launch description: shared-memory budget and grid size.
 huffllm_status finish_args(KernelArgs *k, bool product, const DeviceInfo &dev, uint32_t *grid) {
-    k->part_bytes = product ? 2 * 32 * 16 * k->batch * (uint32_t)sizeof(float) : 0;
+    // (pieces that warps of a CTA exchange: in shared memory up to 8 vectors, in the workspace above)
+    k->part_bytes = product && k->batch <= kKernelBatch ? 2 * 32 * 16 * k->batch * (uint32_t)sizeof(float) : 0;
     // worst case for the table's alignment gap is covered by assuming the window starts within 4 KB of zero
     uint64_t fixed = (uint64_t)k->lut_size + (k->guard_bytes > k->part_bytes ? k->guard_bytes - k->part_bytes : 0) + k->part_bytes + 4096;
     if (fixed + 2ull * k->slot_bytes > k->dyn_smem_bytes)
@@ -336,6 +347,26 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
     if (st != HUFFLLM_OK) return st;
     if (batch == 0 || batch > 64) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be in [1, 64]");
     if ((st = check_product_args(desc, x, y, workspace, workspace_bytes, batch)) != HUFFLLM_OK) return st;
+    if (batch > kKernelBatch && batch <= kTwoTileBatch && two_tile_blob(desc)) {
+        // 9..16 vectors on the default BF16 blobs: the register path with two tiles of activations per decoded block
+        KernelArgs k;
+        uint32_t grid;
+        begin_args(&k, batch, dev);
+        if ((st = add_matrix(&k, desc, blob)) != HUFFLLM_OK) return st;
+        st = finish_args(&k, true, dev, &grid);
+        if (st == HUFFLLM_OK) {
+            k.m[0].x = x;
+            k.m[0].y = y;
+            k.m[0].ws_ticket = (unsigned int *)workspace;
+            k.m[0].ws_partial = (float *)((uint8_t *)workspace + ws_partial_offset(desc));
+            k.m[0].ws_warp_pieces = (float *)((uint8_t *)workspace + ws_partial_offset(desc) + ws_cta_pieces_bytes(batch));
+            k.err = err_flag;
+            cudaError_t e = launch_gemm(k, grid, (cudaStream_t)stream);
+            if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "product launch: %s", cudaGetErrorString(e));
+            return HUFFLLM_OK;
+        }
+        clear_error();      // records too large for shared memory: the paths below decide
+    }
     if (batch > kKernelBatch && desc->lut_bits <= (desc->dtype == HUFFLLM_FP16 ? 8u : 9u)) {
         // tensor-core path: one pass over the compressed weights for the whole batch (tables of up to 9 bits; longer
         // codes take passes of 8 vectors through the register-path kernel and its two-level lookup)

@@ -50,8 +50,11 @@ namespace huffllm {
 // decoder has finished with a slot it says so on a second barrier, which the feeder polls.  All bookkeeping of a
 // chunk is thus one lane's work instead of a whole warp's: the decoder warps, whose issue slots bound the kernel,
 // spend theirs on decoding.
-template <int MODE, int LB, int THREADS, int FMT>
+// NT = 8-column tiles of activations per product: 1 (batch 1..8) or 2 (batch 9..16: twice the multiply-adds on the same
+// decoded registers; the pieces that warps of a CTA exchange then live in the workspace, shared memory has no room for them).
+template <int MODE, int LB, int THREADS, int FMT, int NT = 1>
 __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant__ KernelArgs A) {
+    constexpr int kV = 4 * NT;                                // values a lane holds of a row group's 16 x batch outputs
     constexpr uint32_t kRawBlock = FMT ? 64u : 512u;          // raw bytes of one block of a record
     constexpr uint32_t kRawLane = FMT ? 2u : 16u;             // of which one lane's share
     // raw part of a record with nkb blocks, in record units of 128 bytes (FP16: rounded up to whole units)
@@ -78,7 +81,8 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     const SmemPlan plan = plan_smem(smem_base, A, feeder);
     const uint32_t nw = plan.warps;                            // decoder warps
     const uint32_t vals = 16 * A.batch;
-    float *part_val = (float *)(dyn_smem + A.dyn_smem_bytes - A.part_bytes);  // [2 * warps][16 * batch]
+    // the pieces of row groups that several warps of the CTA share: [2 * warps][16 * batch], in shared memory (NT = 1)
+    float *part_val = (float *)(dyn_smem + A.dyn_smem_bytes - A.part_bytes);
 
     // the matrix this CTA works in, and the CTA's piece of that matrix's chunks
     uint32_t mi = 0;
@@ -229,8 +233,11 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
 
     bool waited_prior = false, failed = false;
 
-    float acc[4] = {0.f, 0.f, 0.f, 0.f};
+    float acc[kV];
+#pragma unroll
+    for (int j = 0; j < kV; ++j) acc[j] = 0.f;
     int cur_rg = -1;
+    if (NT == 2) part_val = k.ws_warp_pieces + (size_t)J * (2 * kMaxWarps) * vals;   // (same-SM traffic: it stays in L1 / L2)
 
     // ---- reduction of a finished row group, without any CTA-wide barrier.
     // A row group whose chunks this warp decoded alone goes straight to y.  Otherwise the warp parks its
@@ -243,11 +250,11 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         return ch < big ? ch / (k.cta_chunks + 1) : k.cta_extra + (ch - big) / k.cta_chunks;
     };
     // lanes 0..vals-1 (looping if vals > 32) hold or produce the value of output o = column * 16 + row
-    auto finish_cta_sum = [&](int rg, float (&v)[4]) {       // v[i] = value of output o = lane + 32 i
+    auto finish_cta_sum = [&](int rg, float (&v)[kV]) {      // v[i] = value of output o = lane + 32 i
         const uint32_t g_lo = (uint32_t)rg * KC, g_hi = g_lo + KC;
         if (cta_beg <= g_lo && cta_end >= g_hi) {             // the CTA held the whole row group
 #pragma unroll
-            for (int i = 0; i < 4; ++i) {
+            for (int i = 0; i < kV; ++i) {
                 uint32_t o = lane + 32 * i;
                 uint64_t r = (uint64_t)rg * 16 + (o & 15);
                 if (o < vals && r < k.rows) k.y[(uint64_t)(o >> 4) * k.rows + r] = v[i];
@@ -257,7 +264,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         // slot 0 holds the piece of the CTA's first row group in this matrix, slot 1 the piece of its last one
         const uint32_t my_slot = (uint32_t)rg == cta_beg / KC ? 0u : 1u;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < kV; ++i) {
             uint32_t o = lane + 32 * i;
             if (o < vals) k.ws_partial[((size_t)J * 2 + my_slot) * vals + o] = v[i];
         }
@@ -270,7 +277,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         }
         if (!__shfl_sync(0xFFFFFFFFu, last, 0)) return;       // somebody else will arrive later and add us in
 #pragma unroll
-        for (int i = 0; i < 4; ++i) {
+        for (int i = 0; i < kV; ++i) {
             uint32_t o = lane + 32 * i;
             if (o >= vals) continue;
             float sum = 0.f;
@@ -290,16 +297,17 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         const uint32_t ent = warp * 2 + ((uint32_t)rg == c_beg / KC ? 0u : 1u);
         float *mine = part_val + (size_t)ent * vals;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            uint32_t col = 2 * t + (j & 1), row = g + 8 * (j >> 1);
+        for (int j = 0; j < kV; ++j) {      // (tile j / 4 of the activations: columns 8 (j / 4) + 2 t, + 1)
+            uint32_t col = 8 * (j >> 2) + 2 * t + (j & 1), row = g + 8 * ((j >> 1) & 1);
             if (col < A.batch) mine[col * 16 + row] = acc[j];
         }
-        acc[0] = acc[1] = acc[2] = acc[3] = 0.f;
+#pragma unroll
+        for (int j = 0; j < kV; ++j) acc[j] = 0.f;
         __syncwarp();
-        float v[4];
+        float v[kV];
         if (alone) {
 #pragma unroll
-            for (int i = 0; i < 4; ++i) v[i] = lane + 32 * i < vals ? mine[lane + 32 * i] : 0.f;
+            for (int i = 0; i < kV; ++i) v[i] = lane + 32 * i < vals ? mine[lane + 32 * i] : 0.f;
             __syncwarp();
             finish_cta_sum(rg, v);
             return;
@@ -318,12 +326,12 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         }
         if (!__shfl_sync(0xFFFFFFFFu, last, 0)) return;
 #pragma unroll
-        for (int i = 0; i < 4; ++i) v[i] = 0.f;
+        for (int i = 0; i < kV; ++i) v[i] = 0.f;
         for (uint32_t m = mask; m; m &= m - 1) {              // pieces in warp order
             const uint32_t w = __ffs(m) - 1;
             const float *piece = part_val + (size_t)(w * 2 + __shfl_sync(0xFFFFFFFFu, slot_of_lane, w)) * vals;
 #pragma unroll
-            for (int i = 0; i < 4; ++i)
+            for (int i = 0; i < kV; ++i)
                 if (lane + 32 * i < vals) v[i] += piece[lane + 32 * i];
         }
         finish_cta_sum(rg, v);
@@ -333,6 +341,8 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         uint32_t rg = c_beg / KC, kc = c_beg - rg * KC;               // tracked incrementally from here on
         // The activation pointer runs on from chunk to chunk: the columns of a row group's chunks follow each other.
         const uint16_t *xq = k.x + (MODE == 1 ? (uint64_t)min(g, A.batch - 1) * k.cols + kc * k.chunk_cols + t * 8u : 0);
+        // (second tile of activations, vectors 8 .. 15: lane g's vector 8 + g lies this many elements further on)
+        const uint64_t x_tile2 = NT == 2 ? (uint64_t)(min(g + 8u, A.batch - 1) - min(g, A.batch - 1)) * k.cols : 0;
         // this chunk's slot (the lane's column of it), its barrier and its note, toggled by XOR from chunk to chunk; parity
         // of the barrier's next completion (each of the two "full" barriers completes every second chunk)
         uint32_t slot_cur = slot_addr(plan, warp, 0, A.slot_bytes) + (lane << 2), bar_cur = bar_w, par = 0, which = 0;
@@ -412,7 +422,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                     }
                     uint4 xv;
                     if (MODE == 1) {
-                        xv = __ldg((const uint4 *)xq);
+                        if (NT == 1) xv = __ldg((const uint4 *)xq);   // (two tiles: both are fetched behind the decoder, registers are short)
                         xq += 32;
                     }
 
@@ -421,12 +431,28 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                     else decode_block<R, SKIP, LONG>(sa, sb, kIdxMask, lut_lane, cur, a, full_base, full_mask);
 
                     if (MODE == 1) {
+                        uint4 xw;
+                        if (NT == 2) {
+                            xv = __ldg((const uint4 *)(xq - 32));
+                            xw = __ldg((const uint4 *)(xq - 32 + x_tile2));
+                        }
+                        float (&acc0)[4] = *reinterpret_cast<float (*)[4]>(&acc[0]);
                         if (FMT) {
-                            mma_f16_16816(acc, a[0], a[4], a[1], a[5], xv.x, xv.y);
-                            mma_f16_16816(acc, a[2], a[6], a[3], a[7], xv.z, xv.w);
+                            mma_f16_16816(acc0, a[0], a[4], a[1], a[5], xv.x, xv.y);
+                            mma_f16_16816(acc0, a[2], a[6], a[3], a[7], xv.z, xv.w);
                         } else {
-                            mma_bf16_16816(acc, a[0], a[4], a[1], a[5], xv.x, xv.y);
-                            mma_bf16_16816(acc, a[2], a[6], a[3], a[7], xv.z, xv.w);
+                            mma_bf16_16816(acc0, a[0], a[4], a[1], a[5], xv.x, xv.y);
+                            mma_bf16_16816(acc0, a[2], a[6], a[3], a[7], xv.z, xv.w);
+                        }
+                        if (NT == 2) {
+                            float (&acc1)[4] = *reinterpret_cast<float (*)[4]>(&acc[4 * (NT - 1)]);
+                            if (FMT) {
+                                mma_f16_16816(acc1, a[0], a[4], a[1], a[5], xw.x, xw.y);
+                                mma_f16_16816(acc1, a[2], a[6], a[3], a[7], xw.z, xw.w);
+                            } else {
+                                mma_bf16_16816(acc1, a[0], a[4], a[1], a[5], xw.x, xw.y);
+                                mma_bf16_16816(acc1, a[2], a[6], a[3], a[7], xw.z, xw.w);
+                            }
                         }
                     } else {
                         const uint32_t col = col0 + kb * 32u;
@@ -552,9 +578,9 @@ cudaError_t launch_stage_copy(void *dst, const void *src, uint64_t bytes, uint32
 
 // ------------------------------------------------------------------------------ launchers
 
-template <int MODE, int LB, int THREADS, int FMT>
+template <int MODE, int LB, int THREADS, int FMT, int NT = 1>
 static cudaError_t launch_one(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
-    auto fn = huff_kernel<MODE, LB, THREADS, FMT>;
+    auto fn = huff_kernel<MODE, LB, THREADS, FMT, NT>;
     static std::atomic<bool> attr_set[64];   // set twice by racing threads at worst: the call is idempotent
     int dev = 0;
     cudaGetDevice(&dev);
@@ -583,6 +609,7 @@ cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t strea
 }
 
 cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
+    if (k.batch > 8) return launch_one<1, 8, kThreads, 0, 2>(k, grid, stream);   // (the entry point sends only BF16 blobs of 8-bit tables here)
     if (k.fmt) return k.lut_bits > 8 ? launch_one<1, 12, kThreads, 1>(k, grid, stream) : launch_one<1, 8, kThreads, 1>(k, grid, stream);
     if (k.lut_bits > 9) return launch_one<1, 12, kThreads, 0>(k, grid, stream);
     return k.lut_bits == 8 ? launch_one<1, 8, kThreads, 0>(k, grid, stream) : launch_one<1, 9, kThreads, 0>(k, grid, stream);

@@ -19,6 +19,7 @@ struct MatArgs {
     const uint16_t *x;         // [batch][cols]
     float *y;                  // [batch][rows]
     float *ws_partial;         // [cta_count * 2][16 * batch]
+    float *ws_warp_pieces;     // batch 9..16 only: [cta_count][2 * 32][16 * batch], the pieces warps of one CTA exchange
     unsigned int *ws_ticket;   // [cta_count] arrival counters, zero between calls
     uint16_t *out;             // decode output
 };
@@ -32,7 +33,7 @@ struct KernelArgs {
     uint32_t guard_bytes;      // readable bytes kept free behind the last slot
     uint32_t part_bytes;       // bytes at the end of dynamic shared memory for the CTA's partial sums (tensor-core path: the stages of activations)
     uint32_t dyn_smem_bytes;
-    uint32_t batch;            // 1..8
+    uint32_t batch;            // 1..8 (register path), 9..16 (register path with two tiles of activations)
     int32_t *err;              // may be null
     // tensor-core small-batch path only
     uint32_t tc_npad;          // batch rounded up to 16, 32 or 64
