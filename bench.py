@@ -53,10 +53,10 @@ def launch_groups(table, fuse: str):
         return [[0, 1, 2], [3], [4, 5], [6]]
     return [[i] for i in range(n)]
 FALLBACK_HBM_GBS = 6650.0
-# dram__bytes_read.sum + dram__bytes_write.sum of one fused-product launch over its algorithmic bytes, from the ncu
-# capture summarised in profiles/huff_kernel_product_llama7b_layer.md (gate+up: 147.0 MB moved for 142.1 MB; down:
-# 72.4 MB for 71.0 MB); traffic = ratio * algorithmic bytes.
-NCU_TRAFFIC_RATIO = 1.03
+# dram__bytes_read.sum + dram__bytes_write.sum of the step's four fused-product launches over their algorithmic bytes, from the
+# ncu capture summarised in profiles/huff_kernel_product_llama7b_layer.md (330.05 MB moved for 318.64 MB);
+# traffic = ratio * algorithmic bytes.
+NCU_TRAFFIC_RATIO = 1.036
 
 
 def max_over_ranks(v: float, dist, device) -> float:
@@ -775,7 +775,7 @@ def main():
                      "traffic": None if NCU_TRAFFIC_RATIO is None else NCU_TRAFFIC_RATIO * alg_bytes / len(groups),
                      "traffic_per_step": None if NCU_TRAFFIC_RATIO is None else NCU_TRAFFIC_RATIO * alg_bytes,
                      "traffic_note": "DRAM bytes read + written per launch (average over the step's launches): algorithmic bytes x the "
-                                     "ratio of the ncu capture in profiles/ (1.03)",
+                                     "ratio of the ncu capture in profiles/ (1.036)",
                      "peak_source": peak_src, "kernel": "huff_kernel<product>" if B <= 8 else "huff_gemm_tc_kernel", "launches_per_step": len(groups), "fuse": args.fuse,
                      "algorithmic_bytes_per_step": alg_bytes, "kernel_ms_per_step": kernel_ms_step,
                      "frac_of_nominal_8TBs": achieved / 8000.0,
