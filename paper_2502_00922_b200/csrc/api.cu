@@ -429,8 +429,11 @@ huffllm_status huffllm_decode_gemm_multi_host_async(uint32_t n, const huffllm_de
     cudaStream_t s = (cudaStream_t)stream;
     for (uint32_t i = 0; i < n; ++i) {     // nothing is enqueued before every argument has been looked at
         if (!descs[i] || !xs_host[i] || !ys_host[i] || !x_stages[i] || !y_stages[i]) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
-        huffllm_status st = check_desc(descs[i]);
+        huffllm_status st = check_product_args(descs[i], x_stages[i], y_stages[i], workspaces ? workspaces[i] : nullptr,
+                                               workspace_bytes_each, batch);
         if (st != HUFFLLM_OK) return st;
+        if (!blobs || !blobs[i] || ((uintptr_t)blobs[i] & 255))
+            return fail(HUFFLLM_ERR_INVALID_ARG, "blob must be a 256-byte aligned device pointer");
     }
     for (uint32_t i = 0; i < n; ++i) {
         cudaError_t e = cudaMemcpyAsync(x_stages[i], xs_host[i], (size_t)batch * descs[i]->cols * 2, cudaMemcpyHostToDevice, s);

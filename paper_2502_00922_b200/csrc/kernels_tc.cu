@@ -313,6 +313,10 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                     uint32_t a[8];
                     if (FMT) decode_block_fp16(sa, sb, lut_lane, raw_c.x, a);   // a chunk that is not ok decodes garbage, never out of range
                     else decode_block<R, SKIP>(sa, sb, kIdxMask, lut_lane, raw_c, a);
+                    if (!ok) {                                    // ... and contributes nothing, as on the register path
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) a[i] = 0u;
+                    }
                     stage_block(a, x_c, gb == gb_item);
                 };
                 uint4 raw_b = make_uint4(0, 0, 0, 0);
