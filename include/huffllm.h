@@ -115,7 +115,7 @@ typedef struct huffllm_desc {
     uint32_t row_groups;      /* ceil(rows / 16)                                           */
     uint32_t col_chunks;      /* ceil(cols / chunk_cols)                                   */
     uint64_t n_chunks;        /* row_groups * col_chunks                                   */
-    uint32_t lut_bits;        /* L_max: BF16: of one weight's coded fields together; FP16: of each field (8 .. 12) */
+    uint32_t lut_bits;        /* L_max: BF16: of one weight's coded fields together (8 .. 12); FP16: of each field (7 .. 12) */
     uint32_t lag_bits;        /* 7 (BF16 blobs), 6 (FP16 blobs)                            */
     uint32_t n_fields;        /* coded fields per weight: 2 (BF16 {1,4,4,7}), 1 ({1,8,7}), 3 (FP16 {1,5,5,5}) */
     uint8_t  caps[4];         /* per-field maximum code length chosen under lut_bits       */
@@ -140,6 +140,7 @@ typedef struct huffllm_desc {
  * capped at (c0, c1) with c0 + c1 <= max_code_len, chosen to minimise the coded size, each code
  * being the optimal length-limited prefix code for its cap; where plain Huffman already fits,
  * the result is plain Huffman.  0 selects the default (8); supported range 8..12.
+ * (FP16 also takes 7: its fields have 32 symbols each, and the device keeps 128-entry tables once per lane.)
  * A field with a single used symbol gets a 1-bit code.  An empty tensor is INVALID_ARG.
  * HUFFLLM_FP16 is the paper's {1,5,5,5} split (Section 3.1): sign raw, exponent and the two mantissa halves each
  * with its own code, each limited to max_code_len on its own (Section 3.2 quotes 12 for these 5-bit fields).

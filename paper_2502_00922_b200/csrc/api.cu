@@ -367,7 +367,7 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
         }
         clear_error();      // records too large for shared memory: the paths below decide
     }
-    if (batch > kKernelBatch && desc->lut_bits <= (desc->dtype == HUFFLLM_FP16 ? 8u : 9u)) {
+    if (batch > kKernelBatch && (desc->dtype == HUFFLLM_FP16 ? desc->lut_bits == 8u : desc->lut_bits <= 9u)) {
         // tensor-core path: one pass over the compressed weights for the whole batch (tables of up to 9 bits; longer
         // codes take passes of 8 vectors through the register-path kernel and its two-level lookup)
         const TcPlan tp = tc_plan(desc, batch, (uint32_t)dev.sms, (uint32_t)dev.smem_optin - kStaticSmem);

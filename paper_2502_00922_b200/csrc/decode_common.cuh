@@ -161,16 +161,29 @@ __device__ __forceinline__ uint32_t stream_step_long(LaneStream &s, uint32_t lut
 //     refill check tests bit 5 and the funnel shift reads bits 0..4.
 __device__ __forceinline__ uint32_t lut_entry_inplace(uint32_t e) { return e | (e >> 16); }
 
+template <bool RELOAD = true>      // false: the low word is copied from the high one (where shared-memory bandwidth is the scarcer resource)
 __device__ __forceinline__ void stream_refill4(LaneStream &s) {
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t.reg .b32 b;\n\t"
-        "setp.ne.u32 q, 0, 0;\n\t"
-        "lop3.or.b32 b|p, %2, 32, 0, 0xC0, q;\n\t"          // p = bit 5 of the pointer: 32 or more bits consumed
-        "@p ld.shared.u32 %0, [%3+-256];\n\t"
-        "@p ld.shared.u32 %1, [%3];\n\t"
-        "@p add.u32 %3, %3, 256;\n\t"
-        "@p add.u32 %2, %2, 0xFFFFFFE0;\n\t}"
-        : "+r"(s.lo), "+r"(s.hi), "+r"(s.pos), "+r"(s.nxt));
+    if (RELOAD) {
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t.reg .b32 b;\n\t"
+            "setp.ne.u32 q, 0, 0;\n\t"
+            "lop3.or.b32 b|p, %2, 32, 0, 0xC0, q;\n\t"          // p = bit 5 of the pointer: 32 or more bits consumed
+            "@p ld.shared.u32 %0, [%3+-256];\n\t"
+            "@p ld.shared.u32 %1, [%3];\n\t"
+            "@p add.u32 %3, %3, 256;\n\t"
+            "@p add.u32 %2, %2, 0xFFFFFFE0;\n\t}"
+            : "+r"(s.lo), "+r"(s.hi), "+r"(s.pos), "+r"(s.nxt));
+    } else {
+        asm volatile(
+            "{\n\t.reg .pred p, q;\n\t.reg .b32 b;\n\t"
+            "setp.ne.u32 q, 0, 0;\n\t"
+            "lop3.or.b32 b|p, %2, 32, 0, 0xC0, q;\n\t"
+            "@p mov.u32 %0, %1;\n\t"
+            "@p ld.shared.u32 %1, [%3];\n\t"
+            "@p add.u32 %3, %3, 256;\n\t"
+            "@p add.u32 %2, %2, 0xFFFFFFE0;\n\t}"
+            : "+r"(s.lo), "+r"(s.hi), "+r"(s.pos), "+r"(s.nxt));
+    }
 }
 // The 32 window bits at the pointer, right after a refill check (pointer below 32: a 32-bit funnel shift is enough,
 // and it reads only the pointer's low 5 bits).
@@ -332,15 +345,65 @@ __device__ __forceinline__ uint32_t fp16_weight_long(LaneStream &s, uint32_t lut
     asm("lop3.b32 %0, %1, %2, %3, 0xFE;" : "=r"(w) : "r"(e0), "r"(e1), "r"(e2));
     return w;
 }
+// Field codes of at most 8 bits, three codewords at a time (the scheme of the 8-bit BF16 decoder): the pointer stands on the
+// codeword (the sequence's 6 leading zero bits are skipped when it is opened); after one check per weight it is below 32,
+// so the low 32 bits of the shifted window hold the weight's three codewords (at most 24 bits).  They are taken out of
+// the window once and shifted in place by each codeword's length, which the shared-memory copy of the tables keeps in an
+// entry's low byte: entry = symbol bits << 8 | length (fp16_entry_inplace), so the OR of a weight's three entries has the
+// weight's low 15 bits at bits 8..22.  The table address is byte 0 of the window times 64 plus the lane's column of the
+// field's table: one byte dot product.  The pointer is advanced once per weight by the sum of the three entries; only its
+// low 6 bits mean anything (lengths add up to at most 24, bits 4..7 of an entry are zero) and nothing reads above them.
+__device__ __forceinline__ uint32_t fp16_entry_inplace(uint32_t e) { return ((e & 0x7FFFu) << 8) | (e >> 16); }
+__device__ __forceinline__ uint32_t fp16_weight_inplace(LaneStream &s, uint32_t lut_lane) {
+    stream_refill4<false>(s);
+    uint32_t t = window_at(s);
+    const uint32_t e0 = lds_lut(__dp4a(t, 0x00000040u, lut_lane));
+    t = shift_by_entry(t, e0);
+    const uint32_t e1 = lds_lut(__dp4a(t, 0x00000040u, lut_lane) + 16384u);
+    t = shift_by_entry(t, e1);
+    const uint32_t e2 = lds_lut(__dp4a(t, 0x00000040u, lut_lane) + 32768u);
+    s.pos = (s.pos + e0) + (e1 + e2);
+    uint32_t w;
+    asm("lop3.b32 %0, %1, %2, %3, 0xFE;" : "=r"(w) : "r"(e0), "r"(e1), "r"(e2));
+    return w;                                      // bits 8..22: exponent and mantissa
+}
+// Field codes of at most 7 bits: the same three-at-a-time scheme on tables of 128 entries, which are small enough to keep
+// once per LANE (entry i of lane l at word 32 i + l, 16 KB per field: the footprint of the sixteen-fold 256-entry tables),
+// so that a warp-wide lookup never has a bank conflict.  Seven index bits are not a byte, so the window is moved up by 7
+// bits once per weight and the table address is (window & index mask) | lane column, one logic operation; the in-place
+// shifts keep the next codeword at bit 7 (25 window bits are valid there: three codewords take at most 21).
+__device__ __forceinline__ uint32_t fp16_weight_lane(LaneStream &s, uint32_t lut_lane) {
+    stream_refill4<false>(s);
+    uint32_t t = window_at(s) << 7, a0, a1, a2;
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(a0) : "r"(t), "r"(0x7Fu << 7), "r"(lut_lane));
+    const uint32_t e0 = lds_lut(a0);
+    t = shift_by_entry(t, e0);
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(a1) : "r"(t), "r"(0x7Fu << 7), "r"(lut_lane));
+    const uint32_t e1 = lds_lut(a1 + 16384u);
+    t = shift_by_entry(t, e1);
+    asm("lop3.b32 %0, %1, %2, %3, 0xEA;" : "=r"(a2) : "r"(t), "r"(0x7Fu << 7), "r"(lut_lane));
+    const uint32_t e2 = lds_lut(a2 + 32768u);
+    s.pos = (s.pos + e0) + (e1 + e2);
+    uint32_t w;
+    asm("lop3.b32 %0, %1, %2, %3, 0xFE;" : "=r"(w) : "r"(e0), "r"(e1), "r"(e2));
+    return w;                                      // bits 8..22: exponent and mantissa
+}
 // Decode one block of an FP16 chunk into 8 packed registers (same order as decode_block).  `signs` is the lane's
 // uint16 of the block: bit p = sign of the first weight of pair p, bit 8 + p = sign of its second weight.
-template <bool LONG = false>
+// INPLACE: the three-at-a-time decoders above: 1 = tables of 8 bits (sixteen-fold), 2 = tables of 7 bits (per lane).
+template <bool LONG = false, int INPLACE = 0>
 __device__ __forceinline__ void decode_block_fp16(LaneStream &sa, LaneStream &sb, uint32_t lut_lane, uint32_t signs,
                                                   uint32_t (&a)[8], uint32_t full_base = 0, uint32_t full_mask = 0) {
     uint32_t w[16];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        if (LONG) {
+        if (INPLACE == 2) {
+            w[i] = fp16_weight_lane(sa, lut_lane);
+            w[8 + i] = fp16_weight_lane(sb, lut_lane);
+        } else if (INPLACE == 1) {
+            w[i] = fp16_weight_inplace(sa, lut_lane);
+            w[8 + i] = fp16_weight_inplace(sb, lut_lane);
+        } else if (LONG) {
             w[i] = fp16_weight_long(sa, lut_lane, full_base, full_mask);
             w[8 + i] = fp16_weight_long(sb, lut_lane, full_base, full_mask);
         } else {
@@ -353,7 +416,7 @@ __device__ __forceinline__ void decode_block_fp16(LaneStream &sa, LaneStream &sb
     const uint32_t s32 = prmt(signs, 0u, 0x4140u);     // first-weight signs in bits 0..7, second-weight signs in bits 16..23
 #pragma unroll
     for (int p = 0; p < 8; ++p) {
-        uint32_t pair = prmt(w[2 * p], w[2 * p + 1], 0x5410u);   // low halves of the two weights
+        uint32_t pair = prmt(w[2 * p], w[2 * p + 1], INPLACE ? 0x6521u : 0x5410u);   // the two weights' 15 bits (in place: from bits 8..22)
         uint32_t sh = s32 << (15 - p);                            // their sign bits at bits 15 and 31
         asm("lop3.b32 %0, %1, %2, 0x7FFF7FFF, 0xE4;" : "=r"(a[p]) : "r"(pair), "r"(sh));   // mask bit set: pair, else sign
     }

@@ -52,7 +52,7 @@ huffllm_status check_desc(const huffllm_desc *d) {
         d->col_chunks != (d->cols + d->chunk_cols - 1) / d->chunk_cols ||
         d->n_chunks != (uint64_t)d->row_groups * d->col_chunks)
         return fail(HUFFLLM_ERR_CORRUPT, "chunk counts do not match the shape");
-    if (d->lut_bits < kMinBudget || d->lut_bits > kMaxBudget) return fail(HUFFLLM_ERR_CORRUPT, "bad lut_bits");
+    if (d->lut_bits < min_budget_for(d->dtype) || d->lut_bits > kMaxBudget) return fail(HUFFLLM_ERR_CORRUPT, "bad lut_bits");
     uint32_t max_steps = d->chunk_cols / kBlockCols * 8;   // per bit sequence
     uint32_t w_bound = (d->lag_bits + max_steps * d->lut_bits * (d->dtype == HUFFLLM_FP16 ? 3 : 1) + 31) / 32;
     if (d->max_words == 0 || d->max_words > w_bound) return fail(HUFFLLM_ERR_CORRUPT, "bad max_words");
@@ -253,8 +253,8 @@ static huffllm_status codebook_from_counts(huffllm_dtype dtype, huffllm_split sp
     if (split != HUFFLLM_SPLIT_PAPER && split != HUFFLLM_SPLIT_WHOLE_EXPONENT) return fail(HUFFLLM_ERR_INVALID_ARG, "bad split");
     if (split == HUFFLLM_SPLIT_WHOLE_EXPONENT && dtype != HUFFLLM_BF16) return fail(HUFFLLM_ERR_UNSUPPORTED, "the whole-exponent split is for bf16");
     uint32_t budget = max_code_len ? max_code_len : kDefaultBudget;
-    if (budget < kMinBudget || budget > kMaxBudget)
-        return fail(HUFFLLM_ERR_UNSUPPORTED, "max_code_len must be 0 or in [%u, %u]", kMinBudget, kMaxBudget);
+    if (budget < min_budget_for(dtype) || budget > kMaxBudget)
+        return fail(HUFFLLM_ERR_UNSUPPORTED, "max_code_len must be 0 or in [%u, %u]", min_budget_for(dtype), kMaxBudget);
     huffllm_codebook *cb = new (std::nothrow) huffllm_codebook();
     if (!cb) return fail(HUFFLLM_ERR_NOMEM, "out of host memory");
     cb->dtype = dtype;

@@ -18,6 +18,9 @@ inline uint32_t lag_bits_for(uint32_t dtype) { return dtype == HUFFLLM_FP16 ? 6u
 constexpr uint32_t kSeqs = 64;          // bit sequences per chunk: two per lane (rows g and g + 8)
 constexpr uint32_t kDefaultBudget = 8;  // default joint code-length bound
 constexpr uint32_t kMinBudget = 8, kMaxBudget = 12;
+// FP16 fields are limited one by one and have 32 symbols each: 7 bits are allowed there as well (128-entry tables, which
+// the device keeps once per lane: lookups without bank conflicts)
+inline uint32_t min_budget_for(uint32_t dtype) { return dtype == HUFFLLM_FP16 ? 7u : kMinBudget; }
 constexpr uint32_t kRecordUnit = 128;   // record offsets are counted in this many bytes
 // Zero bytes behind the payload, part of the blob: the product kernel's requests into L2 run up to 2 KB past the record
 // they are issued in, and with this slack they never leave the blob.

@@ -62,6 +62,8 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     // 8-bit BF16 tables: the decoder starts behind the sequences' leading zero bits and works on four codewords at a
     // time (stream_step4x2)
     constexpr bool SKIP = LB == 8 && FMT == 0;
+    constexpr int SKIP16 = FMT == 1 ? (LB == 8 ? 1 : LB == 7 ? 2 : 0) : 0;   // the same scheme for FP16: three codewords (one weight) at a
+                                                             // time; 2 = field codes of 7 bits, tables once per lane
     constexpr bool LONG = LB > 9;                            // first level of 8 bits, then the whole table (FP16: lut_bits 9..12)
     constexpr uint32_t kLB1 = LONG ? 8u : (uint32_t)LB;      // index bits of the per-lane table
     constexpr int R = SKIP ? 4 : LB == 8 ? 3 : 2;            // decoder steps between two refill checks
@@ -171,8 +173,8 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     // written to shared memory (by the decoder warps alone: the feeder is already asking for records)
     // (FP16: three tables of 256 entries, sixteen copies each: word j holds entry j / 16 of its table)
     // The table goes to shared memory in 16-byte pieces: four neighbouring copies of one entry per piece.
-    constexpr uint32_t kLutWords = FMT ? 3u * 16u * 256u : 32u << kLB1;
-    constexpr uint32_t kLutRep = FMT ? 4u : 5u;            // log2 of the copies per entry
+    constexpr uint32_t kLutWords = FMT ? 3u * 16u * 256u : 32u << kLB1;   // (FP16, 7 bits: 3 x 32 x 128, the same)
+    constexpr uint32_t kLutRep = FMT && LB != 7 ? 4u : 5u; // log2 of the copies per entry
     constexpr uint32_t kLutVecs = kLutWords / 4;
     constexpr uint32_t kLutThreads = THREADS - 32;
     constexpr int kLutLoads = (kLutVecs + kLutThreads - 1) / kLutThreads;
@@ -183,15 +185,16 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         for (int i = 0; i < kLutLoads; ++i) {
             uint32_t v = tid + i * kLutThreads;
             // (entry of vector v: BF16 v / 8; FP16 field v / 1024, entry v / 4 % 256 of that field's table of 1 << lut_bits)
-            const uint32_t src = FMT ? ((v >> 10) << A.lut_bits) + ((v >> 2) & 255u) : v >> (kLutRep - 2);
+            const uint32_t src = FMT ? ((v >> 10) << A.lut_bits) + (LB == 7 ? (v >> 3) & 127u : (v >> 2) & 255u) : v >> (kLutRep - 2);
             lut_v[i] = v < kLutVecs ? __ldg(lut_g + src) : 0u;
             if (SKIP) lut_v[i] = lut_entry_inplace(lut_v[i]);   // the length once more, where an in-place shift reads it
+            if (SKIP16) lut_v[i] = fp16_entry_inplace(lut_v[i]);
             if (LONG && (lut_v[i] >> 16) > 8u) lut_v[i] |= kLongMark;   // a codeword longer than the first level resolves
         }
     }
     // two-level lookup: the whole table (1 << lut_bits entries, one copy) sits behind the per-lane first level
     const uint32_t full_base = plan.lut + (FMT ? 49152u : 128u << kLB1), full_mask = ((1u << A.lut_bits) - 1u) << 2;
-    uint32_t lut_lane = plan.lut | ((FMT ? lane & 15u : lane) << 2);
+    uint32_t lut_lane = plan.lut | ((FMT && LB != 7 ? lane & 15u : lane) << 2);
     asm volatile("mov.u32 %0, %0;" : "+r"(lut_lane));  // keep it in a register: it is an operand of every lookup
     const uint32_t g = lane >> 2, t = lane & 3;
     uint32_t c_beg = 0, c_end = 0;
@@ -393,8 +396,8 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                 const bool has_next = c + 1 < c_end;
                 const uint32_t coded_bytes = (r1 - r0 - raw_units(nkb)) << 7;
                 LaneStream sa, sb;
-                stream_open(sa, slot_cur, SKIP ? 7u : 0u);
-                stream_open(sb, slot_cur + 128u, SKIP ? 7u : 0u);
+                stream_open(sa, slot_cur, SKIP ? 7u : SKIP16 ? 6u : 0u);
+                stream_open(sb, slot_cur + 128u, SKIP ? 7u : SKIP16 ? 6u : 0u);
                 const uint32_t col0 = kc * k.chunk_cols + t * 8u;
                 // (activations: lanes of unused output columns repeat the last vector; cols is a multiple of 32
                 // here, so every block of the chunk lies inside the row and xq ends the chunk where the next begins)
@@ -427,7 +430,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                     }
 
                     uint32_t a[8];
-                    if (FMT) decode_block_fp16<LONG>(sa, sb, lut_lane, cur.x, a, full_base, full_mask);
+                    if (FMT) decode_block_fp16<LONG, SKIP16>(sa, sb, lut_lane, cur.x, a, full_base, full_mask);
                     else decode_block<R, SKIP, LONG>(sa, sb, kIdxMask, lut_lane, cur, a, full_base, full_mask);
 
                     if (MODE == 1) {
@@ -603,6 +606,7 @@ static cudaError_t launch_one(const KernelArgs &k, uint32_t grid, cudaStream_t s
 }
 
 cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
+    if (k.fmt && k.lut_bits == 7) return launch_one<0, 7, kThreads, 1>(k, grid, stream);
     if (k.fmt) return k.lut_bits > 8 ? launch_one<0, 12, kThreads, 1>(k, grid, stream) : launch_one<0, 8, kThreads, 1>(k, grid, stream);
     if (k.lut_bits > 9) return launch_one<0, 12, kThreads, 0>(k, grid, stream);
     return k.lut_bits == 8 ? launch_one<0, 8, kThreads, 0>(k, grid, stream) : launch_one<0, 9, kThreads, 0>(k, grid, stream);
@@ -610,6 +614,7 @@ cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t strea
 
 cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
     if (k.batch > 8) return launch_one<1, 8, kThreads, 0, 2>(k, grid, stream);   // (the entry point sends only BF16 blobs of 8-bit tables here)
+    if (k.fmt && k.lut_bits == 7) return launch_one<1, 7, kThreads, 1>(k, grid, stream);
     if (k.fmt) return k.lut_bits > 8 ? launch_one<1, 12, kThreads, 1>(k, grid, stream) : launch_one<1, 8, kThreads, 1>(k, grid, stream);
     if (k.lut_bits > 9) return launch_one<1, 12, kThreads, 0>(k, grid, stream);
     return k.lut_bits == 8 ? launch_one<1, 8, kThreads, 0>(k, grid, stream) : launch_one<1, 9, kThreads, 0>(k, grid, stream);

@@ -190,6 +190,29 @@ def test_fp16_long_field_codes_decode_and_product(hl, torch, rows, cols, ce, bud
         check_product(gpu_gemm(hl, torch, up, x), w, x, orc.FP16)
 
 
+@pytest.mark.parametrize("rows,cols,ce,gen,batch", [
+    (1024, 1024, 1024, "fp16", 1),                # true fp16 weights
+    (512, 4096, 2048, "fp16_from_bf16", 8),
+    (256, 1024, 1024, "skewed", 3),               # geometric laws: the 7-bit limit bites in all three fields
+    (37, 300, 512, "skewed", 0),                  # ragged rows and columns (decode only)
+    (256, 2048, 1024, "patterns", 0),             # every bit pattern (decode only)
+    (16, 512, 512, "constant", 2),                # single-symbol codes
+    (128, 1024, 1024, "fp16", 16),                # batch above 8: passes of 8 vectors
+])
+def test_fp16_seven_bit_field_codes(hl, torch, rows, cols, ce, gen, batch):
+    """FP16 {1,5,5,5} blobs whose field codes are limited to 7 bits: 128-entry tables that the device keeps once per lane."""
+    w = FP16_GENS[gen](rows, cols, 1500 + rows)
+    up = Uploaded(hl, torch, w, ce, 7, max(batch, 1), dtype=hl.FP16)
+    assert (up.desc.dtype, up.desc.lut_bits) == (hl.FP16, 7)
+    assert np.array_equal(gpu_decode(hl, torch, up), w)
+    if rows * cols <= 600_000:
+        ref, _ = orc.decode_blob(up.blob)
+        assert np.array_equal(ref, w)
+    if batch:
+        x = wl.activations(batch, cols, 1550 + cols, "fp16")
+        check_product(gpu_gemm(hl, torch, up, x), w, x, orc.FP16)
+
+
 def test_fp16_large_chunks_run_with_fewer_warps(hl, torch):
     """Records too large for 32 pairs of shared-memory slots are decoded by as many warps as have room."""
     w = wl.gaussian_weights(64, 4096, 0.02, 990, "fp16")
