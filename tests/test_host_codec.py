@@ -179,7 +179,7 @@ FP16_SETS = {
 
 
 @pytest.mark.parametrize("name", sorted(FP16_SETS))
-@pytest.mark.parametrize("budget", [0, 8, 12])
+@pytest.mark.parametrize("budget", [0, 7, 8, 12])
 def test_fp16_codebook_cost_matches_oracle(name, budget):
     """FP16 {1,5,5,5}: three codes, each limited on its own."""
     w = FP16_SETS[name](64, 1024)
@@ -197,7 +197,8 @@ def test_fp16_codebook_cost_matches_oracle(name, budget):
 
 @pytest.mark.parametrize("rows,cols,ce,budget,gen", [
     (48, 1056, 1024, 8, "fp16"), (37, 300, 1024, 8, "fp16_from_bf16"), (5, 31, 512, 8, "patterns"),
-    (33, 2080, 4096, 12, "fp16"), (16, 512, 512, 8, "constant"), (64, 1024, 2048, 9, "fp16_from_bf16")])
+    (33, 2080, 4096, 12, "fp16"), (16, 512, 512, 8, "constant"), (64, 1024, 2048, 9, "fp16_from_bf16"),
+    (48, 1056, 1024, 7, "fp16"), (37, 300, 512, 7, "patterns")])
 def test_fp16_blob_decodes_with_oracle_and_bits_match(rows, cols, ce, budget, gen):
     w = FP16_SETS[gen](rows, cols)
     cb = hl.build_codebook(w, hl.FP16, budget)
@@ -270,3 +271,38 @@ def test_compression_accounting_on_paper_shaped_weights():
     assert 11.6 <= payload_bits <= 11.9
     total_ratio = 2.0 * n / d.blob_bytes
     assert 1.25 <= total_ratio <= 1.37          # lane padding and side tables cost a few percent
+
+
+def test_device_call_sizes_are_consistent():
+    """Host-only size queries of the device calls: a workspace sized for `batch` vectors serves every smaller batch, its
+    control words come first, the static entry point's limits are what the header says, and the shared-memory plan is the
+    formula the header states."""
+    w = wl.gaussian_weights(528, 4096, 0.02, 91)
+    cb = hl.build_codebook(w)
+    _, d = hl.encode(cb, w, 4096)
+    cb.free()
+    sizes = [hl.workspace_bytes(d, b) for b in range(1, 65)]
+    assert all(a <= b for a, b in zip(sizes, sizes[1:]))
+    ctrl = hl.workspace_control_bytes(d)
+    assert 4096 <= ctrl < sizes[0] and ctrl % 256 == 0
+    assert sizes[hl.STATIC_MAX_BATCH - 1] <= 1 << 20                # fits the static entry point's built-in array
+    plan = hl.decode_smem_plan(d)
+    assert plan["slot_bytes"] == d.max_words * 256
+    assert plan["guard_bytes"] == 256 * (3 + plan["refill_checks_per_block"] * (d.chunk_cols // 32))
+    assert plan["table_bytes"] == 128 << 8
+    with pytest.raises(hl.HuffllmError):
+        hl.workspace_bytes(d, 65)
+
+
+def test_code_length_limits_accepted_per_format():
+    """BF16 budgets 8..12 (the two nibble codes of a weight together); FP16 field limits 7..12."""
+    wb = wl.gaussian_weights(16, 512, 0.02, 92)
+    wh = wl.gaussian_weights(16, 512, 0.02, 93, "fp16")
+    for b in (8, 9, 10, 11, 12):
+        hl.build_codebook(wb, hl.BF16, b).free()
+    for b in (7, 8, 12):
+        hl.build_codebook(wh, hl.FP16, b).free()
+    for dt, w, b in ((hl.BF16, wb, 7), (hl.BF16, wb, 13), (hl.FP16, wh, 6), (hl.FP16, wh, 13)):
+        with pytest.raises(hl.HuffllmError) as e:
+            hl.build_codebook(w, dt, b)
+        assert e.value.status_name == "UNSUPPORTED"
