@@ -444,13 +444,15 @@ def main():
     B = args.batch
     if not 1 <= B <= 64:
         raise SystemExit("--batch must be in [1, 64]")
-    if B > 8:
-        args.fuse = "none"           # the tensor-core path takes one matrix per launch
     fp16 = args.dtype != "bf16"
+    # launches over several matrices take up to 8 vectors, or up to 16 for BF16 blobs with 8-bit tables (two tiles of activations)
+    multi = B <= 8 or (B <= 16 and not fp16 and args.max_code_len in (0, 8))
+    if not multi:
+        args.fuse = "none"           # the tensor-core path takes one matrix per launch
     mats = prepare(args.workload, args.chunk_elems, hl, torch, dev, cpu_mats, split, B, args.dtype, args.max_code_len)
     err = torch.zeros(1, dtype=torch.int32, device=dev)
     L = args.layers
-    if L < 1 or (L > 1 and B > 8):
+    if L < 1 or (L > 1 and not multi):
         raise SystemExit("--layers must be at least 1 (and takes --batch up to 8)")
     n_weights = L * sum(m["rows"] * m["cols"] for m in mats)
     unc_bytes = 2 * n_weights
@@ -467,11 +469,11 @@ def main():
     ws_each = max(m["ws_bytes"] for m in mats)
     raw_stream = stream.cuda_stream
     for c, g in zip(calls, groups):      # argument arrays marshalled once per launch group
-        c["prep"] = hl.PreparedMulti(c["descs"], c["blobs"], c["xs"], min(B, 8), c["ys"], c["wss"], ws_each, err,
+        c["prep"] = hl.PreparedMulti(c["descs"], c["blobs"], c["xs"], B if multi else 8, c["ys"], c["wss"], ws_each, err,
                                      [mats[i]["x_host"] for i in g], [mats[i]["y_host"] for i in g])
 
     def step_device():
-        if B > 8:
+        if not multi:
             for m in mats:
                 hl.decode_gemm(m["desc"], m["blob_dev"], m["x_dev"], B, m["y_dev"], m["ws"], m["ws_bytes"], err, stream)
             return
@@ -482,7 +484,7 @@ def main():
         c["xh"], c["yh"] = [mats[i]["x_host"] for i in g], [mats[i]["y_host"] for i in g]
 
     def step_host():      # host activations in, host results out
-        if B > 8:
+        if not multi:
             # activations staged by a copy kernel, results written to pinned host memory by the kernels, one wait per step
             for m in mats:
                 hl.stage_copy(m["x_dev"], m["x_host"], m["x_host"].numel() * 2, stream)
@@ -549,7 +551,7 @@ def main():
     # ---- the same step as ONE launch over all matrices (valid where the products are independent, as they are here; a
     # decoder layer's data dependencies allow only the default grouping): reported beside the headline, not as it
     one_launch_ms = None
-    if L == 1 and B <= 8 and len(mats) > 1 and len(groups) > 1 and len(mats) <= 8:
+    if L == 1 and multi and len(mats) > 1 and len(groups) > 1 and len(mats) <= 8:
         allp = hl.PreparedMulti([m["desc"] for m in mats], [m["blob_dev"] for m in mats], [m["x_dev"] for m in mats], B,
                                 [m["y_dev"] for m in mats], [m["ws"] for m in mats], ws_each, err)
         for _ in range(args.warmup):
@@ -587,10 +589,10 @@ def main():
     for _ in range(args.warmup):
         step_host()
     barrier()
-    e2e_mode = "stream" if B <= 8 else ("stream; activations staged from pinned host memory by a copy kernel, results written to pinned "
+    e2e_mode = "stream" if multi else ("stream; activations staged from pinned host memory by a copy kernel, results written to pinned "
                                          "host memory by the product kernels, one wait per step")
     run_e2e = step_host
-    if B <= 8:
+    if multi:
         try:
             gstream = torch.cuda.Stream(device=dev)
             graph = torch.cuda.CUDAGraph()
@@ -600,7 +602,7 @@ def main():
             # (last) layer get the pinned host buffers as their y, so the results are written to the host as they are produced.
             n_last = len(calls) // L
             for c, g in zip(calls[-n_last:], groups[-n_last:]):
-                c["prep_host_y"] = hl.PreparedMulti(c["descs"], c["blobs"], c["xs"], min(B, 8), [mats[i]["y_host"] for i in g],
+                c["prep_host_y"] = hl.PreparedMulti(c["descs"], c["blobs"], c["xs"], B if multi else 8, [mats[i]["y_host"] for i in g],
                                                     c["wss"], ws_each, err)
             x_bytes = pk["x_host"].numel() * pk["x_host"].element_size()
             assert x_bytes % 16 == 0
@@ -776,7 +778,7 @@ def main():
                      "traffic_per_step": None if NCU_TRAFFIC_RATIO is None else NCU_TRAFFIC_RATIO * alg_bytes,
                      "traffic_note": "DRAM bytes read + written per launch (average over the step's launches): algorithmic bytes x the "
                                      "ratio of the ncu capture in profiles/ (1.036)",
-                     "peak_source": peak_src, "kernel": "huff_kernel<product>" if B <= 8 else "huff_gemm_tc_kernel", "launches_per_step": len(groups), "fuse": args.fuse,
+                     "peak_source": peak_src, "kernel": "huff_kernel<product>" if B <= 8 else ("huff_kernel<product, two tiles>" if multi else "huff_gemm_tc_kernel"), "launches_per_step": len(groups), "fuse": args.fuse,
                      "algorithmic_bytes_per_step": alg_bytes, "kernel_ms_per_step": kernel_ms_step,
                      "frac_of_nominal_8TBs": achieved / 8000.0,
                      "one_launch": None if not one_launch_ms else {

@@ -317,12 +317,15 @@ huffllm_status huffllm_decode_gemm_multi(uint32_t n, const huffllm_desc *const *
     if (st != HUFFLLM_OK) return st;
     if (!descs || !blobs || !xs || !ys || !workspaces) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
     if (n == 0 || n > kMaxMats) return fail(HUFFLLM_ERR_INVALID_ARG, "between 1 and %u matrices per call", kMaxMats);
-    if (batch == 0 || batch > kKernelBatch) return fail(HUFFLLM_ERR_UNSUPPORTED, "batch must be in [1, %u] here", kKernelBatch);
+    if (batch == 0 || batch > kTwoTileBatch)
+        return fail(HUFFLLM_ERR_UNSUPPORTED, "batch must be in [1, %u] here (above %u: BF16 blobs of max_code_len 8 only)", kTwoTileBatch, kKernelBatch);
     KernelArgs k;
     uint32_t grid;
     begin_args(&k, batch, dev);
     for (uint32_t i = 0; i < n; ++i) {
         if ((st = check_product_args(descs[i], xs[i], ys[i], workspaces[i], workspace_bytes_each, batch)) != HUFFLLM_OK) return st;
+        if (batch > kKernelBatch && !two_tile_blob(descs[i]))
+            return fail(HUFFLLM_ERR_UNSUPPORTED, "more than %u vectors per call take BF16 blobs of max_code_len 8", kKernelBatch);
         for (uint32_t j = 0; j < i; ++j)
             if (workspaces[j] == workspaces[i]) return fail(HUFFLLM_ERR_INVALID_ARG, "matrices %u and %u share a workspace", j, i);
         if ((st = add_matrix(&k, descs[i], blobs[i])) != HUFFLLM_OK) return st;
@@ -331,6 +334,7 @@ huffllm_status huffllm_decode_gemm_multi(uint32_t n, const huffllm_desc *const *
         m.y = ys[i];
         m.ws_ticket = (unsigned int *)workspaces[i];
         m.ws_partial = (float *)((uint8_t *)workspaces[i] + ws_partial_offset(descs[i]));
+        m.ws_warp_pieces = (float *)((uint8_t *)workspaces[i] + ws_partial_offset(descs[i]) + ws_cta_pieces_bytes(batch));   // (used above 8 vectors)
     }
     if ((st = finish_args(&k, true, dev, &grid)) != HUFFLLM_OK) return st;
     k.err = err_flag;
@@ -425,7 +429,7 @@ huffllm_status huffllm_decode_gemm_multi_host_async(uint32_t n, const huffllm_de
     clear_error();
     if (!descs || !xs_host || !ys_host || !x_stages || !y_stages) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
     if (n == 0 || n > kMaxMats) return fail(HUFFLLM_ERR_INVALID_ARG, "between 1 and %u matrices per call", kMaxMats);
-    if (batch == 0 || batch > kKernelBatch) return fail(HUFFLLM_ERR_UNSUPPORTED, "batch must be in [1, %u] here", kKernelBatch);
+    if (batch == 0 || batch > kTwoTileBatch) return fail(HUFFLLM_ERR_UNSUPPORTED, "batch must be in [1, %u] here", kTwoTileBatch);
     cudaStream_t s = (cudaStream_t)stream;
     for (uint32_t i = 0; i < n; ++i) {     // nothing is enqueued before every argument has been looked at
         if (!descs[i] || !xs_host[i] || !ys_host[i] || !x_stages[i] || !y_stages[i]) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
@@ -434,6 +438,8 @@ huffllm_status huffllm_decode_gemm_multi_host_async(uint32_t n, const huffllm_de
         if (st != HUFFLLM_OK) return st;
         if (!blobs || !blobs[i] || ((uintptr_t)blobs[i] & 255))
             return fail(HUFFLLM_ERR_INVALID_ARG, "blob must be a 256-byte aligned device pointer");
+        if (batch > kKernelBatch && !two_tile_blob(descs[i]))
+            return fail(HUFFLLM_ERR_UNSUPPORTED, "more than %u vectors per call take BF16 blobs of max_code_len 8", kKernelBatch);
     }
     for (uint32_t i = 0; i < n; ++i) {
         cudaError_t e = cudaMemcpyAsync(x_stages[i], xs_host[i], (size_t)batch * descs[i]->cols * 2, cudaMemcpyHostToDevice, s);

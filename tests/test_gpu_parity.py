@@ -286,7 +286,7 @@ def test_long_code_tables_decode_and_product(hl, torch, rows, cols, ce, budget, 
         assert np.array_equal(y1, gpu_gemm(hl, torch, up, x)), "results must be bitwise reproducible"
 
 
-@pytest.mark.parametrize("batch", [1, 3])
+@pytest.mark.parametrize("batch", [1, 3, 13])
 def test_several_matrices_in_one_launch(hl, torch, batch):
     """Matrices of different shapes and chunk sizes through huffllm_decode_gemm_multi: every result against the
     oracle, and the launch must leave every workspace's control words zero."""
