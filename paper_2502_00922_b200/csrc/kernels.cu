@@ -535,6 +535,10 @@ __device__ __forceinline__ void fma_bf16x8(float &lo, float &hi, const uint4 &w,
 __global__ void __launch_bounds__(256, 4) plain_gemv_kernel(const __grid_constant__ PlainArgs A) {
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5, nwarps = (gridDim.x * blockDim.x) >> 5;
+    // launched like the compressed path: the next launch may start early, and this one asks for its first weights before
+    // the launch in front of it has finished; x is read only after that
+    pdl_launch_dependents();
+    bool waited_prior = false;
     uint32_t mi = 0;
     for (uint32_t u = warp; u < A.total_rows; u += nwarps) {
         while (mi + 1 < A.n_mats && u >= A.m[mi + 1].row_first) ++mi;
@@ -547,6 +551,10 @@ __global__ void __launch_bounds__(256, 4) plain_gemv_kernel(const __grid_constan
             uint4 p[8];
 #pragma unroll
             for (int j = 0; j < 8; ++j) p[j] = i + 32 * j < nv ? ldg_stream16(wr + i + 32 * j) : make_uint4(0, 0, 0, 0);
+            if (!waited_prior) {
+                pdl_wait_prior_grid();
+                waited_prior = true;
+            }
 #pragma unroll
             for (int j = 0; j < 8; ++j) {
                 const uint4 xv = i + 32 * j < nv ? __ldg(xr + i + 32 * j) : make_uint4(0, 0, 0, 0);
@@ -623,8 +631,16 @@ cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream)
 cudaError_t launch_plain_gemv(const PlainArgs &a, uint32_t sms, cudaStream_t stream) {
     const uint64_t blocks = ((uint64_t)a.total_rows + 7) / 8;               // 8 warps per CTA, a row per warp and turn
     const uint32_t grid = (uint32_t)(blocks < (uint64_t)sms * 4 ? blocks : (uint64_t)sms * 4);
-    plain_gemv_kernel<<<grid, 256, 0, stream>>>(a);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, plain_gemv_kernel, a);
 }
 
 }  // namespace huffllm
