@@ -91,6 +91,28 @@ __device__ __forceinline__ void mma_bf16_16816(float (&d)[4], uint32_t a0, uint3
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
 
+// Two mixed-precision multiply-adds: acc += w.lo * x.lo, then acc += w.hi * x.hi (bf16 halves of the two words).
+// The products are exact in f32; each addition rounds once.
+__device__ __forceinline__ void fma2_bf16(float &acc, uint32_t w, uint32_t x) {
+    asm("{\n\t.reg .b16 wl, wh, xl, xh;\n\t"
+        "mov.b32 {wl, wh}, %1;\n\t"
+        "mov.b32 {xl, xh}, %2;\n\t"
+        "fma.rn.f32.bf16 %0, wl, xl, %0;\n\t"
+        "fma.rn.f32.bf16 %0, wh, xh, %0;\n\t}"
+        : "+f"(acc)
+        : "r"(w), "r"(x));
+}
+
+__device__ __forceinline__ void fma2_f16(float &acc, uint32_t w, uint32_t x) {
+    asm("{\n\t.reg .b16 wl, wh, xl, xh;\n\t"
+        "mov.b32 {wl, wh}, %1;\n\t"
+        "mov.b32 {xl, xh}, %2;\n\t"
+        "fma.rn.f32.f16 %0, wl, xl, %0;\n\t"
+        "fma.rn.f32.f16 %0, wh, xh, %0;\n\t}"
+        : "+f"(acc)
+        : "r"(w), "r"(x));
+}
+
 // Arrival counter bump that publishes this warp's earlier stores and acquires the other arrivals' stores.
 __device__ __forceinline__ uint32_t arrive_acq_rel(unsigned int *counter) {
     uint32_t old;

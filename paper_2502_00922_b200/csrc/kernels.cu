@@ -52,9 +52,12 @@ namespace huffllm {
 // spend theirs on decoding.
 // NT = 8-column tiles of activations per product: 1 (batch 1..8) or 2 (batch 9..16: twice the multiply-adds on the same
 // decoded registers; the pieces that warps of a CTA exchange then live in the workspace, shared memory has no room for them).
+// NT = 0 (BF16 blobs, batch 1): no tensor core at all.  The two mma.sync of a block cost the decoders more issue time
+// than the sixteen mixed-precision multiply-adds (bf16 x bf16 + f32, `fma.rn.f32.bf16`) that a lane needs for its 16
+// weights and one vector: those run on the FMA pipe, which the decoder leaves idle.
 template <int MODE, int LB, int THREADS, int FMT, int NT = 1>
 __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant__ KernelArgs A) {
-    constexpr int kV = 4 * NT;                                // values a lane holds of a row group's 16 x batch outputs
+    constexpr int kV = NT == 2 ? 8 : 4;                       // values a lane holds of a row group's 16 x batch outputs
     constexpr uint32_t kRawBlock = FMT ? 64u : 512u;          // raw bytes of one block of a record
     constexpr uint32_t kRawLane = FMT ? 2u : 16u;             // of which one lane's share
     // raw part of a record with nkb blocks, in record units of 128 bytes (FP16: rounded up to whole units)
@@ -299,6 +302,17 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         // D fragment -> output order (o = column * 16 + row) through this warp's shared-memory entry
         const uint32_t ent = warp * 2 + ((uint32_t)rg == c_beg / KC ? 0u : 1u);
         float *mine = part_val + (size_t)ent * vals;
+        if (NT == 0) {
+            // acc[0]: this lane's eight columns of row g; acc[2]: of row g + 8.  The four lanes of a row add theirs
+            // (always in this order), and lane t = 0 then holds what the D fragment's column 0 would hold.
+            float s_lo = acc[0], s_hi = acc[2];
+            s_lo += __shfl_xor_sync(0xFFFFFFFFu, s_lo, 1);
+            s_hi += __shfl_xor_sync(0xFFFFFFFFu, s_hi, 1);
+            s_lo += __shfl_xor_sync(0xFFFFFFFFu, s_lo, 2);
+            s_hi += __shfl_xor_sync(0xFFFFFFFFu, s_hi, 2);
+            acc[0] = s_lo;
+            acc[2] = s_hi;
+        }
 #pragma unroll
         for (int j = 0; j < kV; ++j) {      // (tile j / 4 of the activations: columns 8 (j / 4) + 2 t, + 1)
             uint32_t col = 8 * (j >> 2) + 2 * t + (j & 1), row = g + 8 * ((j >> 1) & 1);
@@ -425,7 +439,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                     }
                     uint4 xv;
                     if (MODE == 1) {
-                        if (NT == 1) xv = __ldg((const uint4 *)xq);   // (two tiles: both are fetched behind the decoder, registers are short)
+                        if (NT <= 1) xv = __ldg((const uint4 *)xq);   // (two tiles: both are fetched behind the decoder, registers are short)
                         xq += 32;
                     }
 
@@ -440,7 +454,21 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                             xw = __ldg((const uint4 *)(xq - 32 + x_tile2));
                         }
                         float (&acc0)[4] = *reinterpret_cast<float (*)[4]>(&acc[0]);
-                        if (FMT) {
+                        if (NT == 0) {
+                            // the lane's weights a[i] (row g) and a[4 + i] (row g + 8) stand in columns 2 i, 2 i + 1 of its
+                            // eight, and xv holds the vector's entries of the same columns
+                            const uint32_t xs[4] = {xv.x, xv.y, xv.z, xv.w};
+#pragma unroll
+                            for (int i = 0; i < 4; ++i) {
+                                if (FMT) {
+                                    fma2_f16(acc[0], a[i], xs[i]);
+                                    fma2_f16(acc[2], a[4 + i], xs[i]);
+                                } else {
+                                    fma2_bf16(acc[0], a[i], xs[i]);
+                                    fma2_bf16(acc[2], a[4 + i], xs[i]);
+                                }
+                            }
+                        } else if (FMT) {
                             mma_f16_16816(acc0, a[0], a[4], a[1], a[5], xv.x, xv.y);
                             mma_f16_16816(acc0, a[2], a[6], a[3], a[7], xv.z, xv.w);
                         } else {
@@ -448,7 +476,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                             mma_bf16_16816(acc0, a[2], a[6], a[3], a[7], xv.z, xv.w);
                         }
                         if (NT == 2) {
-                            float (&acc1)[4] = *reinterpret_cast<float (*)[4]>(&acc[4 * (NT - 1)]);
+                            float (&acc1)[4] = *reinterpret_cast<float (*)[4]>(&acc[NT == 2 ? 4 : 0]);
                             if (FMT) {
                                 mma_f16_16816(acc1, a[0], a[4], a[1], a[5], xw.x, xw.y);
                                 mma_f16_16816(acc1, a[2], a[6], a[3], a[7], xw.z, xw.w);
@@ -621,6 +649,14 @@ cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t strea
 }
 
 cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
+    if (k.batch == 1 && k.fmt) {                  // one vector: multiply-adds on the FMA pipe
+        if (k.lut_bits == 7) return launch_one<1, 7, kThreads, 1, 0>(k, grid, stream);
+        return k.lut_bits > 8 ? launch_one<1, 12, kThreads, 1, 0>(k, grid, stream) : launch_one<1, 8, kThreads, 1, 0>(k, grid, stream);
+    }
+    if (k.batch == 1) {
+        if (k.lut_bits > 9) return launch_one<1, 12, kThreads, 0, 0>(k, grid, stream);
+        return k.lut_bits == 8 ? launch_one<1, 8, kThreads, 0, 0>(k, grid, stream) : launch_one<1, 9, kThreads, 0, 0>(k, grid, stream);
+    }
     if (k.batch > 8) return launch_one<1, 8, kThreads, 0, 2>(k, grid, stream);   // (the entry point sends only BF16 blobs of 8-bit tables here)
     if (k.fmt && k.lut_bits == 7) return launch_one<1, 7, kThreads, 1>(k, grid, stream);
     if (k.fmt) return k.lut_bits > 8 ? launch_one<1, 12, kThreads, 1>(k, grid, stream) : launch_one<1, 8, kThreads, 1>(k, grid, stream);
