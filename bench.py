@@ -54,9 +54,9 @@ def launch_groups(table, fuse: str):
     return [[i] for i in range(n)]
 FALLBACK_HBM_GBS = 6650.0
 # dram__bytes_read.sum + dram__bytes_write.sum of the step's four fused-product launches over their algorithmic bytes, from the
-# ncu capture summarised in profiles/huff_kernel_product_llama7b_layer.md (330.05 MB moved for 318.64 MB);
+# ncu capture summarised in profiles/huff_kernel_product_llama7b_layer.md (326.48 MB moved for 318.64 MB);
 # traffic = ratio * algorithmic bytes.
-NCU_TRAFFIC_RATIO = 1.036
+NCU_TRAFFIC_RATIO = 1.025
 
 
 def max_over_ranks(v: float, dist, device) -> float:
@@ -329,7 +329,8 @@ def small_batch_leg(hl, torch, dev, stream, chunk_elems: int, peak_for_small: fl
         alg = desc.payload_bytes + 4 * (desc.n_chunks + 1) + (4 << desc.lut_bits) + batch * (2 * cols + 4 * rows)
         out["batches"].append({"batch": batch, "ms": ms, "frac_of_hbm_peak": alg / (ms * 1e-3) / 1e9 / peak_for_small,
                                "uncompressed_GBs": 2.0 * rows * cols / (ms * 1e-3) / 1e9,
-                               "kernel": "huff_kernel<product> (mma.sync on the decoded registers)" if batch <= 8 else
+                               "kernel": "huff_kernel<product, one vector> (mixed-precision fma on the decoded registers)" if batch == 1 else
+                                         "huff_kernel<product> (mma.sync on the decoded registers)" if batch <= 8 else
                                          ("huff_kernel<product, two tiles of activations> (mma.sync on the decoded registers)" if batch <= 16
                                           else "huff_gemm_tc_kernel (tcgen05)")})
     assert int(err.item()) == 0
@@ -777,7 +778,7 @@ def main():
                      "traffic": None if NCU_TRAFFIC_RATIO is None else NCU_TRAFFIC_RATIO * alg_bytes / len(groups),
                      "traffic_per_step": None if NCU_TRAFFIC_RATIO is None else NCU_TRAFFIC_RATIO * alg_bytes,
                      "traffic_note": "DRAM bytes read + written per launch (average over the step's launches): algorithmic bytes x the "
-                                     "ratio of the ncu capture in profiles/ (1.036)",
+                                     "ratio of the ncu capture in profiles/ (1.025)",
                      "peak_source": peak_src, "kernel": "huff_kernel<product>" if B <= 8 else ("huff_kernel<product, two tiles>" if multi else "huff_gemm_tc_kernel"), "launches_per_step": len(groups), "fuse": args.fuse,
                      "algorithmic_bytes_per_step": alg_bytes, "kernel_ms_per_step": kernel_ms_step,
                      "frac_of_nominal_8TBs": achieved / 8000.0,
