@@ -228,6 +228,8 @@ GEMM_CASES = [
     (16, 256, 4096, 0, "gauss", 1),
     (48, 1056, 4096, 0, "gauss", 1),
     (40, 2080, 1024, 0, "student", 3),            # ragged rows, last column chunk holds a single block
+    (40, 2080, 1024, 0, "student", 1),            # the same as a matrix-vector product (multiply-adds on the FMA pipe)
+    (512, 4096, 4096, 9, "student", 1),           # ... with a 512-entry table
     (16, 65536, 4096, 0, "gauss", 1),             # one row group split over every CTA
     (32, 32768, 4096, 0, "gauss", 8),
     (2368, 512, 512, 0, "gauss", 2),
