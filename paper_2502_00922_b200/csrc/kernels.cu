@@ -603,6 +603,7 @@ __global__ void __launch_bounds__(256, 4) plain_gemv_kernel(const __grid_constan
 // address).  For the tens of kilobytes of activations and results of a decode step this is cheaper than a DMA copy:
 // inside a CUDA graph a copy node between kernel nodes costs about 10 microseconds, this kernel about 3.
 __global__ void __launch_bounds__(512) stage_copy_kernel(uint4 *__restrict__ dst, const uint4 *__restrict__ src, uint64_t n16) {
+    pdl_launch_dependents();   // a product kernel behind this copy may do its set-up meanwhile: it waits for the copy before it reads x
     for (uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; i < n16; i += (uint64_t)gridDim.x * blockDim.x) dst[i] = src[i];
 }
 
