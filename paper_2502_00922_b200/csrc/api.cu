@@ -81,7 +81,7 @@ struct TcPlan {
 };
 // Shared memory the tensor-core kernel needs with `tiles` 128-row tiles per CTA.
 // Stages of the tensor-core kernel: four, two at the widest batch padding, where shared memory is short.
-uint32_t tc_stages(uint32_t npad) { return npad == 64 ? 2u : 4u; }
+uint32_t tc_stages(uint32_t npad) { return npad == 64 ? 3u : 4u; }
 uint64_t tc_smem_need(const huffllm_desc *d, uint32_t npad, uint32_t tiles) {
     const bool fp16 = d->dtype == HUFFLLM_FP16;
     const uint32_t checks_per_block = fp16 ? 8 : (d->lut_bits == 8 ? 3 : 4);
@@ -95,7 +95,8 @@ TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn
     p.npad = batch <= 16 ? 16 : (batch <= 32 ? 32 : 64);
     p.tiles = 4;                                    // as many 8-warp tiles as the chunk slots leave room for
     while (p.tiles > 1 && tc_smem_need(d, p.npad, p.tiles) > dyn_smem) --p.tiles;
-    p.m_tiles = (d->row_groups + 8 * p.tiles - 1) / (8 * p.tiles);
+    const uint32_t n_dec = 8 * p.tiles < 31 ? 8 * p.tiles : 31;      // the CTA's last warp issues the MMAs and never decodes
+    p.m_tiles = (d->row_groups + n_dec - 1) / n_dec;
     // Column ranges: the one with the shortest finish time.  A CTA takes items b, b + grid, ... in turn; an item costs its
     // column chunks (ranges of one matrix differ by a chunk when ksplit does not divide the chunk count) plus an epilogue
     // worth about a quarter of a chunk.  Counting whole waves alone would pick many short, unequal ranges.

@@ -112,7 +112,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     constexpr bool SKIP = LB == 8 && FMT == 0 && NPAD < 64;
     constexpr int R = SKIP ? 4 : LB == 8 ? 3 : 2;
     constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
-    constexpr int S = NPAD == 64 ? 2 : kTcStages;          // the host's tc_stages(): shared memory is short at the widest padding
+    constexpr int S = NPAD == 64 ? 3 : kTcStages;          // the host's tc_stages(): shared memory is short at the widest padding
     constexpr uint32_t kBStage = NPAD * 64;                 // bytes of B per stage: NPAD rows x 32 columns of bf16
     constexpr uint32_t kLbo = 128, kSbo = 512;              // core matrices: 4 along K side by side, then the next 8 rows
     constexpr uint32_t kACol0 = kTcTiles * NPAD;            // first tensor-memory column of the A stages
@@ -122,12 +122,15 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     extern __shared__ __align__(128) uint8_t dyn_smem[];
     __shared__ __align__(8) uint64_t bars[kMaxWarps * 2];   // per warp: its two coded-copy barriers
     __shared__ __align__(8) uint64_t empty_bar[S];          // stage may be refilled (arrived on by tcgen05.commit)
+    __shared__ __align__(8) uint64_t full_bar[S];           // every decoder warp's share of the stage is in place
     __shared__ uint32_t s_tmem_base;
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const MatArgs &k = A.m[0];
     const uint32_t smem_base = smem_u32(dyn_smem);
-    const uint32_t n_tiles = A.tc_tiles, n_dec = n_tiles * 8;          // decoder warps; the others leave at once
+    // decoder warps: eight per tile, except that the CTA's last warp never decodes: it issues the MMAs (with four tiles the
+    // last tile has seven row groups; its last 16 rows are never read).  Warps between the decoders and the issuer leave at once.
+    const uint32_t n_tiles = A.tc_tiles, n_dec = min(n_tiles * 8u, 31u), issuer = 31u;
     const SmemPlan plan = plan_smem(smem_base, A, n_dec);
     if (plan.warps < n_dec) {                                   // the entry point sizes shared memory so that this cannot happen
         if (tid == 0 && A.err) atomicExch(A.err, -3);
@@ -156,6 +159,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     }
     if (tid < S) {
         mbar_init(smem_u32(&empty_bar[tid]), 1);
+        mbar_init(smem_u32(&full_bar[tid]), n_dec);
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     if (warp == 0) {
@@ -166,7 +170,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = s_tmem_base;
-    if (warp >= n_dec) {                 // not a decoder warp in this configuration: only the teardown barrier is left
+    if (warp >= n_dec && warp != issuer) {   // neither decoder nor issuer in this configuration: only the teardown barrier is left
         tc_fence_before();
         __syncthreads();
         return;
@@ -233,8 +237,11 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     const uint32_t a_dst0 = tmem + a_lane + kACol0 + tile * S * 16;
     const uint32_t x_dst0 = b_base + (x_n >> 3) * kSbo + x_kap * kLbo + (x_n & 7) * 16;
 
-    // One block of the stage protocol.  `a` = this warp's decoded 16 rows x 32 columns (null if the warp has no rows).
-    auto stage_block = [&](const uint32_t *a, const uint4 &xv, bool first_of_item) {
+    // One block of the stage protocol, decoder side.  `a` = this warp's decoded 16 rows x 32 columns (null if the warp has
+    // no rows).  The warp stores its share, says so on the stage's "full" barrier and goes on decoding: nobody waits for
+    // the other warps here.  A warp can run ahead of the slowest one by the depth of the stage ring and no further (it
+    // needs the stage back, which the issuer's tcgen05.commit announces on the "empty" barrier).
+    auto stage_block = [&](const uint32_t *a, const uint4 &xv) {
         const uint32_t s = gb % S, use = gb / S;
         if (use > 0) bounded_wait(smem_u32(&empty_bar[s]), (use - 1) & 1u);
         tc_fence_after();
@@ -248,21 +255,30 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
         tc_wait_st();
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the B slice must be visible to the tensor core's reads
         tc_fence_before();
-        // every decoder warp's rows and the activations of this block are in place: a hardware barrier, so that a warp
-        // that waits costs no issue slots (the decoders are bound by instruction issue; a polling loop would take
-        // slots from the warps that still decode)
-        asm volatile("bar.sync 1, %0;" ::"r"(n_dec * 32u) : "memory");
-        if (warp == (gb & 7u) && lane == 0) {                   // the first tile's warps take turns in issuing the block's MMAs
+        __syncwarp();
+        if (lane == 0) mbar_arrive(smem_u32(&full_bar[s]));
+        ++gb;
+    };
+    // The same block, issuer side: when every decoder warp has arrived, one lane issues the block's MMAs for every tile
+    // and commits them onto the stage's "empty" barrier.  (After a wait that ran out the commit still goes out: the
+    // stage ring keeps moving and the kernel ends with its error flag set.)
+    auto issue_block = [&](bool first_of_item) {
+        const uint32_t s = gb % S, use = gb / S;
+        bounded_wait(smem_u32(&full_bar[s]), use & 1u);
+        if (lane == 0) {
             tc_fence_after();
             const uint32_t bst = b_base + s * kBStage;
-            for (uint32_t tl = 0; tl < n_tiles; ++tl) {
+            if (!failed) {
+                for (uint32_t tl = 0; tl < n_tiles; ++tl) {
 #pragma unroll
-                for (uint32_t j = 0; j < 2; ++j)      // two K = 16 steps per stage
-                    tc_mma_f16_tmem_a(tmem + tl * NPAD, tmem + kACol0 + (tl * S + s) * 16 + j * 8,
-                                      smem_desc_kmajor(bst + j * 2 * kLbo, kLbo, kSbo), kIdesc, (first_of_item && j == 0) ? 0u : 1u);
+                    for (uint32_t j = 0; j < 2; ++j)      // two K = 16 steps per stage
+                        tc_mma_f16_tmem_a(tmem + tl * NPAD, tmem + kACol0 + (tl * S + s) * 16 + j * 8,
+                                          smem_desc_kmajor(bst + j * 2 * kLbo, kLbo, kSbo), kIdesc, (first_of_item && j == 0) ? 0u : 1u);
+                }
             }
             tc_commit(smem_u32(&empty_bar[s]));
         }
+        __syncwarp();
         ++gb;
     };
 
@@ -280,7 +296,9 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
         uint4 x_a = make_uint4(0, 0, 0, 0), x_b = make_uint4(0, 0, 0, 0);
         load_x(x_a, x_src + col_lo);
 
-        if (active) {
+        if (warp == issuer) {
+            for (uint32_t col_blk = col_lo; col_blk < col_hi; col_blk += 32) issue_block(gb == gb_item);
+        } else if (active) {
             const uint32_t c_beg = rg * KC + kc0, c_end = rg * KC + kc1;
             if (lane == 0) {
                 issue(c_beg, 0);
@@ -317,7 +335,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
 #pragma unroll
                         for (int i = 0; i < 8; ++i) a[i] = 0u;
                     }
-                    stage_block(a, x_c, gb == gb_item);
+                    stage_block(a, x_c);
                 };
                 uint4 raw_b = make_uint4(0, 0, 0, 0);
                 uint32_t kb = 0;
@@ -340,13 +358,14 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
             for (uint32_t col_blk = col_lo; col_blk < col_hi; col_blk += 32) {
                 if (x_p < x_end) load_x(x_b, x_p);
                 x_p += 32;
-                stage_block(nullptr, x_a, gb == gb_item);
+                stage_block(nullptr, x_a);
                 x_a = x_b;
             }
         }
 
         // ---- epilogue of the item: wait for the last stage's MMAs, read this warp's 32 rows x NPAD/2 columns
-        {
+        // (the issuer has a share like every warp of a tile; with fewer than four tiles its tile does not exist)
+        if (tile < n_tiles) {
             const uint32_t gl = gb - 1;
             bounded_wait(smem_u32(&empty_bar[gl % S]), (gl / S) & 1u);
             tc_fence_after();
@@ -356,11 +375,12 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
             tc_fence_before();
             // thread `lane` holds row 32 q + lane of the tile, columns n = h * NPAD/2 + i
             const uint64_t row = (uint64_t)(mt * n_dec + tile * 8) * 16 + 32u * q + lane;
+            const bool row_ok = row < k.rows && tile * 8 + 2 * q + (lane >> 4) < n_dec;   // (the last tile's last row group belongs to the next item)
             const uint32_t n0 = h * (NPAD / 2);
             if (ksplit == 1) {
 #pragma unroll
                 for (int i = 0; i < NPAD / 2; ++i)
-                    if (n0 + i < A.batch && row < k.rows) k.y[(uint64_t)(n0 + i) * k.rows + row] = __uint_as_float(v[i]);
+                    if (n0 + i < A.batch && row_ok) k.y[(uint64_t)(n0 + i) * k.rows + row] = __uint_as_float(v[i]);
             } else {
                 // piece of (item, warp): [NPAD/2][32] floats; the last range to arrive adds the pieces in range order
                 float *piece = A.tc_partial + ((size_t)item * 32 + warp) * (NPAD / 2) * 32;   // 32 piece slots per item, n_dec used
@@ -385,7 +405,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                     }
 #pragma unroll
                     for (int i = 0; i < NPAD / 2; ++i)
-                        if (n0 + i < A.batch && row < k.rows) k.y[(uint64_t)(n0 + i) * k.rows + row] = sum[i];
+                        if (n0 + i < A.batch && row_ok) k.y[(uint64_t)(n0 + i) * k.rows + row] = sum[i];
                 }
             }
         }
