@@ -282,6 +282,15 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
         ++gb;
     };
 
+    // first and last chunk of this warp's row group in a work item (false: the row group lies outside the matrix)
+    auto item_chunks = [&](uint32_t it, uint32_t &cb, uint32_t &ce) -> bool {
+        const uint32_t mt_i = it / ksplit, ks_i = it % ksplit, rg_i = mt_i * n_dec + rgi;
+        cb = rg_i * KC + (uint32_t)((uint64_t)KC * ks_i / ksplit);
+        ce = rg_i * KC + (uint32_t)((uint64_t)KC * (ks_i + 1) / ksplit);
+        return rg_i < RG;
+    };
+    bool primed = false;                 // the item's first two record copies were started at the end of the item before
+
 #pragma unroll 1
     for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
         const uint32_t mt = item / ksplit, ks = item % ksplit;
@@ -300,7 +309,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
             for (uint32_t col_blk = col_lo; col_blk < col_hi; col_blk += 32) issue_block(gb == gb_item);
         } else if (active) {
             const uint32_t c_beg = rg * KC + kc0, c_end = rg * KC + kc1;
-            if (lane == 0) {
+            if (lane == 0 && !primed) {
                 issue(c_beg, 0);
                 if (c_beg + 1 < c_end) issue(c_beg + 1, 1);
             }
@@ -360,6 +369,19 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                 x_p += 32;
                 stage_block(nullptr, x_a);
                 x_a = x_b;
+            }
+        }
+
+        // both slots are free again: the next item's first records are asked for now, so that they arrive behind the epilogue
+        primed = false;
+        if (warp < n_dec && item + gridDim.x < n_items) {
+            uint32_t nb, ne;
+            if (item_chunks(item + gridDim.x, nb, ne)) {
+                if (lane == 0) {
+                    issue(nb, 0);
+                    if (nb + 1 < ne) issue(nb + 1, 1);
+                }
+                primed = true;
             }
         }
 
