@@ -107,9 +107,8 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
         if (FMT) return make_uint4(ldg_stream2(p), 0, 0, 0);
         return ldg_stream16(p);
     };
-    // the decoder that starts behind the leading zero bits (see huff_kernel); at the widest padding, where a block's
-    // time is set by the two-stage hand-over, it measured 1.4 % slower and is left out
-    constexpr bool SKIP = LB == 8 && FMT == 0 && NPAD < 64;
+    // the decoder that starts behind the leading zero bits and takes four codewords at a time (see huff_kernel)
+    constexpr bool SKIP = LB == 8 && FMT == 0;
     constexpr int R = SKIP ? 4 : LB == 8 ? 3 : 2;
     constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
     constexpr int S = NPAD == 64 ? 3 : kTcStages;          // the host's tc_stages(): shared memory is short at the widest padding
