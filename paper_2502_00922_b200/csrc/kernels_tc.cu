@@ -223,6 +223,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     // piece u = 32 warp + lane belongs to vector n = u / 4 and K positions 8 kap .. 8 kap + 7 (kap = u % 4) of the
     // tile, which hold columns base .. base + 3 and base + 8 .. base + 11 of the block, base = 16 (kap & 1) + 4 (kap >> 1).
     const bool x_carrier = warp * 32 + lane < NPAD * 4;
+    const bool x_carrier_warp = warp * 32 < NPAD * 4;            // (NPAD * 4 is a multiple of 32: whole warps carry)
     const uint32_t x_n = (warp * 32 + lane) >> 2, x_kap = lane & 3;
     const uint16_t *x_src = k.x + (uint64_t)x_n * k.cols + (x_kap & 1) * 16 + (x_kap >> 1) * 4;
     const bool x_loads = x_carrier && x_n < A.batch;         // carriers of padding vectors stage zeros
@@ -252,7 +253,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
         if (x_carrier)
             asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(x_dst0 + s * kBStage), "r"(xv.x), "r"(xv.y), "r"(xv.z), "r"(xv.w) : "memory");
         tc_wait_st();
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the B slice must be visible to the tensor core's reads
+        if (x_carrier_warp) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the B slice must be visible to the tensor core's reads
         tc_fence_before();
         __syncwarp();
         if (lane == 0) mbar_arrive(smem_u32(&full_bar[s]));
@@ -326,6 +327,21 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                 bounded_wait(bar0 + which * 8, (phase >> which) & 1u);
                 phase ^= 1u << which;
                 if (!ok && A.err && lane == 0) atomicExch(A.err, (int32_t)min(c + 1, 0x7FFFFFFFu));
+                if (!ok) {
+                    // record offsets out of range (reported above): nothing of the record is touched, zeros go to the stages
+                    const uint32_t zero[8] = {0u, 0u, 0u, 0u, 0u, 0u, 0u, 0u};
+                    for (uint32_t kb = 0; kb < nkb; ++kb) {
+                        if (x_p < x_end) load_x(x_b, x_p);
+                        x_p += 32;
+                        stage_block(zero, x_a);
+                        x_a = x_b;
+                    }
+                    __syncwarp();
+                    if (lane == 0 && c + 2 < c_end) issue(c + 2, which);
+                    r0 = r1;
+                    r1 = r2;
+                    continue;
+                }
                 LaneStream sa, sb;
                 stream_open(sa, slot0 + which * A.slot_bytes + (lane << 2), SKIP ? 7u : 0u);
                 stream_open(sb, slot0 + which * A.slot_bytes + 128u + (lane << 2), SKIP ? 7u : 0u);
@@ -333,16 +349,12 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                 // this one, hand it to the tensor core
                 auto block = [&](const uint4 &raw_c, uint4 &raw_n, const uint4 &x_c, uint4 &x_n2, bool more) {
                     raw_p += kRawBlock;
-                    if (more && ok) raw_n = load_raw(raw_p);
+                    if (more) raw_n = load_raw(raw_p);
                     if (x_p < x_end) load_x(x_n2, x_p);
                     x_p += 32;
                     uint32_t a[8];
-                    if (FMT) decode_block_fp16(sa, sb, lut_lane, raw_c.x, a);   // a chunk that is not ok decodes garbage, never out of range
+                    if (FMT) decode_block_fp16(sa, sb, lut_lane, raw_c.x, a);
                     else decode_block<R, SKIP>(sa, sb, kIdxMask, lut_lane, raw_c, a);
-                    if (!ok) {                                    // ... and contributes nothing, as on the register path
-#pragma unroll
-                        for (int i = 0; i < 8; ++i) a[i] = 0u;
-                    }
                     stage_block(a, x_c);
                 };
                 uint4 raw_b = make_uint4(0, 0, 0, 0);

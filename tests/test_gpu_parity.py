@@ -392,6 +392,19 @@ def test_bad_record_offsets_are_reported_not_followed(hl, torch):
         rg, kc = divmod(c, up.desc.col_chunks)
         good[rg * 16:(rg + 1) * 16, kc * kc_cols:(kc + 1) * kc_cols] = False
     assert np.array_equal(got[good], w[good])
+    # the products, on every consume path (one vector, one tile, two tiles, tensor core): the two chunks add nothing
+    w_skipped = np.where(good, w, np.uint16(0))
+    for batch in (1, 4, 13, 32):
+        x = wl.activations(batch, cols, 50 + batch)
+        x_dev = torch.from_numpy(x.view(np.int16)).cuda()
+        ws_bytes = hl.workspace_bytes(up.desc, batch)
+        ws = torch.zeros(ws_bytes, dtype=torch.uint8, device="cuda")
+        y = torch.full((batch * rows,), float("nan"), dtype=torch.float32, device="cuda")
+        up.err.zero_()
+        hl.decode_gemm(up.desc, dev, x_dev, batch, y, ws, ws_bytes, up.err)
+        torch.cuda.synchronize()
+        assert int(up.err.item()) != 0
+        check_product(y.cpu().numpy().reshape(batch, rows), w_skipped, x)
 
 
 def test_damaged_coded_part_is_reported_and_contained(hl, torch):
