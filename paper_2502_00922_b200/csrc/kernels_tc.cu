@@ -8,16 +8,20 @@
 // produced (Section 1 of the paper: decompress only to multiply) and one pass over the compressed bytes
 // serves the whole batch; the tensor pipe only takes the batch-fold of multiply-adds off the issue slots.
 //
-// Geometry of a CTA: 32 decoder warps = 4 tiles of 8 warps; a tile is 128 rows (8 row groups of 16), warp
-// (q = warp % 4, h = warp / 4 % 2) of a tile owns tensor-memory lanes 32 q + 16 h .. + 15, which is what the
-// 16x256b store shape of a warp can reach.  Tensor memory (512 columns): 4 accumulators of N columns, then
-// 4 tiles x 4 stages x 16 columns of A (a stage = one block of 32 weight columns = two K = 16 steps).
-// A work item is (512 rows) x (a range of column chunks); partial results of the ranges of one row tile are
+// Geometry of a CTA: 4 tiles of 8 warps; a tile is 128 rows (8 row groups of 16), warp (q = warp % 4, h = warp / 4 % 2)
+// of a tile owns tensor-memory lanes 32 q + 16 h .. + 15, which is what the 16x256b store shape of a warp can reach.
+// The CTA's LAST warp does not decode: it issues the MMAs (so a CTA decodes 31 row groups at a time, and the last 16 rows
+// of the fourth tile are never read).  Tensor memory (512 columns): 4 accumulators of N columns, then 4 tiles x S stages
+// x 16 columns of A (a stage = one block of 32 weight columns = two K = 16 steps).
+// A work item is (31 row groups) x (a range of column chunks); partial results of the ranges of one row tile are
 // added in a fixed order by whoever finishes last (per-warp arrival counters, nobody waits).
 //
-// Stage protocol: every warp fills its share of stage s (A rows, a slice of B) and meets the other decoder warps at
-// a hardware barrier; one of them (they take turns) then issues the 8 MMAs of the stage and a tcgen05.commit onto
-// the stage's "empty" mbarrier, which the warps wait on (with a limit) before they reuse the stage four blocks later.
+// Stage protocol: a decoder warp fills its share of stage s (A rows, a slice of B), arrives on the stage's "full"
+// mbarrier and goes on decoding; no warp waits for another one except through the depth of the stage ring.  The issuer
+// warp waits for a stage to be full, issues its 8 MMAs and a tcgen05.commit onto the stage's "empty" mbarrier, which the
+// decoders wait on (with a limit) before they reuse the stage.  (With the issue taking turns among the decoder warps and a
+// barrier after every block, each block cost the CTA its decode time plus the 2000 cycles one warp needs to issue the
+// MMAs: that warp had to decode its next block before the next barrier could open.)
 // BF16 and FP16 {1,5,5,5} blobs share the kernel (template parameter FMT): tables, raw part and operand format differ.
 #include <atomic>
 
