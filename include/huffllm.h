@@ -251,6 +251,17 @@ huffllm_status huffllm_decode_smem_plan(const huffllm_desc *desc, uint32_t *tabl
                                         uint32_t *refill_checks_per_block, uint32_t *guard_bytes);
 
 /*
+ * How a CTA of huffllm_decode (batch 0) or of the products of 1 to 8 vectors is laid out for this blob (host call, no device
+ * needed; any pointer may be null).  `smem_bytes_per_cta`: the GPU's opt-in shared memory per CTA, 0 = the B200's 232448.
+ * slots_per_warp: 2 where every decoder warp can keep two records in shared memory (the next one lands while this one is
+ * decoded), 1 where records are so large that pairs would leave fewer than 31 warps a place and single slots serve at
+ * least a quarter more of them.  decoder_warps: how many of a CTA's 31 decoder warps get a place, at least.
+ * HUFFLLM_ERR_UNSUPPORTED if not even one record fits.
+ */
+huffllm_status huffllm_decode_launch_plan(const huffllm_desc *desc, uint32_t batch, uint32_t smem_bytes_per_cta,
+                                          uint32_t *slots_per_warp, uint32_t *decoder_warps);
+
+/*
  * y = W x with W taken straight from the compressed blob: weights are decoded in registers and
  * multiplied at once, so only compressed bytes cross the memory bus (Section 1: weights are
  * decompressed only when needed, to multiply with activations).  x: device, cols words of the

@@ -48,6 +48,7 @@ _SIGNATURES = {
     "huffllm_workspace_bytes": [C.POINTER(Desc), C.c_uint32, C.POINTER(C.c_size_t)],
     "huffllm_workspace_control_bytes": [C.POINTER(Desc), C.POINTER(C.c_size_t)],
     "huffllm_decode_smem_plan": [C.POINTER(Desc), C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)],
+    "huffllm_decode_launch_plan": [C.POINTER(Desc), C.c_uint32, C.c_uint32, C.POINTER(C.c_uint32), C.POINTER(C.c_uint32)],
     "huffllm_decode": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemv": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
     "huffllm_decode_gemm": [C.POINTER(Desc), C.c_void_p, C.c_void_p, C.c_uint32, C.c_void_p, C.c_void_p, C.c_size_t, C.c_void_p, C.c_void_p],
@@ -211,6 +212,13 @@ def decode_smem_plan(desc: Desc) -> dict:
     t, sl, ch, g = C.c_uint32(), C.c_uint32(), C.c_uint32(), C.c_uint32()
     _check(lib().huffllm_decode_smem_plan(C.byref(desc), C.byref(t), C.byref(sl), C.byref(ch), C.byref(g)))
     return {"table_bytes": t.value, "slot_bytes": sl.value, "refill_checks_per_block": ch.value, "guard_bytes": g.value}
+
+
+def decode_launch_plan(desc: Desc, batch: int = 1, smem_bytes_per_cta: int = 0) -> dict:
+    """huffllm_decode_launch_plan: slots per decoder warp (2, or 1 for large records) and the decoder warps that get a place."""
+    s, w = C.c_uint32(), C.c_uint32()
+    _check(lib().huffllm_decode_launch_plan(C.byref(desc), batch, smem_bytes_per_cta, C.byref(s), C.byref(w)))
+    return {"slots_per_warp": s.value, "decoder_warps": w.value}
 
 
 def decode(desc: Desc, blob_dev, out_dev, err_flag_dev=None, stream=None):

@@ -195,19 +195,28 @@ huffllm_status add_matrix(KernelArgs *k, const huffllm_desc *desc, const void *b
     k->lut_align = need.table_align;
     k->lut_size = need.table_bytes;
     if (need.slot_bytes > k->slot_bytes) k->slot_bytes = need.slot_bytes;
-    k->pair_recip = (uint32_t)(0x100000000ull / (2ull * k->slot_bytes));
     if (need.guard_bytes > k->guard_bytes) k->guard_bytes = need.guard_bytes;
     return HUFFLLM_OK;
 }
 
 // Close a launch description: shared-memory budget and grid size.
-huffllm_status finish_args(KernelArgs *k, bool product, const DeviceInfo &dev, uint32_t *grid) {
+huffllm_status finish_args(KernelArgs *k, bool product, const DeviceInfo &dev, uint32_t *grid, uint32_t *warps_at_least = nullptr) {
     // (pieces that warps of a CTA exchange: in shared memory up to 8 vectors, in the workspace above)
     k->part_bytes = product && k->batch <= kKernelBatch ? 2 * 32 * 16 * k->batch * (uint32_t)sizeof(float) : 0;
     // worst case for the table's alignment gap is covered by assuming the window starts within 4 KB of zero
     uint64_t fixed = (uint64_t)k->lut_size + (k->guard_bytes > k->part_bytes ? k->guard_bytes - k->part_bytes : 0) + k->part_bytes + 4096;
-    if (fixed + 2ull * k->slot_bytes > k->dyn_smem_bytes)
+    if (fixed + k->slot_bytes > k->dyn_smem_bytes)
         return fail(HUFFLLM_ERR_UNSUPPORTED, "chunk records too large for shared memory (slot %u bytes)", k->slot_bytes);
+    // Two slots per decoder warp, so that a warp's next record lands while it decodes this one.  Where records are so large
+    // that this would leave fewer than 31 warps a slot pair, and single slots serve at least a quarter more warps, every
+    // warp gets one slot: more decoders at work outweigh the wait for a copy at every chunk start.
+    const uint64_t room = k->dyn_smem_bytes - fixed, max_w = 31;     // decoder warps of a CTA of 1024 threads
+    uint64_t w2 = room / (2ull * k->slot_bytes), w1 = room / k->slot_bytes;
+    if (w2 > max_w) w2 = max_w;
+    if (w1 > max_w) w1 = max_w;
+    k->slots = w2 < max_w && 4 * w1 >= 5 * w2 ? 1u : 2u;
+    if (warps_at_least) *warps_at_least = (uint32_t)(k->slots == 1 ? w1 : w2);
+    k->pair_recip = (uint32_t)(0x100000000ull / ((uint64_t)k->slots * k->slot_bytes));
     uint64_t g = k->total_chunks < (uint64_t)dev.sms ? k->total_chunks : (uint64_t)dev.sms;
     *grid = (uint32_t)(g < kMaxGrid ? g : kMaxGrid);
     // deal the CTAs out to the matrices: one each, then always to the matrix with the most chunks per CTA, so that
@@ -278,6 +287,25 @@ huffllm_status huffllm_decode_smem_plan(const huffllm_desc *desc, uint32_t *tabl
     if (slot_bytes) *slot_bytes = n.slot_bytes;
     if (refill_checks_per_block) *refill_checks_per_block = n.checks_per_block;
     if (guard_bytes) *guard_bytes = n.guard_bytes;
+    return HUFFLLM_OK;
+}
+
+huffllm_status huffllm_decode_launch_plan(const huffllm_desc *desc, uint32_t batch, uint32_t smem_bytes_per_cta,
+                                          uint32_t *slots_per_warp, uint32_t *decoder_warps) {
+    clear_error();
+    huffllm_status st = check_desc(desc);
+    if (st != HUFFLLM_OK) return st;
+    if (batch > kKernelBatch) return fail(HUFFLLM_ERR_INVALID_ARG, "the plan is that of the register path: batch 0 (decode) to %u", kKernelBatch);
+    DeviceInfo dev = {};
+    dev.sms = 148;
+    dev.smem_optin = smem_bytes_per_cta ? smem_bytes_per_cta : 232448;
+    KernelArgs k;
+    uint32_t grid = 0, warps = 0;
+    begin_args(&k, batch ? batch : 1, dev);
+    if ((st = add_matrix(&k, desc, (const void *)256)) != HUFFLLM_OK) return st;     // (the pointer is only checked for alignment)
+    if ((st = finish_args(&k, batch != 0, dev, &grid, &warps)) != HUFFLLM_OK) return st;
+    if (slots_per_warp) *slots_per_warp = k.slots;
+    if (decoder_warps) *decoder_warps = warps;
     return HUFFLLM_OK;
 }
 
@@ -384,6 +412,8 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
         begin_args(&k, batch, dev);
         if ((st = add_matrix(&k, desc, blob)) != HUFFLLM_OK) return st;
         k.part_bytes = tc_stages(tp.npad) * tp.npad * 64;      // the stages of activations
+        k.slots = 2;
+        k.pair_recip = (uint32_t)(0x100000000ull / (2ull * k.slot_bytes));
         const uint64_t need = tc_smem_need(desc, tp.npad, tp.tiles);
         if (need <= k.dyn_smem_bytes && workspace_bytes >= tp.bytes) {
             k.m[0].x = x;

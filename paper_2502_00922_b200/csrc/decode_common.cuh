@@ -447,7 +447,7 @@ __device__ __forceinline__ void decode_block_fp16(LaneStream &sa, LaneStream &sb
 // ------------------------------------------------------------------------------ shared memory plan
 
 // Dynamic shared memory, laid out at run time from the window's real start address:
-//   [base, lut)            slot pairs (as many as fit)
+//   [base, lut)            slot pairs (single slots where the launch says so), as many as fit
 //   [lut, lut + LUTSZ)     per-lane LUT; lut = base rounded up to a multiple of LUTSZ, so that the
 //                          index bits of a lookup address never overlap the table's base bits
 //   [lut + LUTSZ, ...)     more slot pairs, then a guard area no valid stream ever reads (it may overlap the next area)
@@ -468,7 +468,7 @@ __device__ __forceinline__ SmemPlan plan_smem(uint32_t base, const KernelArgs &k
     p.slotA = a0;
     // (divisions by the slot pair's size as a multiplication by its rounded-down reciprocal and one correction: this
     // runs in every warp of a launch's set-up, which is bound by instruction issue)
-    const uint32_t pair = 2 * k.slot_bytes;
+    const uint32_t pair = k.slots * k.slot_bytes;
     auto div_pair = [&](uint32_t x) -> uint32_t {
         uint32_t q = __umulhi(x, k.pair_recip);
         return x - q * pair >= pair ? q + 1 : q;
@@ -483,9 +483,9 @@ __device__ __forceinline__ SmemPlan plan_smem(uint32_t base, const KernelArgs &k
     return p;
 }
 
-__device__ __forceinline__ uint32_t slot_addr(const SmemPlan &p, uint32_t warp, uint32_t which, uint32_t slot_bytes) {
-    uint32_t pair = warp < p.nA ? p.slotA + warp * 2 * slot_bytes : p.slotB + (warp - p.nA) * 2 * slot_bytes;
-    return pair + which * slot_bytes;
+// First slot of a decoder warp; `pair_bytes` = slots per warp x slot bytes.
+__device__ __forceinline__ uint32_t slot_addr(const SmemPlan &p, uint32_t warp, uint32_t pair_bytes) {
+    return warp < p.nA ? p.slotA + warp * pair_bytes : p.slotB + (warp - p.nA) * pair_bytes;
 }
 
 constexpr int kMaxWarps = 32;

@@ -132,13 +132,15 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         // the barriers exist: the decoders may go on as soon as their table is built; the feeder does not wait for them
         asm volatile("bar.arrive %0, %1;" ::"r"(kSetupBarrier), "r"(THREADS) : "memory");
         uint32_t f_kc = f_ci % KC;
-        const uint32_t slot_units = A.slot_bytes >> 7, slot_w = slot_addr(plan, lane < nw ? lane : 0u, 0, A.slot_bytes);
+        const uint32_t slot_units = A.slot_bytes >> 7, slot_w = slot_addr(plan, lane < nw ? lane : 0u, A.slots * A.slot_bytes);
         const uint32_t note_w = smem_u32(&notes[lane * 2]);
         uint32_t idle = 0;
         while (__any_sync(0xFFFFFFFFu, f_ci < f_ce)) {
             const uint32_t which = f_issued & 1u;
-            // a slot is free for its first chunk, and later once the decoder has handed it back
-            const bool ready = f_ci < f_ce && (f_issued < 2 || mbar_test_wait(bar_w + 16 + 8 * which, ((f_issued >> 1) - 1u) & 1u));
+            // a slot is free for its first chunk, and later once the decoder has handed it back: with two slots that is the
+            // chunk before the last one issued, with one slot the last one (barriers and notes alternate either way)
+            const uint32_t f_back = f_issued - A.slots;
+            const bool ready = f_ci < f_ce && (f_issued < A.slots || mbar_test_wait(bar_w + 16 + 8 * (f_back & 1u), (f_back >> 1) & 1u));
             if (ready) {
                 const uint32_t full = bar_w + 8 * which, nkb = f_kc + 1 == KC ? nkb_tail : nkb_full;
                 // a record is usable if it lies inside the payload, is longer than its raw part and its coded part fits a slot
@@ -147,7 +149,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                 if (ok) {
                     const uint32_t bytes = (f_rb - f_ra - raw_units(nkb)) << 7;
                     mbar_expect_tx(full, bytes);
-                    bulk_g2s(slot_w + which * A.slot_bytes, payload + ((uint64_t)(f_ra + raw_units(nkb)) << 7), bytes, full);
+                    bulk_g2s(slot_w + (which & (A.slots - 1u)) * A.slot_bytes, payload + ((uint64_t)(f_ra + raw_units(nkb)) << 7), bytes, full);
                     // the raw part of the record is asked into L2 with one request (not for a warp's first two chunks: at the
                     // start of a launch every warp's copies are under way at once, and only the decoders' own loads matter)
                     if (f_issued >= 2)
@@ -362,8 +364,8 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         const uint64_t x_tile2 = NT == 2 ? (uint64_t)(min(g + 8u, A.batch - 1) - min(g, A.batch - 1)) * k.cols : 0;
         // this chunk's slot (the lane's column of it), its barrier and its note, toggled by XOR from chunk to chunk; parity
         // of the barrier's next completion (each of the two "full" barriers completes every second chunk)
-        uint32_t slot_cur = slot_addr(plan, warp, 0, A.slot_bytes) + (lane << 2), bar_cur = bar_w, par = 0, which = 0;
-        const uint32_t slot_tog = slot_cur ^ (slot_cur + A.slot_bytes);
+        uint32_t slot_cur = slot_addr(plan, warp, A.slots * A.slot_bytes) + (lane << 2), bar_cur = bar_w, par = 0, which = 0;
+        const uint32_t slot_tog = A.slots == 2 ? slot_cur ^ (slot_cur + A.slot_bytes) : 0u;   // (one slot: every chunk lands in the same place)
         uint32_t note_cur = smem_u32(&notes[warp * 2]);
 
 #pragma unroll 1

@@ -213,14 +213,26 @@ def test_fp16_seven_bit_field_codes(hl, torch, rows, cols, ce, gen, batch):
         check_product(gpu_gemm(hl, torch, up, x), w, x, orc.FP16)
 
 
-def test_fp16_large_chunks_run_with_fewer_warps(hl, torch):
-    """Records too large for 32 pairs of shared-memory slots are decoded by as many warps as have room."""
+def test_fp16_large_chunks_run_on_single_slots(hl, torch):
+    """Records too large for 31 pairs of shared-memory slots: every decoder warp gets one slot instead of a pair
+    (4096-element FP16 chunks keep 22 of 31 warps that way, against 11); still larger ones are decoded by as many warps as have room."""
     w = wl.gaussian_weights(64, 4096, 0.02, 990, "fp16")
     up = Uploaded(hl, torch, w, 16384, 0, 1, dtype=hl.FP16)
     assert up.desc.max_words > 64
+    plan = hl.decode_launch_plan(up.desc, 1)
+    assert plan["slots_per_warp"] == 1 and 2 <= plan["decoder_warps"] < 31
     assert np.array_equal(gpu_decode(hl, torch, up), w)
     x = wl.activations(1, 4096, 991, "fp16")
     check_product(gpu_gemm(hl, torch, up, x), w, x, orc.FP16)
+    # the benchmark chunk size: single slots for two thirds of the warps; many chunks per warp, so that slots are reused
+    w = wl.gaussian_weights(1040, 4096, 0.02, 992, "fp16")
+    up = Uploaded(hl, torch, w, 4096, 0, 3, dtype=hl.FP16)
+    plan = hl.decode_launch_plan(up.desc, 1)
+    assert plan["slots_per_warp"] == 1 and plan["decoder_warps"] >= 20
+    assert np.array_equal(gpu_decode(hl, torch, up), w)
+    for batch in (1, 3):
+        x = wl.activations(batch, 4096, 993 + batch, "fp16")
+        check_product(gpu_gemm(hl, torch, up, x), w, x, orc.FP16)
 
 
 GEMM_CASES = [

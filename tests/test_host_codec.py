@@ -294,6 +294,35 @@ def test_device_call_sizes_are_consistent():
         hl.workspace_bytes(d, 65)
 
 
+def test_launch_plan_slots_per_warp():
+    """Two slots per decoder warp where 31 pairs fit, one where records are large: the plan of a decoder CTA as the library
+    reports it (host only), checked against the shared-memory arithmetic of the header."""
+    smem = 232448
+    for dtype, name, ce, slots in ((hl.BF16, "bf16", 4096, 2), (hl.BF16, "bf16", 8192, 1), (hl.FP16, "fp16", 1024, 2),
+                                   (hl.FP16, "fp16", 4096, 1), (hl.FP16, "fp16", 16384, 1)):
+        w = wl.gaussian_weights(64, 4096, 0.02, 94, name)
+        cb = hl.build_codebook(w, dtype)
+        _, d = hl.encode(cb, w, ce)
+        cb.free()
+        sp = hl.decode_smem_plan(d)
+        for batch in (0, 1, 8):
+            plan = hl.decode_launch_plan(d, batch)
+            assert plan["slots_per_warp"] == slots, (name, ce, batch, plan)
+            assert 1 <= plan["decoder_warps"] <= 31
+            # the reported warps fit: their slots, the table(s) and the guard area lie inside a CTA's shared memory
+            assert plan["decoder_warps"] * slots * sp["slot_bytes"] + sp["table_bytes"] + sp["guard_bytes"] <= smem
+            if slots == 2:
+                assert plan["decoder_warps"] == 31
+            else:   # single slots serve more warps than pairs would
+                assert plan["decoder_warps"] > (smem - sp["table_bytes"] - sp["guard_bytes"]) // (2 * sp["slot_bytes"]) or plan["decoder_warps"] == 31
+        try:     # less shared memory: fewer warps, or no launch at all
+            assert hl.decode_launch_plan(d, 1, 100 * 1024)["decoder_warps"] <= hl.decode_launch_plan(d, 1)["decoder_warps"]
+        except hl.HuffllmError as e:
+            assert "too large for shared memory" in str(e)
+        with pytest.raises(hl.HuffllmError):
+            hl.decode_launch_plan(d, 9)
+
+
 def test_code_length_limits_accepted_per_format():
     """BF16 budgets 8..12 (the two nibble codes of a weight together); FP16 field limits 7..12."""
     wb = wl.gaussian_weights(16, 512, 0.02, 92)
