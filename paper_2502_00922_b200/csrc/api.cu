@@ -214,7 +214,10 @@ huffllm_status finish_args(KernelArgs *k, bool product, const DeviceInfo &dev, u
     uint64_t w2 = room / (2ull * k->slot_bytes), w1 = room / k->slot_bytes;
     if (w2 > max_w) w2 = max_w;
     if (w1 > max_w) w1 = max_w;
-    k->slots = w2 < max_w && 4 * w1 >= 5 * w2 ? 1u : 2u;
+    const bool single_ok = k->fmt || k->lut_bits == 8;                // (the kernels that exist with single slots)
+    k->slots = single_ok && w2 < max_w && 4 * w1 >= 5 * w2 ? 1u : 2u;
+    if (k->slots == 2 && fixed + 2ull * k->slot_bytes > k->dyn_smem_bytes)
+        return fail(HUFFLLM_ERR_UNSUPPORTED, "chunk records too large for shared memory (slot %u bytes)", k->slot_bytes);
     if (warps_at_least) *warps_at_least = (uint32_t)(k->slots == 1 ? w1 : w2);
     k->pair_recip = (uint32_t)(0x100000000ull / ((uint64_t)k->slots * k->slot_bytes));
     uint64_t g = k->total_chunks < (uint64_t)dev.sms ? k->total_chunks : (uint64_t)dev.sms;

@@ -460,7 +460,7 @@ struct SmemPlan {
     uint32_t slotB;  // first slot pair after it
 };
 
-__device__ __forceinline__ SmemPlan plan_smem(uint32_t base, const KernelArgs &k, uint32_t max_warps) {   // k: launch-wide fields only
+__device__ __forceinline__ SmemPlan plan_smem(uint32_t base, const KernelArgs &k, uint32_t max_warps, uint32_t slots = 2) {   // k: launch-wide fields only
     SmemPlan p;
     const uint32_t lut_bytes = k.lut_align;
     uint32_t a0 = (base + 127u) & ~127u;
@@ -468,7 +468,7 @@ __device__ __forceinline__ SmemPlan plan_smem(uint32_t base, const KernelArgs &k
     p.slotA = a0;
     // (divisions by the slot pair's size as a multiplication by its rounded-down reciprocal and one correction: this
     // runs in every warp of a launch's set-up, which is bound by instruction issue)
-    const uint32_t pair = k.slots * k.slot_bytes;
+    const uint32_t pair = slots == 2 ? 2 * k.slot_bytes : k.slot_bytes;
     auto div_pair = [&](uint32_t x) -> uint32_t {
         uint32_t q = __umulhi(x, k.pair_recip);
         return x - q * pair >= pair ? q + 1 : q;
@@ -483,9 +483,14 @@ __device__ __forceinline__ SmemPlan plan_smem(uint32_t base, const KernelArgs &k
     return p;
 }
 
-// First slot of a decoder warp; `pair_bytes` = slots per warp x slot bytes.
-__device__ __forceinline__ uint32_t slot_addr(const SmemPlan &p, uint32_t warp, uint32_t pair_bytes) {
-    return warp < p.nA ? p.slotA + warp * pair_bytes : p.slotB + (warp - p.nA) * pair_bytes;
+// Slot `which` of a decoder warp (two slots per warp).
+__device__ __forceinline__ uint32_t slot_addr(const SmemPlan &p, uint32_t warp, uint32_t which, uint32_t slot_bytes) {
+    uint32_t pair = warp < p.nA ? p.slotA + warp * 2 * slot_bytes : p.slotB + (warp - p.nA) * 2 * slot_bytes;
+    return pair + which * slot_bytes;
+}
+// The one slot of a decoder warp where warps have single slots.
+__device__ __forceinline__ uint32_t slot_addr_single(const SmemPlan &p, uint32_t warp, uint32_t slot_bytes) {
+    return warp < p.nA ? p.slotA + warp * slot_bytes : p.slotB + (warp - p.nA) * slot_bytes;
 }
 
 constexpr int kMaxWarps = 32;

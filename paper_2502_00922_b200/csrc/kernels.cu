@@ -55,7 +55,9 @@ namespace huffllm {
 // NT = 0 (BF16 blobs, batch 1): no tensor core at all.  The two mma.sync of a block cost the decoders more issue time
 // than the sixteen mixed-precision multiply-adds (bf16 x bf16 + f32, `fma.rn.f32.bf16`) that a lane needs for its 16
 // weights and one vector: those run on the FMA pipe, which the decoder leaves idle.
-template <int MODE, int LB, int THREADS, int FMT, int NT = 1>
+// SLOTS = shared-memory slots per decoder warp: 2 (a warp's next record lands while it decodes this one), or 1 for records
+// so large that pairs would leave too few warps a place (the feeder then waits for the slot before every copy).
+template <int MODE, int LB, int THREADS, int FMT, int NT = 1, int SLOTS = 2>
 __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant__ KernelArgs A) {
     constexpr int kV = NT == 2 ? 8 : 4;                       // values a lane holds of a row group's 16 x batch outputs
     constexpr uint32_t kRawBlock = FMT ? 64u : 512u;          // raw bytes of one block of a record
@@ -83,7 +85,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     pdl_launch_dependents();   // the next kernel's set-up may overlap this kernel's tail
     const uint32_t smem_base = smem_u32(dyn_smem);
     const uint32_t feeder = nwarps_launched - 1;
-    const SmemPlan plan = plan_smem(smem_base, A, feeder);
+    const SmemPlan plan = plan_smem(smem_base, A, feeder, SLOTS);
     const uint32_t nw = plan.warps;                            // decoder warps
     const uint32_t vals = 16 * A.batch;
     // the pieces of row groups that several warps of the CTA share: [2 * warps][16 * batch], in shared memory (NT = 1)
@@ -132,15 +134,17 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         // the barriers exist: the decoders may go on as soon as their table is built; the feeder does not wait for them
         asm volatile("bar.arrive %0, %1;" ::"r"(kSetupBarrier), "r"(THREADS) : "memory");
         uint32_t f_kc = f_ci % KC;
-        const uint32_t slot_units = A.slot_bytes >> 7, slot_w = slot_addr(plan, lane < nw ? lane : 0u, A.slots * A.slot_bytes);
+        const uint32_t slot_units = A.slot_bytes >> 7, slot_w = SLOTS == 2 ? slot_addr(plan, lane < nw ? lane : 0u, 0, A.slot_bytes)
+                                                                                : slot_addr_single(plan, lane < nw ? lane : 0u, A.slot_bytes);
         const uint32_t note_w = smem_u32(&notes[lane * 2]);
         uint32_t idle = 0;
         while (__any_sync(0xFFFFFFFFu, f_ci < f_ce)) {
             const uint32_t which = f_issued & 1u;
             // a slot is free for its first chunk, and later once the decoder has handed it back: with two slots that is the
             // chunk before the last one issued, with one slot the last one (barriers and notes alternate either way)
-            const uint32_t f_back = f_issued - A.slots;
-            const bool ready = f_ci < f_ce && (f_issued < A.slots || mbar_test_wait(bar_w + 16 + 8 * (f_back & 1u), (f_back >> 1) & 1u));
+            const bool ready = f_ci < f_ce &&
+                               (SLOTS == 2 ? f_issued < 2 || mbar_test_wait(bar_w + 16 + 8 * which, ((f_issued >> 1) - 1u) & 1u)
+                                           : f_issued < 1 || mbar_test_wait(bar_w + 16 + 8 * (which ^ 1u), ((f_issued - 1u) >> 1) & 1u));
             if (ready) {
                 const uint32_t full = bar_w + 8 * which, nkb = f_kc + 1 == KC ? nkb_tail : nkb_full;
                 // a record is usable if it lies inside the payload, is longer than its raw part and its coded part fits a slot
@@ -149,7 +153,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                 if (ok) {
                     const uint32_t bytes = (f_rb - f_ra - raw_units(nkb)) << 7;
                     mbar_expect_tx(full, bytes);
-                    bulk_g2s(slot_w + (which & (A.slots - 1u)) * A.slot_bytes, payload + ((uint64_t)(f_ra + raw_units(nkb)) << 7), bytes, full);
+                    bulk_g2s(slot_w + (SLOTS == 2 ? which * A.slot_bytes : 0u), payload + ((uint64_t)(f_ra + raw_units(nkb)) << 7), bytes, full);
                     // the raw part of the record is asked into L2 with one request (not for a warp's first two chunks: at the
                     // start of a launch every warp's copies are under way at once, and only the decoders' own loads matter)
                     if (f_issued >= 2)
@@ -364,8 +368,9 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
         const uint64_t x_tile2 = NT == 2 ? (uint64_t)(min(g + 8u, A.batch - 1) - min(g, A.batch - 1)) * k.cols : 0;
         // this chunk's slot (the lane's column of it), its barrier and its note, toggled by XOR from chunk to chunk; parity
         // of the barrier's next completion (each of the two "full" barriers completes every second chunk)
-        uint32_t slot_cur = slot_addr(plan, warp, A.slots * A.slot_bytes) + (lane << 2), bar_cur = bar_w, par = 0, which = 0;
-        const uint32_t slot_tog = A.slots == 2 ? slot_cur ^ (slot_cur + A.slot_bytes) : 0u;   // (one slot: every chunk lands in the same place)
+        uint32_t slot_cur = (SLOTS == 2 ? slot_addr(plan, warp, 0, A.slot_bytes) : slot_addr_single(plan, warp, A.slot_bytes)) + (lane << 2);
+        uint32_t bar_cur = bar_w, par = 0, which = 0;
+        const uint32_t slot_tog = SLOTS == 2 ? slot_cur ^ (slot_cur + A.slot_bytes) : 0u;   // (one slot: every chunk lands in the same place)
         uint32_t note_cur = smem_u32(&notes[warp * 2]);
 
 #pragma unroll 1
@@ -532,7 +537,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
             if (lane == 0) mbar_arrive(bar_cur + 16);                 // the slot goes back to the feeder
             par ^= which;                                         // 0, 0, 1, 1, 0, 0, ...
             which ^= 1u;
-            slot_cur ^= slot_tog;
+            if (SLOTS == 2) slot_cur ^= slot_tog;
             bar_cur ^= 8u;
             note_cur ^= 8u;
             kc = kc + 1 == KC ? 0u : kc + 1;
@@ -620,9 +625,9 @@ cudaError_t launch_stage_copy(void *dst, const void *src, uint64_t bytes, uint32
 
 // ------------------------------------------------------------------------------ launchers
 
-template <int MODE, int LB, int THREADS, int FMT, int NT = 1>
+template <int MODE, int LB, int THREADS, int FMT, int NT = 1, int SLOTS = 2>
 static cudaError_t launch_one(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
-    auto fn = huff_kernel<MODE, LB, THREADS, FMT, NT>;
+    auto fn = huff_kernel<MODE, LB, THREADS, FMT, NT, SLOTS>;
     static std::atomic<bool> attr_set[64];   // set twice by racing threads at worst: the call is idempotent
     int dev = 0;
     cudaGetDevice(&dev);
@@ -644,27 +649,34 @@ static cudaError_t launch_one(const KernelArgs &k, uint32_t grid, cudaStream_t s
     return cudaLaunchKernelEx(&cfg, fn, k);
 }
 
+// One or two slots per decoder warp (the host decides; kernels.h says for which kernels single slots exist).
+template <int MODE, int LB, int FMT, int NT = 1>
+static cudaError_t launch_slots(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
+    if (k.slots == 1) return launch_one<MODE, LB, kThreads, FMT, NT, 1>(k, grid, stream);
+    return launch_one<MODE, LB, kThreads, FMT, NT, 2>(k, grid, stream);
+}
+
 cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
-    if (k.fmt && k.lut_bits == 7) return launch_one<0, 7, kThreads, 1>(k, grid, stream);
-    if (k.fmt) return k.lut_bits > 8 ? launch_one<0, 12, kThreads, 1>(k, grid, stream) : launch_one<0, 8, kThreads, 1>(k, grid, stream);
+    if (k.fmt && k.lut_bits == 7) return launch_slots<0, 7, 1>(k, grid, stream);
+    if (k.fmt) return k.lut_bits > 8 ? launch_slots<0, 12, 1>(k, grid, stream) : launch_slots<0, 8, 1>(k, grid, stream);
     if (k.lut_bits > 9) return launch_one<0, 12, kThreads, 0>(k, grid, stream);
-    return k.lut_bits == 8 ? launch_one<0, 8, kThreads, 0>(k, grid, stream) : launch_one<0, 9, kThreads, 0>(k, grid, stream);
+    return k.lut_bits == 8 ? launch_slots<0, 8, 0>(k, grid, stream) : launch_one<0, 9, kThreads, 0>(k, grid, stream);
 }
 
 cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
     if (k.batch == 1 && k.fmt) {                  // one vector: multiply-adds on the FMA pipe
-        if (k.lut_bits == 7) return launch_one<1, 7, kThreads, 1, 0>(k, grid, stream);
-        return k.lut_bits > 8 ? launch_one<1, 12, kThreads, 1, 0>(k, grid, stream) : launch_one<1, 8, kThreads, 1, 0>(k, grid, stream);
+        if (k.lut_bits == 7) return launch_slots<1, 7, 1, 0>(k, grid, stream);
+        return k.lut_bits > 8 ? launch_slots<1, 12, 1, 0>(k, grid, stream) : launch_slots<1, 8, 1, 0>(k, grid, stream);
     }
     if (k.batch == 1) {
         if (k.lut_bits > 9) return launch_one<1, 12, kThreads, 0, 0>(k, grid, stream);
-        return k.lut_bits == 8 ? launch_one<1, 8, kThreads, 0, 0>(k, grid, stream) : launch_one<1, 9, kThreads, 0, 0>(k, grid, stream);
+        return k.lut_bits == 8 ? launch_slots<1, 8, 0, 0>(k, grid, stream) : launch_one<1, 9, kThreads, 0, 0>(k, grid, stream);
     }
-    if (k.batch > 8) return launch_one<1, 8, kThreads, 0, 2>(k, grid, stream);   // (the entry point sends only BF16 blobs of 8-bit tables here)
-    if (k.fmt && k.lut_bits == 7) return launch_one<1, 7, kThreads, 1>(k, grid, stream);
-    if (k.fmt) return k.lut_bits > 8 ? launch_one<1, 12, kThreads, 1>(k, grid, stream) : launch_one<1, 8, kThreads, 1>(k, grid, stream);
+    if (k.batch > 8) return launch_slots<1, 8, 0, 2>(k, grid, stream);   // (the entry point sends only BF16 blobs of 8-bit tables here)
+    if (k.fmt && k.lut_bits == 7) return launch_slots<1, 7, 1>(k, grid, stream);
+    if (k.fmt) return k.lut_bits > 8 ? launch_slots<1, 12, 1>(k, grid, stream) : launch_slots<1, 8, 1>(k, grid, stream);
     if (k.lut_bits > 9) return launch_one<1, 12, kThreads, 0>(k, grid, stream);
-    return k.lut_bits == 8 ? launch_one<1, 8, kThreads, 0>(k, grid, stream) : launch_one<1, 9, kThreads, 0>(k, grid, stream);
+    return k.lut_bits == 8 ? launch_slots<1, 8, 0>(k, grid, stream) : launch_one<1, 9, kThreads, 0>(k, grid, stream);
 }
 
 cudaError_t launch_plain_gemv(const PlainArgs &a, uint32_t sms, cudaStream_t stream) {

@@ -29,8 +29,6 @@ struct KernelArgs {
     uint32_t fmt;              // 0: BF16 blobs (one table), 1: FP16 blobs (three tables)
     uint32_t lut_align, lut_size;   // shared-memory window of the table(s): a power-of-two alignment above the index bits, and its bytes
     uint32_t slot_bytes;       // shared-memory bytes of one slot: largest max_words * 256
-    uint32_t slots;            // slots per decoder warp: 2 (the next record lands while this one is decoded), or 1 where two would
-                               // leave too few warps a slot (large records: the feeder then waits for a slot before every copy)
     uint32_t pair_recip;       // floor(2^32 / (slots * slot_bytes)): umulhi(x, pair_recip) is x / (slots * slot_bytes) or one less
     uint32_t guard_bytes;      // readable bytes kept free behind the last slot
     uint32_t part_bytes;       // bytes at the end of dynamic shared memory for the CTA's partial sums (tensor-core path: the stages of activations)
@@ -45,6 +43,10 @@ struct KernelArgs {
     float *tc_partial;         // [m_tiles * ksplit][32 warps][npad / 2][32]
     unsigned int *tc_ticket;   // [m_tiles][32], zero between calls
     MatArgs m[kMaxMats];
+    // (behind the matrices, so that the fields the hot loops read keep their places)
+    uint32_t slots;            // slots per decoder warp: 2 (the next record lands while this one is decoded), or 1 where two would
+                               // leave too few warps a slot (large records: the feeder then waits for a slot before every copy).
+                               // Kernels with single slots exist for FP16 blobs and for BF16 blobs with 8-bit tables.
 };
 
 cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t stream);

@@ -143,7 +143,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     uint32_t lut_lane = plan.lut | ((FMT ? lane & 15u : lane) << 2);
     asm volatile("mov.u32 %0, %0;" : "+r"(lut_lane));
     const uint32_t bar0 = smem_u32(&bars[warp * 2]);
-    const uint32_t slot0 = slot_addr(plan, warp, 2 * A.slot_bytes);   // (this kernel always runs with two slots per warp)
+    const uint32_t slot0 = slot_addr(plan, warp, 0, A.slot_bytes);    // (this kernel always runs with two slots per warp)
 
     // ---- set-up: table, barriers, tensor memory
     {
