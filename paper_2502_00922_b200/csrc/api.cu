@@ -81,14 +81,14 @@ struct TcPlan {
 };
 // Shared memory the tensor-core kernel needs with `tiles` 128-row tiles per CTA.
 // Stages of the tensor-core kernel: four, two at the widest batch padding, where shared memory is short.
-uint32_t tc_stages(uint32_t npad) { return npad == 64 ? 3u : 4u; }
+uint32_t tc_stages(uint32_t npad) { return npad == 64 ? 2u : 3u; }
 uint64_t tc_smem_need(const huffllm_desc *d, uint32_t npad, uint32_t tiles) {
     const bool fp16 = d->dtype == HUFFLLM_FP16;
     const uint32_t checks_per_block = fp16 ? 8 : (d->lut_bits == 8 ? 3 : 4);
     uint64_t guard = 256ull * (3 + checks_per_block * (d->chunk_cols / kBlockCols));
     const uint64_t lut = fp16 ? 49152ull : 128ull << d->lut_bits;
-    const uint64_t b_stages = (uint64_t)tc_stages(npad) * npad * 64;          // the guard area may lie over them
-    return lut + (guard > b_stages ? guard - b_stages : 0) + b_stages + 4096 + 2ull * 8 * tiles * d->max_words * 256;
+    const uint64_t b_stages = (uint64_t)tc_stages(npad) * npad * 128;          // the guard area may lie over them
+    return lut + (guard > b_stages ? guard - b_stages : 0) + b_stages + 4096 + 2ull * (8 * tiles < 31 ? 8 * tiles : 31) * d->max_words * 256;
 }
 TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn_smem) {
     TcPlan p;
@@ -414,7 +414,7 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
         uint32_t grid;
         begin_args(&k, batch, dev);
         if ((st = add_matrix(&k, desc, blob)) != HUFFLLM_OK) return st;
-        k.part_bytes = tc_stages(tp.npad) * tp.npad * 64;      // the stages of activations
+        k.part_bytes = tc_stages(tp.npad) * tp.npad * 128;      // the stages of activations
         k.slots = 2;
         k.pair_recip = (uint32_t)(0x100000000ull / (2ull * k.slot_bytes));
         const uint64_t need = tc_smem_need(desc, tp.npad, tp.tiles);

@@ -29,7 +29,7 @@
 
 namespace huffllm {
 
-constexpr int kTcStages = 4;
+constexpr int kTcStages = 3;
 constexpr int kTcTiles = 4;
 
 __device__ __forceinline__ void tmem_alloc(uint32_t smem_dst, uint32_t ncols) {
@@ -115,9 +115,9 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     constexpr bool SKIP = LB == 8 && FMT == 0;
     constexpr int R = SKIP ? 4 : LB == 8 ? 3 : 2;
     constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
-    constexpr int S = NPAD == 64 ? 3 : kTcStages;          // the host's tc_stages(): shared memory is short at the widest padding
-    constexpr uint32_t kBStage = NPAD * 64;                 // bytes of B per stage: NPAD rows x 32 columns of bf16
-    constexpr uint32_t kLbo = 128, kSbo = 512;              // core matrices: 4 along K side by side, then the next 8 rows
+    constexpr int S = NPAD == 64 ? 2 : kTcStages;          // the host's tc_stages(): shared memory is short at the widest padding
+    constexpr uint32_t kBStage = NPAD * 128;                // bytes of B per stage: NPAD rows x 64 columns (two blocks) of bf16
+    constexpr uint32_t kLbo = 128, kSbo = 1024;             // core matrices: 8 along K side by side, then the next 8 rows
     constexpr uint32_t kACol0 = kTcTiles * NPAD;            // first tensor-memory column of the A stages
     // instruction descriptor: fp32 accumulate, bf16 x bf16, both K-major, N = NPAD, M = 128
     constexpr uint32_t kIdesc = (1u << 4) | (FMT ? 0u : (1u << 7) | (1u << 10)) | ((uint32_t)(NPAD >> 3) << 17) | ((128u >> 4) << 24);
@@ -238,24 +238,27 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
         }
     };
     // addresses that change only with the stage: this warp's rows of the A operand, its piece of the B slice
-    const uint32_t a_dst0 = tmem + a_lane + kACol0 + tile * S * 16;
+    const uint32_t a_dst0 = tmem + a_lane + kACol0 + tile * S * 32;
     const uint32_t x_dst0 = b_base + (x_n >> 3) * kSbo + x_kap * kLbo + (x_n & 7) * 16;
 
     // One block of the stage protocol, decoder side.  `a` = this warp's decoded 16 rows x 32 columns (null if the warp has
     // no rows).  The warp stores its share, says so on the stage's "full" barrier and goes on decoding: nobody waits for
     // the other warps here.  A warp can run ahead of the slowest one by the depth of the stage ring and no further (it
     // needs the stage back, which the issuer's tcgen05.commit announces on the "empty" barrier).
-    auto stage_block = [&](const uint32_t *a, const uint4 &xv) {
+    auto stage_block = [&](const uint32_t *a, const uint4 &xv, uint32_t half, bool publish) {
         const uint32_t s = gb % S, use = gb / S;
-        if (use > 0) bounded_wait(smem_u32(&empty_bar[s]), (use - 1) & 1u);
-        tc_fence_after();
+        if (half == 0) {
+            if (use > 0) bounded_wait(smem_u32(&empty_bar[s]), (use - 1) & 1u);
+            tc_fence_after();
+        }
         if (a) {
             // lane (g, t): row g's weights 0..3 -> 32-bit columns 2t, 2t+1; weights 4..7 -> columns 8 + 2t, 8 + 2t + 1
             const uint32_t r[8] = {a[0], a[1], a[4], a[5], a[2], a[3], a[6], a[7]};
-            tc_st_16x256b_x2(a_dst0 + s * 16, r);
+            tc_st_16x256b_x2(a_dst0 + s * 32 + half * 16, r);
         }
         if (x_carrier)
-            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(x_dst0 + s * kBStage), "r"(xv.x), "r"(xv.y), "r"(xv.z), "r"(xv.w) : "memory");
+            asm volatile("st.shared.v4.u32 [%0], {%1, %2, %3, %4};" ::"r"(x_dst0 + s * kBStage + half * 4 * kLbo), "r"(xv.x), "r"(xv.y), "r"(xv.z), "r"(xv.w) : "memory");
+        if (!publish) return;
         tc_wait_st();
         if (x_carrier_warp) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the B slice must be visible to the tensor core's reads
         tc_fence_before();
@@ -266,7 +269,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     // The same block, issuer side: when every decoder warp has arrived, one lane issues the block's MMAs for every tile
     // and commits them onto the stage's "empty" barrier.  (After a wait that ran out the commit still goes out: the
     // stage ring keeps moving and the kernel ends with its error flag set.)
-    auto issue_block = [&](bool first_of_item) {
+    auto issue_block = [&](bool first_of_item, uint32_t halves) {
         const uint32_t s = gb % S, use = gb / S;
         bounded_wait(smem_u32(&full_bar[s]), use & 1u);
         if (lane == 0) {
@@ -275,9 +278,10 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
             if (!failed) {
                 for (uint32_t tl = 0; tl < n_tiles; ++tl) {
 #pragma unroll
-                    for (uint32_t j = 0; j < 2; ++j)      // two K = 16 steps per stage
-                        tc_mma_f16_tmem_a(tmem + tl * NPAD, tmem + kACol0 + (tl * S + s) * 16 + j * 8,
-                                          smem_desc_kmajor(bst + j * 2 * kLbo, kLbo, kSbo), kIdesc, (first_of_item && j == 0) ? 0u : 1u);
+                    for (uint32_t j = 0; j < 4; ++j)      // four K = 16 steps per full stage, two for the odd last block of a chunk
+                        if (j < 2 * halves)
+                            tc_mma_f16_tmem_a(tmem + tl * NPAD, tmem + kACol0 + (tl * S + s) * 32 + j * 8,
+                                              smem_desc_kmajor(bst + j * 2 * kLbo, kLbo, kSbo), kIdesc, (first_of_item && j == 0) ? 0u : 1u);
                 }
             }
             tc_commit(smem_u32(&empty_bar[s]));
@@ -310,7 +314,10 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
         load_x(x_a, x_src + col_lo);
 
         if (warp == issuer) {
-            for (uint32_t col_blk = col_lo; col_blk < col_hi; col_blk += 32) issue_block(gb == gb_item);
+            for (uint32_t kc = kc0; kc < kc1; ++kc) {       // stages are cut like the decoders': pairs of blocks inside a chunk
+                const uint32_t nkb = blocks_of(kc);
+                for (uint32_t kb = 0; kb < nkb; kb += 2) issue_block(gb == gb_item, min(nkb - kb, 2u));
+            }
         } else if (active) {
             const uint32_t c_beg = rg * KC + kc0, c_end = rg * KC + kc1;
             if (lane == 0 && !primed) {
@@ -337,7 +344,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                     for (uint32_t kb = 0; kb < nkb; ++kb) {
                         if (x_p < x_end) load_x(x_b, x_p);
                         x_p += 32;
-                        stage_block(zero, x_a);
+                        stage_block(zero, x_a, kb & 1u, (kb & 1u) || kb + 1 == nkb);
                         x_a = x_b;
                     }
                     __syncwarp();
@@ -351,7 +358,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                 stream_open(sb, slot0 + which * A.slot_bytes + 128u + (lane << 2), SKIP ? 7u : 0u);
                 // one block: fetch the next block's raw bytes and activations into the other register set, decode
                 // this one, hand it to the tensor core
-                auto block = [&](const uint4 &raw_c, uint4 &raw_n, const uint4 &x_c, uint4 &x_n2, bool more) {
+                auto block = [&](const uint4 &raw_c, uint4 &raw_n, const uint4 &x_c, uint4 &x_n2, bool more, uint32_t half, bool publish) {
                     raw_p += kRawBlock;
                     if (more) raw_n = load_raw(raw_p);
                     if (x_p < x_end) load_x(x_n2, x_p);
@@ -359,17 +366,17 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                     uint32_t a[8];
                     if (FMT) decode_block_fp16(sa, sb, lut_lane, raw_c.x, a);
                     else decode_block<R, SKIP>(sa, sb, kIdxMask, lut_lane, raw_c, a);
-                    stage_block(a, x_c);
+                    stage_block(a, x_c, half, publish);
                 };
                 uint4 raw_b = make_uint4(0, 0, 0, 0);
                 uint32_t kb = 0;
 #pragma unroll 1
                 for (; kb + 2 <= nkb; kb += 2) {                  // the usual case: pairs of blocks, two register sets in turn
-                    block(raw_cur, raw_b, x_a, x_b, true);
-                    block(raw_b, raw_cur, x_b, x_a, kb + 2 < nkb);
+                    block(raw_cur, raw_b, x_a, x_b, true, 0, false);
+                    block(raw_b, raw_cur, x_b, x_a, kb + 2 < nkb, 1, true);
                 }
-                if (kb < nkb) {                                   // odd block count (a ragged last chunk)
-                    block(raw_cur, raw_b, x_a, x_b, false);
+                if (kb < nkb) {                                   // odd block count (a ragged last chunk): a stage of one block
+                    block(raw_cur, raw_b, x_a, x_b, false, 0, true);
                     x_a = x_b;
                 }
                 __syncwarp();
@@ -379,11 +386,14 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
             }
         } else {
             // no rows of the matrix for this warp: it still carries its slice of the activations and its arrivals
-            for (uint32_t col_blk = col_lo; col_blk < col_hi; col_blk += 32) {
-                if (x_p < x_end) load_x(x_b, x_p);
-                x_p += 32;
-                stage_block(nullptr, x_a);
-                x_a = x_b;
+            for (uint32_t kc = kc0; kc < kc1; ++kc) {
+                const uint32_t nkb = blocks_of(kc);
+                for (uint32_t kb = 0; kb < nkb; ++kb) {
+                    if (x_p < x_end) load_x(x_b, x_p);
+                    x_p += 32;
+                    stage_block(nullptr, x_a, kb & 1u, (kb & 1u) || kb + 1 == nkb);
+                    x_a = x_b;
+                }
             }
         }
 
