@@ -129,6 +129,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     __shared__ uint32_t s_tmem_base;
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    pdl_launch_dependents();   // the next kernel in the stream may be scheduled early; it waits for this one before it reads results
     const MatArgs &k = A.m[0];
     const uint32_t smem_base = smem_u32(dyn_smem);
     // decoder warps: eight per tile, except that the CTA's last warp never decodes: it issues the MMAs (with four tiles the
@@ -178,6 +179,10 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
         __syncthreads();
         return;
     }
+
+    // the table is built and tensor memory allocated: from here on activations are read and results written, which the
+    // kernel in front of this one in the stream may still be producing
+    pdl_wait_prior_grid();
 
     // ---- roles
     const uint32_t tile = warp >> 3, q = warp & 3, h = (warp >> 2) & 1;
@@ -475,8 +480,17 @@ static cudaError_t launch_tc_one(const KernelArgs &k, uint32_t grid, cudaStream_
         if (e != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev].store(true, std::memory_order_release);
     }
-    fn<<<grid, 1024, k.dyn_smem_bytes, stream>>>(k);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(1024);
+    cfg.dynamicSmemBytes = k.dyn_smem_bytes;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // set-up overlaps the previous kernel's tail
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, fn, k);
 }
 
 cudaError_t launch_gemm_tc(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
