@@ -12,13 +12,14 @@
 // of a tile owns tensor-memory lanes 32 q + 16 h .. + 15, which is what the 16x256b store shape of a warp can reach.
 // The CTA's LAST warp does not decode: it issues the MMAs (so a CTA decodes 31 row groups at a time, and the last 16 rows
 // of the fourth tile are never read).  Tensor memory (512 columns): 4 accumulators of N columns, then 4 tiles x S stages
-// x 16 columns of A (a stage = one block of 32 weight columns = two K = 16 steps).
+// x 32 columns of A (a stage = two blocks of 32 weight columns = four K = 16 steps; a chunk's odd last block makes a
+// stage of one block).
 // A work item is (31 row groups) x (a range of column chunks); partial results of the ranges of one row tile are
 // added in a fixed order by whoever finishes last (per-warp arrival counters, nobody waits).
 //
-// Stage protocol: a decoder warp fills its share of stage s (A rows, a slice of B), arrives on the stage's "full"
-// mbarrier and goes on decoding; no warp waits for another one except through the depth of the stage ring.  The issuer
-// warp waits for a stage to be full, issues its 8 MMAs and a tcgen05.commit onto the stage's "empty" mbarrier, which the
+// Stage protocol: a decoder warp fills its share of stage s (A rows, a slice of B; each block into its half of the stage
+// as soon as it is decoded), arrives on the stage's "full" mbarrier and goes on decoding; no warp waits for another one except through the depth of the stage ring.  The issuer
+// warp waits for a stage to be full, issues its 16 MMAs and a tcgen05.commit onto the stage's "empty" mbarrier, which the
 // decoders wait on (with a limit) before they reuse the stage.  (With the issue taking turns among the decoder warps and a
 // barrier after every block, each block cost the CTA its decode time plus the 2000 cycles one warp needs to issue the
 // MMAs: that warp had to decode its next block before the next barrier could open.)
