@@ -276,7 +276,10 @@ huffllm_status huffllm_decode_gemv(const huffllm_desc *desc, const void *blob_de
 
 /*
  * Small-batch version: x is [batch][cols] row-major (device), y is [batch][rows] floats (device).
- * batch 1..64.
+ * batch 1..64.  Which kernel runs is the library's choice and does not change the result's meaning (sums are fp32, their
+ * order is fixed for a given call): one vector, 2..8 vectors and 9..16 vectors of BF16 blobs with 8-bit tables multiply from
+ * the decoded registers; 17..64 vectors (and 9..16 where that is faster for the matrix's shape, or the only way) go through
+ * the tensor core; blobs neither takes at that batch are done in passes of 8 vectors.
  */
 huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob_dev, const uint16_t *x_dev, uint32_t batch,
                                    float *y_dev, void *workspace_dev, size_t workspace_bytes, int32_t *err_flag_dev,

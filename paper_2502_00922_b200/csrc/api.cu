@@ -386,55 +386,75 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
     if (st != HUFFLLM_OK) return st;
     if (batch == 0 || batch > 64) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be in [1, 64]");
     if ((st = check_product_args(desc, x, y, workspace, workspace_bytes, batch)) != HUFFLLM_OK) return st;
-    if (batch > kKernelBatch && batch <= kTwoTileBatch && two_tile_blob(desc)) {
+    // Paths for more than 8 vectors.  Each returns HUFFLLM_OK with `done` set if it launched, HUFFLLM_OK without if it does
+    // not apply here (the next path decides), or an error.
+    bool done = false;
+    auto two_tiles = [&]() -> huffllm_status {
         // 9..16 vectors on the default BF16 blobs: the register path with two tiles of activations per decoded block
+        if (batch > kTwoTileBatch || !two_tile_blob(desc)) return HUFFLLM_OK;
         KernelArgs k;
         uint32_t grid;
         begin_args(&k, batch, dev);
-        if ((st = add_matrix(&k, desc, blob)) != HUFFLLM_OK) return st;
-        st = finish_args(&k, true, dev, &grid);
-        if (st == HUFFLLM_OK) {
-            k.m[0].x = x;
-            k.m[0].y = y;
-            k.m[0].ws_ticket = (unsigned int *)workspace;
-            k.m[0].ws_partial = (float *)((uint8_t *)workspace + ws_partial_offset(desc));
-            k.m[0].ws_warp_pieces = (float *)((uint8_t *)workspace + ws_partial_offset(desc) + ws_cta_pieces_bytes(batch));
-            k.err = err_flag;
-            cudaError_t e = launch_gemm(k, grid, (cudaStream_t)stream);
-            if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "product launch: %s", cudaGetErrorString(e));
+        huffllm_status s2 = add_matrix(&k, desc, blob);
+        if (s2 != HUFFLLM_OK) return s2;
+        if (finish_args(&k, true, dev, &grid) != HUFFLLM_OK) {
+            clear_error();      // records too large for shared memory: another path decides
             return HUFFLLM_OK;
         }
-        clear_error();      // records too large for shared memory: the paths below decide
-    }
-    if (batch > kKernelBatch && (desc->dtype == HUFFLLM_FP16 ? desc->lut_bits == 8u : desc->lut_bits <= 9u)) {
-        // tensor-core path: one pass over the compressed weights for the whole batch (tables of up to 9 bits; longer
-        // codes take passes of 8 vectors through the register-path kernel and its two-level lookup)
+        k.m[0].x = x;
+        k.m[0].y = y;
+        k.m[0].ws_ticket = (unsigned int *)workspace;
+        k.m[0].ws_partial = (float *)((uint8_t *)workspace + ws_partial_offset(desc));
+        k.m[0].ws_warp_pieces = (float *)((uint8_t *)workspace + ws_partial_offset(desc) + ws_cta_pieces_bytes(batch));
+        k.err = err_flag;
+        cudaError_t e = launch_gemm(k, grid, (cudaStream_t)stream);
+        if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "product launch: %s", cudaGetErrorString(e));
+        done = true;
+        return HUFFLLM_OK;
+    };
+    auto tensor_core = [&](bool other_path_left) -> huffllm_status {
+        // one pass over the compressed weights for the whole batch (tables of up to 9 bits; longer codes take passes of 8
+        // vectors through the register-path kernel and its two-level lookup)
+        if (!(desc->dtype == HUFFLLM_FP16 ? desc->lut_bits == 8u : desc->lut_bits <= 9u)) return HUFFLLM_OK;
         const TcPlan tp = tc_plan(desc, batch, (uint32_t)dev.sms, (uint32_t)dev.smem_optin - kStaticSmem);
         KernelArgs k;
-        uint32_t grid;
         begin_args(&k, batch, dev);
-        if ((st = add_matrix(&k, desc, blob)) != HUFFLLM_OK) return st;
+        huffllm_status s2 = add_matrix(&k, desc, blob);
+        if (s2 != HUFFLLM_OK) return s2;
         k.part_bytes = tc_stages(tp.npad) * tp.npad * 128;      // the stages of activations
         k.slots = 2;
         k.pair_recip = (uint32_t)(0x100000000ull / (2ull * k.slot_bytes));
-        const uint64_t need = tc_smem_need(desc, tp.npad, tp.tiles);
-        if (need <= k.dyn_smem_bytes && workspace_bytes >= tp.bytes) {
-            k.m[0].x = x;
-            k.m[0].y = y;
-            k.tc_npad = tp.npad;
-            k.tc_tiles = tp.tiles;
-            k.tc_m_tiles = tp.m_tiles;
-            k.tc_ksplit = tp.ksplit;
-            k.tc_ticket = (unsigned int *)((uint8_t *)workspace + tp.ticket_off);
-            k.tc_partial = (float *)((uint8_t *)workspace + tp.partial_off);
-            k.err = err_flag;
-            grid = tp.items < (uint32_t)dev.sms ? tp.items : (uint32_t)dev.sms;
-            cudaError_t e = launch_gemm_tc(k, grid, (cudaStream_t)stream);
-            if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "tensor-core product launch: %s", cudaGetErrorString(e));
-            return HUFFLLM_OK;
+        if (tc_smem_need(desc, tp.npad, tp.tiles) > k.dyn_smem_bytes) return HUFFLLM_OK;   // records too large for this kernel's slots
+        if (workspace_bytes < tp.bytes) {
+            if (other_path_left) return HUFFLLM_OK;     // (the register path needs less)
+            return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "workspace too small for batch %u", batch);
         }
-        if (workspace_bytes < tp.bytes) return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "workspace too small for batch %u", batch);
-        // chunk records too large for 32 warps' slots: fall through to passes of 8 vectors
+        k.m[0].x = x;
+        k.m[0].y = y;
+        k.tc_npad = tp.npad;
+        k.tc_tiles = tp.tiles;
+        k.tc_m_tiles = tp.m_tiles;
+        k.tc_ksplit = tp.ksplit;
+        k.tc_ticket = (unsigned int *)((uint8_t *)workspace + tp.ticket_off);
+        k.tc_partial = (float *)((uint8_t *)workspace + tp.partial_off);
+        k.err = err_flag;
+        const uint32_t grid = tp.items < (uint32_t)dev.sms ? tp.items : (uint32_t)dev.sms;
+        cudaError_t e = launch_gemm_tc(k, grid, (cudaStream_t)stream);
+        if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "tensor-core product launch: %s", cudaGetErrorString(e));
+        done = true;
+        return HUFFLLM_OK;
+    };
+    if (batch > kKernelBatch) {
+        // 9..16 vectors: the tensor-core kernel, whose time does not grow with the batch below its padding of 16, is the
+        // faster one for matrices that are at least as wide as tall (few row groups per SM make the register path's
+        // cross-CTA sums of 16-vector pieces expensive), unless they have so few rows that it gets few row tiles; measured
+        // at 12 and 16 vectors on seven shapes from 1024 x 8192 to 28672 x 8192.  Above 16 vectors it is the only one.
+        const bool wide = desc->cols >= desc->rows && desc->rows >= 2048;
+        if (!wide && (st = two_tiles()) != HUFFLLM_OK) return st;
+        if (!done && (st = tensor_core(wide && batch <= kTwoTileBatch && two_tile_blob(desc))) != HUFFLLM_OK) return st;
+        if (!done && wide && (st = two_tiles()) != HUFFLLM_OK) return st;
+        if (done) return HUFFLLM_OK;
+        // neither applies (long codes, or chunk records too large for the slots): passes of 8 vectors
     }
     for (uint32_t b0 = 0; b0 < batch; b0 += kKernelBatch) {
         uint32_t nb = batch - b0 < kKernelBatch ? batch - b0 : kKernelBatch;
