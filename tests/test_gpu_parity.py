@@ -248,7 +248,10 @@ GEMM_CASES = [
     (272, 2080, 16384, 0, "gauss", 4),
     (512, 4096, 4096, 9, "student", 5),
     (256, 2048, 4096, 0, "uniform", 8),
-    (128, 1024, 1024, 0, "gauss", 16),            # batch 9..64 runs on the tcgen05 path
+    (128, 1024, 1024, 0, "gauss", 16),            # 9..16 vectors, few rows: the register path with two tiles of activations
+    (2048, 2048, 4096, 0, "gauss", 13),           # 9..16 vectors, as wide as tall: the tcgen05 path at its smallest padding
+    (2064, 4096, 4096, 0, "student", 16),         # ... ragged rows (129 row groups: five row tiles, the last nearly empty)
+    (4096, 1024, 4096, 0, "gauss", 12),           # 9..16 vectors, tall: two tiles
     (64, 1024, 4096, 0, "gauss", 23),
     (40, 2080, 1024, 0, "student", 9),            # ragged rows, padded batch
     (1040, 4096, 4096, 0, "gauss", 64),           # three row tiles, column chunks cut into ranges
