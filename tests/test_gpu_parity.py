@@ -590,6 +590,24 @@ def test_distribution_stress_full_size(hl, torch, gen, ce):
     assert np.all(np.abs(y[0, rs] - yo[0]) <= TOL * d[0])
 
 
+@pytest.mark.parametrize("dtype,ce", [("fp16", 4096), ("bf16", 8192)])
+def test_single_slots_reused_full_size(hl, torch, dtype, ce):
+    """Records that get one shared-memory slot per decoder warp, on a matrix large enough that every warp goes through
+    its slot several times (4096 x 8192: 8192 or 4096 chunks for at most 148 x 31 warps at FP16, 8192 x 8192 at BF16):
+    decode against the original tensor, products on sampled rows against the oracle."""
+    rows, cols = (4096, 8192) if dtype == "fp16" else (8192, 8192)
+    w = wl.gaussian_weights(rows, cols, 0.02, 3100 + ce, dtype)
+    up = Uploaded(hl, torch, w, ce, 0, 3, dtype=hl.FP16 if dtype == "fp16" else hl.BF16)
+    assert hl.decode_launch_plan(up.desc, 1)["slots_per_warp"] == 1
+    assert np.array_equal(gpu_decode(hl, torch, up), w)
+    rs = np.random.default_rng(2).choice(rows, 32, replace=False)
+    for batch in (1, 3):
+        x = wl.activations(batch, cols, 3600 + batch, dtype)
+        y = gpu_gemm(hl, torch, up, x)
+        yo, d = orc.matmul(w[rs], x, orc.FP16 if dtype == "fp16" else orc.BF16)
+        assert np.all(np.abs(y[:, rs] - yo) <= TOL * d)
+
+
 @pytest.mark.parametrize("rows,cols", [(28672, 8192), (8192, 28672)])
 def test_ffn70b_shapes_small_batch_sampled(hl, torch, rows, cols):
     """70B-FFN shapes at full size, batch 1 / 4 (register path) and 16 / 64 (tensor-core path), sampled rows."""
