@@ -446,10 +446,12 @@ def main():
     if not 1 <= B <= 64:
         raise SystemExit("--batch must be in [1, 64]")
     fp16 = args.dtype != "bf16"
-    # launches over several matrices take up to 8 vectors, or up to 16 for BF16 blobs with 8-bit tables (two tiles of activations)
-    multi = B <= 8 or (B <= 16 and not fp16 and args.max_code_len in (0, 8))
+    # launches over several matrices take up to 8 vectors, up to 16 for BF16 blobs with 8-bit tables (two tiles of activations),
+    # and 17 to 64 on the tensor-core kernel for tables of up to 9 bits (FP16: 8)
+    multi = (B <= 8 or (B <= 16 and not fp16 and args.max_code_len in (0, 8))
+             or (B > 16 and args.max_code_len in ((0, 8) if fp16 else (0, 8, 9))))
     if not multi:
-        args.fuse = "none"           # the tensor-core path takes one matrix per launch
+        args.fuse = "none"           # one matrix per launch (passes of 8 vectors, or the tensor-core kernel at 9..16)
     mats = prepare(args.workload, args.chunk_elems, hl, torch, dev, cpu_mats, split, B, args.dtype, args.max_code_len)
     err = torch.zeros(1, dtype=torch.int32, device=dev)
     L = args.layers
@@ -779,7 +781,7 @@ def main():
                      "traffic_per_step": None if NCU_TRAFFIC_RATIO is None else NCU_TRAFFIC_RATIO * alg_bytes,
                      "traffic_note": "DRAM bytes read + written per launch (average over the step's launches): algorithmic bytes x the "
                                      "ratio of the ncu capture in profiles/ (1.025)",
-                     "peak_source": peak_src, "kernel": "huff_kernel<product>" if B <= 8 else ("huff_kernel<product, two tiles>" if multi else "huff_gemm_tc_kernel"), "launches_per_step": len(groups), "fuse": args.fuse,
+                     "peak_source": peak_src, "kernel": "huff_kernel<product>" if B <= 8 else ("huff_kernel<product, two tiles>" if multi and B <= 16 else "huff_gemm_tc_kernel"), "launches_per_step": len(groups), "fuse": args.fuse,
                      "algorithmic_bytes_per_step": alg_bytes, "kernel_ms_per_step": kernel_ms_step,
                      "frac_of_nominal_8TBs": achieved / 8000.0,
                      "one_launch": None if not one_launch_ms else {

@@ -286,8 +286,8 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob_de
                                    huffllm_stream stream);
 
 /*
- * Several products in ONE launch: y_i = W_i x_i for i < n (n <= 8; batch <= 8, or <= 16 for BF16 blobs of
- * max_code_len 8), e.g. the q, k and v
+ * Several products in ONE launch: y_i = W_i x_i for i < n (n <= 8; batch <= 8 for every blob, 9..16 for BF16 blobs of
+ * max_code_len 8, 17..64 for BF16 blobs of max_code_len 8 or 9 and FP16 blobs of max_code_len 8: UNSUPPORTED otherwise), e.g. the q, k and v
  * projections of a decoder layer, or gate and up.  The chunks of all matrices are spread over the GPU
  * together, so small matrices do not pay a launch, a set-up and a tail each.  Arrays are host arrays
  * of n pointers; every matrix needs its own workspace (each at least workspace_bytes_each long, which must

@@ -62,6 +62,8 @@ size_t ws_partial_offset(const huffllm_desc *d) {
 // 9..16), [kMaxGrid][2 * 32][16 * b] pieces that the warps of one CTA exchange (shared memory has no room for them).
 constexpr uint32_t kTwoTileBatch = 16;    // most activation vectors of the register path with two tiles
 bool two_tile_blob(const huffllm_desc *d) { return d->dtype == HUFFLLM_BF16 && d->lut_bits == 8; }
+// blobs the tensor-core kernel takes: tables of up to 9 bits (FP16: field codes of up to 8 bits)
+bool tc_blob(const huffllm_desc *d) { return d->dtype == HUFFLLM_FP16 ? d->lut_bits == 8u : d->lut_bits <= 9u; }
 size_t ws_cta_pieces_bytes(uint32_t b) { return (size_t)kMaxGrid * 2 * 16 * b * sizeof(float); }
 // (a workspace sized for `batch` vectors serves every smaller batch too)
 size_t ws_bytes_for(const huffllm_desc *d, uint32_t batch) {
@@ -90,10 +92,12 @@ uint64_t tc_smem_need(const huffllm_desc *d, uint32_t npad, uint32_t tiles) {
     const uint64_t b_stages = (uint64_t)tc_stages(npad) * npad * 128;          // the guard area may lie over them
     return lut + (guard > b_stages ? guard - b_stages : 0) + b_stages + 4096 + 2ull * (8 * tiles < 31 ? 8 * tiles : 31) * d->max_words * 256;
 }
-TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn_smem) {
+// `sms`: the CTAs this matrix can have (all SMs, or its share of a launch over several matrices); `tiles_cap`: the tiles
+// the launch's other matrices leave room for.
+TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn_smem, uint32_t tiles_cap = 4) {
     TcPlan p;
     p.npad = batch <= 16 ? 16 : (batch <= 32 ? 32 : 64);
-    p.tiles = 4;                                    // as many 8-warp tiles as the chunk slots leave room for
+    p.tiles = tiles_cap;                            // as many 8-warp tiles as the chunk slots leave room for
     while (p.tiles > 1 && tc_smem_need(d, p.npad, p.tiles) > dyn_smem) --p.tiles;
     const uint32_t n_dec = 8 * p.tiles < 31 ? 8 * p.tiles : 31;      // the CTA's last warp issues the MMAs and never decodes
     p.m_tiles = (d->row_groups + n_dec - 1) / n_dec;
@@ -352,8 +356,55 @@ huffllm_status huffllm_decode_gemm_multi(uint32_t n, const huffllm_desc *const *
     if (st != HUFFLLM_OK) return st;
     if (!descs || !blobs || !xs || !ys || !workspaces) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
     if (n == 0 || n > kMaxMats) return fail(HUFFLLM_ERR_INVALID_ARG, "between 1 and %u matrices per call", kMaxMats);
-    if (batch == 0 || batch > kTwoTileBatch)
-        return fail(HUFFLLM_ERR_UNSUPPORTED, "batch must be in [1, %u] here (above %u: BF16 blobs of max_code_len 8 only)", kTwoTileBatch, kKernelBatch);
+    if (batch == 0 || batch > 64) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be in [1, 64]");
+    if (batch > kTwoTileBatch) {
+        // 17..64 vectors: the tensor-core kernel, its CTAs dealt to the matrices like the other kernels'
+        TcArgs t;
+        memset(&t, 0, sizeof(t));
+        KernelArgs &k = t.k;
+        uint32_t grid;
+        begin_args(&k, batch, dev);
+        for (uint32_t i = 0; i < n; ++i) {
+            if ((st = check_product_args(descs[i], xs[i], ys[i], workspaces[i], workspace_bytes_each, batch)) != HUFFLLM_OK) return st;
+            if (!tc_blob(descs[i]))
+                return fail(HUFFLLM_ERR_UNSUPPORTED, "more than %u vectors per call over several matrices take tables of up to 9 bits (FP16: 8)", kTwoTileBatch);
+            for (uint32_t j = 0; j < i; ++j)
+                if (workspaces[j] == workspaces[i]) return fail(HUFFLLM_ERR_INVALID_ARG, "matrices %u and %u share a workspace", j, i);
+            if ((st = add_matrix(&k, descs[i], blobs[i])) != HUFFLLM_OK) return st;
+            k.m[i].x = xs[i];
+            k.m[i].y = ys[i];
+        }
+        if ((st = finish_args(&k, true, dev, &grid)) != HUFFLLM_OK) return st;      // (deals the CTAs to the matrices by their chunks)
+        const uint32_t npad = batch <= 32 ? 32 : 64;
+        uint32_t tiles = 4;                             // what the matrix with the largest records leaves room for
+        for (uint32_t i = 0; i < n; ++i) {
+            const TcPlan tp = tc_plan(descs[i], batch, (uint32_t)dev.sms, k.dyn_smem_bytes);
+            if (tc_smem_need(descs[i], tp.npad, tp.tiles) > k.dyn_smem_bytes)
+                return fail(HUFFLLM_ERR_UNSUPPORTED, "chunk records of matrix %u too large for the tensor-core kernel's slots", i);
+            if (tp.tiles < tiles) tiles = tp.tiles;
+        }
+        k.part_bytes = tc_stages(npad) * npad * 128;
+        k.slots = 2;
+        k.pair_recip = (uint32_t)(0x100000000ull / (2ull * k.slot_bytes));
+        k.tc_npad = npad;
+        k.tc_tiles = tiles;
+        uint32_t first = 0;
+        for (uint32_t i = 0; i < n; ++i) {
+            const TcPlan tp = tc_plan(descs[i], batch, k.m[i].cta_count, k.dyn_smem_bytes, tiles);
+            if (workspace_bytes_each < tp.bytes) return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "workspace of matrix %u too small for batch %u", i, batch);
+            t.m_tiles[i] = tp.m_tiles;
+            t.ksplit[i] = tp.ksplit;
+            t.ticket[i] = (unsigned int *)((uint8_t *)workspaces[i] + tp.ticket_off);
+            t.partial[i] = (float *)((uint8_t *)workspaces[i] + tp.partial_off);
+            k.m[i].cta_first = first;
+            if (tp.items < k.m[i].cta_count) k.m[i].cta_count = tp.items;
+            first += k.m[i].cta_count;
+        }
+        k.err = err_flag;
+        cudaError_t e = launch_gemm_tc(t, first, (cudaStream_t)stream);
+        if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "tensor-core product launch: %s", cudaGetErrorString(e));
+        return HUFFLLM_OK;
+    }
     KernelArgs k;
     uint32_t grid;
     begin_args(&k, batch, dev);
@@ -415,9 +466,11 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
     auto tensor_core = [&](bool other_path_left) -> huffllm_status {
         // one pass over the compressed weights for the whole batch (tables of up to 9 bits; longer codes take passes of 8
         // vectors through the register-path kernel and its two-level lookup)
-        if (!(desc->dtype == HUFFLLM_FP16 ? desc->lut_bits == 8u : desc->lut_bits <= 9u)) return HUFFLLM_OK;
+        if (!tc_blob(desc)) return HUFFLLM_OK;
         const TcPlan tp = tc_plan(desc, batch, (uint32_t)dev.sms, (uint32_t)dev.smem_optin - kStaticSmem);
-        KernelArgs k;
+        TcArgs t;
+        memset(&t, 0, sizeof(t));
+        KernelArgs &k = t.k;
         begin_args(&k, batch, dev);
         huffllm_status s2 = add_matrix(&k, desc, blob);
         if (s2 != HUFFLLM_OK) return s2;
@@ -433,13 +486,15 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
         k.m[0].y = y;
         k.tc_npad = tp.npad;
         k.tc_tiles = tp.tiles;
-        k.tc_m_tiles = tp.m_tiles;
-        k.tc_ksplit = tp.ksplit;
-        k.tc_ticket = (unsigned int *)((uint8_t *)workspace + tp.ticket_off);
-        k.tc_partial = (float *)((uint8_t *)workspace + tp.partial_off);
+        t.m_tiles[0] = tp.m_tiles;
+        t.ksplit[0] = tp.ksplit;
+        t.ticket[0] = (unsigned int *)((uint8_t *)workspace + tp.ticket_off);
+        t.partial[0] = (float *)((uint8_t *)workspace + tp.partial_off);
         k.err = err_flag;
         const uint32_t grid = tp.items < (uint32_t)dev.sms ? tp.items : (uint32_t)dev.sms;
-        cudaError_t e = launch_gemm_tc(k, grid, (cudaStream_t)stream);
+        k.m[0].cta_first = 0;
+        k.m[0].cta_count = grid;
+        cudaError_t e = launch_gemm_tc(t, grid, (cudaStream_t)stream);
         if (e != cudaSuccess) return fail(HUFFLLM_ERR_CUDA, "tensor-core product launch: %s", cudaGetErrorString(e));
         done = true;
         return HUFFLLM_OK;
@@ -486,7 +541,7 @@ huffllm_status huffllm_decode_gemm_multi_host_async(uint32_t n, const huffllm_de
     clear_error();
     if (!descs || !xs_host || !ys_host || !x_stages || !y_stages) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
     if (n == 0 || n > kMaxMats) return fail(HUFFLLM_ERR_INVALID_ARG, "between 1 and %u matrices per call", kMaxMats);
-    if (batch == 0 || batch > kTwoTileBatch) return fail(HUFFLLM_ERR_UNSUPPORTED, "batch must be in [1, %u] here", kTwoTileBatch);
+    if (batch == 0 || batch > 64) return fail(HUFFLLM_ERR_INVALID_ARG, "batch must be in [1, 64]");
     cudaStream_t s = (cudaStream_t)stream;
     for (uint32_t i = 0; i < n; ++i) {     // nothing is enqueued before every argument has been looked at
         if (!descs[i] || !xs_host[i] || !ys_host[i] || !x_stages[i] || !y_stages[i]) return fail(HUFFLLM_ERR_INVALID_ARG, "null pointer");
@@ -495,8 +550,10 @@ huffllm_status huffllm_decode_gemm_multi_host_async(uint32_t n, const huffllm_de
         if (st != HUFFLLM_OK) return st;
         if (!blobs || !blobs[i] || ((uintptr_t)blobs[i] & 255))
             return fail(HUFFLLM_ERR_INVALID_ARG, "blob must be a 256-byte aligned device pointer");
-        if (batch > kKernelBatch && !two_tile_blob(descs[i]))
-            return fail(HUFFLLM_ERR_UNSUPPORTED, "more than %u vectors per call take BF16 blobs of max_code_len 8", kKernelBatch);
+        if (batch > kKernelBatch && batch <= kTwoTileBatch && !two_tile_blob(descs[i]))
+            return fail(HUFFLLM_ERR_UNSUPPORTED, "9 to %u vectors per call over several matrices take BF16 blobs of max_code_len 8", kTwoTileBatch);
+        if (batch > kTwoTileBatch && !tc_blob(descs[i]))
+            return fail(HUFFLLM_ERR_UNSUPPORTED, "more than %u vectors per call over several matrices take tables of up to 9 bits (FP16: 8)", kTwoTileBatch);
     }
     for (uint32_t i = 0; i < n; ++i) {
         cudaError_t e = cudaMemcpyAsync(x_stages[i], xs_host[i], (size_t)batch * descs[i]->cols * 2, cudaMemcpyHostToDevice, s);

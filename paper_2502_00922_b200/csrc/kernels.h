@@ -38,10 +38,8 @@ struct KernelArgs {
     // tensor-core small-batch path only
     uint32_t tc_npad;          // batch rounded up to 16, 32 or 64
     uint32_t tc_tiles;         // 128-row tiles a CTA decodes side by side (8 warps each): 1..4
-    uint32_t tc_m_tiles;       // row tiles of 128 * tc_tiles rows
-    uint32_t tc_ksplit;        // ranges the column chunks are cut into
-    float *tc_partial;         // [m_tiles * ksplit][32 warps][npad / 2][32]
-    unsigned int *tc_ticket;   // [m_tiles][32], zero between calls
+    uint32_t tc_reserved[2];   // (the per-matrix values of that path live in TcArgs; these words keep the fields behind
+    void *tc_reserved_p[2];    //  them where the register-path kernels were measured with them)
     MatArgs m[kMaxMats];
     // (behind the matrices, so that the fields the hot loops read keep their places)
     uint32_t slots;            // slots per decoder warp: 2 (the next record lands while this one is decoded), or 1 where two would
@@ -49,9 +47,19 @@ struct KernelArgs {
                                // Kernels with single slots exist for FP16 blobs and for BF16 blobs with 8-bit tables.
 };
 
+// Arguments of the tensor-core kernel: the launch description plus, per matrix, its work items and where their pieces meet.
+// (The CTAs of a launch are dealt to the matrices as in the other kernels: m[i].cta_first / cta_count.)
+struct TcArgs {
+    KernelArgs k;
+    uint32_t m_tiles[kMaxMats];        // row tiles (of the decoder warps' row groups) of matrix i
+    uint32_t ksplit[kMaxMats];         // ranges its column chunks are cut into; work items = m_tiles * ksplit
+    float *partial[kMaxMats];          // [m_tiles * ksplit][32 warps][npad / 2][32]
+    unsigned int *ticket[kMaxMats];    // [m_tiles][32], zero between calls
+};
+
 cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t stream);
 cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream);
-cudaError_t launch_gemm_tc(const KernelArgs &k, uint32_t grid, cudaStream_t stream);
+cudaError_t launch_gemm_tc(const TcArgs &t, uint32_t grid, cudaStream_t stream);
 cudaError_t launch_stage_copy(void *dst, const void *src, uint64_t bytes, uint32_t sms, cudaStream_t stream);
 // The dense bf16 comparison product: up to kMaxMats matrices per launch, rows dealt to the warps round-robin.
 struct PlainMat {

@@ -104,7 +104,8 @@ __device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t addr, uint32_t lbo
 // LB = table index bits; NPAD = batch rounded up to 16, 32 or 64 (the MMA's N); FMT = 0: BF16 blobs, 1: FP16 {1,5,5,5} blobs
 // (three tables, sign words as the raw part, f16 operands).
 template <int LB, int NPAD, int FMT>
-__global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_constant__ KernelArgs A) {
+__global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_constant__ TcArgs T) {
+    const KernelArgs &A = T.k;
     constexpr uint32_t kRawBlock = FMT ? 64u : 512u;          // raw bytes of one block of a record
     constexpr uint32_t kRawLane = FMT ? 2u : 16u;             // of which one lane's share
     auto raw_part = [](uint32_t nkb) -> uint32_t { return FMT ? (nkb * 64u + 127u) & ~127u : nkb * 512u; };
@@ -131,7 +132,12 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     pdl_launch_dependents();   // the next kernel in the stream may be scheduled early; it waits for this one before it reads results
-    const MatArgs &k = A.m[0];
+    // the matrix this CTA works in (the launch's CTAs are dealt to its matrices; a CTA builds one table), and the CTA's
+    // number among that matrix's CTAs: it takes the matrix's work items J, J + n_cta, ...
+    uint32_t mi = 0;
+    while (mi + 1 < A.n_mats && blockIdx.x >= A.m[mi + 1].cta_first) ++mi;
+    const MatArgs &k = A.m[mi];
+    const uint32_t J = blockIdx.x - k.cta_first, n_cta = k.cta_count;
     const uint32_t smem_base = smem_u32(dyn_smem);
     // decoder warps: eight per tile, except that the CTA's last warp never decodes: it issues the MMAs (with four tiles the
     // last tile has seven row groups; its last 16 rows are never read).  Warps between the decoders and the issuer leave at once.
@@ -192,7 +198,9 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     const uint32_t KC = k.col_chunks, RG = (uint32_t)((k.rows + 15) / 16);
     const uint32_t *index = (const uint32_t *)(k.blob + k.off_index);
     const uint8_t *payload = k.blob + k.off_payload;
-    const uint32_t ksplit = A.tc_ksplit, n_items = A.tc_m_tiles * ksplit;
+    const uint32_t ksplit = T.ksplit[mi], n_items = T.m_tiles[mi] * ksplit;
+    float *const tc_partial = T.partial[mi];
+    unsigned int *const tc_ticket = T.ticket[mi];
     uint32_t phase = 0, gb = 0;          // coded-copy barrier parities; blocks this CTA has gone through so far
     bool failed = false;                 // a wait ran out: stop waiting, keep moving, report
 
@@ -306,7 +314,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     bool primed = false;                 // the item's first two record copies were started at the end of the item before
 
 #pragma unroll 1
-    for (uint32_t item = blockIdx.x; item < n_items; item += gridDim.x) {
+    for (uint32_t item = J; item < n_items; item += n_cta) {
         const uint32_t mt = item / ksplit, ks = item % ksplit;
         const uint32_t rg = mt * n_dec + rgi;
         const bool active = rg < RG;
@@ -405,9 +413,9 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
 
         // both slots are free again: the next item's first records are asked for now, so that they arrive behind the epilogue
         primed = false;
-        if (warp < n_dec && item + gridDim.x < n_items) {
+        if (warp < n_dec && item + n_cta < n_items) {
             uint32_t nb, ne;
-            if (item_chunks(item + gridDim.x, nb, ne)) {
+            if (item_chunks(item + n_cta, nb, ne)) {
                 if (lane == 0) {
                     issue(nb, 0);
                     if (nb + 1 < ne) issue(nb + 1, 1);
@@ -436,13 +444,13 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                     if (n0 + i < A.batch && row_ok) k.y[(uint64_t)(n0 + i) * k.rows + row] = __uint_as_float(v[i]);
             } else {
                 // piece of (item, warp): [NPAD/2][32] floats; the last range to arrive adds the pieces in range order
-                float *piece = A.tc_partial + ((size_t)item * 32 + warp) * (NPAD / 2) * 32;   // 32 piece slots per item, n_dec used
+                float *piece = tc_partial + ((size_t)item * 32 + warp) * (NPAD / 2) * 32;   // 32 piece slots per item, n_dec used
 #pragma unroll
                 for (int i = 0; i < NPAD / 2; ++i) piece[i * 32 + lane] = __uint_as_float(v[i]);
                 __syncwarp();
                 uint32_t last = 0;
                 if (lane == 0) {
-                    unsigned int *ctr = A.tc_ticket + mt * 32 + warp;
+                    unsigned int *ctr = tc_ticket + mt * 32 + warp;
                     last = arrive_acq_rel(ctr) == ksplit - 1 ? 1u : 0u;
                     if (last) *ctr = 0;
                 }
@@ -452,7 +460,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
 #pragma unroll
                     for (int i = 0; i < NPAD / 2; ++i) sum[i] = 0.f;
                     for (uint32_t s2 = 0; s2 < ksplit; ++s2) {
-                        const float *pc = A.tc_partial + ((size_t)(mt * ksplit + s2) * 32 + warp) * (NPAD / 2) * 32 + lane;
+                        const float *pc = tc_partial + ((size_t)(mt * ksplit + s2) * 32 + warp) * (NPAD / 2) * 32 + lane;
 #pragma unroll
                         for (int i = 0; i < NPAD / 2; ++i) sum[i] += __ldcg(pc + i * 32);
                     }
@@ -471,7 +479,8 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
 }
 
 template <int LB, int NPAD, int FMT>
-static cudaError_t launch_tc_one(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
+static cudaError_t launch_tc_one(const TcArgs &t, uint32_t grid, cudaStream_t stream) {
+    const KernelArgs &k = t.k;
     auto fn = huff_gemm_tc_kernel<LB, NPAD, FMT>;
     static std::atomic<bool> attr_set[64];   // set twice by racing threads at worst: the call is idempotent
     int dev = 0;
@@ -491,23 +500,24 @@ static cudaError_t launch_tc_one(const KernelArgs &k, uint32_t grid, cudaStream_
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, fn, k);
+    return cudaLaunchKernelEx(&cfg, fn, t);
 }
 
-cudaError_t launch_gemm_tc(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
+cudaError_t launch_gemm_tc(const TcArgs &t, uint32_t grid, cudaStream_t stream) {
+    const KernelArgs &k = t.k;
     if (k.fmt) {
-        if (k.tc_npad == 16) return launch_tc_one<8, 16, 1>(k, grid, stream);
-        if (k.tc_npad == 32) return launch_tc_one<8, 32, 1>(k, grid, stream);
-        return launch_tc_one<8, 64, 1>(k, grid, stream);
+        if (k.tc_npad == 16) return launch_tc_one<8, 16, 1>(t, grid, stream);
+        if (k.tc_npad == 32) return launch_tc_one<8, 32, 1>(t, grid, stream);
+        return launch_tc_one<8, 64, 1>(t, grid, stream);
     }
     if (k.lut_bits == 8) {
-        if (k.tc_npad == 16) return launch_tc_one<8, 16, 0>(k, grid, stream);
-        if (k.tc_npad == 32) return launch_tc_one<8, 32, 0>(k, grid, stream);
-        return launch_tc_one<8, 64, 0>(k, grid, stream);
+        if (k.tc_npad == 16) return launch_tc_one<8, 16, 0>(t, grid, stream);
+        if (k.tc_npad == 32) return launch_tc_one<8, 32, 0>(t, grid, stream);
+        return launch_tc_one<8, 64, 0>(t, grid, stream);
     }
-    if (k.tc_npad == 16) return launch_tc_one<9, 16, 0>(k, grid, stream);
-    if (k.tc_npad == 32) return launch_tc_one<9, 32, 0>(k, grid, stream);
-    return launch_tc_one<9, 64, 0>(k, grid, stream);
+    if (k.tc_npad == 16) return launch_tc_one<9, 16, 0>(t, grid, stream);
+    if (k.tc_npad == 32) return launch_tc_one<9, 32, 0>(t, grid, stream);
+    return launch_tc_one<9, 64, 0>(t, grid, stream);
 }
 
 }  // namespace huffllm

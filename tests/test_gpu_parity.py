@@ -303,10 +303,10 @@ def test_long_code_tables_decode_and_product(hl, torch, rows, cols, ce, budget, 
         assert np.array_equal(y1, gpu_gemm(hl, torch, up, x)), "results must be bitwise reproducible"
 
 
-@pytest.mark.parametrize("batch", [1, 3, 13])
+@pytest.mark.parametrize("batch", [1, 3, 13, 33, 64])
 def test_several_matrices_in_one_launch(hl, torch, batch):
-    """Matrices of different shapes and chunk sizes through huffllm_decode_gemm_multi: every result against the
-    oracle, and the launch must leave every workspace's control words zero."""
+    """Matrices of different shapes and chunk sizes through huffllm_decode_gemm_multi (one vector, one tile, two tiles,
+    tensor core): every result against the oracle, and the launch must leave every workspace's control words zero."""
     shapes = [(256, 1024, 4096, "gauss"), (48, 2080, 1024, "student"), (1040, 512, 512, "gauss"), (16, 8192, 4096, "gauss"),
               (2368, 256, 4096, "uniform")]
     ups, xs, x_devs, ys = [], [], [], []
