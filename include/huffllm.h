@@ -120,7 +120,9 @@ typedef struct huffllm_desc {
     uint32_t n_fields;        /* coded fields per weight: 2 (BF16 {1,4,4,7}), 1 ({1,8,7}), 3 (FP16 {1,5,5,5}) */
     uint8_t  caps[4];         /* per-field maximum code length chosen under lut_bits       */
     uint16_t pad_word;        /* weight stored at positions outside the tensor            */
-    uint16_t reserved0;
+    uint16_t flat_fields;     /* FP16 blobs: bit f set = coded field f carries the flat code (all 32 symbols, 5 bits each, the
+                                 codeword of symbol s is s): the decoders then read that field without its table.  Written
+                                 by the encoders; 0 is always valid (every field is decoded through its table)       */
     uint32_t max_words;       /* largest W over all chunks                                 */
     uint64_t off_codebook, off_lut, off_index, off_payload;   /* byte offsets in the blob */
     uint64_t payload_bytes;   /* 128 * index[n_chunks]                                     */

@@ -27,7 +27,7 @@ class Desc(C.Structure):
                 ("rows", C.c_uint64), ("cols", C.c_uint64), ("tile_rows", C.c_uint32), ("chunk_cols", C.c_uint32),
                 ("row_groups", C.c_uint32), ("col_chunks", C.c_uint32), ("n_chunks", C.c_uint64),
                 ("lut_bits", C.c_uint32), ("lag_bits", C.c_uint32), ("n_fields", C.c_uint32), ("caps", C.c_uint8 * 4),
-                ("pad_word", C.c_uint16), ("reserved0", C.c_uint16), ("max_words", C.c_uint32),
+                ("pad_word", C.c_uint16), ("flat_fields", C.c_uint16), ("max_words", C.c_uint32),
                 ("off_codebook", C.c_uint64), ("off_lut", C.c_uint64), ("off_index", C.c_uint64),
                 ("off_payload", C.c_uint64), ("payload_bytes", C.c_uint64), ("blob_bytes", C.c_uint64),
                 ("coded_bits", C.c_uint64), ("raw_bits", C.c_uint64), ("payload_checksum", C.c_uint64),

@@ -195,6 +195,9 @@ huffllm_status add_matrix(KernelArgs *k, const huffllm_desc *desc, const void *b
     m.col_chunks = desc->col_chunks;
     k->total_chunks += m.n_chunks;
     k->lut_bits = desc->lut_bits;
+    // (flat mantissa codes: only if every matrix of the launch has them)
+    const uint32_t flat = fmt && (desc->flat_fields & 6u) == 6u ? 1u : 0u;
+    k->fp16_flat = k->n_mats == 1 ? flat : (k->fp16_flat & flat);
     const SmemNeeds need = smem_needs(desc);
     k->lut_align = need.table_align;
     k->lut_size = need.table_bytes;

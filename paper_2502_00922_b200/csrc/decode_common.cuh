@@ -389,6 +389,19 @@ __device__ __forceinline__ uint32_t fp16_weight_inplace(LaneStream &s, uint32_t 
     asm("lop3.b32 %0, %1, %2, %3, 0xFE;" : "=r"(w) : "r"(e0), "r"(e1), "r"(e2));
     return w;                                      // bits 8..22: exponent and mantissa
 }
+// Both mantissa halves carry the FLAT code (all 32 symbols, 5 bits each: the canonical codeword of symbol s is s, written
+// first bit first), which is what fp16-trained weights give: their mantissa bits are incompressible.  The ten stream bits
+// behind the exponent's codeword are then the weight's ten mantissa bits in reverse order: one bit reversal replaces two
+// table lookups.  (The exponent's table and everything else is as in fp16_weight_inplace; bits 0..7 of the result hold
+// the exponent's length and later stream bits, which the packing step never looks at.)
+__device__ __forceinline__ uint32_t fp16_weight_flat(LaneStream &s, uint32_t lut_lane) {
+    stream_refill4<false>(s);
+    uint32_t t = window_at(s);
+    const uint32_t e0 = lds_lut(__dp4a(t, 0x00000040u, lut_lane));
+    t = shift_by_entry(t, e0);
+    s.pos = s.pos + e0 + 10u;
+    return e0 | (__brev(t) >> 14);                 // bits 8..17: the mantissa, bits 18..22: the exponent
+}
 // Field codes of at most 7 bits: the same three-at-a-time scheme on tables of 128 entries, which are small enough to keep
 // once per LANE (entry i of lane l at word 32 i + l, 16 KB per field: the footprint of the sixteen-fold 256-entry tables),
 // so that a warp-wide lookup never has a bank conflict.  Seven index bits are not a byte, so the window is moved up by 7
@@ -412,14 +425,18 @@ __device__ __forceinline__ uint32_t fp16_weight_lane(LaneStream &s, uint32_t lut
 }
 // Decode one block of an FP16 chunk into 8 packed registers (same order as decode_block).  `signs` is the lane's
 // uint16 of the block: bit p = sign of the first weight of pair p, bit 8 + p = sign of its second weight.
-// INPLACE: the three-at-a-time decoders above: 1 = tables of 8 bits (sixteen-fold), 2 = tables of 7 bits (per lane).
+// INPLACE: the three-at-a-time decoders above: 1 = tables of 8 bits (sixteen-fold), 2 = tables of 7 bits (per lane),
+// 3 = tables of 8 bits with flat codes for both mantissa halves.
 template <bool LONG = false, int INPLACE = 0>
 __device__ __forceinline__ void decode_block_fp16(LaneStream &sa, LaneStream &sb, uint32_t lut_lane, uint32_t signs,
                                                   uint32_t (&a)[8], uint32_t full_base = 0, uint32_t full_mask = 0) {
     uint32_t w[16];
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
-        if (INPLACE == 2) {
+        if (INPLACE == 3) {
+            w[i] = fp16_weight_flat(sa, lut_lane);
+            w[8 + i] = fp16_weight_flat(sb, lut_lane);
+        } else if (INPLACE == 2) {
             w[i] = fp16_weight_lane(sa, lut_lane);
             w[8 + i] = fp16_weight_lane(sb, lut_lane);
         } else if (INPLACE == 1) {

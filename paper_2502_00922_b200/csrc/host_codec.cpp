@@ -48,6 +48,9 @@ huffllm_status check_desc(const huffllm_desc *d) {
     if (d->tile_rows != kTileRows || d->chunk_cols != d->chunk_elems / kTileRows || d->lag_bits != lag_bits_for(d->dtype) ||
         (d->dtype == HUFFLLM_BF16 && d->n_fields != 2 && d->n_fields != 1) || (d->dtype == HUFFLLM_FP16 && d->n_fields != 3))
         return fail(HUFFLLM_ERR_CORRUPT, "bad tile geometry");
+    if (d->flat_fields & ~7u) return fail(HUFFLLM_ERR_CORRUPT, "bad flat_fields");
+    if (d->flat_fields && (d->dtype != HUFFLLM_FP16 || d->lut_bits < 5))
+        return fail(HUFFLLM_ERR_CORRUPT, "flat_fields set where no field can carry the flat code");
     if (d->row_groups != (d->rows + kTileRows - 1) / kTileRows ||
         d->col_chunks != (d->cols + d->chunk_cols - 1) / d->chunk_cols ||
         d->n_chunks != (uint64_t)d->row_groups * d->col_chunks)
@@ -469,6 +472,12 @@ void fill_desc_fixed(const huffllm_codebook *cb, uint64_t rows, uint64_t cols, u
     d.n_fields = cb->n_fields;
     memcpy(d.caps, cb->caps, 4);
     d.pad_word = cb->pad_word;
+    if (cb->dtype == HUFFLLM_FP16)
+        for (int k = 0; k < 3; ++k) {      // flat code: all 32 symbols at 5 bits (canonical codes are then the symbols themselves)
+            bool flat = true;
+            for (int s = 0; s < 32; ++s) flat = flat && cb->len[k][s] == 5;
+            if (flat) d.flat_fields |= (uint16_t)(1u << k);
+        }
     d.off_codebook = 256;
     d.off_lut = 512;
     d.off_index = d.off_lut + align_up((cb->dtype == HUFFLLM_FP16 ? 3 : 1) * (4ull << cb->budget), 256);
@@ -694,6 +703,9 @@ huffllm_status huffllm_validate_blob(const void *blob, size_t bytes, huffllm_des
             memcpy(cb.len[k], base + d.off_codebook + 32 * k, 32);
             if (!check_code(cb.len[k], 32, 32, d.caps[k], k)) return HUFFLLM_ERR_CORRUPT;
             if (d.caps[k] > d.lut_bits) return fail(HUFFLLM_ERR_CORRUPT, "caps exceed lut_bits");
+            if (d.flat_fields >> k & 1u)
+                for (int s = 0; s < 32; ++s)
+                    if (cb.len[k][s] != 5) return fail(HUFFLLM_ERR_CORRUPT, "flat_fields names a field whose code is not flat");
             canonical_codes(cb.len[k], 32, cb.code[k]);
         }
     } else if (d.n_fields == 2) {

@@ -38,7 +38,8 @@ namespace huffllm {
 // MODE 0: write the decoded weights.  MODE 1: y = W x for up to 8 activation vectors.
 // LB = table index bits (the blobs' lut_bits): 8 or 9; LB = 12 stands for every longer limit up to 12 (BF16: 10..12,
 // FP16: 9..12): two-level lookup, the number of bits is A.lut_bits.
-// FMT = 0: BF16 blobs; FMT = 1: FP16 {1,5,5,5} blobs (three lookups per weight, sign bits as the raw part).
+// FMT = 0: BF16 blobs; FMT = 1: FP16 {1,5,5,5} blobs (three lookups per weight, sign bits as the raw part); FMT = 2: the same
+// where both mantissa halves carry the flat 5-bit code (8-bit tables only: one lookup and a bit reversal per weight).
 //
 // One launch works through a LIST of matrices (A.n_mats, usually the matrices of one decoder layer that
 // may run together).  The CTAs are dealt out to the matrices in proportion to their chunks, so every CTA
@@ -67,7 +68,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     // 8-bit BF16 tables: the decoder starts behind the sequences' leading zero bits and works on four codewords at a
     // time (stream_step4x2)
     constexpr bool SKIP = LB == 8 && FMT == 0;
-    constexpr int SKIP16 = FMT == 1 ? (LB == 8 ? 1 : LB == 7 ? 2 : 0) : 0;   // the same scheme for FP16: three codewords (one weight) at a
+    constexpr int SKIP16 = FMT ? (LB == 8 ? (FMT == 2 ? 3 : 1) : LB == 7 ? 2 : 0) : 0;   // the same scheme for FP16: three codewords (one weight) at a
                                                              // time; 2 = field codes of 7 bits, tables once per lane
     constexpr bool LONG = LB > 9;                            // first level of 8 bits, then the whole table (FP16: lut_bits 9..12)
     constexpr uint32_t kLB1 = LONG ? 8u : (uint32_t)LB;      // index bits of the per-lane table
@@ -672,6 +673,7 @@ static cudaError_t launch_slots(const KernelArgs &k, uint32_t grid, cudaStream_t
 
 cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
     if (k.fmt && k.lut_bits == 7) return launch_slots<0, 7, 1>(k, grid, stream);
+    if (k.fmt && k.lut_bits == 8 && k.fp16_flat) return launch_slots<0, 8, 2>(k, grid, stream);
     if (k.fmt) return k.lut_bits > 8 ? launch_slots<0, 12, 1>(k, grid, stream) : launch_slots<0, 8, 1>(k, grid, stream);
     if (k.lut_bits > 9) return launch_one<0, 12, kThreads, 0>(k, grid, stream);
     return k.lut_bits == 8 ? launch_slots<0, 8, 0>(k, grid, stream) : launch_one<0, 9, kThreads, 0>(k, grid, stream);
@@ -680,6 +682,7 @@ cudaError_t launch_decode(const KernelArgs &k, uint32_t grid, cudaStream_t strea
 cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream) {
     if (k.batch == 1 && k.fmt) {                  // one vector: multiply-adds on the FMA pipe
         if (k.lut_bits == 7) return launch_slots<1, 7, 1, 0>(k, grid, stream);
+        if (k.lut_bits == 8 && k.fp16_flat) return launch_slots<1, 8, 2, 0>(k, grid, stream);
         return k.lut_bits > 8 ? launch_slots<1, 12, 1, 0>(k, grid, stream) : launch_slots<1, 8, 1, 0>(k, grid, stream);
     }
     if (k.batch == 1) {
@@ -688,6 +691,7 @@ cudaError_t launch_gemm(const KernelArgs &k, uint32_t grid, cudaStream_t stream)
     }
     if (k.batch > 8) return launch_slots<1, 8, 0, 2>(k, grid, stream);   // (the entry point sends only BF16 blobs of 8-bit tables here)
     if (k.fmt && k.lut_bits == 7) return launch_slots<1, 7, 1>(k, grid, stream);
+    if (k.fmt && k.lut_bits == 8 && k.fp16_flat) return launch_slots<1, 8, 2>(k, grid, stream);
     if (k.fmt) return k.lut_bits > 8 ? launch_slots<1, 12, 1>(k, grid, stream) : launch_slots<1, 8, 1>(k, grid, stream);
     if (k.lut_bits > 9) return launch_one<1, 12, kThreads, 0>(k, grid, stream);
     return k.lut_bits == 8 ? launch_slots<1, 8, 0>(k, grid, stream) : launch_one<1, 9, kThreads, 0>(k, grid, stream);

@@ -45,6 +45,7 @@ struct KernelArgs {
     uint32_t slots;            // slots per decoder warp: 2 (the next record lands while this one is decoded), or 1 where two would
                                // leave too few warps a slot (large records: the feeder then waits for a slot before every copy).
                                // Kernels with single slots exist for FP16 blobs and for BF16 blobs with 8-bit tables.
+    uint32_t fp16_flat;        // FP16 blobs: both mantissa halves of every matrix of the launch carry the flat 5-bit code
 };
 
 // Arguments of the tensor-core kernel: the launch description plus, per matrix, its work items and where their pieces meet.
