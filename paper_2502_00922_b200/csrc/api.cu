@@ -93,8 +93,10 @@ uint64_t tc_smem_need(const huffllm_desc *d, uint32_t npad, uint32_t tiles) {
     return lut + (guard > b_stages ? guard - b_stages : 0) + b_stages + 4096 + 2ull * (8 * tiles < 31 ? 8 * tiles : 31) * d->max_words * 256;
 }
 // `sms`: the CTAs this matrix can have (all SMs, or its share of a launch over several matrices); `tiles_cap`: the tiles
-// the launch's other matrices leave room for.
-TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn_smem, uint32_t tiles_cap = 4) {
+// the launch's other matrices leave room for; `max_bytes`: the workspace at hand (column ranges whose pieces would not
+// fit are not considered: a share of the SMs can favour more ranges than the whole GPU, for which workspaces are sized).
+TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn_smem, uint32_t tiles_cap = 4,
+               size_t max_bytes = ~(size_t)0) {
     TcPlan p;
     p.npad = batch <= 16 ? 16 : (batch <= 32 ? 32 : 64);
     p.tiles = tiles_cap;                            // as many 8-warp tiles as the chunk slots leave room for
@@ -111,6 +113,7 @@ TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn
     uint64_t best_span = ~0ull;
     for (uint32_t ks = 1; ks <= 16 && ks <= d->col_chunks; ++ks) {
         const uint64_t items = (uint64_t)p.m_tiles * ks, grid = items < sms ? items : sms;
+        if (ks > 1 && ws_partial_offset(d) + (size_t)items * 32 * (p.npad / 2) * 32 * sizeof(float) > max_bytes) break;
         uint64_t span = 0;
         for (uint64_t b = 0; b < grid; ++b) {
             uint64_t t = 0;
@@ -393,7 +396,7 @@ huffllm_status huffllm_decode_gemm_multi(uint32_t n, const huffllm_desc *const *
         k.tc_tiles = tiles;
         uint32_t first = 0;
         for (uint32_t i = 0; i < n; ++i) {
-            const TcPlan tp = tc_plan(descs[i], batch, k.m[i].cta_count, k.dyn_smem_bytes, tiles);
+            const TcPlan tp = tc_plan(descs[i], batch, k.m[i].cta_count, k.dyn_smem_bytes, tiles, workspace_bytes_each);
             if (workspace_bytes_each < tp.bytes) return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "workspace of matrix %u too small for batch %u", i, batch);
             t.m_tiles[i] = tp.m_tiles;
             t.ksplit[i] = tp.ksplit;

@@ -101,7 +101,7 @@ __device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t addr, uint32_t lbo
     return (uint64_t)((addr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo >> 4) << 16) | ((uint64_t)(sbo >> 4) << 32) | (1ull << 46);
 }
 
-// LB = table index bits; NPAD = batch rounded up to 16, 32 or 64 (the MMA's N); FMT = 0: BF16 blobs, 1: FP16 {1,5,5,5} blobs
+// LB = table index bits; NPAD = batch rounded up to 16, 32 or 64 (the MMA's N); FMT = 0: BF16 blobs, 1: FP16 {1,5,5,5} blobs, 2: FP16 blobs with flat mantissa codes
 // (three tables, sign words as the raw part, f16 operands).
 template <int LB, int NPAD, int FMT>
 __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_constant__ TcArgs T) {
@@ -115,6 +115,8 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     };
     // the decoder that starts behind the leading zero bits and takes four codewords at a time (see huff_kernel)
     constexpr bool SKIP = LB == 8 && FMT == 0;
+    // FP16 (8-bit tables only here): three codewords at a time with in-place shifts; FMT = 2: flat codes for both mantissa halves
+    constexpr int SKIP16 = FMT ? (FMT == 2 ? 3 : 1) : 0;
     constexpr int R = SKIP ? 4 : LB == 8 ? 3 : 2;
     constexpr uint32_t kIdxMask = ((1u << LB) - 1u) << 7;
     constexpr int S = NPAD == 64 ? 2 : kTcStages;          // the host's tc_stages(): shared memory is short at the widest padding
@@ -161,7 +163,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
         constexpr uint32_t kLutWords = FMT ? 3u * 16u * 256u : 32u << LB;
         for (uint32_t i = tid; i < kLutWords; i += 1024) {
             const uint32_t v = __ldg(lut_g + (i >> (FMT ? 4 : 5)));
-            lut_s[i] = SKIP ? lut_entry_inplace(v) : v;
+            lut_s[i] = SKIP ? lut_entry_inplace(v) : SKIP16 ? fp16_entry_inplace(v) : v;
         }
     }
     if (lane == 0) {
@@ -368,8 +370,8 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                     continue;
                 }
                 LaneStream sa, sb;
-                stream_open(sa, slot0 + which * A.slot_bytes + (lane << 2), SKIP ? 7u : 0u);
-                stream_open(sb, slot0 + which * A.slot_bytes + 128u + (lane << 2), SKIP ? 7u : 0u);
+                stream_open(sa, slot0 + which * A.slot_bytes + (lane << 2), SKIP ? 7u : SKIP16 ? 6u : 0u);
+                stream_open(sb, slot0 + which * A.slot_bytes + 128u + (lane << 2), SKIP ? 7u : SKIP16 ? 6u : 0u);
                 // one block: fetch the next block's raw bytes and activations into the other register set, decode
                 // this one, hand it to the tensor core
                 auto block = [&](const uint4 &raw_c, uint4 &raw_n, const uint4 &x_c, uint4 &x_n2, bool more, uint32_t half, bool publish) {
@@ -378,7 +380,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
                     if (x_p < x_end) load_x(x_n2, x_p);
                     x_p += 32;
                     uint32_t a[8];
-                    if (FMT) decode_block_fp16(sa, sb, lut_lane, raw_c.x, a);
+                    if (FMT) decode_block_fp16<false, SKIP16>(sa, sb, lut_lane, raw_c.x, a);
                     else decode_block<R, SKIP>(sa, sb, kIdxMask, lut_lane, raw_c, a);
                     stage_block(a, x_c, half, publish);
                 };
@@ -505,6 +507,11 @@ static cudaError_t launch_tc_one(const TcArgs &t, uint32_t grid, cudaStream_t st
 
 cudaError_t launch_gemm_tc(const TcArgs &t, uint32_t grid, cudaStream_t stream) {
     const KernelArgs &k = t.k;
+    if (k.fmt && k.fp16_flat) {
+        if (k.tc_npad == 16) return launch_tc_one<8, 16, 2>(t, grid, stream);
+        if (k.tc_npad == 32) return launch_tc_one<8, 32, 2>(t, grid, stream);
+        return launch_tc_one<8, 64, 2>(t, grid, stream);
+    }
     if (k.fmt) {
         if (k.tc_npad == 16) return launch_tc_one<8, 16, 1>(t, grid, stream);
         if (k.tc_npad == 32) return launch_tc_one<8, 32, 1>(t, grid, stream);
