@@ -282,7 +282,7 @@ def decode_tensor(enc) -> np.ndarray:
 # Layout (little endian).  Header, 256 bytes:
 #   0 magic "HFLM" | 4 u32 version | 8 u32 dtype | 12 u32 chunk_elems | 16 u64 rows | 24 u64 cols
 #   32 u32 tile_rows | 36 u32 chunk_cols | 40 u32 row_groups | 44 u32 col_chunks | 48 u64 n_chunks
-#   56 u32 lut_bits | 60 u32 lag_bits | 64 u32 n_fields | 68 u8 caps[4] | 72 u16 pad_word | 74 u16 0
+#   56 u32 lut_bits | 60 u32 lag_bits | 64 u32 n_fields | 68 u8 caps[4] | 72 u16 pad_word | 74 u16 flat_fields (a hint to the device decoders; not used here)
 #   76 u32 max_words | 80 u64 off_codebook | 88 u64 off_lut | 96 u64 off_index | 104 u64 off_payload
 #   112 u64 payload_bytes | 120 u64 blob_bytes | 128 u64 coded_bits | 136 u64 raw_bits | 144 u64 checksum
 # codebook: n_fields == 2: u8 lengths[3][32] (two nibble codes, third row zero); n_fields == 1: u8 lengths[256]

@@ -323,6 +323,47 @@ def test_launch_plan_slots_per_warp():
             hl.decode_launch_plan(d, 9)
 
 
+def test_flat_fields_mark_exactly_the_flat_codes():
+    """FP16 blobs: the descriptor marks the fields whose code is the flat one (all 32 symbols at 5 bits, codeword = symbol):
+    both mantissa halves of fp16-trained weights, only the upper half of bf16-trained weights stored as fp16, none of
+    skewed data; BF16 blobs never.  A mark on a field whose code is not flat is refused by the validator, no mark at all
+    is always accepted (the decoders then use the tables)."""
+    cases = [("fp16", 0b110), ("fp16_from_bf16", 0b010)]
+    for name, want in cases:
+        w = wl.gaussian_weights(64, 4096, 0.02, 95, name)
+        cb = hl.build_codebook(w, hl.FP16)
+        lens = [cb.get(f)[2] for f in range(3)]
+        blob, d = hl.encode(cb, w, 1024)
+        cb.free()
+        flat = sum(1 << f for f in range(3) if all(int(l) == 5 for l in lens[f][:32]))
+        assert d.flat_fields == flat == want, (name, d.flat_fields, flat)
+        # the codewords of a flat field are the symbols themselves (canonical code), which is what lets a decoder skip its table
+        parsed = orc.parse_blob(blob)
+        assert parsed["header"]["_r"] == want
+        hl.validate_blob(blob)
+        unmarked = blob.copy()
+        unmarked[74:76] = 0
+        assert hl.validate_blob(unmarked).flat_fields == 0
+        wrong = blob.copy()
+        wrong[74] = 0b111                      # the exponent's code is never flat on these weights
+        with pytest.raises(hl.HuffllmError):
+            hl.validate_blob(wrong)
+    w = wl.skewed_exponent_weights(64, 1024, 96, dtype="fp16")
+    cb = hl.build_codebook(w, hl.FP16)
+    _, d = hl.encode(cb, w, 1024)
+    cb.free()
+    assert d.flat_fields == 0
+    w = wl.gaussian_weights(64, 1024, 0.02, 97)
+    cb = hl.build_codebook(w)
+    blob, d = hl.encode(cb, w, 1024)
+    cb.free()
+    assert d.flat_fields == 0
+    bad = blob.copy()
+    bad[74] = 2
+    with pytest.raises(hl.HuffllmError):
+        hl.validate_blob(bad)
+
+
 def test_code_length_limits_accepted_per_format():
     """BF16 budgets 8..12 (the two nibble codes of a weight together); FP16 field limits 7..12."""
     wb = wl.gaussian_weights(16, 512, 0.02, 92)
