@@ -337,6 +337,42 @@ def small_batch_leg(hl, torch, dev, stream, chunk_elems: int, peak_for_small: fl
     return out
 
 
+def fp16_leg(hl, torch, dev, stream, chunk_elems: int, peak: float):
+    """The paper's FP16 {1,5,5,5} format (Section 3.1) on one matrix of the layer (gate, 11008 x 4096) with fp16-trained
+    weights, batch 1, at the benchmark's chunk size: ms per product and fraction of the HBM peak on the compressed bytes."""
+    name, rows, cols = "gate", 11008, 4096
+    w = wl.gaussian_weights(rows, cols, 0.02, 1000 + 4, "fp16")
+    cb = hl.build_codebook(w, hl.FP16)
+    blob, desc = hl.encode(cb, w, chunk_elems)
+    cb.free()
+    del w
+    blob_dev = torch.from_numpy(blob).to(dev)
+    err = torch.zeros(1, dtype=torch.int32, device=dev)
+    ws_bytes = hl.workspace_bytes(desc, 1)
+    ws = torch.zeros(ws_bytes, dtype=torch.uint8, device=dev)
+    x = torch.from_numpy(wl.activations(1, cols, 1504, "fp16").view(np.int16).reshape(-1)).to(dev)
+    y = torch.zeros(rows, dtype=torch.float32, device=dev)
+    for _ in range(5):
+        hl.decode_gemv(desc, blob_dev, x, y, ws, ws_bytes, err, stream)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    n = 400
+    a.record(stream)
+    for _ in range(n):
+        hl.decode_gemv(desc, blob_dev, x, y, ws, ws_bytes, err, stream)
+    b.record(stream)
+    torch.cuda.synchronize()
+    assert int(err.item()) == 0
+    ms = a.elapsed_time(b) / n
+    alg = desc.payload_bytes + 4 * (desc.n_chunks + 1) + 3 * (4 << desc.lut_bits) + 2 * cols + 4 * rows
+    plan = hl.decode_launch_plan(desc, 1)
+    return {"matrix": f"{name} {rows}x{cols}", "weights": "fp16-trained (gaussian), FP16 {1,5,5,5}", "chunk_elems": chunk_elems,
+            "compressed_bytes": int(desc.blob_bytes), "compression_ratio_total": 2.0 * rows * cols / desc.blob_bytes,
+            "ms": ms, "frac_of_hbm_peak": alg / (ms * 1e-3) / 1e9 / peak, "uncompressed_GBs": 2.0 * rows * cols / (ms * 1e-3) / 1e9,
+            "flat_fields": int(desc.flat_fields), "slots_per_warp": plan["slots_per_warp"], "decoder_warps": plan["decoder_warps"],
+            "kernel": "huff_kernel<product, one vector, FP16" + (", flat mantissa codes>" if desc.flat_fields & 6 == 6 else ">")}
+
+
 def sweep_8b_leg(hl, torch, dev, stream, chunk_elems: int, peak: float, layers: int = 32):
     """The per-token pass over an 8B-shaped model: `layers` decoder layers, every layer with its own copy of the seven
     blobs in HBM (same content, distinct memory), four launches per layer, batch 1; beside it the dense bf16 sweep of the
@@ -748,8 +784,10 @@ def main():
 
     # ---- one 70B-FFN-shaped matrix at batch 1 / 16 / 64: register path and tensor-core path under the same clock
     small_batch = None
+    fp16_one = None
     if rank == 0 and world == 1 and not args.no_small_batch and not fp16 and args.workload == "llama7b_layer" and L == 1:
         small_batch = small_batch_leg(hl, torch, dev, stream, args.chunk_elems, peak_for_small=measured_peak()[0])
+        fp16_one = fp16_leg(hl, torch, dev, stream, args.chunk_elems, measured_peak()[0])
     sweep_8b = None
     if rank == 0 and world == 1 and not args.no_sweep and not fp16 and args.workload == "llama7b_layer" and L == 1 and B == 1:
         sweep_8b = sweep_8b_leg(hl, torch, dev, stream, args.chunk_elems, measured_peak()[0])
@@ -810,6 +848,7 @@ def main():
                             "note": "own streaming kernel in the same launch groups as the compressed path; the north star asks for "
                                     "speedup_vs_own_dense >= compression_ratio_total"},
         "small_batch": small_batch,
+        "fp16": fp16_one,
         "sweep_8b_32_layers": sweep_8b,
         "cpu_baseline_all_cores": cpu_all,
         "timing": {"regions": R, "steps_per_region": args.steps, "ms_per_step_min": ms_min, "ms_per_step_median": ms_step,
