@@ -84,23 +84,25 @@ struct TcPlan {
 // Shared memory the tensor-core kernel needs with `tiles` 128-row tiles per CTA.
 // Stages of the tensor-core kernel: four, two at the widest batch padding, where shared memory is short.
 uint32_t tc_stages(uint32_t npad) { return npad == 64 ? 2u : 3u; }
-uint64_t tc_smem_need(const huffllm_desc *d, uint32_t npad, uint32_t tiles) {
+// (`flat`: every matrix of the launch has flat FP16 mantissa codes: the exponent's table alone is kept)
+bool flat_fp16(const huffllm_desc *d) { return d->dtype == HUFFLLM_FP16 && d->lut_bits == 8 && (d->flat_fields & 6u) == 6u; }
+uint64_t tc_smem_need(const huffllm_desc *d, uint32_t npad, uint32_t tiles, bool flat) {
     const bool fp16 = d->dtype == HUFFLLM_FP16;
     const uint32_t checks_per_block = fp16 ? 8 : (d->lut_bits == 8 ? 3 : 4);
     uint64_t guard = 256ull * (3 + checks_per_block * (d->chunk_cols / kBlockCols));
-    const uint64_t lut = fp16 ? 49152ull : 128ull << d->lut_bits;
+    const uint64_t lut = fp16 ? (flat ? 16384ull : 49152ull) : 128ull << d->lut_bits;
     const uint64_t b_stages = (uint64_t)tc_stages(npad) * npad * 128;          // the guard area may lie over them
     return lut + (guard > b_stages ? guard - b_stages : 0) + b_stages + 4096 + 2ull * (8 * tiles < 31 ? 8 * tiles : 31) * d->max_words * 256;
 }
 // `sms`: the CTAs this matrix can have (all SMs, or its share of a launch over several matrices); `tiles_cap`: the tiles
 // the launch's other matrices leave room for; `max_bytes`: the workspace at hand (column ranges whose pieces would not
 // fit are not considered: a share of the SMs can favour more ranges than the whole GPU, for which workspaces are sized).
-TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn_smem, uint32_t tiles_cap = 4,
+TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn_smem, bool flat, uint32_t tiles_cap = 4,
                size_t max_bytes = ~(size_t)0) {
     TcPlan p;
     p.npad = batch <= 16 ? 16 : (batch <= 32 ? 32 : 64);
     p.tiles = tiles_cap;                            // as many 8-warp tiles as the chunk slots leave room for
-    while (p.tiles > 1 && tc_smem_need(d, p.npad, p.tiles) > dyn_smem) --p.tiles;
+    while (p.tiles > 1 && tc_smem_need(d, p.npad, p.tiles, flat) > dyn_smem) --p.tiles;
     const uint32_t n_dec = 8 * p.tiles < 31 ? 8 * p.tiles : 31;      // the CTA's last warp issues the MMAs and never decodes
     p.m_tiles = (d->row_groups + n_dec - 1) / n_dec;
     // Column ranges: the one with the shortest finish time.  A CTA takes items b, b + grid, ... in turn; an item costs its
@@ -150,8 +152,11 @@ SmemNeeds smem_needs(const huffllm_desc *desc) {
     // first 8 bits, then one copy of the whole table behind it
     // (FP16: three sixteen-fold tables of 8 bits; fields of 9 bits and more take the second level too)
     const bool two_level = desc->lut_bits > (fmt ? 8u : 9u);
+    // (FP16 blobs whose mantissa codes are flat need the exponent's table only; a launch over several matrices of which
+    // some are not marked takes all three, see fp16_table_bytes)
     n.table_align = fmt ? 16384u : 128u << (two_level ? 8u : desc->lut_bits);
-    n.table_bytes = fmt ? 49152u + (two_level ? 3u * (4u << desc->lut_bits) : 0u)
+    const bool flat = fmt && desc->lut_bits == 8 && (desc->flat_fields & 6u) == 6u;
+    n.table_bytes = fmt ? (flat ? 16384u : 49152u) + (two_level ? 3u * (4u << desc->lut_bits) : 0u)
                         : (two_level ? (128u << 8) + (4u << desc->lut_bits) : 128u << desc->lut_bits);
     // a slot holds the W rows of a record; the window runs one row ahead of what it consumes, and that look-ahead
     // past the last row lands in the next slot, the table or the guard area and is never used
@@ -164,6 +169,10 @@ SmemNeeds smem_needs(const huffllm_desc *desc) {
     n.guard_bytes = 256 * (3 + n.checks_per_block * (desc->chunk_cols / kBlockCols));
     return n;
 }
+
+// Bytes of the FP16 tables a launch keeps in shared memory: three sixteen-fold tables of 8-bit codes, or the exponent's
+// alone where every matrix of the launch has flat mantissa codes (those are read without tables).
+uint32_t fp16_table_bytes(const KernelArgs *k) { return k->lut_bits == 8 && k->fp16_flat ? 16384u : 49152u; }
 
 // Start a launch description.
 void begin_args(KernelArgs *k, uint32_t batch, const DeviceInfo &dev) {
@@ -213,6 +222,7 @@ huffllm_status add_matrix(KernelArgs *k, const huffllm_desc *desc, const void *b
 huffllm_status finish_args(KernelArgs *k, bool product, const DeviceInfo &dev, uint32_t *grid, uint32_t *warps_at_least = nullptr) {
     // (pieces that warps of a CTA exchange: in shared memory up to 8 vectors, in the workspace above)
     k->part_bytes = product && k->batch <= kKernelBatch ? 2 * 32 * 16 * k->batch * (uint32_t)sizeof(float) : 0;
+    if (k->fmt && k->lut_bits <= 8) k->lut_size = fp16_table_bytes(k);
     // worst case for the table's alignment gap is covered by assuming the window starts within 4 KB of zero
     uint64_t fixed = (uint64_t)k->lut_size + (k->guard_bytes > k->part_bytes ? k->guard_bytes - k->part_bytes : 0) + k->part_bytes + 4096;
     if (fixed + k->slot_bytes > k->dyn_smem_bytes)
@@ -275,7 +285,7 @@ huffllm_status huffllm_workspace_bytes(const huffllm_desc *desc, uint32_t batch,
         clear_error();
         const int sms = have ? dev.sms : 148;
         const uint32_t dyn = (have ? (uint32_t)dev.smem_optin : 232448u) - kStaticSmem;
-        size_t tc = tc_plan(desc, batch, (uint32_t)sms, dyn).bytes;
+        size_t tc = tc_plan(desc, batch, (uint32_t)sms, dyn, false).bytes;     // (with all three FP16 tables: the larger plan)
         if (tc > *bytes) *bytes = tc;
     }
     return HUFFLLM_OK;
@@ -384,8 +394,8 @@ huffllm_status huffllm_decode_gemm_multi(uint32_t n, const huffllm_desc *const *
         const uint32_t npad = batch <= 32 ? 32 : 64;
         uint32_t tiles = 4;                             // what the matrix with the largest records leaves room for
         for (uint32_t i = 0; i < n; ++i) {
-            const TcPlan tp = tc_plan(descs[i], batch, (uint32_t)dev.sms, k.dyn_smem_bytes);
-            if (tc_smem_need(descs[i], tp.npad, tp.tiles) > k.dyn_smem_bytes)
+            const TcPlan tp = tc_plan(descs[i], batch, (uint32_t)dev.sms, k.dyn_smem_bytes, k.fp16_flat != 0);
+            if (tc_smem_need(descs[i], tp.npad, tp.tiles, k.fp16_flat != 0) > k.dyn_smem_bytes)
                 return fail(HUFFLLM_ERR_UNSUPPORTED, "chunk records of matrix %u too large for the tensor-core kernel's slots", i);
             if (tp.tiles < tiles) tiles = tp.tiles;
         }
@@ -396,7 +406,7 @@ huffllm_status huffllm_decode_gemm_multi(uint32_t n, const huffllm_desc *const *
         k.tc_tiles = tiles;
         uint32_t first = 0;
         for (uint32_t i = 0; i < n; ++i) {
-            const TcPlan tp = tc_plan(descs[i], batch, k.m[i].cta_count, k.dyn_smem_bytes, tiles, workspace_bytes_each);
+            const TcPlan tp = tc_plan(descs[i], batch, k.m[i].cta_count, k.dyn_smem_bytes, k.fp16_flat != 0, tiles, workspace_bytes_each);
             if (workspace_bytes_each < tp.bytes) return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "workspace of matrix %u too small for batch %u", i, batch);
             t.m_tiles[i] = tp.m_tiles;
             t.ksplit[i] = tp.ksplit;
@@ -473,7 +483,8 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
         // one pass over the compressed weights for the whole batch (tables of up to 9 bits; longer codes take passes of 8
         // vectors through the register-path kernel and its two-level lookup)
         if (!tc_blob(desc)) return HUFFLLM_OK;
-        const TcPlan tp = tc_plan(desc, batch, (uint32_t)dev.sms, (uint32_t)dev.smem_optin - kStaticSmem);
+        // (column ranges are planned within the workspace at hand)
+        const TcPlan tp = tc_plan(desc, batch, (uint32_t)dev.sms, (uint32_t)dev.smem_optin - kStaticSmem, flat_fp16(desc), 4, workspace_bytes);
         TcArgs t;
         memset(&t, 0, sizeof(t));
         KernelArgs &k = t.k;
@@ -483,7 +494,7 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
         k.part_bytes = tc_stages(tp.npad) * tp.npad * 128;      // the stages of activations
         k.slots = 2;
         k.pair_recip = (uint32_t)(0x100000000ull / (2ull * k.slot_bytes));
-        if (tc_smem_need(desc, tp.npad, tp.tiles) > k.dyn_smem_bytes) return HUFFLLM_OK;   // records too large for this kernel's slots
+        if (tc_smem_need(desc, tp.npad, tp.tiles, flat_fp16(desc)) > k.dyn_smem_bytes) return HUFFLLM_OK;   // records too large for this kernel's slots
         if (workspace_bytes < tp.bytes) {
             if (other_path_left) return HUFFLLM_OK;     // (the register path needs less)
             return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "workspace too small for batch %u", batch);

@@ -183,7 +183,8 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
     // written to shared memory (by the decoder warps alone: the feeder is already asking for records)
     // (FP16: three tables of 256 entries, sixteen copies each: word j holds entry j / 16 of its table)
     // The table goes to shared memory in 16-byte pieces: four neighbouring copies of one entry per piece.
-    constexpr uint32_t kLutWords = FMT ? 3u * 16u * 256u : 32u << kLB1;   // (FP16, 7 bits: 3 x 32 x 128, the same)
+    // (FP16, 7 bits: 3 x 32 x 128, the same; flat mantissa codes: the exponent's table alone)
+    constexpr uint32_t kLutWords = FMT == 2 ? 16u * 256u : FMT ? 3u * 16u * 256u : 32u << kLB1;
     constexpr uint32_t kLutRep = FMT && LB != 7 ? 4u : 5u; // log2 of the copies per entry
     constexpr uint32_t kLutVecs = kLutWords / 4;
     constexpr uint32_t kLutThreads = THREADS - 32;

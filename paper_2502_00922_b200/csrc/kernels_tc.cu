@@ -160,7 +160,7 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
         const uint32_t *lut_g = (const uint32_t *)(k.blob + k.off_lut);
         uint32_t *lut_s = (uint32_t *)(dyn_smem + (plan.lut - smem_base));
         // (FP16: three tables of 256 entries, sixteen copies each: word j holds entry j / 16)
-        constexpr uint32_t kLutWords = FMT ? 3u * 16u * 256u : 32u << LB;
+        constexpr uint32_t kLutWords = FMT == 2 ? 16u * 256u : FMT ? 3u * 16u * 256u : 32u << LB;   // (flat mantissa codes: the exponent's table alone)
         for (uint32_t i = tid; i < kLutWords; i += 1024) {
             const uint32_t v = __ldg(lut_g + (i >> (FMT ? 4 : 5)));
             lut_s[i] = SKIP ? lut_entry_inplace(v) : SKIP16 ? fp16_entry_inplace(v) : v;
