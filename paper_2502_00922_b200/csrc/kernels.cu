@@ -430,6 +430,9 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                 // block (the address lies inside the blob whatever that record's offsets turn out to be)
                 const bool has_next = c + 1 < c_end;
                 const uint32_t coded_bytes = (r1 - r0 - raw_units(nkb)) << 7;
+                // from the end of the record's last raw block to the next record: the coded part and, in FP16 records with an
+                // odd number of blocks, the 64 bytes that pad the raw part to a whole unit
+                const uint32_t to_next = FMT ? ((r1 - r0) << 7) - nkb * kRawBlock : coded_bytes;
                 LaneStream sa, sb;
                 stream_open(sa, slot_cur, SKIP ? 7u : SKIP16 ? 6u : 0u);
                 stream_open(sb, slot_cur + 128u, SKIP ? 7u : SKIP16 ? 6u : 0u);
@@ -453,7 +456,7 @@ __global__ void __launch_bounds__(THREADS, 1) huff_kernel(const __grid_constant_
                     raw_p += kRawBlock;
                     if (kPrefetchRaw) asm volatile("prefetch.global.L2 [%0];" ::"l"(raw_p + 3u * kRawBlock));
                     if (decltype(may_be_last)::value) {
-                        if (kb == last) raw_p += coded_bytes;       // the next record's first block
+                        if (kb == last) raw_p += to_next;           // the next record's first block
                         if (kb != last || has_next) nxt = load_raw(raw_p);
                     } else {
                         nxt = load_raw(raw_p);

@@ -590,6 +590,23 @@ def test_distribution_stress_full_size(hl, torch, gen, ce):
     assert np.all(np.abs(y[0, rs] - yo[0]) <= TOL * d[0])
 
 
+@pytest.mark.parametrize("rows,cols,ce,gen", [
+    (586, 4032, 512, "fp16_from_bf16"),      # one block per chunk, several chunks per warp
+    (586, 4032, 512, "fp16"),                # ... through the flat-code decoder
+    (2400, 2080, 1024, "fp16"),              # two blocks per chunk, one in each row's last chunk, more chunks than warps
+])
+def test_fp16_records_with_an_odd_number_of_blocks_in_a_row(hl, torch, rows, cols, ce, gen):
+    """An FP16 record's raw part (64 bytes of signs per block) is padded to a whole 128-byte unit when its chunk has an
+    odd number of blocks; a warp that goes from such a record straight to its next one must step over the padding.
+    (Found by a randomised run: with at most one chunk per warp, as in the smaller cases, the step is never taken.)"""
+    w = wl.gaussian_weights(rows, cols, 0.02, 7002, gen)
+    up = Uploaded(hl, torch, w, ce, 0, 3, dtype=hl.FP16)
+    assert np.array_equal(gpu_decode(hl, torch, up), w)
+    for batch in (1, 3):
+        x = wl.activations(batch, cols, 7100 + batch, "fp16")
+        check_product(gpu_gemm(hl, torch, up, x), w, x, orc.FP16)
+
+
 @pytest.mark.parametrize("dtype,ce", [("fp16", 4096), ("bf16", 8192)])
 def test_single_slots_reused_full_size(hl, torch, dtype, ce):
     """Records that get one shared-memory slot per decoder warp, on a matrix large enough that every warp goes through
