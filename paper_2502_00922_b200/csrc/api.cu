@@ -75,6 +75,56 @@ size_t ws_bytes_for(const huffllm_desc *d, uint32_t batch) {
     return ws_partial_offset(d) + need;
 }
 
+// What a blob asks of a decoder CTA's shared memory.
+struct SmemNeeds {
+    uint32_t table_align, table_bytes;   // window of the decode table(s)
+    uint32_t slot_bytes;                 // one slot: the W rows of the largest record
+    uint32_t checks_per_block;           // refill checks per bit sequence and block of 32 columns
+    uint32_t guard_bytes;                // readable bytes kept behind the last slot
+};
+SmemNeeds smem_needs(const huffllm_desc *desc) {
+    SmemNeeds n;
+    const bool fmt = desc->dtype == HUFFLLM_FP16;
+    // BF16 tables of up to 9 bits are replicated per lane; longer ones are looked up in two levels: a per-lane table of the
+    // first 8 bits, then one copy of the whole table behind it
+    // (FP16: three sixteen-fold tables of 8 bits; fields of 9 bits and more take the second level too)
+    const bool two_level = desc->lut_bits > (fmt ? 8u : 9u);
+    // (FP16 blobs whose mantissa codes are flat need the exponent's table only; a launch over several matrices of which
+    // some are not marked takes all three, see fp16_table_bytes)
+    n.table_align = fmt ? 16384u : 128u << (two_level ? 8u : desc->lut_bits);
+    const bool flat = fmt && desc->lut_bits == 8 && (desc->flat_fields & 6u) == 6u;
+    n.table_bytes = fmt ? (flat ? 16384u : 49152u) + (two_level ? 3u * (4u << desc->lut_bits) : 0u)
+                        : (two_level ? (128u << 8) + (4u << desc->lut_bits) : 128u << desc->lut_bits);
+    // a slot holds the W rows of a record; the window runs one row ahead of what it consumes, and that look-ahead
+    // past the last row lands in the next slot, the table or the guard area and is never used
+    n.slot_bytes = desc->max_words * 256;
+    // A stream can move its read pointer by one row per refill check and no further, whatever its bits and whatever the
+    // table says: a sequence opens on rows 0 and 1, and every check loads at most the next row.  The furthest row a
+    // chunk's decoder can touch is therefore 1 + checks, counted from the slot's first row, and the bytes kept readable
+    // behind the last slot cover that for a slot of any size.
+    n.checks_per_block = fmt ? (two_level ? 24 : 8) : (desc->lut_bits == 8 ? 3 : 4);
+    n.guard_bytes = 256 * (3 + n.checks_per_block * (desc->chunk_cols / kBlockCols));
+    return n;
+}
+
+// How many decoder warps get their slots: the kernels' own shared-memory plan (plan_smem in decode_common.cuh) worked out
+// on the host.  Slots lie in front of and behind the decode table, which sits on a boundary of `lut_align` bytes, so up to a
+// slot pair's bytes are lost on either side; where the dynamic window starts depends on the kernel's static shared memory,
+// which the host does not know exactly: the smallest count over every 128-byte start within kStaticSmem + 1 KB is taken.
+uint32_t planned_warps(uint32_t lut_align, uint32_t lut_size, uint64_t pair_bytes, uint32_t dyn_smem, uint32_t part_bytes,
+                       uint32_t guard_bytes) {
+    const uint64_t guard_extra = guard_bytes > part_bytes ? guard_bytes - part_bytes : 0;
+    uint64_t least = ~0ull;
+    for (uint64_t base = 0; base <= kStaticSmem + 1024; base += 128) {
+        const uint64_t lut = (base + lut_align - 1) / lut_align * lut_align;
+        const uint64_t n_a = lut > base ? (lut - base) / pair_bytes : 0;
+        const uint64_t slot_b = lut + lut_size, end = base + dyn_smem - part_bytes;
+        const uint64_t n_b = end > slot_b + guard_extra ? (end - slot_b - guard_extra) / pair_bytes : 0;
+        if (n_a + n_b < least) least = n_a + n_b;
+    }
+    return (uint32_t)(least > 64 ? 64 : least);
+}
+
 // Geometry of the tensor-core small-batch path (batch 9..64): row tiles of 512 rows, column chunks cut into
 // `ksplit` ranges so that the work items fill the GPU's SMs in whole waves as well as they can.
 struct TcPlan {
@@ -86,13 +136,13 @@ struct TcPlan {
 uint32_t tc_stages(uint32_t npad) { return npad == 64 ? 2u : 3u; }
 // (`flat`: every matrix of the launch has flat FP16 mantissa codes: the exponent's table alone is kept)
 bool flat_fp16(const huffllm_desc *d) { return d->dtype == HUFFLLM_FP16 && d->lut_bits == 8 && (d->flat_fields & 6u) == 6u; }
-uint64_t tc_smem_need(const huffllm_desc *d, uint32_t npad, uint32_t tiles, bool flat) {
-    const bool fp16 = d->dtype == HUFFLLM_FP16;
-    const uint32_t checks_per_block = fp16 ? 8 : (d->lut_bits == 8 ? 3 : 4);
-    uint64_t guard = 256ull * (3 + checks_per_block * (d->chunk_cols / kBlockCols));
-    const uint64_t lut = fp16 ? (flat ? 16384ull : 49152ull) : 128ull << d->lut_bits;
-    const uint64_t b_stages = (uint64_t)tc_stages(npad) * npad * 128;          // the guard area may lie over them
-    return lut + (guard > b_stages ? guard - b_stages : 0) + b_stages + 4096 + 2ull * (8 * tiles < 31 ? 8 * tiles : 31) * d->max_words * 256;
+// Do the slot pairs of `tiles` tiles' decoder warps fit beside the tables and the stages of activations?
+bool tc_fits(const huffllm_desc *d, uint32_t npad, uint32_t tiles, bool flat, uint32_t dyn_smem) {
+    SmemNeeds n = smem_needs(d);
+    if (d->dtype == HUFFLLM_FP16 && d->lut_bits == 8) n.table_bytes = flat ? 16384u : 49152u;   // (a launch-wide choice)
+    const uint32_t b_stages = tc_stages(npad) * npad * 128;          // the guard area may lie over them
+    const uint32_t n_dec = 8 * tiles < 31 ? 8 * tiles : 31;
+    return planned_warps(n.table_align, n.table_bytes, 2ull * n.slot_bytes, dyn_smem, b_stages, n.guard_bytes) >= n_dec;
 }
 // `sms`: the CTAs this matrix can have (all SMs, or its share of a launch over several matrices); `tiles_cap`: the tiles
 // the launch's other matrices leave room for; `max_bytes`: the workspace at hand (column ranges whose pieces would not
@@ -102,7 +152,7 @@ TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn
     TcPlan p;
     p.npad = batch <= 16 ? 16 : (batch <= 32 ? 32 : 64);
     p.tiles = tiles_cap;                            // as many 8-warp tiles as the chunk slots leave room for
-    while (p.tiles > 1 && tc_smem_need(d, p.npad, p.tiles, flat) > dyn_smem) --p.tiles;
+    while (p.tiles > 1 && !tc_fits(d, p.npad, p.tiles, flat, dyn_smem)) --p.tiles;
     const uint32_t n_dec = 8 * p.tiles < 31 ? 8 * p.tiles : 31;      // the CTA's last warp issues the MMAs and never decodes
     p.m_tiles = (d->row_groups + n_dec - 1) / n_dec;
     // Column ranges: the one with the shortest finish time.  A CTA takes items b, b + grid, ... in turn; an item costs its
@@ -136,38 +186,6 @@ TcPlan tc_plan(const huffllm_desc *d, uint32_t batch, uint32_t sms, uint32_t dyn
     p.partial_off = ws_partial_offset(d);
     p.bytes = p.partial_off + (best > 1 ? (size_t)p.items * 32 * (p.npad / 2) * 32 * sizeof(float) : 0);
     return p;
-}
-
-// What a blob asks of a decoder CTA's shared memory.
-struct SmemNeeds {
-    uint32_t table_align, table_bytes;   // window of the decode table(s)
-    uint32_t slot_bytes;                 // one slot: the W rows of the largest record
-    uint32_t checks_per_block;           // refill checks per bit sequence and block of 32 columns
-    uint32_t guard_bytes;                // readable bytes kept behind the last slot
-};
-SmemNeeds smem_needs(const huffllm_desc *desc) {
-    SmemNeeds n;
-    const bool fmt = desc->dtype == HUFFLLM_FP16;
-    // BF16 tables of up to 9 bits are replicated per lane; longer ones are looked up in two levels: a per-lane table of the
-    // first 8 bits, then one copy of the whole table behind it
-    // (FP16: three sixteen-fold tables of 8 bits; fields of 9 bits and more take the second level too)
-    const bool two_level = desc->lut_bits > (fmt ? 8u : 9u);
-    // (FP16 blobs whose mantissa codes are flat need the exponent's table only; a launch over several matrices of which
-    // some are not marked takes all three, see fp16_table_bytes)
-    n.table_align = fmt ? 16384u : 128u << (two_level ? 8u : desc->lut_bits);
-    const bool flat = fmt && desc->lut_bits == 8 && (desc->flat_fields & 6u) == 6u;
-    n.table_bytes = fmt ? (flat ? 16384u : 49152u) + (two_level ? 3u * (4u << desc->lut_bits) : 0u)
-                        : (two_level ? (128u << 8) + (4u << desc->lut_bits) : 128u << desc->lut_bits);
-    // a slot holds the W rows of a record; the window runs one row ahead of what it consumes, and that look-ahead
-    // past the last row lands in the next slot, the table or the guard area and is never used
-    n.slot_bytes = desc->max_words * 256;
-    // A stream can move its read pointer by one row per refill check and no further, whatever its bits and whatever the
-    // table says: a sequence opens on rows 0 and 1, and every check loads at most the next row.  The furthest row a
-    // chunk's decoder can touch is therefore 1 + checks, counted from the slot's first row, and the bytes kept readable
-    // behind the last slot cover that for a slot of any size.
-    n.checks_per_block = fmt ? (two_level ? 24 : 8) : (desc->lut_bits == 8 ? 3 : 4);
-    n.guard_bytes = 256 * (3 + n.checks_per_block * (desc->chunk_cols / kBlockCols));
-    return n;
 }
 
 // Bytes of the FP16 tables a launch keeps in shared memory: three sixteen-fold tables of 8-bit codes, or the exponent's
@@ -223,20 +241,17 @@ huffllm_status finish_args(KernelArgs *k, bool product, const DeviceInfo &dev, u
     // (pieces that warps of a CTA exchange: in shared memory up to 8 vectors, in the workspace above)
     k->part_bytes = product && k->batch <= kKernelBatch ? 2 * 32 * 16 * k->batch * (uint32_t)sizeof(float) : 0;
     if (k->fmt && k->lut_bits <= 8) k->lut_size = fp16_table_bytes(k);
-    // worst case for the table's alignment gap is covered by assuming the window starts within 4 KB of zero
-    uint64_t fixed = (uint64_t)k->lut_size + (k->guard_bytes > k->part_bytes ? k->guard_bytes - k->part_bytes : 0) + k->part_bytes + 4096;
-    if (fixed + k->slot_bytes > k->dyn_smem_bytes)
-        return fail(HUFFLLM_ERR_UNSUPPORTED, "chunk records too large for shared memory (slot %u bytes)", k->slot_bytes);
     // Two slots per decoder warp, so that a warp's next record lands while it decodes this one.  Where records are so large
     // that this would leave fewer than 31 warps a slot pair, and single slots serve at least a quarter more warps, every
     // warp gets one slot: more decoders at work outweigh the wait for a copy at every chunk start.
-    const uint64_t room = k->dyn_smem_bytes - fixed, max_w = 31;     // decoder warps of a CTA of 1024 threads
-    uint64_t w2 = room / (2ull * k->slot_bytes), w1 = room / k->slot_bytes;
+    const uint64_t max_w = 31;                                       // decoder warps of a CTA of 1024 threads
+    uint64_t w2 = planned_warps(k->lut_align, k->lut_size, 2ull * k->slot_bytes, k->dyn_smem_bytes, k->part_bytes, k->guard_bytes);
+    uint64_t w1 = planned_warps(k->lut_align, k->lut_size, k->slot_bytes, k->dyn_smem_bytes, k->part_bytes, k->guard_bytes);
     if (w2 > max_w) w2 = max_w;
     if (w1 > max_w) w1 = max_w;
     const bool single_ok = k->fmt || k->lut_bits == 8;                // (the kernels that exist with single slots)
     k->slots = single_ok && w2 < max_w && 4 * w1 >= 5 * w2 ? 1u : 2u;
-    if (k->slots == 2 && fixed + 2ull * k->slot_bytes > k->dyn_smem_bytes)
+    if ((k->slots == 2 ? w2 : w1) == 0)
         return fail(HUFFLLM_ERR_UNSUPPORTED, "chunk records too large for shared memory (slot %u bytes)", k->slot_bytes);
     if (warps_at_least) *warps_at_least = (uint32_t)(k->slots == 1 ? w1 : w2);
     k->pair_recip = (uint32_t)(0x100000000ull / ((uint64_t)k->slots * k->slot_bytes));
@@ -395,7 +410,7 @@ huffllm_status huffllm_decode_gemm_multi(uint32_t n, const huffllm_desc *const *
         uint32_t tiles = 4;                             // what the matrix with the largest records leaves room for
         for (uint32_t i = 0; i < n; ++i) {
             const TcPlan tp = tc_plan(descs[i], batch, (uint32_t)dev.sms, k.dyn_smem_bytes, k.fp16_flat != 0);
-            if (tc_smem_need(descs[i], tp.npad, tp.tiles, k.fp16_flat != 0) > k.dyn_smem_bytes)
+            if (!tc_fits(descs[i], tp.npad, tp.tiles, k.fp16_flat != 0, k.dyn_smem_bytes))
                 return fail(HUFFLLM_ERR_UNSUPPORTED, "chunk records of matrix %u too large for the tensor-core kernel's slots", i);
             if (tp.tiles < tiles) tiles = tp.tiles;
         }
@@ -494,7 +509,7 @@ huffllm_status huffllm_decode_gemm(const huffllm_desc *desc, const void *blob, c
         k.part_bytes = tc_stages(tp.npad) * tp.npad * 128;      // the stages of activations
         k.slots = 2;
         k.pair_recip = (uint32_t)(0x100000000ull / (2ull * k.slot_bytes));
-        if (tc_smem_need(desc, tp.npad, tp.tiles, flat_fp16(desc)) > k.dyn_smem_bytes) return HUFFLLM_OK;   // records too large for this kernel's slots
+        if (!tc_fits(desc, tp.npad, tp.tiles, flat_fp16(desc), k.dyn_smem_bytes)) return HUFFLLM_OK;   // records too large for this kernel's slots
         if (workspace_bytes < tp.bytes) {
             if (other_path_left) return HUFFLLM_OK;     // (the register path needs less)
             return fail(HUFFLLM_ERR_BUFFER_TOO_SMALL, "workspace too small for batch %u", batch);
