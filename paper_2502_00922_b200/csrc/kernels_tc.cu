@@ -103,7 +103,8 @@ __device__ __forceinline__ uint64_t smem_desc_kmajor(uint32_t addr, uint32_t lbo
 
 // LB = table index bits; NPAD = batch rounded up to 16, 32 or 64 (the MMA's N); FMT = 0: BF16 blobs, 1: FP16 {1,5,5,5} blobs, 2: FP16 blobs with flat mantissa codes
 // (three tables, sign words as the raw part, f16 operands).
-template <int LB, int NPAD, int FMT>
+// MULTI: the launch works through several matrices (a launch over one matrix reads its arguments without an index).
+template <int LB, int NPAD, int FMT, bool MULTI>
 __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_constant__ TcArgs T) {
     const KernelArgs &A = T.k;
     constexpr uint32_t kRawBlock = FMT ? 64u : 512u;          // raw bytes of one block of a record
@@ -137,8 +138,9 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     // the matrix this CTA works in (the launch's CTAs are dealt to its matrices; a CTA builds one table), and the CTA's
     // number among that matrix's CTAs: it takes the matrix's work items J, J + n_cta, ...
     uint32_t mi = 0;
-    while (mi + 1 < A.n_mats && blockIdx.x >= A.m[mi + 1].cta_first) ++mi;
-    const MatArgs &k = A.m[mi];
+    if (MULTI)
+        while (mi + 1 < A.n_mats && blockIdx.x >= A.m[mi + 1].cta_first) ++mi;
+    const MatArgs &k = A.m[MULTI ? mi : 0];
     const uint32_t J = blockIdx.x - k.cta_first, n_cta = k.cta_count;
     const uint32_t smem_base = smem_u32(dyn_smem);
     // decoder warps: eight per tile, except that the CTA's last warp never decodes: it issues the MMAs (with four tiles the
@@ -200,9 +202,9 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     const uint32_t KC = k.col_chunks, RG = (uint32_t)((k.rows + 15) / 16);
     const uint32_t *index = (const uint32_t *)(k.blob + k.off_index);
     const uint8_t *payload = k.blob + k.off_payload;
-    const uint32_t ksplit = T.ksplit[mi], n_items = T.m_tiles[mi] * ksplit;
-    float *const tc_partial = T.partial[mi];
-    unsigned int *const tc_ticket = T.ticket[mi];
+    const uint32_t ksplit = T.ksplit[MULTI ? mi : 0], n_items = T.m_tiles[MULTI ? mi : 0] * ksplit;
+    float *const tc_partial = T.partial[MULTI ? mi : 0];
+    unsigned int *const tc_ticket = T.ticket[MULTI ? mi : 0];
     uint32_t phase = 0, gb = 0;          // coded-copy barrier parities; blocks this CTA has gone through so far
     bool failed = false;                 // a wait ran out: stop waiting, keep moving, report
 
@@ -480,10 +482,10 @@ __global__ void __launch_bounds__(1024, 1) huff_gemm_tc_kernel(const __grid_cons
     if (warp == 0) tmem_dealloc(tmem, 512);
 }
 
-template <int LB, int NPAD, int FMT>
-static cudaError_t launch_tc_one(const TcArgs &t, uint32_t grid, cudaStream_t stream) {
+template <int LB, int NPAD, int FMT, bool MULTI>
+static cudaError_t launch_tc_m(const TcArgs &t, uint32_t grid, cudaStream_t stream) {
     const KernelArgs &k = t.k;
-    auto fn = huff_gemm_tc_kernel<LB, NPAD, FMT>;
+    auto fn = huff_gemm_tc_kernel<LB, NPAD, FMT, MULTI>;
     static std::atomic<bool> attr_set[64];   // set twice by racing threads at worst: the call is idempotent
     int dev = 0;
     cudaGetDevice(&dev);
@@ -503,6 +505,12 @@ static cudaError_t launch_tc_one(const TcArgs &t, uint32_t grid, cudaStream_t st
     cfg.attrs = attr;
     cfg.numAttrs = 1;
     return cudaLaunchKernelEx(&cfg, fn, t);
+}
+
+template <int LB, int NPAD, int FMT>
+static cudaError_t launch_tc_one(const TcArgs &t, uint32_t grid, cudaStream_t stream) {
+    if (t.k.n_mats > 1) return launch_tc_m<LB, NPAD, FMT, true>(t, grid, stream);
+    return launch_tc_m<LB, NPAD, FMT, false>(t, grid, stream);
 }
 
 cudaError_t launch_gemm_tc(const TcArgs &t, uint32_t grid, cudaStream_t stream) {
