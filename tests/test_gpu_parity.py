@@ -258,6 +258,7 @@ GEMM_CASES = [
     (16, 65536, 4096, 0, "gauss", 16),            # one row group, 16 column ranges
     (2368, 512, 512, 0, "uniform", 48),           # several work items per CTA
     (528, 2048, 4096, 9, "student", 32),          # 512-entry table
+    (69, 2496, 4096, 9, "student", 9),            # ... and records of 18 rows: two tiles is all that fits beside a 64 KB table
 ]
 
 
@@ -588,6 +589,43 @@ def test_distribution_stress_full_size(hl, torch, gen, ce):
     rs = np.random.default_rng(1).choice(rows, 48, replace=False)
     yo, d = orc.matmul(w[rs], x)
     assert np.all(np.abs(y[0, rs] - yo[0]) <= TOL * d[0])
+
+
+@pytest.mark.parametrize("seed", [1, 3])
+def test_random_shapes_formats_and_batches(hl, torch, seed):
+    """Seeded random configurations (shape, chunk size, format, code-length limit, split, batch, distribution): decode
+    against the original tensor, the product against the oracle.  Two of the cases such a run first met are kept above
+    as tests of their own (FP16 records with an odd number of blocks; long records with 512-entry tables on the tensor core)."""
+    rng = np.random.default_rng(seed)
+    ran = 0
+    for case in range(70):
+        dtype = rng.choice(["bf16", "bf16", "fp16", "fp16_from_bf16"])
+        rows = int(rng.choice([rng.integers(1, 80), rng.integers(80, 700), rng.integers(700, 2600)]))
+        cols = int(rng.integers(1, 160)) * 32
+        ce = int(rng.choice([512, 1024, 2048, 4096, 8192, 16384]))
+        batch = int(rng.choice([1, 1, 2, 5, 8, 9, 13, 16, 17, 32, 33, 64]))
+        if dtype == "bf16":
+            gen = str(rng.choice(["gauss", "student", "uniform", "skewed"]))
+            budget, split = int(rng.choice([0, 0, 9, 10, 12])), int(rng.choice([0, 0, 1]))
+            w = make(gen, rows, cols, 7000 + case)
+            hd, od = hl.BF16, orc.BF16
+        else:
+            budget, split = int(rng.choice([0, 0, 7, 9, 12])), 0
+            w = (wl.gaussian_weights(rows, cols, 0.02, 7000 + case, str(dtype)) if rng.random() < 0.8
+                 else wl.skewed_exponent_weights(rows, cols, 7000 + case, dtype="fp16"))
+            hd, od = hl.FP16, orc.FP16
+        what = (case, str(dtype), rows, cols, ce, batch, budget, split)
+        up = Uploaded(hl, torch, w, ce, budget, batch, split=split, dtype=hd)
+        try:
+            got = gpu_decode(hl, torch, up)
+        except hl.HuffllmError as e:          # records of the largest chunks may not fit shared memory: refused before any launch
+            assert "too large" in str(e), what
+            continue
+        assert np.array_equal(got, w), what
+        x = wl.activations(batch, cols, 7500 + case, "bf16" if dtype == "bf16" else "fp16")
+        check_product(gpu_gemm(hl, torch, up, x), w, x, od)
+        ran += 1
+    assert ran >= 55
 
 
 @pytest.mark.parametrize("rows,cols,ce,gen", [
